@@ -1,0 +1,380 @@
+"""Python face of the CPU checker (test infrastructure, not the product).
+
+Thin ctypes wrappers over ``ckks_oracle.c`` plus the two composites that are
+easier to read in Python than in C: key derivation helpers and the linear
+projection by diagonals (Eq. 5) in its baby-step/giant-step schedule.
+
+Nothing here imports the CUDA package.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from dataclasses import dataclass
+
+import numpy as np
+
+from . import build as _build
+
+_u64p = C.POINTER(C.c_uint64)
+_i64p = C.POINTER(C.c_int64)
+_f64p = C.POINTER(C.c_double)
+_ldp = C.POINTER(C.c_longdouble)
+
+
+def _p(a, typ):
+    return a.ctypes.data_as(typ) if a is not None else None
+
+
+def _u64(a):
+    a = np.ascontiguousarray(a, dtype=np.uint64)
+    return a
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(_build.build())
+        L.orc_create.restype = C.c_void_p
+        L.orc_create.argtypes = [C.c_uint32] * 4 + [_u64p, _u64p]
+        L.orc_destroy.argtypes = [C.c_void_p]
+        L.orc_root.restype = C.c_uint64
+        L.orc_root.argtypes = [C.c_void_p, C.c_uint32]
+        L.orc_galois_element.restype = C.c_uint64
+        L.orc_galois_element.argtypes = [C.c_void_p, C.c_int64]
+        L.orc_encode_coeffs.restype = C.c_int
+        L.orc_encode.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+@dataclass
+class ProjDesc:
+    """Shape of one linear projection Y = X W in the feature-major token-shard layout."""
+    d_in: int
+    d_out: int
+    tokens_per_shard: int
+    nshards: int
+    baby: int
+    pt_scale: float = 0.0      # 0 => q_{level-1}
+
+
+class Oracle:
+    def __init__(self, log_n: int, q, p, dnum: int):
+        self.log_n, self.N, self.n, self.M = log_n, 1 << log_n, 1 << (log_n - 1), 2 << log_n
+        self.q = [int(x) for x in q]
+        self.p = [int(x) for x in p]
+        self.L, self.K, self.dnum = len(self.q), len(self.p), dnum
+        self.alpha = -(-self.L // dnum)
+        self.mod = self.q + self.p
+        qa = np.array(self.q, dtype=np.uint64)
+        pa = np.array(self.p if self.p else [0], dtype=np.uint64)
+        self._h = C.c_void_p(lib().orc_create(log_n, self.L, self.K, dnum, _p(qa, _u64p), _p(pa, _u64p)))
+
+    def __del__(self):
+        try:
+            lib().orc_destroy(self._h)
+        except Exception:
+            pass
+
+    # ------------------------------------------------------------ parameters
+    def root(self, t: int) -> int:
+        return int(lib().orc_root(self._h, t))
+
+    def galois_element(self, r: int) -> int:
+        return int(lib().orc_galois_element(self._h, r))
+
+    # ------------------------------------------------------------------- NTT
+    def ntt_definition(self, a, t: int):
+        a = _u64(a); out = np.empty_like(a)
+        lib().orc_ntt_definition(self._h, C.c_uint32(t), _p(a, _u64p), _p(out, _u64p))
+        return out
+
+    def intt_definition(self, a, t: int):
+        a = _u64(a); out = np.empty_like(a)
+        lib().orc_intt_definition(self._h, C.c_uint32(t), _p(a, _u64p), _p(out, _u64p))
+        return out
+
+    def ntt(self, polys, first: int = 0):
+        """polys [..., nlimbs, N] -> forward NTT of every limb (copy)."""
+        a = _u64(polys).copy()
+        nl = a.shape[-2] if a.ndim >= 2 else 1
+        batch = a.size // (nl * self.N)
+        lib().orc_ntt_batch(self._h, _p(a, _u64p), C.c_uint32(batch), C.c_uint32(first), C.c_uint32(nl))
+        return a
+
+    def intt(self, polys, first: int = 0):
+        a = _u64(polys).copy()
+        nl = a.shape[-2] if a.ndim >= 2 else 1
+        batch = a.size // (nl * self.N)
+        lib().orc_intt_batch(self._h, _p(a, _u64p), C.c_uint32(batch), C.c_uint32(first), C.c_uint32(nl))
+        return a
+
+    # ---------------------------------------------------------------- encode
+    def encode_coeffs(self, z, scale: float):
+        z = np.asarray(z)
+        re = np.ascontiguousarray(z.real, dtype=np.float64)
+        im = np.ascontiguousarray(z.imag, dtype=np.float64) if np.iscomplexobj(z) else None
+        m = np.empty(self.N, dtype=np.int64)
+        rc = lib().orc_encode_coeffs(self._h, _p(re, _f64p), _p(im, _f64p), C.c_double(scale), _p(m, _i64p))
+        if rc:
+            raise OverflowError("scaled value out of range")
+        return m
+
+    def encode(self, z, scale: float, level: int):
+        z = np.asarray(z)
+        re = np.ascontiguousarray(z.real, dtype=np.float64)
+        im = np.ascontiguousarray(z.imag, dtype=np.float64) if np.iscomplexobj(z) else None
+        out = np.empty((level, self.N), dtype=np.uint64)
+        rc = lib().orc_encode(self._h, _p(re, _f64p), _p(im, _f64p), C.c_double(scale), C.c_uint32(level), _p(out, _u64p))
+        if rc:
+            raise OverflowError("scaled value out of range")
+        return out
+
+    def small_to_limbs(self, poly, first: int, nl: int):
+        poly = np.ascontiguousarray(poly, dtype=np.int64)
+        out = np.empty((nl, self.N), dtype=np.uint64)
+        lib().orc_small_to_limbs(self._h, _p(poly, _i64p), C.c_uint32(first), C.c_uint32(nl), _p(out, _u64p))
+        return out
+
+    def decode(self, coeffs, scale: float, direct: bool = False):
+        m = np.ascontiguousarray(coeffs, dtype=np.longdouble)
+        re = np.empty(self.n); im = np.empty(self.n)
+        f = lib().orc_decode_direct if direct else lib().orc_decode
+        f(self._h, _p(m, _ldp), C.c_double(scale), _p(re, _f64p), _p(im, _f64p))
+        return re + 1j * im
+
+    # ------------------------------------------------- keys, encrypt, decrypt
+    def encrypt(self, pt, a, e, s):
+        pt = _u64(pt); level = pt.shape[0]
+        a = _u64(a); e = np.ascontiguousarray(e, dtype=np.int64); s = np.ascontiguousarray(s, dtype=np.int64)
+        ct = np.empty((2, level, self.N), dtype=np.uint64)
+        lib().orc_encrypt(self._h, _p(pt, _u64p), _p(a, _u64p), _p(e, _i64p), _p(s, _i64p), C.c_uint32(level), _p(ct, _u64p))
+        return ct
+
+    def decrypt(self, ct, s, exact: bool = False):
+        """Centred plaintext coefficients: long double array, or Python ints when exact."""
+        ct = _u64(ct); ncomp, level = ct.shape[0], ct.shape[1]
+        s = np.ascontiguousarray(s, dtype=np.int64)
+        if exact:
+            buf = np.empty((self.N, 2), dtype=np.uint64)
+            lib().orc_decrypt(self._h, _p(ct, _u64p), C.c_uint32(ncomp), C.c_uint32(level), _p(s, _i64p),
+                              C.c_void_p(buf.ctypes.data), None)
+            out = []
+            for lo, hi in buf.tolist():
+                v = (hi << 64) | lo
+                out.append(v - (1 << 128) if v >> 127 else v)
+            return out
+        m = np.empty(self.N, dtype=np.longdouble)
+        lib().orc_decrypt(self._h, _p(ct, _u64p), C.c_uint32(ncomp), C.c_uint32(level), _p(s, _i64p), None, _p(m, _ldp))
+        return m
+
+    def decrypt_decode(self, ct, s, scale: float):
+        return self.decode(self.decrypt(ct, s), scale)
+
+    def switch_keygen(self, s, sprime_limbs, a, e):
+        s = np.ascontiguousarray(s, dtype=np.int64)
+        sp = _u64(sprime_limbs); a = _u64(a); e = np.ascontiguousarray(e, dtype=np.int64)
+        T = self.L + self.K
+        assert sp.shape == (T, self.N) and a.shape == (self.dnum, T, self.N) and e.shape == (self.dnum, self.N)
+        evk = np.empty((self.dnum, 2, T, self.N), dtype=np.uint64)
+        lib().orc_switch_keygen(self._h, _p(s, _i64p), _p(sp, _u64p), _p(a, _u64p), _p(e, _i64p), _p(evk, _u64p))
+        return evk
+
+    def automorphism_small(self, a, g: int):
+        a = np.ascontiguousarray(a, dtype=np.int64); out = np.empty_like(a)
+        lib().orc_automorphism_small(self._h, _p(a, _i64p), C.c_uint64(g), _p(out, _i64p))
+        return out
+
+    def rotation_key(self, s, g: int, a, e):
+        """Key switching sigma_g(s) -> s."""
+        sg = self.automorphism_small(s, g)
+        return self.switch_keygen(s, self.small_to_limbs(sg, 0, self.L + self.K), a, e)
+
+    def relin_key(self, s, a, e):
+        """Key switching s^2 -> s."""
+        T = self.L + self.K
+        sl = self.small_to_limbs(s, 0, T)
+        s2 = np.empty_like(sl)
+        lib().orc_pointwise_mul(self._h, _p(sl, _u64p), _p(sl, _u64p), C.c_uint32(0), C.c_uint32(T), _p(s2, _u64p))
+        return self.switch_keygen(s, s2, a, e)
+
+    # ------------------------------------------------------------- pointwise
+    def mul_plain_acc(self, ct, pt, acc=None):
+        ct = _u64(ct); pt = _u64(pt); level = ct.shape[1]
+        init = acc is None
+        if init:
+            acc = np.empty_like(ct)
+        lib().orc_mul_plain_acc(self._h, _p(ct, _u64p), _p(pt, _u64p), _p(acc, _u64p), C.c_uint32(level), C.c_int(int(init)))
+        return acc
+
+    def add(self, a, b):
+        a = _u64(a); b = _u64(b); out = np.empty_like(a)
+        lib().orc_add(self._h, _p(a, _u64p), _p(b, _u64p), _p(out, _u64p), C.c_uint32(a.shape[0]), C.c_uint32(a.shape[1]))
+        return out
+
+    def automorphism_coeff(self, a, g: int, t: int):
+        a = _u64(a); out = np.empty_like(a)
+        lib().orc_automorphism_coeff(self._h, C.c_uint32(t), _p(a, _u64p), C.c_uint64(g), _p(out, _u64p))
+        return out
+
+    def automorphism_eval(self, a, g: int):
+        a = _u64(a); out = np.empty_like(a)
+        lib().orc_automorphism_eval(self._h, _p(a, _u64p), C.c_uint64(g), _p(out, _u64p))
+        return out
+
+    # ------------------------------------------------------------ key switch
+    def num_digits(self, level: int) -> int:
+        return -(-level // self.alpha)
+
+    def modup_digit(self, d_coeff, j: int):
+        d = _u64(d_coeff); level = d.shape[0]
+        ext = np.empty((level + self.K, self.N), dtype=np.uint64)
+        lib().orc_modup_digit(self._h, _p(d, _u64p), C.c_uint32(level), C.c_uint32(j), _p(ext, _u64p))
+        return ext
+
+    def moddown(self, u, level: int):
+        u = _u64(u); out = np.empty((level, self.N), dtype=np.uint64)
+        lib().orc_moddown(self._h, _p(u, _u64p), C.c_uint32(level), _p(out, _u64p))
+        return out
+
+    def keyswitch(self, d, evk):
+        d = _u64(d); evk = _u64(evk); level = d.shape[0]
+        k = np.empty((2, level, self.N), dtype=np.uint64)
+        lib().orc_keyswitch(self._h, _p(d, _u64p), _p(evk, _u64p), C.c_uint32(level), _p(k, _u64p))
+        return k
+
+    def rotate(self, ct, evk, g: int):
+        ct = _u64(ct); evk = _u64(evk); level = ct.shape[1]
+        out = np.empty_like(ct)
+        lib().orc_rotate(self._h, _p(ct, _u64p), _p(evk, _u64p), C.c_uint64(g), C.c_uint32(level), _p(out, _u64p))
+        return out
+
+    def rotate_hoisted(self, ct, evks, gs):
+        ct = _u64(ct); level = ct.shape[1]; nrot = len(gs)
+        evks = [_u64(k) for k in evks]
+        ptrs = (C.c_void_p * nrot)(*[k.ctypes.data for k in evks])
+        ga = np.array(gs, dtype=np.uint64)
+        outs = np.empty((nrot, 2, level, self.N), dtype=np.uint64)
+        lib().orc_rotate_hoisted(self._h, _p(ct, _u64p), ptrs, _p(ga, _u64p), C.c_uint32(nrot), C.c_uint32(level), _p(outs, _u64p))
+        return outs
+
+    def rescale(self, ct):
+        ct = _u64(ct); ncomp, level = ct.shape[0], ct.shape[1]
+        out = np.empty((ncomp, level - 1, self.N), dtype=np.uint64)
+        lib().orc_rescale(self._h, _p(ct, _u64p), C.c_uint32(ncomp), C.c_uint32(level), _p(out, _u64p))
+        return out
+
+    def tensor(self, a, b):
+        a = _u64(a); b = _u64(b); level = a.shape[1]
+        e = np.empty((3, level, self.N), dtype=np.uint64)
+        lib().orc_tensor(self._h, _p(a, _u64p), _p(b, _u64p), C.c_uint32(level), _p(e, _u64p))
+        return e
+
+    def mul_relin(self, a, b, rlk):
+        a = _u64(a); b = _u64(b); rlk = _u64(rlk); level = a.shape[1]
+        out = np.empty_like(a)
+        lib().orc_mul_relin(self._h, _p(a, _u64p), _p(b, _u64p), _p(rlk, _u64p), C.c_uint32(level), _p(out, _u64p))
+        return out
+
+    # ----------------------------------------------------- linear projection
+    def proj_blocks(self, desc: ProjDesc):
+        """Feature blocks of the input and output: lists of (start, size).  F = n / T_s
+        features fit one ciphertext; a trailing block smaller than F must divide F."""
+        F = self.n // desc.tokens_per_shard
+
+        def split(d):
+            blocks, s = [], 0
+            while s < d:
+                m = min(F, d - s)
+                if F % m:
+                    raise ValueError("remainder block must divide F")
+                blocks.append((s, m)); s += m
+            return blocks
+        return F, split(desc.d_in), split(desc.d_out)
+
+    def proj_rotations(self, desc: ProjDesc):
+        """Slot rotations (hence Galois keys) the schedule uses: baby, giant, fold."""
+        F, ins, outs = self.proj_blocks(desc)
+        T, B = desc.tokens_per_shard, desc.baby
+        rots = set(b * T for b in range(1, B))
+        for (_, mo) in outs:
+            for (_, mi) in ins:
+                nd = min(mi, mo)
+                rots |= set(g * B * T for g in range(1, nd // B))
+                f = mo
+                while f < mi:
+                    rots.add(f * T); f *= 2
+        return sorted(rots)
+
+    @staticmethod
+    def diagonal(Wt_blk, k: int, F: int):
+        """k-th generalised cyclic diagonal of the block A = W^T[out block, in block]
+        (Eq. 5): d_k[r] = A[r mod m_out, (r + k) mod m_in], r < F."""
+        mo, mi = Wt_blk.shape
+        r = np.arange(F)
+        return Wt_blk[r % mo, (r + k) % mi]
+
+    def linear_proj(self, desc: ProjDesc, cts, W, keys: dict, ct_scale: float):
+        """Y = X W on token-shard ciphertexts by the diagonal method (Eq. 5), schedule:
+        baby rotations hoisted per input ciphertext; for every giant step g the
+        pre-rotated diagonals are encoded and multiply-accumulated; acc_g is rotated by
+        g*B*T_s (plain rotation) and summed; optional fold; one rescale.
+
+        cts [nshards * n_in_blocks][2][level][N]; W [d_in][d_out] fp64; keys maps a
+        Galois element to its switching key.  Returns (outs [nshards*n_out_blocks][2]
+        [level-1][N], out_scale).
+        """
+        cts = _u64(cts); level = cts.shape[2]
+        F, ins, outs_b = self.proj_blocks(desc)
+        T, B = desc.tokens_per_shard, desc.baby
+        pt_scale = desc.pt_scale if desc.pt_scale else float(self.q[level - 1])
+        nib, nob = len(ins), len(outs_b)
+        A = np.asarray(W, dtype=np.float64).T                     # [d_out][d_in]
+        outs = np.empty((desc.nshards * nob, 2, level - 1, self.N), dtype=np.uint64)
+        gal = lambda r: self.galois_element(r)
+        # Encoded pre-rotated diagonals are independent of the shard: cache per (ob, ib, g, b).
+        pt_cache = {}
+
+        def plaintext(ob, ib, g, b):
+            key = (ob, ib, g, b)
+            if key not in pt_cache:
+                (os_, mo), (is_, mi) = outs_b[ob], ins[ib]
+                d = self.diagonal(A[os_:os_ + mo, is_:is_ + mi], g * B + b, F)
+                dpre = np.roll(d, g * B)                          # d'[r] = d[(r - gB) mod F]
+                pt_cache[key] = self.encode(np.repeat(dpre, T), pt_scale, level)
+            return pt_cache[key]
+
+        for c in range(desc.nshards):
+            baby = []
+            for ib in range(nib):
+                x = cts[c * nib + ib]
+                gs = [gal(b * T) for b in range(1, B)]
+                rot = self.rotate_hoisted(x, [keys[g] for g in gs], gs) if gs else []
+                baby.append([x] + [rot[i] for i in range(len(gs))])
+            for ob, (os_, mo) in enumerate(outs_b):
+                nds = [min(mi, mo) for (_, mi) in ins]
+                folds = {mi // mo if mi > mo else 1 for (_, mi) in ins}
+                if len(folds) != 1:
+                    raise ValueError("input blocks of one output block need the same fold count")
+                total = None
+                for g in range(max(nds) // B):
+                    acc = None
+                    for ib in range(nib):
+                        if g >= nds[ib] // B:
+                            continue
+                        for b in range(B):
+                            acc = self.mul_plain_acc(baby[ib][b], plaintext(ob, ib, g, b), acc)
+                    if g:
+                        ge = gal(g * B * T)
+                        acc = self.rotate(acc, keys[ge], ge)
+                    total = acc if total is None else self.add(total, acc)
+                f, fold = mo, folds.pop()
+                while fold > 1:
+                    ge = gal(f * T)
+                    total = self.add(total, self.rotate(total, keys[ge], ge))
+                    f *= 2; fold //= 2
+                outs[c * nob + ob] = self.rescale(total)
+        return outs, ct_scale * pt_scale / float(self.q[level - 1])

@@ -1,0 +1,98 @@
+"""Client-side harness for the tests: parameter sets, secret/key/ciphertext
+generation through the CPU checker, big-integer helpers.  The library under
+test never sees a secret key; everything secret lives here."""
+from __future__ import annotations
+
+from functools import lru_cache
+
+import numpy as np
+
+from oracle.ckks_oracle import Oracle
+from paper_2609_12378_b200 import inputs
+
+
+class Params:
+    def __init__(self, log_n, num_q, num_p, dnum, bits=50):
+        self.log_n, self.L, self.K, self.dnum = log_n, num_q, num_p, dnum
+        self.N, self.n = 1 << log_n, 1 << (log_n - 1)
+        self.q, self.p = inputs.prime_chain(log_n, num_q, num_p, bits)
+        self.oracle = Oracle(log_n, self.q, self.p, dnum)
+
+
+@lru_cache(maxsize=None)
+def params(log_n, num_q, num_p, dnum, bits=50) -> Params:
+    return Params(log_n, num_q, num_p, dnum, bits)
+
+
+class Client:
+    """Holds the secret; makes ciphertexts and switching keys with seeded draws."""
+
+    def __init__(self, P: Params, seed: int):
+        self.P, self.o, self.seed = P, P.oracle, seed
+        self.s = inputs.ternary(inputs.rng(seed, 0), P.N)
+        self._stream = 1
+
+    def _g(self):
+        self._stream += 1
+        return inputs.rng(self.seed, self._stream)
+
+    def encrypt_slots(self, z, scale, level):
+        P = self.P
+        pt = self.o.encode(z, scale, level)
+        g = self._g()
+        a = inputs.uniform_residues(g, P.q[:level], P.N)[0]
+        e = inputs.rounded_gaussian(g, P.N)
+        return self.o.encrypt(pt, a, e, self.s)
+
+    def _key_draws(self):
+        P = self.P
+        g = self._g()
+        a = inputs.uniform_residues(g, list(P.q) + list(P.p), P.N, batch=P.dnum)
+        e = inputs.rounded_gaussian(g, (P.dnum, P.N))
+        return a, e
+
+    def rotation_key(self, galois):
+        a, e = self._key_draws()
+        return self.o.rotation_key(self.s, galois, a, e)
+
+    def relin_key(self):
+        a, e = self._key_draws()
+        return self.o.relin_key(self.s, a, e)
+
+    def decrypt_slots(self, ct, scale):
+        return self.o.decrypt_decode(ct, self.s, scale)
+
+
+# ------------------------------------------------------------ big-integer side
+
+def crt(residues, moduli):
+    """The integer in [0, prod moduli) with the given residues (Python ints)."""
+    x, m = 0, 1
+    for r, q in zip(residues, moduli):
+        r, q = int(r), int(q)
+        t = (r - x) * pow(m, -1, q) % q
+        x += m * t
+        m *= q
+    return x, m
+
+
+def centred(x, m):
+    x %= m
+    return x - m if x > m // 2 else x
+
+
+def negacyclic_schoolbook(a, b, q):
+    n = len(a)
+    c = [0] * n
+    for i in range(n):
+        for j in range(n):
+            k = i + j
+            if k < n:
+                c[k] = (c[k] + int(a[i]) * int(b[j])) % q
+            else:
+                c[k - n] = (c[k - n] - int(a[i]) * int(b[j])) % q
+    return c
+
+
+def brev(x, bits):
+    return int(format(x, "0%db" % bits)[::-1], 2) if bits else 0

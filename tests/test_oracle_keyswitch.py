@@ -1,0 +1,202 @@
+"""Pins for the checker's automorphism, ModUp, ModDown, rescale, key switch,
+rotations and relinearised product -- exact big-integer statements on small
+rings, decrypt-level statements on larger ones."""
+import numpy as np
+import pytest
+
+from paper_2609_12378_b200 import inputs
+from tests.harness import Client, centred, crt, params
+
+
+def _coeff_ints(o, limbs_coeff, primes):
+    """Per coefficient, the CRT integer of the given coefficient-domain limbs."""
+    cols = np.asarray(limbs_coeff).T.tolist()
+    return [crt(col, primes)[0] for col in cols]
+
+
+@pytest.mark.parametrize("log_n", [3, 6, 10])
+def test_automorphism_eval_equals_coefficient_definition(log_n):
+    P = params(log_n, 2, 1, 2)
+    o = P.oracle
+    g = inputs.rng(41, log_n)
+    a = inputs.uniform_residues(g, [o.mod[0]], P.N)[0]
+    for gal in (5, 25, 3, 2 * P.N - 1, o.galois_element(3), o.galois_element(-1)):
+        want = o.ntt(o.automorphism_coeff(a[0], gal, 0).reshape(1, -1))[0]
+        assert np.array_equal(o.automorphism_eval(o.ntt(a)[0], gal), want)
+
+
+def test_galois_element_is_left_rotation():
+    """sigma_{5^r} on an encoded vector rotates the slots left by r (Eq. 5's rho^r)."""
+    P = params(8, 2, 1, 2)
+    o = P.oracle
+    z = inputs.rng(42).uniform(-1, 1, P.n)
+    m = o.encode_coeffs(z, 2.0 ** 40)
+    for r in (1, 2, 7, P.n - 1, -3):
+        assert o.galois_element(r) == pow(5, r % P.n, 2 * P.N)
+        back = o.decode(o.automorphism_small(m, o.galois_element(r)).astype(np.longdouble), 2.0 ** 40).real
+        assert np.abs(back - np.roll(z, -r)).max() < 1e-8
+
+
+@pytest.mark.parametrize("log_n,L,K,dnum,level", [(4, 6, 2, 3, 6), (4, 6, 2, 3, 5), (4, 6, 2, 3, 2), (3, 4, 4, 1, 4), (5, 3, 1, 3, 3)])
+def test_modup_big_integer(log_n, L, K, dnum, level):
+    """Extended limbs = (d_c + u Q_j) mod t with one integer u per coefficient, |u| <= |D|/2."""
+    P = params(log_n, L, K, dnum)
+    o = P.oracle
+    d = inputs.uniform_residues(inputs.rng(43, level), P.q[:level], P.N)[0]
+    for j in range(o.num_digits(level)):
+        lo, hi = j * o.alpha, min((j + 1) * o.alpha, level)
+        ext = o.modup_digit(d, j)
+        own = [int(x) for x in P.q[lo:hi]]
+        targets = [int(x) for x in P.q[:level]] + [int(x) for x in P.p]
+        assert ext.shape == (level + K, P.N)
+        for k in range(P.N):
+            v, Qj = crt(d[lo:hi, k], own)
+            dc = centred(v, Qj)
+            us = [u for u in range(-(hi - lo), hi - lo + 1)
+                  if all((dc + u * Qj) % t == int(ext[x, k]) for x, t in enumerate(targets))]
+            assert len(us) == 1 and 2 * abs(us[0]) <= hi - lo
+
+
+@pytest.mark.parametrize("log_n,L,K,dnum,level", [(4, 6, 2, 3, 6), (4, 6, 2, 3, 3), (3, 4, 4, 1, 4), (5, 3, 1, 3, 2)])
+def test_moddown_big_integer(log_n, L, K, dnum, level):
+    """out = (U - r) / P exactly, r = U mod P in centred form up to v P with |v| <= K/2."""
+    P = params(log_n, L, K, dnum)
+    o = P.oracle
+    primes = [int(x) for x in P.q[:level]] + [int(x) for x in P.p]
+    g = inputs.rng(44, level)
+    u_coeff = np.concatenate([inputs.uniform_residues(g, P.q[:level], P.N)[0], inputs.uniform_residues(g, P.p, P.N)[0]])
+    u_eval = np.concatenate([o.ntt(u_coeff[:level]), o.ntt(u_coeff[level:], first=L)])
+    out = o.intt(o.moddown(u_eval, level))
+    Pp = 1
+    for x in P.p:
+        Pp *= int(x)
+    Q = 1
+    for x in P.q[:level]:
+        Q *= int(x)
+    for k in range(P.N):
+        U, _ = crt(u_coeff[:, k], primes)
+        o_int, _ = crt(out[:, k], primes[:level])
+        r0 = centred(U % Pp, Pp)
+        ok = [v for v in range(-K, K + 1) if (U - (r0 + v * Pp)) % Pp == 0 and ((U - (r0 + v * Pp)) // Pp - o_int) % Q == 0]
+        assert ok and 2 * abs(ok[0]) <= K
+
+
+@pytest.mark.parametrize("log_n,level", [(3, 2), (4, 4), (5, 3)])
+def test_rescale_exact_rounding(log_n, level):
+    """out = round(c / q_last) mod Q', per coefficient, exactly (no tie: q_last odd)."""
+    P = params(log_n, 4, 1, 2)
+    o = P.oracle
+    primes = [int(x) for x in P.q[:level]]
+    c_coeff = inputs.uniform_residues(inputs.rng(45, level), P.q[:level], P.N, batch=2)
+    out = o.intt(o.rescale(o.ntt(c_coeff)))
+    ql = primes[-1]
+    Qp = 1
+    for x in primes[:-1]:
+        Qp *= x
+    for comp in range(2):
+        for k in range(P.N):
+            cint, Q = crt(c_coeff[comp, :, k], primes)
+            cc = centred(cint, Q)
+            want = (2 * cc + ql) // (2 * ql)          # floor(c/q + 1/2) = nearest integer
+            assert abs(want * ql - cc) * 2 < ql
+            got, _ = crt(out[comp, :, k], primes[:-1])
+            assert got == want % Qp
+
+
+def _noise_after(cl, o, ct, want_coeffs):
+    got = o.decrypt(ct, cl.s, exact=True)
+    return max(abs(a - b) for a, b in zip(got, want_coeffs))
+
+
+@pytest.mark.parametrize("log_n,L,K,dnum,level", [(10, 6, 2, 3, 6), (10, 6, 2, 3, 3), (10, 6, 1, 6, 6), (10, 4, 4, 1, 4)])
+def test_keyswitch_decrypt_invariant(log_n, L, K, dnum, level):
+    """k0 + k1 s = d s' + small, for s' = sigma_g(s) and s' = s^2."""
+    P = params(log_n, L, K, dnum)
+    o = P.oracle
+    cl = Client(P, 51)
+    d = inputs.uniform_residues(inputs.rng(46, level), P.q[:level], P.N)[0]
+    gal = o.galois_element(5)
+    for sprime_limbs, evk in (
+        (o.small_to_limbs(o.automorphism_small(cl.s, gal), 0, level), cl.rotation_key(gal)),
+        (None, cl.relin_key()),
+    ):
+        if sprime_limbs is None:
+            sl = o.small_to_limbs(cl.s, 0, level)
+            sprime_limbs = np.array([[int(a) * int(a) % o.mod[i] for a in sl[i].tolist()] for i in range(level)], dtype=np.uint64)
+        k = o.keyswitch(d, evk)
+        # want = d * s' as a "ciphertext" (d s', 0): compare decryptions
+        ds = np.array([[int(a) * int(b) % o.mod[i] for a, b in zip(d[i].tolist(), sprime_limbs[i].tolist())] for i in range(level)], dtype=np.uint64)
+        ref = np.stack([ds, np.zeros_like(ds)])
+        diff = o.decrypt(_sub(o, k, ref), cl.s, exact=True)
+        noise = max(abs(x) for x in diff)
+        assert noise < 2 ** 14, noise          # ~ sqrt(beta N) sigma, nowhere near Q
+
+
+def _sub(o, a, b):
+    out = np.empty_like(a)
+    for c in range(a.shape[0]):
+        for i in range(a.shape[1]):
+            m = o.mod[i]
+            out[c, i] = (a[c, i].astype(object) - b[c, i].astype(object)) % m
+    return out
+
+
+@pytest.mark.parametrize("log_n,L,K,dnum,level", [(11, 6, 2, 3, 6), (11, 6, 2, 3, 4), (13, 6, 1, 6, 6)])
+def test_rotate_decrypts_to_rotated_slots(log_n, L, K, dnum, level):
+    P = params(log_n, L, K, dnum)
+    o = P.oracle
+    cl = Client(P, 52)
+    z = inputs.rng(47, log_n).uniform(-1, 1, P.n)
+    scale = 2.0 ** 40
+    ct = cl.encrypt_slots(z, scale, level)
+    rots = [1, 8, P.n - 5]
+    gals = [o.galois_element(r) for r in rots]
+    keys = [cl.rotation_key(g) for g in gals]
+    hoisted = o.rotate_hoisted(ct, keys, gals)
+    for i, r in enumerate(rots):
+        plain = o.rotate(ct, keys[i], gals[i])
+        want = np.roll(z, -r)
+        zp, zh = cl.decrypt_slots(plain, scale), cl.decrypt_slots(hoisted[i], scale)
+        assert np.abs(zp - want).max() < 2.0 ** -20
+        assert np.abs(zh - want).max() < 2.0 ** -20
+        assert np.abs(zp - zh).max() < 2.0 ** -20
+        # slot 0 is where a constant rounding bias would show up (centred lifts keep it out)
+        assert abs(zp[0] - want[0]) < 2.0 ** -22 and abs(zh[0] - want[0]) < 2.0 ** -22
+    # rotate by r then by n - r returns the input slots
+    back = o.rotate(o.rotate(ct, keys[0], gals[0]), cl.rotation_key(o.galois_element(-1)), o.galois_element(-1))
+    assert np.abs(cl.decrypt_slots(back, scale) - z).max() < 2.0 ** -20
+
+
+def test_hoisted_is_its_own_integer_function_but_same_plaintext():
+    P = params(10, 6, 2, 3)
+    o = P.oracle
+    cl = Client(P, 53)
+    ct = cl.encrypt_slots(inputs.rng(48).uniform(-1, 1, P.n), 2.0 ** 40, 6)
+    gal = o.galois_element(3)
+    key = cl.rotation_key(gal)
+    a, b = o.rotate(ct, key, gal), o.rotate_hoisted(ct, [key], [gal])[0]
+    da, db = o.decrypt(a, cl.s, exact=True), o.decrypt(b, cl.s, exact=True)
+    assert max(abs(x - y) for x, y in zip(da, db)) < 2 ** 14
+
+
+@pytest.mark.parametrize("log_n,L,K,dnum,level", [(11, 6, 2, 3, 6), (11, 6, 2, 3, 3)])
+def test_mul_relin_slot_product(log_n, L, K, dnum, level):
+    P = params(log_n, L, K, dnum)
+    o = P.oracle
+    cl = Client(P, 54)
+    g = inputs.rng(49)
+    z, w = g.uniform(-1, 1, P.n), g.uniform(-1, 1, P.n)
+    scale = 2.0 ** 40
+    scale_b = float(P.q[level - 1])          # so that the rescale below lands back on 2^40 exactly
+    ca, cb = cl.encrypt_slots(z, scale, level), cl.encrypt_slots(w, scale_b, level)
+    rlk = cl.relin_key()
+    out = o.mul_relin(ca, cb, rlk)
+    assert np.abs(cl.decrypt_slots(out, scale * scale_b) - z * w).max() < 2.0 ** -20
+    # three-component decrypt before relinearisation = two-component decrypt after, up to key-switch noise
+    d3 = o.decrypt(o.tensor(ca, cb), cl.s, exact=True)
+    d2 = o.decrypt(out, cl.s, exact=True)
+    assert max(abs(x - y) for x, y in zip(d3, d2)) < 2 ** 16
+    # then rescale: slots unchanged, scale divided by q_last
+    rs = o.rescale(out)
+    assert rs.shape[1] == level - 1
+    assert np.abs(cl.decrypt_slots(rs, scale) - z * w).max() < 2.0 ** -20
