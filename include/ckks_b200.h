@@ -1,0 +1,219 @@
+/*
+ * ckks_b200 -- CKKS RNS primitive layer for NVIDIA B200 (sm_100a), C ABI.
+ *
+ * The operations are the ones the paper's server-side evaluation is built
+ * from (Section 2.1, "The CKKS Computation Model": Encode, Add, PCMult, Mult,
+ * Rot_k, KeySwitch, Rescale) plus the diagonal matrix-vector product of
+ * Eq. 5 evaluated baby-step/giant-step over the feature-major token-shard
+ * layout (Sections 1 and 3: feature-major cross-layer state; plaintexts
+ * organised by logical diagonal and reused across token-shard inputs).  The
+ * paper fixes what is called and with which shapes; the arithmetic is the
+ * full-RNS form of the scheme it cites.
+ *
+ * General rules
+ *   - Every function returns a status (0 = CKKS_OK, negative = error) and
+ *     never throws.  Arguments are validated on the host before any launch:
+ *     a failing call launches nothing and writes nothing.
+ *   - The caller owns every device buffer: inputs, outputs, keys, workspace.
+ *     The library allocates device memory only in ckks_context_create (its
+ *     tables) and frees it in ckks_context_destroy.  Calls enqueue work on the
+ *     given stream (a cudaStream_t passed as void*, NULL = default stream) and
+ *     return without synchronising.
+ *   - The library never sees a secret key.
+ *   - "Host" / "device" is stated for every pointer.  Descriptor structs
+ *     (ckks_ct, ckks_pt, ckks_evk, ckks_proj_desc) live in host memory and hold
+ *     device pointers.
+ *
+ * Data layout
+ *   N ring degree, n = N/2 slots.  Prime index space: 0..L-1 are the ciphertext
+ *   primes q_0..q_{L-1}, L..L+K-1 the special primes p_0..p_{K-1}.  All primes
+ *   must lie in (2^49, 2^50) and be 1 mod 2N.  A limb is N uint64 residues in
+ *   [0, prime).  Every stored polynomial is in the evaluation domain in
+ *   bit-reversed order: limb[p] = a(psi^(2*bitrev(p)+1)), psi = the smallest
+ *   primitive 2N-th root of unity modulo the limb's prime.
+ *     ciphertext      [ncomp][level][N]      limbs q_0..q_{level-1}
+ *     plaintext       [level][N]
+ *     switching key   [dnum][2][L+K][N]      component 0 = b, 1 = a
+ *   "level" counts limbs; rescale drops q_{level-1}.  Digit j of the hybrid
+ *   key switch covers limbs j*alpha .. min((j+1)*alpha, level)-1 with
+ *   alpha = ceil(L/dnum); K >= alpha is required.
+ *   Slot j of a plaintext sits at the root zeta^(5^j), zeta = exp(2 pi i / 2N),
+ *   so the Galois element 5^r is a left rotation by r slots (Eq. 5's rho^r).
+ */
+#ifndef CKKS_B200_H
+#define CKKS_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    CKKS_OK = 0,
+    CKKS_ERR_ARG = -1,         /* null pointer, zero count, bad enum                       */
+    CKKS_ERR_LEVEL = -2,       /* level 0, level > L, operand levels differ                */
+    CKKS_ERR_SCALE = -3,       /* scales that must agree differ by more than 2^-30 relative */
+    CKKS_ERR_NO_KEY = -4,      /* a needed Galois element is not among the supplied keys   */
+    CKKS_ERR_WORKSPACE = -5,   /* workspace missing or smaller than ckks_workspace_bytes   */
+    CKKS_ERR_RANGE = -6,       /* encode: a scaled value does not fit 2^62                 */
+    CKKS_ERR_UNSUPPORTED = -7, /* parameters outside what the kernels implement            */
+    CKKS_ERR_CUDA = -8,        /* a CUDA runtime call failed (see ckks_last_cuda_error)    */
+    CKKS_ERR_TIMEOUT = -9      /* reserved for bounded device-side waits                   */
+};
+
+/* Operation selectors for ckks_workspace_bytes. */
+enum {
+    CKKS_OP_ENCODE = 1, CKKS_OP_MUL_RELIN = 2, CKKS_OP_ROTATE = 3,
+    CKKS_OP_ROTATE_HOISTED = 4, CKKS_OP_RESCALE = 5, CKKS_OP_LINEAR_PROJ = 6
+};
+
+typedef struct ckks_ctx ckks_ctx; /* opaque */
+
+/* All fields host-side.  q[num_q], p[num_p] host arrays. */
+typedef struct {
+    uint32_t log_n;       /* 10..16                                             */
+    uint32_t num_q;       /* L                                                  */
+    uint32_t num_p;       /* K  (>= ceil(L/dnum))                               */
+    uint32_t dnum;        /* number of key-switch digits                        */
+    const uint64_t *q;    /* host                                               */
+    const uint64_t *p;    /* host                                               */
+    int32_t device;       /* CUDA device ordinal the tables are placed on       */
+} ckks_params;
+
+typedef struct { uint64_t *data; /* device */ uint32_t level, ncomp; double scale; } ckks_ct;
+typedef struct { uint64_t *data; /* device */ uint32_t level; double scale; } ckks_pt;
+typedef struct { const uint64_t *data; /* device */ uint64_t galois; /* 0 for a relinearisation key */ } ckks_evk;
+
+/*
+ * Shape of one projection Y = X W (Eq. 5 per block, baby-step/giant-step).
+ * Tokens are split into nshards shards of tokens_per_shard (T) tokens; one
+ * ciphertext holds F = n/T features of one shard, slot = f*T + t.  d_in and
+ * d_out are cut into blocks of F features; a trailing block smaller than F
+ * must divide F and is stored repeated F/m times.  For an (input block m_in,
+ * output block m_out) pair the min(m_in, m_out) generalised diagonals
+ * d_k[r] = W^T[r mod m_out, (r + k) mod m_in] are used; `baby` (B) must divide
+ * that count; when m_out < m_in the result is folded by log2(m_in/m_out)
+ * rotate-and-add steps.  pt_scale is the scale the weights are encoded at
+ * (0 selects q_{level-1}, so that the final rescale restores the input scale).
+ */
+typedef struct {
+    uint32_t d_in, d_out, tokens_per_shard, nshards, baby;
+    double pt_scale;
+} ckks_proj_desc;
+
+/* ---- context ----------------------------------------------------------- */
+
+/* Builds the tables (twiddles, conversion constants, permutation helpers) on
+ * params->device.  *out receives the context.  Errors: ARG, UNSUPPORTED
+ * (log_n, prime size, prime not 1 mod 2N, duplicates, K < alpha), CUDA. */
+int32_t ckks_context_create(const ckks_params *params, ckks_ctx **out);
+void ckks_context_destroy(ckks_ctx *ctx);
+
+const char *ckks_status_string(int32_t status);
+/* Text of the last CUDA error seen by this context ("" if none).  Host string owned by the context. */
+const char *ckks_last_cuda_error(const ckks_ctx *ctx);
+
+/* Bytes of caller-provided device workspace `op` needs at this level.  `count`
+ * is the batch size for CKKS_OP_ENCODE and the number of rotations for
+ * CKKS_OP_ROTATE_HOISTED; ignored otherwise.  For CKKS_OP_LINEAR_PROJ use
+ * ckks_linear_proj_workspace_bytes.  Returns 0 for an unknown op. */
+size_t ckks_workspace_bytes(const ckks_ctx *ctx, int32_t op, uint32_t level, uint32_t count);
+
+/* 5^r mod 2N with r taken mod n: Galois element of a left rotation by r slots. */
+uint64_t ckks_galois_element(const ckks_ctx *ctx, int64_t left_rot_slots);
+
+/* ---- NTT --------------------------------------------------------------- */
+
+/* Forward / inverse negacyclic NTT, in place, of `batch * nlimbs` limbs laid
+ * out [batch][nlimbs][N] (device); limb i of every batch entry is taken
+ * modulo prime first_prime + i (prime index space above).  Forward: natural-
+ * order coefficients in, bit-reversed evaluations out; inverse undoes it
+ * (including N^-1).  Inputs must be canonical residues.  Errors: ARG, LEVEL
+ * (prime range outside 0..L+K-1). */
+int32_t ckks_ntt(ckks_ctx *ctx, uint64_t *polys, uint32_t batch, uint32_t first_prime, uint32_t nlimbs, void *stream);
+int32_t ckks_intt(ckks_ctx *ctx, uint64_t *polys, uint32_t batch, uint32_t first_prime, uint32_t nlimbs, void *stream);
+
+/* ---- Encode (Section 2.1, Encode) ----------------------------------------
+ * re, im: device, [batch][n] fp64 slot values (im may be NULL = real input).
+ * out: device, [batch][level][N].  Steps: slot permutation e_j = (5^j mod 2N
+ * - 1)/4, unnormalised inverse DFT of size n by radix-2 butterflies with every
+ * product and sum rounded on its own (no FMA), twist by conj(zeta^k), multiply
+ * by scale/n, round half to even, reduce modulo each prime, NTT.  A scaled
+ * value of magnitude >= 2^62 sets a sticky range flag (the coefficient is
+ * encoded as 0); read it with ckks_encode_range_flag.
+ * Errors: ARG, LEVEL, WORKSPACE. */
+int32_t ckks_encode(ckks_ctx *ctx, const double *re, const double *im, uint32_t batch, double scale,
+                    uint32_t level, uint64_t *out, void *ws, size_t ws_bytes, void *stream);
+/* Synchronises `stream`, returns CKKS_ERR_RANGE if any encode since the last
+ * query overflowed (and clears the flag), else CKKS_OK. */
+int32_t ckks_encode_range_flag(ckks_ctx *ctx, void *stream);
+
+/* ---- PCMult + Add (Section 2.1) -------------------------------------------
+ * accs[s] (+)= cts[s] * pt for s < ncts, both components, all limbs.  cts,
+ * accs: host arrays of descriptors.  init = 1: accs[s] = cts[s]*pt and
+ * accs[s].scale/level/ncomp are set; init = 0: requires cts[s].scale *
+ * pt->scale == accs[s].scale within 2^-30 relative.  Levels must all agree.
+ * accs[s] may not alias cts[s'].  Errors: ARG, LEVEL, SCALE. */
+int32_t ckks_mul_plain_acc(ckks_ctx *ctx, const ckks_ct *cts, uint32_t ncts, const ckks_pt *pt,
+                           ckks_ct *accs, int32_t init, void *stream);
+
+/* Add (Section 2.1): out = a + b, same level, ncomp, scale (2^-30 relative).  out may alias a or b. */
+int32_t ckks_add(ckks_ctx *ctx, const ckks_ct *a, const ckks_ct *b, ckks_ct *out, void *stream);
+
+/* ---- Mult with relinearisation (Section 2.1, Mult + KeySwitch) -------------
+ * out = (a0 b0 + k0, a0 b1 + a1 b0 + k1), (k0, k1) = KeySwitch(a1 b1, rlk).
+ * out->scale = a->scale * b->scale; no rescale inside.  rlk->galois must be 0.
+ * out may alias a or b.  Errors: ARG, LEVEL, NO_KEY, WORKSPACE. */
+int32_t ckks_mul_relin(ckks_ctx *ctx, const ckks_ct *a, const ckks_ct *b, const ckks_evk *rlk, ckks_ct *out,
+                       void *ws, size_t ws_bytes, void *stream);
+
+/* ---- Rot_k (Section 2.1, Rot + KeySwitch) ----------------------------------
+ * Plain: apply sigma_g (g = key->galois) to both components, key-switch the
+ * permuted c1: out = (sigma c0 + k0, k1).  Key switch = iNTT, centred ModUp
+ * per digit, NTT, inner product with the key over the active limbs, centred
+ * ModDown.  out must not alias in.  Errors: ARG, LEVEL, NO_KEY (galois 0 or
+ * even), WORKSPACE. */
+int32_t ckks_rotate(ckks_ctx *ctx, const ckks_ct *in, const ckks_evk *key, ckks_ct *out,
+                    void *ws, size_t ws_bytes, void *stream);
+
+/* Hoisted: one iNTT + ModUp + NTT of c1 shared by nrot rotations; rotation r
+ * permutes the extended digits by sigma_{g_r}, takes the inner product with
+ * keys[r], ModDown, adds sigma(c0).  As an integer function this differs from
+ * ckks_rotate (same plaintext, different low noise bits).  keys, outs: host
+ * arrays of nrot descriptors.  Errors as ckks_rotate. */
+int32_t ckks_rotate_hoisted(ckks_ctx *ctx, const ckks_ct *in, const ckks_evk *keys, uint32_t nrot, ckks_ct *outs,
+                            void *ws, size_t ws_bytes, void *stream);
+
+/* ---- Rescale (Section 2.1) --------------------------------------------------
+ * Drops limb level-1 with exact rounding: out_i = (c_i - [centred c_last]) *
+ * q_last^-1 mod q_i.  out->level = level-1, out->scale = in->scale / q_last.
+ * out may alias in (the result is packed [ncomp][level-1][N]) only if ncomp
+ * == 1; otherwise it must not overlap.  Errors: ARG, LEVEL (level < 2), WORKSPACE. */
+int32_t ckks_rescale(ckks_ctx *ctx, const ckks_ct *in, ckks_ct *out, void *ws, size_t ws_bytes, void *stream);
+
+/* ---- Linear projection (Eq. 5, baby-step/giant-step) -----------------------
+ * in: host array of nshards * n_in_blocks descriptors (index shard * n_in_blocks
+ * + block), all at one level and scale.  W: device, row-major [d_in][d_out]
+ * fp64.  keys: host array of nkeys rotation keys; every rotation the schedule
+ * uses (ckks_linear_proj_rotations) must be present.  out: host array of
+ * nshards * n_out_blocks descriptors with device buffers for level-1 limbs;
+ * level and scale are set.  Schedule: hoisted baby rotations b*T (b < B) of
+ * every input ciphertext; for each giant step g the pre-rotated diagonals are
+ * extracted from W, encoded at pt_scale and multiply-accumulated over b and
+ * over input blocks; the sum is rotated by g*B*T with the plain rotation and
+ * added up; optional fold; one rescale per output ciphertext.
+ * Errors: ARG, LEVEL, SCALE, NO_KEY, WORKSPACE, UNSUPPORTED (shape rules above). */
+int32_t ckks_linear_proj(ckks_ctx *ctx, const ckks_proj_desc *desc, const ckks_ct *in, const double *W,
+                         const ckks_evk *keys, uint32_t nkeys, ckks_ct *out,
+                         void *ws, size_t ws_bytes, void *stream);
+size_t ckks_linear_proj_workspace_bytes(const ckks_ctx *ctx, const ckks_proj_desc *desc, uint32_t level);
+/* Writes up to cap left-rotation amounts (in slots) the schedule needs into
+ * rots (host) and returns how many there are; <0 on a shape error. */
+int32_t ckks_linear_proj_rotations(const ckks_ctx *ctx, const ckks_proj_desc *desc, int64_t *rots, uint32_t cap);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CKKS_B200_H */

@@ -1,0 +1,329 @@
+"""ctypes binding of the ckks_b200 C ABI.  Argument marshalling only: every
+step of every operation runs in the library's CUDA kernels.  torch provides
+device memory and streams."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libckks_b200.so")
+
+OK, ERR_ARG, ERR_LEVEL, ERR_SCALE, ERR_NO_KEY, ERR_WORKSPACE, ERR_RANGE, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT = (
+    0, -1, -2, -3, -4, -5, -6, -7, -8, -9)
+OP_ENCODE, OP_MUL_RELIN, OP_ROTATE, OP_ROTATE_HOISTED, OP_RESCALE, OP_LINEAR_PROJ = 1, 2, 3, 4, 5, 6
+
+EXPORTS = [
+    "ckks_context_create", "ckks_context_destroy", "ckks_status_string", "ckks_last_cuda_error",
+    "ckks_workspace_bytes", "ckks_galois_element", "ckks_ntt", "ckks_intt", "ckks_encode",
+    "ckks_encode_range_flag", "ckks_mul_plain_acc", "ckks_add", "ckks_mul_relin", "ckks_rotate",
+    "ckks_rotate_hoisted", "ckks_rescale", "ckks_linear_proj", "ckks_linear_proj_workspace_bytes",
+    "ckks_linear_proj_rotations",
+]
+
+
+class CParams(C.Structure):
+    _fields_ = [("log_n", C.c_uint32), ("num_q", C.c_uint32), ("num_p", C.c_uint32), ("dnum", C.c_uint32),
+                ("q", C.POINTER(C.c_uint64)), ("p", C.POINTER(C.c_uint64)), ("device", C.c_int32)]
+
+
+class CCt(C.Structure):
+    _fields_ = [("data", C.c_void_p), ("level", C.c_uint32), ("ncomp", C.c_uint32), ("scale", C.c_double)]
+
+
+class CPt(C.Structure):
+    _fields_ = [("data", C.c_void_p), ("level", C.c_uint32), ("scale", C.c_double)]
+
+
+class CEvk(C.Structure):
+    _fields_ = [("data", C.c_void_p), ("galois", C.c_uint64)]
+
+
+class CProjDesc(C.Structure):
+    _fields_ = [("d_in", C.c_uint32), ("d_out", C.c_uint32), ("tokens_per_shard", C.c_uint32),
+                ("nshards", C.c_uint32), ("baby", C.c_uint32), ("pt_scale", C.c_double)]
+
+
+_lib = None
+
+
+def load():
+    """Load the CUDA library.  There is no fallback: a missing library is an error."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_12378_b200.build`")
+    L = C.CDLL(LIB_PATH)
+    vp, u32, u64, i32, i64, sz, dbl = C.c_void_p, C.c_uint32, C.c_uint64, C.c_int32, C.c_int64, C.c_size_t, C.c_double
+    sig = {
+        "ckks_context_create": (i32, [C.POINTER(CParams), C.POINTER(vp)]),
+        "ckks_context_destroy": (None, [vp]),
+        "ckks_status_string": (C.c_char_p, [i32]),
+        "ckks_last_cuda_error": (C.c_char_p, [vp]),
+        "ckks_workspace_bytes": (sz, [vp, i32, u32, u32]),
+        "ckks_galois_element": (u64, [vp, i64]),
+        "ckks_ntt": (i32, [vp, vp, u32, u32, u32, vp]),
+        "ckks_intt": (i32, [vp, vp, u32, u32, u32, vp]),
+        "ckks_encode": (i32, [vp, vp, vp, u32, dbl, u32, vp, vp, sz, vp]),
+        "ckks_encode_range_flag": (i32, [vp, vp]),
+        "ckks_mul_plain_acc": (i32, [vp, C.POINTER(CCt), u32, C.POINTER(CPt), C.POINTER(CCt), i32, vp]),
+        "ckks_add": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), C.POINTER(CCt), vp]),
+        "ckks_mul_relin": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
+        "ckks_rotate": (i32, [vp, C.POINTER(CCt), C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
+        "ckks_rotate_hoisted": (i32, [vp, C.POINTER(CCt), C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
+        "ckks_rescale": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), vp, sz, vp]),
+        "ckks_linear_proj": (i32, [vp, C.POINTER(CProjDesc), C.POINTER(CCt), vp, C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
+        "ckks_linear_proj_workspace_bytes": (sz, [vp, C.POINTER(CProjDesc), u32]),
+        "ckks_linear_proj_rotations": (i32, [vp, C.POINTER(CProjDesc), C.POINTER(i64), u32]),
+    }
+    for name, (res, args) in sig.items():
+        f = getattr(L, name)
+        f.restype, f.argtypes = res, args
+    _lib = L
+    return L
+
+
+class CkksError(RuntimeError):
+    def __init__(self, code: int, detail: str = ""):
+        self.code = code
+        msg = load().ckks_status_string(code).decode()
+        super().__init__(f"ckks_b200 error {code}: {msg}" + (f" ({detail})" if detail else ""))
+
+
+@dataclass
+class Ciphertext:
+    data: torch.Tensor      # uint64 [ncomp][level][N] on the device
+    scale: float
+
+    @property
+    def ncomp(self):
+        return self.data.shape[0]
+
+    @property
+    def level(self):
+        return self.data.shape[1]
+
+
+@dataclass
+class Plaintext:
+    data: torch.Tensor      # uint64 [level][N]
+    scale: float
+
+    @property
+    def level(self):
+        return self.data.shape[0]
+
+
+@dataclass
+class SwitchKey:
+    data: torch.Tensor      # uint64 [dnum][2][L+K][N]
+    galois: int             # 0 for a relinearisation key
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _dev_u64(t: torch.Tensor) -> torch.Tensor:
+    if not (t.is_cuda and t.dtype == torch.uint64 and t.is_contiguous()):
+        raise TypeError("expected a contiguous CUDA uint64 tensor")
+    return t
+
+
+def _cct(ct: Ciphertext) -> CCt:
+    _dev_u64(ct.data)
+    return CCt(ct.data.data_ptr(), ct.level, ct.ncomp, ct.scale)
+
+
+class Context:
+    """Owns a library context (device tables) for one parameter set."""
+
+    def __init__(self, log_n: int, q, p, dnum: int, device: int = 0):
+        L = load()
+        self.q = [int(x) for x in q]
+        self.p = [int(x) for x in p]
+        self.log_n, self.N, self.n = log_n, 1 << log_n, 1 << (log_n - 1)
+        self.L, self.K, self.dnum = len(self.q), len(self.p), dnum
+        self.device = torch.device("cuda", device)
+        qa = (C.c_uint64 * max(1, self.L))(*self.q)
+        pa = (C.c_uint64 * max(1, self.K))(*self.p)
+        prm = CParams(log_n, self.L, self.K, dnum, qa, pa, device)
+        h = C.c_void_p()
+        rc = L.ckks_context_create(C.byref(prm), C.byref(h))
+        if rc:
+            raise CkksError(rc)
+        self._h = h
+        self._ws = None
+
+    def close(self):
+        if getattr(self, "_h", None):
+            load().ckks_context_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -------------------------------------------------------------- helpers
+    def _check(self, rc):
+        if rc:
+            raise CkksError(rc, load().ckks_last_cuda_error(self._h).decode() if rc == ERR_CUDA else "")
+
+    def workspace(self, nbytes: int) -> torch.Tensor:
+        """A cached device scratch buffer of at least nbytes (grown on demand by torch)."""
+        if self._ws is None or self._ws.numel() < nbytes:
+            self._ws = None
+            self._ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=self.device)
+        return self._ws
+
+    def workspace_bytes(self, op: int, level: int, count: int = 0) -> int:
+        return int(load().ckks_workspace_bytes(self._h, op, level, count))
+
+    def galois_element(self, r: int) -> int:
+        return int(load().ckks_galois_element(self._h, r))
+
+    def empty_ct(self, level: int, ncomp: int = 2) -> Ciphertext:
+        return Ciphertext(torch.empty((ncomp, level, self.N), dtype=torch.uint64, device=self.device), 0.0)
+
+    # ------------------------------------------------------------------ ops
+    def ntt(self, polys: torch.Tensor, first_prime: int = 0, stream=None):
+        """In-place forward NTT of [batch][nlimbs][N] (or [nlimbs][N])."""
+        _dev_u64(polys)
+        nl = polys.shape[-2]
+        batch = polys.numel() // (nl * self.N)
+        self._check(load().ckks_ntt(self._h, polys.data_ptr(), batch, first_prime, nl, _stream_ptr(stream)))
+        return polys
+
+    def intt(self, polys: torch.Tensor, first_prime: int = 0, stream=None):
+        _dev_u64(polys)
+        nl = polys.shape[-2]
+        batch = polys.numel() // (nl * self.N)
+        self._check(load().ckks_intt(self._h, polys.data_ptr(), batch, first_prime, nl, _stream_ptr(stream)))
+        return polys
+
+    def encode(self, re: torch.Tensor, im, scale: float, level: int, out: torch.Tensor = None, stream=None):
+        """re/im: fp64 [batch][n] on the device -> uint64 [batch][level][N]."""
+        if not (re.is_cuda and re.dtype == torch.float64 and re.is_contiguous()):
+            raise TypeError("expected a contiguous CUDA float64 tensor")
+        batch = re.numel() // self.n
+        if out is None:
+            out = torch.empty((batch, level, self.N), dtype=torch.uint64, device=self.device)
+        nb = self.workspace_bytes(OP_ENCODE, level, batch)
+        ws = self.workspace(nb)
+        self._check(load().ckks_encode(self._h, re.data_ptr(), im.data_ptr() if im is not None else None, batch,
+                                       float(scale), level, _dev_u64(out).data_ptr(), ws.data_ptr(), ws.numel(),
+                                       _stream_ptr(stream)))
+        return out
+
+    def encode_range_flag(self, stream=None) -> int:
+        return int(load().ckks_encode_range_flag(self._h, _stream_ptr(stream)))
+
+    def mul_plain_acc(self, cts, pt: Plaintext, accs=None, stream=None):
+        """accs[s] (+)= cts[s] * pt.  accs None: fresh accumulators are returned."""
+        init = accs is None
+        if init:
+            accs = [self.empty_ct(pt.level) for _ in cts]
+        n = len(cts)
+        ca = (CCt * n)(*[_cct(c) for c in cts])
+        aa = (CCt * n)(*[_cct(a) for a in accs])
+        cp = CPt(_dev_u64(pt.data).data_ptr(), pt.level, pt.scale)
+        self._check(load().ckks_mul_plain_acc(self._h, ca, n, C.byref(cp), aa, int(init), _stream_ptr(stream)))
+        for a, c in zip(accs, aa):
+            a.scale = c.scale
+        return accs
+
+    def add(self, a: Ciphertext, b: Ciphertext, out: Ciphertext = None, stream=None):
+        out = out or self.empty_ct(a.level, a.ncomp)
+        co = _cct(out)
+        self._check(load().ckks_add(self._h, C.byref(_cct(a)), C.byref(_cct(b)), C.byref(co), _stream_ptr(stream)))
+        out.scale = co.scale
+        return out
+
+    def mul_relin(self, a: Ciphertext, b: Ciphertext, rlk: SwitchKey, out: Ciphertext = None, stream=None):
+        out = out or self.empty_ct(a.level)
+        ws = self.workspace(self.workspace_bytes(OP_MUL_RELIN, a.level))
+        co, ck = _cct(out), CEvk(_dev_u64(rlk.data).data_ptr(), rlk.galois)
+        self._check(load().ckks_mul_relin(self._h, C.byref(_cct(a)), C.byref(_cct(b)), C.byref(ck), C.byref(co),
+                                          ws.data_ptr(), ws.numel(), _stream_ptr(stream)))
+        out.scale = co.scale
+        return out
+
+    def rotate(self, ct: Ciphertext, key: SwitchKey, out: Ciphertext = None, stream=None):
+        out = out or self.empty_ct(ct.level)
+        ws = self.workspace(self.workspace_bytes(OP_ROTATE, ct.level))
+        co, ck = _cct(out), CEvk(_dev_u64(key.data).data_ptr(), key.galois)
+        self._check(load().ckks_rotate(self._h, C.byref(_cct(ct)), C.byref(ck), C.byref(co), ws.data_ptr(), ws.numel(),
+                                       _stream_ptr(stream)))
+        out.scale = co.scale
+        return out
+
+    def rotate_hoisted(self, ct: Ciphertext, keys, outs=None, stream=None):
+        n = len(keys)
+        outs = outs or [self.empty_ct(ct.level) for _ in keys]
+        ws = self.workspace(self.workspace_bytes(OP_ROTATE_HOISTED, ct.level, n))
+        ka = (CEvk * n)(*[CEvk(_dev_u64(k.data).data_ptr(), k.galois) for k in keys])
+        oa = (CCt * n)(*[_cct(o) for o in outs])
+        self._check(load().ckks_rotate_hoisted(self._h, C.byref(_cct(ct)), ka, n, oa, ws.data_ptr(), ws.numel(),
+                                               _stream_ptr(stream)))
+        for o, c in zip(outs, oa):
+            o.scale = c.scale
+        return outs
+
+    def rescale(self, ct: Ciphertext, out: Ciphertext = None, stream=None):
+        out = out or self.empty_ct(ct.level - 1, ct.ncomp)
+        ws = self.workspace(self.workspace_bytes(OP_RESCALE, ct.level))
+        co = _cct(out)
+        co.level = ct.level - 1
+        self._check(load().ckks_rescale(self._h, C.byref(_cct(ct)), C.byref(co), ws.data_ptr(), ws.numel(), _stream_ptr(stream)))
+        out.scale = co.scale
+        return out
+
+    # ----------------------------------------------------- linear projection
+    def _desc(self, d_in, d_out, tokens_per_shard, nshards, baby, pt_scale=0.0):
+        return CProjDesc(d_in, d_out, tokens_per_shard, nshards, baby, float(pt_scale))
+
+    def linear_proj_rotations(self, d_in, d_out, tokens_per_shard, nshards, baby):
+        d = self._desc(d_in, d_out, tokens_per_shard, nshards, baby)
+        n = load().ckks_linear_proj_rotations(self._h, C.byref(d), None, 0)
+        if n < 0:
+            raise CkksError(n)
+        buf = (C.c_int64 * max(n, 1))()
+        load().ckks_linear_proj_rotations(self._h, C.byref(d), buf, n)
+        return list(buf)[:n]
+
+    def linear_proj_workspace_bytes(self, d_in, d_out, tokens_per_shard, nshards, baby, level):
+        d = self._desc(d_in, d_out, tokens_per_shard, nshards, baby)
+        return int(load().ckks_linear_proj_workspace_bytes(self._h, C.byref(d), level))
+
+    def linear_proj(self, cts, W: torch.Tensor, keys, d_in, d_out, tokens_per_shard, nshards, baby, pt_scale=0.0,
+                    outs=None, ws: torch.Tensor = None, stream=None):
+        """Y = X W.  cts: nshards * n_in_blocks ciphertexts; W: fp64 [d_in][d_out] on the device;
+        keys: rotation SwitchKeys.  Returns nshards * n_out_blocks ciphertexts at level - 1."""
+        if not (W.is_cuda and W.dtype == torch.float64 and W.is_contiguous() and tuple(W.shape) == (d_in, d_out)):
+            raise TypeError("W must be a contiguous CUDA float64 [d_in][d_out] tensor")
+        d = self._desc(d_in, d_out, tokens_per_shard, nshards, baby, pt_scale)
+        level = cts[0].level
+        F = self.n // tokens_per_shard
+        nob = -(-d_out // F)
+        if outs is None:
+            outs = [self.empty_ct(level - 1) for _ in range(nshards * nob)]
+        if ws is None:
+            ws = self.workspace(self.linear_proj_workspace_bytes(d_in, d_out, tokens_per_shard, nshards, baby, level))
+        ia = (CCt * len(cts))(*[_cct(c) for c in cts])
+        oa = (CCt * len(outs))(*[_cct(o) for o in outs])
+        for o in oa:
+            o.level = level - 1
+        ka = (CEvk * len(keys))(*[CEvk(_dev_u64(k.data).data_ptr(), k.galois) for k in keys])
+        self._check(load().ckks_linear_proj(self._h, C.byref(d), ia, W.data_ptr(), ka, len(keys), oa, ws.data_ptr(),
+                                            ws.numel(), _stream_ptr(stream)))
+        for o, c in zip(outs, oa):
+            o.scale = c.scale
+        return outs

@@ -1,0 +1,398 @@
+// C ABI layer: argument validation on the host, then the kernel sequences.
+#include <math.h>
+
+#include <algorithm>
+#include <set>
+
+#include "common.cuh"
+
+namespace {
+
+struct DeviceGuard {
+    int prev = 0;
+    explicit DeviceGuard(int dev) { cudaGetDevice(&prev); cudaSetDevice(dev); }
+    ~DeviceGuard() { cudaSetDevice(prev); }
+};
+
+int finish(ckks_ctx *c) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { c->cuda_error = cudaGetErrorString(e); return CKKS_ERR_CUDA; }
+    return CKKS_OK;
+}
+
+bool scales_agree(double a, double b) { return fabs(a - b) <= ldexp(fmax(fabs(a), fabs(b)), -30); }
+bool level_ok(const ckks_ctx *c, uint32_t level) { return level >= 1 && level <= c->L; }
+bool ct_ok(const ckks_ct *ct) { return ct && ct->data; }
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+size_t ks_bytes(const ckks_ctx *c, uint32_t level) { return ks_workspace_limbs(c, level) * c->N * sizeof(u64); }
+size_t rescale_bytes(const ckks_ctx *c, uint32_t level, uint32_t ncomp) { return (size_t)ncomp * level * c->N * sizeof(u64); }
+
+// ---- projection plan -------------------------------------------------------
+struct Block { uint32_t start, size; };
+struct ProjPlan {
+    uint32_t F, T, B, S;
+    std::vector<Block> ins, outs;
+    std::vector<int64_t> rots;
+    uint32_t gmax;   // largest giant-step count over block pairs
+};
+
+int split_blocks(uint32_t d, uint32_t F, std::vector<Block> &out) {
+    for (uint32_t s = 0; s < d;) {
+        uint32_t m = std::min(F, d - s);
+        if (F % m) return CKKS_ERR_UNSUPPORTED;
+        out.push_back({s, m});
+        s += m;
+    }
+    return CKKS_OK;
+}
+
+int make_plan(const ckks_ctx *c, const ckks_proj_desc *d, ProjPlan &p) {
+    if (!d || !d->d_in || !d->d_out || !d->tokens_per_shard || !d->nshards || !d->baby) return CKKS_ERR_ARG;
+    if (c->n % d->tokens_per_shard) return CKKS_ERR_UNSUPPORTED;
+    p.T = d->tokens_per_shard; p.F = c->n / p.T; p.B = d->baby; p.S = d->nshards;
+    int rc;
+    if ((rc = split_blocks(d->d_in, p.F, p.ins)) || (rc = split_blocks(d->d_out, p.F, p.outs))) return rc;
+    std::set<int64_t> rots;
+    for (uint32_t b = 1; b < p.B; b++) rots.insert((int64_t)b * p.T);
+    p.gmax = 0;
+    for (const Block &o : p.outs) {
+        int64_t fold = -1;
+        for (const Block &i : p.ins) {
+            uint32_t nd = std::min(i.size, o.size);
+            if (nd % p.B) return CKKS_ERR_UNSUPPORTED;
+            p.gmax = std::max(p.gmax, nd / p.B);
+            for (uint32_t g = 1; g < nd / p.B; g++) rots.insert((int64_t)g * p.B * p.T);
+            int64_t f = i.size > o.size ? i.size / o.size : 1;
+            if (fold >= 0 && fold != f) return CKKS_ERR_UNSUPPORTED;
+            fold = f;
+            for (uint32_t x = o.size; x < i.size; x *= 2) rots.insert((int64_t)x * p.T);
+        }
+    }
+    p.rots.assign(rots.begin(), rots.end());
+    return CKKS_OK;
+}
+
+struct ProjWs { size_t baby, pts, slots, enc, acc, total, tmp, ks, rs, bytes; };
+
+ProjWs proj_layout(const ckks_ctx *c, const ProjPlan &p, uint32_t level) {
+    const size_t ct = (size_t)2 * level * c->N * sizeof(u64), pt = (size_t)level * c->N * sizeof(u64);
+    const size_t nib = p.ins.size();
+    ProjWs w;
+    size_t off = 0;
+    w.baby = off;  off += align256(ct * p.S * nib * p.B);
+    w.pts = off;   off += align256(pt * nib * p.B);
+    w.slots = off; off += align256((size_t)p.B * c->n * sizeof(double));
+    w.enc = off;   off += align256(encode_workspace_bytes(c, p.B));
+    w.acc = off;   off += align256(ct * p.S);
+    w.total = off; off += align256(ct * p.S);
+    w.tmp = off;   off += align256(ct);
+    w.ks = off;    off += align256(ks_bytes(c, level));
+    w.rs = off;    off += align256(rescale_bytes(c, level, 2));
+    w.bytes = off;
+    return w;
+}
+
+const ckks_evk *find_key(const ckks_evk *keys, uint32_t nkeys, u64 g) {
+    for (uint32_t i = 0; i < nkeys; i++)
+        if (keys[i].galois == g && keys[i].data) return &keys[i];
+    return nullptr;
+}
+
+// acc[s][c][i][p] = sum_{j < J} ct_j[s][c][i][p] * pt_j[i][p], ct_j[s] at base + (s*sstride + j) * ct_limbs
+__global__ void __launch_bounds__(256) mac_sum_kernel(DevTables c, const u64 *baby, size_t sstride, const u64 *pts, uint32_t J,
+                                                      u64 *acc, uint32_t level) {
+    const uint32_t p = blockIdx.x * 256 + threadIdx.x;
+    const uint32_t i = blockIdx.y % level, comp = blockIdx.y / level, s = blockIdx.z;
+    const size_t ctl = (size_t)2 * level * c.N;
+    const u64 q = c.mod[i], mu = c.mu[i];
+    const u64 *ct = baby + (size_t)s * sstride * ctl + ((size_t)comp * level + i) * c.N + p;
+    const u64 *pt = pts + (size_t)i * c.N + p;
+    u64 hi = 0, lo = 0;
+    for (uint32_t j = 0; j < J; j++) mac128(hi, lo, ct[(size_t)j * ctl], pt[(size_t)j * level * c.N]);
+    acc[(size_t)s * ctl + ((size_t)comp * level + i) * c.N + p] = barrett112(hi, lo, q, mu);
+}
+
+}  // namespace
+
+extern "C" size_t ckks_workspace_bytes(const ckks_ctx *c, int32_t op, uint32_t level, uint32_t count) {
+    if (!c || !level_ok(c, level)) return 0;
+    const size_t limb = (size_t)c->N * sizeof(u64);
+    switch (op) {
+        case CKKS_OP_ENCODE: return encode_workspace_bytes(c, count ? count : 1);
+        case CKKS_OP_MUL_RELIN: return ks_bytes(c, level) + (size_t)level * limb;
+        case CKKS_OP_ROTATE:
+        case CKKS_OP_ROTATE_HOISTED: return ks_bytes(c, level);
+        case CKKS_OP_RESCALE: return rescale_bytes(c, level, 2);
+        default: return 0;
+    }
+}
+
+extern "C" int32_t ckks_ntt(ckks_ctx *c, uint64_t *polys, uint32_t batch, uint32_t first, uint32_t nlimbs, void *stream) {
+    if (!c || !polys || !batch || !nlimbs) return CKKS_ERR_ARG;
+    if ((uint64_t)first + nlimbs > c->T) return CKKS_ERR_LEVEL;
+    DeviceGuard g(c->device);
+    launch_ntt(c, (u64 *)polys, batch * nlimbs, LimbMap{0, first, nlimbs, 0, 0, 0, 0}, false, (cudaStream_t)stream);
+    return finish(c);
+}
+
+extern "C" int32_t ckks_intt(ckks_ctx *c, uint64_t *polys, uint32_t batch, uint32_t first, uint32_t nlimbs, void *stream) {
+    if (!c || !polys || !batch || !nlimbs) return CKKS_ERR_ARG;
+    if ((uint64_t)first + nlimbs > c->T) return CKKS_ERR_LEVEL;
+    DeviceGuard g(c->device);
+    launch_ntt(c, (u64 *)polys, batch * nlimbs, LimbMap{0, first, nlimbs, 0, 0, 0, 0}, true, (cudaStream_t)stream);
+    return finish(c);
+}
+
+extern "C" int32_t ckks_encode(ckks_ctx *c, const double *re, const double *im, uint32_t batch, double scale, uint32_t level,
+                               uint64_t *out, void *ws, size_t ws_bytes, void *stream) {
+    if (!c || !re || !out || !batch || !(scale > 0.0) || !isfinite(scale)) return CKKS_ERR_ARG;
+    if (!level_ok(c, level)) return CKKS_ERR_LEVEL;
+    if (!ws || ws_bytes < encode_workspace_bytes(c, batch)) return CKKS_ERR_WORKSPACE;
+    DeviceGuard g(c->device);
+    launch_encode(c, re, im, batch, scale, level, (u64 *)out, ws, (cudaStream_t)stream);
+    return finish(c);
+}
+
+extern "C" int32_t ckks_encode_range_flag(ckks_ctx *c, void *stream) {
+    if (!c) return CKKS_ERR_ARG;
+    DeviceGuard g(c->device);
+    int flag = 0;
+    cudaError_t e = cudaMemcpyAsync(&flag, c->dev.range_flag, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e == cudaSuccess && flag) e = cudaMemsetAsync(c->dev.range_flag, 0, sizeof(int), (cudaStream_t)stream);
+    if (e != cudaSuccess) { c->cuda_error = cudaGetErrorString(e); return CKKS_ERR_CUDA; }
+    return flag ? CKKS_ERR_RANGE : CKKS_OK;
+}
+
+extern "C" int32_t ckks_mul_plain_acc(ckks_ctx *c, const ckks_ct *cts, uint32_t ncts, const ckks_pt *pt, ckks_ct *accs,
+                                      int32_t init, void *stream) {
+    if (!c || !cts || !ncts || !pt || !pt->data || !accs) return CKKS_ERR_ARG;
+    const uint32_t level = pt->level;
+    if (!level_ok(c, level)) return CKKS_ERR_LEVEL;
+    for (uint32_t s = 0; s < ncts; s++) {
+        if (!cts[s].data || !accs[s].data || cts[s].ncomp != 2) return CKKS_ERR_ARG;
+        if (cts[s].level != level) return CKKS_ERR_LEVEL;
+        if (!init) {
+            if (accs[s].ncomp != 2) return CKKS_ERR_ARG;
+            if (accs[s].level != level) return CKKS_ERR_LEVEL;
+            if (!scales_agree(cts[s].scale * pt->scale, accs[s].scale)) return CKKS_ERR_SCALE;
+        }
+    }
+    DeviceGuard g(c->device);
+    std::vector<const u64 *> cp(ncts);
+    std::vector<u64 *> ap(ncts);
+    for (uint32_t s = 0; s < ncts; s++) { cp[s] = (const u64 *)cts[s].data; ap[s] = (u64 *)accs[s].data; }
+    launch_mul_plain_acc(c, cp.data(), ap.data(), ncts, (const u64 *)pt->data, level, init != 0, (cudaStream_t)stream);
+    int rc = finish(c);
+    if (rc == CKKS_OK && init)
+        for (uint32_t s = 0; s < ncts; s++) { accs[s].level = level; accs[s].ncomp = 2; accs[s].scale = cts[s].scale * pt->scale; }
+    return rc;
+}
+
+extern "C" int32_t ckks_add(ckks_ctx *c, const ckks_ct *a, const ckks_ct *b, ckks_ct *out, void *stream) {
+    if (!c || !ct_ok(a) || !ct_ok(b) || !ct_ok(out) || a->ncomp != b->ncomp || !a->ncomp) return CKKS_ERR_ARG;
+    if (!level_ok(c, a->level) || a->level != b->level) return CKKS_ERR_LEVEL;
+    if (!scales_agree(a->scale, b->scale)) return CKKS_ERR_SCALE;
+    DeviceGuard g(c->device);
+    launch_add(c, (const u64 *)a->data, (const u64 *)b->data, (u64 *)out->data, a->ncomp, a->level, (cudaStream_t)stream);
+    int rc = finish(c);
+    if (rc == CKKS_OK) { out->level = a->level; out->ncomp = a->ncomp; out->scale = a->scale; }
+    return rc;
+}
+
+extern "C" int32_t ckks_mul_relin(ckks_ctx *c, const ckks_ct *a, const ckks_ct *b, const ckks_evk *rlk, ckks_ct *out, void *ws,
+                                  size_t ws_bytes, void *stream) {
+    if (!c || !ct_ok(a) || !ct_ok(b) || !ct_ok(out) || a->ncomp != 2 || b->ncomp != 2) return CKKS_ERR_ARG;
+    if (!level_ok(c, a->level) || a->level != b->level) return CKKS_ERR_LEVEL;
+    if (!rlk || !rlk->data || rlk->galois != 0) return CKKS_ERR_NO_KEY;
+    const uint32_t level = a->level;
+    if (!ws || ws_bytes < ckks_workspace_bytes(c, CKKS_OP_MUL_RELIN, level, 0)) return CKKS_ERR_WORKSPACE;
+    DeviceGuard g(c->device);
+    cudaStream_t s = (cudaStream_t)stream;
+    u64 *e2 = (u64 *)ws;
+    KsWorkspace w = ks_carve(c, level, e2 + (size_t)level * c->N);
+    u64 *o = (u64 *)out->data;
+    launch_tensor(c, (const u64 *)a->data, (const u64 *)b->data, o, e2, level, s);
+    ks_modup(c, e2, 1, level, w, s);
+    ks_inner_moddown(c, (const u64 *)rlk->data, level, 1, w, o, o + (size_t)level * c->N, 1, o, s);
+    int rc = finish(c);
+    if (rc == CKKS_OK) { out->level = level; out->ncomp = 2; out->scale = a->scale * b->scale; }
+    return rc;
+}
+
+static int rotate_checks(const ckks_ctx *c, const ckks_ct *in, const ckks_evk *keys, uint32_t nrot, const ckks_ct *outs,
+                         const void *ws, size_t ws_bytes) {
+    if (!c || !ct_ok(in) || !keys || !outs || !nrot || in->ncomp != 2) return CKKS_ERR_ARG;
+    if (!level_ok(c, in->level)) return CKKS_ERR_LEVEL;
+    for (uint32_t r = 0; r < nrot; r++) {
+        if (!outs[r].data || outs[r].data == in->data) return CKKS_ERR_ARG;
+        if (!keys[r].data || !(keys[r].galois & 1) || keys[r].galois >= 2ull * c->N) return CKKS_ERR_NO_KEY;
+    }
+    if (!ws || ws_bytes < ks_bytes(c, in->level)) return CKKS_ERR_WORKSPACE;
+    return CKKS_OK;
+}
+
+extern "C" int32_t ckks_rotate(ckks_ctx *c, const ckks_ct *in, const ckks_evk *key, ckks_ct *out, void *ws, size_t ws_bytes,
+                               void *stream) {
+    int rc = rotate_checks(c, in, key, 1, out, ws, ws_bytes);
+    if (rc) return rc;
+    DeviceGuard g(c->device);
+    cudaStream_t s = (cudaStream_t)stream;
+    const uint32_t level = in->level;
+    KsWorkspace w = ks_carve(c, level, ws);
+    const u64 *c0 = (const u64 *)in->data, *c1 = c0 + (size_t)level * c->N;
+    ks_modup(c, c1, key->galois, level, w, s);
+    ks_inner_moddown(c, (const u64 *)key->data, level, 1, w, c0, nullptr, key->galois, (u64 *)out->data, s);
+    rc = finish(c);
+    if (rc == CKKS_OK) { out->level = level; out->ncomp = 2; out->scale = in->scale; }
+    return rc;
+}
+
+extern "C" int32_t ckks_rotate_hoisted(ckks_ctx *c, const ckks_ct *in, const ckks_evk *keys, uint32_t nrot, ckks_ct *outs,
+                                       void *ws, size_t ws_bytes, void *stream) {
+    int rc = rotate_checks(c, in, keys, nrot, outs, ws, ws_bytes);
+    if (rc) return rc;
+    DeviceGuard g(c->device);
+    cudaStream_t s = (cudaStream_t)stream;
+    const uint32_t level = in->level;
+    KsWorkspace w = ks_carve(c, level, ws);
+    const u64 *c0 = (const u64 *)in->data, *c1 = c0 + (size_t)level * c->N;
+    ks_modup(c, c1, 1, level, w, s);
+    for (uint32_t r = 0; r < nrot; r++)
+        ks_inner_moddown(c, (const u64 *)keys[r].data, level, keys[r].galois, w, c0, nullptr, keys[r].galois, (u64 *)outs[r].data, s);
+    rc = finish(c);
+    if (rc == CKKS_OK)
+        for (uint32_t r = 0; r < nrot; r++) { outs[r].level = level; outs[r].ncomp = 2; outs[r].scale = in->scale; }
+    return rc;
+}
+
+extern "C" int32_t ckks_rescale(ckks_ctx *c, const ckks_ct *in, ckks_ct *out, void *ws, size_t ws_bytes, void *stream) {
+    if (!c || !ct_ok(in) || !ct_ok(out) || !in->ncomp || in->ncomp > 3) return CKKS_ERR_ARG;
+    if (!level_ok(c, in->level) || in->level < 2) return CKKS_ERR_LEVEL;
+    if (in->ncomp > 1 && in->data == out->data) return CKKS_ERR_ARG;
+    if (!ws || ws_bytes < rescale_bytes(c, in->level, in->ncomp)) return CKKS_ERR_WORKSPACE;
+    DeviceGuard g(c->device);
+    launch_rescale(c, (const u64 *)in->data, (u64 *)out->data, in->ncomp, in->level, (u64 *)ws, (cudaStream_t)stream);
+    int rc = finish(c);
+    if (rc == CKKS_OK) {
+        const double ql = (double)c->mod[in->level - 1];
+        out->ncomp = in->ncomp; out->scale = in->scale / ql; out->level = in->level - 1;
+    }
+    return rc;
+}
+
+extern "C" int32_t ckks_linear_proj_rotations(const ckks_ctx *c, const ckks_proj_desc *d, int64_t *rots, uint32_t cap) {
+    if (!c) return CKKS_ERR_ARG;
+    ProjPlan p;
+    int rc = make_plan(c, d, p);
+    if (rc) return rc;
+    for (uint32_t i = 0; i < p.rots.size() && i < cap && rots; i++) rots[i] = p.rots[i];
+    return (int32_t)p.rots.size();
+}
+
+extern "C" size_t ckks_linear_proj_workspace_bytes(const ckks_ctx *c, const ckks_proj_desc *d, uint32_t level) {
+    if (!c || !level_ok(c, level) || level < 2) return 0;
+    ProjPlan p;
+    if (make_plan(c, d, p)) return 0;
+    return proj_layout(c, p, level).bytes;
+}
+
+extern "C" int32_t ckks_linear_proj(ckks_ctx *c, const ckks_proj_desc *d, const ckks_ct *in, const double *W, const ckks_evk *keys,
+                                    uint32_t nkeys, ckks_ct *out, void *ws, size_t ws_bytes, void *stream) {
+    if (!c || !in || !W || !keys || !out) return CKKS_ERR_ARG;
+    ProjPlan p;
+    int rc = make_plan(c, d, p);
+    if (rc) return rc;
+    const uint32_t nib = (uint32_t)p.ins.size(), nob = (uint32_t)p.outs.size(), S = p.S, B = p.B, T = p.T, N = c->N;
+    const uint32_t level = in[0].level;
+    if (!level_ok(c, level) || level < 2) return CKKS_ERR_LEVEL;
+    for (uint32_t x = 0; x < S * nib; x++) {
+        if (!in[x].data || in[x].ncomp != 2) return CKKS_ERR_ARG;
+        if (in[x].level != level) return CKKS_ERR_LEVEL;
+        if (!scales_agree(in[x].scale, in[0].scale)) return CKKS_ERR_SCALE;
+    }
+    for (uint32_t x = 0; x < S * nob; x++)
+        if (!out[x].data) return CKKS_ERR_ARG;
+    for (int64_t r : p.rots)
+        if (!find_key(keys, nkeys, ckks_galois_element(c, r))) return CKKS_ERR_NO_KEY;
+    const ProjWs L = proj_layout(c, p, level);
+    if (!ws || ws_bytes < L.bytes) return CKKS_ERR_WORKSPACE;
+    const double pt_scale = d->pt_scale > 0.0 ? d->pt_scale : (double)c->mod[level - 1];
+
+    DeviceGuard g(c->device);
+    cudaStream_t s = (cudaStream_t)stream;
+    char *base = (char *)ws;
+    const size_t ctl = (size_t)2 * level * N, ptl = (size_t)level * N;
+    u64 *baby = (u64 *)(base + L.baby), *pts = (u64 *)(base + L.pts), *acc = (u64 *)(base + L.acc);
+    u64 *total = (u64 *)(base + L.total), *tmp = (u64 *)(base + L.tmp), *rsw = (u64 *)(base + L.rs);
+    double *slots = (double *)(base + L.slots);
+    void *encw = base + L.enc;
+    KsWorkspace kw = ks_carve(c, level, base + L.ks);
+
+    // baby[(sh*nib + ib)*B + b] = rho^(b T)(x_{sh,ib}), hoisted per input ciphertext
+    for (uint32_t sh = 0; sh < S; sh++)
+        for (uint32_t ib = 0; ib < nib; ib++) {
+            const u64 *x = (const u64 *)in[sh * nib + ib].data;
+            u64 *slot0 = baby + ((size_t)(sh * nib + ib) * B) * ctl;
+            cudaMemcpyAsync(slot0, x, ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+            if (B > 1) {
+                ks_modup(c, x + ptl, 1, level, kw, s);
+                for (uint32_t b = 1; b < B; b++) {
+                    const u64 ge = ckks_galois_element(c, (int64_t)b * T);
+                    ks_inner_moddown(c, (const u64 *)find_key(keys, nkeys, ge)->data, level, ge, kw, x, nullptr, ge, slot0 + (size_t)b * ctl, s);
+                }
+            }
+        }
+
+    for (uint32_t ob = 0; ob < nob; ob++) {
+        const Block &o = p.outs[ob];
+        uint32_t gcount = 0, fold = 1;
+        for (const Block &i : p.ins) {
+            gcount = std::max(gcount, std::min(i.size, o.size) / B);
+            if (i.size > o.size) fold = i.size / o.size;
+        }
+        for (uint32_t gi = 0; gi < gcount; gi++) {
+            // contributing input blocks form a prefix (a smaller trailing block drops out first)
+            uint32_t nact = 0;
+            for (uint32_t ib = 0; ib < nib; ib++)
+                if (gi < std::min(p.ins[ib].size, o.size) / B) nact = ib + 1;
+            for (uint32_t ib = 0; ib < nact; ib++) {
+                const Block &i = p.ins[ib];
+                launch_extract_diagonals(c, W, d->d_out, i.start, i.size, o.start, o.size, p.F, T, gi * B, B, gi * B, slots, s);
+                launch_encode(c, slots, nullptr, B, pt_scale, level, pts + (size_t)ib * B * ptl, encw, s);
+            }
+            u64 *dst = gi == 0 ? total : acc;
+            mac_sum_kernel<<<dim3(N / 256, 2 * level, S), 256, 0, s>>>(c->dev, baby, (size_t)nib * B, pts, nact * B, dst, level);
+            if (gi) {
+                const u64 ge = ckks_galois_element(c, (int64_t)gi * B * T);
+                const u64 *key = (const u64 *)find_key(keys, nkeys, ge)->data;
+                for (uint32_t sh = 0; sh < S; sh++) {
+                    u64 *a = acc + (size_t)sh * ctl, *t = total + (size_t)sh * ctl;
+                    ks_modup(c, a + ptl, ge, level, kw, s);
+                    ks_inner_moddown(c, key, level, 1, kw, a, nullptr, ge, tmp, s);
+                    launch_add(c, t, tmp, t, 2, level, s);
+                }
+            }
+        }
+        for (uint32_t f = o.size; fold > 1; f *= 2, fold /= 2) {
+            const u64 ge = ckks_galois_element(c, (int64_t)f * T);
+            const u64 *key = (const u64 *)find_key(keys, nkeys, ge)->data;
+            for (uint32_t sh = 0; sh < S; sh++) {
+                u64 *t = total + (size_t)sh * ctl;
+                ks_modup(c, t + ptl, ge, level, kw, s);
+                ks_inner_moddown(c, key, level, 1, kw, t, nullptr, ge, tmp, s);
+                launch_add(c, t, tmp, t, 2, level, s);
+            }
+        }
+        for (uint32_t sh = 0; sh < S; sh++)
+            launch_rescale(c, total + (size_t)sh * ctl, (u64 *)out[sh * nob + ob].data, 2, level, rsw, s);
+    }
+    rc = finish(c);
+    if (rc == CKKS_OK)
+        for (uint32_t x = 0; x < S * nob; x++) {
+            out[x].level = level - 1; out[x].ncomp = 2;
+            out[x].scale = in[0].scale * pt_scale / (double)c->mod[level - 1];
+        }
+    return rc;
+}

@@ -1,0 +1,145 @@
+// Shared declarations of the ckks_b200 library: context, device tables,
+// modular arithmetic for 50-bit primes, kernel launch entry points.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "../../include/ckks_b200.h"
+
+typedef unsigned long long u64;
+typedef unsigned __int128 u128;
+
+// ---------------------------------------------------------------------------
+// Device-side view of the context tables (plain pointers, passed by value).
+// Prime index space t: 0..L-1 = q_i, L..L+K-1 = p_k.
+// ---------------------------------------------------------------------------
+struct DevTables {
+    uint32_t log_n, N, L, K, alpha, T, dnum;
+    const u64 *mod;          // [T]
+    const u64 *mu;           // [T] floor(2^112 / prime)
+    const ulonglong2 *tw_fwd;  // [T][N] {psi^bitrev(i), Shoup companion}, index m+i
+    const ulonglong2 *tw_inv;  // [T][N] inverses of the same
+    const ulonglong2 *n_inv;   // [T] {N^-1, Shoup}
+    // ModUp, per level l (1..L), digit j, source a < alpha:
+    const ulonglong2 *up_hat_inv;  // [(L+1)][dnum][alpha]        {qhat^-1 mod q_src, Shoup}
+    const u64 *up_hat_mod;         // [(L+1)][dnum][alpha][T]     qhat mod target
+    // ModDown:
+    const ulonglong2 *dn_hat_inv;  // [K]      {Phat_k^-1 mod p_k, Shoup}
+    const u64 *dn_hat_mod;         // [L][K]   Phat_k mod q_i
+    const ulonglong2 *dn_p_inv;    // [L]      {P^-1 mod q_i, Shoup}
+    // Rescale: [L(last)][L(i)] {q_last^-1 mod q_i, Shoup}
+    const ulonglong2 *rs_inv;
+    // Encode:
+    const uint32_t *enc_src;       // [n] slot index feeding FFT input position pos (bit-reversed e_j)
+    const double2 *enc_omega;      // [n] exp(2 pi i t / n)
+    const double2 *enc_zeta;       // [n] exp(2 pi i k / 2N)
+    int *range_flag;               // sticky encode overflow flag
+};
+
+struct ckks_ctx {
+    uint32_t log_n, N, n, L, K, dnum, alpha, T;
+    int device;
+    std::vector<u64> mod;        // host copy of the primes
+    std::vector<u64> pow5;       // 5^j mod 2N, j < n (host)
+    DevTables dev;               // pointers into `allocs`
+    std::vector<void *> allocs;  // device allocations owned by the context
+    std::string cuda_error;
+};
+
+// ---------------------------------------------------------------------------
+// Limb addressing for batched limb-wise kernels (NTT): limb y of a buffer
+// [..][period][N] -> prime index, or -1 to skip the limb.
+//   kind 0: prime = first + y % period
+//   kind 1: "extended" layout [digit][level + K]: x = y % period is q_x for
+//           x < level, else p_{x-level}; with skip_own the digit's own limbs
+//           (which never leave the evaluation domain) are skipped.
+// ---------------------------------------------------------------------------
+struct LimbMap {
+    uint32_t kind, first, period, level, L, alpha, skip_own;
+};
+
+__host__ __device__ inline int limb_prime(const LimbMap &m, uint32_t y) {
+    uint32_t x = y % m.period;
+    if (m.kind == 0) return (int)(m.first + x);
+    if (m.skip_own) {
+        uint32_t j = y / m.period, lo = j * m.alpha, hi = lo + m.alpha < m.level ? lo + m.alpha : m.level;
+        if (x >= lo && x < hi) return -1;
+    }
+    return x < m.level ? (int)x : (int)(m.L + (x - m.level));
+}
+
+// ---------------------------------------------------------------------------
+// Modular arithmetic, primes in (2^49, 2^50).
+// ---------------------------------------------------------------------------
+
+// x * w mod q for a constant w with companion wp = floor(w 2^64 / q); result in [0, 2q) for ANY 64-bit x.
+__device__ __forceinline__ u64 mul_shoup_lazy(u64 x, u64 w, u64 wp, u64 q) {
+    return x * w - __umul64hi(x, wp) * q;
+}
+__device__ __forceinline__ u64 mul_shoup(u64 x, u64 w, u64 wp, u64 q) {
+    u64 r = mul_shoup_lazy(x, w, wp, q);
+    return r >= q ? r - q : r;
+}
+__device__ __forceinline__ u64 add_mod(u64 a, u64 b, u64 q) { u64 s = a + b; return s >= q ? s - q : s; }
+__device__ __forceinline__ u64 sub_mod(u64 a, u64 b, u64 q) { return a >= b ? a - b : a + q - b; }
+
+// (hi:lo) mod q for a value below 2^112; mu = floor(2^112 / q).
+// qhat = floor((x >> 48) mu / 2^64) is in (x/q - 2, x/q], so one conditional subtraction finishes.
+__device__ __forceinline__ u64 barrett112(u64 hi, u64 lo, u64 q, u64 mu) {
+    u64 xh = (hi << 16) | (lo >> 48);
+    u64 qhat = __umul64hi(xh, mu);
+    u64 r = lo - qhat * q;
+    return r >= q ? r - q : r;
+}
+__device__ __forceinline__ u64 mul_mod(u64 a, u64 b, u64 q, u64 mu) {
+    return barrett112(__umul64hi(a, b), a * b, q, mu);
+}
+// 128-bit lazy accumulator: acc += a * b
+__device__ __forceinline__ void mac128(u64 &hi, u64 &lo, u64 a, u64 b) {
+    u64 pl = a * b, ph = __umul64hi(a, b);
+    lo += pl;
+    hi += ph + (lo < pl);
+}
+// Representative of the centred lift of y (mod src) taken modulo dst, for primes of equal bit length:
+// y <= (src-1)/2 stays, else y - src + dst (positive because dst > src/2).
+__device__ __forceinline__ u64 centred_to(u64 y, u64 src, u64 dst) {
+    return y > (src >> 1) ? y + dst - src : y;
+}
+
+__device__ __forceinline__ uint32_t bitrev_n(uint32_t x, uint32_t bits) { return __brev(x) >> (32 - bits); }
+
+// ---------------------------------------------------------------------------
+// Internal launchers (each validates nothing; the C ABI layer does).
+// ---------------------------------------------------------------------------
+void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbMap &map, bool inverse, cudaStream_t s);
+
+void launch_mul_plain_acc(const ckks_ctx *c, const u64 *const *cts, u64 *const *accs, uint32_t ncts, const u64 *pt,
+                          uint32_t level, bool init, cudaStream_t s);
+void launch_add(const ckks_ctx *c, const u64 *a, const u64 *b, u64 *out, uint32_t ncomp, uint32_t level, cudaStream_t s);
+void launch_automorphism(const ckks_ctx *c, const u64 *in, u64 *out, uint32_t nlimbs, u64 galois, cudaStream_t s);
+void launch_tensor(const ckks_ctx *c, const u64 *a, const u64 *b, u64 *e01, u64 *e2, uint32_t level, cudaStream_t s);
+
+// Key switch pieces.  Sizes in limbs: d [level], ext [beta][level+K], u [2][level+K], conv [2][level].
+struct KsWorkspace { u64 *dcoef, *ext, *u, *conv; };
+size_t ks_workspace_limbs(const ckks_ctx *c, uint32_t level);
+KsWorkspace ks_carve(const ckks_ctx *c, uint32_t level, void *ws);
+// sigma_g(d) (d evaluation domain, [level][N]; g = 1: identity) -> ext (evaluation domain, all digits)
+void ks_modup(const ckks_ctx *c, const u64 *d, u64 galois, uint32_t level, const KsWorkspace &w, cudaStream_t s);
+// inner product with evk (digits read through sigma_{ext_galois}; 1 = identity), ModDown, and the final
+// combination out_c = sigma_{add_galois}(add_c) + k_c.  add0/add1 may be null.
+void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext_galois, const KsWorkspace &w,
+                      const u64 *add0, const u64 *add1, u64 add_galois, u64 *out, cudaStream_t s);
+
+void launch_rescale(const ckks_ctx *c, const u64 *in, u64 *out, uint32_t ncomp, uint32_t level, u64 *ws, cudaStream_t s);
+
+size_t encode_workspace_bytes(const ckks_ctx *c, uint32_t batch);
+void launch_encode(const ckks_ctx *c, const double *re, const double *im, uint32_t batch, double scale, uint32_t level,
+                   u64 *out, void *ws, cudaStream_t s);
+// Slot vectors of pre-rotated generalised diagonals, [count][n] fp64, for k = k0 .. k0+count-1 of one block pair.
+void launch_extract_diagonals(const ckks_ctx *c, const double *W, uint32_t d_out_total, uint32_t in0, uint32_t m_in,
+                              uint32_t out0, uint32_t m_out, uint32_t F, uint32_t T, uint32_t k0, uint32_t count,
+                              uint32_t pre_rot, double *slots, cudaStream_t s);

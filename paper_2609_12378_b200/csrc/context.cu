@@ -1,0 +1,250 @@
+// Context: parameter validation, host-side table construction, upload.
+#include <math.h>
+#include <string.h>
+
+#include <algorithm>
+
+#include "common.cuh"
+
+namespace {
+
+u64 h_mul(u64 a, u64 b, u64 q) { return (u64)((u128)a * b % q); }
+u64 h_pow(u64 a, u64 e, u64 q) {
+    u64 r = 1;
+    a %= q;
+    for (; e; e >>= 1) {
+        if (e & 1) r = h_mul(r, a, q);
+        a = h_mul(a, a, q);
+    }
+    return r;
+}
+u64 h_inv(u64 a, u64 q) { return h_pow(a, q - 2, q); }
+u64 h_shoup(u64 w, u64 q) { return (u64)(((u128)w << 64) / q); }
+ulonglong2 h_pair(u64 w, u64 q) { return make_ulonglong2(w, h_shoup(w, q)); }
+
+bool h_is_prime(u64 n) {
+    static const u64 bases[] = {2, 3, 5, 7, 11, 13, 17, 19, 23, 29, 31, 37};
+    if (n < 2) return false;
+    for (u64 b : bases) {
+        if (n % b == 0) return n == b;
+    }
+    u64 d = n - 1;
+    int s = 0;
+    while (!(d & 1)) { d >>= 1; s++; }
+    for (u64 a : bases) {
+        u64 x = h_pow(a, d, n);
+        if (x == 1 || x == n - 1) continue;
+        bool comp = true;
+        for (int i = 1; i < s && comp; i++) {
+            x = h_mul(x, x, n);
+            if (x == n - 1) comp = false;
+        }
+        if (comp) return false;
+    }
+    return true;
+}
+
+uint32_t h_bitrev(uint32_t x, uint32_t bits) {
+    uint32_t r = 0;
+    for (uint32_t i = 0; i < bits; i++) { r = (r << 1) | ((x >> i) & 1); }
+    return r;
+}
+
+// Smallest primitive 2N-th root of unity mod q: scan the odd powers of any one of them.
+u64 h_min_root(u64 q, u64 N) {
+    u64 r = 0;
+    for (u64 x = 2;; x++) {
+        r = h_pow(x, (q - 1) / (2 * N), q);
+        if (h_pow(r, N, q) == q - 1) break;
+    }
+    u64 r2 = h_mul(r, r, q), cur = r, best = r;
+    for (u64 k = 0; k < N; k++) {
+        best = std::min(best, cur);
+        cur = h_mul(cur, r2, q);
+    }
+    return best;
+}
+
+template <class V>
+int upload(ckks_ctx *c, const std::vector<V> &v, const V **dst) {
+    void *p = nullptr;
+    size_t bytes = std::max<size_t>(v.size(), 1) * sizeof(V);
+    cudaError_t e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) { c->cuda_error = cudaGetErrorString(e); return CKKS_ERR_CUDA; }
+    c->allocs.push_back(p);
+    if (!v.empty()) {
+        e = cudaMemcpy(p, v.data(), v.size() * sizeof(V), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) { c->cuda_error = cudaGetErrorString(e); return CKKS_ERR_CUDA; }
+    }
+    *dst = (const V *)p;
+    return CKKS_OK;
+}
+
+}  // namespace
+
+extern "C" const char *ckks_status_string(int32_t s) {
+    switch (s) {
+        case CKKS_OK: return "ok";
+        case CKKS_ERR_ARG: return "bad argument";
+        case CKKS_ERR_LEVEL: return "bad or mismatched level";
+        case CKKS_ERR_SCALE: return "scale mismatch";
+        case CKKS_ERR_NO_KEY: return "switching key for a needed Galois element is missing";
+        case CKKS_ERR_WORKSPACE: return "workspace missing or too small";
+        case CKKS_ERR_RANGE: return "encode: scaled value out of range";
+        case CKKS_ERR_UNSUPPORTED: return "unsupported parameters";
+        case CKKS_ERR_CUDA: return "CUDA runtime error";
+        case CKKS_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+extern "C" const char *ckks_last_cuda_error(const ckks_ctx *ctx) { return ctx ? ctx->cuda_error.c_str() : ""; }
+
+extern "C" void ckks_context_destroy(ckks_ctx *ctx) {
+    if (!ctx) return;
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaSetDevice(ctx->device);
+    for (void *p : ctx->allocs) cudaFree(p);
+    cudaSetDevice(prev);
+    delete ctx;
+}
+
+extern "C" uint64_t ckks_galois_element(const ckks_ctx *ctx, int64_t r) {
+    if (!ctx) return 0;
+    int64_t n = (int64_t)ctx->n;
+    r %= n;
+    if (r < 0) r += n;
+    return ctx->pow5[(size_t)r];
+}
+
+extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
+    if (!prm || !out || !prm->q || (prm->num_p && !prm->p)) return CKKS_ERR_ARG;
+    *out = nullptr;
+    if (prm->log_n < 10 || prm->log_n > 16) return CKKS_ERR_UNSUPPORTED;
+    if (prm->num_q == 0 || prm->dnum == 0 || prm->dnum > prm->num_q || prm->num_q > 64 || prm->num_p > 64) return CKKS_ERR_UNSUPPORTED;
+    const uint32_t L = prm->num_q, K = prm->num_p, T = L + K, N = 1u << prm->log_n, n = N / 2;
+    const uint32_t alpha = (L + prm->dnum - 1) / prm->dnum;
+    if (K < alpha) return CKKS_ERR_UNSUPPORTED;
+    std::vector<u64> mod(T);
+    for (uint32_t t = 0; t < T; t++) mod[t] = t < L ? prm->q[t] : prm->p[t - L];
+    for (uint32_t t = 0; t < T; t++) {
+        u64 m = mod[t];
+        if (m <= (1ull << 49) || m >= (1ull << 50) || m % (2ull * N) != 1 || !h_is_prime(m)) return CKKS_ERR_UNSUPPORTED;
+        for (uint32_t s = 0; s < t; s++)
+            if (mod[s] == m) return CKKS_ERR_UNSUPPORTED;
+    }
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || prm->device < 0 || prm->device >= ndev) return CKKS_ERR_CUDA;
+
+    ckks_ctx *c = new ckks_ctx();
+    c->log_n = prm->log_n; c->N = N; c->n = n; c->L = L; c->K = K; c->dnum = prm->dnum; c->alpha = alpha; c->T = T;
+    c->device = prm->device;
+    c->mod = mod;
+    c->pow5.resize(n);
+    c->pow5[0] = 1;
+    for (uint32_t j = 1; j < n; j++) c->pow5[j] = c->pow5[j - 1] * 5 % (2ull * N);
+
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaSetDevice(c->device);
+
+    // ---- per-prime scalars and twiddles
+    std::vector<u64> mu(T);
+    std::vector<ulonglong2> ninv(T), twf((size_t)T * N), twi((size_t)T * N);
+    for (uint32_t t = 0; t < T; t++) {
+        u64 m = mod[t];
+        mu[t] = (u64)((((u128)1) << 112) / m);
+        ninv[t] = h_pair(h_inv(N % m, m), m);
+        u64 psi = h_min_root(m, N), psi_inv = h_inv(psi, m);
+        std::vector<u64> pw(N), pwi(N);
+        pw[0] = pwi[0] = 1;
+        for (uint32_t j = 1; j < N; j++) { pw[j] = h_mul(pw[j - 1], psi, m); pwi[j] = h_mul(pwi[j - 1], psi_inv, m); }
+        for (uint32_t i = 0; i < N; i++) {
+            uint32_t r = h_bitrev(i, prm->log_n);
+            twf[(size_t)t * N + i] = h_pair(pw[r], m);
+            twi[(size_t)t * N + i] = h_pair(pwi[r], m);
+        }
+    }
+
+    // ---- ModUp constants for every level
+    const uint32_t dn = prm->dnum;
+    std::vector<ulonglong2> up_inv((size_t)(L + 1) * dn * alpha, make_ulonglong2(0, 0));
+    std::vector<u64> up_mod((size_t)(L + 1) * dn * alpha * T, 0);
+    for (uint32_t lvl = 1; lvl <= L; lvl++)
+        for (uint32_t j = 0; j * alpha < lvl; j++) {
+            uint32_t lo = j * alpha, hi = std::min(lo + alpha, lvl);
+            for (uint32_t a = lo; a < hi; a++) {
+                u64 qa = mod[a], h = 1;
+                for (uint32_t b = lo; b < hi; b++)
+                    if (b != a) h = h_mul(h, mod[b] % qa, qa);
+                size_t base = ((size_t)lvl * dn + j) * alpha + (a - lo);
+                up_inv[base] = h_pair(h_inv(h, qa), qa);
+                for (uint32_t t = 0; t < T; t++) {
+                    u64 mt = mod[t], v = 1;
+                    for (uint32_t b = lo; b < hi; b++)
+                        if (b != a) v = h_mul(v, mod[b] % mt, mt);
+                    up_mod[base * T + t] = v;
+                }
+            }
+        }
+
+    // ---- ModDown constants
+    std::vector<ulonglong2> dn_inv(K), dn_pinv(L);
+    std::vector<u64> dn_mod((size_t)L * K);
+    for (uint32_t a = 0; a < K; a++) {
+        u64 pa = mod[L + a], h = 1;
+        for (uint32_t b = 0; b < K; b++)
+            if (b != a) h = h_mul(h, mod[L + b] % pa, pa);
+        dn_inv[a] = h_pair(h_inv(h, pa), pa);
+    }
+    for (uint32_t i = 0; i < L; i++) {
+        u64 q = mod[i], Pm = 1;
+        for (uint32_t a = 0; a < K; a++) {
+            u64 v = 1;
+            for (uint32_t b = 0; b < K; b++)
+                if (b != a) v = h_mul(v, mod[L + b] % q, q);
+            dn_mod[(size_t)i * K + a] = v;
+            Pm = h_mul(Pm, mod[L + a] % q, q);
+        }
+        dn_pinv[i] = h_pair(h_inv(Pm, q), q);
+    }
+
+    // ---- Rescale constants
+    std::vector<ulonglong2> rs((size_t)L * L, make_ulonglong2(0, 0));
+    for (uint32_t last = 0; last < L; last++)
+        for (uint32_t i = 0; i < L; i++)
+            if (i != last) rs[(size_t)last * L + i] = h_pair(h_inv(mod[last] % mod[i], mod[i]), mod[i]);
+
+    // ---- Encode tables: input permutation and fp64 twiddles from the host libm
+    std::vector<uint32_t> enc_src(n);
+    std::vector<double2> om(n), ze(n);
+    for (uint32_t j = 0; j < n; j++) {
+        uint32_t e = (uint32_t)((c->pow5[j] - 1) / 4);
+        enc_src[h_bitrev(e, prm->log_n - 1)] = j;
+    }
+    for (uint32_t t = 0; t < n; t++) {
+        om[t] = make_double2(cos(2.0 * M_PI * (double)t / (double)n), sin(2.0 * M_PI * (double)t / (double)n));
+        ze[t] = make_double2(cos(2.0 * M_PI * (double)t / (double)(2.0 * N)), sin(2.0 * M_PI * (double)t / (double)(2.0 * N)));
+    }
+
+    DevTables &d = c->dev;
+    d.log_n = prm->log_n; d.N = N; d.L = L; d.K = K; d.alpha = alpha; d.T = T; d.dnum = prm->dnum;
+    int rc = CKKS_OK;
+    std::vector<int> flag(1, 0);
+    const int *flag_dev = nullptr;
+    if ((rc = upload(c, mod, &d.mod)) || (rc = upload(c, mu, &d.mu)) || (rc = upload(c, twf, &d.tw_fwd)) ||
+        (rc = upload(c, twi, &d.tw_inv)) || (rc = upload(c, ninv, &d.n_inv)) || (rc = upload(c, up_inv, &d.up_hat_inv)) ||
+        (rc = upload(c, up_mod, &d.up_hat_mod)) || (rc = upload(c, dn_inv, &d.dn_hat_inv)) ||
+        (rc = upload(c, dn_mod, &d.dn_hat_mod)) || (rc = upload(c, dn_pinv, &d.dn_p_inv)) || (rc = upload(c, rs, &d.rs_inv)) ||
+        (rc = upload(c, enc_src, &d.enc_src)) || (rc = upload(c, om, &d.enc_omega)) || (rc = upload(c, ze, &d.enc_zeta)) ||
+        (rc = upload(c, flag, &flag_dev))) {
+        cudaSetDevice(prev);
+        ckks_context_destroy(c);
+        return rc;
+    }
+    d.range_flag = const_cast<int *>(flag_dev);
+    cudaSetDevice(prev);
+    *out = c;
+    return CKKS_OK;
+}

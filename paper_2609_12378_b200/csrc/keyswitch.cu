@@ -1,0 +1,174 @@
+// Hybrid key switching (dnum digits, K special primes) and rescale.
+//
+// KeySwitch(d, evk):  d (evaluation domain, `level` limbs)
+//   1. to the coefficient domain (inverse NTT)
+//   2. ModUp: every active digit j is extended from its own limbs to all active
+//      q-limbs and all special limbs by a centred fast basis conversion
+//         y_a = centre([d_a * qhat_a^-1]_{q_a}),  ext_j[t] = sum_a y_a (qhat_a mod t)  mod t
+//   3. NTT of the converted limbs (own limbs keep their evaluation values)
+//   4. inner product with the key: u_c[t] = sum_j ext_j[t] * evk_{j,c}[t]
+//   5. ModDown: inverse NTT of the special limbs, centred conversion P -> q_i,
+//      NTT, out_i = (u_i - conv_i) * P^-1 mod q_i.
+// Rescale drops the last limb the same way with a single source limb.
+#include "common.cuh"
+
+namespace {
+
+constexpr uint32_t THREADS = 256;
+
+__device__ __forceinline__ uint32_t galois_src(uint32_t p, u64 g, uint32_t log_n, uint32_t N) {
+    if (g == 1) return p;
+    const u64 e = (g * (2ull * bitrev_n(p, log_n) + 1)) & (2ull * N - 1);
+    return bitrev_n((uint32_t)((e - 1) >> 1), log_n);
+}
+
+// dst[i][p] = src[i][pi_g(p)]  (g = 1: copy)
+__global__ void __launch_bounds__(THREADS) permute_kernel(DevTables c, const u64 *src, u64 *dst, u64 g) {
+    const uint32_t p = blockIdx.x * THREADS + threadIdx.x;
+    const size_t row = (size_t)blockIdx.y * c.N;
+    dst[row + p] = src[row + galois_src(p, g, c.log_n, c.N)];
+}
+
+// ext[j][x][k] for x over q_0..q_{level-1}, p_0..p_{K-1}.  dcoef: sigma_g(d) in the coefficient domain;
+// deval: d in the evaluation domain, read through sigma_g for the digit's own limbs.
+__global__ void __launch_bounds__(THREADS) modup_kernel(DevTables c, const u64 *dcoef, const u64 *deval, u64 g,
+                                                        u64 *ext, uint32_t level) {
+    const uint32_t k = blockIdx.x * THREADS + threadIdx.x;
+    const uint32_t x = blockIdx.y, j = blockIdx.z;
+    const uint32_t nt = level + c.K, lo = j * c.alpha, hi = min(lo + c.alpha, level);
+    u64 *dst = ext + ((size_t)j * nt + x) * c.N + k;
+    if (x >= lo && x < hi) {
+        *dst = deval[(size_t)x * c.N + galois_src(k, g, c.log_n, c.N)];
+        return;
+    }
+    const uint32_t t = x < level ? x : c.L + (x - level);
+    const u64 mt = c.mod[t];
+    const size_t cb = ((size_t)level * c.dnum + j) * c.alpha;
+    u64 ahi = 0, alo = 0;
+    for (uint32_t a = lo; a < hi; a++) {
+        const u64 qa = c.mod[a];
+        const ulonglong2 hinv = c.up_hat_inv[cb + (a - lo)];
+        const u64 y = mul_shoup(dcoef[(size_t)a * c.N + k], hinv.x, hinv.y, qa);
+        mac128(ahi, alo, centred_to(y, qa, mt), c.up_hat_mod[(cb + (a - lo)) * c.T + t]);
+    }
+    *dst = barrett112(ahi, alo, mt, c.mu[t]);
+}
+
+// u[comp][x][p] = sum_j ext[j][x][pi_g(p)] * evk[j][comp][kt(x)][p]
+__global__ void __launch_bounds__(THREADS) inner_product_kernel(DevTables c, const u64 *ext, const u64 *evk, u64 g,
+                                                                u64 *u, uint32_t level) {
+    const uint32_t p = blockIdx.x * THREADS + threadIdx.x;
+    const uint32_t x = blockIdx.y;
+    const uint32_t nt = level + c.K, beta = (level + c.alpha - 1) / c.alpha;
+    const uint32_t kt = x < level ? x : c.L + (x - level);
+    const u64 m = c.mod[kt], mu = c.mu[kt];
+    const uint32_t src = galois_src(p, g, c.log_n, c.N);
+    u64 h0 = 0, l0 = 0, h1 = 0, l1 = 0;
+    for (uint32_t j = 0; j < beta; j++) {
+        const u64 e = ext[((size_t)j * nt + x) * c.N + src];
+        mac128(h0, l0, e, evk[(((size_t)j * 2 + 0) * c.T + kt) * c.N + p]);
+        mac128(h1, l1, e, evk[(((size_t)j * 2 + 1) * c.T + kt) * c.N + p]);
+    }
+    u[((size_t)0 * nt + x) * c.N + p] = barrett112(h0, l0, m, mu);
+    u[((size_t)1 * nt + x) * c.N + p] = barrett112(h1, l1, m, mu);
+}
+
+// conv[comp][i][k] = sum_a centre([u_{p_a} Phat_a^-1]) (Phat_a mod q_i)  mod q_i   (coefficient domain)
+__global__ void __launch_bounds__(THREADS) moddown_conv_kernel(DevTables c, const u64 *u, u64 *conv, uint32_t level) {
+    const uint32_t k = blockIdx.x * THREADS + threadIdx.x;
+    const uint32_t i = blockIdx.y, comp = blockIdx.z;
+    const uint32_t nt = level + c.K;
+    const u64 q = c.mod[i];
+    u64 ahi = 0, alo = 0;
+    for (uint32_t a = 0; a < c.K; a++) {
+        const u64 pa = c.mod[c.L + a];
+        const ulonglong2 hinv = c.dn_hat_inv[a];
+        const u64 y = mul_shoup(u[((size_t)comp * nt + level + a) * c.N + k], hinv.x, hinv.y, pa);
+        mac128(ahi, alo, centred_to(y, pa, q), c.dn_hat_mod[(size_t)i * c.K + a]);
+    }
+    conv[((size_t)comp * level + i) * c.N + k] = barrett112(ahi, alo, q, c.mu[i]);
+}
+
+// out[comp][i][p] = (u[comp][i][p] - conv[comp][i][p]) P^-1 + add_comp[i][pi_g(p)]
+__global__ void __launch_bounds__(THREADS) moddown_final_kernel(DevTables c, const u64 *u, const u64 *conv, const u64 *add0,
+                                                                const u64 *add1, u64 g, u64 *out, uint32_t level) {
+    const uint32_t p = blockIdx.x * THREADS + threadIdx.x;
+    const uint32_t i = blockIdx.y, comp = blockIdx.z;
+    const uint32_t nt = level + c.K;
+    const u64 q = c.mod[i];
+    const ulonglong2 pinv = c.dn_p_inv[i];
+    u64 r = sub_mod(u[((size_t)comp * nt + i) * c.N + p], conv[((size_t)comp * level + i) * c.N + p], q);
+    r = mul_shoup(r, pinv.x, pinv.y, q);
+    const u64 *add = comp ? add1 : add0;
+    if (add) r = add_mod(r, add[(size_t)i * c.N + galois_src(p, g, c.log_n, c.N)], q);
+    out[((size_t)comp * level + i) * c.N + p] = r;
+}
+
+// tmp[comp][i][k] = centred lift of last[comp][k] (mod q_last) taken mod q_i
+__global__ void __launch_bounds__(THREADS) rescale_lift_kernel(DevTables c, const u64 *last, u64 *tmp, uint32_t level) {
+    const uint32_t k = blockIdx.x * THREADS + threadIdx.x;
+    const uint32_t i = blockIdx.y, comp = blockIdx.z;
+    tmp[((size_t)comp * (level - 1) + i) * c.N + k] = centred_to(last[(size_t)comp * c.N + k], c.mod[level - 1], c.mod[i]);
+}
+
+// out[comp][i][p] = (in[comp][i][p] - tmp[comp][i][p]) q_last^-1
+__global__ void __launch_bounds__(THREADS) rescale_final_kernel(DevTables c, const u64 *in, const u64 *tmp, u64 *out, uint32_t level) {
+    const uint32_t p = blockIdx.x * THREADS + threadIdx.x;
+    const uint32_t i = blockIdx.y, comp = blockIdx.z;
+    const u64 q = c.mod[i];
+    const ulonglong2 inv = c.rs_inv[(size_t)(level - 1) * c.L + i];
+    const u64 r = sub_mod(in[((size_t)comp * level + i) * c.N + p], tmp[((size_t)comp * (level - 1) + i) * c.N + p], q);
+    out[((size_t)comp * (level - 1) + i) * c.N + p] = mul_shoup(r, inv.x, inv.y, q);
+}
+
+inline LimbMap plain_map(uint32_t first, uint32_t period) { return LimbMap{0, first, period, 0, 0, 0, 0}; }
+
+}  // namespace
+
+size_t ks_workspace_limbs(const ckks_ctx *c, uint32_t level) {
+    const size_t beta = (level + c->alpha - 1) / c->alpha, nt = level + c->K;
+    return level + beta * nt + 2 * nt + 2 * (size_t)level;
+}
+
+KsWorkspace ks_carve(const ckks_ctx *c, uint32_t level, void *ws) {
+    const size_t beta = (level + c->alpha - 1) / c->alpha, nt = level + c->K, N = c->N;
+    KsWorkspace w;
+    w.dcoef = (u64 *)ws;
+    w.ext = w.dcoef + (size_t)level * N;
+    w.u = w.ext + beta * nt * N;
+    w.conv = w.u + 2 * nt * N;
+    return w;
+}
+
+void ks_modup(const ckks_ctx *c, const u64 *d, u64 galois, uint32_t level, const KsWorkspace &w, cudaStream_t s) {
+    const uint32_t N = c->N, beta = (level + c->alpha - 1) / c->alpha, nt = level + c->K;
+    permute_kernel<<<dim3(N / THREADS, level), THREADS, 0, s>>>(c->dev, d, w.dcoef, galois);
+    launch_ntt(c, w.dcoef, level, plain_map(0, level), true, s);
+    modup_kernel<<<dim3(N / THREADS, nt, beta), THREADS, 0, s>>>(c->dev, w.dcoef, d, galois, w.ext, level);
+    LimbMap em{1, 0, nt, level, c->L, c->alpha, 1};
+    launch_ntt(c, w.ext, beta * nt, em, false, s);
+}
+
+void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext_galois, const KsWorkspace &w,
+                      const u64 *add0, const u64 *add1, u64 add_galois, u64 *out, cudaStream_t s) {
+    const uint32_t N = c->N, nt = level + c->K, K = c->K;
+    inner_product_kernel<<<dim3(N / THREADS, nt), THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level);
+    for (uint32_t comp = 0; comp < 2; comp++)
+        launch_ntt(c, w.u + ((size_t)comp * nt + level) * N, K, plain_map(c->L, K), true, s);
+    moddown_conv_kernel<<<dim3(N / THREADS, level, 2), THREADS, 0, s>>>(c->dev, w.u, w.conv, level);
+    launch_ntt(c, w.conv, 2 * level, plain_map(0, level), false, s);
+    moddown_final_kernel<<<dim3(N / THREADS, level, 2), THREADS, 0, s>>>(c->dev, w.u, w.conv, add0, add1, add_galois, out, level);
+}
+
+// ws: [ncomp][N] last limbs + [ncomp][level-1][N]
+void launch_rescale(const ckks_ctx *c, const u64 *in, u64 *out, uint32_t ncomp, uint32_t level, u64 *ws, cudaStream_t s) {
+    const uint32_t N = c->N;
+    u64 *last = ws, *tmp = ws + (size_t)ncomp * N;
+    for (uint32_t comp = 0; comp < ncomp; comp++)
+        cudaMemcpyAsync(last + (size_t)comp * N, in + ((size_t)comp * level + level - 1) * N, (size_t)N * 8,
+                        cudaMemcpyDeviceToDevice, s);
+    launch_ntt(c, last, ncomp, plain_map(level - 1, 1), true, s);
+    rescale_lift_kernel<<<dim3(N / THREADS, level - 1, ncomp), THREADS, 0, s>>>(c->dev, last, tmp, level);
+    launch_ntt(c, tmp, ncomp * (level - 1), plain_map(0, level - 1), false, s);
+    rescale_final_kernel<<<dim3(N / THREADS, level - 1, ncomp), THREADS, 0, s>>>(c->dev, in, tmp, out, level);
+}

@@ -1,0 +1,105 @@
+// Pointwise (coefficient-wise) kernels on evaluation-domain limbs: ciphertext x
+// plaintext multiply-accumulate, addition, tensor product, Galois automorphism.
+// All are streaming kernels bound by HBM bandwidth: 128-bit loads and stores,
+// one pass over each operand.
+#include "common.cuh"
+
+namespace {
+
+constexpr uint32_t THREADS = 256;
+constexpr uint32_t MAC_MAX = 32;   // ciphertexts per launch
+
+struct MacArgs {
+    const u64 *ct[MAC_MAX];
+    u64 *acc[MAC_MAX];
+};
+
+// acc[s][c][i][k] (+)= ct[s][c][i][k] * pt[i][k]; one thread owns two adjacent coefficients of one (c, i).
+template <bool INIT>
+__global__ void __launch_bounds__(THREADS) mac_kernel(DevTables c, MacArgs a, uint32_t ncts, const u64 *pt, uint32_t level) {
+    const uint32_t half = c.N / 2;
+    const uint32_t x = blockIdx.x * THREADS + threadIdx.x;   // pair index inside the limb
+    const uint32_t limb = blockIdx.y, comp = blockIdx.z;
+    if (x >= half) return;
+    const u64 q = c.mod[limb], mu = c.mu[limb];
+    const ulonglong2 p = reinterpret_cast<const ulonglong2 *>(pt + (size_t)limb * c.N)[x];
+    const size_t off = ((size_t)comp * level + limb) * half + x;
+    for (uint32_t s = 0; s < ncts; s++) {
+        ulonglong2 v = reinterpret_cast<const ulonglong2 *>(a.ct[s])[off];
+        ulonglong2 r;
+        r.x = mul_mod(v.x, p.x, q, mu);
+        r.y = mul_mod(v.y, p.y, q, mu);
+        ulonglong2 *dst = reinterpret_cast<ulonglong2 *>(a.acc[s]) + off;
+        if (!INIT) {
+            ulonglong2 o = *dst;
+            r.x = add_mod(r.x, o.x, q);
+            r.y = add_mod(r.y, o.y, q);
+        }
+        *dst = r;
+    }
+}
+
+__global__ void __launch_bounds__(THREADS) add_kernel(DevTables c, const u64 *a, const u64 *b, u64 *out, uint32_t level) {
+    const uint32_t half = c.N / 2;
+    const uint32_t x = blockIdx.x * THREADS + threadIdx.x;
+    if (x >= half) return;
+    const u64 q = c.mod[blockIdx.y % level];
+    const size_t off = (size_t)blockIdx.y * half + x;
+    ulonglong2 u = reinterpret_cast<const ulonglong2 *>(a)[off], v = reinterpret_cast<const ulonglong2 *>(b)[off];
+    reinterpret_cast<ulonglong2 *>(out)[off] = make_ulonglong2(add_mod(u.x, v.x, q), add_mod(u.y, v.y, q));
+}
+
+// out[y][p] = in[y][pi(p)], 2 bitrev(pi(p)) + 1 = g (2 bitrev(p) + 1) mod 2N
+__global__ void __launch_bounds__(THREADS) automorphism_kernel(DevTables c, const u64 *in, u64 *out, u64 g) {
+    const uint32_t p = blockIdx.x * THREADS + threadIdx.x;
+    if (p >= c.N) return;
+    const u64 e = (g * (2ull * bitrev_n(p, c.log_n) + 1)) & (2ull * c.N - 1);
+    const uint32_t src = bitrev_n((uint32_t)((e - 1) >> 1), c.log_n);
+    out[(size_t)blockIdx.y * c.N + p] = in[(size_t)blockIdx.y * c.N + src];
+}
+
+// (a0 b0, a0 b1 + a1 b0) -> e01 [2][level][N];  a1 b1 -> e2 [level][N]
+__global__ void __launch_bounds__(THREADS) tensor_kernel(DevTables c, const u64 *a, const u64 *b, u64 *e01, u64 *e2, uint32_t level) {
+    const uint32_t k = blockIdx.x * THREADS + threadIdx.x;
+    if (k >= c.N) return;
+    const uint32_t limb = blockIdx.y;
+    const u64 q = c.mod[limb], mu = c.mu[limb];
+    const size_t o0 = (size_t)limb * c.N + k, o1 = o0 + (size_t)level * c.N;
+    const u64 a0 = a[o0], a1 = a[o1], b0 = b[o0], b1 = b[o1];
+    u64 hi = 0, lo = 0;
+    mac128(hi, lo, a0, b1);
+    mac128(hi, lo, a1, b0);
+    const u64 r0 = mul_mod(a0, b0, q, mu), r1 = barrett112(hi, lo, q, mu), r2 = mul_mod(a1, b1, q, mu);
+    e01[o0] = r0;
+    e01[o1] = r1;
+    e2[o0] = r2;
+}
+
+}  // namespace
+
+void launch_mul_plain_acc(const ckks_ctx *c, const u64 *const *cts, u64 *const *accs, uint32_t ncts, const u64 *pt,
+                          uint32_t level, bool init, cudaStream_t s) {
+    dim3 grid((c->N / 2 + THREADS - 1) / THREADS, level, 2);
+    for (uint32_t s0 = 0; s0 < ncts; s0 += MAC_MAX) {
+        MacArgs a;
+        uint32_t n = ncts - s0 < MAC_MAX ? ncts - s0 : MAC_MAX;
+        for (uint32_t i = 0; i < n; i++) { a.ct[i] = cts[s0 + i]; a.acc[i] = accs[s0 + i]; }
+        if (init) mac_kernel<true><<<grid, THREADS, 0, s>>>(c->dev, a, n, pt, level);
+        else mac_kernel<false><<<grid, THREADS, 0, s>>>(c->dev, a, n, pt, level);
+    }
+}
+
+void launch_add(const ckks_ctx *c, const u64 *a, const u64 *b, u64 *out, uint32_t ncomp, uint32_t level, cudaStream_t s) {
+    dim3 grid((c->N / 2 + THREADS - 1) / THREADS, ncomp * level);
+    add_kernel<<<grid, THREADS, 0, s>>>(c->dev, a, b, out, level);
+}
+
+void launch_automorphism(const ckks_ctx *c, const u64 *in, u64 *out, uint32_t nlimbs, u64 galois, cudaStream_t s) {
+    dim3 grid((c->N + THREADS - 1) / THREADS, nlimbs);
+    automorphism_kernel<<<grid, THREADS, 0, s>>>(c->dev, in, out, galois);
+}
+
+void launch_tensor(const ckks_ctx *c, const u64 *a, const u64 *b, u64 *e01, u64 *e2, uint32_t level, cudaStream_t s) {
+    dim3 grid((c->N + THREADS - 1) / THREADS, level);
+    tensor_kernel<<<grid, THREADS, 0, s>>>(c->dev, a, b, e01, e2, level);
+}

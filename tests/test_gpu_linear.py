@@ -1,0 +1,90 @@
+"""GPU parity: the linear projection (Eq. 5, baby-step/giant-step), bit-exact on every
+output limb against the CPU checker, and X W after decryption."""
+import numpy as np
+import pytest
+
+from oracle.ckks_oracle import ProjDesc
+from paper_2609_12378_b200 import binding, inputs
+from tests.harness import Client, params
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(log_n, L, K, dnum, level, d_in, d_out, T, S, B, seed, pt_scale=0.0, check_slots=True):
+    from tests.gpu_util import context, ct_dev, dev, host, key_dev
+    P, ctx = params(log_n, L, K, dnum), context(log_n, L, K, dnum)
+    o = P.oracle
+    cl = Client(P, seed)
+    scale = 2.0 ** 40
+    g = inputs.rng(seed, 1)
+    X = inputs.activations_uniform(g, S * T, d_in)
+    W = inputs.weights_normal(g, d_in, d_out, 0.02)
+    desc = ProjDesc(d_in, d_out, T, S, B, pt_scale)
+    F, ins, outs = o.proj_blocks(desc)
+    cts = []
+    for c in range(S):
+        for (s0, mi) in ins:
+            cts.append(cl.encrypt_slots(inputs.pack_feature_major(X[c * T:(c + 1) * T, s0:s0 + mi], T, o.n)[0], scale, level))
+    rots = o.proj_rotations(desc)
+    assert rots == ctx.linear_proj_rotations(d_in, d_out, T, S, B)
+    keys = {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in rots}
+    want, want_scale = o.linear_proj(desc, np.stack(cts), W, keys, scale)
+    got = ctx.linear_proj([ct_dev(c, scale) for c in cts], dev(W), [key_dev(k, g_) for g_, k in keys.items()],
+                          d_in, d_out, T, S, B, pt_scale)
+    assert len(got) == S * len(outs)
+    Y = X @ W
+    for i, ct in enumerate(got):
+        arr = host(ct.data)
+        assert ct.scale == want_scale and ct.level == level - 1
+        assert np.array_equal(arr, want[i]), i
+        if check_slots:
+            c, ob = divmod(i, len(outs))
+            o0, mo = outs[ob]
+            sl = cl.decrypt_slots(arr, ct.scale).real.reshape(F, T)
+            for r in range(0, F, max(1, F // 16)):
+                assert np.abs(sl[r] - Y[c * T:(c + 1) * T, o0 + r % mo]).max() < 2.0 ** -20
+    return ctx, cts, keys
+
+
+@pytest.mark.parametrize("d_in,d_out,T,S,B", [
+    (16, 16, 32, 2, 4),      # square
+    (16, 4, 32, 2, 2),       # wide with fold (K/V-like)
+    (16, 24, 32, 1, 4),      # several output blocks, remainder output block (gate/up-like)
+    (24, 16, 32, 2, 4),      # several input blocks, remainder input block (down-like)
+    (8, 8, 32, 1, 8),        # replicated small block, single giant step
+    (16, 16, 32, 1, 1),      # no baby rotations at all
+])
+def test_projection_shapes_small_ring(d_in, d_out, T, S, B):
+    _run(10, 4, 2, 2, 4, d_in, d_out, T, S, B, seed=400 + d_in + d_out)
+
+
+def test_projection_explicit_pt_scale_and_lower_level():
+    _run(10, 4, 2, 2, 3, 16, 16, 32, 1, 4, seed=410, pt_scale=2.0 ** 40, check_slots=False)
+
+
+def test_projection_toy_config():
+    """N = 2^13, 6 + 1 primes, dnum = 6, 32 tokens x 64 features times 64 x 64, B = G = 8."""
+    ctx, cts, keys = _run(13, 6, 1, 6, 6, 64, 64, 32, 1, 8, seed=1001)
+    assert len(keys) == 14
+
+
+def test_projection_full_ring_small_shape():
+    """N = 2^16, L = 24, dnum = 3 with 512 tokens per shard: F = 64 features, B = G = 8."""
+    _run(16, 24, 8, 3, 24, 64, 64, 512, 1, 8, seed=420)
+
+
+def test_projection_errors():
+    from tests.gpu_util import context, ct_dev, dev, key_dev
+    P, ctx = params(10, 4, 2, 2), context(10, 4, 2, 2)
+    cl = Client(P, 430)
+    ct = ct_dev(cl.encrypt_slots(np.zeros(P.n), 2.0 ** 40, 4), 2.0 ** 40)
+    W = dev(np.zeros((16, 16)))
+    with pytest.raises(binding.CkksError) as e:
+        ctx.linear_proj([ct], W, [key_dev(np.zeros((2, 2, 6, P.N), dtype=np.uint64), 5)], 16, 16, 32, 1, 4)
+    assert e.value.code == binding.ERR_NO_KEY
+    with pytest.raises(binding.CkksError) as e:
+        ctx.linear_proj_rotations(16, 16, 32, 1, 3)        # B must divide the diagonal count
+    assert e.value.code == binding.ERR_UNSUPPORTED
+    with pytest.raises(binding.CkksError) as e:
+        ctx.linear_proj_rotations(12, 16, 32, 1, 4)        # remainder block 12 does not divide F = 16
+    assert e.value.code == binding.ERR_UNSUPPORTED

@@ -1,0 +1,127 @@
+"""GPU parity: pointwise ops, rescale, rotations, relinearised product -- every RNS
+integer output bit-exact against the CPU checker; decrypted slots within 2^-20."""
+import numpy as np
+import pytest
+
+from paper_2609_12378_b200 import binding, inputs
+from tests.harness import Client, params
+
+pytestmark = pytest.mark.gpu
+
+SETS = [(10, 6, 2, 3), (11, 4, 4, 1), (13, 6, 1, 6), (16, 24, 8, 3)]
+
+
+def _random_ct(P, level, seed, ncomp=2):
+    return inputs.uniform_residues(inputs.rng(seed, level), P.q[:level], P.N, ncomp)
+
+
+@pytest.mark.parametrize("log_n,L,K,dnum", SETS)
+def test_mul_plain_acc_and_add(log_n, L, K, dnum):
+    from tests.gpu_util import context, ct_dev, dev, host
+    P, ctx = params(log_n, L, K, dnum), context(log_n, L, K, dnum)
+    o = P.oracle
+    for level in (L, 1):
+        cts = [_random_ct(P, level, 200 + s) for s in range(3)]
+        pt = inputs.uniform_residues(inputs.rng(210, level), P.q[:level], P.N)[0]
+        pt2 = inputs.uniform_residues(inputs.rng(211, level), P.q[:level], P.N)[0]
+        dcts = [ct_dev(c, 2.0 ** 40) for c in cts]
+        accs = ctx.mul_plain_acc(dcts, binding.Plaintext(dev(pt), 2.0 ** 30))
+        want = [o.mul_plain_acc(c, pt) for c in cts]
+        for a, w in zip(accs, want):
+            assert a.scale == 2.0 ** 70 and np.array_equal(host(a.data), w)
+        ctx.mul_plain_acc(dcts[::-1], binding.Plaintext(dev(pt2), 2.0 ** 30), accs)
+        for a, w, c in zip(accs, want, cts[::-1]):
+            assert np.array_equal(host(a.data), o.mul_plain_acc(c, pt2, w.copy()))
+        s = ctx.add(dcts[0], dcts[1])
+        assert np.array_equal(host(s.data), o.add(cts[0], cts[1]))
+        with pytest.raises(binding.CkksError) as e:
+            ctx.mul_plain_acc(dcts, binding.Plaintext(dev(pt), 2.0 ** 31), accs)
+        assert e.value.code == binding.ERR_SCALE
+
+
+@pytest.mark.parametrize("log_n,L,K,dnum", SETS)
+def test_rescale_bit_exact(log_n, L, K, dnum):
+    from tests.gpu_util import context, ct_dev, host
+    P, ctx = params(log_n, L, K, dnum), context(log_n, L, K, dnum)
+    for level in sorted({L, 2, max(2, L - 1)}):
+        ct = _random_ct(P, level, 220)
+        out = ctx.rescale(ct_dev(ct, 2.0 ** 80))
+        assert out.level == level - 1 and out.scale == 2.0 ** 80 / float(P.q[level - 1])
+        assert np.array_equal(host(out.data), P.oracle.rescale(ct))
+    with pytest.raises(binding.CkksError) as e:
+        ctx.rescale(ct_dev(_random_ct(P, 1, 221), 1.0))
+    assert e.value.code == binding.ERR_LEVEL
+
+
+@pytest.mark.parametrize("log_n,L,K,dnum,levels", [(10, 6, 2, 3, (6, 5, 2, 1)), (11, 4, 4, 1, (4, 3)), (13, 6, 1, 6, (6, 3)), (16, 24, 8, 3, (24, 17))])
+def test_rotate_and_hoisted_bit_exact(log_n, L, K, dnum, levels):
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    P, ctx = params(log_n, L, K, dnum), context(log_n, L, K, dnum)
+    o = P.oracle
+    cl = Client(P, 230)
+    rots = [1, 8, P.n - 3]
+    gals = [o.galois_element(r) for r in rots]
+    assert gals == [ctx.galois_element(r) for r in rots]
+    keys = [cl.rotation_key(g) for g in gals]
+    dkeys = [key_dev(k, g) for k, g in zip(keys, gals)]
+    z = inputs.rng(231, log_n).uniform(-1, 1, P.n)
+    for level in levels:
+        ct = cl.encrypt_slots(z, 2.0 ** 40, level)
+        dct = ct_dev(ct, 2.0 ** 40)
+        for k, dk, g in zip(keys, dkeys, gals):
+            out = ctx.rotate(dct, dk)
+            assert np.array_equal(host(out.data), o.rotate(ct, k, g)), (level, g)
+        outs = ctx.rotate_hoisted(dct, dkeys)
+        want = o.rotate_hoisted(ct, keys, gals)
+        for i, out in enumerate(outs):
+            got = host(out.data)
+            assert np.array_equal(got, want[i]), (level, i)
+            if level >= 2:
+                assert np.abs(cl.decrypt_slots(got, 2.0 ** 40).real - np.roll(z, -rots[i])).max() < 2.0 ** -20
+    # error paths: even Galois element, aliasing, short workspace
+    bad = binding.SwitchKey(dkeys[0].data, 4)
+    with pytest.raises(binding.CkksError) as e:
+        ctx.rotate(dct, bad)
+    assert e.value.code == binding.ERR_NO_KEY
+    with pytest.raises(binding.CkksError) as e:
+        ctx.rotate(dct, dkeys[0], out=dct)
+    assert e.value.code == binding.ERR_ARG
+
+
+@pytest.mark.parametrize("log_n,L,K,dnum,levels", [(10, 6, 2, 3, (6, 4, 1)), (13, 6, 1, 6, (6,)), (16, 24, 8, 3, (24,))])
+def test_mul_relin_bit_exact(log_n, L, K, dnum, levels):
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    P, ctx = params(log_n, L, K, dnum), context(log_n, L, K, dnum)
+    o = P.oracle
+    cl = Client(P, 240)
+    rlk = cl.relin_key()
+    drlk = key_dev(rlk, 0)
+    g = inputs.rng(241, log_n)
+    z, w = g.uniform(-1, 1, P.n), g.uniform(-1, 1, P.n)
+    for level in levels:
+        sb = float(P.q[level - 1])
+        ca, cb = cl.encrypt_slots(z, 2.0 ** 40, level), cl.encrypt_slots(w, sb, level)
+        out = ctx.mul_relin(ct_dev(ca, 2.0 ** 40), ct_dev(cb, sb), drlk)
+        got = host(out.data)
+        assert out.scale == 2.0 ** 40 * sb
+        assert np.array_equal(got, o.mul_relin(ca, cb, rlk)), level
+        if level >= 2:
+            assert np.abs(cl.decrypt_slots(got, out.scale) - z * w).max() < 2.0 ** -20
+            rs = ctx.rescale(out)
+            assert np.abs(cl.decrypt_slots(host(rs.data), rs.scale) - z * w).max() < 2.0 ** -20
+    with pytest.raises(binding.CkksError) as e:
+        ctx.mul_relin(ct_dev(ca, 1.0), ct_dev(cb, 1.0), binding.SwitchKey(drlk.data, 5))
+    assert e.value.code == binding.ERR_NO_KEY
+
+
+def test_repeatability():
+    """Same call twice gives the same bytes (a race would show up as a difference)."""
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    P, ctx = params(13, 6, 1, 6), context(13, 6, 1, 6)
+    cl = Client(P, 250)
+    g = P.oracle.galois_element(5)
+    dk = key_dev(cl.rotation_key(g), g)
+    dct = ct_dev(cl.encrypt_slots(np.ones(P.n), 2.0 ** 40, 6), 2.0 ** 40)
+    a = host(ctx.rotate(dct, dk).data).copy()
+    for _ in range(3):
+        assert np.array_equal(host(ctx.rotate(dct, dk).data), a)
