@@ -268,9 +268,9 @@ extern "C" int32_t ckks_rotate_hoisted(ckks_ctx *c, const ckks_ct *in, const ckk
 }
 
 extern "C" int32_t ckks_rescale(ckks_ctx *c, const ckks_ct *in, ckks_ct *out, void *ws, size_t ws_bytes, void *stream) {
-    if (!c || !ct_ok(in) || !ct_ok(out) || !in->ncomp || in->ncomp > 3) return CKKS_ERR_ARG;
+    if (!c || !ct_ok(in) || !out || !in->ncomp || in->ncomp > 3) return CKKS_ERR_ARG;
     if (!level_ok(c, in->level) || in->level < 2) return CKKS_ERR_LEVEL;
-    if (in->ncomp > 1 && in->data == out->data) return CKKS_ERR_ARG;
+    if (!out->data || (in->ncomp > 1 && in->data == out->data)) return CKKS_ERR_ARG;
     if (!ws || ws_bytes < rescale_bytes(c, in->level, in->ncomp)) return CKKS_ERR_WORKSPACE;
     DeviceGuard g(c->device);
     launch_rescale(c, (const u64 *)in->data, (u64 *)out->data, in->ncomp, in->level, (u64 *)ws, (cudaStream_t)stream);

@@ -1,5 +1,7 @@
 """GPU parity: pointwise ops, rescale, rotations, relinearised product -- every RNS
-integer output bit-exact against the CPU checker; decrypted slots within 2^-20."""
+integer output bit-exact against the CPU checker (so decrypted slots agree with the
+checker's exactly, inside the 2^-20 bar); against the plaintext truth the slots are
+within the scheme's own noise: 2^-20 up to N = 2^13, 2^-17 at N = 2^16 (Delta = 2^40)."""
 import numpy as np
 import pytest
 
@@ -9,6 +11,10 @@ from tests.harness import Client, params
 pytestmark = pytest.mark.gpu
 
 SETS = [(10, 6, 2, 3), (11, 4, 4, 1), (13, 6, 1, 6), (16, 24, 8, 3)]
+
+
+def truth_tol(log_n):
+    return 2.0 ** -17 if log_n >= 16 else 2.0 ** -20
 
 
 def _random_ct(P, level, seed, ncomp=2):
@@ -77,7 +83,7 @@ def test_rotate_and_hoisted_bit_exact(log_n, L, K, dnum, levels):
             got = host(out.data)
             assert np.array_equal(got, want[i]), (level, i)
             if level >= 2:
-                assert np.abs(cl.decrypt_slots(got, 2.0 ** 40).real - np.roll(z, -rots[i])).max() < 2.0 ** -20
+                assert np.abs(cl.decrypt_slots(got, 2.0 ** 40).real - np.roll(z, -rots[i])).max() < truth_tol(log_n)
     # error paths: even Galois element, aliasing, short workspace
     bad = binding.SwitchKey(dkeys[0].data, 4)
     with pytest.raises(binding.CkksError) as e:
@@ -106,9 +112,9 @@ def test_mul_relin_bit_exact(log_n, L, K, dnum, levels):
         assert out.scale == 2.0 ** 40 * sb
         assert np.array_equal(got, o.mul_relin(ca, cb, rlk)), level
         if level >= 2:
-            assert np.abs(cl.decrypt_slots(got, out.scale) - z * w).max() < 2.0 ** -20
+            assert np.abs(cl.decrypt_slots(got, out.scale) - z * w).max() < truth_tol(log_n)
             rs = ctx.rescale(out)
-            assert np.abs(cl.decrypt_slots(host(rs.data), rs.scale) - z * w).max() < 2.0 ** -20
+            assert np.abs(cl.decrypt_slots(host(rs.data), rs.scale) - z * w).max() < truth_tol(log_n)
     with pytest.raises(binding.CkksError) as e:
         ctx.mul_relin(ct_dev(ca, 1.0), ct_dev(cb, 1.0), binding.SwitchKey(drlk.data, 5))
     assert e.value.code == binding.ERR_NO_KEY
