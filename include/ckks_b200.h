@@ -121,6 +121,9 @@ const char *ckks_last_cuda_error(const ckks_ctx *ctx);
  * ckks_linear_proj_workspace_bytes.  Returns 0 for an unknown op. */
 size_t ckks_workspace_bytes(const ckks_ctx *ctx, int32_t op, uint32_t level, uint32_t count);
 
+/* Number of kernels this library has launched since it was loaded (all contexts).  Not thread safe. */
+uint64_t ckks_kernel_launches(void);
+
 /* 5^r mod 2N with r taken mod n: Galois element of a left rotation by r slots. */
 uint64_t ckks_galois_element(const ckks_ctx *ctx, int64_t left_rot_slots);
 

@@ -21,7 +21,7 @@ EXPORTS = [
     "ckks_workspace_bytes", "ckks_galois_element", "ckks_ntt", "ckks_intt", "ckks_encode",
     "ckks_encode_range_flag", "ckks_mul_plain_acc", "ckks_add", "ckks_mul_relin", "ckks_rotate",
     "ckks_rotate_hoisted", "ckks_rescale", "ckks_linear_proj", "ckks_linear_proj_workspace_bytes",
-    "ckks_linear_proj_rotations",
+    "ckks_linear_proj_rotations", "ckks_kernel_launches",
 ]
 
 
@@ -65,6 +65,7 @@ def load():
         "ckks_status_string": (C.c_char_p, [i32]),
         "ckks_last_cuda_error": (C.c_char_p, [vp]),
         "ckks_workspace_bytes": (sz, [vp, i32, u32, u32]),
+        "ckks_kernel_launches": (u64, []),
         "ckks_galois_element": (u64, [vp, i64]),
         "ckks_ntt": (i32, [vp, vp, u32, u32, u32, vp]),
         "ckks_intt": (i32, [vp, vp, u32, u32, u32, vp]),
@@ -85,6 +86,11 @@ def load():
         f.restype, f.argtypes = res, args
     _lib = L
     return L
+
+
+def kernel_launches() -> int:
+    """Kernels launched by the library since it was loaded."""
+    return int(load().ckks_kernel_launches())
 
 
 class CkksError(RuntimeError):

@@ -363,7 +363,7 @@ extern "C" int32_t ckks_linear_proj(ckks_ctx *c, const ckks_proj_desc *d, const 
                 launch_encode(c, slots, nullptr, B, pt_scale, level, pts + (size_t)ib * B * ptl, encw, s);
             }
             u64 *dst = gi == 0 ? total : acc;
-            mac_sum_kernel<<<dim3(N / 256, 2 * level, S), 256, 0, s>>>(c->dev, baby, (size_t)nib * B, pts, nact * B, dst, level);
+            mac_sum_kernel<<<dim3(N / 256, 2 * level, S), 256, 0, s>>>(c->dev, baby, (size_t)nib * B, pts, nact * B, dst, level); count_launches();
             if (gi) {
                 const u64 ge = ckks_galois_element(c, (int64_t)gi * B * T);
                 const u64 *key = (const u64 *)find_key(keys, nkeys, ge)->data;

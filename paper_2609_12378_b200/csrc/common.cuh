@@ -112,6 +112,10 @@ __device__ __forceinline__ u64 centred_to(u64 y, u64 src, u64 dst) {
 
 __device__ __forceinline__ uint32_t bitrev_n(uint32_t x, uint32_t bits) { return __brev(x) >> (32 - bits); }
 
+// Kernel launches issued by this library since it was loaded (all contexts, all streams).
+extern unsigned long long g_kernel_launches;
+inline void count_launches(unsigned n = 1) { g_kernel_launches += n; }
+
 // ---------------------------------------------------------------------------
 // Internal launchers (each validates nothing; the C ABI layer does).
 // ---------------------------------------------------------------------------

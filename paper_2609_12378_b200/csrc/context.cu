@@ -82,6 +82,9 @@ int upload(ckks_ctx *c, const std::vector<V> &v, const V **dst) {
 
 }  // namespace
 
+unsigned long long g_kernel_launches = 0;
+extern "C" uint64_t ckks_kernel_launches(void) { return g_kernel_launches; }
+
 extern "C" const char *ckks_status_string(int32_t s) {
     switch (s) {
         case CKKS_OK: return "ok";

@@ -117,13 +117,13 @@ void launch_encode(const ckks_ctx *c, const double *re, const double *im, uint32
     for (uint32_t b0 = 0; b0 < batch; b0 += 32768) {
         const uint32_t nb = batch - b0 < 32768 ? batch - b0 : 32768;
         fft_chunks<<<dim3(n / ch, nb), THREADS, 0, s>>>(c->dev, re + (size_t)b0 * n, im ? im + (size_t)b0 * n : nullptr,
-                                                         buf + (size_t)b0 * n, n, ch);
+                                                         buf + (size_t)b0 * n, n, ch); count_launches();
         fft_strips_round<<<dim3(ch / COLS, nb), THREADS, (size_t)(n / ch) * COLS * sizeof(double2), s>>>(
-            c->dev, buf + (size_t)b0 * n, coef + (size_t)b0 * N, n, ch, sc);
+            c->dev, buf + (size_t)b0 * n, coef + (size_t)b0 * N, n, ch, sc); count_launches();
     }
     for (uint32_t b0 = 0; b0 < batch; b0 += 32768) {
         const uint32_t nb = batch - b0 < 32768 ? batch - b0 : 32768;
-        reduce_coeffs<<<dim3(N / THREADS, level, nb), THREADS, 0, s>>>(c->dev, coef + (size_t)b0 * N, out + (size_t)b0 * level * N, level);
+        reduce_coeffs<<<dim3(N / THREADS, level, nb), THREADS, 0, s>>>(c->dev, coef + (size_t)b0 * N, out + (size_t)b0 * level * N, level); count_launches();
     }
     LimbMap map{0, 0, level, 0, 0, 0, 0};
     launch_ntt(c, out, batch * level, map, false, s);
@@ -133,5 +133,5 @@ void launch_extract_diagonals(const ckks_ctx *c, const double *W, uint32_t d_out
                               uint32_t out0, uint32_t m_out, uint32_t F, uint32_t T, uint32_t k0, uint32_t count,
                               uint32_t pre_rot, double *slots, cudaStream_t s) {
     extract_diagonals<<<dim3((c->n + THREADS - 1) / THREADS, count), THREADS, 0, s>>>(W, d_out_total, in0, m_in, out0, m_out, F, T, k0,
-                                                                                       pre_rot, slots, c->n);
+                                                                                       pre_rot, slots, c->n); count_launches();
 }

@@ -142,9 +142,9 @@ KsWorkspace ks_carve(const ckks_ctx *c, uint32_t level, void *ws) {
 
 void ks_modup(const ckks_ctx *c, const u64 *d, u64 galois, uint32_t level, const KsWorkspace &w, cudaStream_t s) {
     const uint32_t N = c->N, beta = (level + c->alpha - 1) / c->alpha, nt = level + c->K;
-    permute_kernel<<<dim3(N / THREADS, level), THREADS, 0, s>>>(c->dev, d, w.dcoef, galois);
+    permute_kernel<<<dim3(N / THREADS, level), THREADS, 0, s>>>(c->dev, d, w.dcoef, galois); count_launches();
     launch_ntt(c, w.dcoef, level, plain_map(0, level), true, s);
-    modup_kernel<<<dim3(N / THREADS, nt, beta), THREADS, 0, s>>>(c->dev, w.dcoef, d, galois, w.ext, level);
+    modup_kernel<<<dim3(N / THREADS, nt, beta), THREADS, 0, s>>>(c->dev, w.dcoef, d, galois, w.ext, level); count_launches();
     LimbMap em{1, 0, nt, level, c->L, c->alpha, 1};
     launch_ntt(c, w.ext, beta * nt, em, false, s);
 }
@@ -152,12 +152,12 @@ void ks_modup(const ckks_ctx *c, const u64 *d, u64 galois, uint32_t level, const
 void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext_galois, const KsWorkspace &w,
                       const u64 *add0, const u64 *add1, u64 add_galois, u64 *out, cudaStream_t s) {
     const uint32_t N = c->N, nt = level + c->K, K = c->K;
-    inner_product_kernel<<<dim3(N / THREADS, nt), THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level);
+    inner_product_kernel<<<dim3(N / THREADS, nt), THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level); count_launches();
     for (uint32_t comp = 0; comp < 2; comp++)
         launch_ntt(c, w.u + ((size_t)comp * nt + level) * N, K, plain_map(c->L, K), true, s);
-    moddown_conv_kernel<<<dim3(N / THREADS, level, 2), THREADS, 0, s>>>(c->dev, w.u, w.conv, level);
+    moddown_conv_kernel<<<dim3(N / THREADS, level, 2), THREADS, 0, s>>>(c->dev, w.u, w.conv, level); count_launches();
     launch_ntt(c, w.conv, 2 * level, plain_map(0, level), false, s);
-    moddown_final_kernel<<<dim3(N / THREADS, level, 2), THREADS, 0, s>>>(c->dev, w.u, w.conv, add0, add1, add_galois, out, level);
+    moddown_final_kernel<<<dim3(N / THREADS, level, 2), THREADS, 0, s>>>(c->dev, w.u, w.conv, add0, add1, add_galois, out, level); count_launches();
 }
 
 // ws: [ncomp][N] last limbs + [ncomp][level-1][N]
@@ -168,7 +168,7 @@ void launch_rescale(const ckks_ctx *c, const u64 *in, u64 *out, uint32_t ncomp, 
         cudaMemcpyAsync(last + (size_t)comp * N, in + ((size_t)comp * level + level - 1) * N, (size_t)N * 8,
                         cudaMemcpyDeviceToDevice, s);
     launch_ntt(c, last, ncomp, plain_map(level - 1, 1), true, s);
-    rescale_lift_kernel<<<dim3(N / THREADS, level - 1, ncomp), THREADS, 0, s>>>(c->dev, last, tmp, level);
+    rescale_lift_kernel<<<dim3(N / THREADS, level - 1, ncomp), THREADS, 0, s>>>(c->dev, last, tmp, level); count_launches();
     launch_ntt(c, tmp, ncomp * (level - 1), plain_map(0, level - 1), false, s);
-    rescale_final_kernel<<<dim3(N / THREADS, level - 1, ncomp), THREADS, 0, s>>>(c->dev, in, tmp, out, level);
+    rescale_final_kernel<<<dim3(N / THREADS, level - 1, ncomp), THREADS, 0, s>>>(c->dev, in, tmp, out, level); count_launches();
 }

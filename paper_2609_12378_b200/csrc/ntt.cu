@@ -113,11 +113,11 @@ void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbM
         u64 *b = base + (size_t)y0 * N;
         dim3 gc(ROW / COLS, ny), gr(R / rows, ny);
         if (!inverse) {
-            ntt_cols<false><<<gc, THREADS, smc, s>>>(c->dev, b, map);
-            ntt_rows<false><<<gr, THREADS, 0, s>>>(c->dev, b, map, rows);
+            ntt_cols<false><<<gc, THREADS, smc, s>>>(c->dev, b, map); count_launches();
+            ntt_rows<false><<<gr, THREADS, 0, s>>>(c->dev, b, map, rows); count_launches();
         } else {
-            ntt_rows<true><<<gr, THREADS, 0, s>>>(c->dev, b, map, rows);
-            ntt_cols<true><<<gc, THREADS, smc, s>>>(c->dev, b, map);
+            ntt_rows<true><<<gr, THREADS, 0, s>>>(c->dev, b, map, rows); count_launches();
+            ntt_cols<true><<<gc, THREADS, smc, s>>>(c->dev, b, map); count_launches();
         }
     }
 }

@@ -84,22 +84,22 @@ void launch_mul_plain_acc(const ckks_ctx *c, const u64 *const *cts, u64 *const *
         MacArgs a;
         uint32_t n = ncts - s0 < MAC_MAX ? ncts - s0 : MAC_MAX;
         for (uint32_t i = 0; i < n; i++) { a.ct[i] = cts[s0 + i]; a.acc[i] = accs[s0 + i]; }
-        if (init) mac_kernel<true><<<grid, THREADS, 0, s>>>(c->dev, a, n, pt, level);
-        else mac_kernel<false><<<grid, THREADS, 0, s>>>(c->dev, a, n, pt, level);
+        if (init) { mac_kernel<true><<<grid, THREADS, 0, s>>>(c->dev, a, n, pt, level); count_launches(); }
+        else { mac_kernel<false><<<grid, THREADS, 0, s>>>(c->dev, a, n, pt, level); count_launches(); }
     }
 }
 
 void launch_add(const ckks_ctx *c, const u64 *a, const u64 *b, u64 *out, uint32_t ncomp, uint32_t level, cudaStream_t s) {
     dim3 grid((c->N / 2 + THREADS - 1) / THREADS, ncomp * level);
-    add_kernel<<<grid, THREADS, 0, s>>>(c->dev, a, b, out, level);
+    add_kernel<<<grid, THREADS, 0, s>>>(c->dev, a, b, out, level); count_launches();
 }
 
 void launch_automorphism(const ckks_ctx *c, const u64 *in, u64 *out, uint32_t nlimbs, u64 galois, cudaStream_t s) {
     dim3 grid((c->N + THREADS - 1) / THREADS, nlimbs);
-    automorphism_kernel<<<grid, THREADS, 0, s>>>(c->dev, in, out, galois);
+    automorphism_kernel<<<grid, THREADS, 0, s>>>(c->dev, in, out, galois); count_launches();
 }
 
 void launch_tensor(const ckks_ctx *c, const u64 *a, const u64 *b, u64 *e01, u64 *e2, uint32_t level, cudaStream_t s) {
     dim3 grid((c->N + THREADS - 1) / THREADS, level);
-    tensor_kernel<<<grid, THREADS, 0, s>>>(c->dev, a, b, e01, e2, level);
+    tensor_kernel<<<grid, THREADS, 0, s>>>(c->dev, a, b, e01, e2, level); count_launches();
 }
