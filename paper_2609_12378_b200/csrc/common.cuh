@@ -21,6 +21,7 @@ struct DevTables {
     uint32_t log_n, N, L, K, alpha, T, dnum;
     const u64 *mod;          // [T]
     const u64 *mu;           // [T] floor(2^112 / prime)
+    const u64 *mu64;         // [T] floor(2^64 / prime)
     const ulonglong2 *tw_fwd;  // [T][N] {psi^bitrev(i), Shoup companion}, index m+i
     const ulonglong2 *tw_inv;  // [T][N] inverses of the same
     const ulonglong2 *n_inv;   // [T] {N^-1, Shoup}

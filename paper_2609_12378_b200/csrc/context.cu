@@ -153,11 +153,12 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
     cudaSetDevice(c->device);
 
     // ---- per-prime scalars and twiddles
-    std::vector<u64> mu(T);
+    std::vector<u64> mu(T), mu64(T);
     std::vector<ulonglong2> ninv(T), twf((size_t)T * N), twi((size_t)T * N);
     for (uint32_t t = 0; t < T; t++) {
         u64 m = mod[t];
         mu[t] = (u64)((((u128)1) << 112) / m);
+        mu64[t] = (u64)((((u128)1) << 64) / m);
         ninv[t] = h_pair(h_inv(N % m, m), m);
         u64 psi = h_min_root(m, N), psi_inv = h_inv(psi, m);
         std::vector<u64> pw(N), pwi(N);
@@ -236,7 +237,7 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
     int rc = CKKS_OK;
     std::vector<int> flag(1, 0);
     const int *flag_dev = nullptr;
-    if ((rc = upload(c, mod, &d.mod)) || (rc = upload(c, mu, &d.mu)) || (rc = upload(c, twf, &d.tw_fwd)) ||
+    if ((rc = upload(c, mod, &d.mod)) || (rc = upload(c, mu, &d.mu)) || (rc = upload(c, mu64, &d.mu64)) || (rc = upload(c, twf, &d.tw_fwd)) ||
         (rc = upload(c, twi, &d.tw_inv)) || (rc = upload(c, ninv, &d.n_inv)) || (rc = upload(c, up_inv, &d.up_hat_inv)) ||
         (rc = upload(c, up_mod, &d.up_hat_mod)) || (rc = upload(c, dn_inv, &d.dn_hat_inv)) ||
         (rc = upload(c, dn_mod, &d.dn_hat_mod)) || (rc = upload(c, dn_pinv, &d.dn_p_inv)) || (rc = upload(c, rs, &d.rs_inv)) ||

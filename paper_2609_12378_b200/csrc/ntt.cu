@@ -4,7 +4,7 @@
 // m = 1, 2, .., N/2 with butterfly distance t = N/(2m) and twiddle psi^bitrev(m+i)
 // for block i.  Inverse: Gentleman-Sande, the same stages backwards, then N^-1.
 //
-// A limb is viewed as R rows of 256 coefficients (R = N/256).  The stages with
+// Generic path (N < 2^16).  A limb is viewed as R rows of 256 coefficients (R = N/256).  The stages with
 // distance >= 256 couple rows only ("column pass": a CTA owns all R rows of a
 // 16-column strip in shared memory); the stages with distance < 256 stay inside
 // a row ("row pass": a CTA owns 8 rows).  Each limb therefore makes two trips
@@ -99,10 +99,213 @@ __global__ void __launch_bounds__(THREADS) ntt_rows(DevTables c, u64 *base, Limb
     for (uint32_t x = threadIdx.x; x < rows * ROW; x += THREADS) g[x] = sm[x];
 }
 
+
+// ===========================================================================
+// Fast path for N = 2^16 (256 x 256): every pass is two radix-16 steps held in
+// registers (4 butterfly stages each, 16 coefficients per thread) with a single
+// shared-memory exchange in between, so a limb crosses shared memory once per
+// pass instead of once per stage.
+//
+// Lazy arithmetic.  Residues travel as 64-bit words that are only congruent to
+// the value: with 50-bit primes there are 14 spare bits.  The twiddle product
+// uses an under-estimate of floor(x w'/2^64) built from three 32x32 products
+// (the low x low product is dropped, the cross products keep their high halves),
+// at most 3 below the exact quotient, so the product lands in [0, 5q) for ANY
+// 64-bit x.  Forward (Cooley-Tukey): X' = X + T, Y' = X - T + 5q; magnitudes grow
+// by at most 5q per stage, 81q < 2^57 after 16 stages, one exact reduction at the
+// end.  Inverse (Gentleman-Sande): X' = U + V doubles the bound per stage,
+// Y' = (U - V + bound q) w' is back in [0, 5q); 8 stages keep everything below
+// 1280 q < 2^61, so one lazy reduction between the passes suffices.
+// ===========================================================================
+
+constexpr uint32_t F_THREADS = 256;
+
+__device__ __forceinline__ u64 mulhi_under(u64 x, u64 a) {
+    const uint32_t x0 = (uint32_t)x, x1 = (uint32_t)(x >> 32), a0 = (uint32_t)a, a1 = (uint32_t)(a >> 32);
+    return (u64)x1 * a1 + __umulhi(x1, a0) + __umulhi(x0, a1);
+}
+// x * w mod q up to a multiple of q, in [0, 5q), for any 64-bit x
+__device__ __forceinline__ u64 mul_tw(u64 x, ulonglong2 w, u64 q) { return x * w.x - mulhi_under(x, w.y) * q; }
+
+// 4 Cooley-Tukey stages on 16 registers; stage twiddles tw[ml*base + i], ml = 1,2,4,8
+__device__ __forceinline__ void fwd16(u64 (&x)[16], const ulonglong2 *__restrict__ tw, uint32_t base, u64 q, u64 q5) {
+#pragma unroll
+    for (uint32_t ml = 1; ml < 16; ml <<= 1) {
+        const uint32_t tl = 8 / ml;
+#pragma unroll
+        for (uint32_t i = 0; i < ml; i++) {
+            const ulonglong2 w = __ldg(&tw[ml * base + i]);
+#pragma unroll
+            for (uint32_t j = 0; j < tl; j++) {
+                const uint32_t k1 = 2 * i * tl + j, k2 = k1 + tl;
+                const u64 t = mul_tw(x[k2], w, q);
+                x[k2] = x[k1] + q5 - t;
+                x[k1] = x[k1] + t;
+            }
+        }
+    }
+}
+
+// 4 Gentleman-Sande stages (ml = 8,4,2,1); `bound` = multiple of q bounding the inputs on entry
+template <uint32_t BOUND>
+__device__ __forceinline__ void inv16(u64 (&x)[16], const ulonglong2 *__restrict__ tw, uint32_t base, u64 q) {
+    uint32_t b = BOUND;
+#pragma unroll
+    for (uint32_t ml = 8; ml >= 1; ml >>= 1) {
+        const uint32_t tl = 8 / ml;
+        const u64 off = (u64)b * q;
+#pragma unroll
+        for (uint32_t i = 0; i < ml; i++) {
+            const ulonglong2 w = __ldg(&tw[ml * base + i]);
+#pragma unroll
+            for (uint32_t j = 0; j < tl; j++) {
+                const uint32_t k1 = 2 * i * tl + j, k2 = k1 + tl;
+                const u64 u = x[k1], v = x[k2];
+                x[k1] = u + v;
+                x[k2] = mul_tw(u + off - v, w, q);
+            }
+        }
+        b = 2 * b > 5 ? 2 * b : 5;
+    }
+}
+// bound after the 4 stages of inv16<b>: b -> max(2b, 5) four times, i.e. 1 -> 40, 5 -> 80, 40 -> 640, 80 -> 1280
+
+// exact reduction of a lazy word (< 2^64) to [0, q): qinv64 = floor(2^64 / q)
+__device__ __forceinline__ u64 reduce_exact(u64 x, u64 q, u64 qinv64) {
+    u64 r = x - __umul64hi(x, qinv64) * q;     // in [0, 2q)
+    return r >= q ? r - q : r;
+}
+
+// ---- forward, column pass (stages m = 1..128): CTA = strip of 16 columns -----------------
+__global__ void __launch_bounds__(F_THREADS) ntt16_fwd_cols(DevTables c, u64 *base, LimbMap map) {
+    __shared__ u64 sm[256 * 16];
+    const int prime = limb_prime(map, blockIdx.y);
+    if (prime < 0) return;
+    const u64 q = c.mod[prime], q5 = 5 * q;
+    const ulonglong2 *tw = c.tw_fwd + ((size_t)prime << 16);
+    const uint32_t cc = threadIdx.x & 15, r = threadIdx.x >> 4;
+    u64 *g = base + ((size_t)blockIdx.y << 16) + blockIdx.x * 16 + cc;
+    u64 x[16];
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) x[k] = g[(size_t)(r + 16 * k) * 256];
+    fwd16(x, tw, 1, q, q5);
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) sm[(r + 16 * k) * 16 + cc] = x[k];
+    __syncthreads();
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) x[k] = sm[(16 * r + k) * 16 + cc];
+    fwd16(x, tw, 16 + r, q, q5);
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) g[(size_t)(16 * r + k) * 256] = x[k];
+}
+
+// padded index inside a 256-coefficient row: one spare word per 16 so that both access patterns are conflict free
+__device__ __forceinline__ uint32_t padded(uint32_t i) { return i + (i >> 4); }
+constexpr uint32_t ROW_PAD = 256 + 16;
+
+// ---- forward, row pass (stages m = 256..32768): CTA = 16 rows, 16 threads per row ---------
+__global__ void __launch_bounds__(F_THREADS) ntt16_fwd_rows(DevTables c, u64 *base, LimbMap map) {
+    __shared__ u64 sm[16 * ROW_PAD];
+    const int prime = limb_prime(map, blockIdx.y);
+    if (prime < 0) return;
+    const u64 q = c.mod[prime], q5 = 5 * q;
+    const ulonglong2 *tw = c.tw_fwd + ((size_t)prime << 16);
+    const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
+    u64 *g = base + ((size_t)blockIdx.y << 16) + (size_t)row * 256;
+    u64 *s = sm + rl * ROW_PAD;
+    u64 x[16];
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) x[k] = g[t + 16 * k];
+    fwd16(x, tw, 256 + row, q, q5);
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) s[padded(t + 16 * k)] = x[k];
+    __syncwarp();   // a row lives in one half warp
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) x[k] = s[padded(16 * t + k)];
+    fwd16(x, tw, 16 * (256 + row) + t, q, q5);
+    const u64 qinv64 = c.mu64[prime];
+    __syncwarp();
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) s[padded(16 * t + k)] = reduce_exact(x[k], q, qinv64);
+    __syncwarp();
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) g[t + 16 * k] = s[padded(t + 16 * k)];
+}
+
+// ---- inverse, row pass (stages m = 32768..256) ---------------------------------------------
+__global__ void __launch_bounds__(F_THREADS) ntt16_inv_rows(DevTables c, u64 *base, LimbMap map) {
+    __shared__ u64 sm[16 * ROW_PAD];
+    const int prime = limb_prime(map, blockIdx.y);
+    if (prime < 0) return;
+    const u64 q = c.mod[prime];
+    const ulonglong2 *tw = c.tw_inv + ((size_t)prime << 16);
+    const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
+    u64 *g = base + ((size_t)blockIdx.y << 16) + (size_t)row * 256;
+    u64 *s = sm + rl * ROW_PAD;
+    u64 x[16];
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) s[padded(t + 16 * k)] = g[t + 16 * k];
+    __syncwarp();
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) x[k] = s[padded(16 * t + k)];
+    inv16<1>(x, tw, 16 * (256 + row) + t, q);
+    __syncwarp();
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) s[padded(16 * t + k)] = x[k];
+    __syncwarp();
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) x[k] = s[padded(t + 16 * k)];
+    inv16<40>(x, tw, 256 + row, q);
+    const ulonglong2 one = make_ulonglong2(1, c.mu64[prime]);
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) g[t + 16 * k] = mul_tw(x[k], one, q);   // lazy reduction to [0, 5q)
+}
+
+// ---- inverse, column pass (stages m = 128..1), then N^-1 and the exact reduction -----------
+__global__ void __launch_bounds__(F_THREADS) ntt16_inv_cols(DevTables c, u64 *base, LimbMap map) {
+    __shared__ u64 sm[256 * 16];
+    const int prime = limb_prime(map, blockIdx.y);
+    if (prime < 0) return;
+    const u64 q = c.mod[prime];
+    const ulonglong2 *tw = c.tw_inv + ((size_t)prime << 16);
+    const uint32_t cc = threadIdx.x & 15, r = threadIdx.x >> 4;
+    u64 *g = base + ((size_t)blockIdx.y << 16) + blockIdx.x * 16 + cc;
+    u64 x[16];
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) x[k] = g[(size_t)(16 * r + k) * 256];
+    inv16<5>(x, tw, 16 + r, q);
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) sm[(16 * r + k) * 16 + cc] = x[k];
+    __syncthreads();
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) x[k] = sm[(r + 16 * k) * 16 + cc];
+    inv16<80>(x, tw, 1, q);
+    const ulonglong2 ni = c.n_inv[prime];
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) g[(size_t)(r + 16 * k) * 256] = mul_shoup(x[k], ni.x, ni.y, q);
+}
+
 }  // namespace
 
 void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbMap &map, bool inverse, cudaStream_t s) {
     if (nlimbs_total == 0) return;
+    if (c->log_n == 16) {
+        for (uint32_t y0 = 0; y0 < nlimbs_total;) {
+            const uint32_t chunk = map.period >= 32768 ? map.period : (32768 / map.period) * map.period;
+            const uint32_t ny = nlimbs_total - y0 < chunk ? nlimbs_total - y0 : chunk;
+            u64 *b = base + ((size_t)y0 << 16);
+            dim3 grid(16, ny);
+            if (!inverse) {
+                ntt16_fwd_cols<<<grid, F_THREADS, 0, s>>>(c->dev, b, map); count_launches();
+                ntt16_fwd_rows<<<grid, F_THREADS, 0, s>>>(c->dev, b, map); count_launches();
+            } else {
+                ntt16_inv_rows<<<grid, F_THREADS, 0, s>>>(c->dev, b, map); count_launches();
+                ntt16_inv_cols<<<grid, F_THREADS, 0, s>>>(c->dev, b, map); count_launches();
+            }
+            y0 += ny;
+        }
+        return;
+    }
     const uint32_t N = c->N, R = N / ROW;
     const uint32_t rows = R < ROWS_PER_CTA ? R : ROWS_PER_CTA;   // R >= 4 since N >= 1024
     const size_t smc = (size_t)R * COLS * sizeof(u64);
