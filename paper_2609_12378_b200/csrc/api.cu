@@ -73,18 +73,25 @@ int make_plan(const ckks_ctx *c, const ckks_proj_desc *d, ProjPlan &p) {
     return CKKS_OK;
 }
 
-struct ProjWs { size_t baby, pts, slots, enc, acc, total, tmp, ks, rs, bytes; };
+struct ProjWs { size_t baby, pts, slots, enc, acc, total, tmp, ks, rs, bytes; uint32_t gg; };
+
+constexpr uint32_t MAC_GT = 4, MAC_ST = 2;   // register tile of the multiply-accumulate kernel: giants x shards
 
 ProjWs proj_layout(const ckks_ctx *c, const ProjPlan &p, uint32_t level) {
     const size_t ct = (size_t)2 * level * c->N * sizeof(u64), pt = (size_t)level * c->N * sizeof(u64);
     const size_t nib = p.ins.size();
     ProjWs w;
+    // giant steps are processed in groups of gg: their plaintexts are encoded in one batch and
+    // multiply-accumulated in one launch (about 16 * B plaintexts live at a time)
+    w.gg = std::max<uint32_t>(1, std::min<uint32_t>(p.gmax, 16 / (uint32_t)nib ? 16 / (uint32_t)nib : 1));
+    w.gg = (w.gg + MAC_GT - 1) / MAC_GT * MAC_GT;
+    const size_t npt = (size_t)w.gg * nib * p.B;
     size_t off = 0;
     w.baby = off;  off += align256(ct * p.S * nib * p.B);
-    w.pts = off;   off += align256(pt * nib * p.B);
-    w.slots = off; off += align256((size_t)p.B * c->n * sizeof(double));
-    w.enc = off;   off += align256(encode_workspace_bytes(c, p.B));
-    w.acc = off;   off += align256(ct * p.S);
+    w.pts = off;   off += align256(pt * npt);
+    w.slots = off; off += align256(npt * c->n * sizeof(double));
+    w.enc = off;   off += align256(encode_workspace_bytes(c, (uint32_t)npt));
+    w.acc = off;   off += align256(ct * p.S * w.gg);
     w.total = off; off += align256(ct * p.S);
     w.tmp = off;   off += align256(ct);
     w.ks = off;    off += align256(ks_bytes(c, level));
@@ -99,18 +106,105 @@ const ckks_evk *find_key(const ckks_evk *keys, uint32_t nkeys, u64 g) {
     return nullptr;
 }
 
-// acc[s][c][i][p] = sum_{j < J} ct_j[s][c][i][p] * pt_j[i][p], ct_j[s] at base + (s*sstride + j) * ct_limbs
-__global__ void __launch_bounds__(256) mac_sum_kernel(DevTables c, const u64 *baby, size_t sstride, const u64 *pts, uint32_t J,
-                                                      u64 *acc, uint32_t level) {
-    const uint32_t p = blockIdx.x * 256 + threadIdx.x;
-    const uint32_t i = blockIdx.y % level, comp = blockIdx.y / level, s = blockIdx.z;
-    const size_t ctl = (size_t)2 * level * c.N;
+// Multiply-accumulate of one giant-step group:
+//   acc[g][s][c][i][p] = sum_{j < J} baby[s][j][c][i][p] * pts[g][j][i][p]      (j = input block * B + baby step)
+// A thread owns one coefficient p of one limb i and a register tile of MAC_GT giant steps x MAC_ST shards x 2
+// components; per j it loads MAC_ST*2 ciphertext words and MAC_GT plaintext words for MAC_GT*MAC_ST*2 products.
+//
+// Exact lazy accumulation without carries: every 50-bit word is split at bit 25, x = xh 2^25 + xl, and the
+// three sums  LL = sum xl wl,  HH = sum xh wh,  MM = sum (xl + xh)(wl + wh)  are kept in plain 64-bit
+// registers (each product is below 2^52, so 2^11 terms fit).  The sum of products is then
+// LL + (MM - LL - HH) 2^25 + HH 2^50 < 2^112, reduced once.  Three 32x32->64 multiply-adds per product.
+// Tiles of one coefficient range are adjacent in the grid (blockIdx.x), so re-reads of the same words by other
+// tiles hit L2 rather than HBM.
+struct Split { uint32_t l, h, s; };
+__device__ __forceinline__ Split split25(u64 x) {
+    Split r;
+    r.l = (uint32_t)x & 0x1FFFFFFu;
+    r.h = (uint32_t)(x >> 25);
+    r.s = r.l + r.h;
+    return r;
+}
+
+constexpr uint32_t MAC_THREADS = 128, MAC_DEPTH = 6, MAC_WORDS = MAC_GT + MAC_ST * 2;
+
+__device__ __forceinline__ void cp_async8(void *smem, const void *gmem) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int NLEFT>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(NLEFT) : "memory"); }
+
+// Operands are staged through a MAC_DEPTH-deep ring in shared memory filled by cp.async, so that several j steps
+// of loads are in flight per thread while the products of the current step are formed; a thread only ever reads
+// back the words it requested itself, so no block-wide barrier is needed.
+__global__ void __launch_bounds__(MAC_THREADS) mac_tile_kernel(DevTables c, const u64 *__restrict__ baby, const u64 *__restrict__ pts,
+                                                               u64 *__restrict__ acc, uint32_t J, uint32_t Jstride, uint32_t S,
+                                                               uint32_t G, uint32_t level) {
+    __shared__ u64 ring[MAC_DEPTH][MAC_WORDS][MAC_THREADS];
+    const uint32_t stiles = (S + MAC_ST - 1) / MAC_ST;
+    const uint32_t s0 = (blockIdx.x % stiles) * MAC_ST, g0 = (blockIdx.x / stiles) * MAC_GT;
+    const uint32_t tid = threadIdx.x, p = blockIdx.y * MAC_THREADS + tid, i = blockIdx.z;
+    const size_t lN = (size_t)level * c.N, ctl = 2 * lN;
     const u64 q = c.mod[i], mu = c.mu[i];
-    const u64 *ct = baby + (size_t)s * sstride * ctl + ((size_t)comp * level + i) * c.N + p;
-    const u64 *pt = pts + (size_t)i * c.N + p;
-    u64 hi = 0, lo = 0;
-    for (uint32_t j = 0; j < J; j++) mac128(hi, lo, ct[(size_t)j * ctl], pt[(size_t)j * level * c.N]);
-    acc[(size_t)s * ctl + ((size_t)comp * level + i) * c.N + p] = barrett112(hi, lo, q, mu);
+    const size_t off = (size_t)i * c.N + p;
+    constexpr uint32_t NX = MAC_ST * 2;
+    u64 LL[MAC_GT][NX], HH[MAC_GT][NX], MM[MAC_GT][NX];
+#pragma unroll
+    for (uint32_t g = 0; g < MAC_GT; g++)
+#pragma unroll
+        for (uint32_t x = 0; x < NX; x++) LL[g][x] = HH[g][x] = MM[g][x] = 0;
+    const u64 *wp[MAC_GT], *xp[NX];
+    bool wok[MAC_GT], xok[NX];
+#pragma unroll
+    for (uint32_t g = 0; g < MAC_GT; g++) {
+        wok[g] = g0 + g < G;                      // out-of-range tiles read tile 0 and are never stored
+        wp[g] = pts + (size_t)(wok[g] ? g0 + g : 0) * Jstride * lN + off;
+    }
+#pragma unroll
+    for (uint32_t x = 0; x < NX; x++) {
+        xok[x] = s0 + x / 2 < S;
+        xp[x] = baby + (size_t)(xok[x] ? s0 + x / 2 : 0) * Jstride * ctl + (x & 1) * lN + off;
+    }
+    auto issue = [&](uint32_t j) {
+        if (j < J) {
+            const uint32_t st = j % MAC_DEPTH;
+#pragma unroll
+            for (uint32_t g = 0; g < MAC_GT; g++) cp_async8(&ring[st][g][tid], wp[g] + (size_t)j * lN);
+#pragma unroll
+            for (uint32_t x = 0; x < NX; x++) cp_async8(&ring[st][MAC_GT + x][tid], xp[x] + (size_t)j * ctl);
+        }
+        cp_async_commit();
+    };
+#pragma unroll
+    for (uint32_t j = 0; j < MAC_DEPTH - 1; j++) issue(j);
+    for (uint32_t j = 0; j < J; j++) {
+        cp_async_wait<MAC_DEPTH - 2>();           // step j has landed
+        const uint32_t st = j % MAC_DEPTH;
+        Split w[MAC_GT], x[NX];
+#pragma unroll
+        for (uint32_t g = 0; g < MAC_GT; g++) w[g] = split25(ring[st][g][tid]);
+#pragma unroll
+        for (uint32_t k = 0; k < NX; k++) x[k] = split25(ring[st][MAC_GT + k][tid]);
+        issue(j + MAC_DEPTH - 1);                 // refills the slot read in the previous step
+#pragma unroll
+        for (uint32_t g = 0; g < MAC_GT; g++)
+#pragma unroll
+            for (uint32_t k = 0; k < NX; k++) {
+                LL[g][k] += (u64)x[k].l * w[g].l;
+                HH[g][k] += (u64)x[k].h * w[g].h;
+                MM[g][k] += (u64)x[k].s * w[g].s;
+            }
+    }
+#pragma unroll
+    for (uint32_t g = 0; g < MAC_GT; g++)
+#pragma unroll
+        for (uint32_t k = 0; k < NX; k++)
+            if (wok[g] && xok[k]) {
+                const u64 mid = MM[g][k] - LL[g][k] - HH[g][k];
+                const u128 t = (u128)LL[g][k] + ((u128)mid << 25) + ((u128)HH[g][k] << 50);
+                acc[((size_t)(g0 + g) * S + s0 + k / 2) * ctl + (k & 1) * lN + off] = barrett112((u64)(t >> 64), (u64)t, q, mu);
+            }
 }
 
 }  // namespace
@@ -352,23 +446,43 @@ extern "C" int32_t ckks_linear_proj(ckks_ctx *c, const ckks_proj_desc *d, const 
             gcount = std::max(gcount, std::min(i.size, o.size) / B);
             if (i.size > o.size) fold = i.size / o.size;
         }
-        for (uint32_t gi = 0; gi < gcount; gi++) {
-            // contributing input blocks form a prefix (a smaller trailing block drops out first)
-            uint32_t nact = 0;
-            for (uint32_t ib = 0; ib < nib; ib++)
-                if (gi < std::min(p.ins[ib].size, o.size) / B) nact = ib + 1;
-            for (uint32_t ib = 0; ib < nact; ib++) {
-                const Block &i = p.ins[ib];
-                launch_extract_diagonals(c, W, d->d_out, i.start, i.size, o.start, o.size, p.F, T, gi * B, B, gi * B, slots, s);
-                launch_encode(c, slots, nullptr, B, pt_scale, level, pts + (size_t)ib * B * ptl, encw, s);
+        for (uint32_t g0 = 0; g0 < gcount; g0 += L.gg) {
+            const uint32_t ng = std::min(L.gg, gcount - g0);
+            const uint32_t J = nib * B;
+            // plaintexts of the group: pts[(gl * nib + ib) * B + b]; a block pair that has run out of diagonals
+            // contributes zero plaintexts
+            bool ragged = false;
+            for (uint32_t gl = 0; gl < ng; gl++)
+                for (uint32_t ib = 0; ib < nib; ib++)
+                    if (g0 + gl >= std::min(p.ins[ib].size, o.size) / B) ragged = true;
+            if (ragged) cudaMemsetAsync(pts, 0, (size_t)ng * J * ptl * sizeof(u64), s);
+            for (uint32_t gl = 0; gl < ng; gl++)
+                for (uint32_t ib = 0; ib < nib; ib++) {
+                    const Block &i = p.ins[ib];
+                    const uint32_t gi = g0 + gl;
+                    if (gi >= std::min(i.size, o.size) / B) continue;
+                    const size_t idx = ((size_t)gl * nib + ib) * B;
+                    launch_extract_diagonals(c, W, d->d_out, i.start, i.size, o.start, o.size, p.F, T, gi * B, B, gi * B,
+                                             slots + idx * c->n, s);
+                    if (ragged) launch_encode(c, slots + idx * c->n, nullptr, B, pt_scale, level, pts + idx * ptl, encw, s);
+                }
+            if (!ragged) launch_encode(c, slots, nullptr, ng * J, pt_scale, level, pts, encw, s);
+            {
+                const uint32_t stiles = (S + MAC_ST - 1) / MAC_ST, gtiles = (ng + MAC_GT - 1) / MAC_GT;
+                mac_tile_kernel<<<dim3(stiles * gtiles, N / MAC_THREADS, level), MAC_THREADS, 0, s>>>(c->dev, baby, pts, acc, J, J, S, ng, level);
+                count_launches();
             }
-            u64 *dst = gi == 0 ? total : acc;
-            mac_sum_kernel<<<dim3(N / 256, 2 * level, S), 256, 0, s>>>(c->dev, baby, (size_t)nib * B, pts, nact * B, dst, level); count_launches();
-            if (gi) {
+            for (uint32_t gl = 0; gl < ng; gl++) {
+                const uint32_t gi = g0 + gl;
+                u64 *ag = acc + (size_t)gl * S * ctl;
+                if (gi == 0) {
+                    cudaMemcpyAsync(total, ag, (size_t)S * ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+                    continue;
+                }
                 const u64 ge = ckks_galois_element(c, (int64_t)gi * B * T);
                 const u64 *key = (const u64 *)find_key(keys, nkeys, ge)->data;
                 for (uint32_t sh = 0; sh < S; sh++) {
-                    u64 *a = acc + (size_t)sh * ctl, *t = total + (size_t)sh * ctl;
+                    u64 *a = ag + (size_t)sh * ctl, *t = total + (size_t)sh * ctl;
                     ks_modup(c, a + ptl, ge, level, kw, s);
                     ks_inner_moddown(c, key, level, 1, kw, a, nullptr, ge, tmp, s);
                     launch_add(c, t, tmp, t, 2, level, s);

@@ -29,29 +29,52 @@ __global__ void __launch_bounds__(THREADS) permute_kernel(DevTables c, const u64
     dst[row + p] = src[row + galois_src(p, g, c.log_n, c.N)];
 }
 
+constexpr uint32_t CHUNK = 8;   // targets per CTA row in the basis-conversion kernels
+
 // ext[j][x][k] for x over q_0..q_{level-1}, p_0..p_{K-1}.  dcoef: sigma_g(d) in the coefficient domain;
 // deval: d in the evaluation domain, read through sigma_g for the digit's own limbs.
+// A thread owns one coefficient of one digit: it forms the centred y_a of the digit's limbs once and then
+// walks a chunk of CHUNK target limbs (blockIdx.y), so the source limbs are read once per chunk.
+template <uint32_t ALPHA>
 __global__ void __launch_bounds__(THREADS) modup_kernel(DevTables c, const u64 *dcoef, const u64 *deval, u64 g,
                                                         u64 *ext, uint32_t level) {
     const uint32_t k = blockIdx.x * THREADS + threadIdx.x;
-    const uint32_t x = blockIdx.y, j = blockIdx.z;
-    const uint32_t nt = level + c.K, lo = j * c.alpha, hi = min(lo + c.alpha, level);
-    u64 *dst = ext + ((size_t)j * nt + x) * c.N + k;
-    if (x >= lo && x < hi) {
-        *dst = deval[(size_t)x * c.N + galois_src(k, g, c.log_n, c.N)];
-        return;
-    }
-    const uint32_t t = x < level ? x : c.L + (x - level);
-    const u64 mt = c.mod[t];
+    const uint32_t j = blockIdx.z;
+    const uint32_t nt = level + c.K, lo = j * c.alpha, hi = min(lo + c.alpha, level), nd = hi - lo;
     const size_t cb = ((size_t)level * c.dnum + j) * c.alpha;
-    u64 ahi = 0, alo = 0;
-    for (uint32_t a = lo; a < hi; a++) {
-        const u64 qa = c.mod[a];
-        const ulonglong2 hinv = c.up_hat_inv[cb + (a - lo)];
-        const u64 y = mul_shoup(dcoef[(size_t)a * c.N + k], hinv.x, hinv.y, qa);
-        mac128(ahi, alo, centred_to(y, qa, mt), c.up_hat_mod[(cb + (a - lo)) * c.T + t]);
+    u64 y[ALPHA], qa[ALPHA];
+#pragma unroll
+    for (uint32_t a = 0; a < ALPHA; a++) {
+        if (a < nd) {
+            qa[a] = c.mod[lo + a];
+            const ulonglong2 hinv = c.up_hat_inv[cb + a];
+            y[a] = mul_shoup(dcoef[(size_t)(lo + a) * c.N + k], hinv.x, hinv.y, qa[a]);
+        } else {
+            qa[a] = 1; y[a] = 0;
+        }
     }
-    *dst = barrett112(ahi, alo, mt, c.mu[t]);
+    const uint32_t x0 = blockIdx.y * CHUNK, x1 = min(x0 + CHUNK, nt);
+    for (uint32_t x = x0; x < x1; x++) {
+        u64 *dst = ext + ((size_t)j * nt + x) * c.N + k;
+        if (x >= lo && x < hi) {
+            *dst = deval[(size_t)x * c.N + galois_src(k, g, c.log_n, c.N)];
+            continue;
+        }
+        const uint32_t t = x < level ? x : c.L + (x - level);
+        const u64 mt = c.mod[t];
+        u64 ahi = 0, alo = 0;
+#pragma unroll
+        for (uint32_t a = 0; a < ALPHA; a++)
+            if (a < nd) mac128(ahi, alo, centred_to(y[a], qa[a], mt), c.up_hat_mod[(cb + a) * c.T + t]);
+        *dst = barrett112(ahi, alo, mt, c.mu[t]);
+    }
+}
+
+template <uint32_t ALPHA>
+void launch_modup(const ckks_ctx *c, const u64 *dcoef, const u64 *deval, u64 g, u64 *ext, uint32_t level, cudaStream_t s) {
+    const uint32_t nt = level + c->K, beta = (level + c->alpha - 1) / c->alpha;
+    modup_kernel<ALPHA><<<dim3(c->N / THREADS, (nt + CHUNK - 1) / CHUNK, beta), THREADS, 0, s>>>(c->dev, dcoef, deval, g, ext, level);
+    count_launches();
 }
 
 // u[comp][x][p] = sum_j ext[j][x][pi_g(p)] * evk[j][comp][kt(x)][p]
@@ -74,20 +97,51 @@ __global__ void __launch_bounds__(THREADS) inner_product_kernel(DevTables c, con
 }
 
 // conv[comp][i][k] = sum_a centre([u_{p_a} Phat_a^-1]) (Phat_a mod q_i)  mod q_i   (coefficient domain)
+// Same shape as ModUp: the K centred special residues are formed once per thread, then a chunk of targets is walked.
+template <uint32_t KK>
 __global__ void __launch_bounds__(THREADS) moddown_conv_kernel(DevTables c, const u64 *u, u64 *conv, uint32_t level) {
     const uint32_t k = blockIdx.x * THREADS + threadIdx.x;
-    const uint32_t i = blockIdx.y, comp = blockIdx.z;
+    const uint32_t comp = blockIdx.z;
     const uint32_t nt = level + c.K;
-    const u64 q = c.mod[i];
-    u64 ahi = 0, alo = 0;
-    for (uint32_t a = 0; a < c.K; a++) {
-        const u64 pa = c.mod[c.L + a];
-        const ulonglong2 hinv = c.dn_hat_inv[a];
-        const u64 y = mul_shoup(u[((size_t)comp * nt + level + a) * c.N + k], hinv.x, hinv.y, pa);
-        mac128(ahi, alo, centred_to(y, pa, q), c.dn_hat_mod[(size_t)i * c.K + a]);
+    u64 y[KK], pa[KK];
+#pragma unroll
+    for (uint32_t a = 0; a < KK; a++) {
+        if (a < c.K) {
+            pa[a] = c.mod[c.L + a];
+            const ulonglong2 hinv = c.dn_hat_inv[a];
+            y[a] = mul_shoup(u[((size_t)comp * nt + level + a) * c.N + k], hinv.x, hinv.y, pa[a]);
+        } else {
+            pa[a] = 1; y[a] = 0;
+        }
     }
-    conv[((size_t)comp * level + i) * c.N + k] = barrett112(ahi, alo, q, c.mu[i]);
+    const uint32_t i0 = blockIdx.y * CHUNK, i1 = min(i0 + CHUNK, level);
+    for (uint32_t i = i0; i < i1; i++) {
+        const u64 q = c.mod[i];
+        u64 ahi = 0, alo = 0;
+#pragma unroll
+        for (uint32_t a = 0; a < KK; a++)
+            if (a < c.K) mac128(ahi, alo, centred_to(y[a], pa[a], q), c.dn_hat_mod[(size_t)i * c.K + a]);
+        conv[((size_t)comp * level + i) * c.N + k] = barrett112(ahi, alo, q, c.mu[i]);
+    }
 }
+
+template <uint32_t KK>
+void launch_moddown_conv(const ckks_ctx *c, const u64 *u, u64 *conv, uint32_t level, cudaStream_t s) {
+    moddown_conv_kernel<KK><<<dim3(c->N / THREADS, (level + CHUNK - 1) / CHUNK, 2), THREADS, 0, s>>>(c->dev, u, conv, level);
+    count_launches();
+}
+
+// register-array size for a digit / special-prime count: next of 1, 2, 4, 8, 16, 32, 64
+#define DISPATCH_POW2(n, CALL)                      \
+    do {                                            \
+        if ((n) <= 1) { CALL(1); }                  \
+        else if ((n) <= 2) { CALL(2); }             \
+        else if ((n) <= 4) { CALL(4); }             \
+        else if ((n) <= 8) { CALL(8); }             \
+        else if ((n) <= 16) { CALL(16); }           \
+        else if ((n) <= 32) { CALL(32); }           \
+        else { CALL(64); }                          \
+    } while (0)
 
 // out[comp][i][p] = (u[comp][i][p] - conv[comp][i][p]) P^-1 + add_comp[i][pi_g(p)]
 __global__ void __launch_bounds__(THREADS) moddown_final_kernel(DevTables c, const u64 *u, const u64 *conv, const u64 *add0,
@@ -144,7 +198,9 @@ void ks_modup(const ckks_ctx *c, const u64 *d, u64 galois, uint32_t level, const
     const uint32_t N = c->N, beta = (level + c->alpha - 1) / c->alpha, nt = level + c->K;
     permute_kernel<<<dim3(N / THREADS, level), THREADS, 0, s>>>(c->dev, d, w.dcoef, galois); count_launches();
     launch_ntt(c, w.dcoef, level, plain_map(0, level), true, s);
-    modup_kernel<<<dim3(N / THREADS, nt, beta), THREADS, 0, s>>>(c->dev, w.dcoef, d, galois, w.ext, level); count_launches();
+#define CALL_UP(A) launch_modup<A>(c, w.dcoef, d, galois, w.ext, level, s)
+    DISPATCH_POW2(c->alpha, CALL_UP);
+#undef CALL_UP
     LimbMap em{1, 0, nt, level, c->L, c->alpha, 1};
     launch_ntt(c, w.ext, beta * nt, em, false, s);
 }
@@ -155,7 +211,9 @@ void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext
     inner_product_kernel<<<dim3(N / THREADS, nt), THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level); count_launches();
     for (uint32_t comp = 0; comp < 2; comp++)
         launch_ntt(c, w.u + ((size_t)comp * nt + level) * N, K, plain_map(c->L, K), true, s);
-    moddown_conv_kernel<<<dim3(N / THREADS, level, 2), THREADS, 0, s>>>(c->dev, w.u, w.conv, level); count_launches();
+#define CALL_DN(A) launch_moddown_conv<A>(c, w.u, w.conv, level, s)
+    DISPATCH_POW2(K, CALL_DN);
+#undef CALL_DN
     launch_ntt(c, w.conv, 2 * level, plain_map(0, level), false, s);
     moddown_final_kernel<<<dim3(N / THREADS, level, 2), THREADS, 0, s>>>(c->dev, w.u, w.conv, add0, add1, add_galois, out, level); count_launches();
 }
