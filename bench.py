@@ -148,6 +148,7 @@ def run_cuda(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
+    SH = args.shards if args.profile else SHARDS
     q, p = inputs.prime_chain(LOG_N, L, K)
     allp = [int(x) for x in q] + [int(x) for x in p]
     ctx = binding.Context(LOG_N, q, p, DNUM, device=local)
@@ -163,7 +164,7 @@ def run_cuda(args):
     # (a) NTT inputs
     polys = residues(allp[:L], NTT_BATCH)
     # keys: the projection's rotation set contains the 64 rotations 8b, b = 1..64, of part (b)
-    rots = ctx.linear_proj_rotations(HIDDEN, HIDDEN, T_SHARD, SHARDS, BABY)
+    rots = ctx.linear_proj_rotations(HIDDEN, HIDDEN, T_SHARD, SH, BABY)
     keys = {r: binding.SwitchKey(residues(allp, DNUM, 2), ctx.galois_element(r)) for r in rots}
     rlk = binding.SwitchKey(residues(allp, DNUM, 2), 0)
     rot_keys = [keys[8 * b] for b in range(1, NROT + 1)]
@@ -175,14 +176,14 @@ def run_cuda(args):
     hoist_out = [ctx.empty_ct(LEVEL) for _ in range(NROT)]
     mul_out = ctx.empty_ct(LEVEL)
     # (c) projection inputs
-    cts = [binding.Ciphertext(residues(allp[:L], 2), 2.0 ** 40) for _ in range(SHARDS)]
+    cts = [binding.Ciphertext(residues(allp[:L], 2), 2.0 ** 40) for _ in range(SH)]
     W = (torch.randn((HIDDEN, HIDDEN), generator=gen, device=dev, dtype=torch.float64) * 0.02).contiguous()
-    outs = [ctx.empty_ct(LEVEL - 1) for _ in range(SHARDS)]
-    ws = torch.empty(ctx.linear_proj_workspace_bytes(HIDDEN, HIDDEN, T_SHARD, SHARDS, BABY, LEVEL), dtype=torch.uint8, device=dev)
+    outs = [ctx.empty_ct(LEVEL - 1) for _ in range(SH)]
+    ws = torch.empty(ctx.linear_proj_workspace_bytes(HIDDEN, HIDDEN, T_SHARD, SH, BABY, LEVEL), dtype=torch.uint8, device=dev)
     # e2e host buffers (pinned)
     h_cts = [c.data.cpu().pin_memory() for c in cts]
     h_W = W.cpu().pin_memory()
-    h_outs = [torch.empty((2, LEVEL - 1, N), dtype=torch.uint64).pin_memory() for _ in range(SHARDS)]
+    h_outs = [torch.empty((2, LEVEL - 1, N), dtype=torch.uint64).pin_memory() for _ in range(SH)]
 
     def ev():
         return torch.cuda.Event(enable_timing=True)
@@ -198,10 +199,15 @@ def run_cuda(args):
         ctx.mul_relin(cta, ctb, rlk, out=mul_out)
 
     def part_c():
-        ctx.linear_proj(cts, W, proj_keys, HIDDEN, HIDDEN, T_SHARD, SHARDS, BABY, outs=outs, ws=ws)
+        ctx.linear_proj(cts, W, proj_keys, HIDDEN, HIDDEN, T_SHARD, SH, BABY, outs=outs, ws=ws)
 
     def step(times=None):
         e = [ev() for _ in range(4)]
+        if args.profile:
+            for name, f in (("a", part_a), ("b", part_b), ("c", part_c)):
+                if name in args.parts:
+                    f()
+            return
         e[0].record(); part_a(); e[1].record(); part_b(); e[2].record(); part_c(); e[3].record()
         if times is not None:
             times.append(e)
@@ -311,6 +317,8 @@ def main():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--parts", default="abc", help="with --profile: which parts of the step to run (a: NTT, b: key switching, c: projection)")
+    ap.add_argument("--shards", type=int, default=SHARDS, help="with --profile: token shards in the projection (default 16)")
     ap.add_argument("--profile", action="store_true",
                     help="for profiler captures: honour --warmup below 3 and skip the e2e and CPU legs (prints no bench line)")
     args = ap.parse_args()

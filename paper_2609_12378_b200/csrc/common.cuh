@@ -22,15 +22,21 @@ struct DevTables {
     const u64 *mod;          // [T]
     const u64 *mu;           // [T] floor(2^112 / prime)
     const u64 *mu64;         // [T] floor(2^64 / prime)
+    const double2 *modd;     // [T] {prime, 1/prime} as doubles
     const ulonglong2 *tw_fwd;  // [T][N] {psi^bitrev(i), Shoup companion}, index m+i
     const ulonglong2 *tw_inv;  // [T][N] inverses of the same
     const ulonglong2 *n_inv;   // [T] {N^-1, Shoup}
+    // fp64 copies for the double-precision NTT path (N = 2^16 only): {w, w/q} as doubles, same indexing
+    const double2 *twd_fwd, *twd_inv;   // [T][N]
+    const double2 *n_inv_d;             // [T] {N^-1, N^-1/q}
     // ModUp, per level l (1..L), digit j, source a < alpha:
     const ulonglong2 *up_hat_inv;  // [(L+1)][dnum][alpha]        {qhat^-1 mod q_src, Shoup}
     const u64 *up_hat_mod;         // [(L+1)][dnum][alpha][T]     qhat mod target
+    const double2 *up_hat_mod_d;   // same shape, {c, c / target prime} as doubles
     // ModDown:
     const ulonglong2 *dn_hat_inv;  // [K]      {Phat_k^-1 mod p_k, Shoup}
     const u64 *dn_hat_mod;         // [L][K]   Phat_k mod q_i
+    const double2 *dn_hat_mod_d;   // [L][K]   {c, c / q_i} as doubles
     const ulonglong2 *dn_p_inv;    // [L]      {P^-1 mod q_i, Shoup}
     // Rescale: [L(last)][L(i)] {q_last^-1 mod q_i, Shoup}
     const ulonglong2 *rs_inv;
@@ -49,6 +55,7 @@ struct ckks_ctx {
     DevTables dev;               // pointers into `allocs`
     std::vector<void *> allocs;  // device allocations owned by the context
     std::string cuda_error;
+    uint32_t ntt_fp_share = 8;   // of every 8 limbs, how many take the double-precision NTT path (tuning knob)
 };
 
 // ---------------------------------------------------------------------------
@@ -110,6 +117,32 @@ __device__ __forceinline__ void mac128(u64 &hi, u64 &lo, u64 a, u64 b) {
 __device__ __forceinline__ u64 centred_to(u64 y, u64 src, u64 dst) {
     return y > (src >> 1) ? y + dst - src : y;
 }
+
+// ---------------------------------------------------------------------------
+// Double-precision modular arithmetic for 50-bit primes (FP64 pipe).  Values are
+// signed integers held in doubles, exact while below 2^53 in magnitude.
+//   mulmod_d: y * w - k q with k = round(y * (w/q)); exact; |result| <= (1/2 + |y| 2^-53) q
+//             (COARSE: k rounded to even, valid for |y w / q| < 2^52, |result| <= (1 + ..) q).
+// ---------------------------------------------------------------------------
+constexpr double MAGIC0 = 6755399441055744.0;    // 1.5 * 2^52: rounds |v| < 2^51 to the nearest integer
+constexpr double MAGIC1 = 13510798882111488.0;   // 1.5 * 2^53: rounds |v| < 2^52 to the nearest even integer
+constexpr double TWO52 = 4503599627370496.0;
+
+template <int COARSE>
+__device__ __forceinline__ double mulmod_d(double y, double2 w, double q) {
+    const double p = __dmul_rn(y, w.x);
+    const double e = __fma_rn(y, w.x, -p);
+    const double M = COARSE ? MAGIC1 : MAGIC0;
+    const double k = __dsub_rn(__fma_rn(y, w.y, M), M);
+    return __dadd_rn(__fma_rn(-k, q, p), e);
+}
+__device__ __forceinline__ double reduce_d(double v, double q, double qinv) {   // to |v| <= q/2
+    const double k = __dsub_rn(__fma_rn(v, qinv, MAGIC0), MAGIC0);
+    return __fma_rn(-k, q, v);
+}
+__device__ __forceinline__ double u64_to_d(u64 x) { return __dsub_rn(__longlong_as_double((long long)(x | 0x4330000000000000ull)), TWO52); }
+__device__ __forceinline__ u64 d_to_u64(double v) { return (u64)__double_as_longlong(__dadd_rn(v, TWO52)) & 0x000FFFFFFFFFFFFFull; }
+__device__ __forceinline__ u64 canonical_d(double v, double q) { return d_to_u64(v < 0.0 ? __dadd_rn(v, q) : v); }
 
 __device__ __forceinline__ uint32_t bitrev_n(uint32_t x, uint32_t bits) { return __brev(x) >> (32 - bits); }
 

@@ -1,5 +1,6 @@
 // Context: parameter validation, host-side table construction, upload.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -143,6 +144,7 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
     ckks_ctx *c = new ckks_ctx();
     c->log_n = prm->log_n; c->N = N; c->n = n; c->L = L; c->K = K; c->dnum = prm->dnum; c->alpha = alpha; c->T = T;
     c->device = prm->device;
+    if (const char *e = getenv("CKKS_NTT_FP_SHARE")) c->ntt_fp_share = (uint32_t)atoi(e);
     c->mod = mod;
     c->pow5.resize(n);
     c->pow5[0] = 1;
@@ -154,12 +156,17 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
 
     // ---- per-prime scalars and twiddles
     std::vector<u64> mu(T), mu64(T);
+    std::vector<double2> modd(T);
     std::vector<ulonglong2> ninv(T), twf((size_t)T * N), twi((size_t)T * N);
+    const bool fp = prm->log_n == 16;
+    std::vector<double2> twdf(fp ? (size_t)T * N : 0), twdi(fp ? (size_t)T * N : 0), ninvd(T);
     for (uint32_t t = 0; t < T; t++) {
         u64 m = mod[t];
         mu[t] = (u64)((((u128)1) << 112) / m);
         mu64[t] = (u64)((((u128)1) << 64) / m);
+        modd[t] = make_double2((double)m, 1.0 / (double)m);
         ninv[t] = h_pair(h_inv(N % m, m), m);
+        ninvd[t] = make_double2((double)ninv[t].x, (double)ninv[t].x / (double)m);
         u64 psi = h_min_root(m, N), psi_inv = h_inv(psi, m);
         std::vector<u64> pw(N), pwi(N);
         pw[0] = pwi[0] = 1;
@@ -168,6 +175,10 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
             uint32_t r = h_bitrev(i, prm->log_n);
             twf[(size_t)t * N + i] = h_pair(pw[r], m);
             twi[(size_t)t * N + i] = h_pair(pwi[r], m);
+            if (fp) {
+                twdf[(size_t)t * N + i] = make_double2((double)pw[r], (double)pw[r] / (double)m);
+                twdi[(size_t)t * N + i] = make_double2((double)pwi[r], (double)pwi[r] / (double)m);
+            }
         }
     }
 
@@ -175,6 +186,7 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
     const uint32_t dn = prm->dnum;
     std::vector<ulonglong2> up_inv((size_t)(L + 1) * dn * alpha, make_ulonglong2(0, 0));
     std::vector<u64> up_mod((size_t)(L + 1) * dn * alpha * T, 0);
+    std::vector<double2> up_mod_d(up_mod.size(), make_double2(0.0, 0.0));
     for (uint32_t lvl = 1; lvl <= L; lvl++)
         for (uint32_t j = 0; j * alpha < lvl; j++) {
             uint32_t lo = j * alpha, hi = std::min(lo + alpha, lvl);
@@ -189,6 +201,7 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
                     for (uint32_t b = lo; b < hi; b++)
                         if (b != a) v = h_mul(v, mod[b] % mt, mt);
                     up_mod[base * T + t] = v;
+                    up_mod_d[base * T + t] = make_double2((double)v, (double)v / (double)mt);
                 }
             }
         }
@@ -196,6 +209,7 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
     // ---- ModDown constants
     std::vector<ulonglong2> dn_inv(K), dn_pinv(L);
     std::vector<u64> dn_mod((size_t)L * K);
+    std::vector<double2> dn_mod_d((size_t)L * K);
     for (uint32_t a = 0; a < K; a++) {
         u64 pa = mod[L + a], h = 1;
         for (uint32_t b = 0; b < K; b++)
@@ -209,6 +223,7 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
             for (uint32_t b = 0; b < K; b++)
                 if (b != a) v = h_mul(v, mod[L + b] % q, q);
             dn_mod[(size_t)i * K + a] = v;
+            dn_mod_d[(size_t)i * K + a] = make_double2((double)v, (double)v / (double)q);
             Pm = h_mul(Pm, mod[L + a] % q, q);
         }
         dn_pinv[i] = h_pair(h_inv(Pm, q), q);
@@ -237,9 +252,9 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
     int rc = CKKS_OK;
     std::vector<int> flag(1, 0);
     const int *flag_dev = nullptr;
-    if ((rc = upload(c, mod, &d.mod)) || (rc = upload(c, mu, &d.mu)) || (rc = upload(c, mu64, &d.mu64)) || (rc = upload(c, twf, &d.tw_fwd)) ||
-        (rc = upload(c, twi, &d.tw_inv)) || (rc = upload(c, ninv, &d.n_inv)) || (rc = upload(c, up_inv, &d.up_hat_inv)) ||
-        (rc = upload(c, up_mod, &d.up_hat_mod)) || (rc = upload(c, dn_inv, &d.dn_hat_inv)) ||
+    if ((rc = upload(c, mod, &d.mod)) || (rc = upload(c, mu, &d.mu)) || (rc = upload(c, mu64, &d.mu64)) || (rc = upload(c, modd, &d.modd)) || (rc = upload(c, twf, &d.tw_fwd)) ||
+        (rc = upload(c, twi, &d.tw_inv)) || (rc = upload(c, twdf, &d.twd_fwd)) || (rc = upload(c, twdi, &d.twd_inv)) || (rc = upload(c, ninvd, &d.n_inv_d)) || (rc = upload(c, ninv, &d.n_inv)) || (rc = upload(c, up_inv, &d.up_hat_inv)) ||
+        (rc = upload(c, up_mod, &d.up_hat_mod)) || (rc = upload(c, up_mod_d, &d.up_hat_mod_d)) || (rc = upload(c, dn_mod_d, &d.dn_hat_mod_d)) || (rc = upload(c, dn_inv, &d.dn_hat_inv)) ||
         (rc = upload(c, dn_mod, &d.dn_hat_mod)) || (rc = upload(c, dn_pinv, &d.dn_p_inv)) || (rc = upload(c, rs, &d.rs_inv)) ||
         (rc = upload(c, enc_src, &d.enc_src)) || (rc = upload(c, om, &d.enc_omega)) || (rc = upload(c, ze, &d.enc_zeta)) ||
         (rc = upload(c, flag, &flag_dev))) {

@@ -42,15 +42,16 @@ __global__ void __launch_bounds__(THREADS) modup_kernel(DevTables c, const u64 *
     const uint32_t j = blockIdx.z;
     const uint32_t nt = level + c.K, lo = j * c.alpha, hi = min(lo + c.alpha, level), nd = hi - lo;
     const size_t cb = ((size_t)level * c.dnum + j) * c.alpha;
-    u64 y[ALPHA], qa[ALPHA];
+    // centred y_a = [d_a qhat_a^-1] as signed doubles (integer Shoup product, then the lift)
+    double y[ALPHA];
 #pragma unroll
     for (uint32_t a = 0; a < ALPHA; a++) {
+        y[a] = 0.0;
         if (a < nd) {
-            qa[a] = c.mod[lo + a];
+            const u64 qa = c.mod[lo + a];
             const ulonglong2 hinv = c.up_hat_inv[cb + a];
-            y[a] = mul_shoup(dcoef[(size_t)(lo + a) * c.N + k], hinv.x, hinv.y, qa[a]);
-        } else {
-            qa[a] = 1; y[a] = 0;
+            const u64 v = mul_shoup(dcoef[(size_t)(lo + a) * c.N + k], hinv.x, hinv.y, qa);
+            y[a] = v > (qa >> 1) ? __dsub_rn(u64_to_d(v), (double)qa) : u64_to_d(v);
         }
     }
     const uint32_t x0 = blockIdx.y * CHUNK, x1 = min(x0 + CHUNK, nt);
@@ -61,12 +62,16 @@ __global__ void __launch_bounds__(THREADS) modup_kernel(DevTables c, const u64 *
             continue;
         }
         const uint32_t t = x < level ? x : c.L + (x - level);
-        const u64 mt = c.mod[t];
-        u64 ahi = 0, alo = 0;
+        const double2 md = c.modd[t];
+        const double mt = md.x, mtinv = md.y;
+        // each product is reduced to |r| <= 0.57 m_t on the FP64 pipe; eight of them stay far below 2^53
+        double acc = 0.0;
 #pragma unroll
-        for (uint32_t a = 0; a < ALPHA; a++)
-            if (a < nd) mac128(ahi, alo, centred_to(y[a], qa[a], mt), c.up_hat_mod[(cb + a) * c.T + t]);
-        *dst = barrett112(ahi, alo, mt, c.mu[t]);
+        for (uint32_t a = 0; a < ALPHA; a++) {
+            if (a < nd) acc = __dadd_rn(acc, mulmod_d<0>(y[a], c.up_hat_mod_d[(cb + a) * c.T + t], mt));
+            if ((a & 7) == 7 && a + 1 < ALPHA) acc = reduce_d(acc, mt, mtinv);
+        }
+        *dst = canonical_d(reduce_d(acc, mt, mtinv), mt);
     }
 }
 
@@ -103,25 +108,28 @@ __global__ void __launch_bounds__(THREADS) moddown_conv_kernel(DevTables c, cons
     const uint32_t k = blockIdx.x * THREADS + threadIdx.x;
     const uint32_t comp = blockIdx.z;
     const uint32_t nt = level + c.K;
-    u64 y[KK], pa[KK];
+    double y[KK];
 #pragma unroll
     for (uint32_t a = 0; a < KK; a++) {
+        y[a] = 0.0;
         if (a < c.K) {
-            pa[a] = c.mod[c.L + a];
+            const u64 pa = c.mod[c.L + a];
             const ulonglong2 hinv = c.dn_hat_inv[a];
-            y[a] = mul_shoup(u[((size_t)comp * nt + level + a) * c.N + k], hinv.x, hinv.y, pa[a]);
-        } else {
-            pa[a] = 1; y[a] = 0;
+            const u64 v = mul_shoup(u[((size_t)comp * nt + level + a) * c.N + k], hinv.x, hinv.y, pa);
+            y[a] = v > (pa >> 1) ? __dsub_rn(u64_to_d(v), (double)pa) : u64_to_d(v);
         }
     }
     const uint32_t i0 = blockIdx.y * CHUNK, i1 = min(i0 + CHUNK, level);
     for (uint32_t i = i0; i < i1; i++) {
-        const u64 q = c.mod[i];
-        u64 ahi = 0, alo = 0;
+        const double2 md = c.modd[i];
+        const double q = md.x, qinv = md.y;
+        double acc = 0.0;
 #pragma unroll
-        for (uint32_t a = 0; a < KK; a++)
-            if (a < c.K) mac128(ahi, alo, centred_to(y[a], pa[a], q), c.dn_hat_mod[(size_t)i * c.K + a]);
-        conv[((size_t)comp * level + i) * c.N + k] = barrett112(ahi, alo, q, c.mu[i]);
+        for (uint32_t a = 0; a < KK; a++) {
+            if (a < c.K) acc = __dadd_rn(acc, mulmod_d<0>(y[a], c.dn_hat_mod_d[(size_t)i * c.K + a], q));
+            if ((a & 7) == 7 && a + 1 < KK) acc = reduce_d(acc, q, qinv);
+        }
+        conv[((size_t)comp * level + i) * c.N + k] = canonical_d(reduce_d(acc, q, qinv), q);
     }
 }
 

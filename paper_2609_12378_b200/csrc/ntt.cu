@@ -176,11 +176,90 @@ __device__ __forceinline__ u64 reduce_exact(u64 x, u64 q, u64 qinv64) {
     return r >= q ? r - q : r;
 }
 
+// ---------------------------------------------------------------------------
+// Double-precision variant of the same butterflies.  The FP64 pipe multiplies
+// 53-bit operands in one instruction where the integer pipe needs several
+// 32x32 products, so for 50-bit primes a twiddle product is cheaper there:
+//   p = y w (rounded), e = fma(y, w, -p) (exact low part),
+//   k = round(y * (w/q))  by adding and subtracting 1.5 * 2^52 (or 1.5 * 2^53),
+//   r = fma(-k, q, p) + e  =  y w - k q   exactly, |r| <= (1/2 + eps) q  (or (1 + eps) q).
+// Values are signed integers held in doubles; everything is exact while they stay
+// below 2^53 in magnitude, so each group of four stages starts by reducing its 16
+// values to |v| <= q/2 (forward), and the inverse reduces again after two stages.
+// A limb is handled by the integer or by the double path in BOTH passes (the
+// intermediate written between the passes is a lazy word in one case and a double
+// in the other); the result is the same canonical residue either way.
+// ---------------------------------------------------------------------------
+// 4 Cooley-Tukey stages; inputs of any magnitude below 2^53 (reduced first), outputs below 4.6 q.
+__device__ __forceinline__ void fwd16_d(double (&x)[16], const double2 *__restrict__ tw, uint32_t base, double q, double qinv) {
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) x[k] = reduce_d(x[k], q, qinv);
+#pragma unroll
+    for (uint32_t ml = 1; ml < 16; ml <<= 1) {
+        const uint32_t tl = 8 / ml;
+#pragma unroll
+        for (uint32_t i = 0; i < ml; i++) {
+            const double2 w = __ldg(&tw[ml * base + i]);
+#pragma unroll
+            for (uint32_t j = 0; j < tl; j++) {
+                const uint32_t k1 = 2 * i * tl + j, k2 = k1 + tl;
+                // bounds entering the stages: 0.5, 1.13, 1.9, 2.9 (times q): only the last needs the coarse rounding
+                const double t = ml == 8 ? mulmod_d<1>(x[k2], w, q) : mulmod_d<0>(x[k2], w, q);
+                x[k2] = __dsub_rn(x[k1], t);
+                x[k1] = __dadd_rn(x[k1], t);
+            }
+        }
+    }
+}
+
+// 4 Gentleman-Sande stages; reduced at the start and after two stages; outputs below 2 q.
+__device__ __forceinline__ void inv16_d(double (&x)[16], const double2 *__restrict__ tw, uint32_t base, double q, double qinv) {
+#pragma unroll
+    for (uint32_t ml = 8; ml >= 1; ml >>= 1) {
+        const uint32_t tl = 8 / ml;
+        if (ml == 8 || ml == 2) {
+#pragma unroll
+            for (uint32_t k = 0; k < 16; k++) x[k] = reduce_d(x[k], q, qinv);
+        }
+#pragma unroll
+        for (uint32_t i = 0; i < ml; i++) {
+            const double2 w = __ldg(&tw[ml * base + i]);
+#pragma unroll
+            for (uint32_t j = 0; j < tl; j++) {
+                const uint32_t k1 = 2 * i * tl + j, k2 = k1 + tl;
+                const double u = x[k1], v = x[k2];
+                x[k1] = __dadd_rn(u, v);
+                x[k2] = mulmod_d<0>(__dsub_rn(u, v), w, q);     // |u - v| <= 2q < 2^51
+            }
+        }
+    }
+}
+
 // ---- forward, column pass (stages m = 1..128): CTA = strip of 16 columns -----------------
-__global__ void __launch_bounds__(F_THREADS) ntt16_fwd_cols(DevTables c, u64 *base, LimbMap map) {
+__global__ void __launch_bounds__(F_THREADS) ntt16_fwd_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
     __shared__ u64 sm[256 * 16];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
+    if ((blockIdx.y & 7) < fp_share) {
+        const double q = c.modd[prime].x, qinv = c.modd[prime].y;
+        const double2 *tw = c.twd_fwd + ((size_t)prime << 16);
+        const uint32_t cc = threadIdx.x & 15, r = threadIdx.x >> 4;
+        u64 *g = base + ((size_t)blockIdx.y << 16) + blockIdx.x * 16 + cc;
+        double *smd = reinterpret_cast<double *>(sm);
+        double x[16];
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) x[k] = u64_to_d(g[(size_t)(r + 16 * k) * 256]);
+        fwd16_d(x, tw, 1, q, qinv);
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) smd[(r + 16 * k) * 16 + cc] = x[k];
+        __syncthreads();
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) x[k] = smd[(16 * r + k) * 16 + cc];
+        fwd16_d(x, tw, 16 + r, q, qinv);
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) reinterpret_cast<double *>(g)[(size_t)(16 * r + k) * 256] = x[k];
+        return;
+    }
     const u64 q = c.mod[prime], q5 = 5 * q;
     const ulonglong2 *tw = c.tw_fwd + ((size_t)prime << 16);
     const uint32_t cc = threadIdx.x & 15, r = threadIdx.x >> 4;
@@ -204,10 +283,35 @@ __device__ __forceinline__ uint32_t padded(uint32_t i) { return i + (i >> 4); }
 constexpr uint32_t ROW_PAD = 256 + 16;
 
 // ---- forward, row pass (stages m = 256..32768): CTA = 16 rows, 16 threads per row ---------
-__global__ void __launch_bounds__(F_THREADS) ntt16_fwd_rows(DevTables c, u64 *base, LimbMap map) {
+__global__ void __launch_bounds__(F_THREADS) ntt16_fwd_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
     __shared__ u64 sm[16 * ROW_PAD];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
+    if ((blockIdx.y & 7) < fp_share) {
+        const double q = c.modd[prime].x, qinv = c.modd[prime].y;
+        const double2 *tw = c.twd_fwd + ((size_t)prime << 16);
+        const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
+        u64 *g = base + ((size_t)blockIdx.y << 16) + (size_t)row * 256;
+        double *s = reinterpret_cast<double *>(sm) + rl * ROW_PAD;
+        double x[16];
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) x[k] = reinterpret_cast<const double *>(g)[t + 16 * k];
+        fwd16_d(x, tw, 256 + row, q, qinv);
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) s[padded(t + 16 * k)] = x[k];
+        __syncwarp();
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) x[k] = s[padded(16 * t + k)];
+        fwd16_d(x, tw, 16 * (256 + row) + t, q, qinv);
+        __syncwarp();
+        u64 *su = reinterpret_cast<u64 *>(s);
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) su[padded(16 * t + k)] = canonical_d(reduce_d(x[k], q, qinv), q);
+        __syncwarp();
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) g[t + 16 * k] = su[padded(t + 16 * k)];
+        return;
+    }
     const u64 q = c.mod[prime], q5 = 5 * q;
     const ulonglong2 *tw = c.tw_fwd + ((size_t)prime << 16);
     const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
@@ -233,10 +337,34 @@ __global__ void __launch_bounds__(F_THREADS) ntt16_fwd_rows(DevTables c, u64 *ba
 }
 
 // ---- inverse, row pass (stages m = 32768..256) ---------------------------------------------
-__global__ void __launch_bounds__(F_THREADS) ntt16_inv_rows(DevTables c, u64 *base, LimbMap map) {
+__global__ void __launch_bounds__(F_THREADS) ntt16_inv_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
     __shared__ u64 sm[16 * ROW_PAD];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
+    if ((blockIdx.y & 7) < fp_share) {
+        const double q = c.modd[prime].x, qinv = c.modd[prime].y;
+        const double2 *tw = c.twd_inv + ((size_t)prime << 16);
+        const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
+        u64 *g = base + ((size_t)blockIdx.y << 16) + (size_t)row * 256;
+        double *s = reinterpret_cast<double *>(sm) + rl * ROW_PAD;
+        double x[16];
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) s[padded(t + 16 * k)] = u64_to_d(g[t + 16 * k]);
+        __syncwarp();
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) x[k] = s[padded(16 * t + k)];
+        inv16_d(x, tw, 16 * (256 + row) + t, q, qinv);
+        __syncwarp();
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) s[padded(16 * t + k)] = x[k];
+        __syncwarp();
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) x[k] = s[padded(t + 16 * k)];
+        inv16_d(x, tw, 256 + row, q, qinv);
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) reinterpret_cast<double *>(g)[t + 16 * k] = x[k];
+        return;
+    }
     const u64 q = c.mod[prime];
     const ulonglong2 *tw = c.tw_inv + ((size_t)prime << 16);
     const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
@@ -262,10 +390,31 @@ __global__ void __launch_bounds__(F_THREADS) ntt16_inv_rows(DevTables c, u64 *ba
 }
 
 // ---- inverse, column pass (stages m = 128..1), then N^-1 and the exact reduction -----------
-__global__ void __launch_bounds__(F_THREADS) ntt16_inv_cols(DevTables c, u64 *base, LimbMap map) {
+__global__ void __launch_bounds__(F_THREADS) ntt16_inv_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
     __shared__ u64 sm[256 * 16];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
+    if ((blockIdx.y & 7) < fp_share) {
+        const double q = c.modd[prime].x, qinv = c.modd[prime].y;
+        const double2 *tw = c.twd_inv + ((size_t)prime << 16);
+        const uint32_t cc = threadIdx.x & 15, r = threadIdx.x >> 4;
+        u64 *g = base + ((size_t)blockIdx.y << 16) + blockIdx.x * 16 + cc;
+        double *smd = reinterpret_cast<double *>(sm);
+        double x[16];
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) x[k] = reinterpret_cast<const double *>(g)[(size_t)(16 * r + k) * 256];
+        inv16_d(x, tw, 16 + r, q, qinv);
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) smd[(16 * r + k) * 16 + cc] = x[k];
+        __syncthreads();
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) x[k] = smd[(r + 16 * k) * 16 + cc];
+        inv16_d(x, tw, 1, q, qinv);
+        const double2 ni = c.n_inv_d[prime];
+#pragma unroll
+        for (uint32_t k = 0; k < 16; k++) g[(size_t)(r + 16 * k) * 256] = canonical_d(mulmod_d<0>(x[k], ni, q), q);   // |x| <= 2q < 2^51
+        return;
+    }
     const u64 q = c.mod[prime];
     const ulonglong2 *tw = c.tw_inv + ((size_t)prime << 16);
     const uint32_t cc = threadIdx.x & 15, r = threadIdx.x >> 4;
@@ -296,11 +445,11 @@ void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbM
             u64 *b = base + ((size_t)y0 << 16);
             dim3 grid(16, ny);
             if (!inverse) {
-                ntt16_fwd_cols<<<grid, F_THREADS, 0, s>>>(c->dev, b, map); count_launches();
-                ntt16_fwd_rows<<<grid, F_THREADS, 0, s>>>(c->dev, b, map); count_launches();
+                ntt16_fwd_cols<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share); count_launches();
+                ntt16_fwd_rows<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share); count_launches();
             } else {
-                ntt16_inv_rows<<<grid, F_THREADS, 0, s>>>(c->dev, b, map); count_launches();
-                ntt16_inv_cols<<<grid, F_THREADS, 0, s>>>(c->dev, b, map); count_launches();
+                ntt16_inv_rows<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share); count_launches();
+                ntt16_inv_cols<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share); count_launches();
             }
             y0 += ny;
         }
