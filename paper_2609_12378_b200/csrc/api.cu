@@ -94,7 +94,7 @@ ProjWs proj_layout(const ckks_ctx *c, const ProjPlan &p, uint32_t level) {
     w.acc = off;   off += align256(ct * p.S * w.gg);
     w.total = off; off += align256(ct * p.S);
     w.tmp = off;   off += align256(ct);
-    w.ks = off;    off += align256(ks_bytes(c, level));
+    w.ks = off;    off += align256(ks_bytes(c, level) * p.S * nib);   // all shards' key switches run side by side
     w.rs = off;    off += align256(rescale_bytes(c, level, 2));
     w.bytes = off;
     return w;
@@ -226,7 +226,7 @@ extern "C" int32_t ckks_ntt(ckks_ctx *c, uint64_t *polys, uint32_t batch, uint32
     if (!c || !polys || !batch || !nlimbs) return CKKS_ERR_ARG;
     if ((uint64_t)first + nlimbs > c->T) return CKKS_ERR_LEVEL;
     DeviceGuard g(c->device);
-    launch_ntt(c, (u64 *)polys, batch * nlimbs, LimbMap{0, first, nlimbs, 0, 0, 0, 0}, false, (cudaStream_t)stream);
+    launch_ntt(c, (u64 *)polys, batch * nlimbs, plain_map(first, nlimbs), false, (cudaStream_t)stream);
     return finish(c);
 }
 
@@ -234,7 +234,7 @@ extern "C" int32_t ckks_intt(ckks_ctx *c, uint64_t *polys, uint32_t batch, uint3
     if (!c || !polys || !batch || !nlimbs) return CKKS_ERR_ARG;
     if ((uint64_t)first + nlimbs > c->T) return CKKS_ERR_LEVEL;
     DeviceGuard g(c->device);
-    launch_ntt(c, (u64 *)polys, batch * nlimbs, LimbMap{0, first, nlimbs, 0, 0, 0, 0}, true, (cudaStream_t)stream);
+    launch_ntt(c, (u64 *)polys, batch * nlimbs, plain_map(first, nlimbs), true, (cudaStream_t)stream);
     return finish(c);
 }
 
@@ -422,22 +422,20 @@ extern "C" int32_t ckks_linear_proj(ckks_ctx *c, const ckks_proj_desc *d, const 
     u64 *total = (u64 *)(base + L.total), *tmp = (u64 *)(base + L.tmp), *rsw = (u64 *)(base + L.rs);
     double *slots = (double *)(base + L.slots);
     void *encw = base + L.enc;
-    KsWorkspace kw = ks_carve(c, level, base + L.ks);
+    KsWorkspace kw = ks_carve(c, level, base + L.ks, S * nib);
 
-    // baby[(sh*nib + ib)*B + b] = rho^(b T)(x_{sh,ib}), hoisted per input ciphertext
-    for (uint32_t sh = 0; sh < S; sh++)
-        for (uint32_t ib = 0; ib < nib; ib++) {
-            const u64 *x = (const u64 *)in[sh * nib + ib].data;
-            u64 *slot0 = baby + ((size_t)(sh * nib + ib) * B) * ctl;
-            cudaMemcpyAsync(slot0, x, ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
-            if (B > 1) {
-                ks_modup(c, x + ptl, 1, level, kw, s);
-                for (uint32_t b = 1; b < B; b++) {
-                    const u64 ge = ckks_galois_element(c, (int64_t)b * T);
-                    ks_inner_moddown(c, (const u64 *)find_key(keys, nkeys, ge)->data, level, ge, kw, x, nullptr, ge, slot0 + (size_t)b * ctl, s);
-                }
-            }
+    // baby[(sh*nib + ib)*B + b] = rho^(b T)(x_{sh,ib}): one ModUp for all input ciphertexts at once, then every
+    // baby rotation is applied to all of them in one batch (the key is read once per rotation, not once per shard)
+    for (uint32_t x = 0; x < S * nib; x++)
+        cudaMemcpyAsync(baby + (size_t)x * B * ctl, in[x].data, ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+    if (B > 1) {
+        ks_modup(c, baby + ptl, 1, level, kw, s, S * nib, (size_t)B * ctl);
+        for (uint32_t b = 1; b < B; b++) {
+            const u64 ge = ckks_galois_element(c, (int64_t)b * T);
+            ks_inner_moddown(c, (const u64 *)find_key(keys, nkeys, ge)->data, level, ge, kw, baby, nullptr, ge, baby + (size_t)b * ctl, s,
+                             S * nib, (size_t)B * ctl, (size_t)B * ctl, false);
         }
+    }
 
     for (uint32_t ob = 0; ob < nob; ob++) {
         const Block &o = p.outs[ob];
@@ -481,23 +479,19 @@ extern "C" int32_t ckks_linear_proj(ckks_ctx *c, const ckks_proj_desc *d, const 
                 }
                 const u64 ge = ckks_galois_element(c, (int64_t)gi * B * T);
                 const u64 *key = (const u64 *)find_key(keys, nkeys, ge)->data;
-                for (uint32_t sh = 0; sh < S; sh++) {
-                    u64 *a = ag + (size_t)sh * ctl, *t = total + (size_t)sh * ctl;
-                    ks_modup(c, a + ptl, ge, level, kw, s);
-                    ks_inner_moddown(c, key, level, 1, kw, a, nullptr, ge, tmp, s);
-                    launch_add(c, t, tmp, t, 2, level, s);
-                }
+                // total[sh] += rotate(acc_g[sh]) for all shards in one batch
+                ks_modup(c, ag + ptl, ge, level, kw, s, S, ctl);
+                ks_inner_moddown(c, key, level, 1, kw, ag, nullptr, ge, total, s, S, ctl, ctl, true);
             }
         }
         for (uint32_t f = o.size; fold > 1; f *= 2, fold /= 2) {
             const u64 ge = ckks_galois_element(c, (int64_t)f * T);
             const u64 *key = (const u64 *)find_key(keys, nkeys, ge)->data;
-            for (uint32_t sh = 0; sh < S; sh++) {
-                u64 *t = total + (size_t)sh * ctl;
-                ks_modup(c, t + ptl, ge, level, kw, s);
-                ks_inner_moddown(c, key, level, 1, kw, t, nullptr, ge, tmp, s);
-                launch_add(c, t, tmp, t, 2, level, s);
-            }
+            // total += rotate(total): the rotated copy goes to the (now free) accumulator buffer first
+            ks_modup(c, total + ptl, ge, level, kw, s, S, ctl);
+            ks_inner_moddown(c, key, level, 1, kw, total, nullptr, ge, acc, s, S, ctl, ctl, false);
+            for (uint32_t sh = 0; sh < S; sh++)
+                launch_add(c, total + (size_t)sh * ctl, acc + (size_t)sh * ctl, total + (size_t)sh * ctl, 2, level, s);
         }
         for (uint32_t sh = 0; sh < S; sh++)
             launch_rescale(c, total + (size_t)sh * ctl, (u64 *)out[sh * nob + ob].data, 2, level, rsw, s);

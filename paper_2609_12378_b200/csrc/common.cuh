@@ -62,23 +62,33 @@ struct ckks_ctx {
 // Limb addressing for batched limb-wise kernels (NTT): limb y of a buffer
 // [..][period][N] -> prime index, or -1 to skip the limb.
 //   kind 0: prime = first + y % period
-//   kind 1: "extended" layout [digit][level + K]: x = y % period is q_x for
+//   kind 1: "extended" layout [batch][digit][level + K]: x = y % period is q_x for
 //           x < level, else p_{x-level}; with skip_own the digit's own limbs
 //           (which never leave the evaluation domain) are skipped.
 // ---------------------------------------------------------------------------
 struct LimbMap {
-    uint32_t kind, first, period, level, L, alpha, skip_own;
+    uint32_t kind, first, period, pitch, level, L, alpha, nbeta, skip_own;
 };
+// limbs [..][period][N] contiguous, limb x of every period under prime first + x
+inline LimbMap plain_map(uint32_t first, uint32_t period) { return LimbMap{0, first, period, period, 0, 0, 0, 1, 0}; }
+// same, but consecutive periods start `pitch` limbs apart (a sub-range of limbs of a larger array)
+inline LimbMap pitched_map(uint32_t first, uint32_t period, uint32_t pitch) { return LimbMap{0, first, period, pitch, 0, 0, 0, 1, 0}; }
+// extended digits [batch][beta][level + K]
+inline LimbMap ext_map(uint32_t level, uint32_t K, uint32_t L, uint32_t alpha, uint32_t beta) {
+    return LimbMap{1, 0, level + K, level + K, level, L, alpha, beta, 1};
+}
 
 __host__ __device__ inline int limb_prime(const LimbMap &m, uint32_t y) {
     uint32_t x = y % m.period;
     if (m.kind == 0) return (int)(m.first + x);
     if (m.skip_own) {
-        uint32_t j = y / m.period, lo = j * m.alpha, hi = lo + m.alpha < m.level ? lo + m.alpha : m.level;
+        uint32_t j = (y / m.period) % m.nbeta, lo = j * m.alpha, hi = lo + m.alpha < m.level ? lo + m.alpha : m.level;
         if (x >= lo && x < hi) return -1;
     }
     return x < m.level ? (int)x : (int)(m.L + (x - m.level));
 }
+// index (in limbs) of limb y from the base pointer
+__host__ __device__ inline size_t limb_index(const LimbMap &m, uint32_t y) { return (size_t)(y / m.period) * m.pitch + y % m.period; }
 
 // ---------------------------------------------------------------------------
 // Modular arithmetic, primes in (2^49, 2^50).
@@ -164,13 +174,16 @@ void launch_tensor(const ckks_ctx *c, const u64 *a, const u64 *b, u64 *e01, u64 
 // Key switch pieces.  Sizes in limbs: d [level], ext [beta][level+K], u [2][level+K], conv [2][level].
 struct KsWorkspace { u64 *dcoef, *ext, *u, *conv; };
 size_t ks_workspace_limbs(const ckks_ctx *c, uint32_t level);
-KsWorkspace ks_carve(const ckks_ctx *c, uint32_t level, void *ws);
+KsWorkspace ks_carve(const ckks_ctx *c, uint32_t level, void *ws, uint32_t nb = 1);
+// nb key switches side by side (batch entry b reads d + b * d_stride words):
 // sigma_g(d) (d evaluation domain, [level][N]; g = 1: identity) -> ext (evaluation domain, all digits)
-void ks_modup(const ckks_ctx *c, const u64 *d, u64 galois, uint32_t level, const KsWorkspace &w, cudaStream_t s);
+void ks_modup(const ckks_ctx *c, const u64 *d, u64 galois, uint32_t level, const KsWorkspace &w, cudaStream_t s, uint32_t nb = 1,
+              size_t d_stride = 0);
 // inner product with evk (digits read through sigma_{ext_galois}; 1 = identity), ModDown, and the final
-// combination out_c = sigma_{add_galois}(add_c) + k_c.  add0/add1 may be null.
+// combination out_c (+)= sigma_{add_galois}(add_c) + k_c.  add0/add1 may be null.
 void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext_galois, const KsWorkspace &w,
-                      const u64 *add0, const u64 *add1, u64 add_galois, u64 *out, cudaStream_t s);
+                      const u64 *add0, const u64 *add1, u64 add_galois, u64 *out, cudaStream_t s, uint32_t nb = 1,
+                      size_t add_stride = 0, size_t out_stride = 0, bool accumulate = false);
 
 void launch_rescale(const ckks_ctx *c, const u64 *in, u64 *out, uint32_t ncomp, uint32_t level, u64 *ws, cudaStream_t s);
 

@@ -125,8 +125,7 @@ void launch_encode(const ckks_ctx *c, const double *re, const double *im, uint32
         const uint32_t nb = batch - b0 < 32768 ? batch - b0 : 32768;
         reduce_coeffs<<<dim3(N / THREADS, level, nb), THREADS, 0, s>>>(c->dev, coef + (size_t)b0 * N, out + (size_t)b0 * level * N, level); count_launches();
     }
-    LimbMap map{0, 0, level, 0, 0, 0, 0};
-    launch_ntt(c, out, batch * level, map, false, s);
+    launch_ntt(c, out, batch * level, plain_map(0, level), false, s);
 }
 
 void launch_extract_diagonals(const ckks_ctx *c, const double *W, uint32_t d_out_total, uint32_t in0, uint32_t m_in,

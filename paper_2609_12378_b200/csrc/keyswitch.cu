@@ -22,11 +22,11 @@ __device__ __forceinline__ uint32_t galois_src(uint32_t p, u64 g, uint32_t log_n
     return bitrev_n((uint32_t)((e - 1) >> 1), log_n);
 }
 
-// dst[i][p] = src[i][pi_g(p)]  (g = 1: copy)
-__global__ void __launch_bounds__(THREADS) permute_kernel(DevTables c, const u64 *src, u64 *dst, u64 g) {
+// dst[b][i][p] = src[b][i][pi_g(p)]  (g = 1: copy); batch entries src_stride / dst_stride words apart
+__global__ void __launch_bounds__(THREADS) permute_kernel(DevTables c, const u64 *src, size_t src_stride, u64 *dst, size_t dst_stride, u64 g) {
     const uint32_t p = blockIdx.x * THREADS + threadIdx.x;
     const size_t row = (size_t)blockIdx.y * c.N;
-    dst[row + p] = src[row + galois_src(p, g, c.log_n, c.N)];
+    dst[blockIdx.z * dst_stride + row + p] = src[blockIdx.z * src_stride + row + galois_src(p, g, c.log_n, c.N)];
 }
 
 constexpr uint32_t CHUNK = 8;   // targets per CTA row in the basis-conversion kernels
@@ -36,11 +36,14 @@ constexpr uint32_t CHUNK = 8;   // targets per CTA row in the basis-conversion k
 // A thread owns one coefficient of one digit: it forms the centred y_a of the digit's limbs once and then
 // walks a chunk of CHUNK target limbs (blockIdx.y), so the source limbs are read once per chunk.
 template <uint32_t ALPHA>
-__global__ void __launch_bounds__(THREADS) modup_kernel(DevTables c, const u64 *dcoef, const u64 *deval, u64 g,
+__global__ void __launch_bounds__(THREADS) modup_kernel(DevTables c, const u64 *dcoef, const u64 *deval, size_t deval_stride, u64 g,
                                                         u64 *ext, uint32_t level) {
     const uint32_t k = blockIdx.x * THREADS + threadIdx.x;
-    const uint32_t j = blockIdx.z;
+    const uint32_t beta = (level + c.alpha - 1) / c.alpha, j = blockIdx.z % beta, bz = blockIdx.z / beta;
     const uint32_t nt = level + c.K, lo = j * c.alpha, hi = min(lo + c.alpha, level), nd = hi - lo;
+    dcoef += (size_t)bz * level * c.N;
+    deval += bz * deval_stride;
+    ext += (size_t)bz * beta * nt * c.N;
     const size_t cb = ((size_t)level * c.dnum + j) * c.alpha;
     // centred y_a = [d_a qhat_a^-1] as signed doubles (integer Shoup product, then the lift)
     double y[ALPHA];
@@ -76,9 +79,10 @@ __global__ void __launch_bounds__(THREADS) modup_kernel(DevTables c, const u64 *
 }
 
 template <uint32_t ALPHA>
-void launch_modup(const ckks_ctx *c, const u64 *dcoef, const u64 *deval, u64 g, u64 *ext, uint32_t level, cudaStream_t s) {
+void launch_modup(const ckks_ctx *c, const u64 *dcoef, const u64 *deval, size_t deval_stride, u64 g, u64 *ext, uint32_t level,
+                  uint32_t nb, cudaStream_t s) {
     const uint32_t nt = level + c->K, beta = (level + c->alpha - 1) / c->alpha;
-    modup_kernel<ALPHA><<<dim3(c->N / THREADS, (nt + CHUNK - 1) / CHUNK, beta), THREADS, 0, s>>>(c->dev, dcoef, deval, g, ext, level);
+    modup_kernel<ALPHA><<<dim3(c->N / THREADS, (nt + CHUNK - 1) / CHUNK, beta * nb), THREADS, 0, s>>>(c->dev, dcoef, deval, deval_stride, g, ext, level);
     count_launches();
 }
 
@@ -86,11 +90,13 @@ void launch_modup(const ckks_ctx *c, const u64 *dcoef, const u64 *deval, u64 g, 
 __global__ void __launch_bounds__(THREADS) inner_product_kernel(DevTables c, const u64 *ext, const u64 *evk, u64 g,
                                                                 u64 *u, uint32_t level) {
     const uint32_t p = blockIdx.x * THREADS + threadIdx.x;
-    const uint32_t x = blockIdx.y;
+    const uint32_t x = blockIdx.z, bz = blockIdx.y;     // batch varies faster than the limb: a key limb is reused from L2
     const uint32_t nt = level + c.K, beta = (level + c.alpha - 1) / c.alpha;
     const uint32_t kt = x < level ? x : c.L + (x - level);
     const u64 m = c.mod[kt], mu = c.mu[kt];
     const uint32_t src = galois_src(p, g, c.log_n, c.N);
+    ext += (size_t)bz * beta * nt * c.N;
+    u += (size_t)bz * 2 * nt * c.N;
     u64 h0 = 0, l0 = 0, h1 = 0, l1 = 0;
     for (uint32_t j = 0; j < beta; j++) {
         const u64 e = ext[((size_t)j * nt + x) * c.N + src];
@@ -106,8 +112,10 @@ __global__ void __launch_bounds__(THREADS) inner_product_kernel(DevTables c, con
 template <uint32_t KK>
 __global__ void __launch_bounds__(THREADS) moddown_conv_kernel(DevTables c, const u64 *u, u64 *conv, uint32_t level) {
     const uint32_t k = blockIdx.x * THREADS + threadIdx.x;
-    const uint32_t comp = blockIdx.z;
+    const uint32_t comp = blockIdx.z & 1, bz = blockIdx.z >> 1;
     const uint32_t nt = level + c.K;
+    u += (size_t)bz * 2 * nt * c.N;
+    conv += (size_t)bz * 2 * level * c.N;
     double y[KK];
 #pragma unroll
     for (uint32_t a = 0; a < KK; a++) {
@@ -134,8 +142,8 @@ __global__ void __launch_bounds__(THREADS) moddown_conv_kernel(DevTables c, cons
 }
 
 template <uint32_t KK>
-void launch_moddown_conv(const ckks_ctx *c, const u64 *u, u64 *conv, uint32_t level, cudaStream_t s) {
-    moddown_conv_kernel<KK><<<dim3(c->N / THREADS, (level + CHUNK - 1) / CHUNK, 2), THREADS, 0, s>>>(c->dev, u, conv, level);
+void launch_moddown_conv(const ckks_ctx *c, const u64 *u, u64 *conv, uint32_t level, uint32_t nb, cudaStream_t s) {
+    moddown_conv_kernel<KK><<<dim3(c->N / THREADS, (level + CHUNK - 1) / CHUNK, 2 * nb), THREADS, 0, s>>>(c->dev, u, conv, level);
     count_launches();
 }
 
@@ -151,19 +159,22 @@ void launch_moddown_conv(const ckks_ctx *c, const u64 *u, u64 *conv, uint32_t le
         else { CALL(64); }                          \
     } while (0)
 
-// out[comp][i][p] = (u[comp][i][p] - conv[comp][i][p]) P^-1 + add_comp[i][pi_g(p)]
+// out[b][comp][i][p] (+)= (u[b][comp][i][p] - conv[b][comp][i][p]) P^-1 + add_comp[b][i][pi_g(p)]
 __global__ void __launch_bounds__(THREADS) moddown_final_kernel(DevTables c, const u64 *u, const u64 *conv, const u64 *add0,
-                                                                const u64 *add1, u64 g, u64 *out, uint32_t level) {
+                                                                const u64 *add1, size_t add_stride, u64 g, u64 *out,
+                                                                size_t out_stride, int accumulate, uint32_t level) {
     const uint32_t p = blockIdx.x * THREADS + threadIdx.x;
-    const uint32_t i = blockIdx.y, comp = blockIdx.z;
+    const uint32_t i = blockIdx.y, comp = blockIdx.z & 1, bz = blockIdx.z >> 1;
     const uint32_t nt = level + c.K;
     const u64 q = c.mod[i];
     const ulonglong2 pinv = c.dn_p_inv[i];
-    u64 r = sub_mod(u[((size_t)comp * nt + i) * c.N + p], conv[((size_t)comp * level + i) * c.N + p], q);
+    u64 r = sub_mod(u[(((size_t)bz * 2 + comp) * nt + i) * c.N + p], conv[(((size_t)bz * 2 + comp) * level + i) * c.N + p], q);
     r = mul_shoup(r, pinv.x, pinv.y, q);
     const u64 *add = comp ? add1 : add0;
-    if (add) r = add_mod(r, add[(size_t)i * c.N + galois_src(p, g, c.log_n, c.N)], q);
-    out[((size_t)comp * level + i) * c.N + p] = r;
+    if (add) r = add_mod(r, add[bz * add_stride + (size_t)i * c.N + galois_src(p, g, c.log_n, c.N)], q);
+    u64 *dst = out + bz * out_stride + ((size_t)comp * level + i) * c.N + p;
+    if (accumulate) r = add_mod(r, *dst, q);
+    *dst = r;
 }
 
 // tmp[comp][i][k] = centred lift of last[comp][k] (mod q_last) taken mod q_i
@@ -183,8 +194,6 @@ __global__ void __launch_bounds__(THREADS) rescale_final_kernel(DevTables c, con
     out[((size_t)comp * (level - 1) + i) * c.N + p] = mul_shoup(r, inv.x, inv.y, q);
 }
 
-inline LimbMap plain_map(uint32_t first, uint32_t period) { return LimbMap{0, first, period, 0, 0, 0, 0}; }
-
 }  // namespace
 
 size_t ks_workspace_limbs(const ckks_ctx *c, uint32_t level) {
@@ -192,38 +201,43 @@ size_t ks_workspace_limbs(const ckks_ctx *c, uint32_t level) {
     return level + beta * nt + 2 * nt + 2 * (size_t)level;
 }
 
-KsWorkspace ks_carve(const ckks_ctx *c, uint32_t level, void *ws) {
+// Workspace for nb key switches running side by side: dcoef [nb][level], ext [nb][beta][level+K],
+// u [nb][2][level+K], conv [nb][2][level].
+KsWorkspace ks_carve(const ckks_ctx *c, uint32_t level, void *ws, uint32_t nb) {
     const size_t beta = (level + c->alpha - 1) / c->alpha, nt = level + c->K, N = c->N;
     KsWorkspace w;
     w.dcoef = (u64 *)ws;
-    w.ext = w.dcoef + (size_t)level * N;
-    w.u = w.ext + beta * nt * N;
-    w.conv = w.u + 2 * nt * N;
+    w.ext = w.dcoef + (size_t)nb * level * N;
+    w.u = w.ext + (size_t)nb * beta * nt * N;
+    w.conv = w.u + (size_t)nb * 2 * nt * N;
     return w;
 }
 
-void ks_modup(const ckks_ctx *c, const u64 *d, u64 galois, uint32_t level, const KsWorkspace &w, cudaStream_t s) {
+void ks_modup(const ckks_ctx *c, const u64 *d, u64 galois, uint32_t level, const KsWorkspace &w, cudaStream_t s, uint32_t nb,
+              size_t d_stride) {
     const uint32_t N = c->N, beta = (level + c->alpha - 1) / c->alpha, nt = level + c->K;
-    permute_kernel<<<dim3(N / THREADS, level), THREADS, 0, s>>>(c->dev, d, w.dcoef, galois); count_launches();
-    launch_ntt(c, w.dcoef, level, plain_map(0, level), true, s);
-#define CALL_UP(A) launch_modup<A>(c, w.dcoef, d, galois, w.ext, level, s)
+    permute_kernel<<<dim3(N / THREADS, level, nb), THREADS, 0, s>>>(c->dev, d, d_stride, w.dcoef, (size_t)level * N, galois); count_launches();
+    launch_ntt(c, w.dcoef, nb * level, plain_map(0, level), true, s);
+#define CALL_UP(A) launch_modup<A>(c, w.dcoef, d, d_stride, galois, w.ext, level, nb, s)
     DISPATCH_POW2(c->alpha, CALL_UP);
 #undef CALL_UP
-    LimbMap em{1, 0, nt, level, c->L, c->alpha, 1};
-    launch_ntt(c, w.ext, beta * nt, em, false, s);
+    launch_ntt(c, w.ext, nb * beta * nt, ext_map(level, c->K, c->L, c->alpha, beta), false, s);
 }
 
 void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext_galois, const KsWorkspace &w,
-                      const u64 *add0, const u64 *add1, u64 add_galois, u64 *out, cudaStream_t s) {
+                      const u64 *add0, const u64 *add1, u64 add_galois, u64 *out, cudaStream_t s, uint32_t nb,
+                      size_t add_stride, size_t out_stride, bool accumulate) {
     const uint32_t N = c->N, nt = level + c->K, K = c->K;
-    inner_product_kernel<<<dim3(N / THREADS, nt), THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level); count_launches();
-    for (uint32_t comp = 0; comp < 2; comp++)
-        launch_ntt(c, w.u + ((size_t)comp * nt + level) * N, K, plain_map(c->L, K), true, s);
-#define CALL_DN(A) launch_moddown_conv<A>(c, w.u, w.conv, level, s)
+    inner_product_kernel<<<dim3(N / THREADS, nb, nt), THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level); count_launches();
+    // the K special limbs of every (batch, component): groups of K limbs, nt limbs apart
+    launch_ntt(c, w.u + (size_t)level * N, nb * 2 * K, pitched_map(c->L, K, nt), true, s);
+#define CALL_DN(A) launch_moddown_conv<A>(c, w.u, w.conv, level, nb, s)
     DISPATCH_POW2(K, CALL_DN);
 #undef CALL_DN
-    launch_ntt(c, w.conv, 2 * level, plain_map(0, level), false, s);
-    moddown_final_kernel<<<dim3(N / THREADS, level, 2), THREADS, 0, s>>>(c->dev, w.u, w.conv, add0, add1, add_galois, out, level); count_launches();
+    launch_ntt(c, w.conv, nb * 2 * level, plain_map(0, level), false, s);
+    moddown_final_kernel<<<dim3(N / THREADS, level, 2 * nb), THREADS, 0, s>>>(c->dev, w.u, w.conv, add0, add1, add_stride, add_galois, out,
+                                                                               out_stride, accumulate ? 1 : 0, level);
+    count_launches();
 }
 
 // ws: [ncomp][N] last limbs + [ncomp][level-1][N]

@@ -27,7 +27,7 @@ __global__ void __launch_bounds__(THREADS) ntt_cols(DevTables c, u64 *base, Limb
     const uint32_t N = c.N, R = N / ROW;
     const u64 q = c.mod[prime];
     const ulonglong2 *tw = (INV ? c.tw_inv : c.tw_fwd) + (size_t)prime * N;
-    u64 *g = base + (size_t)blockIdx.y * N + blockIdx.x * COLS;
+    u64 *g = base + limb_index(map, blockIdx.y) * N + blockIdx.x * COLS;
     for (uint32_t x = threadIdx.x; x < R * COLS; x += THREADS) sm[x] = g[(size_t)(x / COLS) * ROW + x % COLS];
     __syncthreads();
     if (!INV) {
@@ -69,7 +69,7 @@ __global__ void __launch_bounds__(THREADS) ntt_rows(DevTables c, u64 *base, Limb
     const u64 q = c.mod[prime];
     const ulonglong2 *tw = (INV ? c.tw_inv : c.tw_fwd) + (size_t)prime * N;
     const uint32_t row0 = blockIdx.x * rows;
-    u64 *g = base + (size_t)blockIdx.y * N + (size_t)row0 * ROW;
+    u64 *g = base + limb_index(map, blockIdx.y) * N + (size_t)row0 * ROW;
     for (uint32_t x = threadIdx.x; x < rows * ROW; x += THREADS) sm[x] = g[x];
     __syncthreads();
     // local stage mp = 1 .. 128: global stage m = R*mp, distance t = 128/mp, twiddle index mp*(R + row) + i_local
@@ -244,7 +244,7 @@ __global__ void __launch_bounds__(F_THREADS) ntt16_fwd_cols(DevTables c, u64 *ba
         const double q = c.modd[prime].x, qinv = c.modd[prime].y;
         const double2 *tw = c.twd_fwd + ((size_t)prime << 16);
         const uint32_t cc = threadIdx.x & 15, r = threadIdx.x >> 4;
-        u64 *g = base + ((size_t)blockIdx.y << 16) + blockIdx.x * 16 + cc;
+        u64 *g = base + (limb_index(map, blockIdx.y) << 16) + blockIdx.x * 16 + cc;
         double *smd = reinterpret_cast<double *>(sm);
         double x[16];
 #pragma unroll
@@ -263,7 +263,7 @@ __global__ void __launch_bounds__(F_THREADS) ntt16_fwd_cols(DevTables c, u64 *ba
     const u64 q = c.mod[prime], q5 = 5 * q;
     const ulonglong2 *tw = c.tw_fwd + ((size_t)prime << 16);
     const uint32_t cc = threadIdx.x & 15, r = threadIdx.x >> 4;
-    u64 *g = base + ((size_t)blockIdx.y << 16) + blockIdx.x * 16 + cc;
+    u64 *g = base + (limb_index(map, blockIdx.y) << 16) + blockIdx.x * 16 + cc;
     u64 x[16];
 #pragma unroll
     for (uint32_t k = 0; k < 16; k++) x[k] = g[(size_t)(r + 16 * k) * 256];
@@ -291,7 +291,7 @@ __global__ void __launch_bounds__(F_THREADS) ntt16_fwd_rows(DevTables c, u64 *ba
         const double q = c.modd[prime].x, qinv = c.modd[prime].y;
         const double2 *tw = c.twd_fwd + ((size_t)prime << 16);
         const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
-        u64 *g = base + ((size_t)blockIdx.y << 16) + (size_t)row * 256;
+        u64 *g = base + (limb_index(map, blockIdx.y) << 16) + (size_t)row * 256;
         double *s = reinterpret_cast<double *>(sm) + rl * ROW_PAD;
         double x[16];
 #pragma unroll
@@ -315,7 +315,7 @@ __global__ void __launch_bounds__(F_THREADS) ntt16_fwd_rows(DevTables c, u64 *ba
     const u64 q = c.mod[prime], q5 = 5 * q;
     const ulonglong2 *tw = c.tw_fwd + ((size_t)prime << 16);
     const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
-    u64 *g = base + ((size_t)blockIdx.y << 16) + (size_t)row * 256;
+    u64 *g = base + (limb_index(map, blockIdx.y) << 16) + (size_t)row * 256;
     u64 *s = sm + rl * ROW_PAD;
     u64 x[16];
 #pragma unroll
@@ -345,7 +345,7 @@ __global__ void __launch_bounds__(F_THREADS) ntt16_inv_rows(DevTables c, u64 *ba
         const double q = c.modd[prime].x, qinv = c.modd[prime].y;
         const double2 *tw = c.twd_inv + ((size_t)prime << 16);
         const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
-        u64 *g = base + ((size_t)blockIdx.y << 16) + (size_t)row * 256;
+        u64 *g = base + (limb_index(map, blockIdx.y) << 16) + (size_t)row * 256;
         double *s = reinterpret_cast<double *>(sm) + rl * ROW_PAD;
         double x[16];
 #pragma unroll
@@ -368,7 +368,7 @@ __global__ void __launch_bounds__(F_THREADS) ntt16_inv_rows(DevTables c, u64 *ba
     const u64 q = c.mod[prime];
     const ulonglong2 *tw = c.tw_inv + ((size_t)prime << 16);
     const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
-    u64 *g = base + ((size_t)blockIdx.y << 16) + (size_t)row * 256;
+    u64 *g = base + (limb_index(map, blockIdx.y) << 16) + (size_t)row * 256;
     u64 *s = sm + rl * ROW_PAD;
     u64 x[16];
 #pragma unroll
@@ -398,7 +398,7 @@ __global__ void __launch_bounds__(F_THREADS) ntt16_inv_cols(DevTables c, u64 *ba
         const double q = c.modd[prime].x, qinv = c.modd[prime].y;
         const double2 *tw = c.twd_inv + ((size_t)prime << 16);
         const uint32_t cc = threadIdx.x & 15, r = threadIdx.x >> 4;
-        u64 *g = base + ((size_t)blockIdx.y << 16) + blockIdx.x * 16 + cc;
+        u64 *g = base + (limb_index(map, blockIdx.y) << 16) + blockIdx.x * 16 + cc;
         double *smd = reinterpret_cast<double *>(sm);
         double x[16];
 #pragma unroll
@@ -418,7 +418,7 @@ __global__ void __launch_bounds__(F_THREADS) ntt16_inv_cols(DevTables c, u64 *ba
     const u64 q = c.mod[prime];
     const ulonglong2 *tw = c.tw_inv + ((size_t)prime << 16);
     const uint32_t cc = threadIdx.x & 15, r = threadIdx.x >> 4;
-    u64 *g = base + ((size_t)blockIdx.y << 16) + blockIdx.x * 16 + cc;
+    u64 *g = base + (limb_index(map, blockIdx.y) << 16) + blockIdx.x * 16 + cc;
     u64 x[16];
 #pragma unroll
     for (uint32_t k = 0; k < 16; k++) x[k] = g[(size_t)(16 * r + k) * 256];
@@ -442,7 +442,7 @@ void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbM
         for (uint32_t y0 = 0; y0 < nlimbs_total;) {
             const uint32_t chunk = map.period >= 32768 ? map.period : (32768 / map.period) * map.period;
             const uint32_t ny = nlimbs_total - y0 < chunk ? nlimbs_total - y0 : chunk;
-            u64 *b = base + ((size_t)y0 << 16);
+            u64 *b = base + (limb_index(map, y0) << 16);
             dim3 grid(16, ny);
             if (!inverse) {
                 ntt16_fwd_cols<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share); count_launches();
@@ -462,7 +462,7 @@ void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbM
     const uint32_t chunk = map.period >= 32768 ? map.period : (32768 / map.period) * map.period;
     for (uint32_t y0 = 0; y0 < nlimbs_total; y0 += chunk) {
         const uint32_t ny = nlimbs_total - y0 < chunk ? nlimbs_total - y0 : chunk;
-        u64 *b = base + (size_t)y0 * N;
+        u64 *b = base + limb_index(map, y0) * N;
         dim3 gc(ROW / COLS, ny), gr(R / rows, ny);
         if (!inverse) {
             ntt_cols<false><<<gc, THREADS, smc, s>>>(c->dev, b, map); count_launches();
