@@ -58,6 +58,16 @@ def test_projection_shapes_small_ring(d_in, d_out, T, S, B):
     _run(10, 4, 2, 2, 4, d_in, d_out, T, S, B, seed=400 + d_in + d_out)
 
 
+@pytest.mark.parametrize("d_in,d_out,T,S,B", [
+    (64, 64, 8, 2, 32),      # J = 32: one k-step of the tensor-core multiply-accumulate
+    (64, 64, 8, 3, 64),      # J = 64, odd shard count (column padding), single giant step
+    (128, 64, 8, 1, 32),     # two input blocks: J = 64
+    (64, 160, 8, 9, 32),     # remainder output block 32 | 64, folded; more than one column tile
+])
+def test_projection_tensor_core_mac_path(d_in, d_out, T, S, B):
+    _run(10, 4, 2, 2, 4, d_in, d_out, T, S, B, seed=440 + d_in + d_out + S)
+
+
 def test_projection_explicit_pt_scale_and_lower_level():
     _run(10, 4, 2, 2, 3, 16, 16, 32, 1, 4, seed=410, pt_scale=2.0 ** 40, check_slots=False)
 
@@ -71,6 +81,11 @@ def test_projection_toy_config():
 def test_projection_full_ring_small_shape():
     """N = 2^16, L = 24, dnum = 3 with 512 tokens per shard: F = 64 features, B = G = 8."""
     _run(16, 24, 8, 3, 24, 64, 64, 512, 1, 8, seed=420)
+
+
+def test_projection_full_ring_tensor_core_mac():
+    """N = 2^16, L = 24, dnum = 3, F = 64 features, B = 32, G = 2: the tensor-core multiply-accumulate at full ring size."""
+    _run(16, 24, 8, 3, 24, 64, 64, 512, 2, 32, seed=421)
 
 
 def test_projection_errors():
