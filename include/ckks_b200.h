@@ -153,6 +153,10 @@ int32_t ckks_encode(ckks_ctx *ctx, const double *re, const double *im, uint32_t 
  * query overflowed (and clears the flag), else CKKS_OK. */
 int32_t ckks_encode_range_flag(ckks_ctx *ctx, void *stream);
 
+/* Synchronises `stream`; returns CKKS_ERR_TIMEOUT if a bounded device-side wait (the TMA pipeline of the
+ * projection's multiply-accumulate) gave up since the last query (and clears the flag), else CKKS_OK. */
+int32_t ckks_device_status(ckks_ctx *ctx, void *stream);
+
 /* ---- PCMult + Add (Section 2.1) -------------------------------------------
  * accs[s] (+)= cts[s] * pt for s < ncts, both components, all limbs.  cts,
  * accs: host arrays of descriptors.  init = 1: accs[s] = cts[s]*pt and

@@ -21,7 +21,7 @@ EXPORTS = [
     "ckks_workspace_bytes", "ckks_galois_element", "ckks_ntt", "ckks_intt", "ckks_encode",
     "ckks_encode_range_flag", "ckks_mul_plain_acc", "ckks_add", "ckks_mul_relin", "ckks_rotate",
     "ckks_rotate_hoisted", "ckks_rescale", "ckks_linear_proj", "ckks_linear_proj_workspace_bytes",
-    "ckks_linear_proj_rotations", "ckks_kernel_launches",
+    "ckks_linear_proj_rotations", "ckks_kernel_launches", "ckks_device_status",
 ]
 
 
@@ -71,6 +71,7 @@ def load():
         "ckks_intt": (i32, [vp, vp, u32, u32, u32, vp]),
         "ckks_encode": (i32, [vp, vp, vp, u32, dbl, u32, vp, vp, sz, vp]),
         "ckks_encode_range_flag": (i32, [vp, vp]),
+        "ckks_device_status": (i32, [vp, vp]),
         "ckks_mul_plain_acc": (i32, [vp, C.POINTER(CCt), u32, C.POINTER(CPt), C.POINTER(CCt), i32, vp]),
         "ckks_add": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), C.POINTER(CCt), vp]),
         "ckks_mul_relin": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
@@ -231,6 +232,9 @@ class Context:
 
     def encode_range_flag(self, stream=None) -> int:
         return int(load().ckks_encode_range_flag(self._h, _stream_ptr(stream)))
+
+    def device_status(self, stream=None) -> int:
+        return int(load().ckks_device_status(self._h, _stream_ptr(stream)))
 
     def mul_plain_acc(self, cts, pt: Plaintext, accs=None, stream=None):
         """accs[s] (+)= cts[s] * pt.  accs None: fresh accumulators are returned."""

@@ -207,139 +207,6 @@ __global__ void __launch_bounds__(MAC_THREADS) mac_tile_kernel(DevTables c, cons
             }
 }
 
-// ---------------------------------------------------------------------------
-// Tensor-core form of the same multiply-accumulate, used when J is a multiple of 32.
-// For one coefficient the group's work is a small dense contraction
-//   out[g][s'] = sum_j w[g][j] x[j][s']        g < 16 giants, s' = 2 shard + component, j < J,
-// which is exact in integer tensor-core arithmetic after splitting every 50-bit word into 7 bytes:
-// the byte products of one weight a + b = d are summed over j by mma.m16n8k32 (u8 x u8 -> s32; J * 7 * 255^2
-// stays far below 2^31), giving 13 diagonal sums D_d per output, and out = sum_d D_d 2^(8d) < 2^110 is
-// reduced once.  A warp owns one coefficient: M = 16 giants, N = 16 columns s' (two n-tiles), K = 32 values
-// of j per step.  A CTA (8 warps) owns 8 adjacent coefficients so that every global read is a 64-byte row;
-// rows are staged by cp.async into a 3-deep ring, stored per coefficient with a pitch of 33 words, which
-// makes the fragment reads (row = lane / 4, four consecutive j per lane) bank-conflict free.
-// ---------------------------------------------------------------------------
-constexpr uint32_t MMA_COEF = 8, MMA_G = 16, MMA_S = 16, MMA_K = 32, MMA_PITCH = 33, MMA_STAGES = 3;
-constexpr uint32_t MMA_TILE = MMA_G * MMA_PITCH;                       // words per coefficient per operand
-constexpr uint32_t MMA_STAGE_WORDS = 2 * MMA_COEF * MMA_TILE;          // W tile + X tile
-constexpr size_t MMA_SMEM = (size_t)MMA_STAGES * MMA_STAGE_WORDS * sizeof(u64);
-
-__device__ __forceinline__ void mma_u8(int (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
-    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
-}
-// byte `plane` of four words, packed lowest word first
-template <uint32_t PLANE>
-__device__ __forceinline__ uint32_t pack_plane(const u64 (&w)[4]) {
-    constexpr uint32_t bsel = PLANE & 3;
-    const uint32_t x0 = PLANE < 4 ? (uint32_t)w[0] : (uint32_t)(w[0] >> 32), x1 = PLANE < 4 ? (uint32_t)w[1] : (uint32_t)(w[1] >> 32);
-    const uint32_t x2 = PLANE < 4 ? (uint32_t)w[2] : (uint32_t)(w[2] >> 32), x3 = PLANE < 4 ? (uint32_t)w[3] : (uint32_t)(w[3] >> 32);
-    const uint32_t t0 = __byte_perm(x0, x1, bsel | ((4 + bsel) << 4)), t1 = __byte_perm(x2, x3, bsel | ((4 + bsel) << 4));
-    return __byte_perm(t0, t1, 0x5410);
-}
-template <uint32_t NREG>
-__device__ __forceinline__ void planes7(const u64 (&w)[NREG][4], uint32_t (&f)[7][NREG]) {
-#pragma unroll
-    for (uint32_t r = 0; r < NREG; r++) {
-        f[0][r] = pack_plane<0>(w[r]); f[1][r] = pack_plane<1>(w[r]); f[2][r] = pack_plane<2>(w[r]); f[3][r] = pack_plane<3>(w[r]);
-        f[4][r] = pack_plane<4>(w[r]); f[5][r] = pack_plane<5>(w[r]); f[6][r] = pack_plane<6>(w[r]);
-    }
-}
-
-__global__ void __launch_bounds__(256, 1) mac_mma_kernel(DevTables c, const u64 *__restrict__ baby, const u64 *__restrict__ pts,
-                                                         u64 *__restrict__ acc, uint32_t J, uint32_t Jstride, uint32_t S,
-                                                         uint32_t G, uint32_t level) {
-    extern __shared__ u64 mma_sm[];
-    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, gid = lane >> 2, tig = lane & 3;
-    const uint32_t p0 = blockIdx.x * MMA_COEF, i = blockIdx.y;
-    const uint32_t ncol = 2 * S, coltiles = (ncol + MMA_S - 1) / MMA_S;
-    const uint32_t col0 = (blockIdx.z % coltiles) * MMA_S, g0 = (blockIdx.z / coltiles) * MMA_G;
-    const size_t lN = (size_t)level * c.N, ctl = 2 * lN, off = (size_t)i * c.N + p0;
-    const uint32_t nk = J / MMA_K;
-
-    // loader: element e -> (coefficient e & 7, row e >> 3); rows 0..511 are W (g, j), rows 512..1023 are X (s', j).
-    // Rows beyond G or beyond the last column re-read row/column 0; their results are never stored.
-    auto issue = [&](uint32_t ks) {
-        if (ks < nk) {
-            u64 *st = mma_sm + (size_t)(ks % MMA_STAGES) * MMA_STAGE_WORDS;
-#pragma unroll 4
-            for (uint32_t it = 0; it < (2 * MMA_G * MMA_K * MMA_COEF) / 256; it++) {
-                const uint32_t e = it * 256 + tid, cf = e & 7, row = e >> 3, r = row & 511, a = r >> 5, j = ks * MMA_K + (r & 31);
-                const u64 *src;
-                if (row < 512) {
-                    const uint32_t g = g0 + a < G ? g0 + a : 0;
-                    src = pts + ((size_t)g * Jstride + j) * lN + off + cf;
-                } else {
-                    const uint32_t col = col0 + a < ncol ? col0 + a : 0;
-                    src = baby + ((size_t)(col >> 1) * Jstride + j) * ctl + (col & 1) * lN + off + cf;
-                }
-                cp_async8(st + (row < 512 ? 0 : MMA_COEF * MMA_TILE) + cf * MMA_TILE + a * MMA_PITCH + (r & 31), src);
-            }
-        }
-        cp_async_commit();
-    };
-
-    int dsum[2][13][4];
-#pragma unroll
-    for (uint32_t n = 0; n < 2; n++)
-#pragma unroll
-        for (uint32_t d = 0; d < 13; d++)
-#pragma unroll
-            for (uint32_t r = 0; r < 4; r++) dsum[n][d][r] = 0;
-
-#pragma unroll
-    for (uint32_t ks = 0; ks < MMA_STAGES - 1; ks++) issue(ks);
-    for (uint32_t ks = 0; ks < nk; ks++) {
-        cp_async_wait<MMA_STAGES - 2>();
-        __syncthreads();                       // everyone's rows of step ks have landed; the slot of step ks-1 is free
-        issue(ks + MMA_STAGES - 1);
-        const u64 *Wt = mma_sm + (size_t)(ks % MMA_STAGES) * MMA_STAGE_WORDS + warp * MMA_TILE;
-        const u64 *Xt = Wt + MMA_COEF * MMA_TILE;
-        uint32_t A[7][4];
-        {
-            u64 w[4][4];                       // fragment register r + 2h: row gid + 8r, j = 16h + 4 tig + e
-#pragma unroll
-            for (uint32_t r = 0; r < 2; r++)
-#pragma unroll
-                for (uint32_t h = 0; h < 2; h++)
-#pragma unroll
-                    for (uint32_t e = 0; e < 4; e++) w[r + 2 * h][e] = Wt[(gid + 8 * r) * MMA_PITCH + 16 * h + 4 * tig + e];
-            planes7<4>(w, A);
-        }
-#pragma unroll
-        for (uint32_t n = 0; n < 2; n++) {
-            uint32_t Bf[7][2];
-            {
-                u64 x[2][4];                   // fragment register h: column 8n + gid, j = 16h + 4 tig + e
-#pragma unroll
-                for (uint32_t h = 0; h < 2; h++)
-#pragma unroll
-                    for (uint32_t e = 0; e < 4; e++) x[h][e] = Xt[(8 * n + gid) * MMA_PITCH + 16 * h + 4 * tig + e];
-                planes7<2>(x, Bf);
-            }
-#pragma unroll
-            for (uint32_t a = 0; a < 7; a++)
-#pragma unroll
-                for (uint32_t b = 0; b < 7; b++) mma_u8(dsum[n][a + b], A[a], Bf[b]);
-        }
-    }
-    cp_async_wait<0>();
-
-    const u64 q = c.mod[i], mu = c.mu[i];
-#pragma unroll
-    for (uint32_t n = 0; n < 2; n++)
-#pragma unroll
-        for (uint32_t r = 0; r < 4; r++) {
-            const uint32_t g = g0 + gid + 8 * (r >> 1), col = col0 + 8 * n + 2 * tig + (r & 1);
-            u128 t = 0;
-#pragma unroll
-            for (uint32_t d = 0; d < 13; d++) t += (u128)(uint32_t)dsum[n][d][r] << (8 * d);
-            if (g < G && col < ncol)
-                acc[((size_t)g * S + (col >> 1)) * ctl + (col & 1) * lN + off + warp] = barrett112((u64)(t >> 64), (u64)t, q, mu);
-        }
-}
-
 }  // namespace
 
 extern "C" size_t ckks_workspace_bytes(const ckks_ctx *c, int32_t op, uint32_t level, uint32_t count) {
@@ -390,6 +257,17 @@ extern "C" int32_t ckks_encode_range_flag(ckks_ctx *c, void *stream) {
     if (e == cudaSuccess && flag) e = cudaMemsetAsync(c->dev.range_flag, 0, sizeof(int), (cudaStream_t)stream);
     if (e != cudaSuccess) { c->cuda_error = cudaGetErrorString(e); return CKKS_ERR_CUDA; }
     return flag ? CKKS_ERR_RANGE : CKKS_OK;
+}
+
+extern "C" int32_t ckks_device_status(ckks_ctx *c, void *stream) {
+    if (!c) return CKKS_ERR_ARG;
+    DeviceGuard g(c->device);
+    int flag = 0;
+    cudaError_t e = cudaMemcpyAsync(&flag, c->dev.range_flag + 1, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e == cudaSuccess && flag) e = cudaMemsetAsync(c->dev.range_flag + 1, 0, sizeof(int), (cudaStream_t)stream);
+    if (e != cudaSuccess) { c->cuda_error = cudaGetErrorString(e); return CKKS_ERR_CUDA; }
+    return flag ? CKKS_ERR_TIMEOUT : CKKS_OK;
 }
 
 extern "C" int32_t ckks_mul_plain_acc(ckks_ctx *c, const ckks_ct *cts, uint32_t ncts, const ckks_pt *pt, ckks_ct *accs,
@@ -600,18 +478,10 @@ extern "C" int32_t ckks_linear_proj(ckks_ctx *c, const ckks_proj_desc *d, const 
             if (!ragged) launch_encode(c, slots, nullptr, ng * J, pt_scale, level, pts, encw, s);
             {
                 const uint32_t stiles = (S + MAC_ST - 1) / MAC_ST, gtiles = (ng + MAC_GT - 1) / MAC_GT;
-                if (J % MMA_K == 0) {
-                    static bool attr_set = false;
-                    if (!attr_set) {
-                        cudaFuncSetAttribute(mac_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MMA_SMEM);
-                        attr_set = true;
-                    }
-                    const uint32_t coltiles = (2 * S + MMA_S - 1) / MMA_S, gt = (ng + MMA_G - 1) / MMA_G;
-                    mac_mma_kernel<<<dim3(N / MMA_COEF, level, coltiles * gt), 256, MMA_SMEM, s>>>(c->dev, baby, pts, acc, J, J, S, ng, level);
-                } else {
+                if (!(mac_mma_supported(c, J) && launch_mac_mma(c, baby, pts, acc, J, J, S, ng, level, s))) {
                     mac_tile_kernel<<<dim3(stiles * gtiles, N / MAC_THREADS, level), MAC_THREADS, 0, s>>>(c->dev, baby, pts, acc, J, J, S, ng, level);
+                    count_launches();
                 }
-                count_launches();
             }
             for (uint32_t gl = 0; gl < ng; gl++) {
                 const uint32_t gi = g0 + gl;

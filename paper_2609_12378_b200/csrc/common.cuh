@@ -44,7 +44,7 @@ struct DevTables {
     const uint32_t *enc_src;       // [n] slot index feeding FFT input position pos (bit-reversed e_j)
     const double2 *enc_omega;      // [n] exp(2 pi i t / n)
     const double2 *enc_zeta;       // [n] exp(2 pi i k / 2N)
-    int *range_flag;               // sticky encode overflow flag
+    int *range_flag;               // [0] sticky encode overflow flag, [1] sticky device-side wait timeout flag
 };
 
 struct ckks_ctx {
@@ -184,6 +184,11 @@ void ks_modup(const ckks_ctx *c, const u64 *d, u64 galois, uint32_t level, const
 void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext_galois, const KsWorkspace &w,
                       const u64 *add0, const u64 *add1, u64 add_galois, u64 *out, cudaStream_t s, uint32_t nb = 1,
                       size_t add_stride = 0, size_t out_stride = 0, bool accumulate = false);
+
+// Tensor-core multiply-accumulate of a giant-step group (mac_mma.cu)
+bool mac_mma_supported(const ckks_ctx *c, uint32_t J);
+bool launch_mac_mma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t Jstride, uint32_t S,
+                    uint32_t G, uint32_t level, cudaStream_t s);
 
 void launch_rescale(const ckks_ctx *c, const u64 *in, u64 *out, uint32_t ncomp, uint32_t level, u64 *ws, cudaStream_t s);
 

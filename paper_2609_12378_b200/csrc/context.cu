@@ -250,7 +250,7 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
     DevTables &d = c->dev;
     d.log_n = prm->log_n; d.N = N; d.L = L; d.K = K; d.alpha = alpha; d.T = T; d.dnum = prm->dnum;
     int rc = CKKS_OK;
-    std::vector<int> flag(1, 0);
+    std::vector<int> flag(2, 0);
     const int *flag_dev = nullptr;
     if ((rc = upload(c, mod, &d.mod)) || (rc = upload(c, mu, &d.mu)) || (rc = upload(c, mu64, &d.mu64)) || (rc = upload(c, modd, &d.modd)) || (rc = upload(c, twf, &d.tw_fwd)) ||
         (rc = upload(c, twi, &d.tw_inv)) || (rc = upload(c, twdf, &d.twd_fwd)) || (rc = upload(c, twdi, &d.twd_inv)) || (rc = upload(c, ninvd, &d.n_inv_d)) || (rc = upload(c, ninv, &d.n_inv)) || (rc = upload(c, up_inv, &d.up_hat_inv)) ||
