@@ -73,7 +73,7 @@ int make_plan(const ckks_ctx *c, const ckks_proj_desc *d, ProjPlan &p) {
     return CKKS_OK;
 }
 
-struct ProjWs { size_t baby, pts, slots, enc, acc, total, tmp, ks, rs, bytes; uint32_t gg; };
+struct ProjWs { size_t baby, xin, pts, ptt, slots, enc, acc, total, tmp, ks, rs, bytes; uint32_t gg; };
 
 constexpr uint32_t MAC_GT = 4, MAC_ST = 2;   // register tile of the multiply-accumulate kernel: giants x shards
 
@@ -87,8 +87,10 @@ ProjWs proj_layout(const ckks_ctx *c, const ProjPlan &p, uint32_t level) {
     w.gg = (w.gg + MAC_GT - 1) / MAC_GT * MAC_GT;
     const size_t npt = (size_t)w.gg * nib * p.B;
     size_t off = 0;
-    w.baby = off;  off += align256(ct * p.S * nib * p.B);
-    w.pts = off;   off += align256(pt * npt);
+    w.baby = off;  off += align256(ct * p.S * nib * p.B);   // tiled: rows (shard * J + j) * 2 + component
+    w.xin = off;   off += align256(ct * p.S * nib);         // the inputs side by side, plain layout
+    w.pts = off;   off += align256(pt * npt);               // encoded plaintexts of a group, plain layout
+    w.ptt = off;   off += align256(pt * npt);               // the same, tiled: rows g * J + j
     w.slots = off; off += align256(npt * c->n * sizeof(double));
     w.enc = off;   off += align256(encode_workspace_bytes(c, (uint32_t)npt));
     w.acc = off;   off += align256(ct * p.S * w.gg);
@@ -139,8 +141,7 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 // of loads are in flight per thread while the products of the current step are formed; a thread only ever reads
 // back the words it requested itself, so no block-wide barrier is needed.
 __global__ void __launch_bounds__(MAC_THREADS) mac_tile_kernel(DevTables c, const u64 *__restrict__ baby, const u64 *__restrict__ pts,
-                                                               u64 *__restrict__ acc, uint32_t J, uint32_t Jstride, uint32_t S,
-                                                               uint32_t G, uint32_t level) {
+                                                               u64 *__restrict__ acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level) {
     __shared__ u64 ring[MAC_DEPTH][MAC_WORDS][MAC_THREADS];
     const uint32_t stiles = (S + MAC_ST - 1) / MAC_ST;
     const uint32_t s0 = (blockIdx.x % stiles) * MAC_ST, g0 = (blockIdx.x / stiles) * MAC_GT;
@@ -154,25 +155,27 @@ __global__ void __launch_bounds__(MAC_THREADS) mac_tile_kernel(DevTables c, cons
     for (uint32_t g = 0; g < MAC_GT; g++)
 #pragma unroll
         for (uint32_t x = 0; x < NX; x++) LL[g][x] = HH[g][x] = MM[g][x] = 0;
+    // operands are tiled (tiled_index): row g J + j of pts, row (s J + j) 2 + c of baby; consecutive j are 64 (128) words apart
     const u64 *wp[MAC_GT], *xp[NX];
     bool wok[MAC_GT], xok[NX];
+    const uint32_t Rw = G * J, Rx = 2 * S * J;
 #pragma unroll
     for (uint32_t g = 0; g < MAC_GT; g++) {
         wok[g] = g0 + g < G;                      // out-of-range tiles read tile 0 and are never stored
-        wp[g] = pts + (size_t)(wok[g] ? g0 + g : 0) * Jstride * lN + off;
+        wp[g] = pts + tiled_index(Rw, c.N, (wok[g] ? g0 + g : 0) * J, i, p);
     }
 #pragma unroll
     for (uint32_t x = 0; x < NX; x++) {
         xok[x] = s0 + x / 2 < S;
-        xp[x] = baby + (size_t)(xok[x] ? s0 + x / 2 : 0) * Jstride * ctl + (x & 1) * lN + off;
+        xp[x] = baby + tiled_index(Rx, c.N, (xok[x] ? s0 + x / 2 : 0) * J * 2 + (x & 1), i, p);
     }
     auto issue = [&](uint32_t j) {
         if (j < J) {
             const uint32_t st = j % MAC_DEPTH;
 #pragma unroll
-            for (uint32_t g = 0; g < MAC_GT; g++) cp_async8(&ring[st][g][tid], wp[g] + (size_t)j * lN);
+            for (uint32_t g = 0; g < MAC_GT; g++) cp_async8(&ring[st][g][tid], wp[g] + (size_t)j * 64);
 #pragma unroll
-            for (uint32_t x = 0; x < NX; x++) cp_async8(&ring[st][MAC_GT + x][tid], xp[x] + (size_t)j * ctl);
+            for (uint32_t x = 0; x < NX; x++) cp_async8(&ring[st][MAC_GT + x][tid], xp[x] + (size_t)j * 128);
         }
         cp_async_commit();
     };
@@ -430,21 +433,28 @@ extern "C" int32_t ckks_linear_proj(ckks_ctx *c, const ckks_proj_desc *d, const 
     char *base = (char *)ws;
     const size_t ctl = (size_t)2 * level * N, ptl = (size_t)level * N;
     u64 *baby = (u64 *)(base + L.baby), *pts = (u64 *)(base + L.pts), *acc = (u64 *)(base + L.acc);
+    u64 *xin = (u64 *)(base + L.xin), *ptt = (u64 *)(base + L.ptt);
     u64 *total = (u64 *)(base + L.total), *tmp = (u64 *)(base + L.tmp), *rsw = (u64 *)(base + L.rs);
     double *slots = (double *)(base + L.slots);
     void *encw = base + L.enc;
     KsWorkspace kw = ks_carve(c, level, base + L.ks, S * nib);
 
-    // baby[(sh*nib + ib)*B + b] = rho^(b T)(x_{sh,ib}): one ModUp for all input ciphertexts at once, then every
-    // baby rotation is applied to all of them in one batch (the key is read once per rotation, not once per shard)
+    // baby row ((sh*nib + ib)*B + b)*2 + comp = component comp of rho^(b T)(x_{sh,ib}), tiled layout: one ModUp for all
+    // input ciphertexts at once, then every baby rotation is applied to all of them in one batch (the key is read
+    // once per rotation, not once per shard) and written straight into the tiled buffer
+    const uint32_t Jall = nib * B, Rx = 2 * S * Jall;
     for (uint32_t x = 0; x < S * nib; x++)
-        cudaMemcpyAsync(baby + (size_t)x * B * ctl, in[x].data, ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+        cudaMemcpyAsync(xin + (size_t)x * ctl, in[x].data, ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+    for (uint32_t comp = 0; comp < 2; comp++)
+        launch_to_tiled(c, xin + comp * ptl, ctl, S * nib, baby, Rx, comp, 2 * B, level, s);
     if (B > 1) {
-        ks_modup(c, baby + ptl, 1, level, kw, s, S * nib, (size_t)B * ctl);
+        ks_modup(c, xin + ptl, 1, level, kw, s, S * nib, ctl);
         for (uint32_t b = 1; b < B; b++) {
             const u64 ge = ckks_galois_element(c, (int64_t)b * T);
-            ks_inner_moddown(c, (const u64 *)find_key(keys, nkeys, ge)->data, level, ge, kw, baby, nullptr, ge, baby + (size_t)b * ctl, s,
-                             S * nib, (size_t)B * ctl, (size_t)B * ctl, false);
+            TiledOut to;
+            to.R = Rx; to.row0 = 2 * b; to.row_stride = 2 * B;
+            ks_inner_moddown(c, (const u64 *)find_key(keys, nkeys, ge)->data, level, ge, kw, xin, nullptr, ge, baby, s, S * nib, ctl, 0,
+                             false, to);
         }
     }
 
@@ -476,12 +486,11 @@ extern "C" int32_t ckks_linear_proj(ckks_ctx *c, const ckks_proj_desc *d, const 
                     if (ragged) launch_encode(c, slots + idx * c->n, nullptr, B, pt_scale, level, pts + idx * ptl, encw, s);
                 }
             if (!ragged) launch_encode(c, slots, nullptr, ng * J, pt_scale, level, pts, encw, s);
-            {
+            launch_to_tiled(c, pts, ptl, ng * J, ptt, ng * J, 0, 1, level, s);
+            if (!launch_mac_mma(c, baby, ptt, acc, J, S, ng, level, s)) {
                 const uint32_t stiles = (S + MAC_ST - 1) / MAC_ST, gtiles = (ng + MAC_GT - 1) / MAC_GT;
-                if (!(mac_mma_supported(c, J) && launch_mac_mma(c, baby, pts, acc, J, J, S, ng, level, s))) {
-                    mac_tile_kernel<<<dim3(stiles * gtiles, N / MAC_THREADS, level), MAC_THREADS, 0, s>>>(c->dev, baby, pts, acc, J, J, S, ng, level);
-                    count_launches();
-                }
+                mac_tile_kernel<<<dim3(stiles * gtiles, N / MAC_THREADS, level), MAC_THREADS, 0, s>>>(c->dev, baby, ptt, acc, J, S, ng, level);
+                count_launches();
             }
             for (uint32_t gl = 0; gl < ng; gl++) {
                 const uint32_t gi = g0 + gl;

@@ -156,6 +156,20 @@ __device__ __forceinline__ u64 canonical_d(double v, double q) { return d_to_u64
 
 __device__ __forceinline__ uint32_t bitrev_n(uint32_t x, uint32_t bits) { return __brev(x) >> (32 - bits); }
 
+// ---------------------------------------------------------------------------
+// "Tiled" operand layout of the projection's multiply-accumulate.  R rows (one row = one plaintext, or one
+// component of one ciphertext) of [level][N] words are stored so that, for a limb i and a block of 64
+// coefficients, all R rows are adjacent:   index(r, i, p) = (((i * N/64) + p/64) * R + r) * 64 + p % 64.
+// The multiply-accumulate walks all rows of a few coefficients; in the plain [row][level][N] layout those
+// words are 12-24 MiB apart (one TLB entry and one DRAM page per 64 bytes), here they are one 512-byte step apart.
+// ---------------------------------------------------------------------------
+__host__ __device__ inline size_t tiled_index(uint32_t R, uint32_t N, uint32_t r, uint32_t i, uint32_t p) {
+    return ((((size_t)i * (N >> 6)) + (p >> 6)) * R + r) * 64 + (p & 63);
+}
+// where a key-switch result goes when it is written straight into a tiled buffer: component c of batch entry b
+// becomes row row0 + b * row_stride + c of a buffer with R rows (R = 0: plain layout)
+struct TiledOut { uint32_t R = 0, row0 = 0, row_stride = 0; };
+
 // Kernel launches issued by this library since it was loaded (all contexts, all streams).
 extern unsigned long long g_kernel_launches;
 inline void count_launches(unsigned n = 1) { g_kernel_launches += n; }
@@ -183,12 +197,16 @@ void ks_modup(const ckks_ctx *c, const u64 *d, u64 galois, uint32_t level, const
 // combination out_c (+)= sigma_{add_galois}(add_c) + k_c.  add0/add1 may be null.
 void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext_galois, const KsWorkspace &w,
                       const u64 *add0, const u64 *add1, u64 add_galois, u64 *out, cudaStream_t s, uint32_t nb = 1,
-                      size_t add_stride = 0, size_t out_stride = 0, bool accumulate = false);
+                      size_t add_stride = 0, size_t out_stride = 0, bool accumulate = false, TiledOut tiled = TiledOut());
+// rows of [level][N] words, src_stride words apart, into rows row0, row0 + row_step, .. of a tiled buffer with R rows
+void launch_to_tiled(const ckks_ctx *c, const u64 *src, size_t src_stride, uint32_t nrows, u64 *dst, uint32_t R, uint32_t row0,
+                     uint32_t row_step, uint32_t level, cudaStream_t s);
 
 // Tensor-core multiply-accumulate of a giant-step group (mac_mma.cu)
 bool mac_mma_supported(const ckks_ctx *c, uint32_t J);
-bool launch_mac_mma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t Jstride, uint32_t S,
-                    uint32_t G, uint32_t level, cudaStream_t s);
+// baby, pts: tiled buffers with 2 * S * J rows ((shard * J + j) * 2 + component) and G * J rows (g * J + j)
+bool launch_mac_mma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level,
+                    cudaStream_t s);
 
 void launch_rescale(const ckks_ctx *c, const u64 *in, u64 *out, uint32_t ncomp, uint32_t level, u64 *ws, cudaStream_t s);
 

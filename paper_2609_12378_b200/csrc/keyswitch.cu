@@ -162,7 +162,7 @@ void launch_moddown_conv(const ckks_ctx *c, const u64 *u, u64 *conv, uint32_t le
 // out[b][comp][i][p] (+)= (u[b][comp][i][p] - conv[b][comp][i][p]) P^-1 + add_comp[b][i][pi_g(p)]
 __global__ void __launch_bounds__(THREADS) moddown_final_kernel(DevTables c, const u64 *u, const u64 *conv, const u64 *add0,
                                                                 const u64 *add1, size_t add_stride, u64 g, u64 *out,
-                                                                size_t out_stride, int accumulate, uint32_t level) {
+                                                                size_t out_stride, int accumulate, uint32_t level, TiledOut tl) {
     const uint32_t p = blockIdx.x * THREADS + threadIdx.x;
     const uint32_t i = blockIdx.y, comp = blockIdx.z & 1, bz = blockIdx.z >> 1;
     const uint32_t nt = level + c.K;
@@ -172,9 +172,18 @@ __global__ void __launch_bounds__(THREADS) moddown_final_kernel(DevTables c, con
     r = mul_shoup(r, pinv.x, pinv.y, q);
     const u64 *add = comp ? add1 : add0;
     if (add) r = add_mod(r, add[bz * add_stride + (size_t)i * c.N + galois_src(p, g, c.log_n, c.N)], q);
-    u64 *dst = out + bz * out_stride + ((size_t)comp * level + i) * c.N + p;
+    u64 *dst = tl.R ? out + tiled_index(tl.R, c.N, tl.row0 + bz * tl.row_stride + comp, i, p)
+                    : out + bz * out_stride + ((size_t)comp * level + i) * c.N + p;
     if (accumulate) r = add_mod(r, *dst, q);
     *dst = r;
+}
+
+// dst row (row0 + r * row_step) of a tiled buffer <- src + r * src_stride ([level][N] words)
+__global__ void __launch_bounds__(THREADS) to_tiled_kernel(DevTables c, const u64 *src, size_t src_stride, u64 *dst, uint32_t R,
+                                                           uint32_t row0, uint32_t row_step) {
+    const uint32_t p = (blockIdx.x * THREADS + threadIdx.x) * 2, i = blockIdx.y, r = blockIdx.z;
+    const ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(src + r * src_stride + (size_t)i * c.N + p);
+    *reinterpret_cast<ulonglong2 *>(dst + tiled_index(R, c.N, row0 + r * row_step, i, p)) = v;
 }
 
 // tmp[comp][i][k] = centred lift of last[comp][k] (mod q_last) taken mod q_i
@@ -226,7 +235,7 @@ void ks_modup(const ckks_ctx *c, const u64 *d, u64 galois, uint32_t level, const
 
 void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext_galois, const KsWorkspace &w,
                       const u64 *add0, const u64 *add1, u64 add_galois, u64 *out, cudaStream_t s, uint32_t nb,
-                      size_t add_stride, size_t out_stride, bool accumulate) {
+                      size_t add_stride, size_t out_stride, bool accumulate, TiledOut tiled) {
     const uint32_t N = c->N, nt = level + c->K, K = c->K;
     inner_product_kernel<<<dim3(N / THREADS, nb, nt), THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level); count_launches();
     // the K special limbs of every (batch, component): groups of K limbs, nt limbs apart
@@ -236,8 +245,18 @@ void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext
 #undef CALL_DN
     launch_ntt(c, w.conv, nb * 2 * level, plain_map(0, level), false, s);
     moddown_final_kernel<<<dim3(N / THREADS, level, 2 * nb), THREADS, 0, s>>>(c->dev, w.u, w.conv, add0, add1, add_stride, add_galois, out,
-                                                                               out_stride, accumulate ? 1 : 0, level);
+                                                                               out_stride, accumulate ? 1 : 0, level, tiled);
     count_launches();
+}
+
+void launch_to_tiled(const ckks_ctx *c, const u64 *src, size_t src_stride, uint32_t nrows, u64 *dst, uint32_t R, uint32_t row0,
+                     uint32_t row_step, uint32_t level, cudaStream_t s) {
+    for (uint32_t r0 = 0; r0 < nrows; r0 += 32768) {
+        const uint32_t nr = nrows - r0 < 32768 ? nrows - r0 : 32768;
+        to_tiled_kernel<<<dim3(c->N / (2 * THREADS), level, nr), THREADS, 0, s>>>(c->dev, src + r0 * src_stride, src_stride, dst, R,
+                                                                                   row0 + r0 * row_step, row_step);
+        count_launches();
+    }
 }
 
 // ws: [ncomp][N] last limbs + [ncomp][level-1][N]

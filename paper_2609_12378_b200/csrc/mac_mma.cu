@@ -9,7 +9,9 @@
 //
 // Mapping.  A warp owns one coefficient: M = 16 giants, N = 16 columns s' (two n-tiles), K = 32 values of j
 // per step.  A CTA (8 warps) owns 8 adjacent coefficients, so a row of operands (one (g, j) or (s', j) pair) is
-// 64 contiguous bytes in HBM, fetched as four 16-byte cp.async.cg chunks into a 3-deep ring.  Rows are stored
+// 64 contiguous bytes; both operand arrays are in the tiled layout (all rows of a 64-coefficient block adjacent, see
+// tiled_index), so the 1024 rows of a step are 512 bytes apart.  A row is fetched as four 16-byte cp.async.cg
+// chunks into a 3-deep ring.  Rows are stored
 // [g or s'][j][8 coefficients] with a pitch of 2112 bytes per g and the 16-byte chunks of a row XOR-swizzled
 // by (j / 4) mod 4, which brings the fragment reads (same coefficient, rows gid and 4 tig + e) down to a
 // two-way bank conflict.  CTAs are persistent and walk tiles (column tile fastest, then coefficient block,
@@ -62,8 +64,8 @@ __device__ __forceinline__ u64 tile_word(const uint8_t *tile, uint32_t a, uint32
 }
 
 __global__ void __launch_bounds__(256, 1) mac_mma_kernel(DevTables c, const u64 *__restrict__ baby, const u64 *__restrict__ pts,
-                                                         u64 *__restrict__ acc, uint32_t J, uint32_t Jstride, uint32_t S, uint32_t G,
-                                                         uint32_t level, uint32_t ntiles) {
+                                                         u64 *__restrict__ acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level,
+                                                         uint32_t ntiles) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *ring = reinterpret_cast<uint8_t *>(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, gid = lane >> 2, tig = lane & 3;
@@ -74,7 +76,7 @@ __global__ void __launch_bounds__(256, 1) mac_mma_kernel(DevTables c, const u64 
     const uint32_t my_tiles = blockIdx.x < ntiles ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
     const uint32_t nsteps = my_tiles * nk;
 
-    struct Tile { uint32_t col0, g0, off; };
+    struct Tile { uint32_t col0, g0, off, i, xb; };
     auto decode = [&](uint32_t t) {
         const uint32_t tile = blockIdx.x + t * gridDim.x;
         const uint32_t z = tile % ztiles, rest = tile / ztiles, xb = rest % xblocks, i = rest / xblocks;
@@ -82,30 +84,33 @@ __global__ void __launch_bounds__(256, 1) mac_mma_kernel(DevTables c, const u64 
         r.col0 = (z % coltiles) * MS;
         r.g0 = (z / coltiles) * MG;
         r.off = i * c.N + xb * COEF;          // position inside the [level][N] plane, < 2^32
+        r.i = i;
+        r.xb = xb;
         return r;
     };
     // loader: a thread always fetches the 16-byte chunk ch = tid & 3 of row j = 32 ks + (tid >> 3) and walks
     // blocks a = (tid >> 2 & 1) + 2 it of W and of X, so every address is a base plus a constant stride
     const uint32_t ch = tid & 3, ah = (tid >> 2) & 1, jj = tid >> 3;
-    const size_t wstride = (size_t)Jstride * lN, xstride = (size_t)Jstride * ctl;
+    const uint32_t Rw = G * J, Rx = 2 * S * J;
     auto issue = [&](uint32_t step) {
         if (step < nsteps) {
             const Tile tl = decode(step / nk);
             const uint32_t j = (step % nk) * MK + jj;
             uint8_t *st = ring + (size_t)(step % STAGES) * STAGE_BYTES;
-            const u64 *wb = pts + (size_t)j * lN + tl.off + 2 * ch;
-            const u64 *xb = baby + (size_t)j * ctl + tl.off + 2 * ch;
+            // tiled_index(R, N, r, i, p) = blk * R * 64 + r * 64 + p % 64, blk = i * N/64 + p/64
+            const size_t blk = (size_t)tl.i * (c.N >> 6) + (tl.xb >> 3);
+            const u64 *wb = pts + blk * Rw * 64 + (tl.xb & 7) * 8 + 2 * ch;
+            const u64 *xb = baby + blk * Rx * 64 + (tl.xb & 7) * 8 + 2 * ch;
             const uint32_t gleft = G - tl.g0, cleft = ncol - tl.col0;      // valid giants / columns in this tile
 #pragma unroll
             for (uint32_t it = 0; it < MG / 2; it++) {
                 const uint32_t a = 2 * it + ah;
-                cp_async16(st + tile_off(a, jj, ch), wb + (a < gleft ? (size_t)(tl.g0 + a) * wstride : 0));
+                cp_async16(st + tile_off(a, jj, ch), wb + (size_t)((a < gleft ? tl.g0 + a : 0) * J + j) * 64);
             }
 #pragma unroll
             for (uint32_t it = 0; it < MS / 2; it++) {
-                const uint32_t a = 2 * it + ah;
-                cp_async16(st + BOX_BYTES + tile_off(a, jj, ch),
-                           xb + (a < cleft ? (size_t)((tl.col0 + a) >> 1) * xstride + (a & 1) * lN : 0));
+                const uint32_t a = 2 * it + ah, col = a < cleft ? tl.col0 + a : 0;
+                cp_async16(st + BOX_BYTES + tile_off(a, jj, ch), xb + (size_t)(((col >> 1) * J + j) * 2 + (col & 1)) * 64);
             }
         }
         cp_commit();
@@ -179,10 +184,10 @@ __global__ void __launch_bounds__(256, 1) mac_mma_kernel(DevTables c, const u64 
 
 bool mac_mma_supported(const ckks_ctx *c, uint32_t J) { return J % MK == 0 && J > 0 && c->N % COEF == 0; }
 
-// acc[g][s][c][i][p] = sum_{j < J} baby[s][j][c][i][p] * pts[g][j][i][p];  baby rows are Jstride ciphertexts apart per
-// shard, pts rows Jstride plaintexts apart per giant step.  Returns false if nothing was launched.
-bool launch_mac_mma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t Jstride, uint32_t S,
-                    uint32_t G, uint32_t level, cudaStream_t s) {
+// acc[g][s][c][i][p] = sum_{j < J} baby[s][j][c][i][p] * pts[g][j][i][p] with baby and pts in the tiled layout
+// (rows (s J + j) 2 + c and g J + j); acc in the plain layout.  Returns false if nothing was launched.
+bool launch_mac_mma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level,
+                    cudaStream_t s) {
     if (!mac_mma_supported(c, J)) return false;
     static bool attr_set = false;
     if (!attr_set) {
@@ -193,7 +198,7 @@ bool launch_mac_mma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc
     const uint32_t ntiles = (c->N / COEF) * level * coltiles * gt;
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
-    mac_mma_kernel<<<ntiles < (uint32_t)sms ? ntiles : (uint32_t)sms, 256, SMEM_BYTES, s>>>(c->dev, baby, pts, acc, J, Jstride, S, G, level, ntiles);
+    mac_mma_kernel<<<ntiles < (uint32_t)sms ? ntiles : (uint32_t)sms, 256, SMEM_BYTES, s>>>(c->dev, baby, pts, acc, J, S, G, level, ntiles);
     count_launches();
     return true;
 }
