@@ -285,10 +285,26 @@ def run_cuda(args):
 
     pk, pk_kind = peaks()
     limb_ntts = NTT_BATCH * L
-    ntt_bytes = limb_ntts * 2 * 8 * N          # algorithmic: each limb read once and written once
-    achieved = ntt_bytes / (ntt_fwd_ms * 1e-3) / 1e9
-    roofline = {"kernel": "ntt_cols+ntt_rows (forward NTT of 768 limbs)", "bound": "hbm", "achieved": achieved,
-                "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": achieved / pk["hbm_gbs"], "traffic": None, "peak_kind": pk_kind}
+    # Roofline of the dominant kernel family (the four ntt16 kernels: 36 % of the step in the ncu launch list).
+    # The butterflies run on the FP64 pipe, which ncu shows to be the busiest unit of the column passes, so the
+    # bound is "alu": algorithmic work = 8 FP64 instructions per butterfly (6 for the exact twiddle product with
+    # its quotient, 2 for the sum and difference), N/2 * log2 N butterflies per limb; peak = 64 FP64 instructions
+    # per clock per SM (the DFMA rate ncu reports for this part) x SM count x the maximum SM clock.
+    sm_count = torch.cuda.get_device_properties(local).multi_processor_count
+    fp64_peak = 64.0 * sm_count * float(pk.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12          # T instr/s
+    ops = limb_ntts * (N // 2) * LOG_N * 8
+    achieved = ops / (ntt_fwd_ms * 1e-3) / 1e12
+    ntt_bytes = limb_ntts * 2 * 8 * N          # algorithmic bytes: each limb read once and written once
+    hbm_achieved = ntt_bytes / (ntt_fwd_ms * 1e-3) / 1e9
+    roofline = {"kernel": "ntt16_fwd_cols + ntt16_fwd_rows (forward NTT of 768 limbs, one launch each)", "bound": "alu",
+                "achieved": achieved, "peak": fp64_peak, "unit": "T FP64 instr/s", "frac": achieved / fp64_peak,
+                "traffic": 1574.0e6,   # ncu: dram read+write of the two launches (profiles/ntt16_768limbs.md), bytes
+                "peak_kind": "derived: 64 DFMA/clk/SM x %d SMs x %.0f MHz" % (sm_count, float(pk.get("sm_max_mhz", 1965.0))),
+                "ms_per_launch_pair": ntt_fwd_ms,
+                "hbm": {"achieved": hbm_achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": hbm_achieved / pk["hbm_gbs"],
+                        "algorithmic_bytes": ntt_bytes, "peak_kind": pk_kind + " copy bandwidth"},
+                "others": {"mac_mma_kernel": "19.5 % of the step; legacy mma.sync issue bound, see profiles/mac_mma_projection_8shards.md",
+                           "inner_product_kernel": "12.9 % of the step; HBM bound (key stream)"}}
     cpu = oracle_sample()
     line = {
         "metric": METRIC, "value": c_ms * 1e-3 / world, "unit": "s/projection", "n_gpus": world, "steps": args.steps,

@@ -29,7 +29,7 @@ __global__ void __launch_bounds__(THREADS) permute_kernel(DevTables c, const u64
     dst[blockIdx.z * dst_stride + row + p] = src[blockIdx.z * src_stride + row + galois_src(p, g, c.log_n, c.N)];
 }
 
-constexpr uint32_t CHUNK = 8;   // targets per CTA row in the basis-conversion kernels
+constexpr uint32_t CHUNK = 32;  // targets per CTA row in the basis-conversion kernels (source limbs are re-read once per chunk)
 
 // ext[j][x][k] for x over q_0..q_{level-1}, p_0..p_{K-1}.  dcoef: sigma_g(d) in the coefficient domain;
 // deval: d in the evaluation domain, read through sigma_g for the digit's own limbs.
