@@ -200,6 +200,25 @@ int32_t ckks_rotate_hoisted(ckks_ctx *ctx, const ckks_ct *in, const ckks_evk *ke
  * == 1; otherwise it must not overlap.  Errors: ARG, LEVEL (level < 2), WORKSPACE. */
 int32_t ckks_rescale(ckks_ctx *ctx, const ckks_ct *in, ckks_ct *out, void *ws, size_t ws_bytes, void *stream);
 
+/* ---- Rescale with built-in scratch ---------------------------------------------
+ * (No counterpart in the paper: an addition for callers that cannot allocate.)
+ * Same result as ckks_rescale, bit for bit, but needs no workspace argument and allocates nothing: its scratch
+ * is a fixed array of CKKS_STATIC_SCRATCH_BYTES inside the library image, present on every GPU that loads the
+ * library until the process exits.  Meant for callers that have no way to get device memory when the call is
+ * made -- inside a stream capture, behind a frozen memory pool, or in an application that only lends this
+ * library fixed buffers.
+ *   - in, out: as for ckks_rescale (host descriptors, device data; out must not overlap in unless ncomp == 1).
+ *   - Inputs with ncomp * level * N * 8 > CKKS_STATIC_SCRATCH_BYTES are refused with CKKS_ERR_WORKSPACE (the
+ *     reason is readable through ckks_last_cuda_error); use ckks_rescale for those.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress); make that first
+ *     call outside any stream capture.  Later calls only launch kernels.
+ *   - All calls on a device share the one array and it keeps the previous call's contents.  Nothing in it needs
+ *     clearing between calls, but two calls whose kernels can overlap on the GPU (different streams without an
+ *     ordering between them) race on it: serialise them.
+ * Errors: ARG, LEVEL, WORKSPACE (too large), UNSUPPORTED (device ordinal >= 64), CUDA. */
+#define CKKS_STATIC_SCRATCH_BYTES (8u << 20)
+int32_t ckks_rescale_static(ckks_ctx *ctx, const ckks_ct *in, ckks_ct *out, void *stream);
+
 /* ---- Linear projection (Eq. 5, baby-step/giant-step) -----------------------
  * in: host array of nshards * n_in_blocks descriptors (index shard * n_in_blocks
  * + block), all at one level and scale.  W: device, row-major [d_in][d_out]

@@ -21,7 +21,7 @@ EXPORTS = [
     "ckks_workspace_bytes", "ckks_galois_element", "ckks_ntt", "ckks_intt", "ckks_encode",
     "ckks_encode_range_flag", "ckks_mul_plain_acc", "ckks_add", "ckks_mul_relin", "ckks_rotate",
     "ckks_rotate_hoisted", "ckks_rescale", "ckks_linear_proj", "ckks_linear_proj_workspace_bytes",
-    "ckks_linear_proj_rotations", "ckks_kernel_launches", "ckks_device_status",
+    "ckks_linear_proj_rotations", "ckks_kernel_launches", "ckks_device_status", "ckks_rescale_static",
 ]
 
 
@@ -78,6 +78,7 @@ def load():
         "ckks_rotate": (i32, [vp, C.POINTER(CCt), C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
         "ckks_rotate_hoisted": (i32, [vp, C.POINTER(CCt), C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
         "ckks_rescale": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), vp, sz, vp]),
+        "ckks_rescale_static": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), vp]),
         "ckks_linear_proj": (i32, [vp, C.POINTER(CProjDesc), C.POINTER(CCt), vp, C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
         "ckks_linear_proj_workspace_bytes": (sz, [vp, C.POINTER(CProjDesc), u32]),
         "ckks_linear_proj_rotations": (i32, [vp, C.POINTER(CProjDesc), C.POINTER(i64), u32]),
