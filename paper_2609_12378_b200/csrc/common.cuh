@@ -26,8 +26,9 @@ struct DevTables {
     const ulonglong2 *tw_fwd;  // [T][N] {psi^bitrev(i), Shoup companion}, index m+i
     const ulonglong2 *tw_inv;  // [T][N] inverses of the same
     const ulonglong2 *n_inv;   // [T] {N^-1, Shoup}
-    // fp64 copies for the double-precision NTT path (N = 2^16 only): {w, w/q} as doubles, same indexing
-    const double2 *twd_fwd, *twd_inv;   // [T][N]
+    // fp64 copies for the double-precision NTT path (N = 2^16 only): w as a double, same indexing (w/q is formed
+    // in the kernel as w * (1/q): half the table bytes for one extra multiply per twiddle)
+    const double *twd_fwd, *twd_inv;    // [T][N]
     const double2 *n_inv_d;             // [T] {N^-1, N^-1/q}
     // ModUp, per level l (1..L), digit j, source a < alpha:
     const ulonglong2 *up_hat_inv;  // [(L+1)][dnum][alpha]        {qhat^-1 mod q_src, Shoup}

@@ -159,7 +159,8 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
     std::vector<double2> modd(T);
     std::vector<ulonglong2> ninv(T), twf((size_t)T * N), twi((size_t)T * N);
     const bool fp = prm->log_n == 16;
-    std::vector<double2> twdf(fp ? (size_t)T * N : 0), twdi(fp ? (size_t)T * N : 0), ninvd(T);
+    std::vector<double> twdf(fp ? (size_t)T * N : 0), twdi(fp ? (size_t)T * N : 0);
+    std::vector<double2> ninvd(T);
     for (uint32_t t = 0; t < T; t++) {
         u64 m = mod[t];
         mu[t] = (u64)((((u128)1) << 112) / m);
@@ -176,8 +177,8 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
             twf[(size_t)t * N + i] = h_pair(pw[r], m);
             twi[(size_t)t * N + i] = h_pair(pwi[r], m);
             if (fp) {
-                twdf[(size_t)t * N + i] = make_double2((double)pw[r], (double)pw[r] / (double)m);
-                twdi[(size_t)t * N + i] = make_double2((double)pwi[r], (double)pwi[r] / (double)m);
+                twdf[(size_t)t * N + i] = (double)pw[r];
+                twdi[(size_t)t * N + i] = (double)pwi[r];
             }
         }
     }

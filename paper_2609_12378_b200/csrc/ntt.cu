@@ -190,59 +190,89 @@ __device__ __forceinline__ u64 reduce_exact(u64 x, u64 q, u64 qinv64) {
 // intermediate written between the passes is a lazy word in one case and a double
 // in the other); the result is the same canonical residue either way.
 // ---------------------------------------------------------------------------
+// ML consecutive twiddles w (ML = 1, 2, 4, 8; the index is a multiple of ML) with the widest loads that fit, each
+// completed to {w, w * (1/q)}.  w * fl(1/q) is within 2^-52 relative of w/q, which the stage bounds allow for.
+template <uint32_t ML>
+__device__ __forceinline__ void load_tw(const double *p, double qinv, double2 (&w)[ML]) {
+    double v[ML];
+    if (ML == 1) v[0] = __ldg(p);
+    if (ML == 2) asm volatile("ld.global.nc.v2.f64 {%0,%1}, [%2];" : "=d"(v[0]), "=d"(v[1]) : "l"(p));
+    if (ML >= 4) {
+#pragma unroll
+        for (uint32_t i = 0; i < ML; i += 4)
+            asm volatile("ld.global.nc.v4.f64 {%0,%1,%2,%3}, [%4];" : "=d"(v[i]), "=d"(v[(i + 1) % ML]), "=d"(v[(i + 2) % ML]), "=d"(v[(i + 3) % ML]) : "l"(p + i));
+    }
+#pragma unroll
+    for (uint32_t i = 0; i < ML; i++) w[i] = make_double2(v[i], __dmul_rn(v[i], qinv));
+}
+__device__ __forceinline__ void stg_4(u64 *p, u64 a, u64 b, u64 c, u64 d) {
+    asm volatile("st.global.v4.b64 [%0], {%1,%2,%3,%4};" ::"l"(p), "l"(a), "l"(b), "l"(c), "l"(d) : "memory");
+}
+__device__ __forceinline__ void ldg_4(const u64 *p, u64 &a, u64 &b, u64 &c, u64 &d) {
+    asm volatile("ld.global.v4.b64 {%0,%1,%2,%3}, [%4];" : "=l"(a), "=l"(b), "=l"(c), "=l"(d) : "l"(p) : "memory");
+}
+
 // 4 Cooley-Tukey stages; inputs of any magnitude below 2^53 (reduced first), outputs below 4.6 q.
-__device__ __forceinline__ void fwd16_d(double (&x)[16], const double2 *__restrict__ tw, uint32_t base, double q, double qinv) {
+template <uint32_t ML>
+__device__ __forceinline__ void fwd_stage_d(double (&x)[16], const double *__restrict__ tw, uint32_t base, double q, double qinv) {
+    constexpr uint32_t tl = 8 / ML;
+    double2 w[ML];
+    load_tw<ML>(tw + ML * base, qinv, w);
+#pragma unroll
+    for (uint32_t i = 0; i < ML; i++)
+#pragma unroll
+        for (uint32_t j = 0; j < tl; j++) {
+            const uint32_t k1 = 2 * i * tl + j, k2 = k1 + tl;
+            // bounds entering the stages: 0.5, 1.13, 1.9, 2.9 (times q): only the last needs the coarse rounding
+            const double t = ML == 8 ? mulmod_d<1>(x[k2], w[i], q) : mulmod_d<0>(x[k2], w[i], q);
+            x[k2] = __dsub_rn(x[k1], t);
+            x[k1] = __dadd_rn(x[k1], t);
+        }
+}
+__device__ __forceinline__ void fwd16_d(double (&x)[16], const double *__restrict__ tw, uint32_t base, double q, double qinv) {
 #pragma unroll
     for (uint32_t k = 0; k < 16; k++) x[k] = reduce_d(x[k], q, qinv);
-#pragma unroll
-    for (uint32_t ml = 1; ml < 16; ml <<= 1) {
-        const uint32_t tl = 8 / ml;
-#pragma unroll
-        for (uint32_t i = 0; i < ml; i++) {
-            const double2 w = __ldg(&tw[ml * base + i]);
-#pragma unroll
-            for (uint32_t j = 0; j < tl; j++) {
-                const uint32_t k1 = 2 * i * tl + j, k2 = k1 + tl;
-                // bounds entering the stages: 0.5, 1.13, 1.9, 2.9 (times q): only the last needs the coarse rounding
-                const double t = ml == 8 ? mulmod_d<1>(x[k2], w, q) : mulmod_d<0>(x[k2], w, q);
-                x[k2] = __dsub_rn(x[k1], t);
-                x[k1] = __dadd_rn(x[k1], t);
-            }
-        }
-    }
+    fwd_stage_d<1>(x, tw, base, q, qinv);
+    fwd_stage_d<2>(x, tw, base, q, qinv);
+    fwd_stage_d<4>(x, tw, base, q, qinv);
+    fwd_stage_d<8>(x, tw, base, q, qinv);
 }
 
 // 4 Gentleman-Sande stages; reduced at the start and after two stages; outputs below 2 q.
-__device__ __forceinline__ void inv16_d(double (&x)[16], const double2 *__restrict__ tw, uint32_t base, double q, double qinv) {
+template <uint32_t ML>
+__device__ __forceinline__ void inv_stage_d(double (&x)[16], const double *__restrict__ tw, uint32_t base, double q, double qinv) {
+    constexpr uint32_t tl = 8 / ML;
+    double2 w[ML];
+    load_tw<ML>(tw + ML * base, qinv, w);
 #pragma unroll
-    for (uint32_t ml = 8; ml >= 1; ml >>= 1) {
-        const uint32_t tl = 8 / ml;
-        if (ml == 8 || ml == 2) {
+    for (uint32_t i = 0; i < ML; i++)
 #pragma unroll
-            for (uint32_t k = 0; k < 16; k++) x[k] = reduce_d(x[k], q, qinv);
+        for (uint32_t j = 0; j < tl; j++) {
+            const uint32_t k1 = 2 * i * tl + j, k2 = k1 + tl;
+            const double u = x[k1], v = x[k2];
+            x[k1] = __dadd_rn(u, v);
+            x[k2] = mulmod_d<0>(__dsub_rn(u, v), w[i], q);     // |u - v| <= 2q < 2^51
         }
+}
+__device__ __forceinline__ void inv16_d(double (&x)[16], const double *__restrict__ tw, uint32_t base, double q, double qinv) {
 #pragma unroll
-        for (uint32_t i = 0; i < ml; i++) {
-            const double2 w = __ldg(&tw[ml * base + i]);
+    for (uint32_t k = 0; k < 16; k++) x[k] = reduce_d(x[k], q, qinv);
+    inv_stage_d<8>(x, tw, base, q, qinv);
+    inv_stage_d<4>(x, tw, base, q, qinv);
 #pragma unroll
-            for (uint32_t j = 0; j < tl; j++) {
-                const uint32_t k1 = 2 * i * tl + j, k2 = k1 + tl;
-                const double u = x[k1], v = x[k2];
-                x[k1] = __dadd_rn(u, v);
-                x[k2] = mulmod_d<0>(__dsub_rn(u, v), w, q);     // |u - v| <= 2q < 2^51
-            }
-        }
-    }
+    for (uint32_t k = 0; k < 16; k++) x[k] = reduce_d(x[k], q, qinv);
+    inv_stage_d<2>(x, tw, base, q, qinv);
+    inv_stage_d<1>(x, tw, base, q, qinv);
 }
 
 // ---- forward, column pass (stages m = 1..128): CTA = strip of 16 columns -----------------
-__global__ void __launch_bounds__(F_THREADS) ntt16_fwd_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
+__global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
     __shared__ u64 sm[256 * 16];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
     if ((blockIdx.y & 7) < fp_share) {
         const double q = c.modd[prime].x, qinv = c.modd[prime].y;
-        const double2 *tw = c.twd_fwd + ((size_t)prime << 16);
+        const double *tw = c.twd_fwd + ((size_t)prime << 16);
         const uint32_t cc = threadIdx.x & 15, r = threadIdx.x >> 4;
         u64 *g = base + (limb_index(map, blockIdx.y) << 16) + blockIdx.x * 16 + cc;
         double *smd = reinterpret_cast<double *>(sm);
@@ -283,13 +313,13 @@ __device__ __forceinline__ uint32_t padded(uint32_t i) { return i + (i >> 4); }
 constexpr uint32_t ROW_PAD = 256 + 16;
 
 // ---- forward, row pass (stages m = 256..32768): CTA = 16 rows, 16 threads per row ---------
-__global__ void __launch_bounds__(F_THREADS) ntt16_fwd_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
+__global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
     __shared__ u64 sm[16 * ROW_PAD];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
     if ((blockIdx.y & 7) < fp_share) {
         const double q = c.modd[prime].x, qinv = c.modd[prime].y;
-        const double2 *tw = c.twd_fwd + ((size_t)prime << 16);
+        const double *tw = c.twd_fwd + ((size_t)prime << 16);
         const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
         u64 *g = base + (limb_index(map, blockIdx.y) << 16) + (size_t)row * 256;
         double *s = reinterpret_cast<double *>(sm) + rl * ROW_PAD;
@@ -303,13 +333,11 @@ __global__ void __launch_bounds__(F_THREADS) ntt16_fwd_rows(DevTables c, u64 *ba
 #pragma unroll
         for (uint32_t k = 0; k < 16; k++) x[k] = s[padded(16 * t + k)];
         fwd16_d(x, tw, 16 * (256 + row) + t, q, qinv);
-        __syncwarp();
-        u64 *su = reinterpret_cast<u64 *>(s);
+        // a thread ends up with 16 consecutive coefficients: four 32-byte stores, each a full sector
 #pragma unroll
-        for (uint32_t k = 0; k < 16; k++) su[padded(16 * t + k)] = canonical_d(reduce_d(x[k], q, qinv), q);
-        __syncwarp();
-#pragma unroll
-        for (uint32_t k = 0; k < 16; k++) g[t + 16 * k] = su[padded(t + 16 * k)];
+        for (uint32_t k = 0; k < 16; k += 4)
+            stg_4(g + 16 * t + k, canonical_d(reduce_d(x[k], q, qinv), q), canonical_d(reduce_d(x[k + 1], q, qinv), q),
+                  canonical_d(reduce_d(x[k + 2], q, qinv), q), canonical_d(reduce_d(x[k + 3], q, qinv), q));
         return;
     }
     const u64 q = c.mod[prime], q5 = 5 * q;
@@ -337,24 +365,24 @@ __global__ void __launch_bounds__(F_THREADS) ntt16_fwd_rows(DevTables c, u64 *ba
 }
 
 // ---- inverse, row pass (stages m = 32768..256) ---------------------------------------------
-__global__ void __launch_bounds__(F_THREADS) ntt16_inv_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
+__global__ void __launch_bounds__(F_THREADS, 4) ntt16_inv_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
     __shared__ u64 sm[16 * ROW_PAD];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
     if ((blockIdx.y & 7) < fp_share) {
         const double q = c.modd[prime].x, qinv = c.modd[prime].y;
-        const double2 *tw = c.twd_inv + ((size_t)prime << 16);
+        const double *tw = c.twd_inv + ((size_t)prime << 16);
         const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
         u64 *g = base + (limb_index(map, blockIdx.y) << 16) + (size_t)row * 256;
         double *s = reinterpret_cast<double *>(sm) + rl * ROW_PAD;
         double x[16];
 #pragma unroll
-        for (uint32_t k = 0; k < 16; k++) s[padded(t + 16 * k)] = u64_to_d(g[t + 16 * k]);
-        __syncwarp();
-#pragma unroll
-        for (uint32_t k = 0; k < 16; k++) x[k] = s[padded(16 * t + k)];
+        for (uint32_t k = 0; k < 16; k += 4) {      // 16 consecutive coefficients per thread, four 32-byte loads
+            u64 a, b, cc, d;
+            ldg_4(g + 16 * t + k, a, b, cc, d);
+            x[k] = u64_to_d(a); x[k + 1] = u64_to_d(b); x[k + 2] = u64_to_d(cc); x[k + 3] = u64_to_d(d);
+        }
         inv16_d(x, tw, 16 * (256 + row) + t, q, qinv);
-        __syncwarp();
 #pragma unroll
         for (uint32_t k = 0; k < 16; k++) s[padded(16 * t + k)] = x[k];
         __syncwarp();
@@ -390,13 +418,13 @@ __global__ void __launch_bounds__(F_THREADS) ntt16_inv_rows(DevTables c, u64 *ba
 }
 
 // ---- inverse, column pass (stages m = 128..1), then N^-1 and the exact reduction -----------
-__global__ void __launch_bounds__(F_THREADS) ntt16_inv_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
+__global__ void __launch_bounds__(F_THREADS, 4) ntt16_inv_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
     __shared__ u64 sm[256 * 16];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
     if ((blockIdx.y & 7) < fp_share) {
         const double q = c.modd[prime].x, qinv = c.modd[prime].y;
-        const double2 *tw = c.twd_inv + ((size_t)prime << 16);
+        const double *tw = c.twd_inv + ((size_t)prime << 16);
         const uint32_t cc = threadIdx.x & 15, r = threadIdx.x >> 4;
         u64 *g = base + (limb_index(map, blockIdx.y) << 16) + blockIdx.x * 16 + cc;
         double *smd = reinterpret_cast<double *>(sm);
