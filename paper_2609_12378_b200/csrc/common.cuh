@@ -60,6 +60,20 @@ struct ckks_ctx {
 };
 
 // ---------------------------------------------------------------------------
+// "Tiled" operand layout of the projection's multiply-accumulate.  R rows (one row = one plaintext, or one
+// component of one ciphertext) of [level][N] words are stored so that, for a limb i and a block of 64
+// coefficients, all R rows are adjacent:   index(r, i, p) = (((i * N/64) + p/64) * R + r) * 64 + p % 64.
+// The multiply-accumulate walks all rows of a few coefficients; in the plain [row][level][N] layout those
+// words are 12-24 MiB apart (one TLB entry and one DRAM page per 64 bytes), here they are one 512-byte step apart.
+// ---------------------------------------------------------------------------
+__host__ __device__ inline size_t tiled_index(uint32_t R, uint32_t N, uint32_t r, uint32_t i, uint32_t p) {
+    return ((((size_t)i * (N >> 6)) + (p >> 6)) * R + r) * 64 + (p & 63);
+}
+// where a key-switch result goes when it is written straight into a tiled buffer: component c of batch entry b
+// becomes row row0 + b * row_stride + c of a buffer with R rows (R = 0: plain layout)
+struct TiledOut { uint32_t R = 0, row0 = 0, row_stride = 0; };
+
+// ---------------------------------------------------------------------------
 // Limb addressing for batched limb-wise kernels (NTT): limb y of a buffer
 // [..][period][N] -> prime index, or -1 to skip the limb.
 //   kind 0: prime = first + y % period
@@ -156,20 +170,12 @@ __device__ __forceinline__ u64 d_to_u64(double v) { return (u64)__double_as_long
 __device__ __forceinline__ u64 canonical_d(double v, double q) { return d_to_u64(v < 0.0 ? __dadd_rn(v, q) : v); }
 
 __device__ __forceinline__ uint32_t bitrev_n(uint32_t x, uint32_t bits) { return __brev(x) >> (32 - bits); }
-
-// ---------------------------------------------------------------------------
-// "Tiled" operand layout of the projection's multiply-accumulate.  R rows (one row = one plaintext, or one
-// component of one ciphertext) of [level][N] words are stored so that, for a limb i and a block of 64
-// coefficients, all R rows are adjacent:   index(r, i, p) = (((i * N/64) + p/64) * R + r) * 64 + p % 64.
-// The multiply-accumulate walks all rows of a few coefficients; in the plain [row][level][N] layout those
-// words are 12-24 MiB apart (one TLB entry and one DRAM page per 64 bytes), here they are one 512-byte step apart.
-// ---------------------------------------------------------------------------
-__host__ __device__ inline size_t tiled_index(uint32_t R, uint32_t N, uint32_t r, uint32_t i, uint32_t p) {
-    return ((((size_t)i * (N >> 6)) + (p >> 6)) * R + r) * 64 + (p & 63);
+// index p' with stored[p] of sigma_g(a) = stored[p'] of a (evaluation domain, bit-reversed); g = 1: identity
+__device__ __forceinline__ uint32_t galois_src(uint32_t p, u64 g, uint32_t log_n, uint32_t N) {
+    if (g == 1) return p;
+    const u64 e = (g * (2ull * bitrev_n(p, log_n) + 1)) & (2ull * N - 1);
+    return bitrev_n((uint32_t)((e - 1) >> 1), log_n);
 }
-// where a key-switch result goes when it is written straight into a tiled buffer: component c of batch entry b
-// becomes row row0 + b * row_stride + c of a buffer with R rows (R = 0: plain layout)
-struct TiledOut { uint32_t R = 0, row0 = 0, row_stride = 0; };
 
 // Kernel launches issued by this library since it was loaded (all contexts, all streams).
 extern unsigned long long g_kernel_launches;
@@ -178,7 +184,20 @@ inline void count_launches(unsigned n = 1) { g_kernel_launches += n; }
 // ---------------------------------------------------------------------------
 // Internal launchers (each validates nothing; the C ABI layer does).
 // ---------------------------------------------------------------------------
-void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbMap &map, bool inverse, cudaStream_t s);
+// Optional epilogue of the forward transform (N = 2^16 path): instead of storing NTT(conv) the last pass finishes the
+// ModDown: out[b][comp][i][p] (+)= (u[b][comp][i][p] - NTT(conv)[p]) P^-1 + sigma_g(add_comp)[b][i][p], for a buffer of
+// limbs laid out [b][comp][level]; `out` in the plain layout (out_stride words per b) or tiled (tl.R != 0).
+struct NttEpilogue {
+    const u64 *u, *add0, *add1;
+    u64 *out;
+    size_t add_stride, out_stride;
+    u64 galois;
+    uint32_t level, nt;
+    int accumulate;
+    TiledOut tl;
+};
+void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbMap &map, bool inverse, cudaStream_t s,
+                const NttEpilogue *ep = nullptr);
 
 void launch_mul_plain_acc(const ckks_ctx *c, const u64 *const *cts, u64 *const *accs, uint32_t ncts, const u64 *pt,
                           uint32_t level, bool init, cudaStream_t s);

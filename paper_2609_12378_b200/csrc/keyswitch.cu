@@ -16,12 +16,6 @@ namespace {
 
 constexpr uint32_t THREADS = 256;
 
-__device__ __forceinline__ uint32_t galois_src(uint32_t p, u64 g, uint32_t log_n, uint32_t N) {
-    if (g == 1) return p;
-    const u64 e = (g * (2ull * bitrev_n(p, log_n) + 1)) & (2ull * N - 1);
-    return bitrev_n((uint32_t)((e - 1) >> 1), log_n);
-}
-
 // dst[b][i][p] = src[b][i][pi_g(p)]  (g = 1: copy); batch entries src_stride / dst_stride words apart
 __global__ void __launch_bounds__(THREADS) permute_kernel(DevTables c, const u64 *src, size_t src_stride, u64 *dst, size_t dst_stride, u64 g) {
     const uint32_t p = blockIdx.x * THREADS + threadIdx.x;
@@ -243,6 +237,11 @@ void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext
 #define CALL_DN(A) launch_moddown_conv<A>(c, w.u, w.conv, level, nb, s)
     DISPATCH_POW2(K, CALL_DN);
 #undef CALL_DN
+    if (c->log_n == 16) {      // the last NTT pass finishes the ModDown itself
+        NttEpilogue ep{w.u, add0, add1, out, add_stride, out_stride, add_galois, level, nt, accumulate ? 1 : 0, tiled};
+        launch_ntt(c, w.conv, nb * 2 * level, plain_map(0, level), false, s, &ep);
+        return;
+    }
     launch_ntt(c, w.conv, nb * 2 * level, plain_map(0, level), false, s);
     moddown_final_kernel<<<dim3(N / THREADS, level, 2 * nb), THREADS, 0, s>>>(c->dev, w.u, w.conv, add0, add1, add_stride, add_galois, out,
                                                                                out_stride, accumulate ? 1 : 0, level, tiled);

@@ -313,7 +313,7 @@ __device__ __forceinline__ uint32_t padded(uint32_t i) { return i + (i >> 4); }
 constexpr uint32_t ROW_PAD = 256 + 16;
 
 // ---- forward, row pass (stages m = 256..32768): CTA = 16 rows, 16 threads per row ---------
-__global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
+__global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, int has_ep, NttEpilogue ep) {
     __shared__ u64 sm[16 * ROW_PAD];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
@@ -333,6 +333,31 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 
 #pragma unroll
         for (uint32_t k = 0; k < 16; k++) x[k] = s[padded(16 * t + k)];
         fwd16_d(x, tw, 16 * (256 + row) + t, q, qinv);
+        if (has_ep) {      // ModDown tail: (u - NTT(conv)) P^-1 + sigma_g(add), written to its final place
+            const uint32_t y = blockIdx.y, i = y % ep.level, comp = (y / ep.level) & 1, bz = y / (2 * ep.level);
+            const u64 qi = c.mod[prime];
+            const ulonglong2 pinv = c.dn_p_inv[i];
+            const uint32_t p0 = row * 256 + 16 * t;
+            const u64 *up = ep.u + (((size_t)bz * 2 + comp) * ep.nt + i) * 65536 + p0;
+            const u64 *add = comp ? ep.add1 : ep.add0;
+            u64 *dst = ep.tl.R ? ep.out + tiled_index(ep.tl.R, 65536, ep.tl.row0 + bz * ep.tl.row_stride + comp, i, p0)
+                               : ep.out + bz * ep.out_stride + ((size_t)comp * ep.level + i) * 65536 + p0;
+#pragma unroll
+            for (uint32_t k = 0; k < 16; k += 4) {
+                u64 uu[4], old[4] = {0, 0, 0, 0}, r[4];
+                ldg_4(up + k, uu[0], uu[1], uu[2], uu[3]);
+                if (ep.accumulate) ldg_4(dst + k, old[0], old[1], old[2], old[3]);
+#pragma unroll
+                for (uint32_t e = 0; e < 4; e++) {
+                    const u64 v = canonical_d(reduce_d(x[k + e], q, qinv), q);
+                    r[e] = mul_shoup(sub_mod(uu[e], v, qi), pinv.x, pinv.y, qi);
+                    if (add) r[e] = add_mod(r[e], add[bz * ep.add_stride + (size_t)i * 65536 + galois_src(p0 + k + e, ep.galois, 16, 65536)], qi);
+                    if (ep.accumulate) r[e] = add_mod(r[e], old[e], qi);
+                }
+                stg_4(dst + k, r[0], r[1], r[2], r[3]);
+            }
+            return;
+        }
         // a thread ends up with 16 consecutive coefficients: four 32-byte stores, each a full sector
 #pragma unroll
         for (uint32_t k = 0; k < 16; k += 4)
@@ -464,7 +489,8 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_inv_cols(DevTables c, u64 
 
 }  // namespace
 
-void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbMap &map, bool inverse, cudaStream_t s) {
+void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbMap &map, bool inverse, cudaStream_t s,
+                const NttEpilogue *ep) {
     if (nlimbs_total == 0) return;
     if (c->log_n == 16) {
         for (uint32_t y0 = 0; y0 < nlimbs_total;) {
@@ -473,8 +499,10 @@ void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbM
             u64 *b = base + (limb_index(map, y0) << 16);
             dim3 grid(16, ny);
             if (!inverse) {
-                ntt16_fwd_cols<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share); count_launches();
-                ntt16_fwd_rows<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share); count_launches();
+                // an epilogue is only implemented on the double-precision path, so it takes all limbs there
+                const uint32_t share = ep ? 8 : c->ntt_fp_share;
+                ntt16_fwd_cols<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share); count_launches();
+                ntt16_fwd_rows<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, ep ? 1 : 0, ep ? *ep : NttEpilogue{}); count_launches();
             } else {
                 ntt16_inv_rows<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share); count_launches();
                 ntt16_inv_cols<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share); count_launches();
