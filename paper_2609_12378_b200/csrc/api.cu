@@ -474,7 +474,7 @@ extern "C" int32_t ckks_linear_proj(ckks_ctx *c, const ckks_proj_desc *d, const 
             for (uint32_t gl = 0; gl < ng; gl++)
                 for (uint32_t ib = 0; ib < nib; ib++)
                     if (g0 + gl >= std::min(p.ins[ib].size, o.size) / B) ragged = true;
-            if (ragged) cudaMemsetAsync(pts, 0, (size_t)ng * J * ptl * sizeof(u64), s);
+            if (ragged) cudaMemsetAsync(ptt, 0, (size_t)ng * J * ptl * sizeof(u64), s);
             for (uint32_t gl = 0; gl < ng; gl++)
                 for (uint32_t ib = 0; ib < nib; ib++) {
                     const Block &i = p.ins[ib];
@@ -483,10 +483,17 @@ extern "C" int32_t ckks_linear_proj(ckks_ctx *c, const ckks_proj_desc *d, const 
                     const size_t idx = ((size_t)gl * nib + ib) * B;
                     launch_extract_diagonals(c, W, d->d_out, i.start, i.size, o.start, o.size, p.F, T, gi * B, B, gi * B,
                                              slots + idx * c->n, s);
-                    if (ragged) launch_encode(c, slots + idx * c->n, nullptr, B, pt_scale, level, pts + idx * ptl, encw, s);
+                    if (ragged) {
+                        TiledOut to;
+                        to.R = ng * J; to.row0 = (uint32_t)idx; to.row_stride = 1;
+                        launch_encode(c, slots + idx * c->n, nullptr, B, pt_scale, level, pts + idx * ptl, encw, s, to, ptt);
+                    }
                 }
-            if (!ragged) launch_encode(c, slots, nullptr, ng * J, pt_scale, level, pts, encw, s);
-            launch_to_tiled(c, pts, ptl, ng * J, ptt, ng * J, 0, 1, level, s);
+            if (!ragged) {
+                TiledOut to;
+                to.R = ng * J; to.row0 = 0; to.row_stride = 1;
+                launch_encode(c, slots, nullptr, ng * J, pt_scale, level, pts, encw, s, to, ptt);
+            }
             if (!launch_mac_mma(c, baby, ptt, acc, J, S, ng, level, s)) {
                 const uint32_t stiles = (S + MAC_ST - 1) / MAC_ST, gtiles = (ng + MAC_GT - 1) / MAC_GT;
                 mac_tile_kernel<<<dim3(stiles * gtiles, N / MAC_THREADS, level), MAC_THREADS, 0, s>>>(c->dev, baby, ptt, acc, J, S, ng, level);

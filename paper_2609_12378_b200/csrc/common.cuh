@@ -187,7 +187,10 @@ inline void count_launches(unsigned n = 1) { g_kernel_launches += n; }
 // Optional epilogue of the forward transform (N = 2^16 path): instead of storing NTT(conv) the last pass finishes the
 // ModDown: out[b][comp][i][p] (+)= (u[b][comp][i][p] - NTT(conv)[p]) P^-1 + sigma_g(add_comp)[b][i][p], for a buffer of
 // limbs laid out [b][comp][level]; `out` in the plain layout (out_stride words per b) or tiled (tl.R != 0).
+// mode 2: the transform's own result is stored, but into a tiled buffer: limb y = b * level + i becomes row
+// tl.row0 + b * tl.row_stride, limb i.
 struct NttEpilogue {
+    int mode;      // 1 = ModDown tail, 2 = tiled store
     const u64 *u, *add0, *add1;
     u64 *out;
     size_t add_stride, out_stride;
@@ -196,8 +199,10 @@ struct NttEpilogue {
     int accumulate;
     TiledOut tl;
 };
+// coef_src (forward, N = 2^16 path only): the first pass reads signed 64-bit coefficients [batch][N] (batch = limb
+// index / map.period) and reduces them modulo the limb's prime on the fly instead of reading `base`.
 void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbMap &map, bool inverse, cudaStream_t s,
-                const NttEpilogue *ep = nullptr);
+                const NttEpilogue *ep = nullptr, const long long *coef_src = nullptr);
 
 void launch_mul_plain_acc(const ckks_ctx *c, const u64 *const *cts, u64 *const *accs, uint32_t ncts, const u64 *pt,
                           uint32_t level, bool init, cudaStream_t s);
@@ -231,8 +236,10 @@ bool launch_mac_mma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc
 void launch_rescale(const ckks_ctx *c, const u64 *in, u64 *out, uint32_t ncomp, uint32_t level, u64 *ws, cudaStream_t s);
 
 size_t encode_workspace_bytes(const ckks_ctx *c, uint32_t batch);
+// tiled.R != 0 (N = 2^16 only): plaintext b is written as row tiled.row0 + b * tiled.row_stride of the tiled buffer
+// `tiled_out`; `out` is then only the scratch between the two NTT passes.
 void launch_encode(const ckks_ctx *c, const double *re, const double *im, uint32_t batch, double scale, uint32_t level,
-                   u64 *out, void *ws, cudaStream_t s);
+                   u64 *out, void *ws, cudaStream_t s, TiledOut tiled = TiledOut(), u64 *tiled_out = nullptr);
 // Slot vectors of pre-rotated generalised diagonals, [count][n] fp64, for k = k0 .. k0+count-1 of one block pair.
 void launch_extract_diagonals(const ckks_ctx *c, const double *W, uint32_t d_out_total, uint32_t in0, uint32_t m_in,
                               uint32_t out0, uint32_t m_out, uint32_t F, uint32_t T, uint32_t k0, uint32_t count,

@@ -109,7 +109,7 @@ size_t encode_workspace_bytes(const ckks_ctx *c, uint32_t batch) {
 }
 
 void launch_encode(const ckks_ctx *c, const double *re, const double *im, uint32_t batch, double scale, uint32_t level,
-                   u64 *out, void *ws, cudaStream_t s) {
+                   u64 *out, void *ws, cudaStream_t s, TiledOut tiled, u64 *tiled_out) {
     const uint32_t n = c->n, N = c->N, ch = n < CH ? n : CH;
     double2 *buf = (double2 *)ws;
     long long *coef = (long long *)(buf + (size_t)batch * n);
@@ -121,11 +121,24 @@ void launch_encode(const ckks_ctx *c, const double *re, const double *im, uint32
         fft_strips_round<<<dim3(ch / COLS, nb), THREADS, (size_t)(n / ch) * COLS * sizeof(double2), s>>>(
             c->dev, buf + (size_t)b0 * n, coef + (size_t)b0 * N, n, ch, sc); count_launches();
     }
+    if (c->log_n == 16 && (uint64_t)batch * level <= 32768) {
+        // the first NTT pass reduces the signed coefficients itself; the last one can write the tiled layout
+        if (tiled.R) {
+            NttEpilogue ep{};
+            ep.mode = 2; ep.out = tiled_out; ep.level = level; ep.tl = tiled;
+            launch_ntt(c, out, batch * level, plain_map(0, level), false, s, &ep, coef);
+        } else {
+            launch_ntt(c, out, batch * level, plain_map(0, level), false, s, nullptr, coef);
+        }
+        return;
+    }
     for (uint32_t b0 = 0; b0 < batch; b0 += 32768) {
         const uint32_t nb = batch - b0 < 32768 ? batch - b0 : 32768;
-        reduce_coeffs<<<dim3(N / THREADS, level, nb), THREADS, 0, s>>>(c->dev, coef + (size_t)b0 * N, out + (size_t)b0 * level * N, level); count_launches();
+        reduce_coeffs<<<dim3(N / THREADS, level, nb), THREADS, 0, s>>>(c->dev, coef + (size_t)b0 * N, out + (size_t)b0 * level * N, level);
+        count_launches();
     }
     launch_ntt(c, out, batch * level, plain_map(0, level), false, s);
+    if (tiled.R) launch_to_tiled(c, out, (size_t)level * N, batch, tiled_out, tiled.R, tiled.row0, tiled.row_stride, level, s);
 }
 
 void launch_extract_diagonals(const ckks_ctx *c, const double *W, uint32_t d_out_total, uint32_t in0, uint32_t m_in,

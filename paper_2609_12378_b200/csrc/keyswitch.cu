@@ -238,7 +238,7 @@ void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext
     DISPATCH_POW2(K, CALL_DN);
 #undef CALL_DN
     if (c->log_n == 16) {      // the last NTT pass finishes the ModDown itself
-        NttEpilogue ep{w.u, add0, add1, out, add_stride, out_stride, add_galois, level, nt, accumulate ? 1 : 0, tiled};
+        NttEpilogue ep{1, w.u, add0, add1, out, add_stride, out_stride, add_galois, level, nt, accumulate ? 1 : 0, tiled};
         launch_ntt(c, w.conv, nb * 2 * level, plain_map(0, level), false, s, &ep);
         return;
     }

@@ -266,7 +266,7 @@ __device__ __forceinline__ void inv16_d(double (&x)[16], const double *__restric
 }
 
 // ---- forward, column pass (stages m = 1..128): CTA = strip of 16 columns -----------------
-__global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
+__global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, const long long *coef_src) {
     __shared__ u64 sm[256 * 16];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
@@ -277,8 +277,19 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_cols(DevTables c, u64 
         u64 *g = base + (limb_index(map, blockIdx.y) << 16) + blockIdx.x * 16 + cc;
         double *smd = reinterpret_cast<double *>(sm);
         double x[16];
+        if (coef_src) {     // signed coefficients shared by all limbs of a batch entry, reduced here
+            const long long *cs = coef_src + ((size_t)(blockIdx.y / map.period) << 16) + blockIdx.x * 16 + cc;
+            const u64 qi = c.mod[prime], mu = c.mu[prime];
 #pragma unroll
-        for (uint32_t k = 0; k < 16; k++) x[k] = u64_to_d(g[(size_t)(r + 16 * k) * 256]);
+            for (uint32_t k = 0; k < 16; k++) {
+                const long long v = cs[(size_t)(r + 16 * k) * 256];
+                const u64 m = barrett112(0, v < 0 ? (u64)(-v) : (u64)v, qi, mu);
+                x[k] = u64_to_d((v < 0 && m) ? qi - m : m);
+            }
+        } else {
+#pragma unroll
+            for (uint32_t k = 0; k < 16; k++) x[k] = u64_to_d(g[(size_t)(r + 16 * k) * 256]);
+        }
         fwd16_d(x, tw, 1, q, qinv);
 #pragma unroll
         for (uint32_t k = 0; k < 16; k++) smd[(r + 16 * k) * 16 + cc] = x[k];
@@ -333,6 +344,15 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 
 #pragma unroll
         for (uint32_t k = 0; k < 16; k++) x[k] = s[padded(16 * t + k)];
         fwd16_d(x, tw, 16 * (256 + row) + t, q, qinv);
+        if (has_ep == 2) {     // the result itself, but into a tiled buffer
+            const uint32_t y = blockIdx.y, i = y % ep.level, b = y / ep.level;
+            u64 *dst = ep.out + tiled_index(ep.tl.R, 65536, ep.tl.row0 + b * ep.tl.row_stride, i, row * 256 + 16 * t);
+#pragma unroll
+            for (uint32_t k = 0; k < 16; k += 4)
+                stg_4(dst + k, canonical_d(reduce_d(x[k], q, qinv), q), canonical_d(reduce_d(x[k + 1], q, qinv), q),
+                      canonical_d(reduce_d(x[k + 2], q, qinv), q), canonical_d(reduce_d(x[k + 3], q, qinv), q));
+            return;
+        }
         if (has_ep) {      // ModDown tail: (u - NTT(conv)) P^-1 + sigma_g(add), written to its final place
             const uint32_t y = blockIdx.y, i = y % ep.level, comp = (y / ep.level) & 1, bz = y / (2 * ep.level);
             const u64 qi = c.mod[prime];
@@ -490,7 +510,7 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_inv_cols(DevTables c, u64 
 }  // namespace
 
 void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbMap &map, bool inverse, cudaStream_t s,
-                const NttEpilogue *ep) {
+                const NttEpilogue *ep, const long long *coef_src) {
     if (nlimbs_total == 0) return;
     if (c->log_n == 16) {
         for (uint32_t y0 = 0; y0 < nlimbs_total;) {
@@ -500,9 +520,9 @@ void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbM
             dim3 grid(16, ny);
             if (!inverse) {
                 // an epilogue is only implemented on the double-precision path, so it takes all limbs there
-                const uint32_t share = ep ? 8 : c->ntt_fp_share;
-                ntt16_fwd_cols<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share); count_launches();
-                ntt16_fwd_rows<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, ep ? 1 : 0, ep ? *ep : NttEpilogue{}); count_launches();
+                const uint32_t share = (ep || coef_src) ? 8 : c->ntt_fp_share;
+                ntt16_fwd_cols<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, coef_src); count_launches();
+                ntt16_fwd_rows<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, ep ? ep->mode : 0, ep ? *ep : NttEpilogue{}); count_launches();
             } else {
                 ntt16_inv_rows<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share); count_launches();
                 ntt16_inv_cols<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share); count_launches();
