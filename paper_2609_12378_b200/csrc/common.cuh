@@ -161,6 +161,13 @@ __device__ __forceinline__ double mulmod_d(double y, double2 w, double q) {
     const double k = __dsub_rn(__fma_rn(y, w.y, M), M);
     return __dadd_rn(__fma_rn(-k, q, p), e);
 }
+// x * y - k q for two variable residues 0 <= x, y < q (as doubles): exact, |result| <= 0.75 q
+__device__ __forceinline__ double mulmod_dd(double x, double y, double q, double qinv) {
+    const double p = __dmul_rn(x, y);
+    const double e = __fma_rn(x, y, -p);
+    const double k = __dsub_rn(__fma_rn(p, qinv, MAGIC0), MAGIC0);
+    return __dadd_rn(__fma_rn(-k, q, p), e);
+}
 __device__ __forceinline__ double reduce_d(double v, double q, double qinv) {   // to |v| <= q/2
     const double k = __dsub_rn(__fma_rn(v, qinv, MAGIC0), MAGIC0);
     return __fma_rn(-k, q, v);

@@ -87,18 +87,20 @@ __global__ void __launch_bounds__(THREADS) inner_product_kernel(DevTables c, con
     const uint32_t x = blockIdx.z, bz = blockIdx.y;     // batch varies faster than the limb: a key limb is reused from L2
     const uint32_t nt = level + c.K, beta = (level + c.alpha - 1) / c.alpha;
     const uint32_t kt = x < level ? x : c.L + (x - level);
-    const u64 m = c.mod[kt], mu = c.mu[kt];
     const uint32_t src = galois_src(p, g, c.log_n, c.N);
     ext += (size_t)bz * beta * nt * c.N;
     u += (size_t)bz * 2 * nt * c.N;
-    u64 h0 = 0, l0 = 0, h1 = 0, l1 = 0;
+    // products on the FP64 pipe: each is reduced to |r| <= 0.75 m as it is formed, the few digits are summed exactly
+    const double2 md = c.modd[kt];
+    double a0 = 0.0, a1 = 0.0;
     for (uint32_t j = 0; j < beta; j++) {
-        const u64 e = ext[((size_t)j * nt + x) * c.N + src];
-        mac128(h0, l0, e, evk[(((size_t)j * 2 + 0) * c.T + kt) * c.N + p]);
-        mac128(h1, l1, e, evk[(((size_t)j * 2 + 1) * c.T + kt) * c.N + p]);
+        const double e = u64_to_d(ext[((size_t)j * nt + x) * c.N + src]);
+        a0 = __dadd_rn(a0, mulmod_dd(e, u64_to_d(evk[(((size_t)j * 2 + 0) * c.T + kt) * c.N + p]), md.x, md.y));
+        a1 = __dadd_rn(a1, mulmod_dd(e, u64_to_d(evk[(((size_t)j * 2 + 1) * c.T + kt) * c.N + p]), md.x, md.y));
+        if ((j & 7) == 7) { a0 = reduce_d(a0, md.x, md.y); a1 = reduce_d(a1, md.x, md.y); }
     }
-    u[((size_t)0 * nt + x) * c.N + p] = barrett112(h0, l0, m, mu);
-    u[((size_t)1 * nt + x) * c.N + p] = barrett112(h1, l1, m, mu);
+    u[((size_t)0 * nt + x) * c.N + p] = canonical_d(reduce_d(a0, md.x, md.y), md.x);
+    u[((size_t)1 * nt + x) * c.N + p] = canonical_d(reduce_d(a1, md.x, md.y), md.x);
 }
 
 // conv[comp][i][k] = sum_a centre([u_{p_a} Phat_a^-1]) (Phat_a mod q_i)  mod q_i   (coefficient domain)
