@@ -462,6 +462,7 @@ void orc_switch_keygen(const orc_ctx *c, const int64_t *s, const uint64_t *sprim
 /* PCMult + Add: acc[c][i][.] (+)= ct[c][i][.] * pt[i][.], c in {0,1}. */
 void orc_mul_plain_acc(const orc_ctx *c, const uint64_t *ct, const uint64_t *pt, uint64_t *acc, uint32_t level, int init) {
     uint64_t N = c->N;
+    #pragma omp parallel for collapse(2)
     for (uint32_t comp = 0; comp < 2; comp++)
         for (uint32_t i = 0; i < level; i++) {
             uint64_t q = c->mod[i];
