@@ -77,3 +77,62 @@ def test_sixty_four_rotations_full_size():
         zh = cl.decrypt_slots(host(hoisted[i].data), scale).real
         want = np.roll(z, -r)
         assert np.abs(zp - want).max() < 2.0 ** -17 and np.abs(zh - want).max() < 2.0 ** -17, i
+
+
+def _full_ring_shape(d_in, d_out, S, B, seed, shards_checked=1):
+    """A decoder-layer projection shape at N = 2^16, level 24: decrypt everything, recompute `shards_checked` shards."""
+    from tests.gpu_util import context, ct_dev, dev, host, key_dev
+    P, ctx = params(16, 24, 8, 3), context(16, 24, 8, 3)
+    o = P.oracle
+    cl = Client(P, seed)
+    level, scale, T = 24, 2.0 ** 40, 8
+    g = inputs.rng(seed, 1)
+    X = inputs.activations_normal(g, S * T, d_in)
+    W = inputs.weights_normal(g, d_in, d_out, 0.02)
+    desc = ProjDesc(d_in, d_out, T, S, B)
+    F, ins, outs_b = o.proj_blocks(desc)
+    rots = o.proj_rotations(desc)
+    assert rots == ctx.linear_proj_rotations(d_in, d_out, T, S, B)
+    cts = []
+    for c in range(S):
+        for (s0, mi) in ins:
+            cts.append(cl.encrypt_slots(inputs.pack_feature_major(X[c * T:(c + 1) * T, s0:s0 + mi], T, o.n)[0], scale, level))
+    keys = {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in rots}
+    outs = ctx.linear_proj([ct_dev(c, scale) for c in cts], dev(W), [key_dev(k, ge) for ge, k in keys.items()], d_in, d_out, T, S, B)
+    assert ctx.device_status() == binding.OK
+    Y = X @ W
+    nib, nob = len(ins), len(outs_b)
+    got = [host(ct.data) for ct in outs]
+    for c in range(S):
+        for ob, (o0, mo) in enumerate(outs_b):
+            sl = cl.decrypt_slots(got[c * nob + ob], outs[c * nob + ob].scale).real.reshape(F, T)
+            for r in range(0, F, 37):
+                assert np.abs(sl[r] - Y[c * T:(c + 1) * T, o0 + r % mo]).max() < 2.0 ** -16, (c, ob, r)
+    for c in range(shards_checked):
+        one = ProjDesc(d_in, d_out, T, 1, B)
+        want, _ = o.linear_proj(one, np.stack(cts[c * nib:(c + 1) * nib]), W, keys, scale)
+        for ob in range(nob):
+            assert np.array_equal(got[c * nob + ob], want[ob]), (c, ob)
+
+
+def test_kv_projection_full_ring():
+    """K / V shape: 4096 -> 1024 (wide block, folded twice), B = G = 32."""
+    _full_ring_shape(4096, 1024, 4, 32, seed=1005)
+
+
+import os  # noqa: E402
+
+heavy = pytest.mark.skipif(os.environ.get("CKKS_RUN_HEAVY") != "1",
+                           reason="ten minutes of CPU checker time per shape; set CKKS_RUN_HEAVY=1")
+
+
+@heavy
+def test_gate_up_projection_full_ring():
+    """gate / up shape: 4096 -> 14336 = 3 x 4096 + 2048 (three square output blocks and a folded remainder block)."""
+    _full_ring_shape(4096, 14336, 2, 64, seed=1006)
+
+
+@heavy
+def test_down_projection_full_ring():
+    """down shape: 14336 -> 4096 (three full input blocks and a repeated remainder block summed before the giant steps)."""
+    _full_ring_shape(14336, 4096, 2, 64, seed=1007)
