@@ -189,7 +189,9 @@ int32_t ckks_rotate(ckks_ctx *ctx, const ckks_ct *in, const ckks_evk *key, ckks_
  * permutes the extended digits by sigma_{g_r}, takes the inner product with
  * keys[r], ModDown, adds sigma(c0).  As an integer function this differs from
  * ckks_rotate (same plaintext, different low noise bits).  keys, outs: host
- * arrays of nrot descriptors.  Errors as ckks_rotate. */
+ * arrays of nrot descriptors.  With the workspace ckks_workspace_bytes(CKKS_OP_ROTATE_HOISTED, level, nrot) asks
+ * for, up to 16 rotations run side by side; any workspace of at least the CKKS_OP_ROTATE size is accepted.
+ * Errors as ckks_rotate. */
 int32_t ckks_rotate_hoisted(ckks_ctx *ctx, const ckks_ct *in, const ckks_evk *keys, uint32_t nrot, ckks_ct *outs,
                             void *ws, size_t ws_bytes, void *stream);
 

@@ -26,6 +26,11 @@ bool ct_ok(const ckks_ct *ct) { return ct && ct->data; }
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 size_t ks_bytes(const ckks_ctx *c, uint32_t level) { return ks_workspace_limbs(c, level) * c->N * sizeof(u64); }
+// hoisted rotations: one set of digits, nbh rotations' worth of inner-product and ModDown buffers side by side
+size_t hoisted_bytes(const ckks_ctx *c, uint32_t level, uint32_t nbh) {
+    const size_t beta = (level + c->alpha - 1) / c->alpha, nt = level + c->K;
+    return (level + beta * nt + (size_t)nbh * (2 * nt + 2 * level)) * c->N * sizeof(u64);
+}
 size_t rescale_bytes(const ckks_ctx *c, uint32_t level, uint32_t ncomp) { return (size_t)ncomp * level * c->N * sizeof(u64); }
 
 // ---- projection plan -------------------------------------------------------
@@ -218,8 +223,8 @@ extern "C" size_t ckks_workspace_bytes(const ckks_ctx *c, int32_t op, uint32_t l
     switch (op) {
         case CKKS_OP_ENCODE: return encode_workspace_bytes(c, count ? count : 1);
         case CKKS_OP_MUL_RELIN: return ks_bytes(c, level) + (size_t)level * limb;
-        case CKKS_OP_ROTATE:
-        case CKKS_OP_ROTATE_HOISTED: return ks_bytes(c, level);
+        case CKKS_OP_ROTATE: return ks_bytes(c, level);
+        case CKKS_OP_ROTATE_HOISTED: return hoisted_bytes(c, level, std::min<uint32_t>(count ? count : 1, KS_MULTI));
         case CKKS_OP_RESCALE: return rescale_bytes(c, level, 2);
         default: return 0;
     }
@@ -364,11 +369,23 @@ extern "C" int32_t ckks_rotate_hoisted(ckks_ctx *c, const ckks_ct *in, const ckk
     DeviceGuard g(c->device);
     cudaStream_t s = (cudaStream_t)stream;
     const uint32_t level = in->level;
-    KsWorkspace w = ks_carve(c, level, ws);
-    const u64 *c0 = (const u64 *)in->data, *c1 = c0 + (size_t)level * c->N;
+    // as many rotations side by side as the workspace allows (one is always possible)
+    uint32_t nbh = std::min<uint32_t>(nrot, KS_MULTI);
+    while (nbh > 1 && hoisted_bytes(c, level, nbh) > ws_bytes) nbh--;
+    const size_t beta = (level + c->alpha - 1) / c->alpha, nt = level + c->K, N = c->N;
+    KsWorkspace w;
+    w.dcoef = (u64 *)ws;
+    w.ext = w.dcoef + (size_t)level * N;
+    w.u = w.ext + beta * nt * N;
+    w.conv = w.u + (size_t)nbh * 2 * nt * N;
+    const u64 *c0 = (const u64 *)in->data, *c1 = c0 + (size_t)level * N;
     ks_modup(c, c1, 1, level, w, s);
-    for (uint32_t r = 0; r < nrot; r++)
-        ks_inner_moddown(c, (const u64 *)keys[r].data, level, keys[r].galois, w, c0, nullptr, keys[r].galois, (u64 *)outs[r].data, s);
+    for (uint32_t r0 = 0; r0 < nrot; r0 += nbh) {
+        const uint32_t nb = std::min(nbh, nrot - r0);
+        KsMulti m{};
+        for (uint32_t b = 0; b < nb; b++) { m.evk[b] = (const u64 *)keys[r0 + b].data; m.galois[b] = keys[r0 + b].galois; m.out[b] = (u64 *)outs[r0 + b].data; }
+        ks_inner_moddown(c, nullptr, level, 1, w, c0, nullptr, 1, nullptr, s, nb, 0, 0, false, TiledOut(), &m);
+    }
     rc = finish(c);
     if (rc == CKKS_OK)
         for (uint32_t r = 0; r < nrot; r++) { outs[r].level = level; outs[r].ncomp = 2; outs[r].scale = in->scale; }

@@ -196,6 +196,15 @@ inline void count_launches(unsigned n = 1) { g_kernel_launches += n; }
 // limbs laid out [b][comp][level]; `out` in the plain layout (out_stride words per b) or tiled (tl.R != 0).
 // mode 2: the transform's own result is stored, but into a tiled buffer: limb y = b * level + i becomes row
 // tl.row0 + b * tl.row_stride, limb i.
+// Up to KS_MULTI key switches that share one set of extended digits but differ in key, Galois element and output
+// buffer (hoisted rotations): batch entry b uses evk[b], galois[b], out[b].
+constexpr uint32_t KS_MULTI = 16;
+struct KsMulti {
+    const u64 *evk[KS_MULTI];
+    u64 galois[KS_MULTI];
+    u64 *out[KS_MULTI];
+};
+
 struct NttEpilogue {
     int mode;      // 1 = ModDown tail, 2 = tiled store
     const u64 *u, *add0, *add1;
@@ -205,6 +214,9 @@ struct NttEpilogue {
     uint32_t level, nt;
     int accumulate;
     TiledOut tl;
+    int multi;             // mode 1: batch entry b adds through mgalois[b] and writes to mout[b]
+    u64 mgalois[KS_MULTI];
+    u64 *mout[KS_MULTI];
 };
 // coef_src (forward, N = 2^16 path only): the first pass reads signed 64-bit coefficients [batch][N] (batch = limb
 // index / map.period) and reduces them modulo the limb's prime on the fly instead of reading `base`.
@@ -229,7 +241,8 @@ void ks_modup(const ckks_ctx *c, const u64 *d, u64 galois, uint32_t level, const
 // combination out_c (+)= sigma_{add_galois}(add_c) + k_c.  add0/add1 may be null.
 void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext_galois, const KsWorkspace &w,
                       const u64 *add0, const u64 *add1, u64 add_galois, u64 *out, cudaStream_t s, uint32_t nb = 1,
-                      size_t add_stride = 0, size_t out_stride = 0, bool accumulate = false, TiledOut tiled = TiledOut());
+                      size_t add_stride = 0, size_t out_stride = 0, bool accumulate = false, TiledOut tiled = TiledOut(),
+                      const KsMulti *multi = nullptr);
 // rows of [level][N] words, src_stride words apart, into rows row0, row0 + row_step, .. of a tiled buffer with R rows
 void launch_to_tiled(const ckks_ctx *c, const u64 *src, size_t src_stride, uint32_t nrows, u64 *dst, uint32_t R, uint32_t row0,
                      uint32_t row_step, uint32_t level, cudaStream_t s);

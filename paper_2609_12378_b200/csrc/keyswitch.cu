@@ -23,7 +23,9 @@ __global__ void __launch_bounds__(THREADS) permute_kernel(DevTables c, const u64
     dst[blockIdx.z * dst_stride + row + p] = src[blockIdx.z * src_stride + row + galois_src(p, g, c.log_n, c.N)];
 }
 
-constexpr uint32_t CHUNK = 32;  // targets per CTA row in the basis-conversion kernels (source limbs are re-read once per chunk)
+// targets per CTA row in the basis-conversion kernels: the source limbs are re-read once per chunk, so large batches
+// take all targets in one chunk and single ciphertexts split them for parallelism
+inline uint32_t conv_chunk(uint32_t nb) { return nb >= 4 ? 32 : 8; }
 
 // ext[j][x][k] for x over q_0..q_{level-1}, p_0..p_{K-1}.  dcoef: sigma_g(d) in the coefficient domain;
 // deval: d in the evaluation domain, read through sigma_g for the digit's own limbs.
@@ -31,7 +33,7 @@ constexpr uint32_t CHUNK = 32;  // targets per CTA row in the basis-conversion k
 // walks a chunk of CHUNK target limbs (blockIdx.y), so the source limbs are read once per chunk.
 template <uint32_t ALPHA>
 __global__ void __launch_bounds__(THREADS) modup_kernel(DevTables c, const u64 *dcoef, const u64 *deval, size_t deval_stride, u64 g,
-                                                        u64 *ext, uint32_t level) {
+                                                        u64 *ext, uint32_t level, uint32_t CHUNK) {
     const uint32_t k = blockIdx.x * THREADS + threadIdx.x;
     const uint32_t beta = (level + c.alpha - 1) / c.alpha, j = blockIdx.z % beta, bz = blockIdx.z / beta;
     const uint32_t nt = level + c.K, lo = j * c.alpha, hi = min(lo + c.alpha, level), nd = hi - lo;
@@ -76,19 +78,21 @@ template <uint32_t ALPHA>
 void launch_modup(const ckks_ctx *c, const u64 *dcoef, const u64 *deval, size_t deval_stride, u64 g, u64 *ext, uint32_t level,
                   uint32_t nb, cudaStream_t s) {
     const uint32_t nt = level + c->K, beta = (level + c->alpha - 1) / c->alpha;
-    modup_kernel<ALPHA><<<dim3(c->N / THREADS, (nt + CHUNK - 1) / CHUNK, beta * nb), THREADS, 0, s>>>(c->dev, dcoef, deval, deval_stride, g, ext, level);
+    const uint32_t CHUNK = conv_chunk(nb);
+    modup_kernel<ALPHA><<<dim3(c->N / THREADS, (nt + CHUNK - 1) / CHUNK, beta * nb), THREADS, 0, s>>>(c->dev, dcoef, deval, deval_stride, g, ext, level, CHUNK);
     count_launches();
 }
 
 // u[comp][x][p] = sum_j ext[j][x][pi_g(p)] * evk[j][comp][kt(x)][p]
 __global__ void __launch_bounds__(THREADS) inner_product_kernel(DevTables c, const u64 *ext, const u64 *evk, u64 g,
-                                                                u64 *u, uint32_t level) {
+                                                                u64 *u, uint32_t level, int has_multi, KsMulti multi) {
     const uint32_t p = blockIdx.x * THREADS + threadIdx.x;
     const uint32_t x = blockIdx.z, bz = blockIdx.y;     // batch varies faster than the limb: a key limb is reused from L2
     const uint32_t nt = level + c.K, beta = (level + c.alpha - 1) / c.alpha;
     const uint32_t kt = x < level ? x : c.L + (x - level);
+    if (has_multi) { evk = multi.evk[bz]; g = multi.galois[bz]; }     // shared digits, per-entry key and permutation
+    else ext += (size_t)bz * beta * nt * c.N;
     const uint32_t src = galois_src(p, g, c.log_n, c.N);
-    ext += (size_t)bz * beta * nt * c.N;
     u += (size_t)bz * 2 * nt * c.N;
     // products on the FP64 pipe: each is reduced to |r| <= 0.75 m as it is formed, the few digits are summed exactly
     const double2 md = c.modd[kt];
@@ -106,7 +110,7 @@ __global__ void __launch_bounds__(THREADS) inner_product_kernel(DevTables c, con
 // conv[comp][i][k] = sum_a centre([u_{p_a} Phat_a^-1]) (Phat_a mod q_i)  mod q_i   (coefficient domain)
 // Same shape as ModUp: the K centred special residues are formed once per thread, then a chunk of targets is walked.
 template <uint32_t KK>
-__global__ void __launch_bounds__(THREADS) moddown_conv_kernel(DevTables c, const u64 *u, u64 *conv, uint32_t level) {
+__global__ void __launch_bounds__(THREADS) moddown_conv_kernel(DevTables c, const u64 *u, u64 *conv, uint32_t level, uint32_t CHUNK) {
     const uint32_t k = blockIdx.x * THREADS + threadIdx.x;
     const uint32_t comp = blockIdx.z & 1, bz = blockIdx.z >> 1;
     const uint32_t nt = level + c.K;
@@ -139,7 +143,8 @@ __global__ void __launch_bounds__(THREADS) moddown_conv_kernel(DevTables c, cons
 
 template <uint32_t KK>
 void launch_moddown_conv(const ckks_ctx *c, const u64 *u, u64 *conv, uint32_t level, uint32_t nb, cudaStream_t s) {
-    moddown_conv_kernel<KK><<<dim3(c->N / THREADS, (level + CHUNK - 1) / CHUNK, 2 * nb), THREADS, 0, s>>>(c->dev, u, conv, level);
+    const uint32_t CHUNK = conv_chunk(nb);
+    moddown_conv_kernel<KK><<<dim3(c->N / THREADS, (level + CHUNK - 1) / CHUNK, 2 * nb), THREADS, 0, s>>>(c->dev, u, conv, level, CHUNK);
     count_launches();
 }
 
@@ -231,9 +236,11 @@ void ks_modup(const ckks_ctx *c, const u64 *d, u64 galois, uint32_t level, const
 
 void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext_galois, const KsWorkspace &w,
                       const u64 *add0, const u64 *add1, u64 add_galois, u64 *out, cudaStream_t s, uint32_t nb,
-                      size_t add_stride, size_t out_stride, bool accumulate, TiledOut tiled) {
+                      size_t add_stride, size_t out_stride, bool accumulate, TiledOut tiled, const KsMulti *multi) {
     const uint32_t N = c->N, nt = level + c->K, K = c->K;
-    inner_product_kernel<<<dim3(N / THREADS, nb, nt), THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level); count_launches();
+    inner_product_kernel<<<dim3(N / THREADS, nb, nt), THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, multi ? 1 : 0,
+                                                                         multi ? *multi : KsMulti{});
+    count_launches();
     // the K special limbs of every (batch, component): groups of K limbs, nt limbs apart
     launch_ntt(c, w.u + (size_t)level * N, nb * 2 * K, pitched_map(c->L, K, nt), true, s);
 #define CALL_DN(A) launch_moddown_conv<A>(c, w.u, w.conv, level, nb, s)
@@ -241,10 +248,21 @@ void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext
 #undef CALL_DN
     if (c->log_n == 16) {      // the last NTT pass finishes the ModDown itself
         NttEpilogue ep{1, w.u, add0, add1, out, add_stride, out_stride, add_galois, level, nt, accumulate ? 1 : 0, tiled};
+        ep.multi = multi ? 1 : 0;
+        if (multi)
+            for (uint32_t b = 0; b < KS_MULTI; b++) { ep.mgalois[b] = multi->galois[b]; ep.mout[b] = multi->out[b]; }
         launch_ntt(c, w.conv, nb * 2 * level, plain_map(0, level), false, s, &ep);
         return;
     }
     launch_ntt(c, w.conv, nb * 2 * level, plain_map(0, level), false, s);
+    if (multi) {
+        for (uint32_t b = 0; b < nb; b++) {
+            moddown_final_kernel<<<dim3(N / THREADS, level, 2), THREADS, 0, s>>>(c->dev, w.u + (size_t)b * 2 * nt * N, w.conv + (size_t)b * 2 * level * N,
+                                                                                  add0, add1, 0, multi->galois[b], multi->out[b], 0, 0, level, TiledOut());
+            count_launches();
+        }
+        return;
+    }
     moddown_final_kernel<<<dim3(N / THREADS, level, 2 * nb), THREADS, 0, s>>>(c->dev, w.u, w.conv, add0, add1, add_stride, add_galois, out,
                                                                                out_stride, accumulate ? 1 : 0, level, tiled);
     count_launches();

@@ -360,8 +360,10 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 
             const uint32_t p0 = row * 256 + 16 * t;
             const u64 *up = ep.u + (((size_t)bz * 2 + comp) * ep.nt + i) * 65536 + p0;
             const u64 *add = comp ? ep.add1 : ep.add0;
-            u64 *dst = ep.tl.R ? ep.out + tiled_index(ep.tl.R, 65536, ep.tl.row0 + bz * ep.tl.row_stride + comp, i, p0)
-                               : ep.out + bz * ep.out_stride + ((size_t)comp * ep.level + i) * 65536 + p0;
+            const u64 gal = ep.multi ? ep.mgalois[bz] : ep.galois;
+            u64 *dst = ep.multi ? ep.mout[bz] + ((size_t)comp * ep.level + i) * 65536 + p0
+                       : ep.tl.R ? ep.out + tiled_index(ep.tl.R, 65536, ep.tl.row0 + bz * ep.tl.row_stride + comp, i, p0)
+                                 : ep.out + bz * ep.out_stride + ((size_t)comp * ep.level + i) * 65536 + p0;
 #pragma unroll
             for (uint32_t k = 0; k < 16; k += 4) {
                 u64 uu[4], old[4] = {0, 0, 0, 0}, r[4];
@@ -371,7 +373,7 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 
                 for (uint32_t e = 0; e < 4; e++) {
                     const u64 v = canonical_d(reduce_d(x[k + e], q, qinv), q);
                     r[e] = mul_shoup(sub_mod(uu[e], v, qi), pinv.x, pinv.y, qi);
-                    if (add) r[e] = add_mod(r[e], add[bz * ep.add_stride + (size_t)i * 65536 + galois_src(p0 + k + e, ep.galois, 16, 65536)], qi);
+                    if (add) r[e] = add_mod(r[e], add[bz * ep.add_stride + (size_t)i * 65536 + galois_src(p0 + k + e, gal, 16, 65536)], qi);
                     if (ep.accumulate) r[e] = add_mod(r[e], old[e], qi);
                 }
                 stg_4(dst + k, r[0], r[1], r[2], r[3]);
