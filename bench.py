@@ -135,6 +135,27 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ----------------------------------------------------------------- multi-rank aggregation (replicas: no data-path collective)
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks of the default process group (identity without one)."""
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor([float(v) for v in values], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_metrics(world, a_ms, b_ms, c_ms):
+    """Whole-job figures from the slowest rank's part times: every rank ran the same step on its own replica."""
+    limb_ntts = NTT_BATCH * L
+    return {"value": c_ms * 1e-3 / world,                                   # seconds per projection, all ranks together
+            "ntt_limbs_per_s": world * 2 * limb_ntts / (a_ms * 1e-3),
+            "key_switches_per_s": world * (2 * NROT + 1) / (b_ms * 1e-3)}
+
+
 # ----------------------------------------------------------------- CUDA leg
 def run_cuda(args):
     import torch
@@ -274,10 +295,7 @@ def run_cuda(args):
     h2d = sum(h.numel() * 8 for h in h_cts) + h_W.numel() * 8
     d2h = sum(h.numel() * 8 for h in h_outs)
 
-    if world > 1:
-        tt = torch.tensor([total_ms, a_ms, b_ms, c_ms, e2e_ms, ntt_fwd_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms, a_ms, b_ms, c_ms, e2e_ms, ntt_fwd_ms = tt.tolist()
+    total_ms, a_ms, b_ms, c_ms, e2e_ms, ntt_fwd_ms = max_over_ranks([total_ms, a_ms, b_ms, c_ms, e2e_ms, ntt_fwd_ms], dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -306,13 +324,13 @@ def run_cuda(args):
                 "others": {"mac_mma_kernel": "19.5 % of the step; legacy mma.sync issue bound, see profiles/mac_mma_projection_8shards.md",
                            "inner_product_kernel": "12.9 % of the step; HBM bound (key stream)"}}
     cpu = oracle_sample()
+    jm = job_metrics(world, a_ms, b_ms, c_ms)
     line = {
-        "metric": METRIC, "value": c_ms * 1e-3 / world, "unit": "s/projection", "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": jm["value"], "unit": "s/projection", "n_gpus": world, "steps": args.steps,
         "warmup": nwarm, "ms_per_step": total_ms / args.steps, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "u64", "data": "synthetic",
         "config": {"workload": WORKLOAD, "l2": "inputs larger than L2 (>= 384 MiB per part)", "parallelism": f"replicas x{world}"},
-        "submetrics": {"ntt_limbs_per_s": world * 2 * limb_ntts / (a_ms * 1e-3),
-                       "key_switches_per_s": world * (2 * NROT + 1) / (b_ms * 1e-3),
+        "submetrics": {"ntt_limbs_per_s": jm["ntt_limbs_per_s"], "key_switches_per_s": jm["key_switches_per_s"],
                        "ms": {"ntt_roundtrip": a_ms, "keyswitch_part": b_ms, "projection": c_ms}},
         "clocks": clocks,
         "e2e": {"value": e2e_ms * 1e-3 / world, "unit": "s/projection", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
