@@ -266,11 +266,12 @@ __device__ __forceinline__ void inv16_d(double (&x)[16], const double *__restric
 }
 
 // ---- forward, column pass (stages m = 1..128): CTA = strip of 16 columns -----------------
+template <bool ALLFP>
 __global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, const long long *coef_src) {
     __shared__ u64 sm[256 * 16];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
-    if ((blockIdx.y & 7) < fp_share) {
+    if (ALLFP || (blockIdx.y & 7) < fp_share) {
         const double q = c.modd[prime].x, qinv = c.modd[prime].y;
         const double *tw = c.twd_fwd + ((size_t)prime << 16);
         const uint32_t cc = threadIdx.x & 15, r = threadIdx.x >> 4;
@@ -301,6 +302,7 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_cols(DevTables c, u64 
         for (uint32_t k = 0; k < 16; k++) reinterpret_cast<double *>(g)[(size_t)(16 * r + k) * 256] = x[k];
         return;
     }
+    if (ALLFP) return;
     const u64 q = c.mod[prime], q5 = 5 * q;
     const ulonglong2 *tw = c.tw_fwd + ((size_t)prime << 16);
     const uint32_t cc = threadIdx.x & 15, r = threadIdx.x >> 4;
@@ -324,11 +326,13 @@ __device__ __forceinline__ uint32_t padded(uint32_t i) { return i + (i >> 4); }
 constexpr uint32_t ROW_PAD = 256 + 16;
 
 // ---- forward, row pass (stages m = 256..32768): CTA = 16 rows, 16 threads per row ---------
-__global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, int has_ep, NttEpilogue ep) {
+template <bool ALLFP, int EP>
+__global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, NttEpilogue ep) {
+    constexpr int has_ep = EP;
     __shared__ u64 sm[16 * ROW_PAD];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
-    if ((blockIdx.y & 7) < fp_share) {
+    if (ALLFP || (blockIdx.y & 7) < fp_share) {
         const double q = c.modd[prime].x, qinv = c.modd[prime].y;
         const double *tw = c.twd_fwd + ((size_t)prime << 16);
         const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
@@ -387,6 +391,7 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 
                   canonical_d(reduce_d(x[k + 2], q, qinv), q), canonical_d(reduce_d(x[k + 3], q, qinv), q));
         return;
     }
+    if (ALLFP) return;
     const u64 q = c.mod[prime], q5 = 5 * q;
     const ulonglong2 *tw = c.tw_fwd + ((size_t)prime << 16);
     const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
@@ -412,11 +417,12 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 
 }
 
 // ---- inverse, row pass (stages m = 32768..256) ---------------------------------------------
+template <bool ALLFP>
 __global__ void __launch_bounds__(F_THREADS, 4) ntt16_inv_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
     __shared__ u64 sm[16 * ROW_PAD];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
-    if ((blockIdx.y & 7) < fp_share) {
+    if (ALLFP || (blockIdx.y & 7) < fp_share) {
         const double q = c.modd[prime].x, qinv = c.modd[prime].y;
         const double *tw = c.twd_inv + ((size_t)prime << 16);
         const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
@@ -440,6 +446,7 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_inv_rows(DevTables c, u64 
         for (uint32_t k = 0; k < 16; k++) reinterpret_cast<double *>(g)[t + 16 * k] = x[k];
         return;
     }
+    if (ALLFP) return;
     const u64 q = c.mod[prime];
     const ulonglong2 *tw = c.tw_inv + ((size_t)prime << 16);
     const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
@@ -465,11 +472,12 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_inv_rows(DevTables c, u64 
 }
 
 // ---- inverse, column pass (stages m = 128..1), then N^-1 and the exact reduction -----------
+template <bool ALLFP>
 __global__ void __launch_bounds__(F_THREADS, 4) ntt16_inv_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
     __shared__ u64 sm[256 * 16];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
-    if ((blockIdx.y & 7) < fp_share) {
+    if (ALLFP || (blockIdx.y & 7) < fp_share) {
         const double q = c.modd[prime].x, qinv = c.modd[prime].y;
         const double *tw = c.twd_inv + ((size_t)prime << 16);
         const uint32_t cc = threadIdx.x & 15, r = threadIdx.x >> 4;
@@ -490,6 +498,7 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_inv_cols(DevTables c, u64 
         for (uint32_t k = 0; k < 16; k++) g[(size_t)(r + 16 * k) * 256] = canonical_d(mulmod_d<0>(x[k], ni, q), q);   // |x| <= 2q < 2^51
         return;
     }
+    if (ALLFP) return;
     const u64 q = c.mod[prime];
     const ulonglong2 *tw = c.tw_inv + ((size_t)prime << 16);
     const uint32_t cc = threadIdx.x & 15, r = threadIdx.x >> 4;
@@ -523,11 +532,21 @@ void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbM
             if (!inverse) {
                 // an epilogue is only implemented on the double-precision path, so it takes all limbs there
                 const uint32_t share = (ep || coef_src) ? 8 : c->ntt_fp_share;
-                ntt16_fwd_cols<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, coef_src); count_launches();
-                ntt16_fwd_rows<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, ep ? ep->mode : 0, ep ? *ep : NttEpilogue{}); count_launches();
+                if (share >= 8) ntt16_fwd_cols<true><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, coef_src);
+                else ntt16_fwd_cols<false><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, coef_src);
+                count_launches();
+                if (share < 8) ntt16_fwd_rows<false, 0><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, NttEpilogue{});
+                else if (!ep) ntt16_fwd_rows<true, 0><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, NttEpilogue{});
+                else if (ep->mode == 1) ntt16_fwd_rows<true, 1><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, *ep);
+                else ntt16_fwd_rows<true, 2><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, *ep);
+                count_launches();
             } else {
-                ntt16_inv_rows<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share); count_launches();
-                ntt16_inv_cols<<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share); count_launches();
+                if (c->ntt_fp_share >= 8) ntt16_inv_rows<true><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, 8);
+                else ntt16_inv_rows<false><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share);
+                count_launches();
+                if (c->ntt_fp_share >= 8) ntt16_inv_cols<true><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, 8);
+                else ntt16_inv_cols<false><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share);
+                count_launches();
             }
             y0 += ny;
         }
