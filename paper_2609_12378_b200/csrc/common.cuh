@@ -39,6 +39,7 @@ struct DevTables {
     const u64 *dn_hat_mod;         // [L][K]   Phat_k mod q_i
     const double2 *dn_hat_mod_d;   // [L][K]   {c, c / q_i} as doubles
     const ulonglong2 *dn_p_inv;    // [L]      {P^-1 mod q_i, Shoup}
+    const double2 *dn_p_inv_d;     // [L]      {P^-1 mod q_i, that / q_i} as doubles
     // Rescale: [L(last)][L(i)] {q_last^-1 mod q_i, Shoup}
     const ulonglong2 *rs_inv;
     // Encode:

@@ -359,8 +359,7 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 
         }
         if (has_ep) {      // ModDown tail: (u - NTT(conv)) P^-1 + sigma_g(add), written to its final place
             const uint32_t y = blockIdx.y, i = y % ep.level, comp = (y / ep.level) & 1, bz = y / (2 * ep.level);
-            const u64 qi = c.mod[prime];
-            const ulonglong2 pinv = c.dn_p_inv[i];
+            const double2 pinv = c.dn_p_inv_d[i];
             const uint32_t p0 = row * 256 + 16 * t;
             const u64 *up = ep.u + (((size_t)bz * 2 + comp) * ep.nt + i) * 65536 + p0;
             const u64 *add = comp ? ep.add1 : ep.add0;
@@ -375,10 +374,11 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 
                 if (ep.accumulate) ldg_4(dst + k, old[0], old[1], old[2], old[3]);
 #pragma unroll
                 for (uint32_t e = 0; e < 4; e++) {
-                    const u64 v = canonical_d(reduce_d(x[k + e], q, qinv), q);
-                    r[e] = mul_shoup(sub_mod(uu[e], v, qi), pinv.x, pinv.y, qi);
-                    if (add) r[e] = add_mod(r[e], add[bz * ep.add_stride + (size_t)i * 65536 + galois_src(p0 + k + e, gal, 16, 65536)], qi);
-                    if (ep.accumulate) r[e] = add_mod(r[e], old[e], qi);
+                    // all on the FP64 pipe: |u - v| < 1.5 q, times P^-1 -> |.| < 0.9 q, plus up to two residues, reduced once
+                    double v = mulmod_d<0>(__dsub_rn(u64_to_d(uu[e]), reduce_d(x[k + e], q, qinv)), pinv, q);
+                    if (add) v = __dadd_rn(v, u64_to_d(add[bz * ep.add_stride + (size_t)i * 65536 + galois_src(p0 + k + e, gal, 16, 65536)]));
+                    if (ep.accumulate) v = __dadd_rn(v, u64_to_d(old[e]));
+                    r[e] = canonical_d(reduce_d(v, q, qinv), q);
                 }
                 stg_4(dst + k, r[0], r[1], r[2], r[3]);
             }
