@@ -303,7 +303,7 @@ def run_cuda(args):
 
     pk, pk_kind = peaks()
     limb_ntts = NTT_BATCH * L
-    # Roofline of the dominant kernel family (the four ntt16 kernels: 36 % of the step in the ncu launch list).
+    # Roofline of the dominant kernel family (the ntt16 kernels: 44 % of the step in the ncu launch list).
     # The butterflies run on the FP64 pipe, which ncu shows to be the busiest unit of the column passes, so the
     # bound is "alu": algorithmic work = 8 FP64 instructions per butterfly (6 for the exact twiddle product with
     # its quotient, 2 for the sum and difference), N/2 * log2 N butterflies per limb; peak = 64 FP64 instructions
@@ -316,13 +316,15 @@ def run_cuda(args):
     hbm_achieved = ntt_bytes / (ntt_fwd_ms * 1e-3) / 1e9
     roofline = {"kernel": "ntt16_fwd_cols + ntt16_fwd_rows (forward NTT of 768 limbs, one launch each)", "bound": "alu",
                 "achieved": achieved, "peak": fp64_peak, "unit": "T FP64 instr/s", "frac": achieved / fp64_peak,
-                "traffic": 1574.0e6,   # ncu: dram read+write of the two launches (profiles/ntt16_768limbs.md), bytes
+                "traffic": 1538.0e6,   # ncu: dram read+write of the two launches (profiles/ntt16_768limbs.md), bytes
+                "fp64_pipe_active_ncu": {"ntt16_fwd_cols": 0.761, "ntt16_fwd_rows": 0.677},
                 "peak_kind": "derived: 64 DFMA/clk/SM x %d SMs x %.0f MHz" % (sm_count, float(pk.get("sm_max_mhz", 1965.0))),
                 "ms_per_launch_pair": ntt_fwd_ms,
                 "hbm": {"achieved": hbm_achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": hbm_achieved / pk["hbm_gbs"],
                         "algorithmic_bytes": ntt_bytes, "peak_kind": pk_kind + " copy bandwidth"},
-                "others": {"mac_mma_kernel": "19.5 % of the step; legacy mma.sync issue bound, see profiles/mac_mma_projection_8shards.md",
-                           "inner_product_kernel": "12.9 % of the step; HBM bound (key stream)"}}
+                "others": {"ntt16 family": "43.9 % of the step (profiles/bench_step_launch_list.md)",
+                           "mac_mma_kernel": "23.7 % of the step; latency bound around legacy mma.sync, see profiles/mac_mma_projection_8shards.md",
+                           "inner_product_kernel": "11.6 % of the step; FP64 products over the key stream"}}
     cpu = oracle_sample()
     jm = job_metrics(world, a_ms, b_ms, c_ms)
     line = {
