@@ -31,16 +31,28 @@ inline uint32_t conv_chunk(uint32_t nb) { return nb >= 4 ? 32 : 8; }
 // deval: d in the evaluation domain, read through sigma_g for the digit's own limbs.
 // A thread owns one coefficient of one digit: it forms the centred y_a of the digit's limbs once and then
 // walks a chunk of CHUNK target limbs (blockIdx.y), so the source limbs are read once per chunk.
+constexpr uint32_t CONV_CHUNK_MAX = 32;
+
 template <uint32_t ALPHA>
 __global__ void __launch_bounds__(THREADS) modup_kernel(DevTables c, const u64 *dcoef, const u64 *deval, size_t deval_stride, u64 g,
                                                         u64 *ext, uint32_t level, uint32_t CHUNK) {
+    // the CTA's conversion constants (qhat_a mod t and its quotient by t; t and 1/t), fetched once: as global loads
+    // inside the loop they kept the L1 busier than the arithmetic kept the FP64 pipe
+    __shared__ double2 s_w[CONV_CHUNK_MAX][ALPHA];
+    __shared__ double2 s_m[CONV_CHUNK_MAX];
     const uint32_t k = blockIdx.x * THREADS + threadIdx.x;
     const uint32_t beta = (level + c.alpha - 1) / c.alpha, j = blockIdx.z % beta, bz = blockIdx.z / beta;
     const uint32_t nt = level + c.K, lo = j * c.alpha, hi = min(lo + c.alpha, level), nd = hi - lo;
+    const uint32_t x0 = blockIdx.y * CHUNK, x1 = min(x0 + CHUNK, nt);
+    const size_t cb = ((size_t)level * c.dnum + j) * c.alpha;
+    for (uint32_t e = threadIdx.x; e < (x1 - x0) * ALPHA; e += THREADS) {
+        const uint32_t xi = e / ALPHA, a = e % ALPHA, x = x0 + xi, t = x < level ? x : c.L + (x - level);
+        s_w[xi][a] = a < nd ? c.up_hat_mod_d[(cb + a) * c.T + t] : make_double2(0.0, 0.0);
+        if (a == 0) s_m[xi] = c.modd[t];
+    }
     dcoef += (size_t)bz * level * c.N;
     deval += bz * deval_stride;
     ext += (size_t)bz * beta * nt * c.N;
-    const size_t cb = ((size_t)level * c.dnum + j) * c.alpha;
     // centred y_a = [d_a qhat_a^-1] as signed doubles (integer Shoup product, then the lift)
     double y[ALPHA];
 #pragma unroll
@@ -53,21 +65,21 @@ __global__ void __launch_bounds__(THREADS) modup_kernel(DevTables c, const u64 *
             y[a] = v > (qa >> 1) ? __dsub_rn(u64_to_d(v), (double)qa) : u64_to_d(v);
         }
     }
-    const uint32_t x0 = blockIdx.y * CHUNK, x1 = min(x0 + CHUNK, nt);
-    for (uint32_t x = x0; x < x1; x++) {
-        u64 *dst = ext + ((size_t)j * nt + x) * c.N + k;
+    __syncthreads();
+    u64 *dst = ext + ((size_t)j * nt + x0) * c.N + k;
+    for (uint32_t x = x0; x < x1; x++, dst += c.N) {
         if (x >= lo && x < hi) {
             *dst = deval[(size_t)x * c.N + galois_src(k, g, c.log_n, c.N)];
             continue;
         }
-        const uint32_t t = x < level ? x : c.L + (x - level);
-        const double2 md = c.modd[t];
+        const double2 md = s_m[x - x0];
         const double mt = md.x, mtinv = md.y;
-        // each product is reduced to |r| <= 0.57 m_t on the FP64 pipe; eight of them stay far below 2^53
+        // each product is reduced to |r| <= 0.57 m_t on the FP64 pipe; eight of them stay far below 2^53 (a missing
+        // source has y = 0 and a zero constant)
         double acc = 0.0;
 #pragma unroll
         for (uint32_t a = 0; a < ALPHA; a++) {
-            if (a < nd) acc = __dadd_rn(acc, mulmod_d<0>(y[a], c.up_hat_mod_d[(cb + a) * c.T + t], mt));
+            acc = __dadd_rn(acc, mulmod_d<0>(y[a], s_w[x - x0][a], mt));
             if ((a & 7) == 7 && a + 1 < ALPHA) acc = reduce_d(acc, mt, mtinv);
         }
         *dst = canonical_d(reduce_d(acc, mt, mtinv), mt);
@@ -83,9 +95,9 @@ void launch_modup(const ckks_ctx *c, const u64 *dcoef, const u64 *deval, size_t 
     count_launches();
 }
 
-// u[comp][x][p] = sum_j ext[j][x][pi_g(p)] * evk[j][comp][kt(x)][p]
-__global__ void __launch_bounds__(THREADS) inner_product_kernel(DevTables c, const u64 *ext, const u64 *evk, u64 g,
-                                                                u64 *u, uint32_t level, int has_multi, KsMulti multi) {
+// u[comp][x][p] = sum_j ext[j][x][pi_g(p)] * evk[j][comp][kt(x)][p]          (any number of digits)
+__global__ void __launch_bounds__(THREADS) inner_product_generic_kernel(DevTables c, const u64 *ext, const u64 *evk, u64 g,
+                                                                        u64 *u, uint32_t level, int has_multi, KsMulti multi) {
     const uint32_t p = blockIdx.x * THREADS + threadIdx.x;
     const uint32_t x = blockIdx.z, bz = blockIdx.y;     // batch varies faster than the limb: a key limb is reused from L2
     const uint32_t nt = level + c.K, beta = (level + c.alpha - 1) / c.alpha;
@@ -107,13 +119,71 @@ __global__ void __launch_bounds__(THREADS) inner_product_kernel(DevTables c, con
     u[((size_t)1 * nt + x) * c.N + p] = canonical_d(reduce_d(a1, md.x, md.y), md.x);
 }
 
+// The same for BETA <= 4 digits, two adjacent coefficients per thread.  pi_g maps the pair (p, p + 1), p even, onto a
+// pair (s, s ^ 1), so digits and key words both move as 16-byte loads.  Without `multi` a thread walks `bch` batch
+// entries (blockIdx.z picks the chunk) with the key words of its pair held in registers; with it, an entry is one
+// of up to KS_MULTI keys applied to the same digits.
+constexpr uint32_t IP_MAX_BETA = 4;
+template <uint32_t BETA>
+__global__ void __launch_bounds__(THREADS) inner_product_kernel(DevTables c, const u64 *ext, const u64 *evk, u64 g, u64 *u,
+                                                                uint32_t level, uint32_t nb, uint32_t bch, int has_multi, KsMulti multi) {
+    const uint32_t p = (blockIdx.x * THREADS + threadIdx.x) * 2;
+    const uint32_t x = blockIdx.y, b0 = blockIdx.z * bch, b1 = min(b0 + bch, nb);
+    const uint32_t nt = level + c.K;
+    const uint32_t kt = x < level ? x : c.L + (x - level);
+    const double2 md = c.modd[kt];
+    const size_t js = (size_t)nt * c.N, ks = (size_t)c.T * c.N;
+    if (has_multi) { evk = multi.evk[b0]; g = multi.galois[b0]; }
+    const uint32_t src = galois_src(p, g, c.log_n, c.N);
+    const bool odd = src & 1;
+    double k[BETA][2][2];                         // [digit][component][coefficient of the pair]
+#pragma unroll
+    for (uint32_t j = 0; j < BETA; j++)
+#pragma unroll
+        for (uint32_t cm = 0; cm < 2; cm++) {
+            const ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(evk + ((size_t)j * 2 + cm) * ks + (size_t)kt * c.N + p);
+            k[j][cm][0] = u64_to_d(v.x);
+            k[j][cm][1] = u64_to_d(v.y);
+        }
+    const u64 *e = ext + (has_multi ? 0 : b0 * BETA * js) + (size_t)x * c.N + (src & ~1u);
+    u64 *o = u + b0 * 2 * js + (size_t)x * c.N + p;
+    for (uint32_t b = b0; b < b1; b++, e += BETA * js, o += 2 * js) {
+        double acc[2][2] = {{0.0, 0.0}, {0.0, 0.0}};
+#pragma unroll
+        for (uint32_t j = 0; j < BETA; j++) {
+            const ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(e + j * js);
+            const double d0 = u64_to_d(odd ? v.y : v.x), d1 = u64_to_d(odd ? v.x : v.y);
+#pragma unroll
+            for (uint32_t cm = 0; cm < 2; cm++) {
+                acc[cm][0] = __dadd_rn(acc[cm][0], mulmod_dd(d0, k[j][cm][0], md.x, md.y));
+                acc[cm][1] = __dadd_rn(acc[cm][1], mulmod_dd(d1, k[j][cm][1], md.x, md.y));
+            }
+        }
+#pragma unroll
+        for (uint32_t cm = 0; cm < 2; cm++) {
+            ulonglong2 r;
+            r.x = canonical_d(reduce_d(acc[cm][0], md.x, md.y), md.x);
+            r.y = canonical_d(reduce_d(acc[cm][1], md.x, md.y), md.x);
+            *reinterpret_cast<ulonglong2 *>(o + cm * js) = r;
+        }
+    }
+}
+
 // conv[comp][i][k] = sum_a centre([u_{p_a} Phat_a^-1]) (Phat_a mod q_i)  mod q_i   (coefficient domain)
 // Same shape as ModUp: the K centred special residues are formed once per thread, then a chunk of targets is walked.
 template <uint32_t KK>
 __global__ void __launch_bounds__(THREADS) moddown_conv_kernel(DevTables c, const u64 *u, u64 *conv, uint32_t level, uint32_t CHUNK) {
+    __shared__ double2 s_w[CONV_CHUNK_MAX][KK];     // Phat_a mod q_i and its quotient by q_i
+    __shared__ double2 s_m[CONV_CHUNK_MAX];         // q_i, 1 / q_i
     const uint32_t k = blockIdx.x * THREADS + threadIdx.x;
     const uint32_t comp = blockIdx.z & 1, bz = blockIdx.z >> 1;
     const uint32_t nt = level + c.K;
+    const uint32_t i0 = blockIdx.y * CHUNK, i1 = min(i0 + CHUNK, level);
+    for (uint32_t e = threadIdx.x; e < (i1 - i0) * KK; e += THREADS) {
+        const uint32_t ii = e / KK, a = e % KK;
+        s_w[ii][a] = a < c.K ? c.dn_hat_mod_d[(size_t)(i0 + ii) * c.K + a] : make_double2(0.0, 0.0);
+        if (a == 0) s_m[ii] = c.modd[i0 + ii];
+    }
     u += (size_t)bz * 2 * nt * c.N;
     conv += (size_t)bz * 2 * level * c.N;
     double y[KK];
@@ -127,17 +197,18 @@ __global__ void __launch_bounds__(THREADS) moddown_conv_kernel(DevTables c, cons
             y[a] = v > (pa >> 1) ? __dsub_rn(u64_to_d(v), (double)pa) : u64_to_d(v);
         }
     }
-    const uint32_t i0 = blockIdx.y * CHUNK, i1 = min(i0 + CHUNK, level);
-    for (uint32_t i = i0; i < i1; i++) {
-        const double2 md = c.modd[i];
+    __syncthreads();
+    u64 *dst = conv + ((size_t)comp * level + i0) * c.N + k;
+    for (uint32_t i = i0; i < i1; i++, dst += c.N) {
+        const double2 md = s_m[i - i0];
         const double q = md.x, qinv = md.y;
         double acc = 0.0;
 #pragma unroll
         for (uint32_t a = 0; a < KK; a++) {
-            if (a < c.K) acc = __dadd_rn(acc, mulmod_d<0>(y[a], c.dn_hat_mod_d[(size_t)i * c.K + a], q));
+            acc = __dadd_rn(acc, mulmod_d<0>(y[a], s_w[i - i0][a], q));
             if ((a & 7) == 7 && a + 1 < KK) acc = reduce_d(acc, q, qinv);
         }
-        conv[((size_t)comp * level + i) * c.N + k] = canonical_d(reduce_d(acc, q, qinv), q);
+        *dst = canonical_d(reduce_d(acc, q, qinv), q);
     }
 }
 
@@ -238,8 +309,25 @@ void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext
                       const u64 *add0, const u64 *add1, u64 add_galois, u64 *out, cudaStream_t s, uint32_t nb,
                       size_t add_stride, size_t out_stride, bool accumulate, TiledOut tiled, const KsMulti *multi) {
     const uint32_t N = c->N, nt = level + c->K, K = c->K;
-    inner_product_kernel<<<dim3(N / THREADS, nb, nt), THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, multi ? 1 : 0,
-                                                                         multi ? *multi : KsMulti{});
+    const uint32_t beta = (level + c->alpha - 1) / c->alpha;
+    bool aligned = ((uintptr_t)w.ext & 15) == 0 && ((uintptr_t)w.u & 15) == 0 && (multi || ((uintptr_t)evk & 15) == 0);
+    if (multi)
+        for (uint32_t b = 0; b < nb; b++) aligned = aligned && ((uintptr_t)multi->evk[b] & 15) == 0;
+    if (beta <= IP_MAX_BETA && N >= 2 * THREADS && aligned) {
+        // batch entries per thread: enough chunks left to fill the machine, key words reused across a chunk
+        const uint32_t bch = multi ? 1 : (nb >= 8 ? 4 : (nb >= 4 ? 2 : 1));
+        const dim3 grid(N / (2 * THREADS), nt, (nb + bch - 1) / bch);
+        const KsMulti m = multi ? *multi : KsMulti{};
+        switch (beta) {
+        case 1: inner_product_kernel<1><<<grid, THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, nb, bch, multi ? 1 : 0, m); break;
+        case 2: inner_product_kernel<2><<<grid, THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, nb, bch, multi ? 1 : 0, m); break;
+        case 3: inner_product_kernel<3><<<grid, THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, nb, bch, multi ? 1 : 0, m); break;
+        default: inner_product_kernel<4><<<grid, THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, nb, bch, multi ? 1 : 0, m); break;
+        }
+    } else {
+        inner_product_generic_kernel<<<dim3(N / THREADS, nb, nt), THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, multi ? 1 : 0,
+                                                                                     multi ? *multi : KsMulti{});
+    }
     count_launches();
     // the K special limbs of every (batch, component): groups of K limbs, nt limbs apart
     launch_ntt(c, w.u + (size_t)level * N, nb * 2 * K, pitched_map(c->L, K, nt), true, s);
