@@ -32,7 +32,7 @@ struct Geo {
     static constexpr uint32_t BOX_BYTES = MG * GPITCH;              // one operand of one stage
     static constexpr uint32_t STAGE_BYTES = 2 * BOX_BYTES;
     static constexpr uint32_t OBUF_BYTES = MG * MS * COEF * 8;      // one tile of results, staged for whole-row stores
-    static constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + OBUF_BYTES + 128 /* alignment slack */;
+    static constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + OBUF_BYTES + 64 /* mbarriers */ + 128 /* alignment slack */;
     // byte offset of (block a, row j, 16-byte chunk ch) inside an operand tile
     static __device__ __forceinline__ uint32_t tile_off(uint32_t a, uint32_t j, uint32_t ch) {
         return a * GPITCH + (((j * CH + ch) ^ (((j >> 2) & 3) * (4 / CH))) << 4);
@@ -267,12 +267,232 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_kernel(DevTa
     if (pend) flush();
 }
 
+// ---------------------------------------------------------------------------
+// The same computation without CTA-wide barriers.  Each ring stage has a "full" mbarrier (every thread's cp.async
+// arrive on it as they complete) and an "empty" one (a warp arrives when it has read its fragments), and the result
+// staging buffer has the same pair, so warps drift up to a step apart: while one splits bytes or reduces results,
+// another keeps the tensor pipe busy.  Every wait is bounded by the clock; on a timeout the kernel raises the
+// context's sticky timeout flag and returns.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cp_async(uint32_t bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+constexpr long long MBAR_WAIT_CYCLES = 2000000000ll;      // about a second
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    const long long t0 = clock64();
+    for (;;) {
+        uint32_t ok;
+        asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+        if (clock64() - t0 > MBAR_WAIT_CYCLES) return false;
+    }
+}
+
 template <uint32_t COEF, uint32_t NW>
+__global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_async_kernel(DevTables c, const u64 *__restrict__ baby,
+                                                                                 const u64 *__restrict__ pts, u64 *__restrict__ acc,
+                                                                                 uint32_t J, uint32_t S, uint32_t G, uint32_t level,
+                                                                                 uint32_t ntiles) {
+    using T = Geo<COEF>;
+    constexpr uint32_t THREADS = COEF * 64 / NW, CH = T::CH, NWARPS = THREADS / 32;
+    constexpr uint32_t AH = THREADS / (CH * MK), NIT = MG / AH, XB64 = 64 / COEF;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *ring = reinterpret_cast<uint8_t *>(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    u64 *obuf = reinterpret_cast<u64 *>(ring + STAGES * T::STAGE_BYTES);
+    // mbarriers behind the staging buffer: full[STAGES], empty[STAGES], results full, results empty
+    const uint32_t bars = (uint32_t)__cvta_generic_to_shared(ring) + STAGES * T::STAGE_BYTES + T::OBUF_BYTES;
+    const uint32_t bar_ofull = bars + 2 * STAGES * 8, bar_oempty = bar_ofull + 8;
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, gid = lane >> 2, tig = lane & 3;
+    if (tid == 0) {
+        for (uint32_t k = 0; k < STAGES; k++) { mbar_init(bars + 8 * k, THREADS); mbar_init(bars + 8 * (STAGES + k), NWARPS); }
+        mbar_init(bar_ofull, NWARPS);
+        mbar_init(bar_oempty, NWARPS);
+    }
+    __syncthreads();
+    const uint32_t coef = NW == 2 ? warp : warp >> 1, n0 = NW == 2 ? 0 : (warp & 1);
+    const uint32_t ncol = 2 * S, coltiles = (ncol + MS - 1) / MS, gtiles = (G + MG - 1) / MG;
+    const uint32_t xblocks = c.N / COEF;
+    const uint32_t nk = J / MK;
+    const uint32_t t_begin = (uint32_t)(((u64)ntiles * blockIdx.x) / gridDim.x), t_end = (uint32_t)(((u64)ntiles * (blockIdx.x + 1)) / gridDim.x);
+    const uint32_t nsteps = (t_end - t_begin) * nk;
+
+    const uint32_t ch = tid % CH, jj = (tid / CH) % MK, arow = tid / (CH * MK);
+    const uint32_t Rw = G * J, Rx = 2 * S * J;
+    const uint32_t sm_thread = (uint32_t)__cvta_generic_to_shared(ring) + T::tile_off(arow, jj, ch);
+    TileIt lt;
+    lt.init(t_begin, coltiles, gtiles, xblocks);
+    uint32_t lks = 0, lstep = 0, lslot = 0, luse = 0;      // luse: how many times the loader has wrapped the ring
+    const u64 *wrow = nullptr, *xrow = nullptr;
+    uint32_t lg0 = 0, lsh0 = 0, lsm = 0;
+    bool alive = true;
+    // addresses of the next step to load; waits until every warp has read the stage's previous contents
+    auto load_begin = [&]() {
+        if (lstep < nsteps) {
+            const size_t blk = (size_t)lt.i * (c.N >> 6) + lt.xb / XB64;
+            const uint32_t in_blk = (lt.xb % XB64) * COEF + 2 * ch, j = lks * MK + jj;
+            wrow = pts + blk * Rw * 64 + in_blk + (size_t)j * 64;
+            xrow = baby + blk * Rx * 64 + in_blk + (size_t)(2 * j + (arow & 1)) * 64;
+            lg0 = lt.zg * MG + arow;
+            lsh0 = lt.zc * (MS / 2) + (arow >> 1);
+            lsm = sm_thread + lslot * T::STAGE_BYTES;
+            if (luse > 0 && !mbar_wait(bars + 8 * (STAGES + lslot), (luse - 1) & 1)) alive = false;
+        }
+    };
+    auto load_w = [&](uint32_t k) {
+        if (lstep < nsteps) {
+            const uint32_t g = min(lg0 + AH * k, G - 1);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(lsm + k * AH * T::GPITCH), "l"(wrow + (size_t)g * J * 64) : "memory");
+        }
+    };
+    auto load_x = [&](uint32_t k) {
+        if (lstep < nsteps) {
+            const uint32_t sh = min(lsh0 + (AH / 2) * k, S - 1);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(lsm + T::BOX_BYTES + k * AH * T::GPITCH), "l"(xrow + (size_t)sh * J * 128)
+                         : "memory");
+        }
+    };
+    auto load_end = [&]() {
+        if (lstep < nsteps) mbar_arrive_cp_async(bars + 8 * lslot);
+        lstep++;
+        if (++lslot == STAGES) { lslot = 0; luse++; }
+        if (++lks == nk) { lks = 0; lt.next(coltiles, gtiles, xblocks); }
+    };
+#pragma unroll 1
+    for (uint32_t s = 0; s < STAGES - 1; s++) {
+        load_begin();
+#pragma unroll
+        for (uint32_t k = 0; k < NIT; k++) { load_w(k); load_x(k); }
+        load_end();
+    }
+
+    TileIt ct;
+    ct.init(t_begin, coltiles, gtiles, xblocks);
+    uint32_t ks = 0, slot = 0, use = 0, qi = ct.i, tiles_done = 0;
+    u64 q = c.mod[qi], mu = c.mu[qi];
+    int dsum[NW][13][4];
+    u64 *pend = nullptr;
+    uint32_t pend_g0 = 0, pend_col0 = 0, pend_tile = 0;
+    const size_t lN = (size_t)level * c.N;
+    auto flush = [&]() {
+        if (!mbar_wait(bar_ofull, pend_tile & 1)) alive = false;
+#pragma unroll
+        for (uint32_t k = 0; k < MG * MS * COEF / THREADS; k++) {
+            const uint32_t row = k * (THREADS / COEF) + tid / COEF, sl = tid % COEF, gl = row >> 4, cl = row & 15;
+            const uint32_t g = pend_g0 + gl, col = pend_col0 + cl;
+            if (alive && g < G && col < ncol) pend[((size_t)g * ncol + col) * lN + (sl ^ (gl % COEF))] = obuf[row * COEF + sl];
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_oempty);
+        pend = nullptr;
+    };
+#pragma unroll 1
+    for (uint32_t step = 0; step < nsteps && alive; step++) {
+        if (ks == 0) {
+#pragma unroll
+            for (uint32_t n = 0; n < NW; n++)
+#pragma unroll
+                for (uint32_t d = 0; d < 13; d++)
+#pragma unroll
+                    for (uint32_t r = 0; r < 4; r++) dsum[n][d][r] = 0;
+        }
+        if (!mbar_wait(bars + 8 * slot, use & 1)) { alive = false; break; }
+        const uint8_t *Wt = ring + (size_t)slot * T::STAGE_BYTES, *Xt = Wt + T::BOX_BYTES;
+        uint32_t A[7][4];
+#pragma unroll
+        for (uint32_t r = 0; r < 2; r++)
+#pragma unroll
+            for (uint32_t h = 0; h < 2; h++) {
+                u64 w[4];
+                uint32_t f[7];
+#pragma unroll
+                for (uint32_t e = 0; e < 4; e++) w[e] = T::tile_word(Wt, gid + 8 * r, 16 * h + 4 * tig + e, coef);
+                planes7(w, f);
+#pragma unroll
+                for (uint32_t pl = 0; pl < 7; pl++) A[pl][r + 2 * h] = f[pl];
+            }
+#pragma unroll
+        for (uint32_t n = 0; n < NW; n++) {
+            uint32_t Bf[7][2];
+#pragma unroll
+            for (uint32_t h = 0; h < 2; h++) {
+                u64 x[4];
+                uint32_t f[7];
+#pragma unroll
+                for (uint32_t e = 0; e < 4; e++) x[e] = T::tile_word(Xt, 8 * (n0 + n) + gid, 16 * h + 4 * tig + e, coef);
+                planes7(x, f);
+#pragma unroll
+                for (uint32_t pl = 0; pl < 7; pl++) Bf[pl][h] = f[pl];
+            }
+            if (n == NW - 1) {
+                // this warp is done with the stage; the loads of the next-but-one step start now, a few between
+                // the products of each plane a
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bars + 8 * (STAGES + slot));
+                load_begin();
+            }
+#pragma unroll
+            for (uint32_t a = 0; a < 7; a++) {
+#pragma unroll
+                for (uint32_t b = 0; b < 7; b++) mma_u8(dsum[n][a + b], A[a], Bf[b]);
+                if (n == NW - 1) {
+                    constexpr uint32_t NCP = 2 * NIT;
+#pragma unroll
+                    for (uint32_t k = 0; k < NCP; k++)
+                        if (k * 7 / NCP == a) {
+                            if (k < NIT) load_w(k); else load_x(k - NIT);
+                        }
+                }
+            }
+        }
+        load_end();
+        if (pend) flush();
+        if (ks == nk - 1 && alive) {
+            if (ct.i != qi) { qi = ct.i; q = c.mod[qi]; mu = c.mu[qi]; }
+            if (tiles_done > 0 && !mbar_wait(bar_oempty, (tiles_done - 1) & 1)) alive = false;
+#pragma unroll
+            for (uint32_t n = 0; n < NW; n++)
+#pragma unroll
+                for (uint32_t r = 0; r < 4; r++) {
+                    const uint32_t gl = gid + 8 * (r >> 1), cl = 8 * (n0 + n) + 2 * tig + (r & 1);
+                    u64 e[3];
+#pragma unroll
+                    for (uint32_t k = 0; k < 3; k++) {
+                        e[k] = mad_wide((uint32_t)dsum[n][4 * k + 1][r], 1u << 8, (u64)(uint32_t)dsum[n][4 * k][r]);
+                        e[k] = mad_wide((uint32_t)dsum[n][4 * k + 2][r], 1u << 16, e[k]);
+                        e[k] = mad_wide((uint32_t)dsum[n][4 * k + 3][r], 1u << 24, e[k]);
+                    }
+                    const u64 lo = e[0] + (e[1] << 32);
+                    const u64 hi = (e[1] >> 32) + e[2] + ((u64)(uint32_t)dsum[n][12][r] << 32) + (lo < e[0]);
+                    obuf[(gl * 16 + cl) * COEF + (coef ^ (gl % COEF))] = barrett112(hi, lo, q, mu);
+                }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_ofull);
+            pend_g0 = ct.zg * MG;
+            pend_col0 = ct.zc * MS;
+            pend_tile = tiles_done++;
+            pend = acc + (size_t)ct.i * c.N + ct.xb * COEF;
+        }
+        if (++ks == nk) { ks = 0; ct.next(coltiles, gtiles, xblocks); }
+        if (++slot == STAGES) { slot = 0; use++; }
+    }
+    if (pend && alive) flush();
+    asm volatile("cp.async.wait_all;\n" ::: "memory");
+    if (!alive) atomicExch(c.range_flag + 1, 1);
+}
+
+template <uint32_t COEF, uint32_t NW, bool ASYNC = false>
 bool launch_as(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level, cudaStream_t s) {
     static bool attr_set = false;
+    auto kernel = ASYNC ? mac_mma_async_kernel<COEF, NW> : mac_mma_kernel<COEF, NW>;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(mac_mma_kernel<COEF, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Geo<COEF>::SMEM_BYTES) != cudaSuccess)
-            return false;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Geo<COEF>::SMEM_BYTES) != cudaSuccess) return false;
         attr_set = true;
     }
     const uint32_t coltiles = (2 * S + MS - 1) / MS, gt = (G + MG - 1) / MG;
@@ -280,8 +500,7 @@ bool launch_as(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uin
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
     const uint32_t ctas = (uint32_t)sms * (8 / COEF);
-    mac_mma_kernel<COEF, NW><<<ntiles < ctas ? ntiles : ctas, COEF * 64 / NW, Geo<COEF>::SMEM_BYTES, s>>>(c->dev, baby, pts, acc, J, S, G, level,
-                                                                                                            ntiles);
+    kernel<<<ntiles < ctas ? ntiles : ctas, COEF * 64 / NW, Geo<COEF>::SMEM_BYTES, s>>>(c->dev, baby, pts, acc, J, S, G, level, ntiles);
     count_launches();
     return true;
 }
@@ -295,10 +514,12 @@ bool mac_mma_supported(const ckks_ctx *c, uint32_t J) { return J % MK == 0 && J 
 bool launch_mac_mma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level,
                     cudaStream_t s) {
     if (!mac_mma_supported(c, J)) return false;
-    // tuning knob: CKKS_MAC_SHAPE = 82 (8 coefficients per CTA, a warp per coefficient: the default), 81 (two warps per
-    // coefficient, 10 % slower) or 42 (4 coefficients per CTA, two CTAs per SM: the products overlap better, but operand
+    // tuning knob: CKKS_MAC_SHAPE = 82 (8 coefficients per CTA, a warp per coefficient: the default), 83 (the same
+    // without CTA-wide barriers: 7 % faster, bounded mbarrier waits), 81 (two warps per coefficient, 10 % slower) or 42 (4 coefficients per CTA, two CTAs per SM: the products overlap better, but operand
     // rows fetched 32 bytes at a time make the loads twice as slow as the whole kernel otherwise is)
-    static const int shape = [] { const char *e = getenv("CKKS_MAC_SHAPE"); return e ? atoi(e) : 82; }();
+    const char *e = getenv("CKKS_MAC_SHAPE");
+    const int shape = e ? atoi(e) : 82;
+    if (shape == 83) return launch_as<8, 2, true>(c, baby, pts, acc, J, S, G, level, s);
     if (shape == 42) return launch_as<4, 2>(c, baby, pts, acc, J, S, G, level, s);
     if (shape == 81) return launch_as<8, 1>(c, baby, pts, acc, J, S, G, level, s);
     return launch_as<8, 2>(c, baby, pts, acc, J, S, G, level, s);

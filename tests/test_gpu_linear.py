@@ -68,6 +68,16 @@ def test_projection_tensor_core_mac_path(d_in, d_out, T, S, B):
     _run(10, 4, 2, 2, 4, d_in, d_out, T, S, B, seed=440 + d_in + d_out + S)
 
 
+@pytest.mark.parametrize("shape", ["81", "83", "42"])
+def test_projection_tensor_core_mac_other_shapes(shape, monkeypatch):
+    """The kernel's other tilings (two warps per coefficient; the barrier-free pipeline; four coefficients per CTA),
+    selected by the CKKS_MAC_SHAPE tuning knob, on a case with two k-steps, two column tiles and column padding."""
+    from tests.gpu_util import context
+    monkeypatch.setenv("CKKS_MAC_SHAPE", shape)
+    ctx, _, _ = _run(10, 4, 2, 2, 4, 64, 160, 8, 9, 32, seed=450)
+    assert ctx.device_status() == 0
+
+
 def test_projection_explicit_pt_scale_and_lower_level():
     _run(10, 4, 2, 2, 3, 16, 16, 32, 1, 4, seed=410, pt_scale=2.0 ** 40, check_slots=False)
 
