@@ -254,6 +254,11 @@ bool mac_mma_supported(const ckks_ctx *c, uint32_t J);
 bool launch_mac_mma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level,
                     cudaStream_t s);
 
+// the same on tcgen05 / TMEM (mac_umma.cu); J <= 64
+bool mac_umma_supported(const ckks_ctx *c, uint32_t J);
+bool launch_mac_umma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level,
+                     cudaStream_t s);
+
 void launch_rescale(const ckks_ctx *c, const u64 *in, u64 *out, uint32_t ncomp, uint32_t level, u64 *ws, cudaStream_t s);
 
 size_t encode_workspace_bytes(const ckks_ctx *c, uint32_t batch);

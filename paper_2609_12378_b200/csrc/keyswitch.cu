@@ -121,14 +121,14 @@ __global__ void __launch_bounds__(THREADS) inner_product_generic_kernel(DevTable
 
 // The same for BETA <= 4 digits, two adjacent coefficients per thread.  pi_g maps the pair (p, p + 1), p even, onto a
 // pair (s, s ^ 1), so digits and key words both move as 16-byte loads.  Without `multi` a thread walks `bch` batch
-// entries (blockIdx.z picks the chunk) with the key words of its pair held in registers; with it, an entry is one
+// entries (blockIdx.y picks the chunk) with the key words of its pair held in registers; with it, an entry is one
 // of up to KS_MULTI keys applied to the same digits.
 constexpr uint32_t IP_MAX_BETA = 4;
 template <uint32_t BETA>
 __global__ void __launch_bounds__(THREADS) inner_product_kernel(DevTables c, const u64 *ext, const u64 *evk, u64 g, u64 *u,
                                                                 uint32_t level, uint32_t nb, uint32_t bch, int has_multi, KsMulti multi) {
     const uint32_t p = (blockIdx.x * THREADS + threadIdx.x) * 2;
-    const uint32_t x = blockIdx.y, b0 = blockIdx.z * bch, b1 = min(b0 + bch, nb);
+    const uint32_t x = blockIdx.z, b0 = blockIdx.y * bch, b1 = min(b0 + bch, nb);     // chunks of a limb run together: its key words come from L2
     const uint32_t nt = level + c.K;
     const uint32_t kt = x < level ? x : c.L + (x - level);
     const double2 md = c.modd[kt];
@@ -316,7 +316,7 @@ void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext
     if (beta <= IP_MAX_BETA && N >= 2 * THREADS && aligned) {
         // batch entries per thread: enough chunks left to fill the machine, key words reused across a chunk
         const uint32_t bch = multi ? 1 : (nb >= 8 ? 4 : (nb >= 4 ? 2 : 1));
-        const dim3 grid(N / (2 * THREADS), nt, (nb + bch - 1) / bch);
+        const dim3 grid(N / (2 * THREADS), (nb + bch - 1) / bch, nt);
         const KsMulti m = multi ? *multi : KsMulti{};
         switch (beta) {
         case 1: inner_product_kernel<1><<<grid, THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, nb, bch, multi ? 1 : 0, m); break;

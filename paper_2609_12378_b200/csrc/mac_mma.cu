@@ -519,6 +519,7 @@ bool launch_mac_mma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc
     // rows fetched 32 bytes at a time make the loads twice as slow as the whole kernel otherwise is)
     const char *e = getenv("CKKS_MAC_SHAPE");
     const int shape = e ? atoi(e) : 82;
+    if (shape == 100 && launch_mac_umma(c, baby, pts, acc, J, S, G, level, s)) return true;
     if (shape == 83) return launch_as<8, 2, true>(c, baby, pts, acc, J, S, G, level, s);
     if (shape == 42) return launch_as<4, 2>(c, baby, pts, acc, J, S, G, level, s);
     if (shape == 81) return launch_as<8, 1>(c, baby, pts, acc, J, S, G, level, s);

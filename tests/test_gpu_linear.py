@@ -68,7 +68,7 @@ def test_projection_tensor_core_mac_path(d_in, d_out, T, S, B):
     _run(10, 4, 2, 2, 4, d_in, d_out, T, S, B, seed=440 + d_in + d_out + S)
 
 
-@pytest.mark.parametrize("shape", ["81", "83", "42"])
+@pytest.mark.parametrize("shape", ["81", "83", "42", "100"])
 def test_projection_tensor_core_mac_other_shapes(shape, monkeypatch):
     """The kernel's other tilings (two warps per coefficient; the barrier-free pipeline; four coefficients per CTA),
     selected by the CKKS_MAC_SHAPE tuning knob, on a case with two k-steps, two column tiles and column padding."""
