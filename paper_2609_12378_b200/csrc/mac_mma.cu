@@ -514,7 +514,8 @@ bool mac_mma_supported(const ckks_ctx *c, uint32_t J) { return J % MK == 0 && J 
 bool launch_mac_mma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level,
                     cudaStream_t s) {
     if (!mac_mma_supported(c, J)) return false;
-    // tuning knob: CKKS_MAC_SHAPE = 82 (8 coefficients per CTA, a warp per coefficient: the default), 83 (the same
+    // tuning knob: CKKS_MAC_SHAPE = 100 (the tcgen05 / TMEM kernel of mac_umma.cu, J <= 64), 82 (mma.sync, 8 coefficients per
+    // CTA, a warp per coefficient: the default), 83 (the same
     // without CTA-wide barriers: 7 % faster, bounded mbarrier waits), 81 (two warps per coefficient, 10 % slower) or 42 (4 coefficients per CTA, two CTAs per SM: the products overlap better, but operand
     // rows fetched 32 bytes at a time make the loads twice as slow as the whole kernel otherwise is)
     const char *e = getenv("CKKS_MAC_SHAPE");

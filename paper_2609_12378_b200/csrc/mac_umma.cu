@@ -16,11 +16,18 @@
 // to the 8 coefficient tiles.
 //
 // Roles in a CTA (one per SM, persistent over blocks of 8 coefficients x 16 giants): 16 epilogue warps, one MMA
-// warp (a single thread issues), two loader warps, one store warp.  W tiles (16 giants x J, 8 coefficients) are
+// warp (a single thread issues), four loader warps, one store warp.  W tiles (16 giants x J, 8 coefficients) are
 // double-buffered per block; X tiles (8 columns x J) stream through a 2-slot ring; 8 TMEM accumulators rotate
 // between the MMA thread and the epilogue warps; finished results are staged per column group and stored as
 // 64-byte rows.  All hand-offs are mbarriers; every wait is bounded by the clock and raises the context's sticky
 // timeout flag instead of hanging.
+//
+// Status: bit-identical to mac_mma.cu and selectable with CKKS_MAC_SHAPE=100, but not the default.  On B200 a
+// giant-step group of the 4096 x 4096 projection (16 shards) takes 18.9 ms here against 13.8 ms with mma.sync: the
+// tensor pipe is idle most of the time and the 16 epilogue warps are busy 85 % of it.  With accumulators in registers
+// the products of equal weight a + b add up inside the MMA (13 sums per output); here all 49 arrive separately and
+// are folded by integer instructions (about 300 per output).  Folding them in the MMA needs the byte-shifted copies
+// of one operand along K (a Toeplitz expansion) and M = 64 giants per tile.
 #include "common.cuh"
 
 namespace {
@@ -30,7 +37,7 @@ constexpr uint32_t UG = 16;                // giants per block: M = 8 * UG = 128
 constexpr uint32_t UCG = 8;                // columns per accumulator: N = 8 * UCG = 64
 constexpr uint32_t UK = 32;                // K of one MMA
 constexpr uint32_t MAX_J = 64;
-constexpr uint32_t E_WARPS = 16, L_WARPS = 2;
+constexpr uint32_t E_WARPS = 16, L_WARPS = 4;      // loader warps: a multiple of 4 (128 threads cover 8 coefficients x 8 j x 2 parities)
 constexpr uint32_t W_MMA = E_WARPS, W_LOAD = E_WARPS + 1, W_STORE = W_LOAD + L_WARPS, U_WARPS = W_STORE + 1;
 constexpr uint32_t U_THREADS = U_WARPS * 32;
 constexpr uint32_t NACC = 8;               // TMEM accumulators of 64 columns
@@ -40,20 +47,20 @@ constexpr uint32_t B_WFULL = 0, B_WEMPTY = 2, B_XFULL = 4, B_XEMPTY = 6, B_TFULL
 
 struct Smem {
     uint32_t tsw, tsx;         // bytes per coefficient tile of W / X (padded by 16)
-    uint32_t w[2], x[2], o[2], bars, tslot, total;
+    uint32_t x0, o0, bars, tslot, total;
+    __host__ __device__ uint32_t w(uint32_t k) const { return k * UC * tsw; }             // two W buffers
+    __host__ __device__ uint32_t x(uint32_t k) const { return x0 + k * UC * tsx; }        // two X slots
+    __host__ __device__ uint32_t o(uint32_t k) const { return o0 + k * OBUF_BYTES; }      // two result buffers
 };
 __host__ __device__ inline Smem smem_plan(uint32_t J) {
     Smem s;
     s.tsw = J * 16 * (UG / 2) + 16;
     s.tsx = J * 16 * (UCG / 2) + 16;
-    uint32_t off = 0;
-    for (int k = 0; k < 2; k++) { s.w[k] = off; off += UC * s.tsw; }
-    for (int k = 0; k < 2; k++) { s.x[k] = off; off += UC * s.tsx; }
-    off = (off + 127) & ~127u;
-    for (int k = 0; k < 2; k++) { s.o[k] = off; off += OBUF_BYTES; }
-    s.bars = off; off += B_COUNT * 8;
-    s.tslot = off; off += 16;
-    s.total = off + 128;       // alignment slack
+    s.x0 = 2 * UC * s.tsw;
+    s.o0 = (s.x0 + 2 * UC * s.tsx + 127) & ~127u;
+    s.bars = s.o0 + 2 * OBUF_BYTES;
+    s.tslot = s.bars + B_COUNT * 8;
+    s.total = s.tslot + 16 + 128;       // alignment slack
     return s;
 }
 
@@ -106,20 +113,11 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
                  : "r"(taddr));
     asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
 }
-__device__ __forceinline__ u64 mad_wide(uint32_t a, uint32_t b, u64 c) {
-    u64 d;
-    asm("mad.wide.u32 %0, %1, %2, %3;\n" : "=l"(d) : "r"(a), "r"(b), "l"(c));
-    return d;
-}
 // multi-word little-endian helpers (32-bit words)
 template <int NW_IN, int NW_OUT>
-__device__ __forceinline__ void mul_small(const uint32_t (&x)[NW_IN], uint32_t m, uint32_t (&r)[NW_OUT]) {     // r = x * m, m < 2^17
-    u64 t = 0;
+__device__ __forceinline__ void shl_words(const uint32_t (&x)[NW_IN], uint32_t sh, uint32_t (&r)[NW_OUT]) {     // r = x << sh, sh < 32
 #pragma unroll
-    for (int i = 0; i < NW_OUT; i++) {
-        t = mad_wide(i < NW_IN ? x[i] : 0u, m, t >> 32);
-        r[i] = (uint32_t)t;
-    }
+    for (int i = 0; i < NW_OUT; i++) r[i] = __funnelshift_l(i ? x[i - 1] : 0u, i < NW_IN ? x[i] : 0u, sh);
 }
 template <int NWD>
 __device__ __forceinline__ void add_words(uint32_t (&a)[NWD], const uint32_t (&b)[NWD]) {
@@ -179,8 +177,10 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
 
     if (warp >= W_LOAD && warp < W_STORE) {
         // ---------------- loaders: 8-byte cp.async, lane -> coefficient p of a row piece ----------------
-        const uint32_t lt = tid - W_LOAD * 32, p = lt & 7, rs = lt >> 3;       // 8 row slots per pass
-        const uint32_t Rw = G * J, Rx = 2 * S * J;
+        // a thread keeps its coefficient p, its j mod 8 and the parity of its giant (column); it walks pairs and j / 8
+        const uint32_t lt = tid - W_LOAD * 32, p = lt & 7, jr = (lt >> 3) & 7, par = (lt >> 6) & 1, sub = lt >> 7;
+        constexpr uint32_t NSUB = L_WARPS / 4;                                  // thread groups sharing the pairs
+        const uint32_t Rw = G * J, Rx = 2 * S * J, njb = J / 8;
         BlockIt it;
         it.init(b_begin, gtiles, xblocks);
         uint32_t cgn = 0;                                                       // column groups issued so far
@@ -188,22 +188,26 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
             const size_t blk = (size_t)it.i * (c.N >> 6) + (it.xb >> 3);
             const uint32_t in_blk = (it.xb & 7) * UC + p;
             if (!wait_empty(bars, B_WEMPTY, b, 2)) { alive = false; break; }
-            const u64 *wsrc = pts + blk * Rw * 64 + in_blk;
-            const uint32_t wdst = sm0 + L.w[b & 1] + p * L.tsw;
-            for (uint32_t r = rs; r < UG * J; r += L_WARPS * 4) {
-                const uint32_t gl = r / J, j = r % J, g = min(it.zg * UG + gl, G - 1);
-                asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(wdst + (gl >> 1) * sbo + j * 16 + (gl & 1) * 8),
-                             "l"(wsrc + (size_t)(g * J + j) * 64) : "memory");
+            const u64 *wsrc = pts + blk * Rw * 64 + in_blk + (size_t)jr * 64;
+            const uint32_t wdst = sm0 + L.w(b & 1) + p * L.tsw + jr * 16 + par * 8;
+            for (uint32_t gp = sub; gp < UG / 2; gp += NSUB) {
+                const uint32_t g = min(it.zg * UG + 2 * gp + par, G - 1);
+                const u64 *src = wsrc + (size_t)g * J * 64;
+                uint32_t dst = wdst + gp * sbo;
+                for (uint32_t jb = 0; jb < njb; jb++, src += 8 * 64, dst += 128)
+                    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(dst), "l"(src) : "memory");
             }
             mbar_arrive_cp_async(bars + 8 * (B_WFULL + (b & 1)));
-            const u64 *xsrc = baby + blk * Rx * 64 + in_blk;
+            const u64 *xsrc = baby + blk * Rx * 64 + in_blk + (size_t)jr * 128;
             for (uint32_t cg = 0; cg < ncg && alive; cg++, cgn++) {
                 if (!wait_empty(bars, B_XEMPTY, cgn, 2)) { alive = false; break; }
-                const uint32_t xdst = sm0 + L.x[cgn & 1] + p * L.tsx;
-                for (uint32_t r = rs; r < UCG * J; r += L_WARPS * 4) {
-                    const uint32_t cl = r / J, j = r % J, col = min(cg * UCG + cl, ncol - 1);
-                    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(xdst + (cl >> 1) * sbo + j * 16 + (cl & 1) * 8),
-                                 "l"(xsrc + (size_t)(((col >> 1) * J + j) * 2 + (col & 1)) * 64) : "memory");
+                const uint32_t xdst = sm0 + L.x(cgn & 1) + p * L.tsx + jr * 16 + par * 8;
+                for (uint32_t cp = sub; cp < UCG / 2; cp += NSUB) {
+                    const uint32_t col = min(cg * UCG + 2 * cp + par, ncol - 1);
+                    const u64 *src = xsrc + ((size_t)(col >> 1) * J * 2 + (col & 1)) * 64;
+                    uint32_t dst = xdst + cp * sbo;
+                    for (uint32_t jb = 0; jb < njb; jb++, src += 16 * 64, dst += 128)
+                        asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(dst), "l"(src) : "memory");
                 }
                 mbar_arrive_cp_async(bars + 8 * (B_XFULL + (cgn & 1)));
             }
@@ -221,7 +225,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
                     for (uint32_t p = 0; p < UC; p++, an++) {
                         if (!wait_empty(bars, B_TEMPTY, an, NACC)) { alive = false; break; }
                         tc_fence_after();
-                        const uint32_t wa = sm0 + L.w[b & 1] + p * L.tsw, xa = sm0 + L.x[cgn & 1] + p * L.tsx;
+                        const uint32_t wa = sm0 + L.w(b & 1) + p * L.tsw, xa = sm0 + L.x(cgn & 1) + p * L.tsx;
                         for (uint32_t ks = 0; ks < nk; ks++)
                             umma_i8(tmem + (an % NACC) * 8 * UCG, umma_desc(wa + ks * UK * 16, 128, sbo), umma_desc(xa + ks * UK * 16, 128, sbo), ks);
                         tc_commit(bars + 8 * (B_TFULL + an % NACC));
@@ -241,7 +245,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
             u64 *obase = acc + (size_t)it.i * c.N + it.xb * UC;
             for (uint32_t cg = 0; cg < ncg && alive; cg++, cgn++) {
                 if (!wait_full(bars, B_OFULL, cgn, 2)) { alive = false; break; }
-                const u64 *ob = reinterpret_cast<const u64 *>(sm + L.o[cgn & 1]);
+                const u64 *ob = reinterpret_cast<const u64 *>(sm + L.o(cgn & 1));
 #pragma unroll 4
                 for (uint32_t k = 0; k < UG * UCG * UC / 32; k++) {
                     const uint32_t row = k * 4 + (lane >> 3), w = lane & 7, gl = row >> 3, cl = row & 7;
@@ -256,7 +260,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
         // ---------------- epilogue: warp = (group eg, lane quarter q); group eg takes coefficients eg and eg + 4 ----------------
         const uint32_t eg = warp >> 2, q = warp & 3;
         const uint32_t a = lane & 7, gl = 4 * q + (lane >> 3);          // TMEM lane 32 q + lane = 8 gl + a
-        const uint32_t m1 = (a & 1) ? 256u : 1u, m2 = (a & 2) ? 65536u : 1u;
+        const uint32_t sh1 = (a & 1) ? 8u : 0u, sh2 = (a & 2) ? 16u : 0u;
         const bool a0 = a & 1, a1 = a & 2, a2 = a & 4;
         BlockIt it;
         it.init(b_begin, gtiles, xblocks);
@@ -278,15 +282,13 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
 #pragma unroll
                         for (uint32_t cc = 0; cc < 4; cc++) {
                             const uint32_t *d = v + 8 * cc;
-                            u64 lo = mad_wide(d[1], 1u << 8, (u64)d[0]);
-                            lo = mad_wide(d[2], 1u << 16, lo);
-                            lo = mad_wide(d[3], 1u << 24, lo);
-                            u64 hi = mad_wide(d[5], 1u << 8, (u64)d[4]);
-                            hi = mad_wide(d[6], 1u << 16, hi);
-                            hi += lo >> 32;
+                            // every D is below 2^22 (J <= 64), so byte pairs combine in 32 bits
+                            const uint32_t t01 = d[0] + (d[1] << 8), t23 = d[2] + (d[3] << 8), t45 = d[4] + (d[5] << 8);
+                            const u64 lo = (u64)t01 + ((u64)t23 << 16);
+                            const u64 hi = (u64)t45 + ((u64)d[6] << 16) + (lo >> 32);
                             // times 2^(8 (a & 1)) before the first exchange
                             const uint32_t s[3] = {(uint32_t)lo, (uint32_t)hi, (uint32_t)(hi >> 32)};
-                            mul_small<3, 3>(s, m1, T[4 * h + cc]);
+                            shl_words<3, 3>(s, sh1, T[4 * h + cc]);
                         }
                     }
                     tc_fence_before();
@@ -310,7 +312,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
                     {
                         uint32_t X4[4][4];
 #pragma unroll
-                        for (uint32_t k = 0; k < 4; k++) mul_small<3, 4>(V[k], m2, X4[k]);
+                        for (uint32_t k = 0; k < 4; k++) shl_words<3, 4>(V[k], sh2, X4[k]);
 #pragma unroll
                         for (uint32_t k = 0; k < 2; k++) {
                             uint32_t r[4];
@@ -338,7 +340,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
                     const uint32_t cl = (a0 ? 4u : 0u) + (a1 ? 2u : 0u) + (a2 ? 1u : 0u);     // the column this lane finished
                     const u64 res = barrett112(((u64)Z[3] << 32) | Z[2], ((u64)Z[1] << 32) | Z[0], qmod, mu);
                     if (!wait_empty(bars, B_OEMPTY, cgn, 2)) { alive = false; break; }
-                    reinterpret_cast<u64 *>(sm + L.o[cgn & 1])[(gl * UCG + cl) * UC + (p ^ (gl & 7))] = res;
+                    reinterpret_cast<u64 *>(sm + L.o(cgn & 1))[(gl * UCG + cl) * UC + (p ^ (gl & 7))] = res;
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bars + 8 * (B_OFULL + (cgn & 1)));
                 }
