@@ -273,6 +273,15 @@ def run_cuda(args):
     s1.record()
     torch.cuda.synchronize()
     ntt_fwd_ms = s0.elapsed_time(s1) / reps
+    # the same butterflies on registers only (no global traffic): what the arithmetic alone sustains on this GPU
+    probe_scratch = torch.zeros(1 << 20, dtype=torch.int64, device=dev).view(torch.uint64)
+    ctx.ntt_butterfly_probe(64, probe_scratch)
+    p0, p1 = ev(), ev()
+    p0.record()
+    probe_bfly = ctx.ntt_butterfly_probe(4096, probe_scratch)
+    p1.record()
+    torch.cuda.synchronize()
+    probe_rate = probe_bfly / (p0.elapsed_time(p1) * 1e-3)          # butterflies per second
 
     # e2e: host buffers in, host buffers out, copies inside the timed region
     def e2e_step():
@@ -320,6 +329,10 @@ def run_cuda(args):
                 "fp64_pipe_active_ncu": {"ntt16_fwd_cols": 0.761, "ntt16_fwd_rows": 0.677},
                 "peak_kind": "derived: 64 DFMA/clk/SM x %d SMs x %.0f MHz" % (sm_count, float(pk.get("sm_max_mhz", 1965.0))),
                 "ms_per_launch_pair": ntt_fwd_ms,
+                "vs_register_resident_butterflies": {
+                    "achieved_gbfly_s": limb_ntts * (N // 2) * LOG_N / (ntt_fwd_ms * 1e-3) / 1e9, "peak_gbfly_s": probe_rate / 1e9,
+                    "frac": limb_ntts * (N // 2) * LOG_N / (ntt_fwd_ms * 1e-3) / probe_rate,
+                    "peak_kind": "measured in this run: the transform's radix-16 butterfly groups on registers, 4 CTAs x 256 threads per SM"},
                 "hbm": {"achieved": hbm_achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": hbm_achieved / pk["hbm_gbs"],
                         "algorithmic_bytes": ntt_bytes, "peak_kind": pk_kind + " copy bandwidth"},
                 "others": {"ntt16 family": "54.0 % of the step (profiles/bench_step_launch_list.md)",

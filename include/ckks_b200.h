@@ -138,6 +138,15 @@ uint64_t ckks_galois_element(const ckks_ctx *ctx, int64_t left_rot_slots);
 int32_t ckks_ntt(ckks_ctx *ctx, uint64_t *polys, uint32_t batch, uint32_t first_prime, uint32_t nlimbs, void *stream);
 int32_t ckks_intt(ckks_ctx *ctx, uint64_t *polys, uint32_t batch, uint32_t first_prime, uint32_t nlimbs, void *stream);
 
+/* Measurement aid (the paper has no counterpart): runs the forward butterflies of the N = 2^16 transform on
+ * registers only -- `iters` groups of 4 stages (32 butterflies) per thread, with the transform's own range
+ * reductions and twiddle fetches, on a grid of four 256-thread CTAs per SM -- so that a caller can time the
+ * launch and compare the transform's butterflies per second with what the arithmetic alone sustains.
+ * scratch: device, at least SMs * 1024 words, never written in practice.  *butterflies (host) receives the
+ * number of butterflies of the launch.  CKKS_ERR_UNSUPPORTED unless log_n = 16. */
+int32_t ckks_ntt_butterfly_probe(ckks_ctx *ctx, uint32_t iters, uint64_t *scratch, size_t scratch_words, uint64_t *butterflies,
+                                 void *stream);
+
 /* ---- Encode (Section 2.1, Encode) ----------------------------------------
  * re, im: device, [batch][n] fp64 slot values (im may be NULL = real input).
  * out: device, [batch][level][N].  Steps: slot permutation e_j = (5^j mod 2N

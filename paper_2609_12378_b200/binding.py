@@ -22,6 +22,7 @@ EXPORTS = [
     "ckks_encode_range_flag", "ckks_mul_plain_acc", "ckks_add", "ckks_mul_relin", "ckks_rotate",
     "ckks_rotate_hoisted", "ckks_rescale", "ckks_linear_proj", "ckks_linear_proj_workspace_bytes",
     "ckks_linear_proj_rotations", "ckks_kernel_launches", "ckks_device_status", "ckks_rescale_static",
+    "ckks_ntt_butterfly_probe",
 ]
 
 
@@ -82,6 +83,7 @@ def load():
         "ckks_linear_proj": (i32, [vp, C.POINTER(CProjDesc), C.POINTER(CCt), vp, C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
         "ckks_linear_proj_workspace_bytes": (sz, [vp, C.POINTER(CProjDesc), u32]),
         "ckks_linear_proj_rotations": (i32, [vp, C.POINTER(CProjDesc), C.POINTER(i64), u32]),
+        "ckks_ntt_butterfly_probe": (i32, [vp, u32, vp, sz, C.POINTER(u64), vp]),
     }
     for name, (res, args) in sig.items():
         f = getattr(L, name)
@@ -216,6 +218,13 @@ class Context:
         batch = polys.numel() // (nl * self.N)
         self._check(load().ckks_intt(self._h, polys.data_ptr(), batch, first_prime, nl, _stream_ptr(stream)))
         return polys
+
+    def ntt_butterfly_probe(self, iters: int, scratch: torch.Tensor, stream=None) -> int:
+        """Launches the register-resident butterfly kernel; returns the number of butterflies it performs."""
+        _dev_u64(scratch)
+        n = C.c_uint64(0)
+        self._check(load().ckks_ntt_butterfly_probe(self._h, iters, scratch.data_ptr(), scratch.numel(), C.byref(n), _stream_ptr(stream)))
+        return int(n.value)
 
     def encode(self, re: torch.Tensor, im, scale: float, level: int, out: torch.Tensor = None, stream=None):
         """re/im: fp64 [batch][n] on the device -> uint64 [batch][level][N]."""

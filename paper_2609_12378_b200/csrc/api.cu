@@ -246,6 +246,18 @@ extern "C" int32_t ckks_intt(ckks_ctx *c, uint64_t *polys, uint32_t batch, uint3
     return finish(c);
 }
 
+extern "C" int32_t ckks_ntt_butterfly_probe(ckks_ctx *c, uint32_t iters, uint64_t *scratch, size_t scratch_words, uint64_t *butterflies,
+                                            void *stream) {
+    if (!c || !scratch || !iters || !butterflies) return CKKS_ERR_ARG;
+    if (c->log_n != 16) return CKKS_ERR_UNSUPPORTED;
+    DeviceGuard g(c->device);
+    int sms = 148;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
+    if (scratch_words < (size_t)sms * 4 * 256) return CKKS_ERR_WORKSPACE;
+    *butterflies = launch_butterfly_probe(c, iters, (u64 *)scratch, (cudaStream_t)stream);
+    return finish(c);
+}
+
 extern "C" int32_t ckks_encode(ckks_ctx *c, const double *re, const double *im, uint32_t batch, double scale, uint32_t level,
                                uint64_t *out, void *ws, size_t ws_bytes, void *stream) {
     if (!c || !re || !out || !batch || !(scale > 0.0) || !isfinite(scale)) return CKKS_ERR_ARG;

@@ -254,6 +254,9 @@ bool mac_mma_supported(const ckks_ctx *c, uint32_t J);
 bool launch_mac_mma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level,
                     cudaStream_t s);
 
+// register-resident forward butterflies (measurement aid, ntt.cu); sink: device scratch of SMs * 4 * 256 words
+uint64_t launch_butterfly_probe(const ckks_ctx *c, uint32_t iters, u64 *sink, cudaStream_t s);
+
 // the same on tcgen05 / TMEM (mac_umma.cu); J <= 64
 bool mac_umma_supported(const ckks_ctx *c, uint32_t J);
 bool launch_mac_umma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level,

@@ -265,6 +265,26 @@ __device__ __forceinline__ void inv16_d(double (&x)[16], const double *__restric
     inv_stage_d<1>(x, tw, base, q, qinv);
 }
 
+// ---- measurement aid: the forward butterflies of the N = 2^16 kernels on registers only ------------------
+// Every thread runs `iters` radix-16 groups (4 stages, 32 butterflies, with the same range reductions and twiddle
+// fetches, the latter from a 64 KiB window that stays in L1/L2) on 16 registers; nothing else touches memory.
+__global__ void __launch_bounds__(F_THREADS, 4) butterfly_probe_kernel(DevTables c, uint32_t iters, u64 *sink) {
+    const double q = c.modd[0].x, qinv = c.modd[0].y;
+    const double *tw = c.twd_fwd;
+    double x[16];
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) x[k] = (double)(threadIdx.x * 16 + k + 1);
+    uint32_t base = 16 + (threadIdx.x & 255);
+    for (uint32_t it = 0; it < iters; it++) {
+        fwd16_d(x, tw, base, q, qinv);
+        base = 16 + ((base * 5 + 1) & 255);
+    }
+    double acc = 0.0;
+#pragma unroll
+    for (uint32_t k = 0; k < 16; k++) acc = __dadd_rn(acc, x[k]);
+    if (acc == 0.5) sink[blockIdx.x * F_THREADS + threadIdx.x] = 1;      // never true for integer-valued sums
+}
+
 // ---- forward, column pass (stages m = 1..128): CTA = strip of 16 columns -----------------
 template <bool ALLFP>
 __global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, const long long *coef_src) {
@@ -570,3 +590,14 @@ void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbM
         }
     }
 }
+
+// grid: four CTAs per SM, the residency of the transform kernels.  Returns the butterflies one launch performs.
+uint64_t launch_butterfly_probe(const ckks_ctx *c, uint32_t iters, u64 *sink, cudaStream_t s) {
+    int sms = 148;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
+    const uint32_t ctas = (uint32_t)sms * 4;
+    butterfly_probe_kernel<<<ctas, F_THREADS, 0, s>>>(c->dev, iters, sink);
+    count_launches();
+    return (uint64_t)ctas * F_THREADS * iters * 32;
+}
+

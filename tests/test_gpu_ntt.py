@@ -67,3 +67,21 @@ def test_ntt_argument_errors():
     lib = binding.load()
     assert lib.ckks_ntt(ctx._h, None, 1, 0, 1, None) == binding.ERR_ARG
     assert lib.ckks_intt(ctx._h, d.data_ptr(), 0, 0, 1, None) == binding.ERR_ARG
+
+
+def test_butterfly_probe_counts_and_errors():
+    """The register-resident butterfly kernel (measurement aid): launch count and argument checks."""
+    import torch
+    from tests.gpu_util import context
+    ctx = context(16, 24, 8, 3)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    scratch = torch.zeros(sms * 1024, dtype=torch.int64, device="cuda").view(torch.uint64)
+    assert ctx.ntt_butterfly_probe(8, scratch) == sms * 4 * 256 * 8 * 32
+    torch.cuda.synchronize()
+    assert int(scratch.view(torch.int64).abs().sum()) == 0          # the sink is never written
+    with pytest.raises(binding.CkksError) as e:
+        ctx.ntt_butterfly_probe(8, scratch[:16])
+    assert e.value.code == binding.ERR_WORKSPACE
+    with pytest.raises(binding.CkksError) as e:
+        context(10, 4, 2, 2).ntt_butterfly_probe(8, scratch)
+    assert e.value.code == binding.ERR_UNSUPPORTED
