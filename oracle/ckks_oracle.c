@@ -693,9 +693,11 @@ void orc_rotate(const orc_ctx *c, const uint64_t *ct, const uint64_t *evk, uint6
 /*
  * Hoisted rotations: one iNTT + ModUp + NTT of c1 shared by all rotations;
  * for each g: permute every extended limb of every digit by sigma_g, inner
- * product with evk_g, ModDown, add sigma_g(c0).  Not bit-identical to the
- * plain form (the centred conversion does not commute with the sign flips of
- * sigma_g), so it is its own function.  evks[r] points at key r; outs is
+ * product with evk_g, ModDown, add sigma_g(c0).  The steps are taken in
+ * this order; the result is bit-identical to the plain form because the
+ * centred conversion is odd (centre(q - v) = -centre(v) for odd q), hence
+ * commutes with the permutation and sign flips of sigma_g (pinned by a test).
+ * evks[r] points at key r; outs is
  * [nrot][2][level][N].
  */
 void orc_rotate_hoisted(const orc_ctx *c, const uint64_t *ct, const uint64_t *const *evks, const uint64_t *gs,

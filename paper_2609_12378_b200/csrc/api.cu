@@ -339,7 +339,7 @@ extern "C" int32_t ckks_mul_relin(ckks_ctx *c, const ckks_ct *a, const ckks_ct *
     KsWorkspace w = ks_carve(c, level, e2 + (size_t)level * c->N);
     u64 *o = (u64 *)out->data;
     launch_tensor(c, (const u64 *)a->data, (const u64 *)b->data, o, e2, level, s);
-    ks_modup(c, e2, 1, level, w, s);
+    ks_modup(c, e2, level, w, s);
     ks_inner_moddown(c, (const u64 *)rlk->data, level, 1, w, o, o + (size_t)level * c->N, 1, o, s);
     int rc = finish(c);
     if (rc == CKKS_OK) { out->level = level; out->ncomp = 2; out->scale = a->scale * b->scale; }
@@ -367,8 +367,8 @@ extern "C" int32_t ckks_rotate(ckks_ctx *c, const ckks_ct *in, const ckks_evk *k
     const uint32_t level = in->level;
     KsWorkspace w = ks_carve(c, level, ws);
     const u64 *c0 = (const u64 *)in->data, *c1 = c0 + (size_t)level * c->N;
-    ks_modup(c, c1, key->galois, level, w, s);
-    ks_inner_moddown(c, (const u64 *)key->data, level, 1, w, c0, nullptr, key->galois, (u64 *)out->data, s);
+    ks_modup(c, c1, level, w, s);
+    ks_inner_moddown(c, (const u64 *)key->data, level, key->galois, w, c0, nullptr, key->galois, (u64 *)out->data, s);
     rc = finish(c);
     if (rc == CKKS_OK) { out->level = level; out->ncomp = 2; out->scale = in->scale; }
     return rc;
@@ -391,7 +391,7 @@ extern "C" int32_t ckks_rotate_hoisted(ckks_ctx *c, const ckks_ct *in, const ckk
     w.u = w.ext + beta * nt * N;
     w.conv = w.u + (size_t)nbh * 2 * nt * N;
     const u64 *c0 = (const u64 *)in->data, *c1 = c0 + (size_t)level * N;
-    ks_modup(c, c1, 1, level, w, s);
+    ks_modup(c, c1, level, w, s);
     for (uint32_t r0 = 0; r0 < nrot; r0 += nbh) {
         const uint32_t nb = std::min(nbh, nrot - r0);
         KsMulti m{};
@@ -477,7 +477,7 @@ extern "C" int32_t ckks_linear_proj(ckks_ctx *c, const ckks_proj_desc *d, const 
     for (uint32_t comp = 0; comp < 2; comp++)
         launch_to_tiled(c, xin + comp * ptl, ctl, S * nib, baby, Rx, comp, 2 * B, level, s);
     if (B > 1) {
-        ks_modup(c, xin + ptl, 1, level, kw, s, S * nib, ctl);
+        ks_modup(c, xin + ptl, level, kw, s, S * nib, ctl);
         for (uint32_t b = 1; b < B; b++) {
             const u64 ge = ckks_galois_element(c, (int64_t)b * T);
             TiledOut to;
@@ -538,16 +538,16 @@ extern "C" int32_t ckks_linear_proj(ckks_ctx *c, const ckks_proj_desc *d, const 
                 const u64 ge = ckks_galois_element(c, (int64_t)gi * B * T);
                 const u64 *key = (const u64 *)find_key(keys, nkeys, ge)->data;
                 // total[sh] += rotate(acc_g[sh]) for all shards in one batch
-                ks_modup(c, ag + ptl, ge, level, kw, s, S, ctl);
-                ks_inner_moddown(c, key, level, 1, kw, ag, nullptr, ge, total, s, S, ctl, ctl, true);
+                ks_modup(c, ag + ptl, level, kw, s, S, ctl);
+                ks_inner_moddown(c, key, level, ge, kw, ag, nullptr, ge, total, s, S, ctl, ctl, true);
             }
         }
         for (uint32_t f = o.size; fold > 1; f *= 2, fold /= 2) {
             const u64 ge = ckks_galois_element(c, (int64_t)f * T);
             const u64 *key = (const u64 *)find_key(keys, nkeys, ge)->data;
             // total += rotate(total): the rotated copy goes to the (now free) accumulator buffer first
-            ks_modup(c, total + ptl, ge, level, kw, s, S, ctl);
-            ks_inner_moddown(c, key, level, 1, kw, total, nullptr, ge, acc, s, S, ctl, ctl, false);
+            ks_modup(c, total + ptl, level, kw, s, S, ctl);
+            ks_inner_moddown(c, key, level, ge, kw, total, nullptr, ge, acc, s, S, ctl, ctl, false);
             for (uint32_t sh = 0; sh < S; sh++)
                 launch_add(c, total + (size_t)sh * ctl, acc + (size_t)sh * ctl, total + (size_t)sh * ctl, 2, level, s);
         }

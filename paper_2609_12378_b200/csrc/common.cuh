@@ -221,8 +221,11 @@ struct NttEpilogue {
 };
 // coef_src (forward, N = 2^16 path only): the first pass reads signed 64-bit coefficients [batch][N] (batch = limb
 // index / map.period) and reduces them modulo the limb's prime on the fly instead of reading `base`.
+// inv_src (inverse, N = 2^16 path only): the first pass reads its limbs from another buffer whose periods start
+// inv_src_pitch limbs apart, so the transform runs out of place and the input stays intact.
 void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbMap &map, bool inverse, cudaStream_t s,
-                const NttEpilogue *ep = nullptr, const long long *coef_src = nullptr);
+                const NttEpilogue *ep = nullptr, const long long *coef_src = nullptr, const u64 *inv_src = nullptr,
+                uint32_t inv_src_pitch = 0);
 
 void launch_mul_plain_acc(const ckks_ctx *c, const u64 *const *cts, u64 *const *accs, uint32_t ncts, const u64 *pt,
                           uint32_t level, bool init, cudaStream_t s);
@@ -234,10 +237,11 @@ void launch_tensor(const ckks_ctx *c, const u64 *a, const u64 *b, u64 *e01, u64 
 struct KsWorkspace { u64 *dcoef, *ext, *u, *conv; };
 size_t ks_workspace_limbs(const ckks_ctx *c, uint32_t level);
 KsWorkspace ks_carve(const ckks_ctx *c, uint32_t level, void *ws, uint32_t nb = 1);
-// nb key switches side by side (batch entry b reads d + b * d_stride words):
-// sigma_g(d) (d evaluation domain, [level][N]; g = 1: identity) -> ext (evaluation domain, all digits)
-void ks_modup(const ckks_ctx *c, const u64 *d, u64 galois, uint32_t level, const KsWorkspace &w, cudaStream_t s, uint32_t nb = 1,
-              size_t d_stride = 0);
+// nb key switches side by side (batch entry b reads d + b * d_stride words, d_stride a multiple of N):
+// d (evaluation domain, [level][N]) -> ext (evaluation domain, all digits).  A rotation applies its sigma_g to the
+// extended digits when the inner product reads them (ext_galois below): the centred conversion commutes with the
+// permutation and the sign flips of sigma_g, so this equals extending sigma_g(d), and d is never copied.
+void ks_modup(const ckks_ctx *c, const u64 *d, uint32_t level, const KsWorkspace &w, cudaStream_t s, uint32_t nb = 1, size_t d_stride = 0);
 // inner product with evk (digits read through sigma_{ext_galois}; 1 = identity), ModDown, and the final
 // combination out_c (+)= sigma_{add_galois}(add_c) + k_c.  add0/add1 may be null.
 void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext_galois, const KsWorkspace &w,

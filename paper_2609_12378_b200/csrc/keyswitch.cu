@@ -294,12 +294,15 @@ KsWorkspace ks_carve(const ckks_ctx *c, uint32_t level, void *ws, uint32_t nb) {
     return w;
 }
 
-void ks_modup(const ckks_ctx *c, const u64 *d, u64 galois, uint32_t level, const KsWorkspace &w, cudaStream_t s, uint32_t nb,
-              size_t d_stride) {
+void ks_modup(const ckks_ctx *c, const u64 *d, uint32_t level, const KsWorkspace &w, cudaStream_t s, uint32_t nb, size_t d_stride) {
     const uint32_t N = c->N, beta = (level + c->alpha - 1) / c->alpha, nt = level + c->K;
-    permute_kernel<<<dim3(N / THREADS, level, nb), THREADS, 0, s>>>(c->dev, d, d_stride, w.dcoef, (size_t)level * N, galois); count_launches();
-    launch_ntt(c, w.dcoef, nb * level, plain_map(0, level), true, s);
-#define CALL_UP(A) launch_modup<A>(c, w.dcoef, d, d_stride, galois, w.ext, level, nb, s)
+    if (c->log_n == 16) {      // the inverse transform reads d and writes the coefficient copy
+        launch_ntt(c, w.dcoef, nb * level, plain_map(0, level), true, s, nullptr, nullptr, d, (uint32_t)(d_stride / N));
+    } else {
+        permute_kernel<<<dim3(N / THREADS, level, nb), THREADS, 0, s>>>(c->dev, d, d_stride, w.dcoef, (size_t)level * N, 1); count_launches();
+        launch_ntt(c, w.dcoef, nb * level, plain_map(0, level), true, s);
+    }
+#define CALL_UP(A) launch_modup<A>(c, w.dcoef, d, d_stride, 1, w.ext, level, nb, s)
     DISPATCH_POW2(c->alpha, CALL_UP);
 #undef CALL_UP
     launch_ntt(c, w.ext, nb * beta * nt, ext_map(level, c->K, c->L, c->alpha, beta), false, s);

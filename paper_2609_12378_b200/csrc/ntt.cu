@@ -438,7 +438,8 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 
 
 // ---- inverse, row pass (stages m = 32768..256) ---------------------------------------------
 template <bool ALLFP>
-__global__ void __launch_bounds__(F_THREADS, 4) ntt16_inv_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
+__global__ void __launch_bounds__(F_THREADS, 4) ntt16_inv_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, const u64 *src,
+                                                                uint32_t src_pitch) {
     __shared__ u64 sm[16 * ROW_PAD];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
@@ -447,12 +448,14 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_inv_rows(DevTables c, u64 
         const double *tw = c.twd_inv + ((size_t)prime << 16);
         const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
         u64 *g = base + (limb_index(map, blockIdx.y) << 16) + (size_t)row * 256;
+        // out of place: the input limbs lie in another buffer, periods src_pitch limbs apart
+        const u64 *gs = src ? src + ((((size_t)(blockIdx.y / map.period) * src_pitch) + blockIdx.y % map.period) << 16) + (size_t)row * 256 : g;
         double *s = reinterpret_cast<double *>(sm) + rl * ROW_PAD;
         double x[16];
 #pragma unroll
         for (uint32_t k = 0; k < 16; k += 4) {      // 16 consecutive coefficients per thread, four 32-byte loads
             u64 a, b, cc, d;
-            ldg_4(g + 16 * t + k, a, b, cc, d);
+            ldg_4(gs + 16 * t + k, a, b, cc, d);
             x[k] = u64_to_d(a); x[k + 1] = u64_to_d(b); x[k + 2] = u64_to_d(cc); x[k + 3] = u64_to_d(d);
         }
         inv16_d(x, tw, 16 * (256 + row) + t, q, qinv);
@@ -471,10 +474,11 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_inv_rows(DevTables c, u64 
     const ulonglong2 *tw = c.tw_inv + ((size_t)prime << 16);
     const uint32_t t = threadIdx.x & 15, rl = threadIdx.x >> 4, row = blockIdx.x * 16 + rl;
     u64 *g = base + (limb_index(map, blockIdx.y) << 16) + (size_t)row * 256;
+    const u64 *gs = src ? src + ((((size_t)(blockIdx.y / map.period) * src_pitch) + blockIdx.y % map.period) << 16) + (size_t)row * 256 : g;
     u64 *s = sm + rl * ROW_PAD;
     u64 x[16];
 #pragma unroll
-    for (uint32_t k = 0; k < 16; k++) s[padded(t + 16 * k)] = g[t + 16 * k];
+    for (uint32_t k = 0; k < 16; k++) s[padded(t + 16 * k)] = gs[t + 16 * k];
     __syncwarp();
 #pragma unroll
     for (uint32_t k = 0; k < 16; k++) x[k] = s[padded(16 * t + k)];
@@ -541,7 +545,7 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_inv_cols(DevTables c, u64 
 }  // namespace
 
 void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbMap &map, bool inverse, cudaStream_t s,
-                const NttEpilogue *ep, const long long *coef_src) {
+                const NttEpilogue *ep, const long long *coef_src, const u64 *inv_src, uint32_t inv_src_pitch) {
     if (nlimbs_total == 0) return;
     if (c->log_n == 16) {
         for (uint32_t y0 = 0; y0 < nlimbs_total;) {
@@ -561,8 +565,9 @@ void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbM
                 else ntt16_fwd_rows<true, 2><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, *ep);
                 count_launches();
             } else {
-                if (c->ntt_fp_share >= 8) ntt16_inv_rows<true><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, 8);
-                else ntt16_inv_rows<false><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share);
+                const u64 *sb = inv_src ? inv_src + (((size_t)(y0 / map.period) * inv_src_pitch) << 16) : nullptr;
+                if (c->ntt_fp_share >= 8) ntt16_inv_rows<true><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, 8, sb, inv_src_pitch);
+                else ntt16_inv_rows<false><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share, sb, inv_src_pitch);
                 count_launches();
                 if (c->ntt_fp_share >= 8) ntt16_inv_cols<true><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, 8);
                 else ntt16_inv_cols<false><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share);
