@@ -294,7 +294,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bars + 8 * (B_TEMPTY + an % NACC));
-                    // fold a over the 8 lanes of a giant.  Round 1 (lane ^ 1): a even keeps columns 0..3, odd keeps 4..7
+                    // fold a over the 8 lanes of a giant.  First exchange (lane ^ 1): a even keeps columns 0..3, odd keeps 4..7
                     uint32_t V[4][3];
 #pragma unroll
                     for (uint32_t k = 0; k < 4; k++) {
@@ -307,7 +307,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
                         }
                         add_words<3>(V[k], r);
                     }
-                    // round 2 (lane ^ 2): weights 2^(16 (a >> 1 & 1)); a1 = 0 keeps the first two of its four columns
+                    // second exchange (lane ^ 2): weights 2^(16 (a >> 1 & 1)); a1 = 0 keeps the first two of its four columns
                     uint32_t U[2][4];
                     {
                         uint32_t X4[4][4];
@@ -325,7 +325,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
                             add_words<4>(U[k], r);
                         }
                     }
-                    // round 3 (lane ^ 4): weights 2^(32 (a >> 2)), a word shift; a2 = 0 keeps the first of its two columns
+                    // third exchange (lane ^ 4): weights 2^(32 (a >> 2)), a word shift; a2 = 0 keeps the first of its two columns
                     uint32_t Z[4];
                     {
                         uint32_t r[4];
