@@ -489,12 +489,9 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_async_kernel
 
 template <uint32_t COEF, uint32_t NW, bool ASYNC = false>
 bool launch_as(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level, cudaStream_t s) {
-    static bool attr_set = false;
     auto kernel = ASYNC ? mac_mma_async_kernel<COEF, NW> : mac_mma_kernel<COEF, NW>;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Geo<COEF>::SMEM_BYTES) != cudaSuccess) return false;
-        attr_set = true;
-    }
+    // per device, so set on every launch (a host-side table update)
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Geo<COEF>::SMEM_BYTES) != cudaSuccess) return false;
     const uint32_t coltiles = (2 * S + MS - 1) / MS, gt = (G + MG - 1) / MG;
     const uint32_t ntiles = (c->N / COEF) * level * coltiles * gt;
     int sms = 148;

@@ -363,11 +363,8 @@ bool launch_mac_umma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *ac
                      cudaStream_t s) {
     if (!mac_umma_supported(c, J)) return false;
     const Smem L = smem_plan(J);
-    static int attr_for = 0;
-    if (attr_for < (int)L.total) {
-        if (cudaFuncSetAttribute(mac_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_plan(MAX_J).total) != cudaSuccess) return false;
-        attr_for = (int)smem_plan(MAX_J).total;
-    }
+    // per device, so set on every launch (a host-side table update)
+    if (cudaFuncSetAttribute(mac_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_plan(MAX_J).total) != cudaSuccess) return false;
     const uint32_t gtiles = (G + UG - 1) / UG, nblocks = (c->N / UC) * level * gtiles;
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
