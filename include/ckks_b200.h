@@ -246,6 +246,20 @@ int32_t ckks_linear_proj(ckks_ctx *ctx, const ckks_proj_desc *desc, const ckks_c
                          const ckks_evk *keys, uint32_t nkeys, ckks_ct *out,
                          void *ws, size_t ws_bytes, void *stream);
 size_t ckks_linear_proj_workspace_bytes(const ckks_ctx *ctx, const ckks_proj_desc *desc, uint32_t level);
+
+/*
+ * Several projections of the same inputs in one call (the query/key/value or the gate/up matrices of a
+ * transformer layer, Section 4: the activations are shared): descs[0..nmat-1] must agree in d_in,
+ * tokens_per_shard, nshards and baby; W[m] is the device matrix of descs[m].  The extension of the inputs to the
+ * key-switching basis and their baby-step rotations are computed once and used by every matrix; each matrix then
+ * runs its own giant steps.  out: host array holding the outputs of matrix 0 (nshards * its output blocks, ordered
+ * as in ckks_linear_proj), then those of matrix 1, and so on; every output is bit-identical to what a separate
+ * ckks_linear_proj call returns.  Keys for the rotations of every matrix must be present.  Errors as
+ * ckks_linear_proj; CKKS_ERR_ARG if the descriptors do not share their input shape.
+ */
+int32_t ckks_linear_proj_multi(ckks_ctx *ctx, const ckks_proj_desc *descs, uint32_t nmat, const ckks_ct *in, const double *const *W,
+                               const ckks_evk *keys, uint32_t nkeys, ckks_ct *out, void *ws, size_t ws_bytes, void *stream);
+size_t ckks_linear_proj_multi_workspace_bytes(const ckks_ctx *ctx, const ckks_proj_desc *descs, uint32_t nmat, uint32_t level);
 /* Writes up to cap left-rotation amounts (in slots) the schedule needs into
  * rots (host) and returns how many there are; <0 on a shape error. */
 int32_t ckks_linear_proj_rotations(const ckks_ctx *ctx, const ckks_proj_desc *desc, int64_t *rots, uint32_t cap);

@@ -22,7 +22,7 @@ EXPORTS = [
     "ckks_encode_range_flag", "ckks_mul_plain_acc", "ckks_add", "ckks_mul_relin", "ckks_rotate",
     "ckks_rotate_hoisted", "ckks_rescale", "ckks_linear_proj", "ckks_linear_proj_workspace_bytes",
     "ckks_linear_proj_rotations", "ckks_kernel_launches", "ckks_device_status", "ckks_rescale_static",
-    "ckks_ntt_butterfly_probe",
+    "ckks_ntt_butterfly_probe", "ckks_linear_proj_multi", "ckks_linear_proj_multi_workspace_bytes",
 ]
 
 
@@ -84,6 +84,8 @@ def load():
         "ckks_linear_proj_workspace_bytes": (sz, [vp, C.POINTER(CProjDesc), u32]),
         "ckks_linear_proj_rotations": (i32, [vp, C.POINTER(CProjDesc), C.POINTER(i64), u32]),
         "ckks_ntt_butterfly_probe": (i32, [vp, u32, vp, sz, C.POINTER(u64), vp]),
+        "ckks_linear_proj_multi": (i32, [vp, C.POINTER(CProjDesc), u32, C.POINTER(CCt), C.POINTER(vp), C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
+        "ckks_linear_proj_multi_workspace_bytes": (sz, [vp, C.POINTER(CProjDesc), u32, u32]),
     }
     for name, (res, args) in sig.items():
         f = getattr(L, name)
@@ -294,6 +296,32 @@ class Context:
         self._check(load().ckks_rotate_hoisted(self._h, C.byref(_cct(ct)), ka, n, oa, ws.data_ptr(), ws.numel(),
                                                _stream_ptr(stream)))
         for o, c in zip(outs, oa):
+            o.scale = c.scale
+        return outs
+
+    def linear_proj_multi(self, cts, Ws, keys, d_in, d_outs, tokens_per_shard, nshards, baby, pt_scale=0.0,
+                          ws: torch.Tensor = None, stream=None):
+        """[X W_0, X W_1, ...] for weight matrices sharing their input (Q/K/V, gate/up): the baby-step rotations of
+        the inputs are computed once.  Returns one list of output ciphertexts per matrix, each bit-identical to a
+        separate linear_proj call."""
+        nmat = len(Ws)
+        for W, d_out in zip(Ws, d_outs):
+            if not (W.is_cuda and W.dtype == torch.float64 and W.is_contiguous() and tuple(W.shape) == (d_in, d_out)):
+                raise TypeError("every W must be a contiguous CUDA float64 [d_in][d_out] tensor")
+        da = (CProjDesc * nmat)(*[self._desc(d_in, d_out, tokens_per_shard, nshards, baby, pt_scale) for d_out in d_outs])
+        level = cts[0].level
+        F = self.n // tokens_per_shard
+        outs = [[self.empty_ct(level - 1) for _ in range(nshards * -(-d_out // F))] for d_out in d_outs]
+        flat = [o for m in outs for o in m]
+        if ws is None:
+            ws = self.workspace(int(load().ckks_linear_proj_multi_workspace_bytes(self._h, da, nmat, level)))
+        ia = (CCt * len(cts))(*[_cct(c) for c in cts])
+        oa = (CCt * len(flat))(*[_cct(o) for o in flat])
+        wa = (C.c_void_p * nmat)(*[W.data_ptr() for W in Ws])
+        ka = (CEvk * len(keys))(*[CEvk(_dev_u64(k.data).data_ptr(), k.galois) for k in keys])
+        self._check(load().ckks_linear_proj_multi(self._h, da, nmat, ia, wa, ka, len(keys), oa, ws.data_ptr(), ws.numel(),
+                                                  _stream_ptr(stream)))
+        for o, c in zip(flat, oa):
             o.scale = c.scale
         return outs
 

@@ -435,13 +435,26 @@ extern "C" size_t ckks_linear_proj_workspace_bytes(const ckks_ctx *c, const ckks
     return proj_layout(c, p, level).bytes;
 }
 
-extern "C" int32_t ckks_linear_proj(ckks_ctx *c, const ckks_proj_desc *d, const ckks_ct *in, const double *W, const ckks_evk *keys,
-                                    uint32_t nkeys, ckks_ct *out, void *ws, size_t ws_bytes, void *stream) {
-    if (!c || !in || !W || !keys || !out) return CKKS_ERR_ARG;
-    ProjPlan p;
-    int rc = make_plan(c, d, p);
-    if (rc) return rc;
-    const uint32_t nib = (uint32_t)p.ins.size(), nob = (uint32_t)p.outs.size(), S = p.S, B = p.B, T = p.T, N = c->N;
+// nmat projections of the same inputs (descriptors agreeing in d_in, tokens_per_shard, nshards, baby): the inputs'
+// ModUp and baby-step rotations are done once, then every matrix runs its giant steps.  out: the outputs of matrix 0
+// (nshards * its output blocks), then those of matrix 1, and so on.
+static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_t nmat, const ckks_ct *in, const double *const *Ws,
+                               const ckks_evk *keys, uint32_t nkeys, ckks_ct *out, void *ws, size_t ws_bytes, void *stream) {
+    if (!c || !descs || !nmat || !in || !Ws || !keys || !out) return CKKS_ERR_ARG;
+    std::vector<ProjPlan> plans(nmat);
+    ProjPlan merged;
+    int rc;
+    for (uint32_t m = 0; m < nmat; m++) {
+        if (!Ws[m]) return CKKS_ERR_ARG;
+        if ((rc = make_plan(c, &descs[m], plans[m]))) return rc;
+        if (descs[m].d_in != descs[0].d_in || descs[m].tokens_per_shard != descs[0].tokens_per_shard || descs[m].nshards != descs[0].nshards ||
+            descs[m].baby != descs[0].baby)
+            return CKKS_ERR_ARG;
+    }
+    merged = plans[0];
+    for (uint32_t m = 1; m < nmat; m++) merged.gmax = std::max(merged.gmax, plans[m].gmax);
+    const ProjPlan &p0 = plans[0];
+    const uint32_t nib = (uint32_t)p0.ins.size(), S = p0.S, B = p0.B, T = p0.T, N = c->N;
     const uint32_t level = in[0].level;
     if (!level_ok(c, level) || level < 2) return CKKS_ERR_LEVEL;
     for (uint32_t x = 0; x < S * nib; x++) {
@@ -449,13 +462,16 @@ extern "C" int32_t ckks_linear_proj(ckks_ctx *c, const ckks_proj_desc *d, const 
         if (in[x].level != level) return CKKS_ERR_LEVEL;
         if (!scales_agree(in[x].scale, in[0].scale)) return CKKS_ERR_SCALE;
     }
-    for (uint32_t x = 0; x < S * nob; x++)
-        if (!out[x].data) return CKKS_ERR_ARG;
-    for (int64_t r : p.rots)
-        if (!find_key(keys, nkeys, ckks_galois_element(c, r))) return CKKS_ERR_NO_KEY;
-    const ProjWs L = proj_layout(c, p, level);
+    uint32_t nout = 0;
+    for (uint32_t m = 0; m < nmat; m++) {
+        for (uint32_t x = 0; x < S * plans[m].outs.size(); x++)
+            if (!out[nout + x].data) return CKKS_ERR_ARG;
+        nout += S * (uint32_t)plans[m].outs.size();
+        for (int64_t r : plans[m].rots)
+            if (!find_key(keys, nkeys, ckks_galois_element(c, r))) return CKKS_ERR_NO_KEY;
+    }
+    const ProjWs L = proj_layout(c, merged, level);
     if (!ws || ws_bytes < L.bytes) return CKKS_ERR_WORKSPACE;
-    const double pt_scale = d->pt_scale > 0.0 ? d->pt_scale : (double)c->mod[level - 1];
 
     DeviceGuard g(c->device);
     cudaStream_t s = (cudaStream_t)stream;
@@ -463,7 +479,7 @@ extern "C" int32_t ckks_linear_proj(ckks_ctx *c, const ckks_proj_desc *d, const 
     const size_t ctl = (size_t)2 * level * N, ptl = (size_t)level * N;
     u64 *baby = (u64 *)(base + L.baby), *pts = (u64 *)(base + L.pts), *acc = (u64 *)(base + L.acc);
     u64 *xin = (u64 *)(base + L.xin), *ptt = (u64 *)(base + L.ptt);
-    u64 *total = (u64 *)(base + L.total), *tmp = (u64 *)(base + L.tmp), *rsw = (u64 *)(base + L.rs);
+    u64 *total = (u64 *)(base + L.total), *rsw = (u64 *)(base + L.rs);
     double *slots = (double *)(base + L.slots);
     void *encw = base + L.enc;
     KsWorkspace kw = ks_carve(c, level, base + L.ks, S * nib);
@@ -487,78 +503,117 @@ extern "C" int32_t ckks_linear_proj(ckks_ctx *c, const ckks_proj_desc *d, const 
         }
     }
 
-    for (uint32_t ob = 0; ob < nob; ob++) {
-        const Block &o = p.outs[ob];
-        uint32_t gcount = 0, fold = 1;
-        for (const Block &i : p.ins) {
-            gcount = std::max(gcount, std::min(i.size, o.size) / B);
-            if (i.size > o.size) fold = i.size / o.size;
-        }
-        for (uint32_t g0 = 0; g0 < gcount; g0 += L.gg) {
-            const uint32_t ng = std::min(L.gg, gcount - g0);
-            const uint32_t J = nib * B;
-            // plaintexts of the group: pts[(gl * nib + ib) * B + b]; a block pair that has run out of diagonals
-            // contributes zero plaintexts
-            bool ragged = false;
-            for (uint32_t gl = 0; gl < ng; gl++)
-                for (uint32_t ib = 0; ib < nib; ib++)
-                    if (g0 + gl >= std::min(p.ins[ib].size, o.size) / B) ragged = true;
-            if (ragged) cudaMemsetAsync(ptt, 0, (size_t)ng * J * ptl * sizeof(u64), s);
-            for (uint32_t gl = 0; gl < ng; gl++)
-                for (uint32_t ib = 0; ib < nib; ib++) {
-                    const Block &i = p.ins[ib];
-                    const uint32_t gi = g0 + gl;
-                    if (gi >= std::min(i.size, o.size) / B) continue;
-                    const size_t idx = ((size_t)gl * nib + ib) * B;
-                    launch_extract_diagonals(c, W, d->d_out, i.start, i.size, o.start, o.size, p.F, T, gi * B, B, gi * B,
-                                             slots + idx * c->n, s);
-                    if (ragged) {
-                        TiledOut to;
-                        to.R = ng * J; to.row0 = (uint32_t)idx; to.row_stride = 1;
-                        launch_encode(c, slots + idx * c->n, nullptr, B, pt_scale, level, pts + idx * ptl, encw, s, to, ptt);
+    ckks_ct *out_m = out;
+    for (uint32_t m = 0; m < nmat; m++) {
+        const ProjPlan &p = plans[m];
+        const ckks_proj_desc *d = &descs[m];
+        const double *W = Ws[m];
+        const uint32_t nob = (uint32_t)p.outs.size();
+        const double pt_scale = d->pt_scale > 0.0 ? d->pt_scale : (double)c->mod[level - 1];
+        for (uint32_t ob = 0; ob < nob; ob++) {
+            const Block &o = p.outs[ob];
+            uint32_t gcount = 0, fold = 1;
+            for (const Block &i : p.ins) {
+                gcount = std::max(gcount, std::min(i.size, o.size) / B);
+                if (i.size > o.size) fold = i.size / o.size;
+            }
+            for (uint32_t g0 = 0; g0 < gcount; g0 += L.gg) {
+                const uint32_t ng = std::min(L.gg, gcount - g0);
+                const uint32_t J = nib * B;
+                // plaintexts of the group: pts[(gl * nib + ib) * B + b]; a block pair that has run out of diagonals
+                // contributes zero plaintexts
+                bool ragged = false;
+                for (uint32_t gl = 0; gl < ng; gl++)
+                    for (uint32_t ib = 0; ib < nib; ib++)
+                        if (g0 + gl >= std::min(p.ins[ib].size, o.size) / B) ragged = true;
+                if (ragged) cudaMemsetAsync(ptt, 0, (size_t)ng * J * ptl * sizeof(u64), s);
+                for (uint32_t gl = 0; gl < ng; gl++)
+                    for (uint32_t ib = 0; ib < nib; ib++) {
+                        const Block &i = p.ins[ib];
+                        const uint32_t gi = g0 + gl;
+                        if (gi >= std::min(i.size, o.size) / B) continue;
+                        const size_t idx = ((size_t)gl * nib + ib) * B;
+                        launch_extract_diagonals(c, W, d->d_out, i.start, i.size, o.start, o.size, p.F, T, gi * B, B, gi * B,
+                                                 slots + idx * c->n, s);
+                        if (ragged) {
+                            TiledOut to;
+                            to.R = ng * J; to.row0 = (uint32_t)idx; to.row_stride = 1;
+                            launch_encode(c, slots + idx * c->n, nullptr, B, pt_scale, level, pts + idx * ptl, encw, s, to, ptt);
+                        }
                     }
+                if (!ragged) {
+                    TiledOut to;
+                    to.R = ng * J; to.row0 = 0; to.row_stride = 1;
+                    launch_encode(c, slots, nullptr, ng * J, pt_scale, level, pts, encw, s, to, ptt);
                 }
-            if (!ragged) {
-                TiledOut to;
-                to.R = ng * J; to.row0 = 0; to.row_stride = 1;
-                launch_encode(c, slots, nullptr, ng * J, pt_scale, level, pts, encw, s, to, ptt);
-            }
-            if (!launch_mac_mma(c, baby, ptt, acc, J, S, ng, level, s)) {
-                const uint32_t stiles = (S + MAC_ST - 1) / MAC_ST, gtiles = (ng + MAC_GT - 1) / MAC_GT;
-                mac_tile_kernel<<<dim3(stiles * gtiles, N / MAC_THREADS, level), MAC_THREADS, 0, s>>>(c->dev, baby, ptt, acc, J, S, ng, level);
-                count_launches();
-            }
-            for (uint32_t gl = 0; gl < ng; gl++) {
-                const uint32_t gi = g0 + gl;
-                u64 *ag = acc + (size_t)gl * S * ctl;
-                if (gi == 0) {
-                    cudaMemcpyAsync(total, ag, (size_t)S * ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
-                    continue;
+                if (!launch_mac_mma(c, baby, ptt, acc, J, S, ng, level, s)) {
+                    const uint32_t stiles = (S + MAC_ST - 1) / MAC_ST, gtiles = (ng + MAC_GT - 1) / MAC_GT;
+                    mac_tile_kernel<<<dim3(stiles * gtiles, N / MAC_THREADS, level), MAC_THREADS, 0, s>>>(c->dev, baby, ptt, acc, J, S, ng, level);
+                    count_launches();
                 }
-                const u64 ge = ckks_galois_element(c, (int64_t)gi * B * T);
+                for (uint32_t gl = 0; gl < ng; gl++) {
+                    const uint32_t gi = g0 + gl;
+                    u64 *ag = acc + (size_t)gl * S * ctl;
+                    if (gi == 0) {
+                        cudaMemcpyAsync(total, ag, (size_t)S * ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+                        continue;
+                    }
+                    const u64 ge = ckks_galois_element(c, (int64_t)gi * B * T);
+                    const u64 *key = (const u64 *)find_key(keys, nkeys, ge)->data;
+                    // total[sh] += rotate(acc_g[sh]) for all shards in one batch
+                    ks_modup(c, ag + ptl, level, kw, s, S, ctl);
+                    ks_inner_moddown(c, key, level, ge, kw, ag, nullptr, ge, total, s, S, ctl, ctl, true);
+                }
+            }
+            for (uint32_t f = o.size; fold > 1; f *= 2, fold /= 2) {
+                const u64 ge = ckks_galois_element(c, (int64_t)f * T);
                 const u64 *key = (const u64 *)find_key(keys, nkeys, ge)->data;
-                // total[sh] += rotate(acc_g[sh]) for all shards in one batch
-                ks_modup(c, ag + ptl, level, kw, s, S, ctl);
-                ks_inner_moddown(c, key, level, ge, kw, ag, nullptr, ge, total, s, S, ctl, ctl, true);
+                // total += rotate(total): the rotated copy goes to the (now free) accumulator buffer first
+                ks_modup(c, total + ptl, level, kw, s, S, ctl);
+                ks_inner_moddown(c, key, level, ge, kw, total, nullptr, ge, acc, s, S, ctl, ctl, false);
+                for (uint32_t sh = 0; sh < S; sh++)
+                    launch_add(c, total + (size_t)sh * ctl, acc + (size_t)sh * ctl, total + (size_t)sh * ctl, 2, level, s);
             }
-        }
-        for (uint32_t f = o.size; fold > 1; f *= 2, fold /= 2) {
-            const u64 ge = ckks_galois_element(c, (int64_t)f * T);
-            const u64 *key = (const u64 *)find_key(keys, nkeys, ge)->data;
-            // total += rotate(total): the rotated copy goes to the (now free) accumulator buffer first
-            ks_modup(c, total + ptl, level, kw, s, S, ctl);
-            ks_inner_moddown(c, key, level, ge, kw, total, nullptr, ge, acc, s, S, ctl, ctl, false);
             for (uint32_t sh = 0; sh < S; sh++)
-                launch_add(c, total + (size_t)sh * ctl, acc + (size_t)sh * ctl, total + (size_t)sh * ctl, 2, level, s);
+                launch_rescale(c, total + (size_t)sh * ctl, (u64 *)out_m[sh * nob + ob].data, 2, level, rsw, s);
         }
-        for (uint32_t sh = 0; sh < S; sh++)
-            launch_rescale(c, total + (size_t)sh * ctl, (u64 *)out[sh * nob + ob].data, 2, level, rsw, s);
+        out_m += S * nob;
     }
     rc = finish(c);
-    if (rc == CKKS_OK)
-        for (uint32_t x = 0; x < S * nob; x++) {
-            out[x].level = level - 1; out[x].ncomp = 2;
-            out[x].scale = in[0].scale * pt_scale / (double)c->mod[level - 1];
+    if (rc == CKKS_OK) {
+        out_m = out;
+        for (uint32_t m = 0; m < nmat; m++) {
+            const uint32_t nob = (uint32_t)plans[m].outs.size();
+            const double pt_scale = descs[m].pt_scale > 0.0 ? descs[m].pt_scale : (double)c->mod[level - 1];
+            for (uint32_t x = 0; x < S * nob; x++) {
+                out_m[x].level = level - 1; out_m[x].ncomp = 2;
+                out_m[x].scale = in[0].scale * pt_scale / (double)c->mod[level - 1];
+            }
+            out_m += S * nob;
         }
+    }
     return rc;
+}
+
+extern "C" int32_t ckks_linear_proj(ckks_ctx *c, const ckks_proj_desc *d, const ckks_ct *in, const double *W, const ckks_evk *keys,
+                                    uint32_t nkeys, ckks_ct *out, void *ws, size_t ws_bytes, void *stream) {
+    if (!d || !W) return CKKS_ERR_ARG;
+    return run_projections(c, d, 1, in, &W, keys, nkeys, out, ws, ws_bytes, stream);
+}
+
+extern "C" int32_t ckks_linear_proj_multi(ckks_ctx *c, const ckks_proj_desc *descs, uint32_t nmat, const ckks_ct *in, const double *const *W,
+                                          const ckks_evk *keys, uint32_t nkeys, ckks_ct *out, void *ws, size_t ws_bytes, void *stream) {
+    return run_projections(c, descs, nmat, in, W, keys, nkeys, out, ws, ws_bytes, stream);
+}
+
+extern "C" size_t ckks_linear_proj_multi_workspace_bytes(const ckks_ctx *c, const ckks_proj_desc *descs, uint32_t nmat, uint32_t level) {
+    if (!c || !descs || !nmat || !level_ok(c, level) || level < 2) return 0;
+    ProjPlan merged;
+    if (make_plan(c, &descs[0], merged)) return 0;
+    for (uint32_t m = 1; m < nmat; m++) {
+        ProjPlan p;
+        if (make_plan(c, &descs[m], p)) return 0;
+        merged.gmax = std::max(merged.gmax, p.gmax);
+    }
+    return proj_layout(c, merged, level).bytes;
 }

@@ -32,7 +32,8 @@ def test_llama_shaped_projection_full_size():
         ge = o.galois_element(r)
         keys[ge] = cl.rotation_key(ge)
         dkeys.append(key_dev(keys[ge], ge))
-    outs = ctx.linear_proj([ct_dev(c, scale) for c in cts], dev(W), dkeys, D, D, T, S, B)
+    dcts = [ct_dev(c, scale) for c in cts]
+    outs = ctx.linear_proj(dcts, dev(W), dkeys, D, D, T, S, B)
     assert ctx.device_status() == binding.OK
     Y = X @ W
     got = [host(ct.data) for ct in outs]
@@ -48,6 +49,18 @@ def test_llama_shaped_projection_full_size():
     want, want_scale = o.linear_proj(one, cts[c][None], W, keys, scale)
     assert want_scale == outs[c].scale
     assert np.array_equal(got[c], want[0])
+    # the same inputs through the square and a key-shaped (4096 x 1024) matrix in one call with shared baby steps:
+    # the square matrix's outputs do not change, the second matrix's decrypt to X Wk (one block, stored four times)
+    Wk = inputs.weights_normal(inputs.rng(1004, 3), D, 1024, 0.02)
+    both = ctx.linear_proj_multi(dcts, [dev(W), dev(Wk)], dkeys, D, [D, 1024], T, S, B)
+    assert ctx.device_status() == binding.OK
+    assert len(both[0]) == S and len(both[1]) == S
+    for a, b in zip(both[0], got):
+        assert np.array_equal(host(a.data), b)
+    Yk = X @ Wk
+    for cc in (0, c, S - 1):
+        sl = cl.decrypt_slots(host(both[1][cc].data), both[1][cc].scale).real.reshape(D, T)
+        assert np.abs(sl - np.tile(Yk[cc * T:(cc + 1) * T].T, (4, 1))).max() < 2.0 ** -16
 
 
 def test_sixty_four_rotations_full_size():

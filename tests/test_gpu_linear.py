@@ -78,6 +78,57 @@ def test_projection_tensor_core_mac_other_shapes(shape, monkeypatch):
     assert ctx.device_status() == 0
 
 
+def test_projection_multi_shares_baby_steps():
+    """Three matrices on the same inputs (query/key/value-like: square, wide with fold, several output blocks):
+    every output equals the checker's per-matrix result, and the shared call launches fewer kernels than three
+    separate ones."""
+    from tests.gpu_util import context, ct_dev, dev, host, key_dev
+    log_n, L, K, dnum, level, d_in, T, S, B = 10, 4, 2, 2, 4, 16, 32, 2, 4
+    d_outs = [16, 4, 24]
+    P, ctx = params(log_n, L, K, dnum), context(log_n, L, K, dnum)
+    o = P.oracle
+    cl = Client(P, 470)
+    scale = 2.0 ** 40
+    g = inputs.rng(470, 1)
+    X = inputs.activations_uniform(g, S * T, d_in)
+    Ws = [inputs.weights_normal(g, d_in, d_out, 0.02) for d_out in d_outs]
+    descs = [ProjDesc(d_in, d_out, T, S, B, 0.0) for d_out in d_outs]
+    F, ins, _ = o.proj_blocks(descs[0])
+    cts = []
+    for c in range(S):
+        for (s0, mi) in ins:
+            cts.append(cl.encrypt_slots(inputs.pack_feature_major(X[c * T:(c + 1) * T, s0:s0 + mi], T, o.n)[0], scale, level))
+    rots = sorted(set(r for d in descs for r in o.proj_rotations(d)))
+    keys = {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in rots}
+    kd = [key_dev(k, g_) for g_, k in keys.items()]
+    cd = [ct_dev(c, scale) for c in cts]
+    n0 = binding.kernel_launches()
+    got = ctx.linear_proj_multi(cd, [dev(W) for W in Ws], kd, d_in, d_outs, T, S, B)
+    n_multi = binding.kernel_launches() - n0
+    n_sep = 0
+    for m, (d, W) in enumerate(zip(descs, Ws)):
+        want, want_scale = o.linear_proj(d, np.stack(cts), W, keys, scale)
+        assert len(got[m]) == len(want)
+        for i, ct in enumerate(got[m]):
+            assert ct.scale == want_scale and ct.level == level - 1
+            assert np.array_equal(host(ct.data), want[i]), (m, i)
+        n1 = binding.kernel_launches()
+        ctx.linear_proj(cd, dev(W), kd, d_in, d_outs[m], T, S, B)
+        n_sep += binding.kernel_launches() - n1
+    assert n_multi < n_sep
+    with pytest.raises(binding.CkksError) as e:       # descriptors must share the input shape
+        lib = binding.load()
+        import ctypes as C
+        da = (binding.CProjDesc * 2)(ctx._desc(16, 16, T, S, B), ctx._desc(16, 16, T, S, 2))
+        ia = (binding.CCt * len(cd))(*[binding._cct(c) for c in cd])
+        oa = (binding.CCt * 4)(*[binding._cct(ctx.empty_ct(level - 1)) for _ in range(4)])
+        wa = (C.c_void_p * 2)(dev(Ws[0]).data_ptr(), dev(Ws[0]).data_ptr())
+        ka = (binding.CEvk * len(kd))(*[binding.CEvk(k.data.data_ptr(), k.galois) for k in kd])
+        ws = ctx.workspace(1 << 20)
+        ctx._check(lib.ckks_linear_proj_multi(ctx._h, da, 2, ia, wa, ka, len(kd), oa, ws.data_ptr(), ws.numel(), None))
+    assert e.value.code == binding.ERR_ARG
+
+
 def test_projection_explicit_pt_scale_and_lower_level():
     _run(10, 4, 2, 2, 3, 16, 16, 32, 1, 4, seed=410, pt_scale=2.0 ** 40, check_slots=False)
 
