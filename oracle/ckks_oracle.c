@@ -782,6 +782,32 @@ void orc_mul_relin(const orc_ctx *c, const uint64_t *a, const uint64_t *b, const
     free(e); free(k);
 }
 
+/*
+ * Sum of n products with one relinearisation (the lazy form of a sum of Mults, Section 4: the attention
+ * products add up many ciphertext x ciphertext terms): e = sum_i tensor(a_i, b_i) component-wise modulo each
+ * prime, (k0,k1) = KeySwitch(e2, rlk), out = (e0 + k0, e1 + k1).  a, b: [n][2][level][N].  For n = 1 this is
+ * orc_mul_relin.  Not the same integers as the sum of n separately relinearised products (the key switch's
+ * rounding acts on the sum once instead of on every term); both decrypt to the sum of the slot products.
+ */
+void orc_mul_relin_sum(const orc_ctx *c, const uint64_t *a, const uint64_t *b, uint32_t n, const uint64_t *rlk, uint32_t level,
+                       uint64_t *out) {
+    uint64_t N = c->N, S = (uint64_t)level * N;
+    uint64_t *e = (uint64_t *)calloc(3 * S, 8), *t = (uint64_t *)malloc(3 * S * 8), *k = (uint64_t *)malloc(2 * S * 8);
+    for (uint32_t i = 0; i < n; i++) {
+        orc_tensor(c, a + (uint64_t)i * 2 * S, b + (uint64_t)i * 2 * S, level, t);
+        for (uint32_t x = 0; x < 3 * level; x++) {
+            uint64_t q = c->mod[x % level];
+            for (uint64_t p = 0; p < N; p++) e[x * N + p] = addmod(e[x * N + p], t[x * N + p], q);
+        }
+    }
+    orc_keyswitch(c, e + 2 * S, rlk, level, k);
+    for (uint32_t x = 0; x < 2 * level; x++) {
+        uint64_t q = c->mod[x % level];
+        for (uint64_t p = 0; p < N; p++) out[x * N + p] = addmod(e[x * N + p], k[x * N + p], q);
+    }
+    free(e); free(t); free(k);
+}
+
 /* Pointwise product of limb arrays under primes first..first+nl-1 (used to form s^2 for the relinearisation key). */
 void orc_pointwise_mul(const orc_ctx *c, const uint64_t *a, const uint64_t *b, uint32_t first, uint32_t nl, uint64_t *out) {
     uint64_t N = c->N;

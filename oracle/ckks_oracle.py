@@ -279,6 +279,13 @@ class Oracle:
         lib().orc_mul_relin(self._h, _p(a, _u64p), _p(b, _u64p), _p(rlk, _u64p), C.c_uint32(level), _p(out, _u64p))
         return out
 
+    def mul_relin_sum(self, a, b, rlk):
+        """relin(sum_i a_i (x) b_i): a, b [n][2][level][N]; one key switch for the whole sum."""
+        a = _u64(a); b = _u64(b); rlk = _u64(rlk); n, level = a.shape[0], a.shape[2]
+        out = np.empty_like(a[0])
+        lib().orc_mul_relin_sum(self._h, _p(a, _u64p), _p(b, _u64p), C.c_uint32(n), _p(rlk, _u64p), C.c_uint32(level), _p(out, _u64p))
+        return out
+
     # ----------------------------------------------------- linear projection
     def proj_blocks(self, desc: ProjDesc):
         """Feature blocks of the input and output: lists of (start, size).  F = n / T_s

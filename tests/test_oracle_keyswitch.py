@@ -201,3 +201,35 @@ def test_mul_relin_slot_product(log_n, L, K, dnum, level):
     rs = o.rescale(out)
     assert rs.shape[1] == level - 1
     assert np.abs(cl.decrypt_slots(rs, scale) - z * w).max() < 2.0 ** -20
+
+
+def test_mul_relin_sum_pins():
+    """Sum of products with one relinearisation: n = 1 is mul_relin bit for bit; the result is the key switch applied
+    to the component-wise sum of the tensor products (checked against the separately exposed pieces); it decrypts
+    to sum_i z_i w_i; and its exact decryption stays within key-switch noise of the three-component sum."""
+    P = params(10, 6, 2, 3)
+    o = P.oracle
+    cl = Client(P, 57)
+    g = inputs.rng(57)
+    level, n, scale = 5, 6, 2.0 ** 40
+    zs, ws = g.uniform(-1, 1, (n, P.n)), g.uniform(-1, 1, (n, P.n))
+    ca = np.stack([cl.encrypt_slots(z, scale, level) for z in zs])
+    cb = np.stack([cl.encrypt_slots(w, scale, level) for w in ws])
+    rlk = cl.relin_key()
+    assert np.array_equal(o.mul_relin_sum(ca[:1], cb[:1], rlk), o.mul_relin(ca[0], cb[0], rlk))
+    out = o.mul_relin_sum(ca, cb, rlk)
+    # the pieces: e = sum of tensor products modulo each prime, then mul_relin's own combination on e
+    q = np.array(P.q[:level], dtype=object)[None, :, None]
+    e = sum(o.tensor(ca[i], cb[i]).astype(object) for i in range(n)) % q
+    e = e.astype(np.uint64)
+    k = o.keyswitch(e[2], rlk)
+    want = ((e[:2].astype(object) + k.astype(object)) % q).astype(np.uint64)
+    assert np.array_equal(out, want)
+    assert np.abs(cl.decrypt_slots(out, scale * scale) - (zs * ws).sum(0)).max() < 2.0 ** -20
+    d3 = o.decrypt(e, cl.s, exact=True)
+    d2 = o.decrypt(out, cl.s, exact=True)
+    assert max(abs(x - y) for x, y in zip(d3, d2)) < 2 ** 16
+    # and it is a different integer function from the sum of separately relinearised products (same plaintext)
+    sep = sum(o.mul_relin(ca[i], cb[i], rlk).astype(object) for i in range(n)) % q
+    assert not np.array_equal(sep.astype(np.uint64), out)
+    assert np.abs(cl.decrypt_slots(sep.astype(np.uint64), scale * scale) - (zs * ws).sum(0)).max() < 2.0 ** -20
