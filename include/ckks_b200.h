@@ -185,6 +185,16 @@ int32_t ckks_add(ckks_ctx *ctx, const ckks_ct *a, const ckks_ct *b, ckks_ct *out
 int32_t ckks_mul_relin(ckks_ctx *ctx, const ckks_ct *a, const ckks_ct *b, const ckks_evk *rlk, ckks_ct *out,
                        void *ws, size_t ws_bytes, void *stream);
 
+/* Sum of n products with one relinearisation (Section 4: the attention products add up many ciphertext x
+ * ciphertext terms): e = sum_i a_i (x) b_i component-wise modulo each prime, then as ckks_mul_relin from the
+ * key switch on.  a, b: host arrays of n two-component ciphertexts, all at one level; the a_i share a scale,
+ * the b_i share a scale; out.scale = a_0.scale * b_0.scale.  n = 1 gives ckks_mul_relin's result bit for bit; for
+ * n > 1 the integers differ from the sum of n ckks_mul_relin results (one rounding of the key switch instead of n)
+ * while the plaintext is the same.  out must not alias an input.  Workspace: CKKS_OP_MUL_RELIN.
+ * Errors: as ckks_mul_relin; CKKS_ERR_SCALE if the a_i (or the b_i) disagree in scale. */
+int32_t ckks_mul_relin_sum(ckks_ctx *ctx, const ckks_ct *a, const ckks_ct *b, uint32_t n, const ckks_evk *rlk, ckks_ct *out,
+                           void *ws, size_t ws_bytes, void *stream);
+
 /* ---- Rot_k (Section 2.1, Rot + KeySwitch) ----------------------------------
  * Plain: apply sigma_g (g = key->galois) to both components, key-switch the
  * permuted c1: out = (sigma c0 + k0, k1).  Key switch = iNTT, centred ModUp

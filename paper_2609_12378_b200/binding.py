@@ -22,7 +22,7 @@ EXPORTS = [
     "ckks_encode_range_flag", "ckks_mul_plain_acc", "ckks_add", "ckks_mul_relin", "ckks_rotate",
     "ckks_rotate_hoisted", "ckks_rescale", "ckks_linear_proj", "ckks_linear_proj_workspace_bytes",
     "ckks_linear_proj_rotations", "ckks_kernel_launches", "ckks_device_status", "ckks_rescale_static",
-    "ckks_ntt_butterfly_probe", "ckks_linear_proj_multi", "ckks_linear_proj_multi_workspace_bytes",
+    "ckks_ntt_butterfly_probe", "ckks_mul_relin_sum", "ckks_linear_proj_multi", "ckks_linear_proj_multi_workspace_bytes",
 ]
 
 
@@ -76,6 +76,7 @@ def load():
         "ckks_mul_plain_acc": (i32, [vp, C.POINTER(CCt), u32, C.POINTER(CPt), C.POINTER(CCt), i32, vp]),
         "ckks_add": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), C.POINTER(CCt), vp]),
         "ckks_mul_relin": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
+        "ckks_mul_relin_sum": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), u32, C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
         "ckks_rotate": (i32, [vp, C.POINTER(CCt), C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
         "ckks_rotate_hoisted": (i32, [vp, C.POINTER(CCt), C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
         "ckks_rescale": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), vp, sz, vp]),
@@ -275,6 +276,21 @@ class Context:
         co, ck = _cct(out), CEvk(_dev_u64(rlk.data).data_ptr(), rlk.galois)
         self._check(load().ckks_mul_relin(self._h, C.byref(_cct(a)), C.byref(_cct(b)), C.byref(ck), C.byref(co),
                                           ws.data_ptr(), ws.numel(), _stream_ptr(stream)))
+        out.scale = co.scale
+        return out
+
+    def mul_relin_sum(self, a, b, rlk: SwitchKey, out: Ciphertext = None, stream=None):
+        """relin(sum_i a[i] (x) b[i]) with a single key switch; a, b: equally long lists of ciphertexts."""
+        if len(a) != len(b) or not a:
+            raise ValueError("a and b must be non-empty lists of the same length")
+        level = a[0].level
+        out = out or self.empty_ct(level)
+        ws = self.workspace(self.workspace_bytes(OP_MUL_RELIN, level))
+        aa = (CCt * len(a))(*[_cct(x) for x in a])
+        ba = (CCt * len(b))(*[_cct(x) for x in b])
+        co, ck = _cct(out), CEvk(_dev_u64(rlk.data).data_ptr(), rlk.galois)
+        self._check(load().ckks_mul_relin_sum(self._h, aa, ba, len(a), C.byref(ck), C.byref(co), ws.data_ptr(), ws.numel(),
+                                              _stream_ptr(stream)))
         out.scale = co.scale
         return out
 

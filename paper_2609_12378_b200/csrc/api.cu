@@ -358,6 +358,35 @@ static int rotate_checks(const ckks_ctx *c, const ckks_ct *in, const ckks_evk *k
     return CKKS_OK;
 }
 
+extern "C" int32_t ckks_mul_relin_sum(ckks_ctx *c, const ckks_ct *a, const ckks_ct *b, uint32_t n, const ckks_evk *rlk, ckks_ct *out,
+                                      void *ws, size_t ws_bytes, void *stream) {
+    if (!c || !a || !b || !n || !ct_ok(out)) return CKKS_ERR_ARG;
+    for (uint32_t i = 0; i < n; i++)
+        if (!ct_ok(&a[i]) || !ct_ok(&b[i]) || a[i].ncomp != 2 || b[i].ncomp != 2) return CKKS_ERR_ARG;
+    const uint32_t level = a[0].level;
+    if (!level_ok(c, level)) return CKKS_ERR_LEVEL;
+    for (uint32_t i = 0; i < n; i++) {
+        if (a[i].level != level || b[i].level != level) return CKKS_ERR_LEVEL;
+        if (!scales_agree(a[i].scale, a[0].scale) || !scales_agree(b[i].scale, b[0].scale)) return CKKS_ERR_SCALE;
+        if (a[i].data == out->data || b[i].data == out->data) return CKKS_ERR_ARG;       // out is written before the last read
+    }
+    if (!rlk || !rlk->data || rlk->galois != 0) return CKKS_ERR_NO_KEY;
+    if (!ws || ws_bytes < ckks_workspace_bytes(c, CKKS_OP_MUL_RELIN, level, 0)) return CKKS_ERR_WORKSPACE;
+    DeviceGuard g(c->device);
+    cudaStream_t s = (cudaStream_t)stream;
+    u64 *e2 = (u64 *)ws;
+    KsWorkspace w = ks_carve(c, level, e2 + (size_t)level * c->N);
+    u64 *o = (u64 *)out->data;
+    std::vector<const u64 *> pa(n), pb(n);
+    for (uint32_t i = 0; i < n; i++) { pa[i] = (const u64 *)a[i].data; pb[i] = (const u64 *)b[i].data; }
+    launch_tensor_sum(c, pa.data(), pb.data(), n, o, e2, level, s);
+    ks_modup(c, e2, level, w, s);
+    ks_inner_moddown(c, (const u64 *)rlk->data, level, 1, w, o, o + (size_t)level * c->N, 1, o, s);
+    int rc = finish(c);
+    if (rc == CKKS_OK) { out->level = level; out->ncomp = 2; out->scale = a[0].scale * b[0].scale; }
+    return rc;
+}
+
 extern "C" int32_t ckks_rotate(ckks_ctx *c, const ckks_ct *in, const ckks_evk *key, ckks_ct *out, void *ws, size_t ws_bytes,
                                void *stream) {
     int rc = rotate_checks(c, in, key, 1, out, ws, ws_bytes);

@@ -75,7 +75,44 @@ __global__ void __launch_bounds__(THREADS) tensor_kernel(DevTables c, const u64 
     e2[o0] = r2;
 }
 
+// e (+)= sum_{i < n} tensor(a_i, b_i): lazy 128-bit sums (n <= TS_MAX pairs per launch: 2 n products stay below
+// 2^112), one Barrett step per component, then the previous partial sum is added unless INIT
+template <bool INIT>
+__global__ void __launch_bounds__(THREADS) tensor_sum_kernel(DevTables c, TensorSumArgs args, uint32_t n, u64 *e01, u64 *e2, uint32_t level) {
+    const uint32_t k = blockIdx.x * THREADS + threadIdx.x;
+    if (k >= c.N) return;
+    const uint32_t limb = blockIdx.y;
+    const u64 q = c.mod[limb], mu = c.mu[limb];
+    const size_t o0 = (size_t)limb * c.N + k, o1 = o0 + (size_t)level * c.N;
+    u64 h0 = 0, l0 = 0, h1 = 0, l1 = 0, h2 = 0, l2 = 0;
+    for (uint32_t i = 0; i < n; i++) {
+        const u64 a0 = args.a[i][o0], a1 = args.a[i][o1], b0 = args.b[i][o0], b1 = args.b[i][o1];
+        mac128(h0, l0, a0, b0);
+        mac128(h1, l1, a0, b1);
+        mac128(h1, l1, a1, b0);
+        mac128(h2, l2, a1, b1);
+    }
+    u64 r0 = barrett112(h0, l0, q, mu), r1 = barrett112(h1, l1, q, mu), r2 = barrett112(h2, l2, q, mu);
+    if (!INIT) { r0 = add_mod(r0, e01[o0], q); r1 = add_mod(r1, e01[o1], q); r2 = add_mod(r2, e2[o0], q); }
+    e01[o0] = r0;
+    e01[o1] = r1;
+    e2[o0] = r2;
+}
+
 }  // namespace
+
+void launch_tensor_sum(const ckks_ctx *c, const u64 *const *a, const u64 *const *b, uint32_t n, u64 *e01, u64 *e2, uint32_t level,
+                       cudaStream_t s) {
+    dim3 grid((c->N + THREADS - 1) / THREADS, level);
+    for (uint32_t i0 = 0; i0 < n; i0 += TS_MAX) {
+        TensorSumArgs args;
+        const uint32_t m = n - i0 < TS_MAX ? n - i0 : TS_MAX;
+        for (uint32_t i = 0; i < m; i++) { args.a[i] = a[i0 + i]; args.b[i] = b[i0 + i]; }
+        if (i0 == 0) tensor_sum_kernel<true><<<grid, THREADS, 0, s>>>(c->dev, args, m, e01, e2, level);
+        else tensor_sum_kernel<false><<<grid, THREADS, 0, s>>>(c->dev, args, m, e01, e2, level);
+        count_launches();
+    }
+}
 
 void launch_mul_plain_acc(const ckks_ctx *c, const u64 *const *cts, u64 *const *accs, uint32_t ncts, const u64 *pt,
                           uint32_t level, bool init, cudaStream_t s) {

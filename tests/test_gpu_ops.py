@@ -120,6 +120,41 @@ def test_mul_relin_bit_exact(log_n, L, K, dnum, levels):
     assert e.value.code == binding.ERR_NO_KEY
 
 
+@pytest.mark.parametrize("log_n,L,K,dnum,level,n", [(10, 6, 2, 3, 5, 1), (10, 6, 2, 3, 6, 7), (11, 4, 2, 2, 3, 20), (16, 24, 8, 3, 24, 3)])
+def test_mul_relin_sum_bit_exact(log_n, L, K, dnum, level, n):
+    """Sum of n products with one relinearisation (n = 20 spans two launches of the accumulating kernel)."""
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    P, ctx = params(log_n, L, K, dnum), context(log_n, L, K, dnum)
+    o = P.oracle
+    cl = Client(P, 260 + n)
+    rlk = cl.relin_key()
+    drlk = key_dev(rlk, 0)
+    g = inputs.rng(261, n)
+    zs, ws = g.uniform(-1, 1, (n, P.n)), g.uniform(-1, 1, (n, P.n))
+    sa, sb = 2.0 ** 40, 2.0 ** 38
+    ca = np.stack([cl.encrypt_slots(z, sa, level) for z in zs])
+    cb = np.stack([cl.encrypt_slots(w, sb, level) for w in ws])
+    da, db = [ct_dev(c, sa) for c in ca], [ct_dev(c, sb) for c in cb]
+    out = ctx.mul_relin_sum(da, db, drlk)
+    got = host(out.data)
+    assert out.scale == sa * sb and out.level == level
+    assert np.array_equal(got, o.mul_relin_sum(ca, cb, rlk))
+    assert np.abs(cl.decrypt_slots(got, out.scale) - (zs * ws).sum(0)).max() < truth_tol(log_n) * n
+    if n == 1:
+        assert np.array_equal(got, host(ctx.mul_relin(da[0], db[0], drlk).data))
+    # errors: mixed scales, output aliasing an input, a rotation key instead of the relinearisation key
+    if n > 1:
+        with pytest.raises(binding.CkksError) as e:
+            ctx.mul_relin_sum([da[0], binding.Ciphertext(da[1].data, 2.0 ** 39)], db[:2], drlk)
+        assert e.value.code == binding.ERR_SCALE
+    with pytest.raises(binding.CkksError) as e:
+        ctx.mul_relin_sum(da, db, drlk, out=da[0])
+    assert e.value.code == binding.ERR_ARG
+    with pytest.raises(binding.CkksError) as e:
+        ctx.mul_relin_sum(da, db, binding.SwitchKey(drlk.data, 5))
+    assert e.value.code == binding.ERR_NO_KEY
+
+
 def test_repeatability():
     """Same call twice gives the same bytes (a race would show up as a difference)."""
     from tests.gpu_util import context, ct_dev, host, key_dev
