@@ -483,6 +483,27 @@ void orc_add(const orc_ctx *c, const uint64_t *a, const uint64_t *b, uint64_t *o
     }
 }
 
+/*
+ * Multiplication and addition of a real constant (Section 2.1: Mult and Add with a plaintext that encodes the
+ * same value in every slot).  Such a plaintext is the constant polynomial v = round(c * scale), whose
+ * evaluation-domain image is v in every position.  v is passed as a signed integer (the caller rounds).
+ *   mul: out = ct * v on every component and limb;   add: out = ct with v added to component 0.
+ */
+void orc_mul_const(const orc_ctx *c, const uint64_t *in, int64_t v, uint32_t ncomp, uint32_t level, uint64_t *out) {
+    uint64_t N = c->N;
+    for (uint32_t x = 0; x < ncomp * level; x++) {
+        uint64_t q = c->mod[x % level], r = reduce_signed((i128)v, q);
+        for (uint64_t k = 0; k < N; k++) out[x * N + k] = mulmod(in[x * N + k], r, q);
+    }
+}
+void orc_add_const(const orc_ctx *c, const uint64_t *in, int64_t v, uint32_t ncomp, uint32_t level, uint64_t *out) {
+    uint64_t N = c->N;
+    for (uint32_t x = 0; x < ncomp * level; x++) {
+        uint64_t q = c->mod[x % level], r = x < level ? reduce_signed((i128)v, q) : 0;
+        for (uint64_t k = 0; k < N; k++) out[x * N + k] = addmod(in[x * N + k], r, q);
+    }
+}
+
 /* Galois automorphism by definition, coefficient domain: a(X) -> a(X^g), X^N = -1. */
 void orc_automorphism_coeff(const orc_ctx *c, uint32_t t, const uint64_t *a, uint64_t g, uint64_t *out) {
     uint64_t q = c->mod[t], N = c->N, M = c->M;

@@ -215,6 +215,38 @@ class Oracle:
         lib().orc_add(self._h, _p(a, _u64p), _p(b, _u64p), _p(out, _u64p), C.c_uint32(a.shape[0]), C.c_uint32(a.shape[1]))
         return out
 
+    def mul_const(self, ct, v: int):
+        """ct times the constant polynomial v (a signed integer)."""
+        ct = _u64(ct); out = np.empty_like(ct)
+        lib().orc_mul_const(self._h, _p(ct, _u64p), C.c_int64(v), C.c_uint32(ct.shape[0]), C.c_uint32(ct.shape[1]), _p(out, _u64p))
+        return out
+
+    def add_const(self, ct, v: int):
+        """ct plus the constant polynomial v (a signed integer), i.e. v added to component 0."""
+        ct = _u64(ct); out = np.empty_like(ct)
+        lib().orc_add_const(self._h, _p(ct, _u64p), C.c_int64(v), C.c_uint32(ct.shape[0]), C.c_uint32(ct.shape[1]), _p(out, _u64p))
+        return out
+
+    def poly_eval(self, x, scale: float, coeffs, rlk):
+        """Horner evaluation of sum_k coeffs[k] x^k (degree d = len(coeffs) - 1 >= 1) on a ciphertext, in this order:
+        r = x * round(c_d * q_{l-1});  rescale;  r += round(c_{d-1} * scale(r));  then for k = d-2 .. 0:
+        r = mul_relin(r, x truncated to r's level);  rescale;  r += round(c_k * scale(r)).
+        Scales are tracked as doubles, multiplied and divided in exactly this order.  Returns (ct, scale) at level
+        l - d."""
+        x = _u64(x); level = x.shape[1]; d = len(coeffs) - 1
+        if d < 1 or level < d + 1:
+            raise ValueError("degree must be >= 1 and the ciphertext needs degree + 1 limbs")
+        cs = float(self.q[level - 1])
+        r = self.mul_const(x, int(np.rint(coeffs[d] * cs)))
+        rs = scale * cs
+        r = self.rescale(r); rs = rs / float(self.q[level - 1]); lvl = level - 1
+        r = self.add_const(r, int(np.rint(coeffs[d - 1] * rs)))
+        for k in range(d - 2, -1, -1):
+            r = self.mul_relin(r, x[:, :lvl], rlk); rs = rs * scale
+            r = self.rescale(r); rs = rs / float(self.q[lvl - 1]); lvl -= 1
+            r = self.add_const(r, int(np.rint(coeffs[k] * rs)))
+        return r, rs
+
     def automorphism_coeff(self, a, g: int, t: int):
         a = _u64(a); out = np.empty_like(a)
         lib().orc_automorphism_coeff(self._h, C.c_uint32(t), _p(a, _u64p), C.c_uint64(g), _p(out, _u64p))

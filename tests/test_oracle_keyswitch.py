@@ -233,3 +233,36 @@ def test_mul_relin_sum_pins():
     sep = sum(o.mul_relin(ca[i], cb[i], rlk).astype(object) for i in range(n)) % q
     assert not np.array_equal(sep.astype(np.uint64), out)
     assert np.abs(cl.decrypt_slots(sep.astype(np.uint64), scale * scale) - (zs * ws).sum(0)).max() < 2.0 ** -20
+
+
+def test_const_ops_and_horner_pins():
+    """Constant multiply / add are the plaintext operations with a constant-slot plaintext (checked against the
+    encode + multiply-accumulate path and against decryption), and the Horner evaluation decrypts to the
+    polynomial of the slots."""
+    P = params(11, 8, 2, 4)
+    o = P.oracle
+    cl = Client(P, 58)
+    g = inputs.rng(58)
+    level = 8
+    scale = float(2 ** 50)
+    z = g.uniform(-1, 1, P.n)
+    ct = cl.encrypt_slots(z, scale, level)
+    # a constant-slot plaintext encodes to the constant polynomial round(c * scale): its limbs are that value everywhere
+    c, cs = 0.37, float(P.q[level - 1])
+    pt = o.encode(np.full(P.n, c), cs, level)
+    v = int(np.rint(c * cs))
+    assert all(np.all(pt[i] == np.uint64(v % P.q[i])) for i in range(level))
+    assert np.array_equal(o.mul_const(ct, v), o.mul_plain_acc(ct, pt))
+    assert np.array_equal(o.mul_const(ct, -v), o.mul_const(o.mul_const(ct, v), -1))
+    assert np.abs(cl.decrypt_slots(o.mul_const(ct, v), scale * cs) - c * z).max() < 2.0 ** -30
+    va = int(np.rint(-1.25 * scale))
+    added = o.add_const(ct, va)
+    assert np.array_equal(added[1], ct[1])
+    assert np.abs(cl.decrypt_slots(added, scale) - (z - 1.25)).max() < 2.0 ** -30
+    # Horner: degree 1 (no ciphertext product), 2 and 5
+    rlk = cl.relin_key()
+    for coeffs in ([0.5, -0.25], [0.1, 0.7, -0.3], [1.0, 1.0, 0.5, 1 / 6, 1 / 24, 1 / 120]):
+        out, s_out = o.poly_eval(ct, scale, coeffs, rlk)
+        assert out.shape[1] == level - (len(coeffs) - 1)
+        want = sum(ck * z ** k for k, ck in enumerate(coeffs))
+        assert np.abs(cl.decrypt_slots(out, s_out) - want).max() < 2.0 ** -25, coeffs
