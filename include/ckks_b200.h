@@ -66,7 +66,7 @@ enum {
 /* Operation selectors for ckks_workspace_bytes. */
 enum {
     CKKS_OP_ENCODE = 1, CKKS_OP_MUL_RELIN = 2, CKKS_OP_ROTATE = 3,
-    CKKS_OP_ROTATE_HOISTED = 4, CKKS_OP_RESCALE = 5, CKKS_OP_LINEAR_PROJ = 6
+    CKKS_OP_ROTATE_HOISTED = 4, CKKS_OP_RESCALE = 5, CKKS_OP_LINEAR_PROJ = 6, CKKS_OP_POLY_EVAL = 7
 };
 
 typedef struct ckks_ctx ckks_ctx; /* opaque */
@@ -194,6 +194,26 @@ int32_t ckks_mul_relin(ckks_ctx *ctx, const ckks_ct *a, const ckks_ct *b, const 
  * Errors: as ckks_mul_relin; CKKS_ERR_SCALE if the a_i (or the b_i) disagree in scale. */
 int32_t ckks_mul_relin_sum(ckks_ctx *ctx, const ckks_ct *a, const ckks_ct *b, uint32_t n, const ckks_evk *rlk, ckks_ct *out,
                            void *ws, size_t ws_bytes, void *stream);
+
+/* ---- Constants and polynomials (Section 2.1 Add / Mult with a constant-slot plaintext; Section 3: the
+ * element-wise polynomials that replace the non-linear layers) -------------------------------------------
+ * A plaintext holding the same real value c in every slot is the constant polynomial v = round(c * scale)
+ * (round half to even); its evaluation-domain image is v in every position, so no encode is needed.
+ *   ckks_mul_const: out = in * v with v = round(c * cscale) on all components; out.scale = in.scale * cscale.
+ *                   cscale = 0 selects q_{level-1}, so that a following rescale restores in.scale.
+ *   ckks_add_const: out = in with v = round(c * in.scale) added to component 0; scale and level unchanged.
+ * out may be in.  CKKS_ERR_RANGE if |c * scale| >= 2^62.
+ *   ckks_poly_eval: sum_k coeffs[k] x^k (coeffs: host, degree + 1 doubles, degree >= 1) by Horner's rule:
+ *                   r = x * round(c_d q_{l-1}); rescale; r += c_{d-1};  then for k = d-2 .. 0:
+ *                   r = Mult+relin(r, x truncated to r's level); rescale; r += c_k   (constants at r's scale).
+ *                   x must have ncomp = 2 and level l >= degree + 1; out is written at level l - degree with the
+ *                   scale obtained by multiplying by x.scale and dividing by the dropped prime at every step, in
+ *                   that order.  Workspace: ckks_workspace_bytes(CKKS_OP_POLY_EVAL, l, 0).  A scale close to the
+ *                   primes (2^50) keeps the precision; errors as ckks_mul_relin, plus CKKS_ERR_RANGE. */
+int32_t ckks_mul_const(ckks_ctx *ctx, const ckks_ct *in, double c, double cscale, ckks_ct *out, void *stream);
+int32_t ckks_add_const(ckks_ctx *ctx, const ckks_ct *in, double c, ckks_ct *out, void *stream);
+int32_t ckks_poly_eval(ckks_ctx *ctx, const ckks_ct *x, const double *coeffs, uint32_t degree, const ckks_evk *rlk, ckks_ct *out,
+                       void *ws, size_t ws_bytes, void *stream);
 
 /* ---- Rot_k (Section 2.1, Rot + KeySwitch) ----------------------------------
  * Plain: apply sigma_g (g = key->galois) to both components, key-switch the

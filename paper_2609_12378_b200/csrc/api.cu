@@ -226,6 +226,8 @@ extern "C" size_t ckks_workspace_bytes(const ckks_ctx *c, int32_t op, uint32_t l
         case CKKS_OP_ROTATE: return ks_bytes(c, level);
         case CKKS_OP_ROTATE_HOISTED: return hoisted_bytes(c, level, std::min<uint32_t>(count ? count : 1, KS_MULTI));
         case CKKS_OP_RESCALE: return rescale_bytes(c, level, 2);
+        // two running ciphertexts, the truncated copy of x, then the Mult and rescale scratch
+        case CKKS_OP_POLY_EVAL: return 3 * (size_t)2 * level * limb + ks_bytes(c, level) + (size_t)level * limb + rescale_bytes(c, level, 2);
         default: return 0;
     }
 }
@@ -384,6 +386,95 @@ extern "C" int32_t ckks_mul_relin_sum(ckks_ctx *c, const ckks_ct *a, const ckks_
     ks_inner_moddown(c, (const u64 *)rlk->data, level, 1, w, o, o + (size_t)level * c->N, 1, o, s);
     int rc = finish(c);
     if (rc == CKKS_OK) { out->level = level; out->ncomp = 2; out->scale = a[0].scale * b[0].scale; }
+    return rc;
+}
+
+static bool const_value(double c, double scale, long long *v) {
+    const double x = c * scale;
+    if (!(fabs(x) < 4611686018427387904.0)) return false;      // 2^62; also rejects NaN
+    *v = llrint(x);                                            // round half to even in the default rounding mode
+    return true;
+}
+
+extern "C" int32_t ckks_mul_const(ckks_ctx *c, const ckks_ct *in, double cv, double cscale, ckks_ct *out, void *stream) {
+    if (!c || !ct_ok(in) || !ct_ok(out) || !in->ncomp || in->ncomp > 3 || !(cscale >= 0.0) || !isfinite(cscale)) return CKKS_ERR_ARG;
+    if (!level_ok(c, in->level)) return CKKS_ERR_LEVEL;
+    const double cs = cscale > 0.0 ? cscale : (double)c->mod[in->level - 1];
+    long long v;
+    if (!const_value(cv, cs, &v)) return CKKS_ERR_RANGE;
+    DeviceGuard g(c->device);
+    launch_const(c, (const u64 *)in->data, v, true, (u64 *)out->data, in->ncomp, in->level, (cudaStream_t)stream);
+    int rc = finish(c);
+    if (rc == CKKS_OK) { out->level = in->level; out->ncomp = in->ncomp; out->scale = in->scale * cs; }
+    return rc;
+}
+
+extern "C" int32_t ckks_add_const(ckks_ctx *c, const ckks_ct *in, double cv, ckks_ct *out, void *stream) {
+    if (!c || !ct_ok(in) || !ct_ok(out) || !in->ncomp || in->ncomp > 3) return CKKS_ERR_ARG;
+    if (!level_ok(c, in->level)) return CKKS_ERR_LEVEL;
+    long long v;
+    if (!const_value(cv, in->scale, &v)) return CKKS_ERR_RANGE;
+    DeviceGuard g(c->device);
+    launch_const(c, (const u64 *)in->data, v, false, (u64 *)out->data, in->ncomp, in->level, (cudaStream_t)stream);
+    int rc = finish(c);
+    if (rc == CKKS_OK) { out->level = in->level; out->ncomp = in->ncomp; out->scale = in->scale; }
+    return rc;
+}
+
+extern "C" int32_t ckks_poly_eval(ckks_ctx *c, const ckks_ct *x, const double *coeffs, uint32_t degree, const ckks_evk *rlk, ckks_ct *out,
+                                  void *ws, size_t ws_bytes, void *stream) {
+    if (!c || !ct_ok(x) || !ct_ok(out) || x->ncomp != 2 || !coeffs || degree < 1) return CKKS_ERR_ARG;
+    const uint32_t level = x->level;
+    if (!level_ok(c, level) || level < degree + 1) return CKKS_ERR_LEVEL;
+    if (degree > 1 && (!rlk || !rlk->data || rlk->galois != 0)) return CKKS_ERR_NO_KEY;
+    if (!ws || ws_bytes < ckks_workspace_bytes(c, CKKS_OP_POLY_EVAL, level, 0)) return CKKS_ERR_WORKSPACE;
+    // every constant is fixed (and range-checked) before anything is launched; the scales follow the documented order
+    std::vector<long long> vs(degree + 1);
+    std::vector<double> scales(degree + 1);
+    {
+        const double cs = (double)c->mod[level - 1];
+        if (!const_value(coeffs[degree], cs, &vs[degree])) return CKKS_ERR_RANGE;
+        double rs = x->scale * cs;
+        rs = rs / (double)c->mod[level - 1];
+        uint32_t lvl = level - 1;
+        if (!const_value(coeffs[degree - 1], rs, &vs[degree - 1])) return CKKS_ERR_RANGE;
+        scales[degree - 1] = rs;
+        for (uint32_t k = degree - 1; k-- > 0;) {
+            rs = rs * x->scale;
+            rs = rs / (double)c->mod[lvl - 1];
+            lvl--;
+            if (!const_value(coeffs[k], rs, &vs[k])) return CKKS_ERR_RANGE;
+            scales[k] = rs;
+        }
+    }
+    DeviceGuard g(c->device);
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t N = c->N, ctw = (size_t)2 * level * N;
+    u64 *ra = (u64 *)ws, *rb = ra + ctw, *xt = rb + ctw, *e2 = xt + ctw;
+    u64 *ksw = e2 + (size_t)level * N;
+    u64 *rsw = (u64 *)((char *)ksw + ks_bytes(c, level));
+    const u64 *xd = (const u64 *)x->data;
+    // r = x * c_d; rescale; + c_{d-1}
+    launch_const(c, xd, vs[degree], true, ra, 2, level, s);
+    launch_rescale(c, ra, rb, 2, level, rsw, s);
+    uint32_t lvl = level - 1;
+    launch_const(c, rb, vs[degree - 1], false, rb, 2, lvl, s);
+    u64 *cur = rb, *other = ra;
+    for (uint32_t k = degree - 1; k-- > 0;) {
+        // x truncated to lvl limbs per component
+        for (uint32_t comp = 0; comp < 2; comp++)
+            cudaMemcpyAsync(xt + (size_t)comp * lvl * N, xd + (size_t)comp * level * N, (size_t)lvl * N * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+        KsWorkspace w = ks_carve(c, lvl, ksw);
+        launch_tensor(c, cur, xt, other, e2, lvl, s);
+        ks_modup(c, e2, lvl, w, s);
+        ks_inner_moddown(c, (const u64 *)rlk->data, lvl, 1, w, other, other + (size_t)lvl * N, 1, other, s);
+        launch_rescale(c, other, cur, 2, lvl, rsw, s);
+        lvl--;
+        launch_const(c, cur, vs[k], false, cur, 2, lvl, s);
+    }
+    cudaMemcpyAsync(out->data, cur, (size_t)2 * lvl * N * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+    int rc = finish(c);
+    if (rc == CKKS_OK) { out->level = lvl; out->ncomp = 2; out->scale = scales[0]; }
     return rc;
 }
 

@@ -75,6 +75,24 @@ __global__ void __launch_bounds__(THREADS) tensor_kernel(DevTables c, const u64 
     e2[o0] = r2;
 }
 
+// out = in * v (MUL) or in + v on component 0 (the constant polynomial v, a signed integer, has the value v mod q in
+// every position of the evaluation domain); blockIdx.y = component * level + limb
+template <bool MUL>
+__global__ void __launch_bounds__(THREADS) const_kernel(DevTables c, const u64 *in, long long v, u64 *out, uint32_t level) {
+    const uint32_t half = c.N / 2;
+    const uint32_t x = blockIdx.x * THREADS + threadIdx.x;
+    if (x >= half) return;
+    const uint32_t limb = blockIdx.y % level;
+    const u64 q = c.mod[limb], mu = c.mu[limb];
+    const u64 m = (u64)(v < 0 ? -v : v) % q;
+    u64 r = (v < 0 && m) ? q - m : m;
+    if (!MUL && blockIdx.y >= level) r = 0;
+    const size_t off = (size_t)blockIdx.y * half + x;
+    const ulonglong2 u = reinterpret_cast<const ulonglong2 *>(in)[off];
+    reinterpret_cast<ulonglong2 *>(out)[off] =
+        MUL ? make_ulonglong2(mul_mod(u.x, r, q, mu), mul_mod(u.y, r, q, mu)) : make_ulonglong2(add_mod(u.x, r, q), add_mod(u.y, r, q));
+}
+
 // e (+)= sum_{i < n} tensor(a_i, b_i): lazy 128-bit sums (n <= TS_MAX pairs per launch: 2 n products stay below
 // 2^112), one Barrett step per component, then the previous partial sum is added unless INIT
 template <bool INIT>
@@ -100,6 +118,13 @@ __global__ void __launch_bounds__(THREADS) tensor_sum_kernel(DevTables c, Tensor
 }
 
 }  // namespace
+
+void launch_const(const ckks_ctx *c, const u64 *in, long long v, bool mul, u64 *out, uint32_t ncomp, uint32_t level, cudaStream_t s) {
+    dim3 grid((c->N / 2 + THREADS - 1) / THREADS, ncomp * level);
+    if (mul) const_kernel<true><<<grid, THREADS, 0, s>>>(c->dev, in, v, out, level);
+    else const_kernel<false><<<grid, THREADS, 0, s>>>(c->dev, in, v, out, level);
+    count_launches();
+}
 
 void launch_tensor_sum(const ckks_ctx *c, const u64 *const *a, const u64 *const *b, uint32_t n, u64 *e01, u64 *e2, uint32_t level,
                        cudaStream_t s) {

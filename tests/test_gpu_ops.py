@@ -155,6 +155,47 @@ def test_mul_relin_sum_bit_exact(log_n, L, K, dnum, level, n):
     assert e.value.code == binding.ERR_NO_KEY
 
 
+@pytest.mark.parametrize("log_n,L,K,dnum,level,coeffs", [
+    (11, 8, 2, 4, 8, [0.5, -0.25]),                                   # degree 1: no ciphertext product
+    (11, 8, 2, 4, 8, [1.0, 1.0, 0.5, 1 / 6, 1 / 24, 1 / 120]),        # exp, degree 5
+    (11, 8, 2, 4, 6, [0.1, 0.7, -0.3]),                               # below the top level
+    (16, 24, 8, 3, 24, [0.0, 0.5, 0.0, -1 / 24, 0.0, 1 / 720, 0.0]),  # full ring, degree 6 with a zero leading coefficient
+])
+def test_const_ops_and_poly_eval_bit_exact(log_n, L, K, dnum, level, coeffs):
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    P, ctx = params(log_n, L, K, dnum), context(log_n, L, K, dnum)
+    o = P.oracle
+    cl = Client(P, 270)
+    rlk = cl.relin_key()
+    drlk = key_dev(rlk, 0)
+    z = inputs.rng(271, log_n).uniform(-1, 1, P.n)
+    scale = float(2 ** 50)
+    ct = cl.encrypt_slots(z, scale, level)
+    d = ct_dev(ct, scale)
+    # constants
+    cs = float(P.q[level - 1])
+    m = ctx.mul_const(d, -0.37)
+    assert m.scale == scale * cs and np.array_equal(host(m.data), o.mul_const(ct, int(np.rint(-0.37 * cs))))
+    m2 = ctx.mul_const(d, 3.0, 2.0 ** 20)
+    assert m2.scale == scale * 2.0 ** 20 and np.array_equal(host(m2.data), o.mul_const(ct, 3 << 20))
+    a = ctx.add_const(d, 1.25)
+    assert a.scale == scale and np.array_equal(host(a.data), o.add_const(ct, int(np.rint(1.25 * scale))))
+    with pytest.raises(binding.CkksError) as e:
+        ctx.add_const(d, 1.0e4)                  # 10^4 * 2^50 does not fit 2^62
+    assert e.value.code == binding.ERR_RANGE
+    # polynomial
+    out = ctx.poly_eval(d, coeffs, drlk)
+    want, want_scale = o.poly_eval(ct, scale, coeffs, rlk)
+    assert out.level == level - (len(coeffs) - 1) and out.scale == want_scale
+    got = host(out.data)
+    assert np.array_equal(got, want)
+    truth = sum(ck * z ** k for k, ck in enumerate(coeffs))
+    assert np.abs(cl.decrypt_slots(got, out.scale) - truth).max() < 2.0 ** -22
+    with pytest.raises(binding.CkksError) as e:
+        ctx.poly_eval(d, [1.0] * (level + 1), drlk)          # degree = level: not enough limbs
+    assert e.value.code == binding.ERR_LEVEL
+
+
 def test_repeatability():
     """Same call twice gives the same bytes (a race would show up as a difference)."""
     from tests.gpu_util import context, ct_dev, host, key_dev
