@@ -312,7 +312,7 @@ def run_cuda(args):
 
     pk, pk_kind = peaks()
     limb_ntts = NTT_BATCH * L
-    # Roofline of the dominant kernel family (the ntt16 kernels: 54 % of the step in the ncu launch list).
+    # Roofline of the dominant kernel family (the ntt16 kernels: 55 % of the step in the ncu launch list).
     # The butterflies run on the FP64 pipe, which ncu shows to be the busiest unit of the column passes, so the
     # bound is "alu": algorithmic work = 8 FP64 instructions per butterfly (6 for the exact twiddle product with
     # its quotient, 2 for the sum and difference), N/2 * log2 N butterflies per limb; peak = 64 FP64 instructions
@@ -335,9 +335,9 @@ def run_cuda(args):
                     "peak_kind": "measured in this run: the transform's radix-16 butterfly groups on registers, 4 CTAs x 256 threads per SM"},
                 "hbm": {"achieved": hbm_achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": hbm_achieved / pk["hbm_gbs"],
                         "algorithmic_bytes": ntt_bytes, "peak_kind": pk_kind + " copy bandwidth"},
-                "others": {"ntt16 family": "54.0 % of the step (profiles/bench_step_launch_list.md)",
-                           "mac_mma_kernel": "14.8 % of the step; legacy tensor path 32 % busy, DRAM 51 %, see profiles/mac_mma_projection_8shards.md",
-                           "modup + moddown_conv + inner_product": "27.5 % of the step; FP64 pipe 67 % (conversions), DRAM 72 % (inner product)"}}
+                "others": {"ntt16 family": "55.0 % of the step (profiles/bench_step_launch_list.md)",
+                           "mac_mma_kernel": "15.0 % of the step; legacy tensor path 32 % busy, DRAM 51 %, see profiles/mac_mma_projection_8shards.md",
+                           "modup + moddown_conv + inner_product": "27.8 % of the step; FP64 pipe 67 % (conversions), DRAM 72 % (inner product)"}}
     cpu = oracle_sample()
     jm = job_metrics(world, a_ms, b_ms, c_ms)
     line = {
