@@ -247,6 +247,38 @@ class Oracle:
             r = self.add_const(r, int(np.rint(coeffs[k] * rs)))
         return r, rs
 
+    def poly_eval_tree(self, x, scale: float, coeffs, rlk):
+        """sum_k coeffs[k] x^k (degree d >= 2) in depth ceil(log2 d) + 1 instead of d.  Order of steps:
+        powers: pw[1] = x; for k = 2..d: a = k // 2, b = k - a, lv = min(level[a], level[b]),
+          pw[k] = rescale(mul_relin(pw[a][:, :lv], pw[b][:, :lv])), scale[k] = scale[a] * scale[b] / q_{lv-1};
+        combination at level Lt = level[d] and scale T = scale(x) * q_{Lt-1}:
+          acc = sum over k = 1..d with coeffs[k] != 0, in increasing k, of pw[k][:, :Lt] * round(coeffs[k] * (T / scale[k]));
+        result = rescale(acc) + round(coeffs[0] * (T / q_{Lt-1})).  Returns (ct, scale) at level Lt - 1."""
+        x = _u64(x); level = x.shape[1]; d = len(coeffs) - 1
+        depth = (d - 1).bit_length()
+        if d < 2 or level < depth + 2:
+            raise ValueError("degree must be >= 2 and the ciphertext needs ceil(log2 degree) + 2 limbs")
+        pw, sc = {1: x}, {1: scale}
+        for k in range(2, d + 1):
+            a = k // 2; b = k - a
+            lv = min(pw[a].shape[1], pw[b].shape[1])
+            t = self.mul_relin(pw[a][:, :lv], pw[b][:, :lv], rlk)
+            pw[k] = self.rescale(t)
+            sc[k] = sc[a] * sc[b] / float(self.q[lv - 1])
+        Lt = pw[d].shape[1]
+        T = scale * float(self.q[Lt - 1])
+        acc = None
+        for k in range(1, d + 1):
+            if coeffs[k] == 0.0:
+                continue
+            term = self.mul_const(pw[k][:, :Lt], int(np.rint(coeffs[k] * (T / sc[k]))))
+            acc = term if acc is None else self.add(acc, term)
+        if acc is None:
+            raise ValueError("all non-constant coefficients are zero")
+        out = self.rescale(acc)
+        so = T / float(self.q[Lt - 1])
+        return self.add_const(out, int(np.rint(coeffs[0] * so))), so
+
     def automorphism_coeff(self, a, g: int, t: int):
         a = _u64(a); out = np.empty_like(a)
         lib().orc_automorphism_coeff(self._h, C.c_uint32(t), _p(a, _u64p), C.c_uint64(g), _p(out, _u64p))

@@ -266,3 +266,26 @@ def test_const_ops_and_horner_pins():
         assert out.shape[1] == level - (len(coeffs) - 1)
         want = sum(ck * z ** k for k, ck in enumerate(coeffs))
         assert np.abs(cl.decrypt_slots(out, s_out) - want).max() < 2.0 ** -25, coeffs
+
+
+def test_poly_eval_tree_pins():
+    """Log-depth polynomial evaluation: uses ceil(log2 d) + 1 levels, decrypts to the polynomial of the slots, and
+    agrees with the Horner form (a different sequence of integer operations) to within the scheme's noise."""
+    P = params(11, 8, 2, 4)
+    o = P.oracle
+    cl = Client(P, 59)
+    z = inputs.rng(59).uniform(-1, 1, P.n)
+    level, scale = 8, float(2 ** 50)
+    ct = cl.encrypt_slots(z, scale, level)
+    rlk = cl.relin_key()
+    for coeffs in ([0.1, 0.7, -0.3], [1.0, 1.0, 0.5, 1 / 6, 1 / 24, 1 / 120], [0.0, 1.0, 0.0, -1 / 6, 0.0, 1 / 120, 0.0, -1 / 5040],
+                   [0.3] + [(-1) ** k / (k + 1) for k in range(1, 16)]):
+        d = len(coeffs) - 1
+        out, so = o.poly_eval_tree(ct, scale, coeffs, rlk)
+        assert out.shape[1] == level - ((d - 1).bit_length() + 1)
+        want = sum(ck * z ** k for k, ck in enumerate(coeffs))
+        got = cl.decrypt_slots(out, so)
+        assert np.abs(got - want).max() < 2.0 ** -25, d
+        if d <= 7:
+            h, sh = o.poly_eval(ct, scale, coeffs, rlk)
+            assert np.abs(cl.decrypt_slots(h, sh) - got).max() < 2.0 ** -25
