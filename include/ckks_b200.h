@@ -66,7 +66,8 @@ enum {
 /* Operation selectors for ckks_workspace_bytes. */
 enum {
     CKKS_OP_ENCODE = 1, CKKS_OP_MUL_RELIN = 2, CKKS_OP_ROTATE = 3,
-    CKKS_OP_ROTATE_HOISTED = 4, CKKS_OP_RESCALE = 5, CKKS_OP_LINEAR_PROJ = 6, CKKS_OP_POLY_EVAL = 7
+    CKKS_OP_ROTATE_HOISTED = 4, CKKS_OP_RESCALE = 5, CKKS_OP_LINEAR_PROJ = 6, CKKS_OP_POLY_EVAL = 7,
+    CKKS_OP_POLY_EVAL_TREE = 8 /* count = degree */
 };
 
 typedef struct ckks_ctx ckks_ctx; /* opaque */
@@ -214,6 +215,14 @@ int32_t ckks_mul_const(ckks_ctx *ctx, const ckks_ct *in, double c, double cscale
 int32_t ckks_add_const(ckks_ctx *ctx, const ckks_ct *in, double c, ckks_ct *out, void *stream);
 int32_t ckks_poly_eval(ckks_ctx *ctx, const ckks_ct *x, const double *coeffs, uint32_t degree, const ckks_evk *rlk, ckks_ct *out,
                        void *ws, size_t ws_bytes, void *stream);
+/* The same polynomial in depth ceil(log2 degree) + 1 (degree >= 2, level >= depth + 1): powers x^k = x^(k/2) *
+ * x^(k - k/2) for k = 2..degree (Mult + relinearisation, rescale; operands truncated to the lower of their levels),
+ * then, at the level Lt of x^degree and the scale T = x.scale * q_{Lt-1}, acc = sum over k >= 1 with coeffs[k] != 0, in
+ * increasing k, of x^k * round(coeffs[k] * (T / scale(x^k))), a rescale, and round(coeffs[0] * scale) added last.
+ * out is written at level Lt - 1 with scale T / q_{Lt-1}.  Workspace: ckks_workspace_bytes(CKKS_OP_POLY_EVAL_TREE,
+ * level, degree).  CKKS_ERR_ARG if all non-constant coefficients are zero. */
+int32_t ckks_poly_eval_tree(ckks_ctx *ctx, const ckks_ct *x, const double *coeffs, uint32_t degree, const ckks_evk *rlk, ckks_ct *out,
+                            void *ws, size_t ws_bytes, void *stream);
 
 /* ---- Rot_k (Section 2.1, Rot + KeySwitch) ----------------------------------
  * Plain: apply sigma_g (g = key->galois) to both components, key-switch the

@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(_HERE, "libckks_b200.so")
 
 OK, ERR_ARG, ERR_LEVEL, ERR_SCALE, ERR_NO_KEY, ERR_WORKSPACE, ERR_RANGE, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT = (
     0, -1, -2, -3, -4, -5, -6, -7, -8, -9)
-OP_ENCODE, OP_MUL_RELIN, OP_ROTATE, OP_ROTATE_HOISTED, OP_RESCALE, OP_LINEAR_PROJ, OP_POLY_EVAL = 1, 2, 3, 4, 5, 6, 7
+OP_ENCODE, OP_MUL_RELIN, OP_ROTATE, OP_ROTATE_HOISTED, OP_RESCALE, OP_LINEAR_PROJ, OP_POLY_EVAL, OP_POLY_EVAL_TREE = 1, 2, 3, 4, 5, 6, 7, 8
 
 EXPORTS = [
     "ckks_context_create", "ckks_context_destroy", "ckks_status_string", "ckks_last_cuda_error",
@@ -22,7 +22,7 @@ EXPORTS = [
     "ckks_encode_range_flag", "ckks_mul_plain_acc", "ckks_add", "ckks_mul_relin", "ckks_rotate",
     "ckks_rotate_hoisted", "ckks_rescale", "ckks_linear_proj", "ckks_linear_proj_workspace_bytes",
     "ckks_linear_proj_rotations", "ckks_kernel_launches", "ckks_device_status", "ckks_rescale_static",
-    "ckks_ntt_butterfly_probe", "ckks_mul_relin_sum", "ckks_mul_const", "ckks_add_const", "ckks_poly_eval", "ckks_linear_proj_multi", "ckks_linear_proj_multi_workspace_bytes",
+    "ckks_ntt_butterfly_probe", "ckks_mul_relin_sum", "ckks_mul_const", "ckks_add_const", "ckks_poly_eval", "ckks_poly_eval_tree", "ckks_linear_proj_multi", "ckks_linear_proj_multi_workspace_bytes",
 ]
 
 
@@ -80,6 +80,7 @@ def load():
         "ckks_mul_const": (i32, [vp, C.POINTER(CCt), dbl, dbl, C.POINTER(CCt), vp]),
         "ckks_add_const": (i32, [vp, C.POINTER(CCt), dbl, C.POINTER(CCt), vp]),
         "ckks_poly_eval": (i32, [vp, C.POINTER(CCt), C.POINTER(dbl), u32, C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
+        "ckks_poly_eval_tree": (i32, [vp, C.POINTER(CCt), C.POINTER(dbl), u32, C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
         "ckks_rotate": (i32, [vp, C.POINTER(CCt), C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
         "ckks_rotate_hoisted": (i32, [vp, C.POINTER(CCt), C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
         "ckks_rescale": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), vp, sz, vp]),
@@ -307,6 +308,20 @@ class Context:
         ck = CEvk(_dev_u64(rlk.data).data_ptr() if rlk is not None else None, rlk.galois if rlk is not None else 0)
         self._check(load().ckks_poly_eval(self._h, C.byref(_cct(x)), ca, d, C.byref(ck), C.byref(co), ws.data_ptr(), ws.numel(),
                                           _stream_ptr(stream)))
+        out.scale = co.scale
+        return out
+
+    def poly_eval_tree(self, x: Ciphertext, coeffs, rlk: SwitchKey, stream=None):
+        """sum_k coeffs[k] x^k in depth ceil(log2 degree) + 1; returns a ciphertext at level x.level - depth - 1."""
+        d = len(coeffs) - 1
+        depth = max(d - 1, 0).bit_length()
+        out = self.empty_ct(max(x.level - depth - 1, 1))
+        ws = self.workspace(self.workspace_bytes(OP_POLY_EVAL_TREE, x.level, d))
+        ca = (C.c_double * (d + 1))(*[float(v) for v in coeffs])
+        co = _cct(out)
+        ck = CEvk(_dev_u64(rlk.data).data_ptr(), rlk.galois)
+        self._check(load().ckks_poly_eval_tree(self._h, C.byref(_cct(x)), ca, d, C.byref(ck), C.byref(co), ws.data_ptr(), ws.numel(),
+                                               _stream_ptr(stream)))
         out.scale = co.scale
         return out
 

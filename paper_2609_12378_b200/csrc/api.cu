@@ -228,6 +228,9 @@ extern "C" size_t ckks_workspace_bytes(const ckks_ctx *c, int32_t op, uint32_t l
         case CKKS_OP_RESCALE: return rescale_bytes(c, level, 2);
         // two running ciphertexts, the truncated copy of x, then the Mult and rescale scratch
         case CKKS_OP_POLY_EVAL: return 3 * (size_t)2 * level * limb + ks_bytes(c, level) + (size_t)level * limb + rescale_bytes(c, level, 2);
+        // the powers x^2..x^degree, two truncated operands, the product, the accumulator and a term, then the scratch
+        case CKKS_OP_POLY_EVAL_TREE:
+            return ((size_t)(count > 1 ? count - 1 : 1) + 5) * 2 * level * limb + ks_bytes(c, level) + (size_t)level * limb + rescale_bytes(c, level, 2);
         default: return 0;
     }
 }
@@ -475,6 +478,77 @@ extern "C" int32_t ckks_poly_eval(ckks_ctx *c, const ckks_ct *x, const double *c
     cudaMemcpyAsync(out->data, cur, (size_t)2 * lvl * N * sizeof(u64), cudaMemcpyDeviceToDevice, s);
     int rc = finish(c);
     if (rc == CKKS_OK) { out->level = lvl; out->ncomp = 2; out->scale = scales[0]; }
+    return rc;
+}
+
+extern "C" int32_t ckks_poly_eval_tree(ckks_ctx *c, const ckks_ct *x, const double *coeffs, uint32_t degree, const ckks_evk *rlk,
+                                       ckks_ct *out, void *ws, size_t ws_bytes, void *stream) {
+    if (!c || !ct_ok(x) || !ct_ok(out) || x->ncomp != 2 || !coeffs || degree < 2) return CKKS_ERR_ARG;
+    const uint32_t level = x->level;
+    uint32_t depth = 0;
+    while ((1u << depth) < degree) depth++;
+    if (!level_ok(c, level) || level < depth + 2) return CKKS_ERR_LEVEL;
+    if (!rlk || !rlk->data || rlk->galois != 0) return CKKS_ERR_NO_KEY;
+    if (!ws || ws_bytes < ckks_workspace_bytes(c, CKKS_OP_POLY_EVAL_TREE, level, degree)) return CKKS_ERR_WORKSPACE;
+    // levels and scales of the powers, the combination's constants: all fixed and range-checked before the first launch
+    std::vector<uint32_t> lvl(degree + 1);
+    std::vector<double> sc(degree + 1);
+    lvl[1] = level; sc[1] = x->scale;
+    for (uint32_t k = 2; k <= degree; k++) {
+        const uint32_t a = k / 2, b = k - a, lv = std::min(lvl[a], lvl[b]);
+        sc[k] = sc[a] * sc[b] / (double)c->mod[lv - 1];
+        lvl[k] = lv - 1;
+    }
+    const uint32_t Lt = lvl[degree];
+    const double T = x->scale * (double)c->mod[Lt - 1], so = T / (double)c->mod[Lt - 1];
+    std::vector<long long> vs(degree + 1, 0);
+    bool any = false;
+    for (uint32_t k = 1; k <= degree; k++) {
+        if (coeffs[k] == 0.0) continue;
+        any = true;
+        if (!const_value(coeffs[k], T / sc[k], &vs[k])) return CKKS_ERR_RANGE;
+    }
+    if (!any) return CKKS_ERR_ARG;
+    if (!const_value(coeffs[0], so, &vs[0])) return CKKS_ERR_RANGE;
+
+    DeviceGuard g(c->device);
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t N = c->N, ctw = (size_t)2 * level * N;
+    u64 *pw = (u64 *)ws;                                        // x^k at pw + (k - 2) * ctw, k >= 2
+    u64 *ta = pw + (size_t)(degree - 1) * ctw, *tb = ta + ctw, *prod = tb + ctw, *acc = prod + ctw, *term = acc + ctw;
+    u64 *e2 = term + ctw, *ksw = e2 + (size_t)level * N;
+    u64 *rsw = (u64 *)((char *)ksw + ks_bytes(c, level));
+    const u64 *xd = (const u64 *)x->data;
+    auto power = [&](uint32_t k) { return k == 1 ? xd : pw + (size_t)(k - 2) * ctw; };
+    // [2][from][N] -> [2][to][N], to <= from
+    auto truncate = [&](const u64 *src, uint32_t from, uint32_t to, u64 *dst) {
+        for (uint32_t comp = 0; comp < 2; comp++)
+            cudaMemcpyAsync(dst + (size_t)comp * to * N, src + (size_t)comp * from * N, (size_t)to * N * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+    };
+    for (uint32_t k = 2; k <= degree; k++) {
+        const uint32_t a = k / 2, b = k - a, lv = std::min(lvl[a], lvl[b]);
+        const u64 *pa = power(a), *pb = power(b);
+        if (lvl[a] != lv) { truncate(pa, lvl[a], lv, ta); pa = ta; }
+        if (lvl[b] != lv) { truncate(pb, lvl[b], lv, tb); pb = tb; }
+        KsWorkspace w = ks_carve(c, lv, ksw);
+        launch_tensor(c, pa, pb, prod, e2, lv, s);
+        ks_modup(c, e2, lv, w, s);
+        ks_inner_moddown(c, (const u64 *)rlk->data, lv, 1, w, prod, prod + (size_t)lv * N, 1, prod, s);
+        launch_rescale(c, prod, pw + (size_t)(k - 2) * ctw, 2, lv, rsw, s);
+    }
+    bool first = true;
+    for (uint32_t k = 1; k <= degree; k++) {
+        if (coeffs[k] == 0.0) continue;
+        const u64 *pk = power(k);
+        if (lvl[k] != Lt) { truncate(pk, lvl[k], Lt, ta); pk = ta; }
+        launch_const(c, pk, vs[k], true, first ? acc : term, 2, Lt, s);
+        if (!first) launch_add(c, acc, term, acc, 2, Lt, s);
+        first = false;
+    }
+    launch_rescale(c, acc, (u64 *)out->data, 2, Lt, rsw, s);
+    launch_const(c, (const u64 *)out->data, vs[0], false, (u64 *)out->data, 2, Lt - 1, s);
+    int rc = finish(c);
+    if (rc == CKKS_OK) { out->level = Lt - 1; out->ncomp = 2; out->scale = so; }
     return rc;
 }
 

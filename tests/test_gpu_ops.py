@@ -196,6 +196,35 @@ def test_const_ops_and_poly_eval_bit_exact(log_n, L, K, dnum, level, coeffs):
     assert e.value.code == binding.ERR_LEVEL
 
 
+@pytest.mark.parametrize("log_n,L,K,dnum,level,coeffs", [
+    (11, 8, 2, 4, 8, [0.1, 0.7, -0.3]),
+    (11, 8, 2, 4, 8, [0.0, 1.0, 0.0, -1 / 6, 0.0, 1 / 120, 0.0, -1 / 5040]),           # zero coefficients are skipped
+    (11, 8, 2, 4, 7, [0.3] + [(-1) ** k / (k + 1) for k in range(1, 16)]),                # degree 15 in 5 levels
+    (16, 24, 8, 3, 24, [1.0, 1.0, 0.5, 1 / 6, 1 / 24, 1 / 120, 1 / 720, 1 / 5040, 1 / 40320]),   # full ring, degree 8
+])
+def test_poly_eval_tree_bit_exact(log_n, L, K, dnum, level, coeffs):
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    P, ctx = params(log_n, L, K, dnum), context(log_n, L, K, dnum)
+    o = P.oracle
+    cl = Client(P, 280)
+    rlk = cl.relin_key()
+    drlk = key_dev(rlk, 0)
+    z = inputs.rng(281, log_n).uniform(-1, 1, P.n)
+    scale = float(2 ** 50)
+    ct = cl.encrypt_slots(z, scale, level)
+    out = ctx.poly_eval_tree(ct_dev(ct, scale), coeffs, drlk)
+    want, want_scale = o.poly_eval_tree(ct, scale, coeffs, rlk)
+    d = len(coeffs) - 1
+    assert out.level == level - ((d - 1).bit_length() + 1) and out.scale == want_scale
+    got = host(out.data)
+    assert np.array_equal(got, want)
+    truth = sum(ck * z ** k for k, ck in enumerate(coeffs))
+    assert np.abs(cl.decrypt_slots(got, out.scale) - truth).max() < 2.0 ** -22
+    with pytest.raises(binding.CkksError) as e:
+        ctx.poly_eval_tree(ct_dev(ct, scale), [1.0] + [0.0] * d, drlk)
+    assert e.value.code == binding.ERR_ARG
+
+
 def test_repeatability():
     """Same call twice gives the same bytes (a race would show up as a difference)."""
     from tests.gpu_util import context, ct_dev, host, key_dev
