@@ -27,7 +27,8 @@
 // tensor pipe is idle most of the time and the 16 epilogue warps are busy 85 % of it.  With accumulators in registers
 // the products of equal weight a + b add up inside the MMA (13 sums per output); here all 49 arrive separately and
 // are folded by integer instructions (about 300 per output).  Folding them in the MMA needs the byte-shifted copies
-// of one operand along K (a Toeplitz expansion) and M = 64 giants per tile.
+// of one operand along K (a Toeplitz expansion) and M = 64 giants per tile.  More read-back warps (20 or 24 instead of
+// 16) change nothing (18.9 - 19.4 ms): the read-back is bound by instruction issue, not by latency.
 #include "common.cuh"
 
 namespace {
