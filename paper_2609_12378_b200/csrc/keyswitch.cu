@@ -172,7 +172,7 @@ __global__ void __launch_bounds__(THREADS) inner_product_kernel(DevTables c, con
 // conv[comp][i][k] = sum_a centre([u_{p_a} Phat_a^-1]) (Phat_a mod q_i)  mod q_i   (coefficient domain)
 // Same shape as ModUp: the K centred special residues are formed once per thread, then a chunk of targets is walked.
 template <uint32_t KK>
-__global__ void __launch_bounds__(THREADS) moddown_conv_kernel(DevTables c, const u64 *u, u64 *conv, uint32_t level, uint32_t CHUNK) {
+__global__ void __launch_bounds__(THREADS, 6) moddown_conv_kernel(DevTables c, const u64 *u, u64 *conv, uint32_t level, uint32_t CHUNK) {
     __shared__ double2 s_w[CONV_CHUNK_MAX][KK];     // Phat_a mod q_i and its quotient by q_i
     __shared__ double2 s_m[CONV_CHUNK_MAX];         // q_i, 1 / q_i
     const uint32_t k = blockIdx.x * THREADS + threadIdx.x;
