@@ -78,7 +78,7 @@ int make_plan(const ckks_ctx *c, const ckks_proj_desc *d, ProjPlan &p) {
     return CKKS_OK;
 }
 
-struct ProjWs { size_t baby, xin, pts, ptt, slots, enc, acc, total, tmp, ks, rs, bytes; uint32_t gg; };
+struct ProjWs { size_t baby, xin, pts, ptt, slots, enc, acc, total, tmp, ks, rs, bytes; uint32_t gg; bool per_block; };
 
 constexpr uint32_t MAC_GT = 4, MAC_ST = 2;   // register tile of the multiply-accumulate kernel: giants x shards
 
@@ -87,10 +87,14 @@ ProjWs proj_layout(const ckks_ctx *c, const ProjPlan &p, uint32_t level) {
     const size_t nib = p.ins.size();
     ProjWs w;
     // giant steps are processed in groups of gg: their plaintexts are encoded in one batch and
-    // multiply-accumulated in one launch (about 16 * B plaintexts live at a time)
-    w.gg = std::max<uint32_t>(1, std::min<uint32_t>(p.gmax, 16 / (uint32_t)nib ? 16 / (uint32_t)nib : 1));
+    // multiply-accumulated in one launch (about 16 * B plaintexts live at a time).  With the tensor-core kernel a
+    // group is 16 giants and the input blocks are taken one after the other (accumulating launches), so its 16-row
+    // tiles are full whatever the number of input blocks; the fallback kernel takes all blocks at once.
+    w.per_block = mac_mma_supported(c, p.B);
+    if (w.per_block) w.gg = std::max<uint32_t>(1, std::min<uint32_t>(p.gmax, 16));
+    else w.gg = std::max<uint32_t>(1, std::min<uint32_t>(p.gmax, 16 / (uint32_t)nib ? 16 / (uint32_t)nib : 1));
     w.gg = (w.gg + MAC_GT - 1) / MAC_GT * MAC_GT;
-    const size_t npt = (size_t)w.gg * nib * p.B;
+    const size_t npt = (size_t)w.gg * (w.per_block ? 1 : nib) * p.B;
     size_t off = 0;
     w.baby = off;  off += align256(ct * p.S * nib * p.B);   // tiled: rows (shard * J + j) * 2 + component
     w.xin = off;   off += align256(ct * p.S * nib);         // the inputs side by side, plain layout
@@ -714,6 +718,26 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
             for (uint32_t g0 = 0; g0 < gcount; g0 += L.gg) {
                 const uint32_t ng = std::min(L.gg, gcount - g0);
                 const uint32_t J = nib * B;
+                if (L.per_block) {
+                    // one input block at a time: encode its ng x B diagonals, multiply-accumulate them with that block's
+                    // baby rows into the group's accumulators.  A block that has run out of diagonals takes part with
+                    // fewer giants; the accumulators are then cleared first so that every launch can accumulate.
+                    bool full0 = g0 + ng <= std::min(p.ins[0].size, o.size) / B;
+                    if (!full0) cudaMemsetAsync(acc, 0, (size_t)ng * S * ctl * sizeof(u64), s);
+                    for (uint32_t ib = 0; ib < nib; ib++) {
+                        const Block &i = p.ins[ib];
+                        const uint32_t cnt = std::min(i.size, o.size) / B;
+                        if (g0 >= cnt) continue;
+                        const uint32_t ngi = std::min(ng, cnt - g0);
+                        for (uint32_t gl = 0; gl < ngi; gl++)
+                            launch_extract_diagonals(c, W, d->d_out, i.start, i.size, o.start, o.size, p.F, T, (g0 + gl) * B, B, (g0 + gl) * B,
+                                                     slots + (size_t)gl * B * c->n, s);
+                        TiledOut to;
+                        to.R = ngi * B; to.row0 = 0; to.row_stride = 1;
+                        launch_encode(c, slots, nullptr, ngi * B, pt_scale, level, pts, encw, s, to, ptt);
+                        launch_mac_mma(c, baby, ptt, acc, B, S, ngi, level, s, J, ib * B, !full0 || ib > 0);
+                    }
+                } else {
                 // plaintexts of the group: pts[(gl * nib + ib) * B + b]; a block pair that has run out of diagonals
                 // contributes zero plaintexts
                 bool ragged = false;
@@ -744,6 +768,7 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
                     const uint32_t stiles = (S + MAC_ST - 1) / MAC_ST, gtiles = (ng + MAC_GT - 1) / MAC_GT;
                     mac_tile_kernel<<<dim3(stiles * gtiles, N / MAC_THREADS, level), MAC_THREADS, 0, s>>>(c->dev, baby, ptt, acc, J, S, ng, level);
                     count_launches();
+                }
                 }
                 for (uint32_t gl = 0; gl < ng; gl++) {
                     const uint32_t gi = g0 + gl;

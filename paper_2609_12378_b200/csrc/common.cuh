@@ -262,8 +262,10 @@ void launch_to_tiled(const ckks_ctx *c, const u64 *src, size_t src_stride, uint3
 // Tensor-core multiply-accumulate of a giant-step group (mac_mma.cu)
 bool mac_mma_supported(const ckks_ctx *c, uint32_t J);
 // baby, pts: tiled buffers with 2 * S * J rows ((shard * J + j) * 2 + component) and G * J rows (g * J + j)
+// the baby buffer may hold Jx >= J rows per shard and component, of which rows j0 .. j0 + J - 1 are used (Jx = 0: J);
+// accumulate: add to acc instead of overwriting it
 bool launch_mac_mma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level,
-                    cudaStream_t s);
+                    cudaStream_t s, uint32_t Jx = 0, uint32_t j0 = 0, bool accumulate = false);
 
 // register-resident forward butterflies (measurement aid, ntt.cu); sink: device scratch of SMs * 4 * 256 words
 uint64_t launch_butterfly_probe(const ckks_ctx *c, uint32_t iters, u64 *sink, cudaStream_t s);
@@ -271,7 +273,7 @@ uint64_t launch_butterfly_probe(const ckks_ctx *c, uint32_t iters, u64 *sink, cu
 // the same on tcgen05 / TMEM (mac_umma.cu); J <= 64
 bool mac_umma_supported(const ckks_ctx *c, uint32_t J);
 bool launch_mac_umma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level,
-                     cudaStream_t s);
+                     cudaStream_t s, uint32_t Jx = 0, uint32_t j0 = 0, bool accumulate = false);
 
 void launch_rescale(const ckks_ctx *c, const u64 *in, u64 *out, uint32_t ncomp, uint32_t level, u64 *ws, cudaStream_t s);
 

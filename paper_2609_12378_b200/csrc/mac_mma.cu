@@ -93,7 +93,8 @@ struct TileIt {
 template <uint32_t COEF, uint32_t NW>
 __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_kernel(DevTables c, const u64 *__restrict__ baby,
                                                                            const u64 *__restrict__ pts, u64 *__restrict__ acc, uint32_t J,
-                                                                           uint32_t S, uint32_t G, uint32_t level, uint32_t ntiles) {
+                                                                           uint32_t S, uint32_t G, uint32_t level, uint32_t ntiles,
+                                                                           uint32_t Jx, uint32_t j0, uint32_t accumulate) {
     using T = Geo<COEF>;
     constexpr uint32_t THREADS = COEF * 64 / NW, CH = T::CH;
     constexpr uint32_t AH = THREADS / (CH * MK);      // blocks a loaded side by side; a thread walks a = arow + AH it
@@ -114,7 +115,7 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_kernel(DevTa
     // loader: a thread always fetches the 16-byte chunk ch of row jj of the step and walks blocks a = arow + AH it of
     // W and of X, so its shared-memory addresses are one base plus constants
     const uint32_t ch = tid % CH, jj = (tid / CH) % MK, arow = tid / (CH * MK);
-    const uint32_t Rw = G * J, Rx = 2 * S * J;
+    const uint32_t Rw = G * J, Rx = 2 * S * Jx;          // the baby buffer has Jx rows per shard and component; this launch uses rows j0 .. j0 + J - 1
     const uint32_t sm_thread = (uint32_t)__cvta_generic_to_shared(ring) + T::tile_off(arow, jj, ch);
     TileIt lt;                                    // tile of the step the loader issues next
     lt.init(t_begin, coltiles, gtiles, xblocks);
@@ -127,7 +128,7 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_kernel(DevTa
             const size_t blk = (size_t)lt.i * (c.N >> 6) + lt.xb / XB64;
             const uint32_t in_blk = (lt.xb % XB64) * COEF + 2 * ch, j = lks * MK + jj;
             wrow = pts + blk * Rw * 64 + in_blk + (size_t)j * 64;
-            xrow = baby + blk * Rx * 64 + in_blk + (size_t)(2 * j + (arow & 1)) * 64;
+            xrow = baby + blk * Rx * 64 + in_blk + (size_t)(2 * (j0 + j) + (arow & 1)) * 64;
             lg0 = lt.zg * MG + arow;
             lsh0 = lt.zc * (MS / 2) + (arow >> 1);
             lsm = sm_thread + (lstep % STAGES) * T::STAGE_BYTES;
@@ -143,7 +144,7 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_kernel(DevTa
     auto load_x = [&](uint32_t k) {
         if (lstep < nsteps) {
             const uint32_t sh = min(lsh0 + (AH / 2) * k, S - 1);
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(lsm + T::BOX_BYTES + k * AH * T::GPITCH), "l"(xrow + (size_t)sh * J * 128)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(lsm + T::BOX_BYTES + k * AH * T::GPITCH), "l"(xrow + (size_t)sh * Jx * 128)
                          : "memory");
         }
     };
@@ -169,13 +170,18 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_kernel(DevTa
     // next barrier, COEF lanes per row
     u64 *pend = nullptr;
     uint32_t pend_g0 = 0, pend_col0 = 0;
+    u64 pend_q = 0;
     const size_t lN = (size_t)level * c.N;
     auto flush = [&]() {
 #pragma unroll
         for (uint32_t k = 0; k < MG * MS * COEF / THREADS; k++) {
             const uint32_t row = k * (THREADS / COEF) + tid / COEF, sl = tid % COEF, gl = row >> 4, cl = row & 15;
             const uint32_t g = pend_g0 + gl, col = pend_col0 + cl;
-            if (g < G && col < ncol) pend[((size_t)g * ncol + col) * lN + (sl ^ (gl % COEF))] = obuf[row * COEF + sl];
+            if (g < G && col < ncol) {
+                u64 *dst = pend + ((size_t)g * ncol + col) * lN + (sl ^ (gl % COEF));
+                const u64 v = obuf[row * COEF + sl];
+                *dst = accumulate ? add_mod(v, *dst, pend_q) : v;
+            }
         }
         pend = nullptr;
     };
@@ -257,6 +263,7 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_kernel(DevTa
                 }
             pend_g0 = ct.zg * MG;
             pend_col0 = ct.zc * MS;
+            pend_q = q;
             pend = acc + (size_t)ct.i * c.N + ct.xb * COEF;
         }
         if (++ks == nk) { ks = 0; ct.next(coltiles, gtiles, xblocks); }
@@ -299,7 +306,7 @@ template <uint32_t COEF, uint32_t NW>
 __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_async_kernel(DevTables c, const u64 *__restrict__ baby,
                                                                                  const u64 *__restrict__ pts, u64 *__restrict__ acc,
                                                                                  uint32_t J, uint32_t S, uint32_t G, uint32_t level,
-                                                                                 uint32_t ntiles) {
+                                                                                 uint32_t ntiles, uint32_t Jx, uint32_t j0, uint32_t accumulate) {
     using T = Geo<COEF>;
     constexpr uint32_t THREADS = COEF * 64 / NW, CH = T::CH, NWARPS = THREADS / 32;
     constexpr uint32_t AH = THREADS / (CH * MK), NIT = MG / AH, XB64 = 64 / COEF;
@@ -324,7 +331,7 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_async_kernel
     const uint32_t nsteps = (t_end - t_begin) * nk;
 
     const uint32_t ch = tid % CH, jj = (tid / CH) % MK, arow = tid / (CH * MK);
-    const uint32_t Rw = G * J, Rx = 2 * S * J;
+    const uint32_t Rw = G * J, Rx = 2 * S * Jx;          // the baby buffer has Jx rows per shard and component; this launch uses rows j0 .. j0 + J - 1
     const uint32_t sm_thread = (uint32_t)__cvta_generic_to_shared(ring) + T::tile_off(arow, jj, ch);
     TileIt lt;
     lt.init(t_begin, coltiles, gtiles, xblocks);
@@ -338,7 +345,7 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_async_kernel
             const size_t blk = (size_t)lt.i * (c.N >> 6) + lt.xb / XB64;
             const uint32_t in_blk = (lt.xb % XB64) * COEF + 2 * ch, j = lks * MK + jj;
             wrow = pts + blk * Rw * 64 + in_blk + (size_t)j * 64;
-            xrow = baby + blk * Rx * 64 + in_blk + (size_t)(2 * j + (arow & 1)) * 64;
+            xrow = baby + blk * Rx * 64 + in_blk + (size_t)(2 * (j0 + j) + (arow & 1)) * 64;
             lg0 = lt.zg * MG + arow;
             lsh0 = lt.zc * (MS / 2) + (arow >> 1);
             lsm = sm_thread + lslot * T::STAGE_BYTES;
@@ -354,7 +361,7 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_async_kernel
     auto load_x = [&](uint32_t k) {
         if (lstep < nsteps) {
             const uint32_t sh = min(lsh0 + (AH / 2) * k, S - 1);
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(lsm + T::BOX_BYTES + k * AH * T::GPITCH), "l"(xrow + (size_t)sh * J * 128)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(lsm + T::BOX_BYTES + k * AH * T::GPITCH), "l"(xrow + (size_t)sh * Jx * 128)
                          : "memory");
         }
     };
@@ -379,6 +386,7 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_async_kernel
     int dsum[NW][13][4];
     u64 *pend = nullptr;
     uint32_t pend_g0 = 0, pend_col0 = 0, pend_tile = 0;
+    u64 pend_q = 0;
     const size_t lN = (size_t)level * c.N;
     auto flush = [&]() {
         if (!mbar_wait(bar_ofull, pend_tile & 1)) alive = false;
@@ -386,7 +394,11 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_async_kernel
         for (uint32_t k = 0; k < MG * MS * COEF / THREADS; k++) {
             const uint32_t row = k * (THREADS / COEF) + tid / COEF, sl = tid % COEF, gl = row >> 4, cl = row & 15;
             const uint32_t g = pend_g0 + gl, col = pend_col0 + cl;
-            if (alive && g < G && col < ncol) pend[((size_t)g * ncol + col) * lN + (sl ^ (gl % COEF))] = obuf[row * COEF + sl];
+            if (alive && g < G && col < ncol) {
+                u64 *dst = pend + ((size_t)g * ncol + col) * lN + (sl ^ (gl % COEF));
+                const u64 v = obuf[row * COEF + sl];
+                *dst = accumulate ? add_mod(v, *dst, pend_q) : v;
+            }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_oempty);
@@ -477,6 +489,7 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_async_kernel
             pend_g0 = ct.zg * MG;
             pend_col0 = ct.zc * MS;
             pend_tile = tiles_done++;
+            pend_q = q;
             pend = acc + (size_t)ct.i * c.N + ct.xb * COEF;
         }
         if (++ks == nk) { ks = 0; ct.next(coltiles, gtiles, xblocks); }
@@ -488,7 +501,8 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_async_kernel
 }
 
 template <uint32_t COEF, uint32_t NW, bool ASYNC = false>
-bool launch_as(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level, cudaStream_t s) {
+bool launch_as(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level, cudaStream_t s,
+               uint32_t Jx, uint32_t j0, bool accumulate) {
     auto kernel = ASYNC ? mac_mma_async_kernel<COEF, NW> : mac_mma_kernel<COEF, NW>;
     // per device, so set on every launch (a host-side table update)
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Geo<COEF>::SMEM_BYTES) != cudaSuccess) return false;
@@ -497,7 +511,8 @@ bool launch_as(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uin
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
     const uint32_t ctas = (uint32_t)sms * (8 / COEF);
-    kernel<<<ntiles < ctas ? ntiles : ctas, COEF * 64 / NW, Geo<COEF>::SMEM_BYTES, s>>>(c->dev, baby, pts, acc, J, S, G, level, ntiles);
+    kernel<<<ntiles < ctas ? ntiles : ctas, COEF * 64 / NW, Geo<COEF>::SMEM_BYTES, s>>>(c->dev, baby, pts, acc, J, S, G, level, ntiles, Jx, j0,
+                                                                                       accumulate ? 1u : 0u);
     count_launches();
     return true;
 }
@@ -506,20 +521,23 @@ bool launch_as(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uin
 
 bool mac_mma_supported(const ckks_ctx *c, uint32_t J) { return J % MK == 0 && J > 0 && c->N % 64 == 0; }
 
-// acc[g][s][c][i][p] = sum_{j < J} baby[s][j][c][i][p] * pts[g][j][i][p] with baby and pts in the tiled layout
-// (rows (s J + j) 2 + c and g J + j); acc in the plain layout.  Returns false if nothing was launched.
+// acc[g][s][c][i][p] (+)= sum_{j < J} baby[s][j0 + j][c][i][p] * pts[g][j][i][p] with baby and pts in the tiled layout
+// (baby rows (s Jx + j) 2 + c, pts rows g J + j); acc in the plain layout.  Jx = 0 means Jx = J.  Returns false if
+// nothing was launched.
 bool launch_mac_mma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level,
-                    cudaStream_t s) {
+                    cudaStream_t s, uint32_t Jx, uint32_t j0, bool accumulate) {
     if (!mac_mma_supported(c, J)) return false;
+    if (!Jx) Jx = J;
     // tuning knob: CKKS_MAC_SHAPE = 100 (the tcgen05 / TMEM kernel of mac_umma.cu, J <= 64), 82 (mma.sync, 8 coefficients per
     // CTA, a warp per coefficient: the default), 83 (the same
-    // without CTA-wide barriers: 7 % faster, bounded mbarrier waits), 81 (two warps per coefficient, 10 % slower) or 42 (4 coefficients per CTA, two CTAs per SM: the products overlap better, but operand
+    // without CTA-wide barriers: 7 % faster, bounded mbarrier waits), 81 (two warps per coefficient, 10 % slower) or 42
+    // (4 coefficients per CTA, two CTAs per SM: the products overlap better, but operand
     // rows fetched 32 bytes at a time make the loads twice as slow as the whole kernel otherwise is)
     const char *e = getenv("CKKS_MAC_SHAPE");
     const int shape = e ? atoi(e) : 82;
-    if (shape == 100 && launch_mac_umma(c, baby, pts, acc, J, S, G, level, s)) return true;
-    if (shape == 83) return launch_as<8, 2, true>(c, baby, pts, acc, J, S, G, level, s);
-    if (shape == 42) return launch_as<4, 2>(c, baby, pts, acc, J, S, G, level, s);
-    if (shape == 81) return launch_as<8, 1>(c, baby, pts, acc, J, S, G, level, s);
-    return launch_as<8, 2>(c, baby, pts, acc, J, S, G, level, s);
+    if (shape == 100 && launch_mac_umma(c, baby, pts, acc, J, S, G, level, s, Jx, j0, accumulate)) return true;
+    if (shape == 83) return launch_as<8, 2, true>(c, baby, pts, acc, J, S, G, level, s, Jx, j0, accumulate);
+    if (shape == 42) return launch_as<4, 2>(c, baby, pts, acc, J, S, G, level, s, Jx, j0, accumulate);
+    if (shape == 81) return launch_as<8, 1>(c, baby, pts, acc, J, S, G, level, s, Jx, j0, accumulate);
+    return launch_as<8, 2>(c, baby, pts, acc, J, S, G, level, s, Jx, j0, accumulate);
 }

@@ -146,7 +146,7 @@ struct BlockIt {           // blocks of a CTA: giant tile fastest, then coeffici
 
 __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, const u64 *__restrict__ baby, const u64 *__restrict__ pts,
                                                                 u64 *__restrict__ acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level,
-                                                                uint32_t nblocks) {
+                                                                uint32_t nblocks, uint32_t Jx, uint32_t j0, uint32_t accumulate) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sm = reinterpret_cast<uint8_t *>(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
     const uint32_t sm0 = (uint32_t)__cvta_generic_to_shared(sm);
@@ -181,7 +181,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
         // a thread keeps its coefficient p, its j mod 8 and the parity of its giant (column); it walks pairs and j / 8
         const uint32_t lt = tid - W_LOAD * 32, p = lt & 7, jr = (lt >> 3) & 7, par = (lt >> 6) & 1, sub = lt >> 7;
         constexpr uint32_t NSUB = L_WARPS / 4;                                  // thread groups sharing the pairs
-        const uint32_t Rw = G * J, Rx = 2 * S * J, njb = J / 8;
+        const uint32_t Rw = G * J, Rx = 2 * S * Jx, njb = J / 8;      // baby rows j0 .. j0 + J - 1 of Jx per shard and component
         BlockIt it;
         it.init(b_begin, gtiles, xblocks);
         uint32_t cgn = 0;                                                       // column groups issued so far
@@ -199,13 +199,13 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
                     asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(dst), "l"(src) : "memory");
             }
             mbar_arrive_cp_async(bars + 8 * (B_WFULL + (b & 1)));
-            const u64 *xsrc = baby + blk * Rx * 64 + in_blk + (size_t)jr * 128;
+            const u64 *xsrc = baby + blk * Rx * 64 + in_blk + (size_t)(j0 + jr) * 128;
             for (uint32_t cg = 0; cg < ncg && alive; cg++, cgn++) {
                 if (!wait_empty(bars, B_XEMPTY, cgn, 2)) { alive = false; break; }
                 const uint32_t xdst = sm0 + L.x(cgn & 1) + p * L.tsx + jr * 16 + par * 8;
                 for (uint32_t cp = sub; cp < UCG / 2; cp += NSUB) {
                     const uint32_t col = min(cg * UCG + 2 * cp + par, ncol - 1);
-                    const u64 *src = xsrc + ((size_t)(col >> 1) * J * 2 + (col & 1)) * 64;
+                    const u64 *src = xsrc + ((size_t)(col >> 1) * Jx * 2 + (col & 1)) * 64;
                     uint32_t dst = xdst + cp * sbo;
                     for (uint32_t jb = 0; jb < njb; jb++, src += 16 * 64, dst += 128)
                         asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(dst), "l"(src) : "memory");
@@ -251,7 +251,11 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
                 for (uint32_t k = 0; k < UG * UCG * UC / 32; k++) {
                     const uint32_t row = k * 4 + (lane >> 3), w = lane & 7, gl = row >> 3, cl = row & 7;
                     const uint32_t g = it.zg * UG + gl, col = cg * UCG + cl;
-                    if (g < G && col < ncol) obase[((size_t)g * ncol + col) * lN + (w ^ (gl & 7))] = ob[row * UC + w];
+                    if (g < G && col < ncol) {
+                        u64 *dst = obase + ((size_t)g * ncol + col) * lN + (w ^ (gl & 7));
+                        const u64 v = ob[row * UC + w];
+                        *dst = accumulate ? add_mod(v, *dst, c.mod[it.i]) : v;
+                    }
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bars + 8 * (B_OEMPTY + (cgn & 1)));
@@ -361,15 +365,17 @@ bool mac_umma_supported(const ckks_ctx *c, uint32_t J) { return J % UK == 0 && J
 
 // Same contract as launch_mac_mma.
 bool launch_mac_umma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level,
-                     cudaStream_t s) {
+                     cudaStream_t s, uint32_t Jx, uint32_t j0, bool accumulate) {
     if (!mac_umma_supported(c, J)) return false;
+    if (!Jx) Jx = J;
     const Smem L = smem_plan(J);
     // per device, so set on every launch (a host-side table update)
     if (cudaFuncSetAttribute(mac_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_plan(MAX_J).total) != cudaSuccess) return false;
     const uint32_t gtiles = (G + UG - 1) / UG, nblocks = (c->N / UC) * level * gtiles;
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
-    mac_umma_kernel<<<nblocks < (uint32_t)sms ? nblocks : (uint32_t)sms, U_THREADS, L.total, s>>>(c->dev, baby, pts, acc, J, S, G, level, nblocks);
+    mac_umma_kernel<<<nblocks < (uint32_t)sms ? nblocks : (uint32_t)sms, U_THREADS, L.total, s>>>(c->dev, baby, pts, acc, J, S, G, level, nblocks, Jx, j0,
+                                                                                                  accumulate ? 1u : 0u);
     count_launches();
     return true;
 }

@@ -63,6 +63,8 @@ def test_projection_shapes_small_ring(d_in, d_out, T, S, B):
     (64, 64, 8, 3, 64),      # J = 64, odd shard count (column padding), single giant step
     (128, 64, 8, 1, 32),     # two input blocks: J = 64
     (64, 160, 8, 9, 32),     # remainder output block 32 | 64, folded; more than one column tile
+    (96, 64, 8, 3, 32),      # remainder input block: the second block has one giant step, the first two
+    (224, 64, 8, 2, 32),     # four input blocks (64, 64, 64, 32): four accumulating launches per group
 ])
 def test_projection_tensor_core_mac_path(d_in, d_out, T, S, B):
     _run(10, 4, 2, 2, 4, d_in, d_out, T, S, B, seed=440 + d_in + d_out + S)
