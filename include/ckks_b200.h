@@ -117,9 +117,10 @@ const char *ckks_status_string(int32_t status);
 const char *ckks_last_cuda_error(const ckks_ctx *ctx);
 
 /* Bytes of caller-provided device workspace `op` needs at this level.  `count`
- * is the batch size for CKKS_OP_ENCODE and the number of rotations for
- * CKKS_OP_ROTATE_HOISTED; ignored otherwise.  For CKKS_OP_LINEAR_PROJ use
- * ckks_linear_proj_workspace_bytes.  Returns 0 for an unknown op. */
+ * is the batch size for CKKS_OP_ENCODE, the number of rotations for
+ * CKKS_OP_ROTATE_HOISTED and the degree for CKKS_OP_POLY_EVAL_TREE; ignored
+ * otherwise.  For CKKS_OP_LINEAR_PROJ use ckks_linear_proj_workspace_bytes.
+ * Returns 0 for an unknown op. */
 size_t ckks_workspace_bytes(const ckks_ctx *ctx, int32_t op, uint32_t level, uint32_t count);
 
 /* Number of kernels this library has launched since it was loaded (all contexts).  Not thread safe. */
