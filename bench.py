@@ -302,6 +302,10 @@ def run_cuda(args):
         pa, pb = [cta, ctb] * 64, [ctb, cta] * 64
         extras["sum_of_128_products_one_relin_ms"] = once(lambda: ctx.mul_relin_sum(pa, pb, rlk, out=mul_out))
         extras["mul_relin_128_calls_ms"] = once(lambda: [ctx.mul_relin(x_, y_, rlk, out=mul_out) for x_, y_ in zip(pa, pb)])
+        bouts = [ctx.empty_ct(LEVEL) for _ in range(16)] * 8
+        bws = ctx.workspace(ctx.workspace_bytes(binding.OP_MUL_RELIN_BATCH, LEVEL, 128))
+        extras["mul_relin_batch_128_ms"] = once(lambda: ctx.mul_relin_batch(pa, pb, rlk, outs=bouts, ws=bws))
+        del bouts, bws
         del Wk, Wv
 
     # e2e: host buffers in, host buffers out, copies inside the timed region

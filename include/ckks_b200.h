@@ -67,7 +67,7 @@ enum {
 enum {
     CKKS_OP_ENCODE = 1, CKKS_OP_MUL_RELIN = 2, CKKS_OP_ROTATE = 3,
     CKKS_OP_ROTATE_HOISTED = 4, CKKS_OP_RESCALE = 5, CKKS_OP_LINEAR_PROJ = 6, CKKS_OP_POLY_EVAL = 7,
-    CKKS_OP_POLY_EVAL_TREE = 8 /* count = degree */
+    CKKS_OP_POLY_EVAL_TREE = 8 /* count = degree */, CKKS_OP_MUL_RELIN_BATCH = 9 /* count = products */
 };
 
 typedef struct ckks_ctx ckks_ctx; /* opaque */
@@ -118,7 +118,8 @@ const char *ckks_last_cuda_error(const ckks_ctx *ctx);
 
 /* Bytes of caller-provided device workspace `op` needs at this level.  `count`
  * is the batch size for CKKS_OP_ENCODE, the number of rotations for
- * CKKS_OP_ROTATE_HOISTED and the degree for CKKS_OP_POLY_EVAL_TREE; ignored
+ * CKKS_OP_ROTATE_HOISTED, the degree for CKKS_OP_POLY_EVAL_TREE and the number
+ * of products for CKKS_OP_MUL_RELIN_BATCH; ignored
  * otherwise.  For CKKS_OP_LINEAR_PROJ use ckks_linear_proj_workspace_bytes.
  * Returns 0 for an unknown op. */
 size_t ckks_workspace_bytes(const ckks_ctx *ctx, int32_t op, uint32_t level, uint32_t count);
@@ -186,6 +187,13 @@ int32_t ckks_add(ckks_ctx *ctx, const ckks_ct *a, const ckks_ct *b, ckks_ct *out
  * out may alias a or b.  Errors: ARG, LEVEL, NO_KEY, WORKSPACE. */
 int32_t ckks_mul_relin(ckks_ctx *ctx, const ckks_ct *a, const ckks_ct *b, const ckks_evk *rlk, ckks_ct *out,
                        void *ws, size_t ws_bytes, void *stream);
+
+/* n independent products out[i] = Mult+relin(a[i], b[i]) in one call: the key switches of up to 16 products run side by
+ * side (one batched ModUp, inner product and ModDown), which fills the GPU where a single ciphertext does not.
+ * Every out[i] is bit-identical to ckks_mul_relin(a[i], b[i]).  a, b, out: host arrays of n ciphertexts at one
+ * level; out[i] may be a[i] or b[i].  Workspace: ckks_workspace_bytes(CKKS_OP_MUL_RELIN_BATCH, level, n). */
+int32_t ckks_mul_relin_batch(ckks_ctx *ctx, const ckks_ct *a, const ckks_ct *b, uint32_t n, const ckks_evk *rlk, ckks_ct *out,
+                             void *ws, size_t ws_bytes, void *stream);
 
 /* Sum of n products with one relinearisation (Section 4: the attention products add up many ciphertext x
  * ciphertext terms): e = sum_i a_i (x) b_i component-wise modulo each prime, then as ckks_mul_relin from the

@@ -31,6 +31,7 @@ size_t hoisted_bytes(const ckks_ctx *c, uint32_t level, uint32_t nbh) {
     const size_t beta = (level + c->alpha - 1) / c->alpha, nt = level + c->K;
     return (level + beta * nt + (size_t)nbh * (2 * nt + 2 * level)) * c->N * sizeof(u64);
 }
+constexpr uint32_t MRB_CHUNK = 16;      // products key-switched side by side by ckks_mul_relin_batch
 size_t rescale_bytes(const ckks_ctx *c, uint32_t level, uint32_t ncomp) { return (size_t)ncomp * level * c->N * sizeof(u64); }
 
 // ---- projection plan -------------------------------------------------------
@@ -230,6 +231,9 @@ extern "C" size_t ckks_workspace_bytes(const ckks_ctx *c, int32_t op, uint32_t l
         case CKKS_OP_ROTATE: return ks_bytes(c, level);
         case CKKS_OP_ROTATE_HOISTED: return hoisted_bytes(c, level, std::min<uint32_t>(count ? count : 1, KS_MULTI));
         case CKKS_OP_RESCALE: return rescale_bytes(c, level, 2);
+        // per product of a chunk (at most MRB_CHUNK): the staged result, e_2 and a key-switch workspace
+        case CKKS_OP_MUL_RELIN_BATCH:
+            return (size_t)std::min<uint32_t>(count ? count : 1, MRB_CHUNK) * ((size_t)3 * level * limb + ks_bytes(c, level));
         // two running ciphertexts, the truncated copy of x, then the Mult and rescale scratch
         case CKKS_OP_POLY_EVAL: return 3 * (size_t)2 * level * limb + ks_bytes(c, level) + (size_t)level * limb + rescale_bytes(c, level, 2);
         // the powers x^2..x^degree, two truncated operands, the product, the accumulator and a term, then the scratch
@@ -365,6 +369,38 @@ static int rotate_checks(const ckks_ctx *c, const ckks_ct *in, const ckks_evk *k
     }
     if (!ws || ws_bytes < ks_bytes(c, in->level)) return CKKS_ERR_WORKSPACE;
     return CKKS_OK;
+}
+
+extern "C" int32_t ckks_mul_relin_batch(ckks_ctx *c, const ckks_ct *a, const ckks_ct *b, uint32_t n, const ckks_evk *rlk, ckks_ct *out,
+                                        void *ws, size_t ws_bytes, void *stream) {
+    if (!c || !a || !b || !out || !n) return CKKS_ERR_ARG;
+    for (uint32_t i = 0; i < n; i++)
+        if (!ct_ok(&a[i]) || !ct_ok(&b[i]) || !ct_ok(&out[i]) || a[i].ncomp != 2 || b[i].ncomp != 2) return CKKS_ERR_ARG;
+    const uint32_t level = a[0].level;
+    if (!level_ok(c, level)) return CKKS_ERR_LEVEL;
+    for (uint32_t i = 0; i < n; i++)
+        if (a[i].level != level || b[i].level != level) return CKKS_ERR_LEVEL;
+    if (!rlk || !rlk->data || rlk->galois != 0) return CKKS_ERR_NO_KEY;
+    if (!ws || ws_bytes < ckks_workspace_bytes(c, CKKS_OP_MUL_RELIN_BATCH, level, n)) return CKKS_ERR_WORKSPACE;
+    DeviceGuard g(c->device);
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t N = c->N, ctl = (size_t)2 * level * N, ptl = (size_t)level * N;
+    for (uint32_t i0 = 0; i0 < n; i0 += MRB_CHUNK) {
+        const uint32_t m = std::min(MRB_CHUNK, n - i0);
+        u64 *stage = (u64 *)ws, *e2 = stage + (size_t)m * ctl;
+        KsWorkspace w = ks_carve(c, level, e2 + (size_t)m * ptl, m);
+        for (uint32_t i = 0; i < m; i++)
+            launch_tensor(c, (const u64 *)a[i0 + i].data, (const u64 *)b[i0 + i].data, stage + (size_t)i * ctl, e2 + (size_t)i * ptl, level, s);
+        // the m key switches run side by side: one ModUp, one inner product, one ModDown over the whole chunk
+        ks_modup(c, e2, level, w, s, m, ptl);
+        ks_inner_moddown(c, (const u64 *)rlk->data, level, 1, w, stage, stage + ptl, 1, stage, s, m, ctl, ctl, false);
+        for (uint32_t i = 0; i < m; i++)
+            cudaMemcpyAsync(out[i0 + i].data, stage + (size_t)i * ctl, ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+    }
+    int rc = finish(c);
+    if (rc == CKKS_OK)
+        for (uint32_t i = 0; i < n; i++) { out[i].level = level; out[i].ncomp = 2; out[i].scale = a[i].scale * b[i].scale; }
+    return rc;
 }
 
 extern "C" int32_t ckks_mul_relin_sum(ckks_ctx *c, const ckks_ct *a, const ckks_ct *b, uint32_t n, const ckks_evk *rlk, ckks_ct *out,

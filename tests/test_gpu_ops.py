@@ -225,6 +225,28 @@ def test_poly_eval_tree_bit_exact(log_n, L, K, dnum, level, coeffs):
     assert e.value.code == binding.ERR_ARG
 
 
+@pytest.mark.parametrize("log_n,L,K,dnum,level,n", [(10, 6, 2, 3, 6, 3), (11, 4, 2, 2, 3, 19), (16, 24, 8, 3, 24, 4)])
+def test_mul_relin_batch_bit_exact(log_n, L, K, dnum, level, n):
+    """n independent products with batched key switches (n = 19 spans two chunks): each equals mul_relin."""
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    P, ctx = params(log_n, L, K, dnum), context(log_n, L, K, dnum)
+    o = P.oracle
+    cl = Client(P, 290 + n)
+    rlk = cl.relin_key()
+    drlk = key_dev(rlk, 0)
+    g = inputs.rng(291, n)
+    ca = [cl.encrypt_slots(g.uniform(-1, 1, P.n), 2.0 ** 40, level) for _ in range(n)]
+    cb = [cl.encrypt_slots(g.uniform(-1, 1, P.n), 2.0 ** 38, level) for _ in range(n)]
+    outs = ctx.mul_relin_batch([ct_dev(c, 2.0 ** 40) for c in ca], [ct_dev(c, 2.0 ** 38) for c in cb], drlk)
+    assert len(outs) == n
+    for i in (range(n) if log_n < 16 else (0, n - 1)):
+        assert outs[i].scale == 2.0 ** 78 and outs[i].level == level
+        assert np.array_equal(host(outs[i].data), o.mul_relin(ca[i], cb[i], rlk)), i
+    with pytest.raises(binding.CkksError) as e:
+        ctx.mul_relin_batch([ct_dev(ca[0], 1.0)], [ct_dev(cb[0], 1.0)], binding.SwitchKey(drlk.data, 3))
+    assert e.value.code == binding.ERR_NO_KEY
+
+
 def test_repeatability():
     """Same call twice gives the same bytes (a race would show up as a difference)."""
     from tests.gpu_util import context, ct_dev, host, key_dev
