@@ -306,6 +306,11 @@ def run_cuda(args):
         bws = ctx.workspace(ctx.workspace_bytes(binding.OP_MUL_RELIN_BATCH, LEVEL, 128))
         extras["mul_relin_batch_128_ms"] = once(lambda: ctx.mul_relin_batch(pa, pb, rlk, outs=bouts, ws=bws))
         del bouts, bws
+        rin, routs = [cta, ctb] * 32, [ctx.empty_ct(LEVEL) for _ in range(16)] * 4
+        rws = ctx.workspace(ctx.workspace_bytes(binding.OP_ROTATE_BATCH, LEVEL, 64))
+        extras["rotate_64_calls_ms"] = once(lambda: [ctx.rotate(x_, rot_keys[0], out=rot_out) for x_ in rin])
+        extras["rotate_batch_64_ms"] = once(lambda: ctx.rotate_batch(rin, rot_keys[0], outs=routs, ws=rws))
+        del routs, rws
         del Wk, Wv
 
     # e2e: host buffers in, host buffers out, copies inside the timed region

@@ -67,7 +67,7 @@ enum {
 enum {
     CKKS_OP_ENCODE = 1, CKKS_OP_MUL_RELIN = 2, CKKS_OP_ROTATE = 3,
     CKKS_OP_ROTATE_HOISTED = 4, CKKS_OP_RESCALE = 5, CKKS_OP_LINEAR_PROJ = 6, CKKS_OP_POLY_EVAL = 7,
-    CKKS_OP_POLY_EVAL_TREE = 8 /* count = degree */, CKKS_OP_MUL_RELIN_BATCH = 9 /* count = products */
+    CKKS_OP_POLY_EVAL_TREE = 8 /* count = degree */, CKKS_OP_MUL_RELIN_BATCH = 9 /* count = products */, CKKS_OP_ROTATE_BATCH = 10 /* count = ciphertexts */
 };
 
 typedef struct ckks_ctx ckks_ctx; /* opaque */
@@ -119,7 +119,7 @@ const char *ckks_last_cuda_error(const ckks_ctx *ctx);
 /* Bytes of caller-provided device workspace `op` needs at this level.  `count`
  * is the batch size for CKKS_OP_ENCODE, the number of rotations for
  * CKKS_OP_ROTATE_HOISTED, the degree for CKKS_OP_POLY_EVAL_TREE and the number
- * of products for CKKS_OP_MUL_RELIN_BATCH; ignored
+ * of products / ciphertexts for CKKS_OP_MUL_RELIN_BATCH / CKKS_OP_ROTATE_BATCH; ignored
  * otherwise.  For CKKS_OP_LINEAR_PROJ use ckks_linear_proj_workspace_bytes.
  * Returns 0 for an unknown op. */
 size_t ckks_workspace_bytes(const ckks_ctx *ctx, int32_t op, uint32_t level, uint32_t count);
@@ -241,6 +241,13 @@ int32_t ckks_poly_eval_tree(ckks_ctx *ctx, const ckks_ct *x, const double *coeff
  * even), WORKSPACE. */
 int32_t ckks_rotate(ckks_ctx *ctx, const ckks_ct *in, const ckks_evk *key, ckks_ct *out,
                     void *ws, size_t ws_bytes, void *stream);
+
+/* The same rotation of n ciphertexts (one key) in one call: the key switches of up to 16 ciphertexts run side by
+ * side and the key is read once per chunk.  Every out[i] is bit-identical to ckks_rotate(in[i], key).  in, out: host
+ * arrays of n two-component ciphertexts at one level; out[i] may be in[i].  Workspace:
+ * ckks_workspace_bytes(CKKS_OP_ROTATE_BATCH, level, n). */
+int32_t ckks_rotate_batch(ckks_ctx *ctx, const ckks_ct *in, uint32_t n, const ckks_evk *key, ckks_ct *out, void *ws, size_t ws_bytes,
+                          void *stream);
 
 /* Hoisted: one iNTT + ModUp + NTT of c1 shared by nrot rotations; rotation r
  * permutes the extended digits by sigma_{g_r}, takes the inner product with

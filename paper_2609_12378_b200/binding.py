@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(_HERE, "libckks_b200.so")
 
 OK, ERR_ARG, ERR_LEVEL, ERR_SCALE, ERR_NO_KEY, ERR_WORKSPACE, ERR_RANGE, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT = (
     0, -1, -2, -3, -4, -5, -6, -7, -8, -9)
-OP_ENCODE, OP_MUL_RELIN, OP_ROTATE, OP_ROTATE_HOISTED, OP_RESCALE, OP_LINEAR_PROJ, OP_POLY_EVAL, OP_POLY_EVAL_TREE, OP_MUL_RELIN_BATCH = 1, 2, 3, 4, 5, 6, 7, 8, 9
+OP_ENCODE, OP_MUL_RELIN, OP_ROTATE, OP_ROTATE_HOISTED, OP_RESCALE, OP_LINEAR_PROJ, OP_POLY_EVAL, OP_POLY_EVAL_TREE, OP_MUL_RELIN_BATCH, OP_ROTATE_BATCH = 1, 2, 3, 4, 5, 6, 7, 8, 9, 10
 
 EXPORTS = [
     "ckks_context_create", "ckks_context_destroy", "ckks_status_string", "ckks_last_cuda_error",
@@ -22,7 +22,7 @@ EXPORTS = [
     "ckks_encode_range_flag", "ckks_mul_plain_acc", "ckks_add", "ckks_mul_relin", "ckks_rotate",
     "ckks_rotate_hoisted", "ckks_rescale", "ckks_linear_proj", "ckks_linear_proj_workspace_bytes",
     "ckks_linear_proj_rotations", "ckks_kernel_launches", "ckks_device_status", "ckks_rescale_static",
-    "ckks_ntt_butterfly_probe", "ckks_mul_relin_sum", "ckks_mul_relin_batch", "ckks_mul_const", "ckks_add_const", "ckks_poly_eval", "ckks_poly_eval_tree", "ckks_linear_proj_multi", "ckks_linear_proj_multi_workspace_bytes",
+    "ckks_ntt_butterfly_probe", "ckks_mul_relin_sum", "ckks_mul_relin_batch", "ckks_rotate_batch", "ckks_mul_const", "ckks_add_const", "ckks_poly_eval", "ckks_poly_eval_tree", "ckks_linear_proj_multi", "ckks_linear_proj_multi_workspace_bytes",
 ]
 
 
@@ -76,6 +76,7 @@ def load():
         "ckks_mul_plain_acc": (i32, [vp, C.POINTER(CCt), u32, C.POINTER(CPt), C.POINTER(CCt), i32, vp]),
         "ckks_add": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), C.POINTER(CCt), vp]),
         "ckks_mul_relin": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
+        "ckks_rotate_batch": (i32, [vp, C.POINTER(CCt), u32, C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
         "ckks_mul_relin_batch": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), u32, C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
         "ckks_mul_relin_sum": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), u32, C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
         "ckks_mul_const": (i32, [vp, C.POINTER(CCt), dbl, dbl, C.POINTER(CCt), vp]),
@@ -325,6 +326,20 @@ class Context:
                                                _stream_ptr(stream)))
         out.scale = co.scale
         return out
+
+    def rotate_batch(self, cts, key: SwitchKey, outs=None, ws: torch.Tensor = None, stream=None):
+        """[rotate(ct, key) for ct in cts] with the key switches of up to 16 ciphertexts running side by side."""
+        level = cts[0].level
+        outs = outs or [self.empty_ct(level) for _ in cts]
+        if ws is None:
+            ws = self.workspace(self.workspace_bytes(OP_ROTATE_BATCH, level, len(cts)))
+        ia = (CCt * len(cts))(*[_cct(x) for x in cts])
+        oa = (CCt * len(outs))(*[_cct(x) for x in outs])
+        ck = CEvk(_dev_u64(key.data).data_ptr(), key.galois)
+        self._check(load().ckks_rotate_batch(self._h, ia, len(cts), C.byref(ck), oa, ws.data_ptr(), ws.numel(), _stream_ptr(stream)))
+        for o, c in zip(outs, oa):
+            o.scale = c.scale
+        return outs
 
     def mul_relin_batch(self, a, b, rlk: SwitchKey, outs=None, ws: torch.Tensor = None, stream=None):
         """[mul_relin(a[i], b[i]) for i] with the key switches of up to 16 products running side by side."""

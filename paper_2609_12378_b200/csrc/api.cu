@@ -232,6 +232,9 @@ extern "C" size_t ckks_workspace_bytes(const ckks_ctx *c, int32_t op, uint32_t l
         case CKKS_OP_ROTATE_HOISTED: return hoisted_bytes(c, level, std::min<uint32_t>(count ? count : 1, KS_MULTI));
         case CKKS_OP_RESCALE: return rescale_bytes(c, level, 2);
         // per product of a chunk (at most MRB_CHUNK): the staged result, e_2 and a key-switch workspace
+        // per ciphertext of a chunk: staged input, staged output and a key-switch workspace
+        case CKKS_OP_ROTATE_BATCH:
+            return (size_t)std::min<uint32_t>(count ? count : 1, MRB_CHUNK) * ((size_t)4 * level * limb + ks_bytes(c, level));
         case CKKS_OP_MUL_RELIN_BATCH:
             return (size_t)std::min<uint32_t>(count ? count : 1, MRB_CHUNK) * ((size_t)3 * level * limb + ks_bytes(c, level));
         // two running ciphertexts, the truncated copy of x, then the Mult and rescale scratch
@@ -605,6 +608,37 @@ extern "C" int32_t ckks_rotate(ckks_ctx *c, const ckks_ct *in, const ckks_evk *k
     ks_inner_moddown(c, (const u64 *)key->data, level, key->galois, w, c0, nullptr, key->galois, (u64 *)out->data, s);
     rc = finish(c);
     if (rc == CKKS_OK) { out->level = level; out->ncomp = 2; out->scale = in->scale; }
+    return rc;
+}
+
+extern "C" int32_t ckks_rotate_batch(ckks_ctx *c, const ckks_ct *in, uint32_t n, const ckks_evk *key, ckks_ct *out, void *ws,
+                                     size_t ws_bytes, void *stream) {
+    if (!c || !in || !out || !n) return CKKS_ERR_ARG;
+    for (uint32_t i = 0; i < n; i++)
+        if (!ct_ok(&in[i]) || !ct_ok(&out[i]) || in[i].ncomp != 2) return CKKS_ERR_ARG;
+    const uint32_t level = in[0].level;
+    if (!level_ok(c, level)) return CKKS_ERR_LEVEL;
+    for (uint32_t i = 0; i < n; i++)
+        if (in[i].level != level) return CKKS_ERR_LEVEL;
+    if (!key || !key->data || key->galois == 0) return CKKS_ERR_NO_KEY;
+    if (!ws || ws_bytes < ckks_workspace_bytes(c, CKKS_OP_ROTATE_BATCH, level, n)) return CKKS_ERR_WORKSPACE;
+    DeviceGuard g(c->device);
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t N = c->N, ctl = (size_t)2 * level * N, ptl = (size_t)level * N;
+    for (uint32_t i0 = 0; i0 < n; i0 += MRB_CHUNK) {
+        const uint32_t m = std::min(MRB_CHUNK, n - i0);
+        u64 *xin = (u64 *)ws, *xout = xin + (size_t)m * ctl;
+        KsWorkspace w = ks_carve(c, level, xout + (size_t)m * ctl, m);
+        for (uint32_t i = 0; i < m; i++)
+            cudaMemcpyAsync(xin + (size_t)i * ctl, in[i0 + i].data, ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+        ks_modup(c, xin + ptl, level, w, s, m, ctl);
+        ks_inner_moddown(c, (const u64 *)key->data, level, key->galois, w, xin, nullptr, key->galois, xout, s, m, ctl, ctl, false);
+        for (uint32_t i = 0; i < m; i++)
+            cudaMemcpyAsync(out[i0 + i].data, xout + (size_t)i * ctl, ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+    }
+    int rc = finish(c);
+    if (rc == CKKS_OK)
+        for (uint32_t i = 0; i < n; i++) { out[i].level = level; out[i].ncomp = 2; out[i].scale = in[i].scale; }
     return rc;
 }
 

@@ -247,6 +247,27 @@ def test_mul_relin_batch_bit_exact(log_n, L, K, dnum, level, n):
     assert e.value.code == binding.ERR_NO_KEY
 
 
+@pytest.mark.parametrize("log_n,L,K,dnum,level,n", [(10, 6, 2, 3, 5, 3), (11, 4, 2, 2, 4, 18), (16, 24, 8, 3, 24, 3)])
+def test_rotate_batch_bit_exact(log_n, L, K, dnum, level, n):
+    """One key, n ciphertexts, key switches side by side (n = 18 spans two chunks): each equals the plain rotation."""
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    P, ctx = params(log_n, L, K, dnum), context(log_n, L, K, dnum)
+    o = P.oracle
+    cl = Client(P, 300 + n)
+    gal = o.galois_element(5)
+    key = cl.rotation_key(gal)
+    dkey = key_dev(key, gal)
+    g = inputs.rng(301, n)
+    cts = [cl.encrypt_slots(g.uniform(-1, 1, P.n), 2.0 ** 40, level) for _ in range(n)]
+    outs = ctx.rotate_batch([ct_dev(c, 2.0 ** 40) for c in cts], dkey)
+    for i in (range(n) if log_n < 16 else (0, n - 1)):
+        assert outs[i].scale == 2.0 ** 40 and outs[i].level == level
+        assert np.array_equal(host(outs[i].data), o.rotate(cts[i], key, gal)), i
+    with pytest.raises(binding.CkksError) as e:
+        ctx.rotate_batch([ct_dev(cts[0], 1.0)], binding.SwitchKey(dkey.data, 0))
+    assert e.value.code == binding.ERR_NO_KEY
+
+
 def test_repeatability():
     """Same call twice gives the same bytes (a race would show up as a difference)."""
     from tests.gpu_util import context, ct_dev, host, key_dev
