@@ -656,15 +656,14 @@ void orc_modup_all(const orc_ctx *c, const uint64_t *d, uint32_t level, uint64_t
 }
 
 /*
- * Evaluation-key inner product and ModDown: ext [beta][level+K][N] evaluation
- * domain, evk [dnum][2][L+K][N].  u_c[t] = sum_j ext_j[t] * evk_{j,c}[t] over
- * the active limbs (key limbs of dropped q's are skipped), then ModDown each
- * component.  k is [2][level][N].
+ * Evaluation-key inner product in the extended basis: ext [beta][level+K][N]
+ * evaluation domain, evk [dnum][2][L+K][N].  u_c[t] = sum_j ext_j[t] * evk_{j,c}[t]
+ * over the active limbs (key limbs of dropped q's are skipped).  u is
+ * [2][level+K][N].
  */
-void orc_inner_moddown(const orc_ctx *c, const uint64_t *ext, const uint64_t *evk, uint32_t level, uint64_t *k) {
+void orc_inner_product(const orc_ctx *c, const uint64_t *ext, const uint64_t *evk, uint32_t level, uint64_t *u) {
     uint64_t N = c->N;
     uint32_t beta = num_digits(c, level), nt = level + c->K, T = c->L + c->K;
-    uint64_t *u = (uint64_t *)malloc(2ull * nt * N * 8);
     #pragma omp parallel for
     for (uint32_t x = 0; x < 2 * nt; x++) {
         uint32_t comp = x / nt, lx = x % nt;
@@ -678,6 +677,14 @@ void orc_inner_moddown(const orc_ctx *c, const uint64_t *ext, const uint64_t *ev
             u[(uint64_t)x * N + p] = acc;
         }
     }
+}
+
+/* The inner product followed by the ModDown of each component.  k is [2][level][N]. */
+void orc_inner_moddown(const orc_ctx *c, const uint64_t *ext, const uint64_t *evk, uint32_t level, uint64_t *k) {
+    uint64_t N = c->N;
+    uint32_t nt = level + c->K;
+    uint64_t *u = (uint64_t *)malloc(2ull * nt * N * 8);
+    orc_inner_product(c, ext, evk, level, u);
     orc_moddown(c, u, level, k);
     orc_moddown(c, u + (uint64_t)nt * N, level, k + (uint64_t)level * N);
     free(u);
@@ -709,6 +716,43 @@ void orc_rotate(const orc_ctx *c, const uint64_t *ct, const uint64_t *evk, uint6
         }
     }
     free(perm); free(k);
+}
+
+/*
+ * A sum of rotated ciphertexts with one ModDown ("lazy" ModDown: the sum is
+ * formed in the extended basis, where the key-switched terms live before
+ * they are divided by P):
+ *   U = sum_i <ModUp(sigma_{g_i} c1_i), evk_i>   over the limbs of Q_level P,
+ *   out = (sum_i sigma_{g_i} c0_i + ModDown(U_0), ModDown(U_1)).
+ * It decrypts to the same sum as adding up orc_rotate's results, with one
+ * division rounding instead of n.  cts is [n][2][level][N], evks[i] points at
+ * the key of Galois element gs[i].
+ */
+void orc_rotate_sum(const orc_ctx *c, const uint64_t *cts, const uint64_t *const *evks, const uint64_t *gs, uint32_t n,
+                    uint32_t level, uint64_t *out) {
+    uint64_t N = c->N;
+    uint32_t beta = num_digits(c, level), nt = level + c->K;
+    uint64_t *perm = (uint64_t *)malloc(2ull * level * N * 8), *ext = (uint64_t *)malloc((uint64_t)beta * nt * N * 8);
+    uint64_t *u = (uint64_t *)malloc(2ull * nt * N * 8), *U = (uint64_t *)calloc(2ull * nt * N, 8);
+    uint64_t *z = (uint64_t *)calloc((uint64_t)level * N, 8);
+    for (uint32_t r = 0; r < n; r++) {
+        const uint64_t *ct = cts + (uint64_t)r * 2 * level * N;
+        for (uint32_t x = 0; x < 2 * level; x++) orc_automorphism_eval(c, ct + (uint64_t)x * N, gs[r], perm + (uint64_t)x * N);
+        orc_modup_all(c, perm + (uint64_t)level * N, level, ext);
+        orc_inner_product(c, ext, evks[r], level, u);
+        for (uint32_t x = 0; x < 2 * nt; x++) {
+            uint32_t lx = x % nt;
+            uint64_t m = c->mod[lx < level ? lx : c->L + (lx - level)];
+            for (uint64_t p = 0; p < N; p++) U[(uint64_t)x * N + p] = addmod(U[(uint64_t)x * N + p], u[(uint64_t)x * N + p], m);
+        }
+        for (uint32_t i = 0; i < level; i++)
+            for (uint64_t p = 0; p < N; p++) z[(uint64_t)i * N + p] = addmod(z[(uint64_t)i * N + p], perm[(uint64_t)i * N + p], c->mod[i]);
+    }
+    orc_moddown(c, U, level, out);
+    orc_moddown(c, U + (uint64_t)nt * N, level, out + (uint64_t)level * N);
+    for (uint32_t i = 0; i < level; i++)
+        for (uint64_t p = 0; p < N; p++) out[(uint64_t)i * N + p] = addmod(out[(uint64_t)i * N + p], z[(uint64_t)i * N + p], c->mod[i]);
+    free(perm); free(ext); free(u); free(U); free(z);
 }
 
 /*

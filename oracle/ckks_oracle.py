@@ -59,6 +59,7 @@ class ProjDesc:
     nshards: int
     baby: int
     pt_scale: float = 0.0      # 0 => q_{level-1}
+    lazy_moddown: bool = False  # giant-step results summed in the extended basis, one ModDown per output
 
 
 class Oracle:
@@ -325,6 +326,30 @@ class Oracle:
         lib().orc_rotate_hoisted(self._h, _p(ct, _u64p), ptrs, _p(ga, _u64p), C.c_uint32(nrot), C.c_uint32(level), _p(outs, _u64p))
         return outs
 
+    def modup_all(self, d):
+        """d [level][N] evaluation domain -> all digits extended and transformed, [beta][level+K][N]."""
+        d = _u64(d); level = d.shape[0]
+        ext = np.empty((self.num_digits(level), level + self.K, self.N), dtype=np.uint64)
+        lib().orc_modup_all(self._h, _p(d, _u64p), C.c_uint32(level), _p(ext, _u64p))
+        return ext
+
+    def inner_product(self, ext, evk):
+        """<ext, evk> in the extended basis: [2][level+K][N], before any ModDown."""
+        ext = _u64(ext); evk = _u64(evk); level = ext.shape[1] - self.K
+        u = np.empty((2, level + self.K, self.N), dtype=np.uint64)
+        lib().orc_inner_product(self._h, _p(ext, _u64p), _p(evk, _u64p), C.c_uint32(level), _p(u, _u64p))
+        return u
+
+    def rotate_sum(self, cts, evks, gs):
+        """sum_i rotate(cts[i], evks[i], gs[i]) with the sum taken in the extended basis and one ModDown."""
+        cts = _u64(cts); n, level = cts.shape[0], cts.shape[2]
+        evks = [_u64(k) for k in evks]
+        ptrs = (C.c_void_p * n)(*[k.ctypes.data for k in evks])
+        ga = np.array(gs, dtype=np.uint64)
+        out = np.empty((2, level, self.N), dtype=np.uint64)
+        lib().orc_rotate_sum(self._h, _p(cts, _u64p), ptrs, _p(ga, _u64p), C.c_uint32(n), C.c_uint32(level), _p(out, _u64p))
+        return out
+
     def rescale(self, ct):
         ct = _u64(ct); ncomp, level = ct.shape[0], ct.shape[1]
         out = np.empty((ncomp, level - 1, self.N), dtype=np.uint64)
@@ -392,7 +417,9 @@ class Oracle:
         """Y = X W on token-shard ciphertexts by the diagonal method (Eq. 5), schedule:
         baby rotations hoisted per input ciphertext; for every giant step g the
         pre-rotated diagonals are encoded and multiply-accumulated; acc_g is rotated by
-        g*B*T_s (plain rotation) and summed; optional fold; one rescale.
+        g*B*T_s (plain rotation) and summed; optional fold; one rescale.  With
+        desc.lazy_moddown the rotated accumulators of g >= 1 are summed by rotate_sum
+        (one ModDown for all of them) and added to acc_0.
 
         cts [nshards * n_in_blocks][2][level][N]; W [d_in][d_out] fp64; keys maps a
         Galois element to its switching key.  Returns (outs [nshards*n_out_blocks][2]
@@ -430,7 +457,7 @@ class Oracle:
                 folds = {mi // mo if mi > mo else 1 for (_, mi) in ins}
                 if len(folds) != 1:
                     raise ValueError("input blocks of one output block need the same fold count")
-                total = None
+                total, later = None, []
                 for g in range(max(nds) // B):
                     acc = None
                     for ib in range(nib):
@@ -438,10 +465,16 @@ class Oracle:
                             continue
                         for b in range(B):
                             acc = self.mul_plain_acc(baby[ib][b], plaintext(ob, ib, g, b), acc)
+                    if g and desc.lazy_moddown:
+                        later.append(acc)
+                        continue
                     if g:
                         ge = gal(g * B * T)
                         acc = self.rotate(acc, keys[ge], ge)
                     total = acc if total is None else self.add(total, acc)
+                if later:
+                    ges = [gal(g * B * T) for g in range(1, len(later) + 1)]
+                    total = self.add(total, self.rotate_sum(np.stack(later), [keys[ge] for ge in ges], ges))
                 f, fold = mo, folds.pop()
                 while fold > 1:
                     ge = gal(f * T)

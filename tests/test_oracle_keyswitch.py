@@ -180,6 +180,65 @@ def test_hoisted_equals_plain_rotation_bit_for_bit():
         assert np.array_equal(o.rotate(ct, key, gal), o.rotate_hoisted(ct, [key], [gal])[0])
 
 
+def test_rotate_sum_pins():
+    """A sum of rotations with one ModDown: n = 1 is rotate bit for bit; the extended-basis inner product is the
+    big-integer sum of digit x key products; the result is ModDown of the summed inner products plus the permuted
+    c0's (re-composed here from the separately pinned pieces); every coefficient differs from the sum of separate
+    rotations by at most (n + 1) K / 2 (one conversion error instead of n); it decrypts to the sum of rotated slots."""
+    log_n, L, K, dnum, level, n = 6, 6, 2, 3, 5, 4
+    P = params(log_n, L, K, dnum)
+    o = P.oracle
+    cl = Client(P, 58)
+    g = inputs.rng(58)
+    scale = 2.0 ** 40
+    zs = g.uniform(-1, 1, (n, P.n))
+    rots = [1, 4, 9, P.n - 2]
+    gals = [o.galois_element(r) for r in rots]
+    keys = [cl.rotation_key(x) for x in gals]
+    cts = np.stack([cl.encrypt_slots(z, scale, level) for z in zs])
+    assert np.array_equal(o.rotate_sum(cts[:1], keys[:1], gals[:1]), o.rotate(cts[0], keys[0], gals[0]))
+    out = o.rotate_sum(cts, keys, gals)
+    primes = [int(x) for x in P.q[:level]] + [int(x) for x in P.p]
+    kidx = list(range(level)) + [L + a for a in range(K)]
+    U = np.zeros((2, level + K, P.N), dtype=object)
+    z0 = np.zeros((level, P.N), dtype=object)
+    for i in range(n):
+        perm = np.stack([[o.automorphism_eval(cts[i][c][t], gals[i]) for t in range(level)] for c in range(2)])
+        ext = o.modup_all(perm[1])
+        u = o.inner_product(ext, keys[i])
+        for c in range(2):
+            for x, (m, kt) in enumerate(zip(primes, kidx)):
+                want = sum(ext[j, x].astype(object) * keys[i][j, c, kt].astype(object) for j in range(ext.shape[0])) % m
+                assert np.array_equal(u[c, x].astype(object), want)
+                U[c, x] = (U[c, x] + want) % m
+        z0 = z0 + perm[0].astype(object)
+    q = np.array(primes[:level], dtype=object)[:, None]
+    want0 = (o.moddown(U[0].astype(np.uint64), level).astype(object) + z0) % q
+    assert np.array_equal(out[0].astype(object), want0)
+    assert np.array_equal(out[1], o.moddown(U[1].astype(np.uint64), level))
+    # against the sum of separate rotations, coefficient by coefficient
+    sep = sum(o.rotate(cts[i], keys[i], gals[i]).astype(object) for i in range(n)) % q[None]
+    diff = ((out.astype(object) - sep) % q[None]).astype(np.uint64)
+    assert diff.any()
+    for c in range(2):
+        dc = o.intt(diff[c][None])[0]
+        worst = max(abs(centred(*crt(dc[:, k], primes[:level]))) for k in range(P.N))
+        assert worst <= (n + 1) * K / 2
+
+    P = params(11, 6, 2, 3)
+    o = P.oracle
+    cl = Client(P, 59)
+    zs = g.uniform(-1, 1, (3, P.n))
+    rots = [8, 64, P.n - 16]
+    gals = [o.galois_element(r) for r in rots]
+    keys = [cl.rotation_key(x) for x in gals]
+    for level in (6, 4):
+        cts = np.stack([cl.encrypt_slots(z, scale, level) for z in zs])
+        got = cl.decrypt_slots(o.rotate_sum(cts, keys, gals), scale)
+        want = sum(np.roll(z, -r) for z, r in zip(zs, rots))
+        assert np.abs(got - want).max() < 2.0 ** -20
+
+
 @pytest.mark.parametrize("log_n,L,K,dnum,level", [(11, 6, 2, 3, 6), (11, 6, 2, 3, 3)])
 def test_mul_relin_slot_product(log_n, L, K, dnum, level):
     P = params(log_n, L, K, dnum)

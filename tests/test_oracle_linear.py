@@ -147,6 +147,39 @@ def test_encrypted_projection_small_ring(d_in, d_out, T, B):
     assert np.array_equal(Yc2[len(outs):], Yc[len(outs):]) and np.array_equal(Yc2[:len(outs)], Yc[len(outs):])
 
 
+@pytest.mark.parametrize("d_in,d_out,T,B", [(16, 16, 32, 4), (16, 4, 32, 2), (24, 16, 32, 4), (16, 16, 32, 16)])
+def test_lazy_moddown_projection(d_in, d_out, T, B):
+    """Giant steps summed in the extended basis: the same plaintext result (X W) within the same bound; equal to the
+    eager schedule bit for bit when there is no giant step to sum, and otherwise within one unit per residue after the
+    rescale (the two differ by a few units before the division by q_last, which almost always rounds them away)."""
+    P = params(10, 4, 2, 2)
+    o = P.oracle
+    cl = Client(P, 64)
+    level, scale = 4, 2.0 ** 40
+    g = inputs.rng(65, d_in * 100 + d_out)
+    X, W = inputs.activations_uniform(g, T, d_in), inputs.weights_normal(g, d_in, d_out, 0.05)
+    eager, lazy = ProjDesc(d_in, d_out, T, 1, B), ProjDesc(d_in, d_out, T, 1, B, lazy_moddown=True)
+    F, ins, outs = o.proj_blocks(eager)
+    cts = np.stack([cl.encrypt_slots(inputs.pack_feature_major(X[:, s0:s0 + mi], T, o.n)[0], scale, level) for (s0, mi) in ins])
+    keys = {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in o.proj_rotations(eager)}
+    Ye, se = o.linear_proj(eager, cts, W, keys, scale)
+    Yl, sl = o.linear_proj(lazy, cts, W, keys, scale)
+    assert se == sl and Ye.shape == Yl.shape
+    giants = max(min(mi, mo) for (_, mi) in ins for (_, mo) in outs) // B
+    if giants == 1:
+        assert np.array_equal(Ye, Yl)
+    q = np.array(P.q[:level - 1], dtype=np.int64)[None, None, :, None]
+    d = (Yl.astype(np.int64) - Ye.astype(np.int64)) % q
+    assert np.minimum(d, q - d).max() <= 1
+    Y = X @ W
+    for ob, (o0, mo) in enumerate(outs):
+        got = cl.decrypt_slots(Yl[ob], sl).real.reshape(F, T)
+        ref = cl.decrypt_slots(Ye[ob], se).real.reshape(F, T)
+        for r in range(F):
+            assert np.abs(got[r] - Y[:, o0 + r % mo]).max() < 2.0 ** -20
+        assert np.abs(got - ref).max() < 2.0 ** -24
+
+
 def test_toy_config_projection():
     """Config 1: N = 2^13, 6+1 primes, dnum 6, 32 tokens x 64 features, 64x64 weights, B = G = 8."""
     P = params(13, 6, 1, 6)
