@@ -36,7 +36,12 @@ TOKENS, HIDDEN, T_SHARD, SHARDS, BABY = 128, 4096, 8, 16, 64
 NTT_BATCH, NROT = 32, 64
 METRIC = "key-switches/s & NTT limbs/s at N=2^16; s per 128-token Llama-3-8B projection"
 WORKLOAD = ("one pass of the hot path at N=2^16 L=24 K=8 dnum=3: NTT fwd+inv of 32x24 limbs; 64 plain + 64 hoisted "
-            "rotations + 1 mul_relin; 128-token 4096x4096 projection (16 shard ciphertexts, B=G=64)")
+            "rotations + 1 mul_relin; 128-token 4096x4096 projection (16 shard ciphertexts, B=G=64, giant steps ")
+LAZY = True
+
+
+def workload():
+    return WORKLOAD + ("summed before one ModDown per output)" if LAZY else "with one ModDown each)")
 
 
 def peaks():
@@ -82,7 +87,7 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------- CPU checker leg
-def oracle_sample(threads_note=True):
+def oracle_sample(lazy=True):
     """Time the CPU checker on a bounded sample of the projection workload and scale to one projection."""
     import numpy as np
 
@@ -102,16 +107,22 @@ def oracle_sample(threads_note=True):
     t0 = time.perf_counter(); acc = orc.mul_plain_acc(ct, pts[0]); acc = orc.mul_plain_acc(ct, pts[1], acc); t["mac"] = (time.perf_counter() - t0) / 2
     t0 = time.perf_counter(); orc.rotate_hoisted(ct, keys, gals); t["hoisted_2"] = time.perf_counter() - t0
     t0 = time.perf_counter(); orc.rotate(ct, keys[0], gals[0]); t["rotate"] = time.perf_counter() - t0
+    t0 = time.perf_counter(); orc.rotate_sum(np.stack([ct, ct]), keys, gals); t["rotate_sum_2"] = time.perf_counter() - t0
     t0 = time.perf_counter(); orc.rescale(acc); t["rescale"] = time.perf_counter() - t0
     t0 = time.perf_counter(); x = inputs.uniform_residues(g, q, N, 1); orc.intt(orc.ntt(x)); t["ntt_pair_24"] = time.perf_counter() - t0
     G = HIDDEN // BABY
     # a hoisted rotation costs (hoisted_2 - shared ModUp)/2; approximate the shared part by rotate - per-rotation part
     per_h = t["hoisted_2"] / 2
+    # a two-term rotate_sum is two extended-basis terms and one ModDown, a rotation one term and one ModDown
+    term = max(t["rotate_sum_2"] - t["rotate"], 0.0)
+    moddown = max(t["rotate"] - term, 0.0)
+    giant = (G - 1) * term + moddown if lazy else (G - 1) * t["rotate"]
     proj = (HIDDEN * t["encode"] + HIDDEN * SHARDS * t["mac"] + SHARDS * (BABY - 1) * per_h
-            + SHARDS * (G - 1) * t["rotate"] + SHARDS * t["rescale"])
+            + SHARDS * giant + SHARDS * t["rescale"])
     cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
-    sample = ("2 encodes, 2 ct x pt MACs, 2 hoisted + 1 plain rotation, 1 rescale, 24 NTT round trips at full size; "
-              "scaled by the projection's counts (4096 encodes, 65536 MACs, 1008 hoisted, 1008 plain, 16 rescales)")
+    sample = ("2 encodes, 2 ct x pt MACs, 2 hoisted + 1 plain rotation, 1 two-term rotate_sum, 1 rescale, 24 NTT round trips at "
+              "full size; scaled by the projection's counts (4096 encodes, 65536 MACs, 1008 hoisted rotations, "
+              + ("1008 giant-step terms + 16 ModDowns" if lazy else "1008 plain rotations") + ", 16 rescales)")
     return {"proj_s": proj, "ntt_limbs_per_s": 48 / t["ntt_pair_24"], "key_switches_per_s": 1.0 / t["rotate"],
             "parts_s": t, "cores": cores, "sample": sample}
 
@@ -121,14 +132,14 @@ def run_reference(args):
     if rank != 0:
         return
     for _ in range(args.warmup if args.warmup < 2 else 1):
-        oracle_sample()
-    vals = [oracle_sample() for _ in range(max(1, args.steps))]
+        oracle_sample(LAZY)
+    vals = [oracle_sample(LAZY) for _ in range(max(1, args.steps))]
     v = statistics.mean(x["proj_s"] for x in vals)
     last = vals[-1]
     line = {"impl": "reference", "metric": METRIC, "value": v, "unit": "s/projection", "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": v * 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "u64", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "note": "CPU checker timed on a bounded sample, scaled by operation counts"},
+            "config": {"workload": workload(), "note": "CPU checker timed on a bounded sample, scaled by operation counts"},
             "submetrics": {"ntt_limbs_per_s": last["ntt_limbs_per_s"], "key_switches_per_s": last["key_switches_per_s"]},
             "cpu_baseline": {"value": v, "unit": "s/projection", "cores": last["cores"], "kind": "oracle", "sample": last["sample"]},
             "e2e": {"value": v, "unit": "s/projection", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -200,7 +211,7 @@ def run_cuda(args):
     cts = [binding.Ciphertext(residues(allp[:L], 2), 2.0 ** 40) for _ in range(SH)]
     W = (torch.randn((HIDDEN, HIDDEN), generator=gen, device=dev, dtype=torch.float64) * 0.02).contiguous()
     outs = [ctx.empty_ct(LEVEL - 1) for _ in range(SH)]
-    ws = torch.empty(ctx.linear_proj_workspace_bytes(HIDDEN, HIDDEN, T_SHARD, SH, BABY, LEVEL), dtype=torch.uint8, device=dev)
+    ws = torch.empty(ctx.linear_proj_workspace_bytes(HIDDEN, HIDDEN, T_SHARD, SH, BABY, LEVEL, True), dtype=torch.uint8, device=dev)
     # e2e host buffers (pinned)
     h_cts = [c.data.cpu().pin_memory() for c in cts]
     h_W = W.cpu().pin_memory()
@@ -220,7 +231,7 @@ def run_cuda(args):
         ctx.mul_relin(cta, ctb, rlk, out=mul_out)
 
     def part_c():
-        ctx.linear_proj(cts, W, proj_keys, HIDDEN, HIDDEN, T_SHARD, SH, BABY, outs=outs, ws=ws)
+        ctx.linear_proj(cts, W, proj_keys, HIDDEN, HIDDEN, T_SHARD, SH, BABY, outs=outs, ws=ws, lazy_moddown=LAZY)
 
     def step(times=None):
         e = [ev() for _ in range(4)]
@@ -294,6 +305,8 @@ def run_cuda(args):
 
     extras = {}
     if rank == 0 and not args.no_extras:
+        extras["projection_%s_moddown_ms" % ("eager" if LAZY else "lazy")] = once(
+            lambda: ctx.linear_proj(cts, W, proj_keys, HIDDEN, HIDDEN, T_SHARD, SH, BABY, outs=outs, ws=ws, lazy_moddown=not LAZY))
         Wk = (torch.randn((HIDDEN, HIDDEN // 4), generator=gen, device=dev, dtype=torch.float64) * 0.02).contiguous()
         Wv = (torch.randn((HIDDEN, HIDDEN // 4), generator=gen, device=dev, dtype=torch.float64) * 0.02).contiguous()
         douts = [HIDDEN, HIDDEN // 4, HIDDEN // 4]
@@ -368,13 +381,13 @@ def run_cuda(args):
                 "others": {"ntt16 family": "55.0 % of the step (profiles/bench_step_launch_list.md)",
                            "mac_mma_kernel": "15.0 % of the step; legacy tensor path 32 % busy, DRAM 51 %, see profiles/mac_mma_projection_8shards.md",
                            "modup + moddown_conv + inner_product": "27.8 % of the step; FP64 pipe 67 % (conversions), DRAM 72 % (inner product)"}}
-    cpu = oracle_sample()
+    cpu = oracle_sample(LAZY)
     jm = job_metrics(world, a_ms, b_ms, c_ms)
     line = {
         "metric": METRIC, "value": jm["value"], "unit": "s/projection", "n_gpus": world, "steps": args.steps,
         "warmup": nwarm, "ms_per_step": total_ms / args.steps, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "u64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "l2": "inputs larger than L2 (>= 384 MiB per part)", "parallelism": f"replicas x{world}"},
+        "config": {"workload": workload(), "l2": "inputs larger than L2 (>= 384 MiB per part)", "parallelism": f"replicas x{world}"},
         "extras": extras,
         "submetrics": {"ntt_limbs_per_s": jm["ntt_limbs_per_s"], "key_switches_per_s": jm["key_switches_per_s"],
                        "ms": {"ntt_roundtrip": a_ms, "keyswitch_part": b_ms, "projection": c_ms}},
@@ -399,10 +412,14 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--parts", default="abc", help="with --profile: which parts of the step to run (a: NTT, b: key switching, c: projection)")
     ap.add_argument("--shards", type=int, default=SHARDS, help="with --profile: token shards in the projection (default 16)")
+    ap.add_argument("--eager-moddown", action="store_true",
+                    help="one ModDown per giant-step rotation instead of one per output ciphertext")
     ap.add_argument("--no-extras", action="store_true", help="skip the untimed one-off measurements of the composite calls")
     ap.add_argument("--profile", action="store_true",
                     help="for profiler captures: honour --warmup below 3 and skip the e2e and CPU legs (prints no bench line)")
     args = ap.parse_args()
+    global LAZY
+    LAZY = not args.eager_moddown
     if args.impl == "reference":
         run_reference(args)
     else:

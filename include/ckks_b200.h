@@ -67,7 +67,7 @@ enum {
 enum {
     CKKS_OP_ENCODE = 1, CKKS_OP_MUL_RELIN = 2, CKKS_OP_ROTATE = 3,
     CKKS_OP_ROTATE_HOISTED = 4, CKKS_OP_RESCALE = 5, CKKS_OP_LINEAR_PROJ = 6, CKKS_OP_POLY_EVAL = 7,
-    CKKS_OP_POLY_EVAL_TREE = 8 /* count = degree */, CKKS_OP_MUL_RELIN_BATCH = 9 /* count = products */, CKKS_OP_ROTATE_BATCH = 10 /* count = ciphertexts */
+    CKKS_OP_POLY_EVAL_TREE = 8 /* count = degree */, CKKS_OP_MUL_RELIN_BATCH = 9 /* count = products */, CKKS_OP_ROTATE_BATCH = 10 /* count = ciphertexts */, CKKS_OP_ROTATE_SUM = 11 /* count = ciphertexts */
 };
 
 typedef struct ckks_ctx ckks_ctx; /* opaque */
@@ -98,9 +98,14 @@ typedef struct { const uint64_t *data; /* device */ uint64_t galois; /* 0 for a 
  * that count; when m_out < m_in the result is folded by log2(m_in/m_out)
  * rotate-and-add steps.  pt_scale is the scale the weights are encoded at
  * (0 selects q_{level-1}, so that the final rescale restores the input scale).
+ * flags: 0, or CKKS_PROJ_LAZY_MODDOWN: the rotated giant-step accumulators of an output ciphertext are summed in the
+ * key-switching basis Q_level P and divided by P once (ckks_rotate_sum's function) instead of once per rotation.
+ * The two settings are different integer functions with the same plaintext result; after the final rescale their
+ * residues differ by at most one unit.
  */
+#define CKKS_PROJ_LAZY_MODDOWN 1u
 typedef struct {
-    uint32_t d_in, d_out, tokens_per_shard, nshards, baby;
+    uint32_t d_in, d_out, tokens_per_shard, nshards, baby, flags;
     double pt_scale;
 } ckks_proj_desc;
 
@@ -119,7 +124,7 @@ const char *ckks_last_cuda_error(const ckks_ctx *ctx);
 /* Bytes of caller-provided device workspace `op` needs at this level.  `count`
  * is the batch size for CKKS_OP_ENCODE, the number of rotations for
  * CKKS_OP_ROTATE_HOISTED, the degree for CKKS_OP_POLY_EVAL_TREE and the number
- * of products / ciphertexts for CKKS_OP_MUL_RELIN_BATCH / CKKS_OP_ROTATE_BATCH; ignored
+ * of products / ciphertexts for CKKS_OP_MUL_RELIN_BATCH / CKKS_OP_ROTATE_BATCH / CKKS_OP_ROTATE_SUM; ignored
  * otherwise.  For CKKS_OP_LINEAR_PROJ use ckks_linear_proj_workspace_bytes.
  * Returns 0 for an unknown op. */
 size_t ckks_workspace_bytes(const ckks_ctx *ctx, int32_t op, uint32_t level, uint32_t count);
@@ -248,6 +253,15 @@ int32_t ckks_rotate(ckks_ctx *ctx, const ckks_ct *in, const ckks_evk *key, ckks_
  * ckks_workspace_bytes(CKKS_OP_ROTATE_BATCH, level, n). */
 int32_t ckks_rotate_batch(ckks_ctx *ctx, const ckks_ct *in, uint32_t n, const ckks_evk *key, ckks_ct *out, void *ws, size_t ws_bytes,
                           void *stream);
+
+/* out = sum_i rotate(in[i], keys[i]) with the sum taken before the division by P ("lazy" ModDown, Section 2.1's key
+ * switch): U = sum_i <ModUp(c1_i) read through sigma_{g_i}, key_i> over the limbs of Q_level P, then
+ * out = (sum_i sigma_{g_i}(c0_i) + ModDown(U_0), ModDown(U_1)).  One division rounding instead of n, and one ModDown's
+ * worth of transforms; n = 1 is ckks_rotate bit for bit.  in: host array of n two-component ciphertexts at one level
+ * and scale; keys: host array of n rotation keys (keys[i] for in[i]); out may be any in[i].  Workspace:
+ * ckks_workspace_bytes(CKKS_OP_ROTATE_SUM, level, n).  Errors: ARG, LEVEL, SCALE, NO_KEY, WORKSPACE. */
+int32_t ckks_rotate_sum(ckks_ctx *ctx, const ckks_ct *in, const ckks_evk *keys, uint32_t n, ckks_ct *out, void *ws, size_t ws_bytes,
+                        void *stream);
 
 /* Hoisted: one iNTT + ModUp + NTT of c1 shared by nrot rotations; rotation r
  * permutes the extended digits by sigma_{g_r}, takes the inner product with

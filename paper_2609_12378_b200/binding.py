@@ -14,7 +14,8 @@ LIB_PATH = os.path.join(_HERE, "libckks_b200.so")
 
 OK, ERR_ARG, ERR_LEVEL, ERR_SCALE, ERR_NO_KEY, ERR_WORKSPACE, ERR_RANGE, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT = (
     0, -1, -2, -3, -4, -5, -6, -7, -8, -9)
-OP_ENCODE, OP_MUL_RELIN, OP_ROTATE, OP_ROTATE_HOISTED, OP_RESCALE, OP_LINEAR_PROJ, OP_POLY_EVAL, OP_POLY_EVAL_TREE, OP_MUL_RELIN_BATCH, OP_ROTATE_BATCH = 1, 2, 3, 4, 5, 6, 7, 8, 9, 10
+OP_ENCODE, OP_MUL_RELIN, OP_ROTATE, OP_ROTATE_HOISTED, OP_RESCALE, OP_LINEAR_PROJ, OP_POLY_EVAL, OP_POLY_EVAL_TREE, OP_MUL_RELIN_BATCH, OP_ROTATE_BATCH, OP_ROTATE_SUM = 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11
+PROJ_LAZY_MODDOWN = 1
 
 EXPORTS = [
     "ckks_context_create", "ckks_context_destroy", "ckks_status_string", "ckks_last_cuda_error",
@@ -22,7 +23,7 @@ EXPORTS = [
     "ckks_encode_range_flag", "ckks_mul_plain_acc", "ckks_add", "ckks_mul_relin", "ckks_rotate",
     "ckks_rotate_hoisted", "ckks_rescale", "ckks_linear_proj", "ckks_linear_proj_workspace_bytes",
     "ckks_linear_proj_rotations", "ckks_kernel_launches", "ckks_device_status", "ckks_rescale_static",
-    "ckks_ntt_butterfly_probe", "ckks_mul_relin_sum", "ckks_mul_relin_batch", "ckks_rotate_batch", "ckks_mul_const", "ckks_add_const", "ckks_poly_eval", "ckks_poly_eval_tree", "ckks_linear_proj_multi", "ckks_linear_proj_multi_workspace_bytes",
+    "ckks_ntt_butterfly_probe", "ckks_mul_relin_sum", "ckks_mul_relin_batch", "ckks_rotate_batch", "ckks_rotate_sum", "ckks_mul_const", "ckks_add_const", "ckks_poly_eval", "ckks_poly_eval_tree", "ckks_linear_proj_multi", "ckks_linear_proj_multi_workspace_bytes",
 ]
 
 
@@ -45,7 +46,7 @@ class CEvk(C.Structure):
 
 class CProjDesc(C.Structure):
     _fields_ = [("d_in", C.c_uint32), ("d_out", C.c_uint32), ("tokens_per_shard", C.c_uint32),
-                ("nshards", C.c_uint32), ("baby", C.c_uint32), ("pt_scale", C.c_double)]
+                ("nshards", C.c_uint32), ("baby", C.c_uint32), ("flags", C.c_uint32), ("pt_scale", C.c_double)]
 
 
 _lib = None
@@ -76,6 +77,7 @@ def load():
         "ckks_mul_plain_acc": (i32, [vp, C.POINTER(CCt), u32, C.POINTER(CPt), C.POINTER(CCt), i32, vp]),
         "ckks_add": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), C.POINTER(CCt), vp]),
         "ckks_mul_relin": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
+        "ckks_rotate_sum": (i32, [vp, C.POINTER(CCt), C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
         "ckks_rotate_batch": (i32, [vp, C.POINTER(CCt), u32, C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
         "ckks_mul_relin_batch": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), u32, C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
         "ckks_mul_relin_sum": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), u32, C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
@@ -327,6 +329,19 @@ class Context:
         out.scale = co.scale
         return out
 
+    def rotate_sum(self, cts, keys, out: Ciphertext = None, ws: torch.Tensor = None, stream=None):
+        """sum_i rotate(cts[i], keys[i]) formed in the key-switching basis and divided by P once."""
+        level = cts[0].level
+        out = out or self.empty_ct(level)
+        if ws is None:
+            ws = self.workspace(self.workspace_bytes(OP_ROTATE_SUM, level, len(cts)))
+        ia = (CCt * len(cts))(*[_cct(x) for x in cts])
+        ka = (CEvk * len(keys))(*[CEvk(_dev_u64(k.data).data_ptr(), k.galois) for k in keys])
+        co = _cct(out)
+        self._check(load().ckks_rotate_sum(self._h, ia, ka, len(cts), C.byref(co), ws.data_ptr(), ws.numel(), _stream_ptr(stream)))
+        out.scale = co.scale
+        return out
+
     def rotate_batch(self, cts, key: SwitchKey, outs=None, ws: torch.Tensor = None, stream=None):
         """[rotate(ct, key) for ct in cts] with the key switches of up to 16 ciphertexts running side by side."""
         level = cts[0].level
@@ -395,7 +410,7 @@ class Context:
         return outs
 
     def linear_proj_multi(self, cts, Ws, keys, d_in, d_outs, tokens_per_shard, nshards, baby, pt_scale=0.0,
-                          ws: torch.Tensor = None, stream=None):
+                          ws: torch.Tensor = None, stream=None, lazy_moddown=False):
         """[X W_0, X W_1, ...] for weight matrices sharing their input (Q/K/V, gate/up): the baby-step rotations of
         the inputs are computed once.  Returns one list of output ciphertexts per matrix, each bit-identical to a
         separate linear_proj call."""
@@ -403,7 +418,7 @@ class Context:
         for W, d_out in zip(Ws, d_outs):
             if not (W.is_cuda and W.dtype == torch.float64 and W.is_contiguous() and tuple(W.shape) == (d_in, d_out)):
                 raise TypeError("every W must be a contiguous CUDA float64 [d_in][d_out] tensor")
-        da = (CProjDesc * nmat)(*[self._desc(d_in, d_out, tokens_per_shard, nshards, baby, pt_scale) for d_out in d_outs])
+        da = (CProjDesc * nmat)(*[self._desc(d_in, d_out, tokens_per_shard, nshards, baby, pt_scale, lazy_moddown) for d_out in d_outs])
         level = cts[0].level
         F = self.n // tokens_per_shard
         outs = [[self.empty_ct(level - 1) for _ in range(nshards * -(-d_out // F))] for d_out in d_outs]
@@ -430,8 +445,8 @@ class Context:
         return out
 
     # ----------------------------------------------------- linear projection
-    def _desc(self, d_in, d_out, tokens_per_shard, nshards, baby, pt_scale=0.0):
-        return CProjDesc(d_in, d_out, tokens_per_shard, nshards, baby, float(pt_scale))
+    def _desc(self, d_in, d_out, tokens_per_shard, nshards, baby, pt_scale=0.0, lazy_moddown=False):
+        return CProjDesc(d_in, d_out, tokens_per_shard, nshards, baby, PROJ_LAZY_MODDOWN if lazy_moddown else 0, float(pt_scale))
 
     def linear_proj_rotations(self, d_in, d_out, tokens_per_shard, nshards, baby):
         d = self._desc(d_in, d_out, tokens_per_shard, nshards, baby)
@@ -442,24 +457,24 @@ class Context:
         load().ckks_linear_proj_rotations(self._h, C.byref(d), buf, n)
         return list(buf)[:n]
 
-    def linear_proj_workspace_bytes(self, d_in, d_out, tokens_per_shard, nshards, baby, level):
-        d = self._desc(d_in, d_out, tokens_per_shard, nshards, baby)
+    def linear_proj_workspace_bytes(self, d_in, d_out, tokens_per_shard, nshards, baby, level, lazy_moddown=False):
+        d = self._desc(d_in, d_out, tokens_per_shard, nshards, baby, 0.0, lazy_moddown)
         return int(load().ckks_linear_proj_workspace_bytes(self._h, C.byref(d), level))
 
     def linear_proj(self, cts, W: torch.Tensor, keys, d_in, d_out, tokens_per_shard, nshards, baby, pt_scale=0.0,
-                    outs=None, ws: torch.Tensor = None, stream=None):
+                    outs=None, ws: torch.Tensor = None, stream=None, lazy_moddown=False):
         """Y = X W.  cts: nshards * n_in_blocks ciphertexts; W: fp64 [d_in][d_out] on the device;
         keys: rotation SwitchKeys.  Returns nshards * n_out_blocks ciphertexts at level - 1."""
         if not (W.is_cuda and W.dtype == torch.float64 and W.is_contiguous() and tuple(W.shape) == (d_in, d_out)):
             raise TypeError("W must be a contiguous CUDA float64 [d_in][d_out] tensor")
-        d = self._desc(d_in, d_out, tokens_per_shard, nshards, baby, pt_scale)
+        d = self._desc(d_in, d_out, tokens_per_shard, nshards, baby, pt_scale, lazy_moddown)
         level = cts[0].level
         F = self.n // tokens_per_shard
         nob = -(-d_out // F)
         if outs is None:
             outs = [self.empty_ct(level - 1) for _ in range(nshards * nob)]
         if ws is None:
-            ws = self.workspace(self.linear_proj_workspace_bytes(d_in, d_out, tokens_per_shard, nshards, baby, level))
+            ws = self.workspace(self.linear_proj_workspace_bytes(d_in, d_out, tokens_per_shard, nshards, baby, level, lazy_moddown))
         ia = (CCt * len(cts))(*[_cct(c) for c in cts])
         oa = (CCt * len(outs))(*[_cct(o) for o in outs])
         for o in oa:

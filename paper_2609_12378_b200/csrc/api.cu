@@ -79,11 +79,11 @@ int make_plan(const ckks_ctx *c, const ckks_proj_desc *d, ProjPlan &p) {
     return CKKS_OK;
 }
 
-struct ProjWs { size_t baby, xin, pts, ptt, slots, enc, acc, total, tmp, ks, rs, bytes; uint32_t gg; bool per_block; };
+struct ProjWs { size_t baby, xin, pts, ptt, slots, enc, acc, total, tmp, ks, ksx, rs, bytes; uint32_t gg; bool per_block; };
 
 constexpr uint32_t MAC_GT = 4, MAC_ST = 2;   // register tile of the multiply-accumulate kernel: giants x shards
 
-ProjWs proj_layout(const ckks_ctx *c, const ProjPlan &p, uint32_t level) {
+ProjWs proj_layout(const ckks_ctx *c, const ProjPlan &p, uint32_t level, bool lazy) {
     const size_t ct = (size_t)2 * level * c->N * sizeof(u64), pt = (size_t)level * c->N * sizeof(u64);
     const size_t nib = p.ins.size();
     ProjWs w;
@@ -107,6 +107,9 @@ ProjWs proj_layout(const ckks_ctx *c, const ProjPlan &p, uint32_t level) {
     w.total = off; off += align256(ct * p.S);
     w.tmp = off;   off += align256(ct);
     w.ks = off;    off += align256(ks_bytes(c, level) * p.S * nib);   // all shards' key switches run side by side
+    // lazy giant steps: coefficient copies and extended digits of IP_TERMS giant steps of every shard
+    const size_t kbeta = (level + c->alpha - 1) / c->alpha;
+    w.ksx = off;   off += lazy ? align256((size_t)IP_TERMS * p.S * (level + kbeta * (level + c->K)) * c->N * sizeof(u64)) : 0;
     w.rs = off;    off += align256(rescale_bytes(c, level, 2));
     w.bytes = off;
     return w;
@@ -235,6 +238,9 @@ extern "C" size_t ckks_workspace_bytes(const ckks_ctx *c, int32_t op, uint32_t l
         // per ciphertext of a chunk: staged input, staged output and a key-switch workspace
         case CKKS_OP_ROTATE_BATCH:
             return (size_t)std::min<uint32_t>(count ? count : 1, MRB_CHUNK) * ((size_t)4 * level * limb + ks_bytes(c, level));
+        // a chunk of staged inputs with their key-switch workspaces
+        case CKKS_OP_ROTATE_SUM:
+            return (size_t)std::min<uint32_t>(count ? count : 1, MRB_CHUNK) * ((size_t)2 * level * limb + ks_bytes(c, level));
         case CKKS_OP_MUL_RELIN_BATCH:
             return (size_t)std::min<uint32_t>(count ? count : 1, MRB_CHUNK) * ((size_t)3 * level * limb + ks_bytes(c, level));
         // two running ciphertexts, the truncated copy of x, then the Mult and rescale scratch
@@ -642,6 +648,52 @@ extern "C" int32_t ckks_rotate_batch(ckks_ctx *c, const ckks_ct *in, uint32_t n,
     return rc;
 }
 
+extern "C" int32_t ckks_rotate_sum(ckks_ctx *c, const ckks_ct *in, const ckks_evk *keys, uint32_t n, ckks_ct *out, void *ws, size_t ws_bytes,
+                                   void *stream) {
+    if (!c || !in || !keys || !out || !n || !ct_ok(out)) return CKKS_ERR_ARG;
+    for (uint32_t i = 0; i < n; i++)
+        if (!ct_ok(&in[i]) || in[i].ncomp != 2) return CKKS_ERR_ARG;
+    const uint32_t level = in[0].level;
+    if (!level_ok(c, level)) return CKKS_ERR_LEVEL;
+    for (uint32_t i = 0; i < n; i++) {
+        if (in[i].level != level) return CKKS_ERR_LEVEL;
+        if (!scales_agree(in[i].scale, in[0].scale)) return CKKS_ERR_SCALE;
+        if (!keys[i].data || keys[i].galois == 0) return CKKS_ERR_NO_KEY;
+    }
+    if (!ws || ws_bytes < ckks_workspace_bytes(c, CKKS_OP_ROTATE_SUM, level, n)) return CKKS_ERR_WORKSPACE;
+    DeviceGuard g(c->device);
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t N = c->N, ctl = (size_t)2 * level * N, ptl = (size_t)level * N;
+    const uint32_t beta = (level + c->alpha - 1) / c->alpha, nt = level + c->K;
+    const uint32_t mmax = std::min(MRB_CHUNK, n);
+    u64 *xin = (u64 *)ws;
+    KsWorkspace w = ks_carve(c, level, xin + (size_t)mmax * ctl, mmax);
+    for (uint32_t i0 = 0; i0 < n; i0 += MRB_CHUNK) {
+        const uint32_t m = std::min(MRB_CHUNK, n - i0);
+        for (uint32_t i = 0; i < m; i++)
+            cudaMemcpyAsync(xin + (size_t)i * ctl, in[i0 + i].data, ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+        ks_modup(c, xin + ptl, level, w, s, m, ctl);
+        // every term has its own digits, key and first component; all of them add into entry 0 of the inner-product
+        // buffer, the first components multiplied by P so that the one ModDown returns them unchanged
+        for (uint32_t t0 = 0; t0 < m; t0 += IP_TERMS) {
+            const uint32_t nterm = std::min(IP_TERMS, m - t0);
+            IpTerms tm{};
+            for (uint32_t t = 0; t < nterm; t++) {
+                tm.evk[t] = (const u64 *)keys[i0 + t0 + t].data;
+                tm.galois[t] = keys[i0 + t0 + t].galois;
+                tm.c0[t] = xin + (size_t)(t0 + t) * ctl;
+            }
+            KsWorkspace wt = w;
+            wt.ext = w.ext + (size_t)t0 * beta * nt * N;
+            ks_inner_terms(c, level, wt, (size_t)beta * nt * N, tm, nterm, 0, s, 1, i0 + t0 > 0);
+        }
+    }
+    ks_moddown(c, level, w, nullptr, nullptr, 1, (u64 *)out->data, s);
+    int rc = finish(c);
+    if (rc == CKKS_OK) { out->level = level; out->ncomp = 2; out->scale = in[0].scale; }
+    return rc;
+}
+
 extern "C" int32_t ckks_rotate_hoisted(ckks_ctx *c, const ckks_ct *in, const ckks_evk *keys, uint32_t nrot, ckks_ct *outs,
                                        void *ws, size_t ws_bytes, void *stream) {
     int rc = rotate_checks(c, in, keys, nrot, outs, ws, ws_bytes);
@@ -700,7 +752,7 @@ extern "C" size_t ckks_linear_proj_workspace_bytes(const ckks_ctx *c, const ckks
     if (!c || !level_ok(c, level) || level < 2) return 0;
     ProjPlan p;
     if (make_plan(c, d, p)) return 0;
-    return proj_layout(c, p, level).bytes;
+    return proj_layout(c, p, level, (d->flags & CKKS_PROJ_LAZY_MODDOWN) != 0).bytes;
 }
 
 // nmat projections of the same inputs (descriptors agreeing in d_in, tokens_per_shard, nshards, baby): the inputs'
@@ -718,6 +770,7 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
         if (descs[m].d_in != descs[0].d_in || descs[m].tokens_per_shard != descs[0].tokens_per_shard || descs[m].nshards != descs[0].nshards ||
             descs[m].baby != descs[0].baby)
             return CKKS_ERR_ARG;
+        if (descs[m].flags & ~CKKS_PROJ_LAZY_MODDOWN) return CKKS_ERR_ARG;
     }
     merged = plans[0];
     for (uint32_t m = 1; m < nmat; m++) merged.gmax = std::max(merged.gmax, plans[m].gmax);
@@ -738,7 +791,9 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
         for (int64_t r : plans[m].rots)
             if (!find_key(keys, nkeys, ckks_galois_element(c, r))) return CKKS_ERR_NO_KEY;
     }
-    const ProjWs L = proj_layout(c, merged, level);
+    bool any_lazy = false;
+    for (uint32_t m = 0; m < nmat; m++) any_lazy = any_lazy || (descs[m].flags & CKKS_PROJ_LAZY_MODDOWN) != 0;
+    const ProjWs L = proj_layout(c, merged, level, any_lazy);
     if (!ws || ws_bytes < L.bytes) return CKKS_ERR_WORKSPACE;
 
     DeviceGuard g(c->device);
@@ -751,6 +806,11 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
     double *slots = (double *)(base + L.slots);
     void *encw = base + L.enc;
     KsWorkspace kw = ks_carve(c, level, base + L.ks, S * nib);
+    // lazy giant steps: digits of IP_TERMS x S accumulators side by side; the running sum and the ModDown use kw's buffers
+    const uint32_t kbeta = (level + c->alpha - 1) / c->alpha, knt = level + c->K;
+    KsWorkspace kx = kw;
+    kx.dcoef = (u64 *)(base + L.ksx);
+    kx.ext = kx.dcoef + (size_t)IP_TERMS * S * level * N;
 
     // baby row ((sh*nib + ib)*B + b)*2 + comp = component comp of rho^(b T)(x_{sh,ib}), tiled layout: one ModUp for all
     // input ciphertexts at once, then every baby rotation is applied to all of them in one batch (the key is read
@@ -781,6 +841,8 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
         for (uint32_t ob = 0; ob < nob; ob++) {
             const Block &o = p.outs[ob];
             uint32_t gcount = 0, fold = 1;
+            const bool lazy = (d->flags & CKKS_PROJ_LAZY_MODDOWN) != 0;
+            bool u_live = false;        // the inner-product buffer holds a running sum of giant steps
             for (const Block &i : p.ins) {
                 gcount = std::max(gcount, std::min(i.size, o.size) / B);
                 if (i.size > o.size) fold = i.size / o.size;
@@ -840,7 +902,7 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
                     count_launches();
                 }
                 }
-                for (uint32_t gl = 0; gl < ng; gl++) {
+                for (uint32_t gl = 0; gl < ng && !lazy; gl++) {
                     const uint32_t gi = g0 + gl;
                     u64 *ag = acc + (size_t)gl * S * ctl;
                     if (gi == 0) {
@@ -853,7 +915,30 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
                     ks_modup(c, ag + ptl, level, kw, s, S, ctl);
                     ks_inner_moddown(c, key, level, ge, kw, ag, nullptr, ge, total, s, S, ctl, ctl, true);
                 }
+                // lazy: the key-switched parts of up to IP_TERMS giant steps (all shards) are extended in one batch and
+                // added to the running sum in the key-switching basis in one pass, their first components with them
+                for (uint32_t gl = 0; gl < ng && lazy;) {
+                    if (g0 + gl == 0) {
+                        cudaMemcpyAsync(total, acc, (size_t)S * ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+                        gl++;
+                        continue;
+                    }
+                    const uint32_t nterm = std::min(IP_TERMS, ng - gl);
+                    u64 *ag = acc + (size_t)gl * S * ctl;
+                    ks_modup(c, ag + ptl, level, kx, s, nterm * S, ctl);
+                    IpTerms tm{};
+                    for (uint32_t t = 0; t < nterm; t++) {
+                        const u64 ge = ckks_galois_element(c, (int64_t)(g0 + gl + t) * B * T);
+                        tm.evk[t] = (const u64 *)find_key(keys, nkeys, ge)->data;
+                        tm.galois[t] = ge;
+                        tm.c0[t] = ag + (size_t)t * S * ctl;
+                    }
+                    ks_inner_terms(c, level, kx, (size_t)S * kbeta * knt * N, tm, nterm, ctl, s, S, u_live);
+                    u_live = true;
+                    gl += nterm;
+                }
             }
+            if (u_live) ks_moddown(c, level, kw, total, total + ptl, 1, total, s, S, ctl, ctl, false);
             for (uint32_t f = o.size; fold > 1; f *= 2, fold /= 2) {
                 const u64 ge = ckks_galois_element(c, (int64_t)f * T);
                 const u64 *key = (const u64 *)find_key(keys, nkeys, ge)->data;
@@ -899,10 +984,12 @@ extern "C" size_t ckks_linear_proj_multi_workspace_bytes(const ckks_ctx *c, cons
     if (!c || !descs || !nmat || !level_ok(c, level) || level < 2) return 0;
     ProjPlan merged;
     if (make_plan(c, &descs[0], merged)) return 0;
+    bool lazy = (descs[0].flags & CKKS_PROJ_LAZY_MODDOWN) != 0;
     for (uint32_t m = 1; m < nmat; m++) {
         ProjPlan p;
         if (make_plan(c, &descs[m], p)) return 0;
         merged.gmax = std::max(merged.gmax, p.gmax);
+        lazy = lazy || (descs[m].flags & CKKS_PROJ_LAZY_MODDOWN) != 0;
     }
-    return proj_layout(c, merged, level).bytes;
+    return proj_layout(c, merged, level, lazy).bytes;
 }

@@ -40,6 +40,7 @@ struct DevTables {
     const double2 *dn_hat_mod_d;   // [L][K]   {c, c / q_i} as doubles
     const ulonglong2 *dn_p_inv;    // [L]      {P^-1 mod q_i, Shoup}
     const double2 *dn_p_inv_d;     // [L]      {P^-1 mod q_i, that / q_i} as doubles
+    const double *dn_p_mod_d;      // [L]      P mod q_i as a double
     // Rescale: [L(last)][L(i)] {q_last^-1 mod q_i, Shoup}
     const ulonglong2 *rs_inv;
     // Encode:
@@ -255,6 +256,26 @@ void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext
                       const u64 *add0, const u64 *add1, u64 add_galois, u64 *out, cudaStream_t s, uint32_t nb = 1,
                       size_t add_stride = 0, size_t out_stride = 0, bool accumulate = false, TiledOut tiled = TiledOut(),
                       const KsMulti *multi = nullptr);
+// The two halves of ks_inner_moddown.  ks_inner leaves u = <digits, evk> in the extended basis (w.u, nb entries); with
+// acc_u it adds to what w.u holds, so that a sum of key-switched terms can share one ks_moddown.
+void ks_inner(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext_galois, const KsWorkspace &w, cudaStream_t s, uint32_t nb = 1,
+              bool acc_u = false, const KsMulti *multi = nullptr);
+void ks_moddown(const ckks_ctx *c, uint32_t level, const KsWorkspace &w, const u64 *add0, const u64 *add1, u64 add_galois, u64 *out,
+                cudaStream_t s, uint32_t nb = 1, size_t add_stride = 0, size_t out_stride = 0, bool accumulate = false,
+                TiledOut tiled = TiledOut(), const KsMulti *multi = nullptr);
+// A sum of up to IP_TERMS key-switched terms in one pass over the extended basis:
+//   u[b] (+)= sum_t ( <ext[t][b] read through sigma_{g_t}, evk_t>  +  P sigma_{g_t}(c0_t[b]) on component 0's q-limbs )
+// ext holds term t's digits of batch entry b at ext + t * term_stride + b * beta * (level + K) * N words; c0[t]
+// (may be null) points at term t's first-component limbs, entries c0_stride words apart.  Adding P c0 before the
+// ModDown equals adding c0 after it, exactly.
+constexpr uint32_t IP_TERMS = 4;
+struct IpTerms {
+    const u64 *evk[IP_TERMS];
+    u64 galois[IP_TERMS];
+    const u64 *c0[IP_TERMS];
+};
+void ks_inner_terms(const ckks_ctx *c, uint32_t level, const KsWorkspace &w, size_t term_stride, const IpTerms &terms, uint32_t nterm,
+                    size_t c0_stride, cudaStream_t s, uint32_t nb, bool acc_u);
 // rows of [level][N] words, src_stride words apart, into rows row0, row0 + row_step, .. of a tiled buffer with R rows
 void launch_to_tiled(const ckks_ctx *c, const u64 *src, size_t src_stride, uint32_t nrows, u64 *dst, uint32_t R, uint32_t row0,
                      uint32_t row_step, uint32_t level, cudaStream_t s);

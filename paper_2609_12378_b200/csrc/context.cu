@@ -210,6 +210,7 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
     // ---- ModDown constants
     std::vector<ulonglong2> dn_inv(K), dn_pinv(L);
     std::vector<double2> dn_pinv_d(L);
+    std::vector<double> dn_pmod_d(L);
     std::vector<u64> dn_mod((size_t)L * K);
     std::vector<double2> dn_mod_d((size_t)L * K);
     for (uint32_t a = 0; a < K; a++) {
@@ -230,6 +231,7 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
         }
         dn_pinv[i] = h_pair(h_inv(Pm, q), q);
         dn_pinv_d[i] = make_double2((double)dn_pinv[i].x, (double)dn_pinv[i].x / (double)q);
+        dn_pmod_d[i] = (double)Pm;
     }
 
     // ---- Rescale constants
@@ -258,7 +260,7 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
     if ((rc = upload(c, mod, &d.mod)) || (rc = upload(c, mu, &d.mu)) || (rc = upload(c, mu64, &d.mu64)) || (rc = upload(c, modd, &d.modd)) || (rc = upload(c, twf, &d.tw_fwd)) ||
         (rc = upload(c, twi, &d.tw_inv)) || (rc = upload(c, twdf, &d.twd_fwd)) || (rc = upload(c, twdi, &d.twd_inv)) || (rc = upload(c, ninvd, &d.n_inv_d)) || (rc = upload(c, ninv, &d.n_inv)) || (rc = upload(c, up_inv, &d.up_hat_inv)) ||
         (rc = upload(c, up_mod, &d.up_hat_mod)) || (rc = upload(c, up_mod_d, &d.up_hat_mod_d)) || (rc = upload(c, dn_mod_d, &d.dn_hat_mod_d)) || (rc = upload(c, dn_inv, &d.dn_hat_inv)) ||
-        (rc = upload(c, dn_mod, &d.dn_hat_mod)) || (rc = upload(c, dn_pinv, &d.dn_p_inv)) || (rc = upload(c, dn_pinv_d, &d.dn_p_inv_d)) || (rc = upload(c, rs, &d.rs_inv)) ||
+        (rc = upload(c, dn_mod, &d.dn_hat_mod)) || (rc = upload(c, dn_pinv, &d.dn_p_inv)) || (rc = upload(c, dn_pinv_d, &d.dn_p_inv_d)) || (rc = upload(c, dn_pmod_d, &d.dn_p_mod_d)) || (rc = upload(c, rs, &d.rs_inv)) ||
         (rc = upload(c, enc_src, &d.enc_src)) || (rc = upload(c, om, &d.enc_omega)) || (rc = upload(c, ze, &d.enc_zeta)) ||
         (rc = upload(c, flag, &flag_dev))) {
         cudaSetDevice(prev);

@@ -97,7 +97,7 @@ void launch_modup(const ckks_ctx *c, const u64 *dcoef, const u64 *deval, size_t 
 
 // u[comp][x][p] = sum_j ext[j][x][pi_g(p)] * evk[j][comp][kt(x)][p]          (any number of digits)
 __global__ void __launch_bounds__(THREADS) inner_product_generic_kernel(DevTables c, const u64 *ext, const u64 *evk, u64 g,
-                                                                        u64 *u, uint32_t level, int has_multi, KsMulti multi) {
+                                                                        u64 *u, uint32_t level, int has_multi, KsMulti multi, int acc_u) {
     const uint32_t p = blockIdx.x * THREADS + threadIdx.x;
     const uint32_t x = blockIdx.z, bz = blockIdx.y;     // batch varies faster than the limb: a key limb is reused from L2
     const uint32_t nt = level + c.K, beta = (level + c.alpha - 1) / c.alpha;
@@ -115,8 +115,14 @@ __global__ void __launch_bounds__(THREADS) inner_product_generic_kernel(DevTable
         a1 = __dadd_rn(a1, mulmod_dd(e, u64_to_d(evk[(((size_t)j * 2 + 1) * c.T + kt) * c.N + p]), md.x, md.y));
         if ((j & 7) == 7) { a0 = reduce_d(a0, md.x, md.y); a1 = reduce_d(a1, md.x, md.y); }
     }
-    u[((size_t)0 * nt + x) * c.N + p] = canonical_d(reduce_d(a0, md.x, md.y), md.x);
-    u[((size_t)1 * nt + x) * c.N + p] = canonical_d(reduce_d(a1, md.x, md.y), md.x);
+    u64 r0 = canonical_d(reduce_d(a0, md.x, md.y), md.x), r1 = canonical_d(reduce_d(a1, md.x, md.y), md.x);
+    if (acc_u) {        // a sum of key-switched terms kept in the extended basis
+        const u64 m = c.mod[kt];
+        r0 = add_mod(r0, u[((size_t)0 * nt + x) * c.N + p], m);
+        r1 = add_mod(r1, u[((size_t)1 * nt + x) * c.N + p], m);
+    }
+    u[((size_t)0 * nt + x) * c.N + p] = r0;
+    u[((size_t)1 * nt + x) * c.N + p] = r1;
 }
 
 // The same for BETA <= 4 digits, two adjacent coefficients per thread.  pi_g maps the pair (p, p + 1), p even, onto a
@@ -126,7 +132,8 @@ __global__ void __launch_bounds__(THREADS) inner_product_generic_kernel(DevTable
 constexpr uint32_t IP_MAX_BETA = 4;
 template <uint32_t BETA>
 __global__ void __launch_bounds__(THREADS) inner_product_kernel(DevTables c, const u64 *ext, const u64 *evk, u64 g, u64 *u,
-                                                                uint32_t level, uint32_t nb, uint32_t bch, int has_multi, KsMulti multi) {
+                                                                uint32_t level, uint32_t nb, uint32_t bch, int has_multi, KsMulti multi,
+                                                                int acc_u) {
     const uint32_t p = (blockIdx.x * THREADS + threadIdx.x) * 2;
     const uint32_t x = blockIdx.z, b0 = blockIdx.y * bch, b1 = min(b0 + bch, nb);     // chunks of a limb run together: its key words come from L2
     const uint32_t nt = level + c.K;
@@ -164,6 +171,94 @@ __global__ void __launch_bounds__(THREADS) inner_product_kernel(DevTables c, con
             ulonglong2 r;
             r.x = canonical_d(reduce_d(acc[cm][0], md.x, md.y), md.x);
             r.y = canonical_d(reduce_d(acc[cm][1], md.x, md.y), md.x);
+            if (acc_u) {
+                const ulonglong2 old = *reinterpret_cast<const ulonglong2 *>(o + cm * js);
+                const u64 m = c.mod[kt];
+                r.x = add_mod(r.x, old.x, m);
+                r.y = add_mod(r.y, old.y, m);
+            }
+            *reinterpret_cast<ulonglong2 *>(o + cm * js) = r;
+        }
+    }
+}
+
+// The inner product of several terms at once (see ks_inner_terms): like inner_product_kernel, but every term has its
+// own digits, key, permutation and first component, and the running sums of a chunk of IP_BCH batch entries stay in
+// registers over the terms.
+constexpr uint32_t IP_BCH = 4;
+template <uint32_t BETA>
+__global__ void __launch_bounds__(THREADS, 3) inner_product_terms_kernel(DevTables c, const u64 *ext, size_t term_stride,
+                                                                         const __grid_constant__ IpTerms tm, uint32_t nterm, size_t c0_stride,
+                                                                         u64 *u, uint32_t level, uint32_t nb, int acc_u) {
+    const uint32_t p = (blockIdx.x * THREADS + threadIdx.x) * 2;
+    const uint32_t x = blockIdx.z, b0 = blockIdx.y * IP_BCH;
+    const uint32_t nt = level + c.K;
+    const uint32_t kt = x < level ? x : c.L + (x - level);
+    const double2 md = c.modd[kt];
+    const size_t js = (size_t)nt * c.N, ks = (size_t)c.T * c.N;
+    const double pq = x < level ? c.dn_p_mod_d[x] : 0.0;
+    double acc[IP_BCH][2][2];
+#pragma unroll
+    for (uint32_t bi = 0; bi < IP_BCH; bi++) acc[bi][0][0] = acc[bi][0][1] = acc[bi][1][0] = acc[bi][1][1] = 0.0;
+    for (uint32_t t = 0; t < nterm; t++) {
+        const uint32_t src = galois_src(p, tm.galois[t], c.log_n, c.N);
+        const bool odd = src & 1;
+        const u64 *evk = tm.evk[t];
+        double k[BETA][2][2];
+#pragma unroll
+        for (uint32_t j = 0; j < BETA; j++)
+#pragma unroll
+            for (uint32_t cm = 0; cm < 2; cm++) {
+                const ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(evk + ((size_t)j * 2 + cm) * ks + (size_t)kt * c.N + p);
+                k[j][cm][0] = u64_to_d(v.x);
+                k[j][cm][1] = u64_to_d(v.y);
+            }
+        const u64 *e = ext + t * term_stride + (size_t)b0 * BETA * js + (size_t)x * c.N + (src & ~1u);
+        const u64 *z = (x < level && tm.c0[t]) ? tm.c0[t] + b0 * c0_stride + (size_t)x * c.N + (src & ~1u) : nullptr;
+        // no branch in here, so that the loads of all entries of the chunk are in flight together: an entry past the end
+        // of the batch repeats the last one and is not stored
+#pragma unroll
+        for (uint32_t bi = 0; bi < IP_BCH; bi++) {
+            const uint32_t bc = min(bi, nb - 1 - b0);
+            double sum[2][2] = {{0.0, 0.0}, {0.0, 0.0}};
+#pragma unroll
+            for (uint32_t j = 0; j < BETA; j++) {
+                const ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(e + ((size_t)bc * BETA + j) * js);
+                const double d0 = u64_to_d(odd ? v.y : v.x), d1 = u64_to_d(odd ? v.x : v.y);
+#pragma unroll
+                for (uint32_t cm = 0; cm < 2; cm++) {
+                    sum[cm][0] = __dadd_rn(sum[cm][0], mulmod_dd(d0, k[j][cm][0], md.x, md.y));
+                    sum[cm][1] = __dadd_rn(sum[cm][1], mulmod_dd(d1, k[j][cm][1], md.x, md.y));
+                }
+            }
+            if (z) {
+                const ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(z + bc * c0_stride);
+                sum[0][0] = __dadd_rn(sum[0][0], mulmod_dd(u64_to_d(odd ? v.y : v.x), pq, md.x, md.y));
+                sum[0][1] = __dadd_rn(sum[0][1], mulmod_dd(u64_to_d(odd ? v.x : v.y), pq, md.x, md.y));
+            }
+            // at most BETA + 1 products of size 0.75 m on top of a reduced sum: far below 2^53
+#pragma unroll
+            for (uint32_t cm = 0; cm < 2; cm++) {
+                acc[bi][cm][0] = reduce_d(__dadd_rn(acc[bi][cm][0], sum[cm][0]), md.x, md.y);
+                acc[bi][cm][1] = reduce_d(__dadd_rn(acc[bi][cm][1], sum[cm][1]), md.x, md.y);
+            }
+        }
+    }
+    const u64 m = c.mod[kt];
+#pragma unroll
+    for (uint32_t bi = 0; bi < IP_BCH; bi++) {
+        if (b0 + bi >= nb) break;
+        u64 *o = u + (size_t)(b0 + bi) * 2 * js + (size_t)x * c.N + p;
+#pragma unroll
+        for (uint32_t cm = 0; cm < 2; cm++) {
+            ulonglong2 r;
+            r.x = canonical_d(acc[bi][cm][0], md.x);
+            r.y = canonical_d(acc[bi][cm][1], md.x);
+            if (acc_u) {
+                const ulonglong2 old = *reinterpret_cast<const ulonglong2 *>(o + cm * js);
+                r.x = add_mod(r.x, old.x, m);
+                r.y = add_mod(r.y, old.y, m);
+            }
             *reinterpret_cast<ulonglong2 *>(o + cm * js) = r;
         }
     }
@@ -275,6 +370,15 @@ __global__ void __launch_bounds__(THREADS) rescale_final_kernel(DevTables c, con
     out[((size_t)comp * (level - 1) + i) * c.N + p] = mul_shoup(r, inv.x, inv.y, q);
 }
 
+// u[b][0][i][p] += P sigma_g(c0[b][i])[p]   (first component's q-limbs of the extended-basis sum)
+__global__ void __launch_bounds__(THREADS) p_c0_acc_kernel(DevTables c, const u64 *c0, size_t c0_stride, u64 g, u64 *u, size_t u_stride) {
+    const uint32_t p = blockIdx.x * THREADS + threadIdx.x, i = blockIdx.y, b = blockIdx.z;
+    const double2 md = c.modd[i];
+    u64 *d = u + b * u_stride + (size_t)i * c.N + p;
+    const double v = mulmod_dd(u64_to_d(c0[b * c0_stride + (size_t)i * c.N + galois_src(p, g, c.log_n, c.N)]), c.dn_p_mod_d[i], md.x, md.y);
+    *d = add_mod(*d, canonical_d(reduce_d(v, md.x, md.y), md.x), c.mod[i]);
+}
+
 }  // namespace
 
 size_t ks_workspace_limbs(const ckks_ctx *c, uint32_t level) {
@@ -308,11 +412,11 @@ void ks_modup(const ckks_ctx *c, const u64 *d, uint32_t level, const KsWorkspace
     launch_ntt(c, w.ext, nb * beta * nt, ext_map(level, c->K, c->L, c->alpha, beta), false, s);
 }
 
-void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext_galois, const KsWorkspace &w,
-                      const u64 *add0, const u64 *add1, u64 add_galois, u64 *out, cudaStream_t s, uint32_t nb,
-                      size_t add_stride, size_t out_stride, bool accumulate, TiledOut tiled, const KsMulti *multi) {
-    const uint32_t N = c->N, nt = level + c->K, K = c->K;
+void ks_inner(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext_galois, const KsWorkspace &w, cudaStream_t s, uint32_t nb,
+              bool acc_u, const KsMulti *multi) {
+    const uint32_t N = c->N, nt = level + c->K;
     const uint32_t beta = (level + c->alpha - 1) / c->alpha;
+    const int au = acc_u ? 1 : 0;
     bool aligned = ((uintptr_t)w.ext & 15) == 0 && ((uintptr_t)w.u & 15) == 0 && (multi || ((uintptr_t)evk & 15) == 0);
     if (multi)
         for (uint32_t b = 0; b < nb; b++) aligned = aligned && ((uintptr_t)multi->evk[b] & 15) == 0;
@@ -322,16 +426,21 @@ void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext
         const dim3 grid(N / (2 * THREADS), (nb + bch - 1) / bch, nt);
         const KsMulti m = multi ? *multi : KsMulti{};
         switch (beta) {
-        case 1: inner_product_kernel<1><<<grid, THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, nb, bch, multi ? 1 : 0, m); break;
-        case 2: inner_product_kernel<2><<<grid, THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, nb, bch, multi ? 1 : 0, m); break;
-        case 3: inner_product_kernel<3><<<grid, THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, nb, bch, multi ? 1 : 0, m); break;
-        default: inner_product_kernel<4><<<grid, THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, nb, bch, multi ? 1 : 0, m); break;
+        case 1: inner_product_kernel<1><<<grid, THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, nb, bch, multi ? 1 : 0, m, au); break;
+        case 2: inner_product_kernel<2><<<grid, THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, nb, bch, multi ? 1 : 0, m, au); break;
+        case 3: inner_product_kernel<3><<<grid, THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, nb, bch, multi ? 1 : 0, m, au); break;
+        default: inner_product_kernel<4><<<grid, THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, nb, bch, multi ? 1 : 0, m, au); break;
         }
     } else {
         inner_product_generic_kernel<<<dim3(N / THREADS, nb, nt), THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, multi ? 1 : 0,
-                                                                                     multi ? *multi : KsMulti{});
+                                                                                     multi ? *multi : KsMulti{}, au);
     }
     count_launches();
+}
+
+void ks_moddown(const ckks_ctx *c, uint32_t level, const KsWorkspace &w, const u64 *add0, const u64 *add1, u64 add_galois, u64 *out,
+                cudaStream_t s, uint32_t nb, size_t add_stride, size_t out_stride, bool accumulate, TiledOut tiled, const KsMulti *multi) {
+    const uint32_t N = c->N, nt = level + c->K, K = c->K;
     // the K special limbs of every (batch, component): groups of K limbs, nt limbs apart
     launch_ntt(c, w.u + (size_t)level * N, nb * 2 * K, pitched_map(c->L, K, nt), true, s);
 #define CALL_DN(A) launch_moddown_conv<A>(c, w.u, w.conv, level, nb, s)
@@ -357,6 +466,42 @@ void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext
     moddown_final_kernel<<<dim3(N / THREADS, level, 2 * nb), THREADS, 0, s>>>(c->dev, w.u, w.conv, add0, add1, add_stride, add_galois, out,
                                                                                out_stride, accumulate ? 1 : 0, level, tiled);
     count_launches();
+}
+
+void ks_inner_moddown(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext_galois, const KsWorkspace &w,
+                      const u64 *add0, const u64 *add1, u64 add_galois, u64 *out, cudaStream_t s, uint32_t nb,
+                      size_t add_stride, size_t out_stride, bool accumulate, TiledOut tiled, const KsMulti *multi) {
+    ks_inner(c, evk, level, ext_galois, w, s, nb, false, multi);
+    ks_moddown(c, level, w, add0, add1, add_galois, out, s, nb, add_stride, out_stride, accumulate, tiled, multi);
+}
+
+void ks_inner_terms(const ckks_ctx *c, uint32_t level, const KsWorkspace &w, size_t term_stride, const IpTerms &terms, uint32_t nterm,
+                    size_t c0_stride, cudaStream_t s, uint32_t nb, bool acc_u) {
+    const uint32_t N = c->N, nt = level + c->K, beta = (level + c->alpha - 1) / c->alpha;
+    bool aligned = ((uintptr_t)w.ext & 15) == 0 && ((uintptr_t)w.u & 15) == 0 && (term_stride & 1) == 0 && (c0_stride & 1) == 0;
+    for (uint32_t t = 0; t < nterm; t++) aligned = aligned && ((uintptr_t)terms.evk[t] & 15) == 0 && ((uintptr_t)terms.c0[t] & 15) == 0;
+    if (beta <= IP_MAX_BETA && N >= 2 * THREADS && aligned) {
+        const dim3 grid(N / (2 * THREADS), (nb + IP_BCH - 1) / IP_BCH, nt);
+        const int au = acc_u ? 1 : 0;
+        switch (beta) {
+        case 1: inner_product_terms_kernel<1><<<grid, THREADS, 0, s>>>(c->dev, w.ext, term_stride, terms, nterm, c0_stride, w.u, level, nb, au); break;
+        case 2: inner_product_terms_kernel<2><<<grid, THREADS, 0, s>>>(c->dev, w.ext, term_stride, terms, nterm, c0_stride, w.u, level, nb, au); break;
+        case 3: inner_product_terms_kernel<3><<<grid, THREADS, 0, s>>>(c->dev, w.ext, term_stride, terms, nterm, c0_stride, w.u, level, nb, au); break;
+        default: inner_product_terms_kernel<4><<<grid, THREADS, 0, s>>>(c->dev, w.ext, term_stride, terms, nterm, c0_stride, w.u, level, nb, au); break;
+        }
+        count_launches();
+        return;
+    }
+    // any number of digits, any alignment: one term at a time through the generic kernel, then its P c0
+    for (uint32_t t = 0; t < nterm; t++) {
+        inner_product_generic_kernel<<<dim3(N / THREADS, nb, nt), THREADS, 0, s>>>(c->dev, w.ext + t * term_stride, terms.evk[t], terms.galois[t],
+                                                                                     w.u, level, 0, KsMulti{}, (acc_u || t > 0) ? 1 : 0);
+        count_launches();
+        if (terms.c0[t]) {
+            p_c0_acc_kernel<<<dim3(N / THREADS, level, nb), THREADS, 0, s>>>(c->dev, terms.c0[t], c0_stride, terms.galois[t], w.u, (size_t)2 * nt * N);
+            count_launches();
+        }
+    }
 }
 
 void launch_to_tiled(const ckks_ctx *c, const u64 *src, size_t src_stride, uint32_t nrows, u64 *dst, uint32_t R, uint32_t row0,

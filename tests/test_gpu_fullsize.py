@@ -49,6 +49,16 @@ def test_llama_shaped_projection_full_size():
     want, want_scale = o.linear_proj(one, cts[c][None], W, keys, scale)
     assert want_scale == outs[c].scale
     assert np.array_equal(got[c], want[0])
+    # the schedule with the giant steps summed before one ModDown: all shards decrypt to X W, the sampled shard is the
+    # checker's lazy variant bit for bit
+    lazy = ctx.linear_proj(dcts, dev(W), dkeys, D, D, T, S, B, lazy_moddown=True)
+    assert ctx.device_status() == binding.OK
+    for cc in range(S):
+        sl = cl.decrypt_slots(host(lazy[cc].data), lazy[cc].scale).real.reshape(D, T)
+        assert np.abs(sl - Y[cc * T:(cc + 1) * T].T).max() < 2.0 ** -16
+    want_lazy, _ = o.linear_proj(ProjDesc(D, D, T, 1, B, lazy_moddown=True), cts[c][None], W, keys, scale)
+    assert np.array_equal(host(lazy[c].data), want_lazy[0])
+    del lazy
     # the same inputs through the square and a key-shaped (4096 x 1024) matrix in one call with shared baby steps:
     # the square matrix's outputs do not change, the second matrix's decrypt to X Wk (one block, stored four times)
     Wk = inputs.weights_normal(inputs.rng(1004, 3), D, 1024, 0.02)

@@ -10,7 +10,7 @@ from tests.harness import Client, params
 pytestmark = pytest.mark.gpu
 
 
-def _run(log_n, L, K, dnum, level, d_in, d_out, T, S, B, seed, pt_scale=0.0, check_slots=True):
+def _run(log_n, L, K, dnum, level, d_in, d_out, T, S, B, seed, pt_scale=0.0, check_slots=True, lazy=False):
     from tests.gpu_util import context, ct_dev, dev, host, key_dev
     P, ctx = params(log_n, L, K, dnum), context(log_n, L, K, dnum)
     o = P.oracle
@@ -19,7 +19,7 @@ def _run(log_n, L, K, dnum, level, d_in, d_out, T, S, B, seed, pt_scale=0.0, che
     g = inputs.rng(seed, 1)
     X = inputs.activations_uniform(g, S * T, d_in)
     W = inputs.weights_normal(g, d_in, d_out, 0.02)
-    desc = ProjDesc(d_in, d_out, T, S, B, pt_scale)
+    desc = ProjDesc(d_in, d_out, T, S, B, pt_scale, lazy_moddown=lazy)
     F, ins, outs = o.proj_blocks(desc)
     cts = []
     for c in range(S):
@@ -30,7 +30,7 @@ def _run(log_n, L, K, dnum, level, d_in, d_out, T, S, B, seed, pt_scale=0.0, che
     keys = {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in rots}
     want, want_scale = o.linear_proj(desc, np.stack(cts), W, keys, scale)
     got = ctx.linear_proj([ct_dev(c, scale) for c in cts], dev(W), [key_dev(k, g_) for g_, k in keys.items()],
-                          d_in, d_out, T, S, B, pt_scale)
+                          d_in, d_out, T, S, B, pt_scale, lazy_moddown=lazy)
     assert len(got) == S * len(outs)
     Y = X @ W
     for i, ct in enumerate(got):
@@ -68,6 +68,26 @@ def test_projection_shapes_small_ring(d_in, d_out, T, S, B):
 ])
 def test_projection_tensor_core_mac_path(d_in, d_out, T, S, B):
     _run(10, 4, 2, 2, 4, d_in, d_out, T, S, B, seed=440 + d_in + d_out + S)
+
+
+@pytest.mark.parametrize("d_in,d_out,T,S,B", [
+    (16, 16, 32, 2, 4),      # three giant steps summed before one ModDown
+    (16, 4, 32, 2, 2),       # followed by a fold
+    (24, 16, 32, 2, 4),      # input blocks with different giant counts
+    (8, 8, 32, 1, 8),        # no giant step to sum: the eager result
+    (64, 160, 8, 9, 32),     # tensor-core path, several output blocks
+    (224, 64, 8, 2, 32),     # four input blocks
+])
+def test_projection_lazy_moddown(d_in, d_out, T, S, B):
+    """Giant steps summed in the key-switching basis, one ModDown per output ciphertext: bit-exact against the checker's
+    variant of the schedule."""
+    _run(10, 4, 2, 2, 4, d_in, d_out, T, S, B, seed=480 + d_in + d_out, lazy=True)
+
+
+def test_projection_lazy_moddown_many_groups():
+    """More giant steps than one group of accumulators holds (32 > 16): the running sum survives the next group's
+    encode and multiply-accumulate."""
+    _run(11, 4, 2, 2, 3, 128, 128, 8, 2, 4, seed=490, lazy=True)
 
 
 @pytest.mark.parametrize("shape", ["81", "83", "42", "100"])

@@ -268,6 +268,35 @@ def test_rotate_batch_bit_exact(log_n, L, K, dnum, level, n):
     assert e.value.code == binding.ERR_NO_KEY
 
 
+@pytest.mark.parametrize("log_n,L,K,dnum,level,n", [(10, 6, 2, 3, 5, 4), (11, 4, 2, 2, 4, 19), (10, 4, 1, 4, 3, 1), (10, 6, 1, 6, 6, 5), (16, 24, 8, 3, 24, 6)])
+def test_rotate_sum_bit_exact(log_n, L, K, dnum, level, n):
+    """sum_i rotate(ct_i, key_i) formed in the key-switching basis with one ModDown (n = 19 spans two chunks; n = 1 is the
+    plain rotation)."""
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    P, ctx = params(log_n, L, K, dnum), context(log_n, L, K, dnum)
+    o = P.oracle
+    cl = Client(P, 310 + n)
+    rots = [1 + 3 * i for i in range(min(n, 5))]
+    gals = [o.galois_element(r) for r in rots]
+    hk = [cl.rotation_key(x) for x in gals]
+    dk = [key_dev(k, x) for k, x in zip(hk, gals)]
+    g = inputs.rng(311, n)
+    cts = np.stack([cl.encrypt_slots(g.uniform(-1, 1, P.n), 2.0 ** 40, level) for _ in range(n)])
+    pick = [i % len(rots) for i in range(n)]
+    out = ctx.rotate_sum([ct_dev(c, 2.0 ** 40) for c in cts], [dk[j] for j in pick])
+    assert out.scale == 2.0 ** 40 and out.level == level
+    assert np.array_equal(host(out.data), o.rotate_sum(cts, [hk[j] for j in pick], [gals[j] for j in pick]))
+    if n == 1:
+        assert np.array_equal(host(out.data), o.rotate(cts[0], hk[0], gals[0]))
+    # in place on one of the inputs
+    d = [ct_dev(c, 2.0 ** 40) for c in cts]
+    ctx.rotate_sum(d, [dk[j] for j in pick], out=d[-1])
+    assert np.array_equal(host(d[-1].data), host(out.data))
+    with pytest.raises(binding.CkksError) as e:
+        ctx.rotate_sum(d[:1], [binding.SwitchKey(dk[0].data, 0)])
+    assert e.value.code == binding.ERR_NO_KEY
+
+
 def test_repeatability():
     """Same call twice gives the same bytes (a race would show up as a difference)."""
     from tests.gpu_util import context, ct_dev, host, key_dev
