@@ -138,6 +138,23 @@ def test_projection_multi_shares_baby_steps():
         ctx.linear_proj(cd, dev(W), kd, d_in, d_outs[m], T, S, B)
         n_sep += binding.kernel_launches() - n1
     assert n_multi < n_sep
+    # the same call with the giant steps summed before one ModDown: every matrix equals the checker's lazy schedule
+    got = ctx.linear_proj_multi(cd, [dev(W) for W in Ws], kd, d_in, d_outs, T, S, B, lazy_moddown=True)
+    for m, (d_out, W) in enumerate(zip(d_outs, Ws)):
+        want, _ = o.linear_proj(ProjDesc(d_in, d_out, T, S, B, 0.0, lazy_moddown=True), np.stack(cts), W, keys, scale)
+        for i, ct in enumerate(got[m]):
+            assert np.array_equal(host(ct.data), want[i]), (m, i)
+    with pytest.raises(binding.CkksError) as e:       # unknown descriptor flags are refused
+        bad = ctx._desc(16, 16, T, S, B)
+        bad.flags = 2
+        ws = ctx.workspace(1 << 20)
+        ia = (binding.CCt * len(cd))(*[binding._cct(c) for c in cd])
+        oa = (binding.CCt * 2)(*[binding._cct(ctx.empty_ct(level - 1)) for _ in range(2)])
+        ka = (binding.CEvk * len(kd))(*[binding.CEvk(k.data.data_ptr(), k.galois) for k in kd])
+        import ctypes as C
+        ctx._check(binding.load().ckks_linear_proj(ctx._h, C.byref(bad), ia, dev(Ws[0]).data_ptr(), ka, len(kd), oa, ws.data_ptr(),
+                                                   ws.numel(), None))
+    assert e.value.code == binding.ERR_ARG
     with pytest.raises(binding.CkksError) as e:       # descriptors must share the input shape
         lib = binding.load()
         import ctypes as C
