@@ -81,6 +81,7 @@ int make_plan(const ckks_ctx *c, const ckks_proj_desc *d, ProjPlan &p) {
 
 struct ProjWs { size_t baby, xin, pts, ptt, slots, enc, acc, total, tmp, ks, ksx, rs, bytes; uint32_t gg; bool per_block; };
 
+constexpr uint32_t BABY_ROTS = 4;            // baby-step rotations per key-switch pass (N = 2^16)
 constexpr uint32_t MAC_GT = 4, MAC_ST = 2;   // register tile of the multiply-accumulate kernel: giants x shards
 
 ProjWs proj_layout(const ckks_ctx *c, const ProjPlan &p, uint32_t level, bool lazy) {
@@ -106,7 +107,10 @@ ProjWs proj_layout(const ckks_ctx *c, const ProjPlan &p, uint32_t level, bool la
     w.acc = off;   off += align256(ct * p.S * w.gg);
     w.total = off; off += align256(ct * p.S);
     w.tmp = off;   off += align256(ct);
-    w.ks = off;    off += align256(ks_bytes(c, level) * p.S * nib);   // all shards' key switches run side by side
+    // all shards' key switches run side by side; the baby steps take BABY_ROTS rotations per pass, which needs that
+    // many inner-product and conversion buffers per input ciphertext
+    const size_t knt = level + c->K;
+    w.ks = off;    off += align256(ks_bytes(c, level) * p.S * nib + (size_t)(BABY_ROTS - 1) * p.S * nib * (2 * knt + 2 * level) * c->N * sizeof(u64));
     // lazy giant steps: coefficient copies and extended digits of IP_TERMS giant steps of every shard
     const size_t kbeta = (level + c->alpha - 1) / c->alpha;
     w.ksx = off;   off += lazy ? align256((size_t)IP_TERMS * p.S * (level + kbeta * (level + c->K)) * c->N * sizeof(u64)) : 0;
@@ -822,12 +826,29 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
         launch_to_tiled(c, xin + comp * ptl, ctl, S * nib, baby, Rx, comp, 2 * B, level, s);
     if (B > 1) {
         ks_modup(c, xin + ptl, level, kw, s, S * nib, ctl);
-        for (uint32_t b = 1; b < B; b++) {
-            const u64 ge = ckks_galois_element(c, (int64_t)b * T);
+        // N = 2^16: BABY_ROTS rotations of all inputs per pass (the digits of a limb are fetched once for all of them and
+        // the launches are four times larger); the inner-product and conversion buffers follow the digits
+        const uint32_t rots = c->log_n == 16 ? BABY_ROTS : 1;       // the grouped ModDown tail exists for N = 2^16 only
+        KsWorkspace kb = kw;
+        kb.u = kw.ext + (size_t)S * nib * kbeta * knt * N;
+        kb.conv = kb.u + (size_t)rots * S * nib * 2 * knt * N;
+        for (uint32_t b = 1; b < B; b += rots) {
+            const uint32_t nr = std::min(rots, B - b);
             TiledOut to;
             to.R = Rx; to.row0 = 2 * b; to.row_stride = 2 * B;
-            ks_inner_moddown(c, (const u64 *)find_key(keys, nkeys, ge)->data, level, ge, kw, xin, nullptr, ge, baby, s, S * nib, ctl, 0,
-                             false, to);
+            if (rots == 1) {
+                const u64 ge = ckks_galois_element(c, (int64_t)b * T);
+                ks_inner_moddown(c, (const u64 *)find_key(keys, nkeys, ge)->data, level, ge, kw, xin, nullptr, ge, baby, s, S * nib, ctl, 0,
+                                 false, to);
+                continue;
+            }
+            KsMulti m{};
+            m.group = S * nib; m.rot_rows = 2;
+            for (uint32_t r = 0; r < nr; r++) {
+                m.galois[r] = ckks_galois_element(c, (int64_t)(b + r) * T);
+                m.evk[r] = (const u64 *)find_key(keys, nkeys, m.galois[r])->data;
+            }
+            ks_inner_moddown(c, nullptr, level, 1, kb, xin, nullptr, 1, baby, s, nr * S * nib, ctl, 0, false, to, &m);
         }
     }
 

@@ -205,6 +205,10 @@ struct KsMulti {
     const u64 *evk[KS_MULTI];
     u64 galois[KS_MULTI];
     u64 *out[KS_MULTI];
+    // group > 0 (N = 2^16 only): `group` ciphertexts with their own digits take every one of the keys; batch entry
+    // b = r * group + m is key r applied to member m's digits, added to member m's addend, and written to the tiled
+    // row  row0 + r * rot_rows + m * row_stride + component  (out[] is not used)
+    uint32_t group, rot_rows;
 };
 
 struct NttEpilogue {
@@ -219,6 +223,7 @@ struct NttEpilogue {
     int multi;             // mode 1: batch entry b adds through mgalois[b] and writes to mout[b]
     u64 mgalois[KS_MULTI];
     u64 *mout[KS_MULTI];
+    uint32_t group, rot_rows;   // KsMulti's grouped form
 };
 // coef_src (forward, N = 2^16 path only): the first pass reads signed 64-bit coefficients [batch][N] (batch = limb
 // index / map.period) and reduces them modulo the limb's prime on the fly instead of reading `base`.

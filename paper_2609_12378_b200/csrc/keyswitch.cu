@@ -135,12 +135,19 @@ __global__ void __launch_bounds__(THREADS) inner_product_kernel(DevTables c, con
                                                                 uint32_t level, uint32_t nb, uint32_t bch, int has_multi, KsMulti multi,
                                                                 int acc_u) {
     const uint32_t p = (blockIdx.x * THREADS + threadIdx.x) * 2;
-    const uint32_t x = blockIdx.z, b0 = blockIdx.y * bch, b1 = min(b0 + bch, nb);     // chunks of a limb run together: its key words come from L2
+    const uint32_t x = blockIdx.z;     // chunks of a limb run together: its key words (and shared digits) come from L2
+    uint32_t b0 = blockIdx.y * bch, b1 = min(b0 + bch, nb), e0 = has_multi ? 0 : b0;      // entries; first digits entry
     const uint32_t nt = level + c.K;
     const uint32_t kt = x < level ? x : c.L + (x - level);
     const double2 md = c.modd[kt];
     const size_t js = (size_t)nt * c.N, ks = (size_t)c.T * c.N;
-    if (has_multi) { evk = multi.evk[b0]; g = multi.galois[b0]; }
+    if (has_multi && multi.group) {     // key r on a chunk of the group's members
+        const uint32_t cpr = (multi.group + bch - 1) / bch, r = blockIdx.y / cpr, ch = blockIdx.y % cpr;
+        e0 = ch * bch;
+        b0 = r * multi.group + e0;
+        b1 = min(b0 + bch, (r + 1) * multi.group);
+        evk = multi.evk[r]; g = multi.galois[r];
+    } else if (has_multi) { evk = multi.evk[b0]; g = multi.galois[b0]; }
     const uint32_t src = galois_src(p, g, c.log_n, c.N);
     const bool odd = src & 1;
     double k[BETA][2][2];                         // [digit][component][coefficient of the pair]
@@ -152,7 +159,7 @@ __global__ void __launch_bounds__(THREADS) inner_product_kernel(DevTables c, con
             k[j][cm][0] = u64_to_d(v.x);
             k[j][cm][1] = u64_to_d(v.y);
         }
-    const u64 *e = ext + (has_multi ? 0 : b0 * BETA * js) + (size_t)x * c.N + (src & ~1u);
+    const u64 *e = ext + e0 * BETA * js + (size_t)x * c.N + (src & ~1u);
     u64 *o = u + b0 * 2 * js + (size_t)x * c.N + p;
     for (uint32_t b = b0; b < b1; b++, e += BETA * js, o += 2 * js) {
         double acc[2][2] = {{0.0, 0.0}, {0.0, 0.0}};
@@ -418,12 +425,22 @@ void ks_inner(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext_galois,
     const uint32_t beta = (level + c->alpha - 1) / c->alpha;
     const int au = acc_u ? 1 : 0;
     bool aligned = ((uintptr_t)w.ext & 15) == 0 && ((uintptr_t)w.u & 15) == 0 && (multi || ((uintptr_t)evk & 15) == 0);
-    if (multi)
-        for (uint32_t b = 0; b < nb; b++) aligned = aligned && ((uintptr_t)multi->evk[b] & 15) == 0;
-    if (beta <= IP_MAX_BETA && N >= 2 * THREADS && aligned) {
+    const uint32_t nkeys = multi ? (multi->group ? nb / multi->group : nb) : 0;
+    for (uint32_t b = 0; b < nkeys; b++) aligned = aligned && ((uintptr_t)multi->evk[b] & 15) == 0;
+    const bool fast = beta <= IP_MAX_BETA && N >= 2 * THREADS && aligned;
+    if (multi && multi->group && !fast) {       // grouped entries without the fast kernel: one key at a time
+        for (uint32_t r = 0; r < nkeys; r++) {
+            KsWorkspace wr = w;
+            wr.u = w.u + (size_t)r * multi->group * 2 * nt * N;
+            ks_inner(c, multi->evk[r], level, multi->galois[r], wr, s, multi->group, acc_u, nullptr);
+        }
+        return;
+    }
+    if (fast) {
         // batch entries per thread: enough chunks left to fill the machine, key words reused across a chunk
-        const uint32_t bch = multi ? 1 : (nb >= 8 ? 4 : (nb >= 4 ? 2 : 1));
-        const dim3 grid(N / (2 * THREADS), (nb + bch - 1) / bch, nt);
+        const uint32_t grp = multi ? multi->group : 0, per = grp ? grp : nb;
+        const uint32_t bch = (multi && !grp) ? 1 : (per >= 8 ? 4 : (per >= 4 ? 2 : 1));
+        const dim3 grid(N / (2 * THREADS), grp ? (nb / grp) * ((grp + bch - 1) / bch) : (nb + bch - 1) / bch, nt);
         const KsMulti m = multi ? *multi : KsMulti{};
         switch (beta) {
         case 1: inner_product_kernel<1><<<grid, THREADS, 0, s>>>(c->dev, w.ext, evk, ext_galois, w.u, level, nb, bch, multi ? 1 : 0, m, au); break;
@@ -449,6 +466,8 @@ void ks_moddown(const ckks_ctx *c, uint32_t level, const KsWorkspace &w, const u
     if (c->log_n == 16) {      // the last NTT pass finishes the ModDown itself
         NttEpilogue ep{1, w.u, add0, add1, out, add_stride, out_stride, add_galois, level, nt, accumulate ? 1 : 0, tiled};
         ep.multi = multi ? 1 : 0;
+        ep.group = multi ? multi->group : 0;
+        ep.rot_rows = multi ? multi->rot_rows : 0;
         if (multi)
             for (uint32_t b = 0; b < KS_MULTI; b++) { ep.mgalois[b] = multi->galois[b]; ep.mout[b] = multi->out[b]; }
         launch_ntt(c, w.conv, nb * 2 * level, plain_map(0, level), false, s, &ep);

@@ -383,8 +383,11 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 
             const uint32_t p0 = row * 256 + 16 * t;
             const u64 *up = ep.u + (((size_t)bz * 2 + comp) * ep.nt + i) * 65536 + p0;
             const u64 *add = comp ? ep.add1 : ep.add0;
-            const u64 gal = ep.multi ? ep.mgalois[bz] : ep.galois;
-            u64 *dst = ep.multi ? ep.mout[bz] + ((size_t)comp * ep.level + i) * 65536 + p0
+            // grouped: entry bz is key bz / group applied to member bz % group
+            const uint32_t rot = ep.group ? bz / ep.group : bz, mem = ep.group ? bz % ep.group : bz;
+            const u64 gal = ep.multi ? ep.mgalois[rot] : ep.galois;
+            u64 *dst = ep.group ? ep.out + tiled_index(ep.tl.R, 65536, ep.tl.row0 + rot * ep.rot_rows + mem * ep.tl.row_stride + comp, i, p0)
+                       : ep.multi ? ep.mout[bz] + ((size_t)comp * ep.level + i) * 65536 + p0
                        : ep.tl.R ? ep.out + tiled_index(ep.tl.R, 65536, ep.tl.row0 + bz * ep.tl.row_stride + comp, i, p0)
                                  : ep.out + bz * ep.out_stride + ((size_t)comp * ep.level + i) * 65536 + p0;
 #pragma unroll
@@ -396,7 +399,7 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 
                 for (uint32_t e = 0; e < 4; e++) {
                     // all on the FP64 pipe: |u - v| < 1.5 q, times P^-1 -> |.| < 0.9 q, plus up to two residues, reduced once
                     double v = mulmod_d<0>(__dsub_rn(u64_to_d(uu[e]), reduce_d(x[k + e], q, qinv)), pinv, q);
-                    if (add) v = __dadd_rn(v, u64_to_d(add[bz * ep.add_stride + (size_t)i * 65536 + galois_src(p0 + k + e, gal, 16, 65536)]));
+                    if (add) v = __dadd_rn(v, u64_to_d(add[mem * ep.add_stride + (size_t)i * 65536 + galois_src(p0 + k + e, gal, 16, 65536)]));
                     if (ep.accumulate) v = __dadd_rn(v, u64_to_d(old[e]));
                     r[e] = canonical_d(reduce_d(v, q, qinv), q);
                 }
