@@ -41,6 +41,13 @@ struct DevTables {
     const ulonglong2 *dn_p_inv;    // [L]      {P^-1 mod q_i, Shoup}
     const double2 *dn_p_inv_d;     // [L]      {P^-1 mod q_i, that / q_i} as doubles
     const double *dn_p_mod_d;      // [L]      P mod q_i as a double
+    // Tensor-core basis conversion (conv_mma.cu; conv_groups = 0 when alpha or K exceeds 8 sources): byte matrices of
+    // the conversion constants in the B-fragment order of mma.m16n8k32, [group of 8 targets][13 diagonals][2 k-steps]
+    // [lane][2] words; targets are the non-own limbs of the digit in ascending order (ModUp) or q_0.. (ModDown)
+    const uint32_t *up_bmat;       // [(L+1)][dnum][conv_groups][13][2][64]
+    const uint32_t *dn_bmat;       // [conv_groups][13][2][64]
+    const double2 *two52_d;        // [T] {2^52 mod prime, that / prime}
+    uint32_t conv_groups;
     // Rescale: [L(last)][L(i)] {q_last^-1 mod q_i, Shoup}
     const ulonglong2 *rs_inv;
     // Encode:
@@ -281,6 +288,11 @@ struct IpTerms {
 };
 void ks_inner_terms(const ckks_ctx *c, uint32_t level, const KsWorkspace &w, size_t term_stride, const IpTerms &terms, uint32_t nterm,
                     size_t c0_stride, cudaStream_t s, uint32_t nb, bool acc_u);
+// The basis conversions on the tensor cores (N = 2^16 layout rules: any N that is a multiple of 1024).  Return false if
+// the context has no byte matrices (more than 8 sources) and nothing was launched.
+bool launch_modup_mma(const ckks_ctx *c, const u64 *dcoef, const u64 *deval, size_t deval_stride, u64 *ext, uint32_t level, uint32_t nb,
+                      cudaStream_t s);
+bool launch_moddown_conv_mma(const ckks_ctx *c, const u64 *u, u64 *conv, uint32_t level, uint32_t nb, cudaStream_t s);
 // rows of [level][N] words, src_stride words apart, into rows row0, row0 + row_step, .. of a tiled buffer with R rows
 void launch_to_tiled(const ckks_ctx *c, const u64 *src, size_t src_stride, uint32_t nrows, u64 *dst, uint32_t R, uint32_t row0,
                      uint32_t row_step, uint32_t level, cudaStream_t s);

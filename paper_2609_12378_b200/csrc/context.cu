@@ -234,6 +234,58 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
         dn_pmod_d[i] = (double)Pm;
     }
 
+    // ---- Byte matrices for the tensor-core basis conversion.  Row k = 8 a + b of the k-dimension is byte b of source
+    // a's centred-lift word (b = 7: the "negative" flag); column (x, d) collects the byte products of weight 2^(8 d):
+    // byte d - b of the constant C[a][x] for b < 7, and byte d of (-q_a C[a][x]) mod t for the flag, so that the
+    // 13 diagonal sums recombine to sum_a centre(v_a) C[a][x] modulo t.
+    const uint32_t conv_groups = (alpha <= 8 && K <= 8) ? (L + K + 7) / 8 : 0;
+    const size_t gwords = 13 * 2 * 64;
+    auto fill_bmat = [&](uint32_t *out, uint32_t nsrc, uint32_t ntgt, auto &&konst) {
+        for (uint32_t gr = 0; gr < conv_groups; gr++)
+            for (uint32_t d = 0; d < 13; d++)
+                for (uint32_t ks = 0; ks < 2; ks++)
+                    for (uint32_t lane = 0; lane < 32; lane++)
+                        for (uint32_t half = 0; half < 2; half++) {
+                            const uint32_t n = lane >> 2, t = lane & 3, x = gr * 8 + n, a = ks * 4 + half * 2 + (t >> 1), bb = (t & 1) * 4;
+                            uint32_t word = 0;
+                            if (x < ntgt && a < nsrc) {
+                                u64 C, Kn;
+                                konst(a, x, C, Kn);
+                                for (uint32_t i = 0; i < 4; i++) {
+                                    const uint32_t b = bb + i;
+                                    uint32_t byte = 0;
+                                    if (b < 7) { if (d >= b && d - b <= 6) byte = (uint32_t)(C >> (8 * (d - b))) & 255u; }
+                                    else if (d <= 6) byte = (uint32_t)(Kn >> (8 * d)) & 255u;
+                                    word |= byte << (8 * i);
+                                }
+                            }
+                            out[((size_t)(gr * 13 + d) * 2 + ks) * 64 + lane * 2 + half] = word;
+                        }
+    };
+    std::vector<uint32_t> up_bmat((size_t)(L + 1) * dn * conv_groups * gwords, 0), dn_bmat((size_t)conv_groups * gwords, 0);
+    std::vector<double2> two52(T);
+    for (uint32_t t = 0; t < T; t++) {
+        const u64 v = (u64)(((u128)1 << 52) % mod[t]);
+        two52[t] = make_double2((double)v, (double)v / (double)mod[t]);
+    }
+    if (conv_groups) {
+        for (uint32_t lvl = 1; lvl <= L; lvl++)
+            for (uint32_t j = 0; j * alpha < lvl; j++) {
+                const uint32_t lo = j * alpha, hi = std::min(lo + alpha, lvl), nd = hi - lo, nt = lvl + K;
+                fill_bmat(up_bmat.data() + ((size_t)lvl * dn + j) * conv_groups * gwords, nd, nt - nd, [&](uint32_t a, uint32_t x, u64 &C, u64 &Kn) {
+                    const uint32_t xp = x < lo ? x : x + nd, t = xp < lvl ? xp : L + (xp - lvl);
+                    C = up_mod[(((size_t)lvl * dn + j) * alpha + a) * T + t];
+                    const u64 m = h_mul(mod[lo + a] % mod[t], C, mod[t]);
+                    Kn = m ? mod[t] - m : 0;
+                });
+            }
+        fill_bmat(dn_bmat.data(), K, L, [&](uint32_t a, uint32_t x, u64 &C, u64 &Kn) {
+            C = dn_mod[(size_t)x * K + a];
+            const u64 m = h_mul(mod[L + a] % mod[x], C, mod[x]);
+            Kn = m ? mod[x] - m : 0;
+        });
+    }
+
     // ---- Rescale constants
     std::vector<ulonglong2> rs((size_t)L * L, make_ulonglong2(0, 0));
     for (uint32_t last = 0; last < L; last++)
@@ -253,14 +305,14 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
     }
 
     DevTables &d = c->dev;
-    d.log_n = prm->log_n; d.N = N; d.L = L; d.K = K; d.alpha = alpha; d.T = T; d.dnum = prm->dnum;
+    d.conv_groups = conv_groups; d.log_n = prm->log_n; d.N = N; d.L = L; d.K = K; d.alpha = alpha; d.T = T; d.dnum = prm->dnum;
     int rc = CKKS_OK;
     std::vector<int> flag(2, 0);
     const int *flag_dev = nullptr;
     if ((rc = upload(c, mod, &d.mod)) || (rc = upload(c, mu, &d.mu)) || (rc = upload(c, mu64, &d.mu64)) || (rc = upload(c, modd, &d.modd)) || (rc = upload(c, twf, &d.tw_fwd)) ||
         (rc = upload(c, twi, &d.tw_inv)) || (rc = upload(c, twdf, &d.twd_fwd)) || (rc = upload(c, twdi, &d.twd_inv)) || (rc = upload(c, ninvd, &d.n_inv_d)) || (rc = upload(c, ninv, &d.n_inv)) || (rc = upload(c, up_inv, &d.up_hat_inv)) ||
         (rc = upload(c, up_mod, &d.up_hat_mod)) || (rc = upload(c, up_mod_d, &d.up_hat_mod_d)) || (rc = upload(c, dn_mod_d, &d.dn_hat_mod_d)) || (rc = upload(c, dn_inv, &d.dn_hat_inv)) ||
-        (rc = upload(c, dn_mod, &d.dn_hat_mod)) || (rc = upload(c, dn_pinv, &d.dn_p_inv)) || (rc = upload(c, dn_pinv_d, &d.dn_p_inv_d)) || (rc = upload(c, dn_pmod_d, &d.dn_p_mod_d)) || (rc = upload(c, rs, &d.rs_inv)) ||
+        (rc = upload(c, dn_mod, &d.dn_hat_mod)) || (rc = upload(c, dn_pinv, &d.dn_p_inv)) || (rc = upload(c, dn_pinv_d, &d.dn_p_inv_d)) || (rc = upload(c, dn_pmod_d, &d.dn_p_mod_d)) || (rc = upload(c, up_bmat, &d.up_bmat)) || (rc = upload(c, dn_bmat, &d.dn_bmat)) || (rc = upload(c, two52, &d.two52_d)) || (rc = upload(c, rs, &d.rs_inv)) ||
         (rc = upload(c, enc_src, &d.enc_src)) || (rc = upload(c, om, &d.enc_omega)) || (rc = upload(c, ze, &d.enc_zeta)) ||
         (rc = upload(c, flag, &flag_dev))) {
         cudaSetDevice(prev);

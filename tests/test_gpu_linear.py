@@ -100,6 +100,15 @@ def test_projection_tensor_core_mac_other_shapes(shape, monkeypatch):
     assert ctx.device_status() == 0
 
 
+def test_projection_with_tensor_core_basis_conversion(monkeypatch):
+    """ModUp's and ModDown's conversion matrices on the tensor cores (the CKKS_CONV=mma tuning knob): the same integers,
+    on a shape with a fold, several output blocks and a partial last digit."""
+    monkeypatch.setenv("CKKS_CONV", "mma")
+    ctx, _, _ = _run(10, 6, 2, 3, 5, 16, 24, 32, 2, 4, seed=455)
+    assert ctx.device_status() == 0
+    _run(10, 4, 2, 2, 4, 64, 160, 8, 3, 32, seed=456, lazy=True)
+
+
 def test_projection_multi_shares_baby_steps():
     """Three matrices on the same inputs (query/key/value-like: square, wide with fold, several output blocks):
     every output equals the checker's per-matrix result, and the shared call launches fewer kernels than three
