@@ -13,9 +13,9 @@
 // creation in the B-fragment order (context.cu).
 //
 // Status: opt-in (CKKS_CONV=mma).  On B200 it is no faster than the FP64 kernels (ModDown conversion of 16 entries:
-// 302 us against 258-290 us; 4096 x 4096 projection 300 ms against 293 ms): putting the 13 sums together costs about 70
-// instructions per output, the kernel issues on 45 % of its cycles with 16 warps per SM (120 registers), and the
-// tensor, FP64 and integer pipes each stay below 30 %.
+// 297 us against 258-290 us; 4096 x 4096 projection 299 ms against 293 ms): putting the 13 sums together and reducing
+// them costs about 50 instructions per output, the kernel issues on 45 % of its cycles with 16 warps per SM (122
+// registers), and the tensor, FP64 and integer pipes each stay below 30 %.
 #include "common.cuh"
 
 namespace {
@@ -27,6 +27,28 @@ __device__ __forceinline__ void mma_u8(int (&d)[4], const uint32_t (&a)[4], uint
     asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
                  : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// sum_q E_q 2^(16 q), q < 7, E_q < 2^31, as four 32-bit words (the value stays below 2^103)
+__device__ __forceinline__ void assemble7(const uint32_t (&E)[7], uint32_t &w0, uint32_t &w1, uint32_t &w2, uint32_t &w3) {
+    asm("{\n"
+        ".reg .u32 a1, b1, t1, a3, b3, t2, a5, b5, t3;\n"
+        "shl.b32 a1, %5, 16;\n"
+        "shr.u32 b1, %5, 16;\n"
+        "add.u32 t1, b1, %6;\n"
+        "shl.b32 a3, %7, 16;\n"
+        "shr.u32 b3, %7, 16;\n"
+        "add.u32 t2, b3, %8;\n"
+        "shl.b32 a5, %9, 16;\n"
+        "shr.u32 b5, %9, 16;\n"
+        "add.u32 t3, b5, %10;\n"
+        "add.cc.u32 %0, %4, a1;\n"
+        "addc.cc.u32 %1, t1, a3;\n"
+        "addc.cc.u32 %2, t2, a5;\n"
+        "addc.u32 %3, t3, 0;\n"
+        "}\n"
+        : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3)
+        : "r"(E[0]), "r"(E[1]), "r"(E[2]), "r"(E[3]), "r"(E[4]), "r"(E[5]), "r"(E[6]));
 }
 
 // MODE 0: ModUp.   item = (batch b, digit j); sources dcoef[b][lo + a]; targets the limbs of ext[b][j] outside the digit.
@@ -100,6 +122,12 @@ __global__ void __launch_bounds__(CM_THREADS, 2) conv_mma_kernel(DevTables c, co
     const bool hi_half = t & 1;
     const uint2 *bs2 = reinterpret_cast<const uint2 *>(bs);
 
+    // the source words of a tile are fetched while the tile before it is converted
+    u64 nxt[2][2];
+#pragma unroll
+    for (uint32_t i = 0; i < 2; i++)
+#pragma unroll
+        for (uint32_t r = 0; r < 2; r++) nxt[i][r] = qa[i] ? sbase[(size_t)(4 * i + t) * N + kcta + warp * 16 + g + 8 * r] : 0;
     for (uint32_t tile = 0; tile < CM_TILES; tile++) {
         const uint32_t k0 = kcta + tile * 128 + warp * 16;
         uint32_t wlo[2][2], whi[2][2];
@@ -109,8 +137,9 @@ __global__ void __launch_bounds__(CM_THREADS, 2) conv_mma_kernel(DevTables c, co
             for (uint32_t r = 0; r < 2; r++) {
                 u64 wd = 0;
                 if (qa[i]) {
-                    const u64 v = mul_shoup(sbase[(size_t)(4 * i + t) * N + k0 + g + 8 * r], hv[i].x, hv[i].y, qa[i]);
+                    const u64 v = mul_shoup(nxt[i][r], hv[i].x, hv[i].y, qa[i]);
                     wd = v | ((u64)(v > (qa[i] >> 1)) << 56);
+                    if (tile + 1 < CM_TILES) nxt[i][r] = sbase[(size_t)(4 * i + t) * N + k0 + 128 + g + 8 * r];
                 }
                 wlo[i][r] = (uint32_t)wd;
                 whi[i][r] = (uint32_t)(wd >> 32);
@@ -148,12 +177,11 @@ __global__ void __launch_bounds__(CM_THREADS, 2) conv_mma_kernel(DevTables c, co
 #pragma unroll
                 for (uint32_t q = 0; q < 6; q++) E[q] = (uint32_t)acc[2 * q][o] + ((uint32_t)acc[2 * q + 1][o] << 8);
                 E[6] = (uint32_t)acc[12][o];
-                const u64 A = (u64)E[0] + ((u64)E[1] << 16) + ((u64)E[2] << 32);
-                const u64 B = (u64)E[3] + ((u64)E[4] << 16) + ((u64)E[5] << 32);
-                const u64 vlo = A + (B << 48);
-                const u64 vhi = (B >> 16) + ((u64)E[6] << 32) + (vlo < A ? 1 : 0);
-                const double dlo = u64_to_d(vlo & 0x000FFFFFFFFFFFFFull);
-                const double dhi = u64_to_d((vlo >> 52) | (vhi << 12));          // below 2^51
+                uint32_t w0, w1, w2, w3;
+                assemble7(E, w0, w1, w2, w3);
+                // split at bit 52; both parts go into the mantissa of 2^52 (an integer below 2^52 each)
+                const double dlo = __dsub_rn(__hiloint2double((int)((w1 & 0x000FFFFFu) | 0x43300000u), (int)w0), TWO52);
+                const double dhi = __dsub_rn(__hiloint2double((int)(__funnelshift_r(w2, w3, 20) | 0x43300000u), (int)__funnelshift_r(w1, w2, 20)), TWO52);
                 const double r = __dadd_rn(mulmod_d<0>(dhi, c52, md.x), reduce_d(dlo, md.x, md.y));
                 const u64 res = canonical_d(reduce_d(r, md.x, md.y), md.x);
                 if (limb != 0xffffffffu) dbase[(size_t)limb * N + k0 + g + 8 * (o >> 1)] = res;

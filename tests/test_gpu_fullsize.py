@@ -102,7 +102,7 @@ def test_sixty_four_rotations_full_size():
         assert np.abs(zp - want).max() < 2.0 ** -17 and np.abs(zh - want).max() < 2.0 ** -17, i
 
 
-def _full_ring_shape(d_in, d_out, S, B, seed, shards_checked=1):
+def _full_ring_shape(d_in, d_out, S, B, seed, shards_checked=1, lazy=False):
     """A decoder-layer projection shape at N = 2^16, level 24: decrypt everything, recompute `shards_checked` shards."""
     from tests.gpu_util import context, ct_dev, dev, host, key_dev
     P, ctx = params(16, 24, 8, 3), context(16, 24, 8, 3)
@@ -112,7 +112,7 @@ def _full_ring_shape(d_in, d_out, S, B, seed, shards_checked=1):
     g = inputs.rng(seed, 1)
     X = inputs.activations_normal(g, S * T, d_in)
     W = inputs.weights_normal(g, d_in, d_out, 0.02)
-    desc = ProjDesc(d_in, d_out, T, S, B)
+    desc = ProjDesc(d_in, d_out, T, S, B, lazy_moddown=lazy)
     F, ins, outs_b = o.proj_blocks(desc)
     rots = o.proj_rotations(desc)
     assert rots == ctx.linear_proj_rotations(d_in, d_out, T, S, B)
@@ -121,7 +121,8 @@ def _full_ring_shape(d_in, d_out, S, B, seed, shards_checked=1):
         for (s0, mi) in ins:
             cts.append(cl.encrypt_slots(inputs.pack_feature_major(X[c * T:(c + 1) * T, s0:s0 + mi], T, o.n)[0], scale, level))
     keys = {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in rots}
-    outs = ctx.linear_proj([ct_dev(c, scale) for c in cts], dev(W), [key_dev(k, ge) for ge, k in keys.items()], d_in, d_out, T, S, B)
+    outs = ctx.linear_proj([ct_dev(c, scale) for c in cts], dev(W), [key_dev(k, ge) for ge, k in keys.items()], d_in, d_out, T, S, B,
+                           lazy_moddown=lazy)
     assert ctx.device_status() == binding.OK
     Y = X @ W
     nib, nob = len(ins), len(outs_b)
@@ -132,15 +133,15 @@ def _full_ring_shape(d_in, d_out, S, B, seed, shards_checked=1):
             for r in range(0, F, 37):
                 assert np.abs(sl[r] - Y[c * T:(c + 1) * T, o0 + r % mo]).max() < 2.0 ** -16, (c, ob, r)
     for c in range(shards_checked):
-        one = ProjDesc(d_in, d_out, T, 1, B)
+        one = ProjDesc(d_in, d_out, T, 1, B, lazy_moddown=lazy)
         want, _ = o.linear_proj(one, np.stack(cts[c * nib:(c + 1) * nib]), W, keys, scale)
         for ob in range(nob):
             assert np.array_equal(got[c * nob + ob], want[ob]), (c, ob)
 
 
 def test_kv_projection_full_ring():
-    """K / V shape: 4096 -> 1024 (wide block, folded twice), B = G = 32."""
-    _full_ring_shape(4096, 1024, 4, 32, seed=1005)
+    """K / V shape: 4096 -> 1024 (wide block, folded twice), B = G = 32, giant steps summed before one ModDown."""
+    _full_ring_shape(4096, 1024, 4, 32, seed=1005, lazy=True)
 
 
 import os  # noqa: E402
@@ -158,4 +159,4 @@ def test_gate_up_projection_full_ring():
 @heavy
 def test_down_projection_full_ring():
     """down shape: 14336 -> 4096 (three full input blocks and a repeated remainder block summed before the giant steps)."""
-    _full_ring_shape(14336, 4096, 2, 64, seed=1007)
+    _full_ring_shape(14336, 4096, 2, 64, seed=1007, lazy=True)
