@@ -372,6 +372,9 @@ def run_cuda(args):
                 "fp64_pipe_active_ncu": {"ntt16_fwd_cols": 0.761, "ntt16_fwd_rows": 0.677},
                 "peak_kind": "derived: 64 DFMA/clk/SM x %d SMs x %.0f MHz" % (sm_count, float(pk.get("sm_max_mhz", 1965.0))),
                 "ms_per_launch_pair": ntt_fwd_ms,
+                # the same fraction against the clock the SMs held under the power cap during the timed steps
+                "frac_at_sampled_clock": (achieved / (fp64_peak * float(clocks["sm_mhz"]) / float(pk.get("sm_max_mhz", 1965.0)))
+                                          if clocks and clocks.get("sm_mhz") else None),
                 "vs_register_resident_butterflies": {
                     "achieved_gbfly_s": limb_ntts * (N // 2) * LOG_N / (ntt_fwd_ms * 1e-3) / 1e9, "peak_gbfly_s": probe_rate / 1e9,
                     "frac": limb_ntts * (N // 2) * LOG_N / (ntt_fwd_ms * 1e-3) / probe_rate,
