@@ -84,6 +84,15 @@ def test_projection_lazy_moddown(d_in, d_out, T, S, B):
     _run(10, 4, 2, 2, 4, d_in, d_out, T, S, B, seed=480 + d_in + d_out, lazy=True)
 
 
+@pytest.mark.parametrize("log_n,L,K,dnum,level,d_in,d_out,T,S,B", [
+    (10, 6, 2, 3, 5, 16, 16, 32, 2, 4),     # level below L, partial last digit
+    (13, 6, 1, 6, 6, 64, 64, 32, 3, 8),     # six digits: the any-number-of-digits inner product, three shards
+    (10, 4, 1, 4, 3, 16, 4, 32, 2, 2),      # one special prime, fold after the lazy sum
+])
+def test_projection_lazy_moddown_other_parameters(log_n, L, K, dnum, level, d_in, d_out, T, S, B):
+    _run(log_n, L, K, dnum, level, d_in, d_out, T, S, B, seed=485 + log_n + dnum, lazy=True)
+
+
 def test_projection_lazy_moddown_many_groups():
     """More giant steps than one group of accumulators holds (32 > 16): the running sum survives the next group's
     encode and multiply-accumulate."""
