@@ -280,6 +280,38 @@ class Oracle:
         so = T / float(self.q[Lt - 1])
         return self.add_const(out, int(np.rint(coeffs[0] * so))), so
 
+    def softmax_doubling(self, x, scale: float, shift: float, rounds: int, row_len: int, exp_coeffs, rsqrt_coeffs, rlk, keys: dict):
+        """Softmax by doubling with a public shift (Algorithm 1) on one ciphertext of score rows.  Row r holds its
+        row_len scores in slots i * (n / row_len) + r, so that rotations by (n / row_len) 2^i, i < log2 row_len,
+        add up a whole row in every one of its slots.  exp_coeffs: the polynomial p_exp(z / 2^k) as a polynomial in z;
+        rsqrt_coeffs[j]: round j's inverse-square-root polynomial.  Order of steps:
+          z = x + round(-shift * scale);  u = poly_eval_tree(z, exp_coeffs);
+          per round: sq = rescale(mul_relin(u, u));  s = sq, then s = s + rotate(s, (n / row_len) 2^i) for i = 0, 1, ..;
+                     lam = poly_eval_tree(s, rsqrt_coeffs[j]);  v = rescale(mul_relin(lam, u truncated to lam's level));
+                     u = rescale(mul_relin(v, v)).
+        Scales are doubles, multiplied and divided in this order.  keys maps a Galois element to its key.
+        Returns (ct, scale)."""
+        x = _u64(x)
+        stride = self.n // row_len
+        if row_len < 2 or row_len & (row_len - 1) or self.n % row_len:
+            raise ValueError("row_len must be a power of two dividing the slot count")
+        z = self.add_const(x, int(np.rint(-shift * scale)))
+        u, su = self.poly_eval_tree(z, scale, exp_coeffs, rlk)
+        for j in range(rounds):
+            lv = u.shape[1]
+            sq = self.rescale(self.mul_relin(u, u, rlk)); ss = su * su / float(self.q[lv - 1])
+            s = sq
+            i = 1
+            while i < row_len:
+                ge = self.galois_element(stride * i)
+                s = self.add(s, self.rotate(s, keys[ge], ge))
+                i *= 2
+            lam, sl = self.poly_eval_tree(s, ss, rsqrt_coeffs[j], rlk)
+            ll = lam.shape[1]
+            v = self.rescale(self.mul_relin(lam, u[:, :ll], rlk)); sv = sl * su / float(self.q[ll - 1])
+            u = self.rescale(self.mul_relin(v, v, rlk)); su = sv * sv / float(self.q[ll - 2])
+        return u, su
+
     def automorphism_coeff(self, a, g: int, t: int):
         a = _u64(a); out = np.empty_like(a)
         lib().orc_automorphism_coeff(self._h, C.c_uint32(t), _p(a, _u64p), C.c_uint64(g), _p(out, _u64p))

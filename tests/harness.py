@@ -96,3 +96,44 @@ def negacyclic_schoolbook(a, b, q):
 
 def brev(x, bits):
     return int(format(x, "0%db" % bits)[::-1], 2) if bits else 0
+
+
+# ------------------------------------------------------------ Softmax by doubling (Algorithm 1), synthetic case
+
+def softmax_case(P: Params, seed: int, row_len: int = 16, rounds: int = 2, degree: int = 4, spread: float = 11.0):
+    """Scores in [shift - spread, shift] laid out row by row with stride n / row_len, polynomial fits of exp on
+    [-spread / 2^rounds, 0] and of 1 / sqrt on the measured range of every round's row sums (times a safety factor),
+    and the same pipeline evaluated in the clear.  Returns (slots, shift, exp_coeffs_in_z, rsqrt_coeffs, clear_result,
+    true_softmax), all per slot."""
+    n, stride = P.n, P.n // row_len
+    g = inputs.rng(seed, 7)
+    shift = 3.0
+    rows = shift - spread * g.uniform(0.0, 1.0, (stride, row_len)) ** 2      # row r, element i
+    rows[:, 0] = shift - 0.25                                                # one score near the top of every row
+    x = np.empty(n)
+    for i in range(row_len):
+        x[i * stride:(i + 1) * stride] = rows[:, i]
+
+    def fit(f, lo, hi, deg):
+        t = np.cos(np.pi * (np.arange(64) + 0.5) / 64) * (hi - lo) / 2 + (hi + lo) / 2
+        return np.polynomial.polynomial.polyfit(t, f(t), deg)
+
+    ce = fit(np.exp, -spread / 2 ** rounds, 0.0, degree)
+    exp_in_z = ce / (2.0 ** rounds) ** np.arange(degree + 1)                 # p_exp(z / 2^k) as a polynomial in z
+    pv = np.polynomial.polynomial.polyval
+    u = pv(rows - shift, exp_in_z)
+    rs = []
+    for _ in range(rounds):
+        s = (u * u).sum(1)
+        c = fit(lambda t: 1.0 / np.sqrt(t), s.min() / 1.3, s.max() * 1.3, degree)
+        rs.append(c)
+        u = (pv(s, c)[:, None] * u) ** 2
+    clear = np.empty(n)
+    for i in range(row_len):
+        clear[i * stride:(i + 1) * stride] = u[:, i]
+    e = np.exp(rows - rows.max(1, keepdims=True))
+    true = e / e.sum(1, keepdims=True)
+    truth = np.empty(n)
+    for i in range(row_len):
+        truth[i * stride:(i + 1) * stride] = true[:, i]
+    return x, shift, exp_in_z, np.stack(rs), clear, truth
