@@ -324,6 +324,12 @@ def run_cuda(args):
         extras["rotate_64_calls_ms"] = once(lambda: [ctx.rotate(x_, rot_keys[0], out=rot_out) for x_ in rin])
         extras["rotate_batch_64_ms"] = once(lambda: ctx.rotate_batch(rin, rot_keys[0], outs=routs, ws=rws))
         del routs, rws
+        # Softmax by doubling on 256 rows of 128 scores (one ciphertext), two rounds, degree-4 polynomials: 7 + 2 x 11 products,
+        # 14 rotations
+        sm_keys = [keys[256 << i] for i in range(7)]
+        sm_in = binding.Ciphertext(cta.data, 2.0 ** 50)
+        poly = [1.0, 0.25, 0.03, 0.002, 0.0001]
+        extras["softmax_256x128_two_rounds_ms"] = once(lambda: ctx.softmax(sm_in, 3.0, 2, 128, poly, [poly, poly], rlk, sm_keys))
         del Wk, Wv
 
     # e2e: host buffers in, host buffers out, copies inside the timed region

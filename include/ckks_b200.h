@@ -238,6 +238,27 @@ int32_t ckks_poly_eval(ckks_ctx *ctx, const ckks_ct *x, const double *coeffs, ui
 int32_t ckks_poly_eval_tree(ckks_ctx *ctx, const ckks_ct *x, const double *coeffs, uint32_t degree, const ckks_evk *rlk, ckks_ct *out,
                             void *ws, size_t ws_bytes, void *stream);
 
+/* ---- Softmax by doubling with a public shift (Algorithm 1) --------------------
+ * One ciphertext of score rows: row r holds its row_len scores (a power of two dividing n) in slots
+ * i * (n / row_len) + r, so that rotations by (n / row_len) 2^i, i < log2 row_len, leave a row's sum in every one of its
+ * slots (keys for these rotations must be among `keys`).  exp_coeffs (host, exp_degree + 1 values, degree >= 2): the
+ * polynomial p_exp(z / 2^rounds) written as a polynomial in z = x - shift; rsqrt_coeffs (host, rounds x
+ * (rsqrt_degree + 1) values): round j's inverse-square-root polynomial.  Steps, all on the device:
+ *   z = x - shift;  u = p_exp(z);  per round: s = row sums of u^2;  lambda = p_rsqrt_j(s);  u = (lambda u)^2,
+ * every product followed by a rescale, both polynomials evaluated as ckks_poly_eval_tree does.  No bootstrapping:
+ * the input needs (d_e + 1) + rounds * (d_r + 4) limbs more than the output keeps, d = ceil(log2 degree).  Scores should
+ * be encrypted at a scale near the primes.  out: level and scale as they come out.  Workspace:
+ * ckks_softmax_workspace_bytes.  Errors: ARG, LEVEL, NO_KEY, RANGE (a constant beyond 2^62), WORKSPACE. */
+typedef struct {
+    double shift;
+    uint32_t rounds, row_len, exp_degree, rsqrt_degree;
+    const double *exp_coeffs;   /* host */
+    const double *rsqrt_coeffs; /* host */
+} ckks_softmax_desc;
+int32_t ckks_softmax(ckks_ctx *ctx, const ckks_softmax_desc *desc, const ckks_ct *in, const ckks_evk *rlk, const ckks_evk *keys,
+                     uint32_t nkeys, ckks_ct *out, void *ws, size_t ws_bytes, void *stream);
+size_t ckks_softmax_workspace_bytes(const ckks_ctx *ctx, const ckks_softmax_desc *desc, uint32_t level);
+
 /* ---- Rot_k (Section 2.1, Rot + KeySwitch) ----------------------------------
  * Plain: apply sigma_g (g = key->galois) to both components, key-switch the
  * permuted c1: out = (sigma c0 + k0, k1).  Key switch = iNTT, centred ModUp

@@ -23,7 +23,7 @@ EXPORTS = [
     "ckks_encode_range_flag", "ckks_mul_plain_acc", "ckks_add", "ckks_mul_relin", "ckks_rotate",
     "ckks_rotate_hoisted", "ckks_rescale", "ckks_linear_proj", "ckks_linear_proj_workspace_bytes",
     "ckks_linear_proj_rotations", "ckks_kernel_launches", "ckks_device_status", "ckks_rescale_static",
-    "ckks_ntt_butterfly_probe", "ckks_mul_relin_sum", "ckks_mul_relin_batch", "ckks_rotate_batch", "ckks_rotate_sum", "ckks_mul_const", "ckks_add_const", "ckks_poly_eval", "ckks_poly_eval_tree", "ckks_linear_proj_multi", "ckks_linear_proj_multi_workspace_bytes",
+    "ckks_ntt_butterfly_probe", "ckks_mul_relin_sum", "ckks_mul_relin_batch", "ckks_rotate_batch", "ckks_rotate_sum", "ckks_softmax", "ckks_softmax_workspace_bytes", "ckks_mul_const", "ckks_add_const", "ckks_poly_eval", "ckks_poly_eval_tree", "ckks_linear_proj_multi", "ckks_linear_proj_multi_workspace_bytes",
 ]
 
 
@@ -42,6 +42,11 @@ class CPt(C.Structure):
 
 class CEvk(C.Structure):
     _fields_ = [("data", C.c_void_p), ("galois", C.c_uint64)]
+
+
+class CSoftmaxDesc(C.Structure):
+    _fields_ = [("shift", C.c_double), ("rounds", C.c_uint32), ("row_len", C.c_uint32), ("exp_degree", C.c_uint32),
+                ("rsqrt_degree", C.c_uint32), ("exp_coeffs", C.POINTER(C.c_double)), ("rsqrt_coeffs", C.POINTER(C.c_double))]
 
 
 class CProjDesc(C.Structure):
@@ -77,6 +82,8 @@ def load():
         "ckks_mul_plain_acc": (i32, [vp, C.POINTER(CCt), u32, C.POINTER(CPt), C.POINTER(CCt), i32, vp]),
         "ckks_add": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), C.POINTER(CCt), vp]),
         "ckks_mul_relin": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
+        "ckks_softmax": (i32, [vp, C.POINTER(CSoftmaxDesc), C.POINTER(CCt), C.POINTER(CEvk), C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
+        "ckks_softmax_workspace_bytes": (sz, [vp, C.POINTER(CSoftmaxDesc), u32]),
         "ckks_rotate_sum": (i32, [vp, C.POINTER(CCt), C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
         "ckks_rotate_batch": (i32, [vp, C.POINTER(CCt), u32, C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
         "ckks_mul_relin_batch": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), u32, C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
@@ -328,6 +335,30 @@ class Context:
                                                _stream_ptr(stream)))
         out.scale = co.scale
         return out
+
+    def softmax(self, ct: Ciphertext, shift: float, rounds: int, row_len: int, exp_coeffs, rsqrt_coeffs, rlk: SwitchKey, keys,
+                ws: torch.Tensor = None, stream=None):
+        """Softmax by doubling with a public shift on one ciphertext of score rows (row r in slots i * (n / row_len) + r).
+        exp_coeffs: p_exp(z / 2^rounds) as a polynomial in z; rsqrt_coeffs: [rounds][degree + 1]."""
+        ec = (C.c_double * len(exp_coeffs))(*[float(v) for v in exp_coeffs])
+        flat = [float(v) for row in rsqrt_coeffs for v in row]
+        rc = (C.c_double * max(1, len(flat)))(*flat)
+        rdeg = (len(rsqrt_coeffs[0]) - 1) if rounds else 0
+        d = CSoftmaxDesc(float(shift), rounds, row_len, len(exp_coeffs) - 1, rdeg, C.cast(ec, C.POINTER(C.c_double)),
+                         C.cast(rc, C.POINTER(C.c_double)))
+        need = int(load().ckks_softmax_workspace_bytes(self._h, C.byref(d), ct.level))
+        if need == 0:
+            raise CkksError(ERR_ARG)
+        if ws is None:
+            ws = self.workspace(need)
+        out = self.empty_ct(ct.level)
+        ci, co = _cct(ct), _cct(out)
+        crlk = CEvk(_dev_u64(rlk.data).data_ptr(), 0)
+        ka = (CEvk * max(1, len(keys)))(*[CEvk(_dev_u64(k.data).data_ptr(), k.galois) for k in keys])
+        self._check(load().ckks_softmax(self._h, C.byref(d), C.byref(ci), C.byref(crlk), ka, len(keys), C.byref(co), ws.data_ptr(), ws.numel(),
+                                        _stream_ptr(stream)))
+        res = Ciphertext(out.data.view(-1)[: 2 * co.level * self.N].view(2, co.level, self.N), co.scale)
+        return res
 
     def rotate_sum(self, cts, keys, out: Ciphertext = None, ws: torch.Tensor = None, stream=None):
         """sum_i rotate(cts[i], keys[i]) formed in the key-switching basis and divided by P once."""

@@ -605,6 +605,81 @@ extern "C" int32_t ckks_poly_eval_tree(ckks_ctx *c, const ckks_ct *x, const doub
     return rc;
 }
 
+// ---- Softmax by doubling (Algorithm 1): a composition of the entry points above on buffers carved from the workspace
+static uint32_t log2_ceil(uint32_t x) { uint32_t d = 0; while ((1u << d) < x) d++; return d; }
+static size_t softmax_scratch_bytes(const ckks_ctx *c, const ckks_softmax_desc *d, uint32_t level) {
+    const uint32_t deg = std::max(d->exp_degree, d->rsqrt_degree);
+    return align256(std::max(ckks_workspace_bytes(c, CKKS_OP_POLY_EVAL_TREE, level, deg),
+                             std::max(ckks_workspace_bytes(c, CKKS_OP_MUL_RELIN, level, 0), ckks_workspace_bytes(c, CKKS_OP_RESCALE, level, 0))));
+}
+static bool softmax_desc_ok(const ckks_ctx *c, const ckks_softmax_desc *d) {
+    return d && d->exp_coeffs && d->exp_degree >= 2 && (d->rounds == 0 || (d->rsqrt_coeffs && d->rsqrt_degree >= 2)) && d->row_len >= 2 &&
+           !(d->row_len & (d->row_len - 1)) && c->n % d->row_len == 0;
+}
+
+extern "C" size_t ckks_softmax_workspace_bytes(const ckks_ctx *c, const ckks_softmax_desc *d, uint32_t level) {
+    if (!c || !softmax_desc_ok(c, d) || !level_ok(c, level)) return 0;
+    return 4 * align256((size_t)2 * level * c->N * sizeof(u64)) + softmax_scratch_bytes(c, d, level);
+}
+
+extern "C" int32_t ckks_softmax(ckks_ctx *c, const ckks_softmax_desc *d, const ckks_ct *in, const ckks_evk *rlk, const ckks_evk *keys,
+                                uint32_t nkeys, ckks_ct *out, void *ws, size_t ws_bytes, void *stream) {
+    if (!c || !softmax_desc_ok(c, d) || !ct_ok(in) || !ct_ok(out) || in->ncomp != 2) return CKKS_ERR_ARG;
+    const uint32_t level = in->level;
+    const uint32_t de = log2_ceil(d->exp_degree), dr = d->rounds ? log2_ceil(d->rsqrt_degree) : 0;
+    if (!level_ok(c, level) || level < (de + 1) + d->rounds * (dr + 4) + 1) return CKKS_ERR_LEVEL;
+    if (!rlk || !rlk->data || rlk->galois != 0) return CKKS_ERR_NO_KEY;
+    const uint32_t stride = c->n / d->row_len;
+    std::vector<const ckks_evk *> rk;
+    for (uint32_t i = 1; i < d->row_len && d->rounds; i *= 2) {
+        const ckks_evk *k = keys ? find_key(keys, nkeys, ckks_galois_element(c, (int64_t)stride * i)) : nullptr;
+        if (!k) return CKKS_ERR_NO_KEY;
+        rk.push_back(k);
+    }
+    if (!ws || ws_bytes < ckks_softmax_workspace_bytes(c, d, level)) return CKKS_ERR_WORKSPACE;
+    const size_t ctb = align256((size_t)2 * level * c->N * sizeof(u64)), scratch = softmax_scratch_bytes(c, d, level);
+    char *base = (char *)ws;
+    ckks_ct U{(uint64_t *)base, level, 2, 0.0}, A{(uint64_t *)(base + ctb), level, 2, 0.0}, B{(uint64_t *)(base + 2 * ctb), level, 2, 0.0},
+        S{(uint64_t *)(base + 3 * ctb), level, 2, 0.0};
+    void *sw = base + 4 * ctb;
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t N = c->N;
+    int rc;
+    // z = x - shift;  u = p_exp(z)
+    if ((rc = ckks_add_const(c, in, -d->shift, &A, stream))) return rc;
+    if ((rc = ckks_poly_eval_tree(c, &A, d->exp_coeffs, d->exp_degree, rlk, &U, sw, scratch, stream))) return rc;
+    for (uint32_t j = 0; j < d->rounds; j++) {
+        // s = row sums of u^2
+        if ((rc = ckks_mul_relin(c, &U, &U, rlk, &A, sw, scratch, stream))) return rc;
+        if ((rc = ckks_rescale(c, &A, &S, sw, scratch, stream))) return rc;
+        for (const ckks_evk *k : rk) {
+            if ((rc = ckks_rotate(c, &S, k, &A, sw, scratch, stream))) return rc;
+            if ((rc = ckks_add(c, &S, &A, &S, stream))) return rc;
+        }
+        // lambda = p_rsqrt_j(s);  u = (lambda u)^2
+        if ((rc = ckks_poly_eval_tree(c, &S, d->rsqrt_coeffs + (size_t)j * (d->rsqrt_degree + 1), d->rsqrt_degree, rlk, &B, sw, scratch, stream)))
+            return rc;
+        {
+            DeviceGuard g(c->device);       // u truncated to lambda's level
+            for (uint32_t comp = 0; comp < 2; comp++)
+                cudaMemcpyAsync((u64 *)A.data + (size_t)comp * B.level * N, (const u64 *)U.data + (size_t)comp * U.level * N,
+                                (size_t)B.level * N * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+            A.level = B.level; A.ncomp = 2; A.scale = U.scale;
+        }
+        if ((rc = ckks_mul_relin(c, &B, &A, rlk, &S, sw, scratch, stream))) return rc;
+        if ((rc = ckks_rescale(c, &S, &A, sw, scratch, stream))) return rc;
+        if ((rc = ckks_mul_relin(c, &A, &A, rlk, &S, sw, scratch, stream))) return rc;
+        if ((rc = ckks_rescale(c, &S, &U, sw, scratch, stream))) return rc;
+    }
+    {
+        DeviceGuard g(c->device);
+        cudaMemcpyAsync(out->data, U.data, (size_t)2 * U.level * N * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+    }
+    rc = finish(c);
+    if (rc == CKKS_OK) { out->level = U.level; out->ncomp = 2; out->scale = U.scale; }
+    return rc;
+}
+
 extern "C" int32_t ckks_rotate(ckks_ctx *c, const ckks_ct *in, const ckks_evk *key, ckks_ct *out, void *ws, size_t ws_bytes,
                                void *stream) {
     int rc = rotate_checks(c, in, key, 1, out, ws, ws_bytes);

@@ -297,6 +297,38 @@ def test_rotate_sum_bit_exact(log_n, L, K, dnum, level, n):
     assert e.value.code == binding.ERR_NO_KEY
 
 
+def test_softmax_by_doubling_bit_exact():
+    """Algorithm 1 with synthetic polynomials on 32 rows of 16 scores (two rounds, degree 4): the composite entry point
+    returns the checker's integers, which decrypt to the same pipeline in the clear and to the Softmax of every row."""
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    from tests.harness import softmax_case
+    P, ctx = params(10, 17, 4, 5), context(10, 17, 4, 5)
+    o = P.oracle
+    cl = Client(P, 71)
+    row_len, rounds, level, scale = 16, 2, 17, 2.0 ** 50
+    x, shift, ce, cr, clear, truth = softmax_case(P, 71, row_len, rounds)
+    ct = cl.encrypt_slots(x, scale, level)
+    rlk = cl.relin_key()
+    keys, i = {}, 1
+    while i < row_len:
+        ge = o.galois_element(P.n // row_len * i)
+        keys[ge] = cl.rotation_key(ge)
+        i *= 2
+    want, want_scale = o.softmax_doubling(ct, scale, shift, rounds, row_len, ce, cr, rlk, keys)
+    got = ctx.softmax(ct_dev(ct, scale), shift, rounds, row_len, ce, cr, key_dev(rlk, 0), [key_dev(k, g) for g, k in keys.items()])
+    assert got.level == want.shape[1] == 2 and got.scale == want_scale
+    arr = host(got.data)
+    assert np.array_equal(arr, want)
+    slots = cl.decrypt_slots(arr, got.scale).real
+    assert np.abs(slots - clear).max() < 2.0 ** -20 and np.abs(slots - truth).max() < 0.05
+    with pytest.raises(binding.CkksError) as e:          # a rotation key of the ladder is missing
+        ctx.softmax(ct_dev(ct, scale), shift, rounds, row_len, ce, cr, key_dev(rlk, 0), [key_dev(k, g) for g, k in list(keys.items())[1:]])
+    assert e.value.code == binding.ERR_NO_KEY
+    with pytest.raises(binding.CkksError) as e:          # not enough levels for the rounds
+        ctx.softmax(ct_dev(ct[:, :10], scale), shift, rounds, row_len, ce, cr, key_dev(rlk, 0), [key_dev(k, g) for g, k in keys.items()])
+    assert e.value.code == binding.ERR_LEVEL
+
+
 def test_repeatability():
     """Same call twice gives the same bytes (a race would show up as a difference)."""
     from tests.gpu_util import context, ct_dev, host, key_dev
