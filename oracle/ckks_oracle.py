@@ -280,6 +280,71 @@ class Oracle:
         so = T / float(self.q[Lt - 1])
         return self.add_const(out, int(np.rint(coeffs[0] * so))), so
 
+    def poly_eval_bsgs(self, x, scale: float, coeffs, rlk, m: int):
+        """sum_k coeffs[k] x^k by baby steps and giant steps (m a power of two, 2 <= m <= degree): about m + 2 d / m
+        products instead of the tree's d - 1, one key switch for the whole giant-step sum.  With blocks
+        B_i(x) = sum_{j<m} coeffs[i m + j] x^j, G = d // m + 1 and y = x^m the polynomial is sum_{i<G} B_i(x) y^i.
+        Order of steps:
+          baby powers pw[k], k = 2..m, and giant powers gp[i] = y^i, i = 2..G-1, as poly_eval_tree forms its powers
+            (operands k // 2 and k - k // 2, truncated to their common level; mul_relin; rescale);
+          Lb = level of pw[m-1] (of x for m = 2), Lc = min(level of gp[G-1], Lb - 1), Tp = scale(x) * q_{Lc-1};
+          block i >= 1 with a non-constant part: at level Lb and scale Ti = (Tp / scale(gp[i])) * q_{Lb-1} the sum over
+            j = 1..m-1 (coefficient != 0, increasing j) of pw[j][:Lb] * round(c (Ti / scale(pw[j]))), rescaled, plus
+            round(coeffs[i m] * (Ti / q_{Lb-1})); a block that is only a constant enters as gp[i][:Lc] * round(c (Tp / scale(gp[i])));
+          S = mul_relin_sum of the non-constant blocks (truncated to Lc) with their gp[i][:Lc], in increasing i;
+          then block 0's terms pw[j][:Lc] * round(c_j (Tp / scale(pw[j]))), j = 1..m-1, and the constant-only blocks are added
+          to S in that order; result = rescale(S) + round(coeffs[0] * (Tp / q_{Lc-1})).
+        Returns (ct, scale = Tp / q_{Lc-1}) at level Lc - 1."""
+        x = _u64(x); level = x.shape[1]; d = len(coeffs) - 1
+        if m < 2 or m & (m - 1) or m > d:
+            raise ValueError("m must be a power of two between 2 and the degree")
+        G = d // m + 1
+        c = lambda k: float(coeffs[k]) if k <= d else 0.0
+        q = lambda l: float(self.q[l - 1])
+
+        def powers(base, sbase, top):
+            pw, sc = {1: base}, {1: sbase}
+            for k in range(2, top + 1):
+                a = k // 2; b = k - a
+                lv = min(pw[a].shape[1], pw[b].shape[1])
+                pw[k] = self.rescale(self.mul_relin(pw[a][:, :lv], pw[b][:, :lv], rlk))
+                sc[k] = sc[a] * sc[b] / q(lv)
+            return pw, sc
+        pw, sc = powers(x, scale, m)
+        gp, sg = powers(pw[m], sc[m], G - 1)
+        Lb = pw[m - 1].shape[1]
+        Lc = min(gp[G - 1].shape[1], Lb - 1)
+        if Lc < 2:
+            raise ValueError("not enough limbs")
+        Tp = scale * q(Lc)
+        A, B, consts = [], [], []
+        for i in range(1, G):
+            Ti = (Tp / sg[i]) * q(Lb)
+            acc = None
+            for j in range(1, m):
+                if c(i * m + j) == 0.0:
+                    continue
+                term = self.mul_const(pw[j][:, :Lb], int(np.rint(c(i * m + j) * (Ti / sc[j]))))
+                acc = term if acc is None else self.add(acc, term)
+            if acc is None:
+                if c(i * m) != 0.0:
+                    consts.append(self.mul_const(gp[i][:, :Lc], int(np.rint(c(i * m) * (Tp / sg[i])))))
+                continue
+            blk = self.add_const(self.rescale(acc), int(np.rint(c(i * m) * (Ti / q(Lb)))))
+            A.append(blk[:, :Lc]); B.append(gp[i][:, :Lc])
+        S = self.mul_relin_sum(np.stack(A), np.stack(B), rlk) if A else None
+        for j in range(1, m):
+            if c(j) == 0.0:
+                continue
+            term = self.mul_const(pw[j][:, :Lc], int(np.rint(c(j) * (Tp / sc[j]))))
+            S = term if S is None else self.add(S, term)
+        for t in consts:
+            S = t if S is None else self.add(S, t)
+        if S is None:
+            raise ValueError("all non-constant coefficients are zero")
+        so = Tp / q(Lc)
+        return self.add_const(self.rescale(S), int(np.rint(c(0) * so))), so
+
     def softmax_doubling(self, x, scale: float, shift: float, rounds: int, row_len: int, exp_coeffs, rsqrt_coeffs, rlk, keys: dict):
         """Softmax by doubling with a public shift (Algorithm 1) on one ciphertext of score rows.  Row r holds its
         row_len scores in slots i * (n / row_len) + r, so that rotations by (n / row_len) 2^i, i < log2 row_len,

@@ -348,3 +348,33 @@ def test_poly_eval_tree_pins():
         if d <= 7:
             h, sh = o.poly_eval(ct, scale, coeffs, rlk)
             assert np.abs(cl.decrypt_slots(h, sh) - got).max() < 2.0 ** -25
+
+
+def test_poly_eval_bsgs_pins():
+    """Baby-step / giant-step polynomial evaluation: the polynomial of the slots (as poly_eval_tree's pin), the tree's
+    result within noise, the level it ends on, and the special shapes (a block that is only a constant, zero coefficients,
+    a degree that does not fill the last block)."""
+    P = params(11, 9, 3, 3)
+    o = P.oracle
+    cl = Client(P, 81)
+    g = inputs.rng(81)
+    level, scale = 9, 2.0 ** 50
+    z = g.uniform(-1, 1, P.n)
+    ct = cl.encrypt_slots(z, scale, level)
+    rlk = cl.relin_key()
+    pv = np.polynomial.polynomial.polyval
+    for d, m in [(15, 4), (9, 4), (7, 2), (31, 8), (5, 4)]:
+        coeffs = g.uniform(-1, 1, d + 1) / (1 + np.arange(d + 1))
+        if d == 15:
+            coeffs[[5, 6, 7]] = 0.0          # block 1 is only a constant
+            coeffs[9] = 0.0
+        out, so = o.poly_eval_bsgs(ct, scale, coeffs, rlk, m)
+        G = d // m + 1
+        lb = level - max(m - 2, 0).bit_length()                       # level of x^(m-1)
+        lg = level - (m - 1).bit_length() - max(G - 2, 0).bit_length()  # level of y^(G-1)
+        assert out.shape[1] == min(lg, lb - 1) - 1
+        got = cl.decrypt_slots(out, so).real
+        assert np.abs(got - pv(z, coeffs)).max() < 2.0 ** -20, (d, m)
+        if d <= 15:
+            tree, st = o.poly_eval_tree(ct, scale, coeffs, rlk)
+            assert np.abs(cl.decrypt_slots(tree, st).real - got).max() < 2.0 ** -22
