@@ -324,6 +324,10 @@ def run_cuda(args):
         extras["rotate_64_calls_ms"] = once(lambda: [ctx.rotate(x_, rot_keys[0], out=rot_out) for x_ in rin])
         extras["rotate_batch_64_ms"] = once(lambda: ctx.rotate_batch(rin, rot_keys[0], outs=routs, ws=rws))
         del routs, rws
+        # a degree-63 polynomial (the paper's SiLU degree per layer) by the power tree and by baby steps / giant steps
+        c63 = [1.0 / (1 + k) for k in range(64)]
+        extras["poly_degree63_tree_ms"] = once(lambda: ctx.poly_eval_tree(binding.Ciphertext(cta.data, 2.0 ** 50), c63, rlk))
+        extras["poly_degree63_bsgs_m8_ms"] = once(lambda: ctx.poly_eval_bsgs(binding.Ciphertext(cta.data, 2.0 ** 50), c63, 8, rlk))
         # Softmax by doubling on 256 rows of 128 scores (one ciphertext), two rounds, degree-4 polynomials: 7 + 2 x 11 products,
         # 14 rotations
         sm_keys = [keys[256 << i] for i in range(7)]

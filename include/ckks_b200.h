@@ -238,6 +238,17 @@ int32_t ckks_poly_eval(ckks_ctx *ctx, const ckks_ct *x, const double *coeffs, ui
 int32_t ckks_poly_eval_tree(ckks_ctx *ctx, const ckks_ct *x, const double *coeffs, uint32_t degree, const ckks_evk *rlk, ckks_ct *out,
                             void *ws, size_t ws_bytes, void *stream);
 
+/* The same polynomial by baby steps and giant steps: blocks of m coefficients (m a power of two, 2 <= m <= degree) over
+ * the baby powers x .. x^(m-1), times the giant powers (x^m)^i, i < G = degree / m + 1, the giant-step sum relinearised
+ * once (ckks_mul_relin_sum): about m + 2 degree / m products instead of degree - 1, at most one level more than
+ * ckks_poly_eval_tree.  The powers are formed as ckks_poly_eval_tree forms them; blocks are encoded so that every
+ * product lands on the scale x.scale * q at the common level Lc = min(level of x^(m (G-1)), level of x^(m-1) - 1); the
+ * result has level Lc - 1 and scale x.scale * q_{Lc-1} / q_{Lc-1}.  Workspace: ckks_poly_eval_bsgs_workspace_bytes.
+ * Errors as ckks_poly_eval_tree; CKKS_ERR_ARG for an m that is not a power of two in [2, degree]. */
+int32_t ckks_poly_eval_bsgs(ckks_ctx *ctx, const ckks_ct *x, const double *coeffs, uint32_t degree, uint32_t m, const ckks_evk *rlk,
+                            ckks_ct *out, void *ws, size_t ws_bytes, void *stream);
+size_t ckks_poly_eval_bsgs_workspace_bytes(const ckks_ctx *ctx, uint32_t level, uint32_t degree, uint32_t m);
+
 /* ---- Softmax by doubling with a public shift (Algorithm 1) --------------------
  * One ciphertext of score rows: row r holds its row_len scores (a power of two dividing n) in slots
  * i * (n / row_len) + r, so that rotations by (n / row_len) 2^i, i < log2 row_len, leave a row's sum in every one of its

@@ -23,7 +23,7 @@ EXPORTS = [
     "ckks_encode_range_flag", "ckks_mul_plain_acc", "ckks_add", "ckks_mul_relin", "ckks_rotate",
     "ckks_rotate_hoisted", "ckks_rescale", "ckks_linear_proj", "ckks_linear_proj_workspace_bytes",
     "ckks_linear_proj_rotations", "ckks_kernel_launches", "ckks_device_status", "ckks_rescale_static",
-    "ckks_ntt_butterfly_probe", "ckks_mul_relin_sum", "ckks_mul_relin_batch", "ckks_rotate_batch", "ckks_rotate_sum", "ckks_softmax", "ckks_softmax_workspace_bytes", "ckks_mul_const", "ckks_add_const", "ckks_poly_eval", "ckks_poly_eval_tree", "ckks_linear_proj_multi", "ckks_linear_proj_multi_workspace_bytes",
+    "ckks_ntt_butterfly_probe", "ckks_mul_relin_sum", "ckks_mul_relin_batch", "ckks_rotate_batch", "ckks_rotate_sum", "ckks_softmax", "ckks_softmax_workspace_bytes", "ckks_poly_eval_bsgs", "ckks_poly_eval_bsgs_workspace_bytes", "ckks_mul_const", "ckks_add_const", "ckks_poly_eval", "ckks_poly_eval_tree", "ckks_linear_proj_multi", "ckks_linear_proj_multi_workspace_bytes",
 ]
 
 
@@ -82,6 +82,8 @@ def load():
         "ckks_mul_plain_acc": (i32, [vp, C.POINTER(CCt), u32, C.POINTER(CPt), C.POINTER(CCt), i32, vp]),
         "ckks_add": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), C.POINTER(CCt), vp]),
         "ckks_mul_relin": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
+        "ckks_poly_eval_bsgs": (i32, [vp, C.POINTER(CCt), C.POINTER(C.c_double), u32, u32, C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
+        "ckks_poly_eval_bsgs_workspace_bytes": (sz, [vp, u32, u32, u32]),
         "ckks_softmax": (i32, [vp, C.POINTER(CSoftmaxDesc), C.POINTER(CCt), C.POINTER(CEvk), C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
         "ckks_softmax_workspace_bytes": (sz, [vp, C.POINTER(CSoftmaxDesc), u32]),
         "ckks_rotate_sum": (i32, [vp, C.POINTER(CCt), C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
@@ -335,6 +337,21 @@ class Context:
                                                _stream_ptr(stream)))
         out.scale = co.scale
         return out
+
+    def poly_eval_bsgs(self, x: Ciphertext, coeffs, m: int, rlk: SwitchKey, stream=None):
+        """sum_k coeffs[k] x^k by baby steps (blocks of m coefficients) and giant steps with one key switch for their sum."""
+        d = len(coeffs) - 1
+        need = int(load().ckks_poly_eval_bsgs_workspace_bytes(self._h, x.level, d, m))
+        if need == 0:
+            raise CkksError(ERR_ARG)
+        ws = self.workspace(need)
+        out = self.empty_ct(x.level)
+        ca = (C.c_double * (d + 1))(*[float(v) for v in coeffs])
+        co = _cct(out)
+        ck = CEvk(_dev_u64(rlk.data).data_ptr(), rlk.galois)
+        self._check(load().ckks_poly_eval_bsgs(self._h, C.byref(_cct(x)), ca, d, m, C.byref(ck), C.byref(co), ws.data_ptr(), ws.numel(),
+                                               _stream_ptr(stream)))
+        return Ciphertext(out.data.view(-1)[: 2 * co.level * self.N].view(2, co.level, self.N), co.scale)
 
     def softmax(self, ct: Ciphertext, shift: float, rounds: int, row_len: int, exp_coeffs, rsqrt_coeffs, rlk: SwitchKey, keys,
                 ws: torch.Tensor = None, stream=None):

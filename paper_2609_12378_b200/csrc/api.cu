@@ -605,6 +605,142 @@ extern "C" int32_t ckks_poly_eval_tree(ckks_ctx *c, const ckks_ct *x, const doub
     return rc;
 }
 
+// ---- Baby-step / giant-step polynomial evaluation: a composition of the entry points above
+static bool bsgs_shape_ok(uint32_t degree, uint32_t m) { return m >= 2 && !(m & (m - 1)) && m <= degree; }
+static size_t bsgs_scratch_bytes(const ckks_ctx *c, uint32_t level) {
+    return align256(std::max(ckks_workspace_bytes(c, CKKS_OP_MUL_RELIN, level, 0), ckks_workspace_bytes(c, CKKS_OP_RESCALE, level, 0)));
+}
+static uint32_t bsgs_buffers(uint32_t degree, uint32_t m) {
+    const uint32_t G = degree / m + 1;
+    return (m - 1) + (G > 2 ? G - 2 : 0) + 2 * (G - 1) + 6;      // baby powers, giant powers, blocks and truncated giants, temporaries
+}
+
+extern "C" size_t ckks_poly_eval_bsgs_workspace_bytes(const ckks_ctx *c, uint32_t level, uint32_t degree, uint32_t m) {
+    if (!c || !level_ok(c, level) || !bsgs_shape_ok(degree, m)) return 0;
+    return (size_t)bsgs_buffers(degree, m) * align256((size_t)2 * level * c->N * sizeof(u64)) + bsgs_scratch_bytes(c, level);
+}
+
+extern "C" int32_t ckks_poly_eval_bsgs(ckks_ctx *c, const ckks_ct *x, const double *coeffs, uint32_t degree, uint32_t m, const ckks_evk *rlk,
+                                       ckks_ct *out, void *ws, size_t ws_bytes, void *stream) {
+    if (!c || !ct_ok(x) || !ct_ok(out) || x->ncomp != 2 || !coeffs || !bsgs_shape_ok(degree, m)) return CKKS_ERR_ARG;
+    const uint32_t level = x->level, G = degree / m + 1;
+    if (!level_ok(c, level)) return CKKS_ERR_LEVEL;
+    if (!rlk || !rlk->data || rlk->galois != 0) return CKKS_ERR_NO_KEY;
+    // levels of the powers (operands k / 2 and k - k / 2, one level per product)
+    std::vector<uint32_t> lb(m + 1), lg(G);
+    lb[1] = level;
+    for (uint32_t k = 2; k <= m; k++) {
+        const uint32_t lv = std::min(lb[k / 2], lb[k - k / 2]);
+        if (lv < 2) return CKKS_ERR_LEVEL;
+        lb[k] = lv - 1;
+    }
+    lg[1] = lb[m];
+    for (uint32_t i = 2; i < G; i++) {
+        const uint32_t lv = std::min(lg[i / 2], lg[i - i / 2]);
+        if (lv < 2) return CKKS_ERR_LEVEL;
+        lg[i] = lv - 1;
+    }
+    const uint32_t Lb = lb[m - 1], Lc = std::min(lg[G - 1], Lb - 1);
+    if (Lb < 2 || Lc < 2) return CKKS_ERR_LEVEL;
+    if (!ws || ws_bytes < ckks_poly_eval_bsgs_workspace_bytes(c, level, degree, m)) return CKKS_ERR_WORKSPACE;
+    auto coef = [&](uint32_t k) { return k <= degree ? coeffs[k] : 0.0; };
+    auto q = [&](uint32_t l) { return (double)c->mod[l - 1]; };
+
+    const size_t N = c->N, ctb = align256((size_t)2 * level * N * sizeof(u64)), scratch = bsgs_scratch_bytes(c, level);
+    char *base = (char *)ws;
+    uint32_t next = 0;
+    auto buffer = [&]() { return ckks_ct{(uint64_t *)(base + (size_t)(next++) * ctb), level, 2, 0.0}; };
+    std::vector<ckks_ct> pw(m + 1), gp(G);
+    pw[1] = *x;
+    for (uint32_t k = 2; k <= m; k++) pw[k] = buffer();
+    for (uint32_t i = 2; i < G; i++) gp[i] = buffer();
+    std::vector<ckks_ct> blk(G), gpt(G);
+    for (uint32_t i = 1; i < G; i++) { blk[i] = buffer(); gpt[i] = buffer(); }
+    ckks_ct ta = buffer(), tb = buffer(), prod = buffer(), acc = buffer(), term = buffer(), S = buffer();
+    void *sw = base + (size_t)bsgs_buffers(degree, m) * ctb;
+    cudaStream_t s = (cudaStream_t)stream;
+    DeviceGuard guard(c->device);
+    // src cut down to `to` limbs per component (a copy into dst), or src itself if it has that many
+    auto at_level = [&](const ckks_ct &src, uint32_t to, ckks_ct &dst) -> ckks_ct {
+        if (src.level == to) return src;
+        for (uint32_t comp = 0; comp < 2; comp++)
+            cudaMemcpyAsync(dst.data + (size_t)comp * to * N, src.data + (size_t)comp * src.level * N, (size_t)to * N * sizeof(u64),
+                            cudaMemcpyDeviceToDevice, s);
+        dst.level = to; dst.ncomp = 2; dst.scale = src.scale;
+        return dst;
+    };
+    int rc;
+    auto powers = [&](std::vector<ckks_ct> &p, uint32_t top) -> int {
+        for (uint32_t k = 2; k <= top; k++) {
+            const uint32_t a = k / 2, b = k - a, lv = std::min(p[a].level, p[b].level);
+            const ckks_ct pa = at_level(p[a], lv, ta), pb = at_level(p[b], lv, tb);
+            int r;
+            if ((r = ckks_mul_relin(c, &pa, &pb, rlk, &prod, sw, scratch, stream))) return r;
+            if ((r = ckks_rescale(c, &prod, &p[k], sw, scratch, stream))) return r;
+        }
+        return CKKS_OK;
+    };
+    if ((rc = powers(pw, m))) return rc;
+    gp[1] = pw[m];
+    if ((rc = powers(gp, G - 1))) return rc;
+    const double Tp = x->scale * q(Lc);
+    // the blocks B_i, i >= 1, encoded so that B_i y^i has scale Tp; constant-only blocks are kept for later
+    std::vector<ckks_ct> A, B;
+    std::vector<uint32_t> const_only;
+    for (uint32_t i = 1; i < G; i++) {
+        const double Ti = (Tp / gp[i].scale) * q(Lb);
+        bool first = true;
+        for (uint32_t j = 1; j < m; j++) {
+            if (coef(i * m + j) == 0.0) continue;
+            const ckks_ct pj = at_level(pw[j], Lb, ta);
+            ckks_ct &dst = first ? acc : term;
+            if ((rc = ckks_mul_const(c, &pj, coef(i * m + j), Ti / pw[j].scale, &dst, stream))) return rc;
+            if (!first && (rc = ckks_add(c, &acc, &term, &acc, stream))) return rc;
+            first = false;
+        }
+        if (first) {
+            if (coef(i * m) != 0.0) const_only.push_back(i);
+            continue;
+        }
+        acc.scale = Ti;
+        if ((rc = ckks_rescale(c, &acc, &prod, sw, scratch, stream))) return rc;
+        if ((rc = ckks_add_const(c, &prod, coef(i * m), &prod, stream))) return rc;
+        ckks_ct a = at_level(prod, Lc, blk[i]);
+        if (a.data == prod.data) {       // already at the common level: keep a copy, prod is reused
+            cudaMemcpyAsync(blk[i].data, prod.data, (size_t)2 * Lc * N * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+            blk[i].level = Lc; blk[i].ncomp = 2;
+            a = blk[i];
+        }
+        ckks_ct b = at_level(gp[i], Lc, gpt[i]);
+        a.scale = 1.0; b.scale = Tp;      // the products agree in scale (Tp up to rounding); the factors need not
+        A.push_back(a); B.push_back(b);
+    }
+    bool have = false;
+    if (!A.empty()) {
+        if ((rc = ckks_mul_relin_sum(c, A.data(), B.data(), (uint32_t)A.size(), rlk, &S, sw, scratch, stream))) return rc;
+        have = true;
+    }
+    auto add_in = [&](const ckks_ct &src, double cv, double cs) -> int {
+        const ckks_ct p = at_level(src, Lc, ta);
+        ckks_ct &dst = have ? term : S;
+        int r;
+        if ((r = ckks_mul_const(c, &p, cv, cs, &dst, stream))) return r;
+        dst.scale = Tp;
+        if (have && (r = ckks_add(c, &S, &term, &S, stream))) return r;
+        have = true;
+        return CKKS_OK;
+    };
+    S.scale = Tp;
+    for (uint32_t j = 1; j < m; j++)
+        if (coef(j) != 0.0 && (rc = add_in(pw[j], coef(j), Tp / pw[j].scale))) return rc;
+    for (uint32_t i : const_only)
+        if ((rc = add_in(gp[i], coef(i * m), Tp / gp[i].scale))) return rc;
+    if (!have) return CKKS_ERR_ARG;
+    S.scale = Tp;
+    if ((rc = ckks_rescale(c, &S, out, sw, scratch, stream))) return rc;
+    return ckks_add_const(c, out, coef(0), out, stream);
+}
+
 // ---- Softmax by doubling (Algorithm 1): a composition of the entry points above on buffers carved from the workspace
 static uint32_t log2_ceil(uint32_t x) { uint32_t d = 0; while ((1u << d) < x) d++; return d; }
 static size_t softmax_scratch_bytes(const ckks_ctx *c, const ckks_softmax_desc *d, uint32_t level) {

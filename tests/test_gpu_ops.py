@@ -297,6 +297,40 @@ def test_rotate_sum_bit_exact(log_n, L, K, dnum, level, n):
     assert e.value.code == binding.ERR_NO_KEY
 
 
+@pytest.mark.parametrize("log_n,d,m", [(11, 15, 4), (11, 9, 4), (11, 7, 2), (11, 31, 8), (11, 5, 4), (16, 31, 8)])
+def test_poly_eval_bsgs_bit_exact(log_n, d, m):
+    """Baby-step / giant-step polynomial evaluation: the checker's integers (constant-only block and zero coefficients at
+    degree 15; a partial last block; N = 2^16 at level 24) and the error paths."""
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    cfg = (11, 9, 3, 3) if log_n == 11 else (16, 24, 8, 3)
+    P, ctx = params(*cfg), context(*cfg)
+    o = P.oracle
+    cl = Client(P, 81)
+    g = inputs.rng(81, d)
+    level, scale = cfg[1], 2.0 ** 50
+    z = g.uniform(-1, 1, P.n)
+    ct = cl.encrypt_slots(z, scale, level)
+    rlk = cl.relin_key()
+    coeffs = g.uniform(-1, 1, d + 1) / (1 + np.arange(d + 1))
+    if d == 15:
+        coeffs[[5, 6, 7]] = 0.0
+        coeffs[9] = 0.0
+    want, so = o.poly_eval_bsgs(ct, scale, coeffs, rlk, m)
+    got = ctx.poly_eval_bsgs(ct_dev(ct, scale), coeffs, m, key_dev(rlk, 0))
+    assert got.level == want.shape[1] and got.scale == so
+    arr = host(got.data)
+    assert np.array_equal(arr, want)
+    assert np.abs(cl.decrypt_slots(arr, so).real - np.polynomial.polynomial.polyval(z, coeffs)).max() < 2.0 ** -20
+    if d == 15:
+        for bad_m in (3, 16, 1):
+            with pytest.raises(binding.CkksError) as e:
+                ctx.poly_eval_bsgs(ct_dev(ct, scale), coeffs, bad_m, key_dev(rlk, 0))
+            assert e.value.code == binding.ERR_ARG
+        with pytest.raises(binding.CkksError) as e:
+            ctx.poly_eval_bsgs(ct_dev(ct[:, :3], scale), coeffs, 4, key_dev(rlk, 0))
+        assert e.value.code == binding.ERR_LEVEL
+
+
 def test_softmax_by_doubling_bit_exact():
     """Algorithm 1 with synthetic polynomials on 32 rows of 16 scores (two rounds, degree 4): the composite entry point
     returns the checker's integers, which decrypt to the same pipeline in the clear and to the Softmax of every row."""
