@@ -256,7 +256,8 @@ size_t ckks_poly_eval_bsgs_workspace_bytes(const ckks_ctx *ctx, uint32_t level, 
  * polynomial p_exp(z / 2^rounds) written as a polynomial in z = x - shift; rsqrt_coeffs (host, rounds x
  * (rsqrt_degree + 1) values): round j's inverse-square-root polynomial.  Steps, all on the device:
  *   z = x - shift;  u = p_exp(z);  per round: s = row sums of u^2;  lambda = p_rsqrt_j(s);  u = (lambda u)^2,
- * every product followed by a rescale, both polynomials evaluated as ckks_poly_eval_tree does.  No bootstrapping:
+ * every product followed by a rescale, both polynomials evaluated as ckks_poly_eval_tree does, or, where exp_m /
+ * rsqrt_m is not 0, as ckks_poly_eval_bsgs does with blocks of that size.  No bootstrapping: with the power tree
  * the input needs (d_e + 1) + rounds * (d_r + 4) limbs more than the output keeps, d = ceil(log2 degree).  Scores should
  * be encrypted at a scale near the primes.  out: level and scale as they come out.  Workspace:
  * ckks_softmax_workspace_bytes.  Errors: ARG, LEVEL, NO_KEY, RANGE (a constant beyond 2^62), WORKSPACE. */
@@ -265,6 +266,7 @@ typedef struct {
     uint32_t rounds, row_len, exp_degree, rsqrt_degree;
     const double *exp_coeffs;   /* host */
     const double *rsqrt_coeffs; /* host */
+    uint32_t exp_m, rsqrt_m;    /* 0: power tree; else the block size of ckks_poly_eval_bsgs */
 } ckks_softmax_desc;
 int32_t ckks_softmax(ckks_ctx *ctx, const ckks_softmax_desc *desc, const ckks_ct *in, const ckks_evk *rlk, const ckks_evk *keys,
                      uint32_t nkeys, ckks_ct *out, void *ws, size_t ws_bytes, void *stream);

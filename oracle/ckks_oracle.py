@@ -345,7 +345,8 @@ class Oracle:
         so = Tp / q(Lc)
         return self.add_const(self.rescale(S), int(np.rint(c(0) * so))), so
 
-    def softmax_doubling(self, x, scale: float, shift: float, rounds: int, row_len: int, exp_coeffs, rsqrt_coeffs, rlk, keys: dict):
+    def softmax_doubling(self, x, scale: float, shift: float, rounds: int, row_len: int, exp_coeffs, rsqrt_coeffs, rlk, keys: dict,
+                         exp_m: int = 0, rsqrt_m: int = 0):
         """Softmax by doubling with a public shift (Algorithm 1) on one ciphertext of score rows.  Row r holds its
         row_len scores in slots i * (n / row_len) + r, so that rotations by (n / row_len) 2^i, i < log2 row_len,
         add up a whole row in every one of its slots.  exp_coeffs: the polynomial p_exp(z / 2^k) as a polynomial in z;
@@ -355,13 +356,15 @@ class Oracle:
                      lam = poly_eval_tree(s, rsqrt_coeffs[j]);  v = rescale(mul_relin(lam, u truncated to lam's level));
                      u = rescale(mul_relin(v, v)).
         Scales are doubles, multiplied and divided in this order.  keys maps a Galois element to its key.
+        exp_m / rsqrt_m != 0 evaluate that polynomial by poly_eval_bsgs with blocks of m instead of the power tree.
         Returns (ct, scale)."""
         x = _u64(x)
         stride = self.n // row_len
         if row_len < 2 or row_len & (row_len - 1) or self.n % row_len:
             raise ValueError("row_len must be a power of two dividing the slot count")
         z = self.add_const(x, int(np.rint(-shift * scale)))
-        u, su = self.poly_eval_tree(z, scale, exp_coeffs, rlk)
+        poly = lambda c_, s_, co, m_: self.poly_eval_bsgs(c_, s_, co, rlk, m_) if m_ else self.poly_eval_tree(c_, s_, co, rlk)
+        u, su = poly(z, scale, exp_coeffs, exp_m)
         for j in range(rounds):
             lv = u.shape[1]
             sq = self.rescale(self.mul_relin(u, u, rlk)); ss = su * su / float(self.q[lv - 1])
@@ -371,7 +374,7 @@ class Oracle:
                 ge = self.galois_element(stride * i)
                 s = self.add(s, self.rotate(s, keys[ge], ge))
                 i *= 2
-            lam, sl = self.poly_eval_tree(s, ss, rsqrt_coeffs[j], rlk)
+            lam, sl = poly(s, ss, rsqrt_coeffs[j], rsqrt_m)
             ll = lam.shape[1]
             v = self.rescale(self.mul_relin(lam, u[:, :ll], rlk)); sv = sl * su / float(self.q[ll - 1])
             u = self.rescale(self.mul_relin(v, v, rlk)); su = sv * sv / float(self.q[ll - 2])

@@ -46,7 +46,8 @@ class CEvk(C.Structure):
 
 class CSoftmaxDesc(C.Structure):
     _fields_ = [("shift", C.c_double), ("rounds", C.c_uint32), ("row_len", C.c_uint32), ("exp_degree", C.c_uint32),
-                ("rsqrt_degree", C.c_uint32), ("exp_coeffs", C.POINTER(C.c_double)), ("rsqrt_coeffs", C.POINTER(C.c_double))]
+                ("rsqrt_degree", C.c_uint32), ("exp_coeffs", C.POINTER(C.c_double)), ("rsqrt_coeffs", C.POINTER(C.c_double)),
+                ("exp_m", C.c_uint32), ("rsqrt_m", C.c_uint32)]
 
 
 class CProjDesc(C.Structure):
@@ -354,7 +355,7 @@ class Context:
         return Ciphertext(out.data.view(-1)[: 2 * co.level * self.N].view(2, co.level, self.N), co.scale)
 
     def softmax(self, ct: Ciphertext, shift: float, rounds: int, row_len: int, exp_coeffs, rsqrt_coeffs, rlk: SwitchKey, keys,
-                ws: torch.Tensor = None, stream=None):
+                ws: torch.Tensor = None, stream=None, exp_m: int = 0, rsqrt_m: int = 0):
         """Softmax by doubling with a public shift on one ciphertext of score rows (row r in slots i * (n / row_len) + r).
         exp_coeffs: p_exp(z / 2^rounds) as a polynomial in z; rsqrt_coeffs: [rounds][degree + 1]."""
         ec = (C.c_double * len(exp_coeffs))(*[float(v) for v in exp_coeffs])
@@ -362,7 +363,7 @@ class Context:
         rc = (C.c_double * max(1, len(flat)))(*flat)
         rdeg = (len(rsqrt_coeffs[0]) - 1) if rounds else 0
         d = CSoftmaxDesc(float(shift), rounds, row_len, len(exp_coeffs) - 1, rdeg, C.cast(ec, C.POINTER(C.c_double)),
-                         C.cast(rc, C.POINTER(C.c_double)))
+                         C.cast(rc, C.POINTER(C.c_double)), exp_m, rsqrt_m)
         need = int(load().ckks_softmax_workspace_bytes(self._h, C.byref(d), ct.level))
         if need == 0:
             raise CkksError(ERR_ARG)

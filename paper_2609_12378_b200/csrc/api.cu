@@ -745,12 +745,16 @@ extern "C" int32_t ckks_poly_eval_bsgs(ckks_ctx *c, const ckks_ct *x, const doub
 static uint32_t log2_ceil(uint32_t x) { uint32_t d = 0; while ((1u << d) < x) d++; return d; }
 static size_t softmax_scratch_bytes(const ckks_ctx *c, const ckks_softmax_desc *d, uint32_t level) {
     const uint32_t deg = std::max(d->exp_degree, d->rsqrt_degree);
-    return align256(std::max(ckks_workspace_bytes(c, CKKS_OP_POLY_EVAL_TREE, level, deg),
-                             std::max(ckks_workspace_bytes(c, CKKS_OP_MUL_RELIN, level, 0), ckks_workspace_bytes(c, CKKS_OP_RESCALE, level, 0))));
+    size_t b = std::max(ckks_workspace_bytes(c, CKKS_OP_POLY_EVAL_TREE, level, deg),
+                        std::max(ckks_workspace_bytes(c, CKKS_OP_MUL_RELIN, level, 0), ckks_workspace_bytes(c, CKKS_OP_RESCALE, level, 0)));
+    if (d->exp_m) b = std::max(b, ckks_poly_eval_bsgs_workspace_bytes(c, level, d->exp_degree, d->exp_m));
+    if (d->rsqrt_m && d->rounds) b = std::max(b, ckks_poly_eval_bsgs_workspace_bytes(c, level, d->rsqrt_degree, d->rsqrt_m));
+    return align256(b);
 }
 static bool softmax_desc_ok(const ckks_ctx *c, const ckks_softmax_desc *d) {
     return d && d->exp_coeffs && d->exp_degree >= 2 && (d->rounds == 0 || (d->rsqrt_coeffs && d->rsqrt_degree >= 2)) && d->row_len >= 2 &&
-           !(d->row_len & (d->row_len - 1)) && c->n % d->row_len == 0;
+           !(d->row_len & (d->row_len - 1)) && c->n % d->row_len == 0 && (!d->exp_m || bsgs_shape_ok(d->exp_degree, d->exp_m)) &&
+           (!d->rsqrt_m || !d->rounds || bsgs_shape_ok(d->rsqrt_degree, d->rsqrt_m));
 }
 
 extern "C" size_t ckks_softmax_workspace_bytes(const ckks_ctx *c, const ckks_softmax_desc *d, uint32_t level) {
@@ -763,7 +767,8 @@ extern "C" int32_t ckks_softmax(ckks_ctx *c, const ckks_softmax_desc *d, const c
     if (!c || !softmax_desc_ok(c, d) || !ct_ok(in) || !ct_ok(out) || in->ncomp != 2) return CKKS_ERR_ARG;
     const uint32_t level = in->level;
     const uint32_t de = log2_ceil(d->exp_degree), dr = d->rounds ? log2_ceil(d->rsqrt_degree) : 0;
-    if (!level_ok(c, level) || level < (de + 1) + d->rounds * (dr + 4) + 1) return CKKS_ERR_LEVEL;
+    if (!level_ok(c, level)) return CKKS_ERR_LEVEL;
+    if (!d->exp_m && !d->rsqrt_m && level < (de + 1) + d->rounds * (dr + 4) + 1) return CKKS_ERR_LEVEL;    // else the steps report it
     if (!rlk || !rlk->data || rlk->galois != 0) return CKKS_ERR_NO_KEY;
     const uint32_t stride = c->n / d->row_len;
     std::vector<const ckks_evk *> rk;
@@ -783,7 +788,10 @@ extern "C" int32_t ckks_softmax(ckks_ctx *c, const ckks_softmax_desc *d, const c
     int rc;
     // z = x - shift;  u = p_exp(z)
     if ((rc = ckks_add_const(c, in, -d->shift, &A, stream))) return rc;
-    if ((rc = ckks_poly_eval_tree(c, &A, d->exp_coeffs, d->exp_degree, rlk, &U, sw, scratch, stream))) return rc;
+    auto poly = [&](const ckks_ct *x, const double *co, uint32_t deg, uint32_t bm, ckks_ct *o) {
+        return bm ? ckks_poly_eval_bsgs(c, x, co, deg, bm, rlk, o, sw, scratch, stream) : ckks_poly_eval_tree(c, x, co, deg, rlk, o, sw, scratch, stream);
+    };
+    if ((rc = poly(&A, d->exp_coeffs, d->exp_degree, d->exp_m, &U))) return rc;
     for (uint32_t j = 0; j < d->rounds; j++) {
         // s = row sums of u^2
         if ((rc = ckks_mul_relin(c, &U, &U, rlk, &A, sw, scratch, stream))) return rc;
@@ -793,8 +801,7 @@ extern "C" int32_t ckks_softmax(ckks_ctx *c, const ckks_softmax_desc *d, const c
             if ((rc = ckks_add(c, &S, &A, &S, stream))) return rc;
         }
         // lambda = p_rsqrt_j(s);  u = (lambda u)^2
-        if ((rc = ckks_poly_eval_tree(c, &S, d->rsqrt_coeffs + (size_t)j * (d->rsqrt_degree + 1), d->rsqrt_degree, rlk, &B, sw, scratch, stream)))
-            return rc;
+        if ((rc = poly(&S, d->rsqrt_coeffs + (size_t)j * (d->rsqrt_degree + 1), d->rsqrt_degree, d->rsqrt_m, &B))) return rc;
         {
             DeviceGuard g(c->device);       // u truncated to lambda's level
             for (uint32_t comp = 0; comp < 2; comp++)

@@ -363,6 +363,29 @@ def test_softmax_by_doubling_bit_exact():
     assert e.value.code == binding.ERR_LEVEL
 
 
+def test_softmax_with_block_polynomials_bit_exact():
+    """One round with degree-8 polynomials evaluated by baby steps and giant steps (blocks of 4)."""
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    from tests.harness import softmax_case
+    P, ctx = params(10, 13, 4, 4), context(10, 13, 4, 4)
+    o = P.oracle
+    cl = Client(P, 73)
+    row_len, rounds, level, scale = 16, 1, 13, 2.0 ** 50
+    x, shift, ce, cr, clear, truth = softmax_case(P, 73, row_len, rounds, degree=8, spread=5.0)
+    ct = cl.encrypt_slots(x, scale, level)
+    rlk = cl.relin_key()
+    keys, i = {}, 1
+    while i < row_len:
+        ge = o.galois_element(P.n // row_len * i)
+        keys[ge] = cl.rotation_key(ge)
+        i *= 2
+    want, want_scale = o.softmax_doubling(ct, scale, shift, rounds, row_len, ce, cr, rlk, keys, exp_m=4, rsqrt_m=4)
+    got = ctx.softmax(ct_dev(ct, scale), shift, rounds, row_len, ce, cr, key_dev(rlk, 0), [key_dev(k, g) for g, k in keys.items()],
+                      exp_m=4, rsqrt_m=4)
+    assert got.level == want.shape[1] and got.scale == want_scale
+    assert np.array_equal(host(got.data), want)
+
+
 def test_repeatability():
     """Same call twice gives the same bytes (a race would show up as a difference)."""
     from tests.gpu_util import context, ct_dev, host, key_dev

@@ -32,6 +32,22 @@ def test_softmax_doubling_matches_clear_pipeline_and_softmax():
     assert np.abs(got.reshape(row_len, stride).sum(0) - 1.0).max() < 0.1       # every row sums to about one
 
 
+def test_softmax_doubling_with_block_polynomials():
+    """The same loop with both polynomials (degree 8) evaluated by baby steps and giant steps: one round, the clear
+    pipeline and the true Softmax again."""
+    P = params(10, 13, 4, 4)
+    o = P.oracle
+    cl = Client(P, 73)
+    row_len, rounds, level, scale = 16, 1, 13, 2.0 ** 50
+    x, shift, ce, cr, clear, truth = softmax_case(P, 73, row_len, rounds, degree=8, spread=5.0)
+    ct = cl.encrypt_slots(x, scale, level)
+    out, so = o.softmax_doubling(ct, scale, shift, rounds, row_len, ce, cr, cl.relin_key(), _keys(cl, o, row_len), exp_m=4, rsqrt_m=4)
+    assert out.shape[1] == level - 4 - 7
+    got = cl.decrypt_slots(out, so).real
+    assert np.abs(got - clear).max() < 2.0 ** -20
+    assert np.abs(got - truth).max() < 0.02
+
+
 def test_row_sum_by_strided_rotations():
     """The rotate-and-add ladder the Softmax rounds use: rotations by (n / R) 2^i leave the row sum in every slot of the row."""
     P = params(10, 4, 2, 2)
