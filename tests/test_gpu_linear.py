@@ -186,6 +186,48 @@ def test_projection_multi_shares_baby_steps():
     assert e.value.code == binding.ERR_ARG
 
 
+def test_projection_replays_from_a_cuda_graph():
+    """The projection issues only stream work (kernels, device copies, memsets): captured once into a CUDA graph, it
+    replays on new contents of the same buffers and returns what the direct call returns."""
+    import torch
+    from tests.gpu_util import context, ct_dev, dev, host, key_dev
+    log_n, L, K, dnum, level, d_in, d_out, T, S, B = 10, 4, 2, 2, 4, 64, 64, 8, 2, 32
+    P, ctx = params(log_n, L, K, dnum), context(log_n, L, K, dnum)
+    o = P.oracle
+    cl = Client(P, 495)
+    scale = 2.0 ** 40
+    g = inputs.rng(495, 1)
+    W = dev(inputs.weights_normal(g, d_in, d_out, 0.02))
+    desc = ProjDesc(d_in, d_out, T, S, B)
+    keys = [key_dev(cl.rotation_key(o.galois_element(r)), o.galois_element(r)) for r in o.proj_rotations(desc)]
+
+    def fresh():
+        X = inputs.activations_uniform(g, S * T, d_in)
+        return [cl.encrypt_slots(inputs.pack_feature_major(X[c * T:(c + 1) * T], T, o.n)[0], scale, level) for c in range(S)]
+    first, second = fresh(), fresh()
+    cts = [ct_dev(c, scale) for c in first]
+    outs = [ctx.empty_ct(level - 1) for _ in range(S)]
+    ws = torch.empty(ctx.linear_proj_workspace_bytes(d_in, d_out, T, S, B, level, True), dtype=torch.uint8, device="cuda")
+    run = lambda: ctx.linear_proj(cts, W, keys, d_in, d_out, T, S, B, outs=outs, ws=ws, lazy_moddown=True)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        run()                                        # warm-up outside the capture
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        run()
+    for src in (second, first):
+        for c, h in zip(cts, src):
+            c.data.copy_(dev(h))
+        graph.replay()
+        replayed = [host(x.data).copy() for x in outs]
+        run()
+        for a, x in zip(replayed, outs):
+            assert np.array_equal(a, host(x.data))
+    assert ctx.device_status() == 0
+
+
 def test_projection_explicit_pt_scale_and_lower_level():
     _run(10, 4, 2, 2, 3, 16, 16, 32, 1, 4, seed=410, pt_scale=2.0 ** 40, check_slots=False)
 
