@@ -363,6 +363,39 @@ def test_softmax_by_doubling_bit_exact():
     assert e.value.code == binding.ERR_LEVEL
 
 
+def test_softmax_without_rounds_is_the_exponential_polynomial():
+    """rounds = 0: the shift and p_exp only, i.e. poly_eval_tree of x - shift; no rotation key is needed."""
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    P, ctx = params(10, 6, 2, 3), context(10, 6, 2, 3)
+    o = P.oracle
+    cl = Client(P, 74)
+    level, scale, shift = 6, 2.0 ** 50, 1.5
+    z = inputs.rng(74, 1).uniform(-1, 1, P.n)
+    ct = cl.encrypt_slots(z, scale, level)
+    rlk = cl.relin_key()
+    coeffs = [1.0, 0.5, 0.125, 0.02, 0.003]
+    want, ws = o.softmax_doubling(ct, scale, shift, 0, 16, coeffs, [], rlk, {})
+    tree, ts = o.poly_eval_tree(o.add_const(ct, int(np.rint(-shift * scale))), scale, coeffs, rlk)
+    assert np.array_equal(want, tree) and ws == ts
+    got = ctx.softmax(ct_dev(ct, scale), shift, 0, 16, coeffs, [], key_dev(rlk, 0), [])
+    assert got.scale == ws and np.array_equal(host(got.data), want)
+
+
+def test_rotate_batch_in_place():
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    P, ctx = params(10, 6, 2, 3), context(10, 6, 2, 3)
+    o = P.oracle
+    cl = Client(P, 320)
+    gal = o.galois_element(7)
+    key = cl.rotation_key(gal)
+    g = inputs.rng(321, 1)
+    cts = [cl.encrypt_slots(g.uniform(-1, 1, P.n), 2.0 ** 40, 4) for _ in range(3)]
+    d = [ct_dev(c, 2.0 ** 40) for c in cts]
+    ctx.rotate_batch(d, key_dev(key, gal), outs=d)
+    for i in range(3):
+        assert np.array_equal(host(d[i].data), o.rotate(cts[i], key, gal))
+
+
 def test_softmax_with_block_polynomials_bit_exact():
     """One round with degree-8 polynomials evaluated by baby steps and giant steps (blocks of 4)."""
     from tests.gpu_util import context, ct_dev, host, key_dev
