@@ -416,8 +416,8 @@ def run_cuda(args):
     hbm_achieved = ntt_bytes / (ntt_fwd_ms * 1e-3) / 1e9
     roofline = {"kernel": "ntt16_fwd_cols + ntt16_fwd_rows (forward NTT of 768 limbs, one launch each)", "bound": "alu",
                 "achieved": achieved, "peak": fp64_peak, "unit": "T FP64 instr/s", "frac": achieved / fp64_peak,
-                "traffic": 1538.0e6,   # ncu: dram read+write of the two launches (profiles/ntt16_768limbs.md), bytes
-                "fp64_pipe_active_ncu": {"ntt16_fwd_cols": 0.761, "ntt16_fwd_rows": 0.677},
+                "traffic": 1523.0e6,   # ncu: dram read+write of the two launches (profiles/ntt16_768limbs.md), bytes
+                "fp64_pipe_active_ncu": {"ntt16_fwd_cols": 0.761, "ntt16_fwd_rows": 0.670},
                 "peak_kind": "derived: 64 DFMA/clk/SM x %d SMs x %.0f MHz" % (sm_count, float(pk.get("sm_max_mhz", 1965.0))),
                 "ms_per_launch_pair": ntt_fwd_ms,
                 # the same fraction against the clock the SMs held under the power cap during the timed steps
@@ -426,7 +426,7 @@ def run_cuda(args):
                 "vs_register_resident_butterflies": {
                     "achieved_gbfly_s": limb_ntts * (N // 2) * LOG_N / (ntt_fwd_ms * 1e-3) / 1e9, "peak_gbfly_s": probe_rate / 1e9,
                     "frac": limb_ntts * (N // 2) * LOG_N / (ntt_fwd_ms * 1e-3) / probe_rate,
-                    "peak_kind": "measured in this run: the transform's radix-16 butterfly groups on registers, 4 CTAs x 256 threads per SM"},
+                    "peak_kind": "measured in this run: the transform's radix-16 butterfly groups on registers, 3 CTAs x 256 threads per SM"},
                 "hbm": {"achieved": hbm_achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": hbm_achieved / pk["hbm_gbs"],
                         "algorithmic_bytes": ntt_bytes, "peak_kind": pk_kind + " copy bandwidth"},
                 "others": ({"ntt16 family": "50.7 % of the step (profiles/bench_step_launch_list.md)",

@@ -148,7 +148,7 @@ int32_t ckks_intt(ckks_ctx *ctx, uint64_t *polys, uint32_t batch, uint32_t first
 
 /* Measurement aid (the paper has no counterpart): runs the forward butterflies of the N = 2^16 transform on
  * registers only -- `iters` groups of 4 stages (32 butterflies) per thread, with the transform's own range
- * reductions and twiddle fetches, on a grid of four 256-thread CTAs per SM -- so that a caller can time the
+ * reductions and twiddle fetches, on a grid of three 256-thread CTAs per SM -- so that a caller can time the
  * launch and compare the transform's butterflies per second with what the arithmetic alone sustains.
  * scratch: device, at least SMs * 1024 words, never written in practice.  *butterflies (host) receives the
  * number of butterflies of the launch.  CKKS_ERR_UNSUPPORTED unless log_n = 16. */

@@ -268,7 +268,7 @@ __device__ __forceinline__ void inv16_d(double (&x)[16], const double *__restric
 // ---- measurement aid: the forward butterflies of the N = 2^16 kernels on registers only ------------------
 // Every thread runs `iters` radix-16 groups (4 stages, 32 butterflies, with the same range reductions and twiddle
 // fetches, the latter from a 64 KiB window that stays in L1/L2) on 16 registers; nothing else touches memory.
-__global__ void __launch_bounds__(F_THREADS, 4) butterfly_probe_kernel(DevTables c, uint32_t iters, u64 *sink) {
+__global__ void __launch_bounds__(F_THREADS, 3) butterfly_probe_kernel(DevTables c, uint32_t iters, u64 *sink) {
     const double q = c.modd[0].x, qinv = c.modd[0].y;
     const double *tw = c.twd_fwd;
     double x[16];
@@ -287,7 +287,7 @@ __global__ void __launch_bounds__(F_THREADS, 4) butterfly_probe_kernel(DevTables
 
 // ---- forward, column pass (stages m = 1..128): CTA = strip of 16 columns -----------------
 template <bool ALLFP>
-__global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, const long long *coef_src) {
+__global__ void __launch_bounds__(F_THREADS, 3) ntt16_fwd_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, const long long *coef_src) {
     __shared__ u64 sm[256 * 16];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
@@ -347,7 +347,7 @@ constexpr uint32_t ROW_PAD = 256 + 16;
 
 // ---- forward, row pass (stages m = 256..32768): CTA = 16 rows, 16 threads per row ---------
 template <bool ALLFP, int EP>
-__global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, NttEpilogue ep) {
+__global__ void __launch_bounds__(F_THREADS, 3) ntt16_fwd_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, NttEpilogue ep) {
     constexpr int has_ep = EP;
     __shared__ u64 sm[16 * ROW_PAD];
     const int prime = limb_prime(map, blockIdx.y);
@@ -441,7 +441,7 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_fwd_rows(DevTables c, u64 
 
 // ---- inverse, row pass (stages m = 32768..256) ---------------------------------------------
 template <bool ALLFP>
-__global__ void __launch_bounds__(F_THREADS, 4) ntt16_inv_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, const u64 *src,
+__global__ void __launch_bounds__(F_THREADS, 3) ntt16_inv_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, const u64 *src,
                                                                 uint32_t src_pitch) {
     __shared__ u64 sm[16 * ROW_PAD];
     const int prime = limb_prime(map, blockIdx.y);
@@ -500,7 +500,7 @@ __global__ void __launch_bounds__(F_THREADS, 4) ntt16_inv_rows(DevTables c, u64 
 
 // ---- inverse, column pass (stages m = 128..1), then N^-1 and the exact reduction -----------
 template <bool ALLFP>
-__global__ void __launch_bounds__(F_THREADS, 4) ntt16_inv_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
+__global__ void __launch_bounds__(F_THREADS, 3) ntt16_inv_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
     __shared__ u64 sm[256 * 16];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
@@ -599,11 +599,11 @@ void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbM
     }
 }
 
-// grid: four CTAs per SM, the residency of the transform kernels.  Returns the butterflies one launch performs.
+// grid: three CTAs per SM, the residency of the transform kernels.  Returns the butterflies one launch performs.
 uint64_t launch_butterfly_probe(const ckks_ctx *c, uint32_t iters, u64 *sink, cudaStream_t s) {
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
-    const uint32_t ctas = (uint32_t)sms * 4;
+    const uint32_t ctas = (uint32_t)sms * 3;
     butterfly_probe_kernel<<<ctas, F_THREADS, 0, s>>>(c->dev, iters, sink);
     count_launches();
     return (uint64_t)ctas * F_THREADS * iters * 32;

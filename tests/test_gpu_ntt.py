@@ -76,7 +76,7 @@ def test_butterfly_probe_counts_and_errors():
     ctx = context(16, 24, 8, 3)
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     scratch = torch.zeros(sms * 1024, dtype=torch.int64, device="cuda").view(torch.uint64)
-    assert ctx.ntt_butterfly_probe(8, scratch) == sms * 4 * 256 * 8 * 32
+    assert ctx.ntt_butterfly_probe(8, scratch) == sms * 3 * 256 * 8 * 32
     torch.cuda.synchronize()
     assert int(scratch.view(torch.int64).abs().sum()) == 0          # the sink is never written
     with pytest.raises(binding.CkksError) as e:
