@@ -429,9 +429,9 @@ def run_cuda(args):
                     "peak_kind": "measured in this run: the transform's radix-16 butterfly groups on registers, 3 CTAs x 256 threads per SM"},
                 "hbm": {"achieved": hbm_achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": hbm_achieved / pk["hbm_gbs"],
                         "algorithmic_bytes": ntt_bytes, "peak_kind": pk_kind + " copy bandwidth"},
-                "others": ({"ntt16 family": "50.7 % of the step (profiles/bench_step_launch_list.md)",
-                            "mac_mma_kernel": "18.6 % of the step; legacy tensor path 32 % busy, DRAM 51 %, see profiles/mac_mma_projection_8shards.md",
-                            "modup + moddown_conv + inner_product(_terms)": "28.0 % of the step; FP64 pipe 67 % (conversions), DRAM 60-72 % (inner products)"}
+                "others": ({"ntt16 family": "49.6 % of the step (profiles/bench_step_launch_list.md)",
+                            "mac_mma_kernel": "19.3 % of the step; legacy tensor path 32 % busy, DRAM 51 %, see profiles/mac_mma_projection_8shards.md",
+                            "modup + moddown_conv + inner_product(_terms)": "28.3 % of the step; FP64 pipe 67 % (conversions), DRAM 60-72 % (inner products)"}
                            if LAZY else
                            {"ntt16 family": "55.0 % of the step (profiles/bench_step_launch_list.md)",
                             "mac_mma_kernel": "15.0 % of the step; legacy tensor path 32 % busy, DRAM 51 %, see profiles/mac_mma_projection_8shards.md",
