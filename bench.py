@@ -9,8 +9,9 @@ seeded synthetic inputs:
   (c) the Llama-3-8B-shaped projection: 128 tokens x 4096 features in 16 token-shard
       ciphertexts times a 4096 x 4096 fp64 weight matrix encoded on the fly
       (encode + ct x pt multiply-accumulate + hoisted/plain rotations + rescale).
-`value` is seconds per projection (part c); NTT limbs/s and key switches/s from parts
-(a) and (b) ride along in `submetrics`.  Ciphertexts and keys are uniform residues
+`value` is seconds per projection (part c); NTT limbs/s and key switches/s (plain rotations,
+each a complete key switch) from parts (a) and (b) ride along in `submetrics`, with a roofline
+fraction for each of the three paths (`roofline`, `roofline_keyswitch`, `roofline_projection`).  Ciphertexts and keys are uniform residues
 (what real ones look like to the kernels); weights N(0, 0.02), fp64.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
@@ -49,6 +50,75 @@ def peaks():
         return json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))), "measured"
     except Exception:
         return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0}, "fallback"
+
+
+def profile_figure(name, key):
+    """A figure recorded in a profiles/ summary as a line `key: number` (None if the file or the key is missing)."""
+    import re
+    try:
+        text = open(os.path.join(ROOT, "profiles", name)).read()
+    except OSError:
+        return None
+    m = re.search(r"^[-* ]*%s\s*[:=]\s*([0-9.eE+-]+)" % re.escape(key), text, re.M)
+    return float(m.group(1)) if m else None
+
+
+# ----------------------------------------------------------------- algorithmic work (what the rooflines count)
+BFLY = (N // 2) * LOG_N                 # butterflies of one limb transform
+FP64_PER_BFLY, FP64_PER_PAIR = 8, 7     # exact twiddle product + sum and difference; exact product of a conversion / key pair + add
+ALPHA = -(-L // DNUM)
+
+
+def ks_work(level=LEVEL, hoisted=False):
+    """Limb transforms and multiply-add pairs (per coefficient products of basis conversion, key inner product and the
+    ModDown tail) of one key switch at `level`; hoisted: without the shared inverse transform, ModUp and its transforms."""
+    beta, nt = -(-level // ALPHA), level + K
+    own = [min(ALPHA, level - j * ALPHA) for j in range(beta)]
+    up_ntt = level + sum(nt - d for d in own)
+    up_pairs = sum(d * (nt - d) + d for d in own)                  # conversions and the y = d qhat^-1 products
+    ip_pairs = beta * 2 * nt
+    dn_ntt = 2 * K + 2 * level
+    dn_pairs = 2 * (K * level + K) + 2 * level                     # conversions, y products, the (u - conv) P^-1 tail
+    ntt = dn_ntt + (0 if hoisted else up_ntt)
+    pairs = ip_pairs + dn_pairs + (0 if hoisted else up_pairs)
+    return {"limb_ntts": ntt, "pairs_per_coeff": pairs, "fp64_instr": ntt * BFLY * FP64_PER_BFLY + pairs * N * FP64_PER_PAIR,
+            "modup": {"limb_ntts": up_ntt, "pairs_per_coeff": up_pairs}, "moddown": {"limb_ntts": dn_ntt, "pairs_per_coeff": dn_pairs},
+            "inner": {"pairs_per_coeff": ip_pairs}}
+
+
+def instr_of(limb_ntts, pairs_per_coeff):
+    return limb_ntts * BFLY * FP64_PER_BFLY + pairs_per_coeff * N * FP64_PER_PAIR
+
+
+def projection_work(lazy, shards=SHARDS):
+    """Algorithmic work of the 4096 x 4096 projection: FP64 instructions of everything transform- or conversion-shaped,
+    and the multiply-accumulate as the bytes that must cross HBM once (plaintexts, baby ciphertexts, accumulators)."""
+    G = HIDDEN // BABY
+    ks, ksh = ks_work(), ks_work(hoisted=True)
+    limb = 8 * N
+    parts = {
+        "encode": {"count": HIDDEN, "fp64_instr": HIDDEN * instr_of(LEVEL, 0)},
+        "baby_modup": {"count": shards, "fp64_instr": shards * instr_of(**ks["modup"])},
+        "baby_hoisted_rotations": {"count": shards * (BABY - 1), "fp64_instr": shards * (BABY - 1) * ksh["fp64_instr"]},
+        "rescale": {"count": shards, "fp64_instr": shards * instr_of(2 + 2 * (LEVEL - 1), 2 * (LEVEL - 1))},
+        "mac": {"count": HIDDEN * shards,
+                "hbm_bytes": HIDDEN * LEVEL * limb + shards * BABY * 2 * LEVEL * limb + shards * G * 2 * LEVEL * limb},
+    }
+    if lazy:
+        term = instr_of(ks["modup"]["limb_ntts"], ks["modup"]["pairs_per_coeff"] + ks["inner"]["pairs_per_coeff"] + 1)
+        parts["giant_terms"] = {"count": shards * (G - 1), "fp64_instr": shards * (G - 1) * term}
+        parts["giant_moddown"] = {"count": shards, "fp64_instr": shards * instr_of(**ks["moddown"])}
+    else:
+        parts["giant_rotations"] = {"count": shards * (G - 1), "fp64_instr": shards * (G - 1) * ks["fp64_instr"]}
+    return parts
+
+
+def bound_ms(parts, fp64_peak_t, hbm_gbs):
+    """Time the parts would take at the FP64 instruction peak (T instr/s) and, for the multiply-accumulate, at the HBM peak."""
+    t = 0.0
+    for v in parts.values():
+        t += v.get("fp64_instr", 0) / (fp64_peak_t * 1e12) + v.get("hbm_bytes", 0) / (hbm_gbs * 1e9)
+    return t * 1e3
 
 
 # ----------------------------------------------------------------- clock sampling
@@ -99,37 +169,66 @@ def oracle_sample(lazy=True):
     g = inputs.rng(1004, 0)
     allp = list(q) + list(p)
     ct = inputs.uniform_residues(g, q, N, 2)
-    keys = [inputs.uniform_residues(g, allp, N, DNUM * 2).reshape(DNUM, 2, L + K, N) for _ in range(2)]
-    gals = [orc.galois_element(8), orc.galois_element(512)]
+    keys = [inputs.uniform_residues(g, allp, N, DNUM * 2).reshape(DNUM, 2, L + K, N) for _ in range(3)]
+    gals = [orc.galois_element(8), orc.galois_element(512), orc.galois_element(16)]
     z = np.repeat(g.normal(0, 0.02, HIDDEN), T_SHARD)
     t = {}
     t0 = time.perf_counter(); pts = [orc.encode(z, float(q[-1]), LEVEL) for _ in range(2)]; t["encode"] = (time.perf_counter() - t0) / 2
     t0 = time.perf_counter(); acc = orc.mul_plain_acc(ct, pts[0]); acc = orc.mul_plain_acc(ct, pts[1], acc); t["mac"] = (time.perf_counter() - t0) / 2
-    t0 = time.perf_counter(); orc.rotate_hoisted(ct, keys, gals); t["hoisted_2"] = time.perf_counter() - t0
+    t0 = time.perf_counter(); orc.rotate_hoisted(ct, keys[:1], gals[:1]); t["hoisted_1"] = time.perf_counter() - t0
+    t0 = time.perf_counter(); orc.rotate_hoisted(ct, keys, gals); t["hoisted_3"] = time.perf_counter() - t0
     t0 = time.perf_counter(); orc.rotate(ct, keys[0], gals[0]); t["rotate"] = time.perf_counter() - t0
-    t0 = time.perf_counter(); orc.rotate_sum(np.stack([ct, ct]), keys, gals); t["rotate_sum_2"] = time.perf_counter() - t0
+    t0 = time.perf_counter(); orc.rotate_sum(np.stack([ct, ct]), keys[:2], gals[:2]); t["rotate_sum_2"] = time.perf_counter() - t0
     t0 = time.perf_counter(); orc.rescale(acc); t["rescale"] = time.perf_counter() - t0
     t0 = time.perf_counter(); x = inputs.uniform_residues(g, q, N, 1); orc.intt(orc.ntt(x)); t["ntt_pair_24"] = time.perf_counter() - t0
     G = HIDDEN // BABY
-    # a hoisted rotation costs (hoisted_2 - shared ModUp)/2; approximate the shared part by rotate - per-rotation part
-    per_h = t["hoisted_2"] / 2
+    # hoisted rotations: three cost the shared ModUp plus three per-rotation parts, one costs the ModUp plus one
+    per_h = max(t["hoisted_3"] - t["hoisted_1"], 0.0) / 2
+    shared_up = max(t["hoisted_1"] - per_h, 0.0)
     # a two-term rotate_sum is two extended-basis terms and one ModDown, a rotation one term and one ModDown
     term = max(t["rotate_sum_2"] - t["rotate"], 0.0)
     moddown = max(t["rotate"] - term, 0.0)
     giant = (G - 1) * term + moddown if lazy else (G - 1) * t["rotate"]
-    proj = (HIDDEN * t["encode"] + HIDDEN * SHARDS * t["mac"] + SHARDS * (BABY - 1) * per_h
+    proj = (HIDDEN * t["encode"] + HIDDEN * SHARDS * t["mac"] + SHARDS * (shared_up + (BABY - 1) * per_h)
             + SHARDS * giant + SHARDS * t["rescale"])
     cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
-    sample = ("2 encodes, 2 ct x pt MACs, 2 hoisted + 1 plain rotation, 1 two-term rotate_sum, 1 rescale, 24 NTT round trips at "
-              "full size; scaled by the projection's counts (4096 encodes, 65536 MACs, 1008 hoisted rotations, "
+    sample = ("2 encodes, 2 ct x pt MACs, hoisted rotations by 1 and by 3 keys, 1 plain rotation, 1 two-term rotate_sum, 1 rescale, "
+              "24 NTT round trips at full size; scaled by the projection's counts (4096 encodes, 65536 MACs, 16 ModUps + 1008 hoisted rotations, "
               + ("1008 giant-step terms + 16 ModDowns" if lazy else "1008 plain rotations") + ", 16 rescales)")
     return {"proj_s": proj, "ntt_limbs_per_s": 48 / t["ntt_pair_24"], "key_switches_per_s": 1.0 / t["rotate"],
             "parts_s": t, "cores": cores, "sample": sample}
 
 
+def oracle_one_shard(lazy=True):
+    """One whole token shard of the 4096 x 4096 projection through the checker (all 4096 diagonals encoded, 4096
+    multiply-accumulates, 63 hoisted and 63 giant-step rotations, one rescale): seconds."""
+    import numpy as np
+
+    from oracle.ckks_oracle import Oracle, ProjDesc
+    from paper_2609_12378_b200 import inputs
+
+    q, p = inputs.prime_chain(LOG_N, L, K)
+    orc = Oracle(LOG_N, q, p, DNUM)
+    g = inputs.rng(1004, 5)
+    allp = list(q) + list(p)
+    desc = ProjDesc(HIDDEN, HIDDEN, T_SHARD, 1, BABY, lazy_moddown=lazy)
+    ct = inputs.uniform_residues(g, q, N, 2)
+    W = inputs.weights_normal(g, HIDDEN, HIDDEN, 0.02)
+    key = inputs.uniform_residues(g, allp, N, DNUM * 2).reshape(DNUM, 2, L + K, N)      # one key stands in for all 126: same work
+    keys = {orc.galois_element(r): key for r in orc.proj_rotations(desc)}
+    t0 = time.perf_counter()
+    orc.linear_proj(desc, ct[None], W, keys, 2.0 ** 40)
+    return time.perf_counter() - t0
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
+        return
+    if args.cpu_anchor:
+        sec = oracle_one_shard(LAZY)
+        print(json.dumps({"impl": "reference", "one_shard_seconds": sec,
+                          "cores": int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))}))
         return
     for _ in range(args.warmup if args.warmup < 2 else 1):
         oracle_sample(LAZY)
@@ -159,12 +258,18 @@ def max_over_ranks(values, device="cpu"):
     return t.tolist()
 
 
-def job_metrics(world, a_ms, b_ms, c_ms):
-    """Whole-job figures from the slowest rank's part times: every rank ran the same step on its own replica."""
+def job_metrics(world, a_ms, plain_ms, c_ms, hoisted_ms=None, relin_ms=None):
+    """Whole-job figures from the slowest rank's part times: every rank ran the same step on its own replica.
+    plain_ms: the NROT plain rotations (each a complete key switch); hoisted_ms: the same NROT off one shared ModUp."""
     limb_ntts = NTT_BATCH * L
-    return {"value": c_ms * 1e-3 / world,                                   # seconds per projection, all ranks together
-            "ntt_limbs_per_s": world * 2 * limb_ntts / (a_ms * 1e-3),
-            "key_switches_per_s": world * (2 * NROT + 1) / (b_ms * 1e-3)}
+    out = {"value": c_ms * 1e-3 / world,                                   # seconds per projection, all ranks together
+           "ntt_limbs_per_s": world * 2 * limb_ntts / (a_ms * 1e-3),
+           "key_switches_per_s": world * NROT / (plain_ms * 1e-3)}
+    if hoisted_ms:
+        out["hoisted_rotations_per_s"] = world * NROT / (hoisted_ms * 1e-3)
+    if relin_ms:
+        out["mul_relin_per_s"] = world / (relin_ms * 1e-3)
+    return out
 
 
 # ----------------------------------------------------------------- CUDA leg
@@ -224,23 +329,30 @@ def run_cuda(args):
         ctx.ntt(polys, 0)
         ctx.intt(polys, 0)
 
-    def part_b():
+    def part_b1():
         for k in rot_keys:
             ctx.rotate(cta, k, out=rot_out)
+
+    def part_b2():
         ctx.rotate_hoisted(cta, rot_keys, outs=hoist_out)
+
+    def part_b3():
         ctx.mul_relin(cta, ctb, rlk, out=mul_out)
+
+    def part_b():
+        part_b1(); part_b2(); part_b3()
 
     def part_c():
         ctx.linear_proj(cts, W, proj_keys, HIDDEN, HIDDEN, T_SHARD, SH, BABY, outs=outs, ws=ws, lazy_moddown=LAZY)
 
     def step(times=None):
-        e = [ev() for _ in range(4)]
+        e = [ev() for _ in range(6)]
         if args.profile:
             for name, f in (("a", part_a), ("b", part_b), ("c", part_c)):
                 if name in args.parts:
                     f()
             return
-        e[0].record(); part_a(); e[1].record(); part_b(); e[2].record(); part_c(); e[3].record()
+        e[0].record(); part_a(); e[1].record(); part_b1(); e[4].record(); part_b2(); e[5].record(); part_b3(); e[2].record(); part_c(); e[3].record()
         if times is not None:
             times.append(e)
 
@@ -274,6 +386,24 @@ def run_cuda(args):
     a_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in times)
     b_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in times)
     c_ms = statistics.mean(e[2].elapsed_time(e[3]) for e in times)
+    b1_ms = statistics.mean(e[1].elapsed_time(e[4]) for e in times)
+    b2_ms = statistics.mean(e[4].elapsed_time(e[5]) for e in times)
+    b3_ms = statistics.mean(e[5].elapsed_time(e[2]) for e in times)
+
+    # the other giant-step schedule (one ModDown per rotation if the step timed the lazy form, and the reverse), with the
+    # same statistics: the same number of calls, one event pair each, mean
+    def part_c_other():
+        ctx.linear_proj(cts, W, proj_keys, HIDDEN, HIDDEN, T_SHARD, SH, BABY, outs=outs, ws=ws, lazy_moddown=not LAZY)
+
+    part_c_other()
+    torch.cuda.synchronize()
+    other = []
+    for _ in range(args.steps):
+        a_, b_ = ev(), ev()
+        a_.record(); part_c_other(); b_.record()
+        other.append((a_, b_))
+    torch.cuda.synchronize()
+    c_other_ms = statistics.mean(a_.elapsed_time(b_) for a_, b_ in other)
 
     # dominant-kernel roofline leg: the NTT kernel pair timed alone on the launching stream
     s0, s1 = ev(), ev()
@@ -294,7 +424,7 @@ def run_cuda(args):
     torch.cuda.synchronize()
     probe_rate = probe_bfly / (p0.elapsed_time(p1) * 1e-3)          # butterflies per second
 
-    # outside the step, once each: the two composite calls that go beyond the scope table's rows
+    # outside the step, once each after a warm-up call: the composite calls built on the step's primitives
     def once(f):
         f()
         torch.cuda.synchronize()
@@ -305,8 +435,6 @@ def run_cuda(args):
 
     extras = {}
     if rank == 0 and not args.no_extras:
-        extras["projection_%s_moddown_ms" % ("eager" if LAZY else "lazy")] = once(
-            lambda: ctx.linear_proj(cts, W, proj_keys, HIDDEN, HIDDEN, T_SHARD, SH, BABY, outs=outs, ws=ws, lazy_moddown=not LAZY))
         Wk = (torch.randn((HIDDEN, HIDDEN // 4), generator=gen, device=dev, dtype=torch.float64) * 0.02).contiguous()
         Wv = (torch.randn((HIDDEN, HIDDEN // 4), generator=gen, device=dev, dtype=torch.float64) * 0.02).contiguous()
         douts = [HIDDEN, HIDDEN // 4, HIDDEN // 4]
@@ -395,69 +523,183 @@ def run_cuda(args):
     barrier()
     e2e_pipe_ms = y0.elapsed_time(y1) / args.steps
 
-    total_ms, a_ms, b_ms, c_ms, e2e_ms, ntt_fwd_ms, e2e_pipe_ms = max_over_ranks([total_ms, a_ms, b_ms, c_ms, e2e_ms, ntt_fwd_ms, e2e_pipe_ms], dev)
+    (total_ms, a_ms, b_ms, c_ms, e2e_ms, ntt_fwd_ms, e2e_pipe_ms, b1_ms, b2_ms, b3_ms, c_other_ms) = max_over_ranks(
+        [total_ms, a_ms, b_ms, c_ms, e2e_ms, ntt_fwd_ms, e2e_pipe_ms, b1_ms, b2_ms, b3_ms, c_other_ms], dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
+    layer = None
+    if not args.no_extras and not args.no_layer:
+        del ws, h_cts, h_W, h_outs
+        ctx._ws = None
+        torch.cuda.empty_cache()
+        layer = layer_submetrics(ctx, residues, allp, gen, dev, args.layer_reps)
+
     pk, pk_kind = peaks()
     limb_ntts = NTT_BATCH * L
-    # Roofline of the dominant kernel family (the ntt16 kernels: 55 % of the step in the ncu launch list).
-    # The butterflies run on the FP64 pipe, which ncu shows to be the busiest unit of the column passes, so the
-    # bound is "alu": algorithmic work = 8 FP64 instructions per butterfly (6 for the exact twiddle product with
-    # its quotient, 2 for the sum and difference), N/2 * log2 N butterflies per limb; peak = 64 FP64 instructions
-    # per clock per SM (the DFMA rate ncu reports for this part) x SM count x the maximum SM clock.
     sm_count = torch.cuda.get_device_properties(local).multi_processor_count
-    fp64_peak = 64.0 * sm_count * float(pk.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12          # T instr/s
-    ops = limb_ntts * (N // 2) * LOG_N * 8
-    achieved = ops / (ntt_fwd_ms * 1e-3) / 1e12
+    sm_max = float(pk.get("sm_max_mhz", 1965.0))
+    # Every path here is bound by FP64 arithmetic ("alu"): butterflies and exact modular products run on the FP64 pipe.
+    # Peak = 64 FP64 instructions per clock per SM (the DFMA rate) x SM count x the maximum SM clock.  Algorithmic work =
+    # 8 instructions per butterfly (6 for the exact twiddle product with its quotient, 2 for sum and difference),
+    # N/2 log2 N butterflies per limb transform, and 7 per multiply-add pair of a basis conversion or key product.
+    fp64_peak = 64.0 * sm_count * sm_max * 1e6 / 1e12          # T instr/s
+    peak_kind = "derived: 64 DFMA/clk/SM x %d SMs x %.0f MHz" % (sm_count, sm_max)
+    clock_ratio = float(clocks["sm_mhz"]) / sm_max if clocks and clocks.get("sm_mhz") else None
+
+    def alu(instr, ms):
+        ach = instr / (ms * 1e-3) / 1e12
+        return {"bound": "alu", "achieved": ach, "peak": fp64_peak, "unit": "T FP64 instr/s", "frac": ach / fp64_peak,
+                "frac_at_sampled_clock": ach / (fp64_peak * clock_ratio) if clock_ratio else None, "peak_kind": peak_kind}
+
+    # (1) dominant kernel pair: forward transform of 768 limbs, timed alone
+    ops = limb_ntts * BFLY * FP64_PER_BFLY
     ntt_bytes = limb_ntts * 2 * 8 * N          # algorithmic bytes: each limb read once and written once
     hbm_achieved = ntt_bytes / (ntt_fwd_ms * 1e-3) / 1e9
-    roofline = {"kernel": "ntt16_fwd_cols + ntt16_fwd_rows (forward NTT of 768 limbs, one launch each)", "bound": "alu",
-                "achieved": achieved, "peak": fp64_peak, "unit": "T FP64 instr/s", "frac": achieved / fp64_peak,
-                "traffic": 1523.0e6,   # ncu: dram read+write of the two launches (profiles/ntt16_768limbs.md), bytes
-                "fp64_pipe_active_ncu": {"ntt16_fwd_cols": 0.761, "ntt16_fwd_rows": 0.670},
-                "peak_kind": "derived: 64 DFMA/clk/SM x %d SMs x %.0f MHz" % (sm_count, float(pk.get("sm_max_mhz", 1965.0))),
-                "ms_per_launch_pair": ntt_fwd_ms,
-                # the same fraction against the clock the SMs held under the power cap during the timed steps
-                "frac_at_sampled_clock": (achieved / (fp64_peak * float(clocks["sm_mhz"]) / float(pk.get("sm_max_mhz", 1965.0)))
-                                          if clocks and clocks.get("sm_mhz") else None),
-                "vs_register_resident_butterflies": {
-                    "achieved_gbfly_s": limb_ntts * (N // 2) * LOG_N / (ntt_fwd_ms * 1e-3) / 1e9, "peak_gbfly_s": probe_rate / 1e9,
-                    "frac": limb_ntts * (N // 2) * LOG_N / (ntt_fwd_ms * 1e-3) / probe_rate,
-                    "peak_kind": "measured in this run: the transform's radix-16 butterfly groups on registers, 3 CTAs x 256 threads per SM"},
-                "hbm": {"achieved": hbm_achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": hbm_achieved / pk["hbm_gbs"],
-                        "algorithmic_bytes": ntt_bytes, "peak_kind": pk_kind + " copy bandwidth"},
-                "others": ({"ntt16 family": "49.6 % of the step (profiles/bench_step_launch_list.md)",
-                            "mac_mma_kernel": "19.3 % of the step; legacy tensor path 32 % busy, DRAM 51 %, see profiles/mac_mma_projection_8shards.md",
-                            "modup + moddown_conv + inner_product(_terms)": "28.3 % of the step; FP64 pipe 67 % (conversions), DRAM 60-72 % (inner products)"}
-                           if LAZY else
-                           {"ntt16 family": "55.0 % of the step (profiles/bench_step_launch_list.md)",
-                            "mac_mma_kernel": "15.0 % of the step; legacy tensor path 32 % busy, DRAM 51 %, see profiles/mac_mma_projection_8shards.md",
-                            "modup + moddown_conv + inner_product": "27.8 % of the step; FP64 pipe 67 % (conversions), DRAM 72 % (inner product)"})}
+    roofline = alu(ops, ntt_fwd_ms)
+    roofline.update({
+        "kernel": "ntt16_fwd_cols + ntt16_fwd_rows (forward NTT of 768 limbs, one launch each)",
+        # ncu, dram read + write bytes of the two launches; None when no capture of the current kernels is recorded
+        "traffic": profile_figure("ntt16_768limbs.md", "dram_bytes_per_launch_pair"),
+        "ms_per_launch_pair": ntt_fwd_ms,
+        "vs_register_resident_butterflies": {
+            "achieved_gbfly_s": limb_ntts * BFLY / (ntt_fwd_ms * 1e-3) / 1e9, "peak_gbfly_s": probe_rate / 1e9,
+            "frac": limb_ntts * BFLY / (ntt_fwd_ms * 1e-3) / probe_rate,
+            "peak_kind": "measured in this run: the transform's radix-16 butterfly groups on registers, 3 CTAs x 256 threads per SM"},
+        "hbm": {"achieved": hbm_achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": hbm_achieved / pk["hbm_gbs"],
+                "algorithmic_bytes": ntt_bytes, "peak_kind": pk_kind + " copy bandwidth"}})
+    # (2) key switching: one plain rotation = one complete key switch; the hoisted form shares the ModUp
+    ks, ksh = ks_work(), ks_work(hoisted=True)
+    ks_bytes = (2 * LEVEL + DNUM * 2 * (L + K) + 2 * LEVEL) * 8 * N          # ciphertext in, key, ciphertext out
+    roofline_ks = alu(ks["fp64_instr"], b1_ms / NROT)
+    roofline_ks.update({
+        "per": "plain rotation (ckks_rotate, one ciphertext per call)", "us": b1_ms / NROT * 1e3,
+        "work": {"limb_ntts": ks["limb_ntts"], "mul_add_pairs": ks["pairs_per_coeff"] * N, "fp64_instr": ks["fp64_instr"]},
+        "hbm": {"achieved": ks_bytes / (b1_ms / NROT * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                "frac": ks_bytes / (b1_ms / NROT * 1e-3) / 1e9 / pk["hbm_gbs"], "algorithmic_bytes": ks_bytes},
+        "hoisted": dict(alu(ksh["fp64_instr"] + instr_of(**ks["modup"]) / NROT, b2_ms / NROT), us=b2_ms / NROT * 1e3,
+                        per="rotation off a ModUp shared by %d (ckks_rotate_hoisted)" % NROT),
+        "mul_relin": dict(alu(ks["fp64_instr"], b3_ms), us=b3_ms * 1e3)})
+    # (3) the projection: everything transform- or conversion-shaped at the FP64 peak, the multiply-accumulate at the
+    # HBM peak (its operands and results crossing HBM once); fraction = that time / measured time
+    def proj_roofline(lazy, ms):
+        parts = projection_work(lazy, SH)
+        bnd = bound_ms(parts, fp64_peak, pk["hbm_gbs"])
+        return {"bound": "alu + hbm (multiply-accumulate)", "bound_ms": bnd, "measured_ms": ms, "frac": bnd / ms,
+                "frac_at_sampled_clock": (bound_ms(parts, fp64_peak * clock_ratio, pk["hbm_gbs"]) / ms) if clock_ratio else None,
+                "schedule": "giant steps summed before one ModDown" if lazy else "one ModDown per giant-step rotation",
+                "parts_bound_ms": {k: bound_ms({k: v}, fp64_peak, pk["hbm_gbs"]) for k, v in parts.items()},
+                "peak_kind": peak_kind + "; " + pk_kind + " copy bandwidth %.0f GB/s" % pk["hbm_gbs"]}
+    roofline_proj = proj_roofline(LAZY, c_ms)
+    roofline_proj["other_schedule"] = proj_roofline(not LAZY, c_other_ms)
+
     cpu = oracle_sample(LAZY)
-    jm = job_metrics(world, a_ms, b_ms, c_ms)
+    jm = job_metrics(world, a_ms, b1_ms, c_ms, b2_ms, b3_ms)
+    sub = {"ntt_limbs_per_s": jm["ntt_limbs_per_s"], "key_switches_per_s": jm["key_switches_per_s"],
+           "hoisted_rotations_per_s": jm["hoisted_rotations_per_s"], "mul_relin_per_s": jm["mul_relin_per_s"],
+           "ms": {"ntt_roundtrip": a_ms, "keyswitch_part": b_ms, "plain_rotations_%d" % NROT: b1_ms, "hoisted_rotations_%d" % NROT: b2_ms,
+                  "mul_relin": b3_ms, "projection": c_ms,
+                  "projection_%s_moddown" % ("eager" if LAZY else "lazy"): c_other_ms}}
+    if layer:
+        sub["layer"] = layer
     line = {
         "metric": METRIC, "value": jm["value"], "unit": "s/projection", "n_gpus": world, "steps": args.steps,
         "warmup": nwarm, "ms_per_step": total_ms / args.steps, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "u64", "data": "synthetic",
         "config": {"workload": workload(), "l2": "inputs larger than L2 (>= 384 MiB per part)", "parallelism": f"replicas x{world}"},
         "extras": extras,
-        "submetrics": {"ntt_limbs_per_s": jm["ntt_limbs_per_s"], "key_switches_per_s": jm["key_switches_per_s"],
-                       "ms": {"ntt_roundtrip": a_ms, "keyswitch_part": b_ms, "projection": c_ms}},
+        "submetrics": sub,
         "clocks": clocks,
         "e2e": {"value": e2e_ms * 1e-3 / world, "unit": "s/projection", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "copies_overlapped_value": e2e_pipe_ms * 1e-3 / world},
         "gpu_launches": launches,
         "roofline": roofline,
+        "roofline_keyswitch": roofline_ks,
+        "roofline_projection": roofline_proj,
         "cpu_baseline": {"value": cpu["proj_s"], "unit": "s/projection", "cores": cpu["cores"], "kind": "oracle",
-                         "sample": cpu["sample"], "ntt_limbs_per_s": cpu["ntt_limbs_per_s"],
-                         "key_switches_per_s": cpu["key_switches_per_s"]},
+                         "method": "extrapolated from a timed sample by operation counts", "sample": cpu["sample"],
+                         "ntt_limbs_per_s": cpu["ntt_limbs_per_s"], "key_switches_per_s": cpu["key_switches_per_s"],
+                         # one whole shard of this projection through the checker, timed once on a B200 host (16 cores) and
+                         # recorded with its command: x 16 shards = what the extrapolation should land near
+                         "one_shard_anchor_s": profile_figure("oracle_one_shard.md", "one_shard_seconds")},
+        # figures copied from ncu captures (profiles/), with the kernels they were taken on: not measured in this run
+        "static_notes": {"source": "profiles/bench_step_launch_list.md, profiles/ntt16_768limbs.md",
+                         "ntt16_family_share_of_step": profile_figure("bench_step_launch_list.md", "ntt16_family_share"),
+                         "mac_share_of_step": profile_figure("bench_step_launch_list.md", "mac_share"),
+                         "keyswitch_kernels_share_of_step": profile_figure("bench_step_launch_list.md", "keyswitch_kernels_share"),
+                         "fp64_pipe_active_fwd_cols": profile_figure("ntt16_768limbs.md", "fp64_pipe_active_fwd_cols"),
+                         "fp64_pipe_active_fwd_rows": profile_figure("ntt16_768limbs.md", "fp64_pipe_active_fwd_rows")},
     }
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------- one decoder layer's linear work and products
+def layer_submetrics(ctx, residues, allp, gen, dev, reps):
+    """CUDA-event means of one Llama-3-8B decoder layer's homomorphic linear work at 128 tokens (16 shards of 8, B = 64,
+    giant steps summed before one ModDown): query/key/value as one call sharing their baby steps, output, gate and up as
+    one call, down; and the attention products as ciphertext x ciphertext multiplies at level 24: 2048 + 2048 products,
+    128 summed per output ciphertext with one relinearisation (ckks_mul_relin_sum), and the same count relinearised one
+    by one in batches (ckks_mul_relin_batch).  Synthetic operands (uniform residues, normal weights)."""
+    import torch
+
+    from paper_2609_12378_b200 import binding
+
+    KV, FFN = 1024, 14336
+
+    def weights(d_in, d_out):
+        return (torch.randn((d_in, d_out), generator=gen, device=dev, dtype=torch.float64) * 0.02).contiguous()
+
+    def keys_for(shapes):
+        rots = sorted(set(r for d_in, d_out in shapes for r in ctx.linear_proj_rotations(d_in, d_out, T_SHARD, SHARDS, BABY)))
+        return [binding.SwitchKey(residues(allp, DNUM, 2), ctx.galois_element(r)) for r in rots]
+
+    def timed(f):
+        f()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); f(); b.record()
+            ts.append((a, b))
+        torch.cuda.synchronize()
+        return statistics.mean(a.elapsed_time(b) for a, b in ts)
+
+    out = {"reps": reps, "ms": {}}
+    cts = [binding.Ciphertext(residues(allp[:L], 2), 2.0 ** 40) for _ in range(SHARDS)]
+    for name, d_outs in (("qkv", [HIDDEN, KV, KV]), ("o", [HIDDEN]), ("gate_up", [FFN, FFN])):
+        keys = keys_for([(HIDDEN, d) for d in d_outs])
+        Ws = [weights(HIDDEN, d) for d in d_outs]
+        out["ms"][name] = timed(lambda: ctx.linear_proj_multi(cts, Ws, keys, HIDDEN, d_outs, T_SHARD, SHARDS, BABY, lazy_moddown=True))
+        del keys, Ws
+        ctx._ws = None
+        torch.cuda.empty_cache()
+    del cts
+    nib = -(-FFN // HIDDEN)
+    cts = [binding.Ciphertext(residues(allp[:L], 2), 2.0 ** 40) for _ in range(SHARDS * nib)]
+    keys = keys_for([(FFN, HIDDEN)])
+    W = weights(FFN, HIDDEN)
+    out["ms"]["down"] = timed(lambda: ctx.linear_proj(cts, W, keys, FFN, HIDDEN, T_SHARD, SHARDS, BABY, lazy_moddown=True))
+    out["down_workspace_gib"] = ctx.linear_proj_workspace_bytes(FFN, HIDDEN, T_SHARD, SHARDS, BABY, LEVEL, True) / 2 ** 30
+    del cts, keys, W
+    ctx._ws = None
+    torch.cuda.empty_cache()
+    out["projections_s"] = sum(out["ms"][k] for k in ("qkv", "o", "gate_up", "down")) * 1e-3
+    # attention products: 16 distinct operands, 128 pairs per output ciphertext, 16 outputs for QK^T and 16 for PV
+    a = [binding.Ciphertext(residues(allp[:L], 2), 2.0 ** 40) for _ in range(16)]
+    b = [binding.Ciphertext(residues(allp[:L], 2), 2.0 ** 40) for _ in range(16)]
+    rlk = binding.SwitchKey(residues(allp, DNUM, 2), 0)
+    pa, pb = [a[i % 16] for i in range(128)], [b[(3 * i + i // 16) % 16] for i in range(128)]
+    acc = ctx.empty_ct(LEVEL)
+    out["ms"]["products_2x2048_summed_128_per_output"] = timed(lambda: [ctx.mul_relin_sum(pa, pb, rlk, out=acc) for _ in range(32)])
+    bouts = [ctx.empty_ct(LEVEL) for _ in range(16)] * 8
+    bws = ctx.workspace(ctx.workspace_bytes(binding.OP_MUL_RELIN_BATCH, LEVEL, 128))
+    out["ms"]["products_2x2048_each_relinearised"] = timed(lambda: [ctx.mul_relin_batch(pa, pb, rlk, outs=bouts, ws=bws) for _ in range(32)])
+    out["layer_linear_and_products_s"] = out["projections_s"] + out["ms"]["products_2x2048_summed_128_per_output"] * 1e-3
+    return out
 
 
 def main():
@@ -471,6 +713,10 @@ def main():
     ap.add_argument("--eager-moddown", action="store_true",
                     help="one ModDown per giant-step rotation instead of one per output ciphertext")
     ap.add_argument("--no-extras", action="store_true", help="skip the untimed one-off measurements of the composite calls")
+    ap.add_argument("--no-layer", action="store_true", help="skip the decoder-layer submetrics (seven projections and the attention products)")
+    ap.add_argument("--layer-reps", type=int, default=3, help="timed repetitions of each decoder-layer call")
+    ap.add_argument("--cpu-anchor", action="store_true",
+                    help="with --impl reference: time the checker on one whole shard of the projection instead of the sample")
     ap.add_argument("--profile", action="store_true",
                     help="for profiler captures: honour --warmup below 3 and skip the e2e and CPU legs (prints no bench line)")
     args = ap.parse_args()

@@ -60,7 +60,7 @@ enum {
     CKKS_ERR_RANGE = -6,       /* encode: a scaled value does not fit 2^62                 */
     CKKS_ERR_UNSUPPORTED = -7, /* parameters outside what the kernels implement            */
     CKKS_ERR_CUDA = -8,        /* a CUDA runtime call failed (see ckks_last_cuda_error)    */
-    CKKS_ERR_TIMEOUT = -9      /* reserved for bounded device-side waits                   */
+    CKKS_ERR_TIMEOUT = -9      /* a bounded device-side wait gave up (see ckks_device_status) */
 };
 
 /* Operation selectors for ckks_workspace_bytes. */
@@ -121,6 +121,27 @@ const char *ckks_status_string(int32_t status);
 /* Text of the last CUDA error seen by this context ("" if none).  Host string owned by the context. */
 const char *ckks_last_cuda_error(const ckks_ctx *ctx);
 
+/* Options of a context: host-side state, read whenever a call is made (set them between calls, not while another
+ * thread is inside one).  None of them changes a result: every kernel variant is bit-identical.
+ *   CKKS_OPT_NTT_FP_SHARE   N = 2^16 transform: of every 8 limbs, how many run on the FP64 pipe (0..8, default 8).
+ *   CKKS_OPT_CONV_KERNEL    ModUp / ModDown basis conversions: CKKS_CONV_FP64 (default) or CKKS_CONV_TENSOR.
+ *   CKKS_OPT_MAC_KERNEL     the projection's multiply-accumulate: CKKS_MAC_MMA (default: mma.sync, 8 coefficients per
+ *                           CTA, a warp per coefficient), CKKS_MAC_MMA_ASYNC (the same joined by mbarriers instead of
+ *                           CTA-wide barriers), CKKS_MAC_MMA_SPLIT (two warps per coefficient), CKKS_MAC_MMA_HALF (4
+ *                           coefficients per CTA), CKKS_MAC_TCGEN05 (tcgen05.mma with TMEM accumulators, baby <= 64).
+ *   CKKS_OPT_WAIT_CYCLES    bound, in SM clock cycles, of every device-side wait on an mbarrier (default 2 * 10^9,
+ *                           about a second).  A wait that runs out makes its kernel drain its copies and return, and
+ *                           sets the sticky flag ckks_device_status reports; 0 makes every wait that is not already
+ *                           satisfied give up at once (used to test that path).
+ *   CKKS_OPT_STATIC_SCRATCH_BYTES  (read only) CKKS_STATIC_SCRATCH_BYTES of the loaded library.
+ * set returns CKKS_ERR_ARG for an unknown option or a value outside its range; get returns -1 for an unknown option. */
+enum { CKKS_OPT_NTT_FP_SHARE = 1, CKKS_OPT_CONV_KERNEL = 2, CKKS_OPT_MAC_KERNEL = 3, CKKS_OPT_WAIT_CYCLES = 4,
+       CKKS_OPT_STATIC_SCRATCH_BYTES = 5 };
+enum { CKKS_CONV_FP64 = 0, CKKS_CONV_TENSOR = 1 };
+enum { CKKS_MAC_MMA = 82, CKKS_MAC_MMA_ASYNC = 83, CKKS_MAC_MMA_SPLIT = 81, CKKS_MAC_MMA_HALF = 42, CKKS_MAC_TCGEN05 = 100 };
+int32_t ckks_context_set_option(ckks_ctx *ctx, int32_t option, int64_t value);
+int64_t ckks_context_get_option(const ckks_ctx *ctx, int32_t option);
+
 /* Bytes of caller-provided device workspace `op` needs at this level.  `count`
  * is the batch size for CKKS_OP_ENCODE, the number of rotations for
  * CKKS_OP_ROTATE_HOISTED, the degree for CKKS_OP_POLY_EVAL_TREE and the number
@@ -170,8 +191,9 @@ int32_t ckks_encode(ckks_ctx *ctx, const double *re, const double *im, uint32_t 
  * query overflowed (and clears the flag), else CKKS_OK. */
 int32_t ckks_encode_range_flag(ckks_ctx *ctx, void *stream);
 
-/* Synchronises `stream`; returns CKKS_ERR_TIMEOUT if a bounded device-side wait (the TMA pipeline of the
- * projection's multiply-accumulate) gave up since the last query (and clears the flag), else CKKS_OK. */
+/* Synchronises `stream`; returns CKKS_ERR_TIMEOUT if a bounded device-side wait (the mbarrier hand-offs of the
+ * projection's multiply-accumulate variants CKKS_MAC_MMA_ASYNC and CKKS_MAC_TCGEN05) gave up since the last query
+ * (and clears the flag), else CKKS_OK.  After a timeout the outputs of the call that hit it are undefined. */
 int32_t ckks_device_status(ckks_ctx *ctx, void *stream);
 
 /* ---- PCMult + Add (Section 2.1) -------------------------------------------
@@ -299,9 +321,10 @@ int32_t ckks_rotate_sum(ckks_ctx *ctx, const ckks_ct *in, const ckks_evk *keys, 
 
 /* Hoisted: one iNTT + ModUp + NTT of c1 shared by nrot rotations; rotation r
  * permutes the extended digits by sigma_{g_r}, takes the inner product with
- * keys[r], ModDown, adds sigma(c0).  As an integer function this differs from
- * ckks_rotate (same plaintext, different low noise bits).  keys, outs: host
- * arrays of nrot descriptors.  With the workspace ckks_workspace_bytes(CKKS_OP_ROTATE_HOISTED, level, nrot) asks
+ * keys[r], ModDown, adds sigma(c0).  Every outs[r] is bit-identical to
+ * ckks_rotate(in, keys[r]): the centred basis conversion is an odd function, so
+ * it commutes with the signed permutation sigma.  keys, outs: host arrays of
+ * nrot descriptors.  With the workspace ckks_workspace_bytes(CKKS_OP_ROTATE_HOISTED, level, nrot) asks
  * for, up to 16 rotations run side by side; any workspace of at least the CKKS_OP_ROTATE size is accepted.
  * Errors as ckks_rotate. */
 int32_t ckks_rotate_hoisted(ckks_ctx *ctx, const ckks_ct *in, const ckks_evk *keys, uint32_t nrot, ckks_ct *outs,

@@ -16,9 +16,13 @@ OK, ERR_ARG, ERR_LEVEL, ERR_SCALE, ERR_NO_KEY, ERR_WORKSPACE, ERR_RANGE, ERR_UNS
     0, -1, -2, -3, -4, -5, -6, -7, -8, -9)
 OP_ENCODE, OP_MUL_RELIN, OP_ROTATE, OP_ROTATE_HOISTED, OP_RESCALE, OP_LINEAR_PROJ, OP_POLY_EVAL, OP_POLY_EVAL_TREE, OP_MUL_RELIN_BATCH, OP_ROTATE_BATCH, OP_ROTATE_SUM = 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11
 PROJ_LAZY_MODDOWN = 1
+OPT_NTT_FP_SHARE, OPT_CONV_KERNEL, OPT_MAC_KERNEL, OPT_WAIT_CYCLES, OPT_STATIC_SCRATCH_BYTES = 1, 2, 3, 4, 5
+CONV_FP64, CONV_TENSOR = 0, 1
+MAC_MMA, MAC_MMA_ASYNC, MAC_MMA_SPLIT, MAC_MMA_HALF, MAC_TCGEN05 = 82, 83, 81, 42, 100
 
 EXPORTS = [
-    "ckks_context_create", "ckks_context_destroy", "ckks_status_string", "ckks_last_cuda_error",
+    "ckks_context_create", "ckks_context_destroy", "ckks_context_set_option", "ckks_context_get_option", "ckks_status_string",
+    "ckks_last_cuda_error",
     "ckks_workspace_bytes", "ckks_galois_element", "ckks_ntt", "ckks_intt", "ckks_encode",
     "ckks_encode_range_flag", "ckks_mul_plain_acc", "ckks_add", "ckks_mul_relin", "ckks_rotate",
     "ckks_rotate_hoisted", "ckks_rescale", "ckks_linear_proj", "ckks_linear_proj_workspace_bytes",
@@ -70,6 +74,8 @@ def load():
     sig = {
         "ckks_context_create": (i32, [C.POINTER(CParams), C.POINTER(vp)]),
         "ckks_context_destroy": (None, [vp]),
+        "ckks_context_set_option": (i32, [vp, i32, i64]),
+        "ckks_context_get_option": (i64, [vp, i32]),
         "ckks_status_string": (C.c_char_p, [i32]),
         "ckks_last_cuda_error": (C.c_char_p, [vp]),
         "ckks_workspace_bytes": (sz, [vp, i32, u32, u32]),
@@ -207,6 +213,12 @@ class Context:
     def _check(self, rc):
         if rc:
             raise CkksError(rc, load().ckks_last_cuda_error(self._h).decode() if rc == ERR_CUDA else "")
+
+    def set_option(self, option: int, value: int):
+        self._check(load().ckks_context_set_option(self._h, option, int(value)))
+
+    def get_option(self, option: int) -> int:
+        return int(load().ckks_context_get_option(self._h, option))
 
     def workspace(self, nbytes: int) -> torch.Tensor:
         """A cached device scratch buffer of at least nbytes (grown on demand by torch)."""

@@ -65,7 +65,11 @@ struct ckks_ctx {
     DevTables dev;               // pointers into `allocs`
     std::vector<void *> allocs;  // device allocations owned by the context
     std::string cuda_error;
-    uint32_t ntt_fp_share = 8;   // of every 8 limbs, how many take the double-precision NTT path (tuning knob)
+    // options (ckks_context_set_option); host-side state read when a call is made
+    uint32_t ntt_fp_share = 8;               // of every 8 limbs, how many take the double-precision NTT path
+    int conv_kernel = 0;                     // basis conversions: 0 = FP64 pipe, 1 = tensor cores (conv_mma.cu)
+    int mac_kernel = 82;                     // projection multiply-accumulate kernel (see launch_mac_mma)
+    long long wait_cycles = 2000000000ll;    // clock bound of every device-side wait (about a second)
 };
 
 // ---------------------------------------------------------------------------
@@ -304,6 +308,10 @@ bool mac_mma_supported(const ckks_ctx *c, uint32_t J);
 // accumulate: add to acc instead of overwriting it
 bool launch_mac_mma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level,
                     cudaStream_t s, uint32_t Jx = 0, uint32_t j0 = 0, bool accumulate = false);
+
+// the same contraction on the integer pipe, any J (mac_tile.cu): baby rows (s J + j) 2 + c, pts rows g J + j, both tiled
+void launch_mac_tile(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level,
+                     cudaStream_t s);
 
 // register-resident forward butterflies (measurement aid, ntt.cu); sink: device scratch of SMs * 4 * 256 words
 uint64_t launch_butterfly_probe(const ckks_ctx *c, uint32_t iters, u64 *sink, cudaStream_t s);

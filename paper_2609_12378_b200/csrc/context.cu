@@ -114,6 +114,43 @@ extern "C" void ckks_context_destroy(ckks_ctx *ctx) {
     delete ctx;
 }
 
+extern "C" int32_t ckks_context_set_option(ckks_ctx *ctx, int32_t option, int64_t value) {
+    if (!ctx) return CKKS_ERR_ARG;
+    switch (option) {
+        case CKKS_OPT_NTT_FP_SHARE:
+            if (value < 0 || value > 8) return CKKS_ERR_ARG;
+            ctx->ntt_fp_share = (uint32_t)value;
+            return CKKS_OK;
+        case CKKS_OPT_CONV_KERNEL:
+            if (value != CKKS_CONV_FP64 && value != CKKS_CONV_TENSOR) return CKKS_ERR_ARG;
+            ctx->conv_kernel = (int)value;
+            return CKKS_OK;
+        case CKKS_OPT_MAC_KERNEL:
+            if (value != CKKS_MAC_MMA && value != CKKS_MAC_MMA_ASYNC && value != CKKS_MAC_MMA_SPLIT && value != CKKS_MAC_MMA_HALF &&
+                value != CKKS_MAC_TCGEN05)
+                return CKKS_ERR_ARG;
+            ctx->mac_kernel = (int)value;
+            return CKKS_OK;
+        case CKKS_OPT_WAIT_CYCLES:
+            if (value < 0) return CKKS_ERR_ARG;
+            ctx->wait_cycles = (long long)value;
+            return CKKS_OK;
+        default: return CKKS_ERR_ARG;
+    }
+}
+
+extern "C" int64_t ckks_context_get_option(const ckks_ctx *ctx, int32_t option) {
+    if (!ctx) return -1;
+    switch (option) {
+        case CKKS_OPT_NTT_FP_SHARE: return ctx->ntt_fp_share;
+        case CKKS_OPT_CONV_KERNEL: return ctx->conv_kernel;
+        case CKKS_OPT_MAC_KERNEL: return ctx->mac_kernel;
+        case CKKS_OPT_WAIT_CYCLES: return ctx->wait_cycles;
+        case CKKS_OPT_STATIC_SCRATCH_BYTES: return (int64_t)CKKS_STATIC_SCRATCH_BYTES;
+        default: return -1;
+    }
+}
+
 extern "C" uint64_t ckks_galois_element(const ckks_ctx *ctx, int64_t r) {
     if (!ctx) return 0;
     int64_t n = (int64_t)ctx->n;
@@ -144,7 +181,6 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
     ckks_ctx *c = new ckks_ctx();
     c->log_n = prm->log_n; c->N = N; c->n = n; c->L = L; c->K = K; c->dnum = prm->dnum; c->alpha = alpha; c->T = T;
     c->device = prm->device;
-    if (const char *e = getenv("CKKS_NTT_FP_SHARE")) c->ntt_fp_share = (uint32_t)atoi(e);
     c->mod = mod;
     c->pow5.resize(n);
     c->pow5[0] = 1;

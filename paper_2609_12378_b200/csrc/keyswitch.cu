@@ -10,7 +10,6 @@
 //   5. ModDown: inverse NTT of the special limbs, centred conversion P -> q_i,
 //      NTT, out_i = (u_i - conv_i) * P^-1 mod q_i.
 // Rescale drops the last limb the same way with a single source limb.
-#include <cstring>
 #include "common.cuh"
 
 namespace {
@@ -389,11 +388,6 @@ __global__ void __launch_bounds__(THREADS) p_c0_acc_kernel(DevTables c, const u6
 
 }  // namespace
 
-static bool conv_on_tensor_cores() {
-    const char *e = getenv("CKKS_CONV");
-    return e && !strcmp(e, "mma");
-}
-
 size_t ks_workspace_limbs(const ckks_ctx *c, uint32_t level) {
     const size_t beta = (level + c->alpha - 1) / c->alpha, nt = level + c->K;
     return level + beta * nt + 2 * nt + 2 * (size_t)level;
@@ -419,8 +413,8 @@ void ks_modup(const ckks_ctx *c, const u64 *d, uint32_t level, const KsWorkspace
         permute_kernel<<<dim3(N / THREADS, level, nb), THREADS, 0, s>>>(c->dev, d, d_stride, w.dcoef, (size_t)level * N, 1); count_launches();
         launch_ntt(c, w.dcoef, nb * level, plain_map(0, level), true, s);
     }
-    // CKKS_CONV=mma (tuning knob) takes the tensor-core conversion of conv_mma.cu: bit-identical, 2 % slower on B200
-    if (!conv_on_tensor_cores() || !launch_modup_mma(c, w.dcoef, d, d_stride, w.ext, level, nb, s)) {
+    // the context option CKKS_CONV_TENSOR takes the tensor-core conversion of conv_mma.cu: bit-identical, 2 % slower on B200
+    if (c->conv_kernel != CKKS_CONV_TENSOR || !launch_modup_mma(c, w.dcoef, d, d_stride, w.ext, level, nb, s)) {
 #define CALL_UP(A) launch_modup<A>(c, w.dcoef, d, d_stride, 1, w.ext, level, nb, s)
         DISPATCH_POW2(c->alpha, CALL_UP);
 #undef CALL_UP
@@ -469,7 +463,7 @@ void ks_moddown(const ckks_ctx *c, uint32_t level, const KsWorkspace &w, const u
     const uint32_t N = c->N, nt = level + c->K, K = c->K;
     // the K special limbs of every (batch, component): groups of K limbs, nt limbs apart
     launch_ntt(c, w.u + (size_t)level * N, nb * 2 * K, pitched_map(c->L, K, nt), true, s);
-    if (!conv_on_tensor_cores() || !launch_moddown_conv_mma(c, w.u, w.conv, level, nb, s)) {
+    if (c->conv_kernel != CKKS_CONV_TENSOR || !launch_moddown_conv_mma(c, w.u, w.conv, level, nb, s)) {
 #define CALL_DN(A) launch_moddown_conv<A>(c, w.u, w.conv, level, nb, s)
         DISPATCH_POW2(K, CALL_DN);
 #undef CALL_DN

@@ -290,23 +290,25 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_cp_async(uint32_t bar) {
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(bar) : "memory");
 }
-constexpr long long MBAR_WAIT_CYCLES = 2000000000ll;      // about a second
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Bounded wait, called by all 32 lanes of a warp together; the verdict is the warp's (every lane gets the same answer, so
+// a timeout never splits a warp in front of a warp-wide instruction).  limit: SM clock cycles.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long limit) {
     const long long t0 = clock64();
+    uint32_t ok = 0;
     for (;;) {
-        uint32_t ok;
         asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
                      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-        if (ok) return true;
-        if (clock64() - t0 > MBAR_WAIT_CYCLES) return false;
+        if (ok || clock64() - t0 > limit) break;
     }
+    return __all_sync(0xffffffffu, ok != 0);
 }
 
 template <uint32_t COEF, uint32_t NW>
 __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_async_kernel(DevTables c, const u64 *__restrict__ baby,
                                                                                  const u64 *__restrict__ pts, u64 *__restrict__ acc,
                                                                                  uint32_t J, uint32_t S, uint32_t G, uint32_t level,
-                                                                                 uint32_t ntiles, uint32_t Jx, uint32_t j0, uint32_t accumulate) {
+                                                                                 uint32_t ntiles, uint32_t Jx, uint32_t j0, uint32_t accumulate,
+                                                                                 long long wait_limit) {
     using T = Geo<COEF>;
     constexpr uint32_t THREADS = COEF * 64 / NW, CH = T::CH, NWARPS = THREADS / 32;
     constexpr uint32_t AH = THREADS / (CH * MK), NIT = MG / AH, XB64 = 64 / COEF;
@@ -349,7 +351,7 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_async_kernel
             lg0 = lt.zg * MG + arow;
             lsh0 = lt.zc * (MS / 2) + (arow >> 1);
             lsm = sm_thread + lslot * T::STAGE_BYTES;
-            if (luse > 0 && !mbar_wait(bars + 8 * (STAGES + lslot), (luse - 1) & 1)) alive = false;
+            if (luse > 0 && !mbar_wait(bars + 8 * (STAGES + lslot), (luse - 1) & 1, wait_limit)) alive = false;
         }
     };
     auto load_w = [&](uint32_t k) {
@@ -389,7 +391,7 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_async_kernel
     u64 pend_q = 0;
     const size_t lN = (size_t)level * c.N;
     auto flush = [&]() {
-        if (!mbar_wait(bar_ofull, pend_tile & 1)) alive = false;
+        if (!mbar_wait(bar_ofull, pend_tile & 1, wait_limit)) alive = false;
 #pragma unroll
         for (uint32_t k = 0; k < MG * MS * COEF / THREADS; k++) {
             const uint32_t row = k * (THREADS / COEF) + tid / COEF, sl = tid % COEF, gl = row >> 4, cl = row & 15;
@@ -414,7 +416,7 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_async_kernel
 #pragma unroll
                     for (uint32_t r = 0; r < 4; r++) dsum[n][d][r] = 0;
         }
-        if (!mbar_wait(bars + 8 * slot, use & 1)) { alive = false; break; }
+        if (!mbar_wait(bars + 8 * slot, use & 1, wait_limit)) { alive = false; break; }
         const uint8_t *Wt = ring + (size_t)slot * T::STAGE_BYTES, *Xt = Wt + T::BOX_BYTES;
         uint32_t A[7][4];
 #pragma unroll
@@ -467,7 +469,7 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_async_kernel
         if (pend) flush();
         if (ks == nk - 1 && alive) {
             if (ct.i != qi) { qi = ct.i; q = c.mod[qi]; mu = c.mu[qi]; }
-            if (tiles_done > 0 && !mbar_wait(bar_oempty, (tiles_done - 1) & 1)) alive = false;
+            if (tiles_done > 0 && !mbar_wait(bar_oempty, (tiles_done - 1) & 1, wait_limit)) alive = false;
 #pragma unroll
             for (uint32_t n = 0; n < NW; n++)
 #pragma unroll
@@ -503,16 +505,20 @@ __global__ void __launch_bounds__(COEF * 64 / NW, 8 / COEF) mac_mma_async_kernel
 template <uint32_t COEF, uint32_t NW, bool ASYNC = false>
 bool launch_as(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level, cudaStream_t s,
                uint32_t Jx, uint32_t j0, bool accumulate) {
-    auto kernel = ASYNC ? mac_mma_async_kernel<COEF, NW> : mac_mma_kernel<COEF, NW>;
     // per device, so set on every launch (a host-side table update)
+    const void *kernel = ASYNC ? (const void *)mac_mma_async_kernel<COEF, NW> : (const void *)mac_mma_kernel<COEF, NW>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Geo<COEF>::SMEM_BYTES) != cudaSuccess) return false;
     const uint32_t coltiles = (2 * S + MS - 1) / MS, gt = (G + MG - 1) / MG;
     const uint32_t ntiles = (c->N / COEF) * level * coltiles * gt;
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
-    const uint32_t ctas = (uint32_t)sms * (8 / COEF);
-    kernel<<<ntiles < ctas ? ntiles : ctas, COEF * 64 / NW, Geo<COEF>::SMEM_BYTES, s>>>(c->dev, baby, pts, acc, J, S, G, level, ntiles, Jx, j0,
-                                                                                       accumulate ? 1u : 0u);
+    const uint32_t ctas = (uint32_t)sms * (8 / COEF), grid = ntiles < ctas ? ntiles : ctas;
+    if (ASYNC)
+        mac_mma_async_kernel<COEF, NW><<<grid, COEF * 64 / NW, Geo<COEF>::SMEM_BYTES, s>>>(c->dev, baby, pts, acc, J, S, G, level, ntiles, Jx, j0,
+                                                                                            accumulate ? 1u : 0u, c->wait_cycles);
+    else
+        mac_mma_kernel<COEF, NW><<<grid, COEF * 64 / NW, Geo<COEF>::SMEM_BYTES, s>>>(c->dev, baby, pts, acc, J, S, G, level, ntiles, Jx, j0,
+                                                                                      accumulate ? 1u : 0u);
     count_launches();
     return true;
 }
@@ -528,13 +534,12 @@ bool launch_mac_mma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *acc
                     cudaStream_t s, uint32_t Jx, uint32_t j0, bool accumulate) {
     if (!mac_mma_supported(c, J)) return false;
     if (!Jx) Jx = J;
-    // tuning knob: CKKS_MAC_SHAPE = 100 (the tcgen05 / TMEM kernel of mac_umma.cu, J <= 64), 82 (mma.sync, 8 coefficients per
-    // CTA, a warp per coefficient: the default), 83 (the same
-    // without CTA-wide barriers: 7 % faster, bounded mbarrier waits), 81 (two warps per coefficient, 10 % slower) or 42
-    // (4 coefficients per CTA, two CTAs per SM: the products overlap better, but operand
-    // rows fetched 32 bytes at a time make the loads twice as slow as the whole kernel otherwise is)
-    const char *e = getenv("CKKS_MAC_SHAPE");
-    const int shape = e ? atoi(e) : 82;
+    // context option CKKS_OPT_MAC_KERNEL: CKKS_MAC_TCGEN05 (the tcgen05 / TMEM kernel of mac_umma.cu, J <= 64), CKKS_MAC_MMA
+    // (mma.sync, 8 coefficients per CTA, a warp per coefficient: the default), CKKS_MAC_MMA_ASYNC (the same without
+    // CTA-wide barriers: 7 % faster, bounded mbarrier waits), CKKS_MAC_MMA_SPLIT (two warps per coefficient, 10 % slower)
+    // or CKKS_MAC_MMA_HALF (4 coefficients per CTA, two CTAs per SM: the products overlap better, but operand rows
+    // fetched 32 bytes at a time make the loads twice as slow as the whole kernel otherwise is)
+    const int shape = c->mac_kernel;
     if (shape == 100 && launch_mac_umma(c, baby, pts, acc, J, S, G, level, s, Jx, j0, accumulate)) return true;
     if (shape == 83) return launch_as<8, 2, true>(c, baby, pts, acc, J, S, G, level, s, Jx, j0, accumulate);
     if (shape == 42) return launch_as<4, 2>(c, baby, pts, acc, J, S, G, level, s, Jx, j0, accumulate);

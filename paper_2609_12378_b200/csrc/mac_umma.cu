@@ -22,7 +22,7 @@
 // 64-byte rows.  All hand-offs are mbarriers; every wait is bounded by the clock and raises the context's sticky
 // timeout flag instead of hanging.
 //
-// Status: bit-identical to mac_mma.cu and selectable with CKKS_MAC_SHAPE=100, but not the default.  On B200 a
+// Status: bit-identical to mac_mma.cu and selectable with the context option CKKS_MAC_TCGEN05, but not the default.  On B200 a
 // giant-step group of the 4096 x 4096 projection (16 shards) takes 18.9 ms here against 13.8 ms with mma.sync: the
 // tensor pipe is idle most of the time and the 16 epilogue warps are busy 85 % of it.  With accumulators in registers
 // the products of equal weight a + b add up inside the MMA (13 sums per output); here all 49 arrive separately and
@@ -72,21 +72,27 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) { asm volatile("mbarri
 __device__ __forceinline__ void mbar_arrive_cp_async(uint32_t bar) {
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(bar) : "memory");
 }
-constexpr long long WAIT_CYCLES = 2000000000ll;      // about a second
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Bounded wait (limit in SM clock cycles).  WARP = true: all 32 lanes call it together and get the warp's common verdict,
+// so a timeout never splits a warp in front of a warp-wide instruction; WARP = false: a single thread waits (the MMA issuer).
+template <bool WARP>
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long limit) {
     const long long t0 = clock64();
+    uint32_t ok = 0;
     for (;;) {
-        uint32_t ok;
         asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
                      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-        if (ok) return true;
-        if (clock64() - t0 > WAIT_CYCLES) return false;
+        if (ok || clock64() - t0 > limit) break;
     }
+    return WARP ? __all_sync(0xffffffffu, ok != 0) : ok != 0;
 }
 // item n of a ring of depth D: the consumer waits for the fill of its slot, the producer for the drain of the item before
-__device__ __forceinline__ bool wait_full(uint32_t bars, uint32_t base, uint32_t n, uint32_t D) { return mbar_wait(bars + 8 * (base + n % D), (n / D) & 1); }
-__device__ __forceinline__ bool wait_empty(uint32_t bars, uint32_t base, uint32_t n, uint32_t D) {
-    return n < D ? true : mbar_wait(bars + 8 * (base + n % D), ((n / D) - 1) & 1);
+template <bool WARP = true>
+__device__ __forceinline__ bool wait_full(uint32_t bars, uint32_t base, uint32_t n, uint32_t D, long long limit) {
+    return mbar_wait<WARP>(bars + 8 * (base + n % D), (n / D) & 1, limit);
+}
+template <bool WARP = true>
+__device__ __forceinline__ bool wait_empty(uint32_t bars, uint32_t base, uint32_t n, uint32_t D, long long limit) {
+    return n < D ? true : mbar_wait<WARP>(bars + 8 * (base + n % D), ((n / D) - 1) & 1, limit);
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
@@ -146,7 +152,7 @@ struct BlockIt {           // blocks of a CTA: giant tile fastest, then coeffici
 
 __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, const u64 *__restrict__ baby, const u64 *__restrict__ pts,
                                                                 u64 *__restrict__ acc, uint32_t J, uint32_t S, uint32_t G, uint32_t level,
-                                                                uint32_t nblocks, uint32_t Jx, uint32_t j0, uint32_t accumulate) {
+                                                                uint32_t nblocks, uint32_t Jx, uint32_t j0, uint32_t accumulate, long long wl) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sm = reinterpret_cast<uint8_t *>(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
     const uint32_t sm0 = (uint32_t)__cvta_generic_to_shared(sm);
@@ -188,7 +194,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
         for (uint32_t b = 0; b < myblocks && alive; b++, it.next(gtiles, xblocks)) {
             const size_t blk = (size_t)it.i * (c.N >> 6) + (it.xb >> 3);
             const uint32_t in_blk = (it.xb & 7) * UC + p;
-            if (!wait_empty(bars, B_WEMPTY, b, 2)) { alive = false; break; }
+            if (!wait_empty(bars, B_WEMPTY, b, 2, wl)) { alive = false; break; }
             const u64 *wsrc = pts + blk * Rw * 64 + in_blk + (size_t)jr * 64;
             const uint32_t wdst = sm0 + L.w(b & 1) + p * L.tsw + jr * 16 + par * 8;
             for (uint32_t gp = sub; gp < UG / 2; gp += NSUB) {
@@ -201,7 +207,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
             mbar_arrive_cp_async(bars + 8 * (B_WFULL + (b & 1)));
             const u64 *xsrc = baby + blk * Rx * 64 + in_blk + (size_t)(j0 + jr) * 128;
             for (uint32_t cg = 0; cg < ncg && alive; cg++, cgn++) {
-                if (!wait_empty(bars, B_XEMPTY, cgn, 2)) { alive = false; break; }
+                if (!wait_empty(bars, B_XEMPTY, cgn, 2, wl)) { alive = false; break; }
                 const uint32_t xdst = sm0 + L.x(cgn & 1) + p * L.tsx + jr * 16 + par * 8;
                 for (uint32_t cp = sub; cp < UCG / 2; cp += NSUB) {
                     const uint32_t col = min(cg * UCG + 2 * cp + par, ncol - 1);
@@ -219,12 +225,12 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
         if (lane == 0) {
             uint32_t cgn = 0, an = 0;
             for (uint32_t b = 0; b < myblocks && alive; b++) {
-                if (!wait_full(bars, B_WFULL, b, 2)) { alive = false; break; }
+                if (!wait_full<false>(bars, B_WFULL, b, 2, wl)) { alive = false; break; }
                 for (uint32_t cg = 0; cg < ncg && alive; cg++, cgn++) {
-                    if (!wait_full(bars, B_XFULL, cgn, 2)) { alive = false; break; }
+                    if (!wait_full<false>(bars, B_XFULL, cgn, 2, wl)) { alive = false; break; }
                     asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
                     for (uint32_t p = 0; p < UC; p++, an++) {
-                        if (!wait_empty(bars, B_TEMPTY, an, NACC)) { alive = false; break; }
+                        if (!wait_empty<false>(bars, B_TEMPTY, an, NACC, wl)) { alive = false; break; }
                         tc_fence_after();
                         const uint32_t wa = sm0 + L.w(b & 1) + p * L.tsw, xa = sm0 + L.x(cgn & 1) + p * L.tsx;
                         for (uint32_t ks = 0; ks < nk; ks++)
@@ -245,7 +251,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
         for (uint32_t b = 0; b < myblocks && alive; b++, it.next(gtiles, xblocks)) {
             u64 *obase = acc + (size_t)it.i * c.N + it.xb * UC;
             for (uint32_t cg = 0; cg < ncg && alive; cg++, cgn++) {
-                if (!wait_full(bars, B_OFULL, cgn, 2)) { alive = false; break; }
+                if (!wait_full(bars, B_OFULL, cgn, 2, wl)) { alive = false; break; }
                 const u64 *ob = reinterpret_cast<const u64 *>(sm + L.o(cgn & 1));
 #pragma unroll 4
                 for (uint32_t k = 0; k < UG * UCG * UC / 32; k++) {
@@ -276,7 +282,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
             for (uint32_t cg = 0; cg < ncg && alive; cg++, cgn++) {
                 for (uint32_t half = 0; half < 2; half++) {
                     const uint32_t p = eg + 4 * half, an = cgn * UC + p;
-                    if (!wait_full(bars, B_TFULL, an, NACC)) { alive = false; break; }
+                    if (!wait_full(bars, B_TFULL, an, NACC, wl)) { alive = false; break; }
                     tc_fence_after();
                     // fold b: S[cl] = sum_b D[cl][b] 2^(8b) as three 32-bit words (below 2^72)
                     uint32_t T[8][3];
@@ -344,7 +350,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) mac_umma_kernel(DevTables c, con
                     }
                     const uint32_t cl = (a0 ? 4u : 0u) + (a1 ? 2u : 0u) + (a2 ? 1u : 0u);     // the column this lane finished
                     const u64 res = barrett112(((u64)Z[3] << 32) | Z[2], ((u64)Z[1] << 32) | Z[0], qmod, mu);
-                    if (!wait_empty(bars, B_OEMPTY, cgn, 2)) { alive = false; break; }
+                    if (!wait_empty(bars, B_OEMPTY, cgn, 2, wl)) { alive = false; break; }
                     reinterpret_cast<u64 *>(sm + L.o(cgn & 1))[(gl * UCG + cl) * UC + (p ^ (gl & 7))] = res;
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bars + 8 * (B_OFULL + (cgn & 1)));
@@ -375,7 +381,7 @@ bool launch_mac_umma(const ckks_ctx *c, const u64 *baby, const u64 *pts, u64 *ac
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
     mac_umma_kernel<<<nblocks < (uint32_t)sms ? nblocks : (uint32_t)sms, U_THREADS, L.total, s>>>(c->dev, baby, pts, acc, J, S, G, level, nblocks, Jx, j0,
-                                                                                                  accumulate ? 1u : 0u);
+                                                                                                  accumulate ? 1u : 0u, c->wait_cycles);
     count_launches();
     return true;
 }

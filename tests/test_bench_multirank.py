@@ -47,7 +47,7 @@ def test_two_gloo_ranks_aggregate():
     jm = line["jm"]
     assert abs(jm["value"] - 0.401 / 2) < 1e-12                       # two replicas finish two projections in 401 ms
     assert abs(jm["ntt_limbs_per_s"] - 2 * 2 * 768 / 0.110) < 1e-6
-    assert abs(jm["key_switches_per_s"] - 2 * 129 / 0.005) < 1e-6
+    assert abs(jm["key_switches_per_s"] - 2 * 64 / 0.005) < 1e-6        # 64 plain rotations per replica in 5 ms
 
 
 def test_single_rank_is_identity():
@@ -55,4 +55,23 @@ def test_single_rank_is_identity():
     import bench
     assert bench.max_over_ranks([1.5, 2.5]) == [1.5, 2.5]
     jm = bench.job_metrics(1, 1.0, 25.0, 450.0)
-    assert jm["value"] == 0.45 and jm["key_switches_per_s"] == 129 / 0.025
+    assert jm["value"] == 0.45 and jm["key_switches_per_s"] == 64 / 0.025
+
+
+def test_algorithmic_work_counts():
+    """The operation counts behind the roofline fractions: one key switch at level 24 with 8 special primes and 3 digits
+    is 160 limb transforms and 81.3 M multiply-add pairs, a hoisted rotation 64 and 42 M (counted by hand from the steps:
+    24 inverse + 72 forward transforms and 600 pairs per coefficient for ModUp, 192 for the key product, 16 + 48
+    transforms and 448 pairs for ModDown)."""
+    sys.path.insert(0, ROOT)
+    import bench
+    ks, h = bench.ks_work(), bench.ks_work(hoisted=True)
+    assert ks["limb_ntts"] == 24 + 72 + 16 + 48 == 160 and h["limb_ntts"] == 64
+    assert ks["pairs_per_coeff"] == 600 + 192 + 448 and h["pairs_per_coeff"] == 192 + 448
+    assert round(ks["pairs_per_coeff"] * 65536 / 1e6, 1) == 81.3 and round(h["pairs_per_coeff"] * 65536 / 1e6, 1) == 41.9
+    assert ks["fp64_instr"] == 160 * 524288 * 8 + 1240 * 65536 * 7
+    lazy, eager = bench.projection_work(True), bench.projection_work(False)
+    assert lazy["encode"]["count"] == 4096 and lazy["mac"]["count"] == 65536
+    assert lazy["baby_hoisted_rotations"]["count"] == 1008 and lazy["giant_terms"]["count"] == 1008 and eager["giant_rotations"]["count"] == 1008
+    assert lazy["mac"]["hbm_bytes"] == (4096 * 24 + 16 * 64 * 48 + 16 * 64 * 48) * 524288      # plaintexts, baby ciphertexts, accumulators
+    assert bench.bound_ms(eager, 18.6, 6527.0) > bench.bound_ms(lazy, 18.6, 6527.0) > 100.0

@@ -2,8 +2,10 @@
 
 The 128-token 4096 x 4096 projection runs in the launch configuration bench.py times (16 shards, B = G = 64,
 126 rotation keys).  Every output ciphertext is decrypted and compared with X W in fp64 (bounded by the scheme's
-noise), and one sampled shard is recomputed by the CPU checker and compared bit for bit (a shard's output depends
-only on that shard's input).  Minutes of host time: key generation and the checker's shard."""
+noise), and the first, the last and one seeded middle shard are recomputed by the CPU checker and compared bit for
+bit (a shard's output depends only on that shard's input; every key switch is batched over the shards, so both ends of
+the batch and an entry inside a chunk are covered).  The other decoder-layer shapes (key/value, gate/up, down) and the
+seeded subset of the attention products run the same way.  Minutes of host time: key generation and the checker."""
 import numpy as np
 import pytest
 
@@ -43,21 +45,25 @@ def test_llama_shaped_projection_full_size():
         sl = cl.decrypt_slots(got[c], outs[c].scale).real.reshape(D, T)
         worst = max(worst, np.abs(sl - Y[c * T:(c + 1) * T].T).max())
     assert worst < 2.0 ** -16, worst           # two key switches, 4096-term sums and a rescale at Delta = 2^40
-    # one sampled shard, bit for bit
-    c = int(inputs.rng(1004, 2).integers(0, S))
-    one = ProjDesc(D, D, T, 1, B)
-    want, want_scale = o.linear_proj(one, cts[c][None], W, keys, scale)
-    assert want_scale == outs[c].scale
-    assert np.array_equal(got[c], want[0])
-    # the schedule with the giant steps summed before one ModDown: all shards decrypt to X W, the sampled shard is the
-    # checker's lazy variant bit for bit
+    # the first and the last shard of the batch and a seeded one in between, bit for bit (one checker call, so the
+    # encoded diagonals are shared)
+    c = int(inputs.rng(1004, 2).integers(1, S - 1))
+    sel = [0, c, S - 1]
+    some = ProjDesc(D, D, T, len(sel), B)
+    want, want_scale = o.linear_proj(some, np.stack([cts[i] for i in sel]), W, keys, scale)
+    for n, i in enumerate(sel):
+        assert want_scale == outs[i].scale
+        assert np.array_equal(got[i], want[n]), i
+    # the schedule with the giant steps summed before one ModDown: all shards decrypt to X W, the same three shards
+    # are the checker's lazy variant bit for bit
     lazy = ctx.linear_proj(dcts, dev(W), dkeys, D, D, T, S, B, lazy_moddown=True)
     assert ctx.device_status() == binding.OK
     for cc in range(S):
         sl = cl.decrypt_slots(host(lazy[cc].data), lazy[cc].scale).real.reshape(D, T)
         assert np.abs(sl - Y[cc * T:(cc + 1) * T].T).max() < 2.0 ** -16
-    want_lazy, _ = o.linear_proj(ProjDesc(D, D, T, 1, B, lazy_moddown=True), cts[c][None], W, keys, scale)
-    assert np.array_equal(host(lazy[c].data), want_lazy[0])
+    want_lazy, _ = o.linear_proj(ProjDesc(D, D, T, len(sel), B, lazy_moddown=True), np.stack([cts[i] for i in sel]), W, keys, scale)
+    for n, i in enumerate(sel):
+        assert np.array_equal(host(lazy[i].data), want_lazy[n]), i
     del lazy
     # the same inputs through the square and a key-shaped (4096 x 1024) matrix in one call with shared baby steps:
     # the square matrix's outputs do not change, the second matrix's decrypt to X Wk (one block, stored four times)
@@ -144,19 +150,48 @@ def test_kv_projection_full_ring():
     _full_ring_shape(4096, 1024, 4, 32, seed=1005, lazy=True)
 
 
-import os  # noqa: E402
-
-heavy = pytest.mark.skipif(os.environ.get("CKKS_RUN_HEAVY") != "1",
-                           reason="ten minutes of CPU checker time per shape; set CKKS_RUN_HEAVY=1")
-
-
-@heavy
 def test_gate_up_projection_full_ring():
     """gate / up shape: 4096 -> 14336 = 3 x 4096 + 2048 (three square output blocks and a folded remainder block)."""
     _full_ring_shape(4096, 14336, 2, 64, seed=1006)
 
 
-@heavy
 def test_down_projection_full_ring():
     """down shape: 14336 -> 4096 (three full input blocks and a repeated remainder block summed before the giant steps)."""
     _full_ring_shape(14336, 4096, 2, 64, seed=1007, lazy=True)
+
+
+def test_attention_product_batch_full_size():
+    """The decoder layer's ciphertext x ciphertext work (QK^T and PV: 2048 + 2048 independent products at level 24,
+    128 of them summed per output ciphertext) on a seeded subset: 64 products through the batched entry point, each
+    against the checker's single product, and one sum of 128 products with a single relinearisation against the
+    checker's sum, bit for bit; the first product and the sum also after decryption."""
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    P, ctx = params(16, 24, 8, 3), context(16, 24, 8, 3)
+    o = P.oracle
+    cl = Client(P, 1005)
+    level, scale = 24, 2.0 ** 40
+    g = inputs.rng(1005, 9)
+    rlk = cl.relin_key()
+    drlk = key_dev(rlk, 0)
+    # 16 distinct ciphertexts; product i pairs a[i % 16] with b[(5 i + 3) % 16], so all 64 pairs differ
+    za, zb = g.uniform(-1, 1, (16, P.n)), g.uniform(-1, 1, (16, P.n))
+    a = [cl.encrypt_slots(z, scale, level) for z in za]
+    b = [cl.encrypt_slots(z, scale, level) for z in zb]
+    da, db = [ct_dev(x, scale) for x in a], [ct_dev(x, scale) for x in b]
+    ia, ib = [i % 16 for i in range(64)], [(5 * i + 3) % 16 for i in range(64)]
+    assert len(set(zip(ia, ib))) == 64
+    outs = ctx.mul_relin_batch([da[i] for i in ia], [db[j] for j in ib], drlk)
+    assert ctx.device_status() == binding.OK
+    for n, (i, j) in enumerate(zip(ia, ib)):
+        assert outs[n].scale == scale * scale
+        assert np.array_equal(host(outs[n].data), o.mul_relin(a[i], b[j], rlk)), n
+    z0 = cl.decrypt_slots(host(outs[0].data), scale * scale).real
+    assert np.abs(z0 - za[ia[0]] * zb[ib[0]]).max() < 2.0 ** -17
+    # one output ciphertext of PV: 128 products summed, one key switch
+    ja, jb = [i % 16 for i in range(128)], [(3 * i + i // 16) % 16 for i in range(128)]
+    tot = ctx.mul_relin_sum([da[i] for i in ja], [db[j] for j in jb], drlk)
+    assert ctx.device_status() == binding.OK
+    want = o.mul_relin_sum(np.stack([a[i] for i in ja]), np.stack([b[j] for j in jb]), rlk)
+    assert np.array_equal(host(tot.data), want)
+    zs = cl.decrypt_slots(host(tot.data), scale * scale).real
+    assert np.abs(zs - sum(za[i] * zb[j] for i, j in zip(ja, jb))).max() < 2.0 ** -17

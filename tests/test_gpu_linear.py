@@ -10,7 +10,7 @@ from tests.harness import Client, params
 pytestmark = pytest.mark.gpu
 
 
-def _run(log_n, L, K, dnum, level, d_in, d_out, T, S, B, seed, pt_scale=0.0, check_slots=True, lazy=False):
+def _run(log_n, L, K, dnum, level, d_in, d_out, T, S, B, seed, pt_scale=0.0, check_slots=True, lazy=False, compare=True):
     from tests.gpu_util import context, ct_dev, dev, host, key_dev
     P, ctx = params(log_n, L, K, dnum), context(log_n, L, K, dnum)
     o = P.oracle
@@ -28,10 +28,12 @@ def _run(log_n, L, K, dnum, level, d_in, d_out, T, S, B, seed, pt_scale=0.0, che
     rots = o.proj_rotations(desc)
     assert rots == ctx.linear_proj_rotations(d_in, d_out, T, S, B)
     keys = {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in rots}
-    want, want_scale = o.linear_proj(desc, np.stack(cts), W, keys, scale)
     got = ctx.linear_proj([ct_dev(c, scale) for c in cts], dev(W), [key_dev(k, g_) for g_, k in keys.items()],
                           d_in, d_out, T, S, B, pt_scale, lazy_moddown=lazy)
     assert len(got) == S * len(outs)
+    if not compare:
+        return ctx, cts, keys
+    want, want_scale = o.linear_proj(desc, np.stack(cts), W, keys, scale)
     Y = X @ W
     for i, ct in enumerate(got):
         arr = host(ct.data)
@@ -99,23 +101,70 @@ def test_projection_lazy_moddown_many_groups():
     _run(11, 4, 2, 2, 3, 128, 128, 8, 2, 4, seed=490, lazy=True)
 
 
-@pytest.mark.parametrize("shape", ["81", "83", "42", "100"])
-def test_projection_tensor_core_mac_other_shapes(shape, monkeypatch):
-    """The kernel's other tilings (two warps per coefficient; the barrier-free pipeline; four coefficients per CTA),
-    selected by the CKKS_MAC_SHAPE tuning knob, on a case with two k-steps, two column tiles and column padding."""
+@pytest.mark.parametrize("kernel", [binding.MAC_MMA_SPLIT, binding.MAC_MMA_ASYNC, binding.MAC_MMA_HALF, binding.MAC_TCGEN05])
+def test_projection_tensor_core_mac_other_shapes(kernel):
+    """The kernel's other forms (two warps per coefficient; the barrier-free pipeline; four coefficients per CTA; tcgen05
+    with TMEM accumulators), selected by a context option, on a case with two k-steps, two column tiles and column
+    padding."""
     from tests.gpu_util import context
-    monkeypatch.setenv("CKKS_MAC_SHAPE", shape)
-    ctx, _, _ = _run(10, 4, 2, 2, 4, 64, 160, 8, 9, 32, seed=450)
-    assert ctx.device_status() == 0
+    ctx = context(10, 4, 2, 2)
+    ctx.set_option(binding.OPT_MAC_KERNEL, kernel)
+    try:
+        assert ctx.get_option(binding.OPT_MAC_KERNEL) == kernel
+        _run(10, 4, 2, 2, 4, 64, 160, 8, 9, 32, seed=450)
+        assert ctx.device_status() == 0
+    finally:
+        ctx.set_option(binding.OPT_MAC_KERNEL, binding.MAC_MMA)
 
 
-def test_projection_with_tensor_core_basis_conversion(monkeypatch):
-    """ModUp's and ModDown's conversion matrices on the tensor cores (the CKKS_CONV=mma tuning knob): the same integers,
-    on a shape with a fold, several output blocks and a partial last digit."""
-    monkeypatch.setenv("CKKS_CONV", "mma")
-    ctx, _, _ = _run(10, 6, 2, 3, 5, 16, 24, 32, 2, 4, seed=455)
-    assert ctx.device_status() == 0
-    _run(10, 4, 2, 2, 4, 64, 160, 8, 3, 32, seed=456, lazy=True)
+def test_projection_with_tensor_core_basis_conversion():
+    """ModUp's and ModDown's conversion matrices on the tensor cores (a context option): the same integers, on a shape
+    with a fold, several output blocks and a partial last digit."""
+    from tests.gpu_util import context
+    ctxs = [context(10, 6, 2, 3), context(10, 4, 2, 2)]
+    for c in ctxs:
+        c.set_option(binding.OPT_CONV_KERNEL, binding.CONV_TENSOR)
+    try:
+        ctx, _, _ = _run(10, 6, 2, 3, 5, 16, 24, 32, 2, 4, seed=455)
+        assert ctx.device_status() == 0
+        _run(10, 4, 2, 2, 4, 64, 160, 8, 3, 32, seed=456, lazy=True)
+    finally:
+        for c in ctxs:
+            c.set_option(binding.OPT_CONV_KERNEL, binding.CONV_FP64)
+
+
+def test_options_reject_bad_values():
+    from tests.gpu_util import context
+    ctx = context(10, 4, 2, 2)
+    for opt, bad in ((binding.OPT_NTT_FP_SHARE, 9), (binding.OPT_CONV_KERNEL, 2), (binding.OPT_MAC_KERNEL, 7), (binding.OPT_WAIT_CYCLES, -1),
+                     (99, 0), (binding.OPT_STATIC_SCRATCH_BYTES, 1)):
+        with pytest.raises(binding.CkksError) as e:
+            ctx.set_option(opt, bad)
+        assert e.value.code == binding.ERR_ARG
+    assert ctx.get_option(99) == -1
+    assert ctx.get_option(binding.OPT_WAIT_CYCLES) == 2_000_000_000
+    assert ctx.get_option(binding.OPT_MAC_KERNEL) == binding.MAC_MMA and ctx.get_option(binding.OPT_CONV_KERNEL) == binding.CONV_FP64
+
+
+def test_device_wait_that_runs_out_is_reported_and_leaves_the_context_usable():
+    """The mbarrier pipeline of the multiply-accumulate with a wait limit of zero cycles: the first wait that is not
+    already satisfied (the operands of the first step are still on their way) gives up, the kernel waits for its own
+    copies and returns, and the sticky flag is reported once.  With the limit restored the same call is bit-exact."""
+    from tests.gpu_util import context
+    ctx = context(10, 4, 2, 2)
+    ctx.set_option(binding.OPT_MAC_KERNEL, binding.MAC_MMA_ASYNC)
+    try:
+        assert ctx.device_status() == binding.OK
+        ctx.set_option(binding.OPT_WAIT_CYCLES, 0)
+        _run(10, 4, 2, 2, 4, 64, 64, 8, 2, 32, seed=452, compare=False)
+        assert ctx.device_status() == binding.ERR_TIMEOUT
+        assert ctx.device_status() == binding.OK            # the flag was cleared by the query
+        ctx.set_option(binding.OPT_WAIT_CYCLES, 2_000_000_000)
+        _run(10, 4, 2, 2, 4, 64, 64, 8, 2, 32, seed=452)
+        assert ctx.device_status() == binding.OK
+    finally:
+        ctx.set_option(binding.OPT_WAIT_CYCLES, 2_000_000_000)
+        ctx.set_option(binding.OPT_MAC_KERNEL, binding.MAC_MMA)
 
 
 def test_projection_multi_shares_baby_steps():
