@@ -62,6 +62,19 @@ class ProjDesc:
     lazy_moddown: bool = False  # giant-step results summed in the extended basis, one ModDown per output
 
 
+@dataclass
+class AttnDesc:
+    """Shape of one attention block in the diagonal-block layout.  Every operand and every score ciphertext uses the slot
+    index ((e * tokens + i) * heads + h) * R + r: i a token position, h a head, e < diag_block one of the score diagonals
+    a ciphertext holds side by side, r < R = n / (diag_block * tokens * heads) trailing copies."""
+    tokens: int
+    heads: int
+    diag_block: int
+
+    def groups(self) -> int:
+        return self.tokens // self.diag_block
+
+
 class Oracle:
     def __init__(self, log_n: int, q, p, dnum: int):
         self.log_n, self.N, self.n, self.M = log_n, 1 << log_n, 1 << (log_n - 1), 2 << log_n
@@ -379,6 +392,108 @@ class Oracle:
             v = self.rescale(self.mul_relin(lam, u[:, :ll], rlk)); sv = sl * su / float(self.q[ll - 1])
             u = self.rescale(self.mul_relin(v, v, rlk)); su = sv * sv / float(self.q[ll - 2])
         return u, su
+
+    # -------------------------------------------------------------- attention
+    def attention_rotations(self, desc: AttnDesc):
+        """(token rotations, ladder rotations) in slots: key rotations by g * diag_block tokens, g = 1 .. groups - 1, and
+        the rotate-and-add ladder over the diag_block blocks of a ciphertext (by tokens * heads * R * 2^k slots)."""
+        E, Tk, H = desc.diag_block, desc.tokens, desc.heads
+        if Tk % E or self.n % (E * Tk * H) or E & (E - 1) or Tk & (Tk - 1):
+            raise ValueError("diag_block must divide tokens, and diag_block * tokens * heads the slot count (powers of two)")
+        R = self.n // (E * Tk * H)
+        tok = [g * E * H * R for g in range(1, desc.groups())]
+        lad, k = [], 1
+        while k < E:
+            lad.append(Tk * H * R * k); k *= 2
+        return tok, lad
+
+    def attention_scores(self, desc: AttnDesc, q, k, rlk, keys: dict):
+        """Score ciphertexts S_g, g < groups = tokens / diag_block, from the channel operands q[d], k[d] (d < dim,
+        [dim][2][level][N], layout of AttnDesc with the query repeated in every block e and the key operand holding token
+        i + e in block e):  S_g = rescale(mul_relin_sum_d(q[d], rotate(k[d], g * diag_block tokens))).
+        Slot (e, i, h) of S_g is the score of query i and head h against one key token; over all g and e every key token
+        occurs exactly once, so the score row of (i, h) is spread over the groups x diag_block slots (e, i, h) of the S_g.
+        One relinearisation per S_g; the products of a group are summed before it.  Returns [groups][2][level-1][N]."""
+        q = _u64(q); k = _u64(k); level = q.shape[2]
+        tok, _ = self.attention_rotations(desc)
+        out = np.empty((desc.groups(), 2, level - 1, self.N), dtype=np.uint64)
+        for g in range(desc.groups()):
+            if g == 0:
+                kr = k
+            else:
+                ge = self.galois_element(tok[g - 1])
+                kr = np.stack([self.rotate(k[d], keys[ge], ge) for d in range(k.shape[0])])
+            out[g] = self.rescale(self.mul_relin_sum(q, kr, rlk))
+        return out
+
+    def _block_ladder(self, desc: AttnDesc, s, keys: dict):
+        _, lad = self.attention_rotations(desc)
+        for r in lad:
+            ge = self.galois_element(r)
+            s = self.add(s, self.rotate(s, keys[ge], ge))
+        return s
+
+    def softmax_rows(self, desc: AttnDesc, S, scale: float, shift: float, rounds: int, exp_coeffs, rsqrt_coeffs, rlk, keys: dict):
+        """Softmax by doubling with a public shift (Algorithm 1) on score rows spread over several ciphertexts: the row of
+        (i, h) consists of the slots (e, i, h), e < diag_block, of every S_g.  Order of steps:
+          u_g = poly_eval_tree(S_g + round(-shift * scale), exp_coeffs) for every g;
+          per round: t = rescale(mul_relin_sum_g(u_g, u_g)); t = t + rotate(t, r) for the ladder rotations r in ascending
+                     order (the row sum, in every slot of the row); lam = poly_eval_tree(t, rsqrt_coeffs[j]);
+                     for every g: v = rescale(mul_relin(lam, u_g truncated to lam's level)); u_g = rescale(mul_relin(v, v)).
+        The row sums and the inverse square root are formed once for all groups.  Returns ([groups][2][l][N], scale)."""
+        S = _u64(S)
+        G = S.shape[0]
+        u, su = [], None
+        for g in range(G):
+            z = self.add_const(S[g], int(np.rint(-shift * scale)))
+            ug, su = self.poly_eval_tree(z, scale, exp_coeffs, rlk)
+            u.append(ug)
+        for j in range(rounds):
+            lv = u[0].shape[1]
+            U = np.stack(u)
+            t = self.rescale(self.mul_relin_sum(U, U, rlk)); st = su * su / float(self.q[lv - 1])
+            t = self._block_ladder(desc, t, keys)
+            lam, sl = self.poly_eval_tree(t, st, rsqrt_coeffs[j], rlk)
+            ll = lam.shape[1]
+            sv = sl * su / float(self.q[ll - 1])
+            for g in range(G):
+                v = self.rescale(self.mul_relin(lam, u[g][:, :ll], rlk))
+                u[g] = self.rescale(self.mul_relin(v, v, rlk))
+            su = sv * sv / float(self.q[ll - 2])
+        return np.stack(u), su
+
+    def attention_values(self, desc: AttnDesc, P, v, rlk, keys: dict):
+        """Output channels from the probability ciphertexts P_g ([groups][2][lp][N], layout of the scores) and the value
+        operands v[d] ([dim_v][2][level][N], level >= lp, layout of the key operand):
+          vt = v[d] truncated to lp limbs;  o = rescale(mul_relin_sum_g(P_g, rotate(vt, g * diag_block tokens)));
+          o = o + rotate(o, r) for the ladder rotations in ascending order.
+        Slot (e, i, h) of output d then holds sum over all key tokens of probability x value for query i, head h, in every
+        block e (the layout of the query operand).  Returns [dim_v][2][lp-1][N]."""
+        P = _u64(P); v = _u64(v)
+        G, lp = P.shape[0], P.shape[2]
+        tok, _ = self.attention_rotations(desc)
+        out = np.empty((v.shape[0], 2, lp - 1, self.N), dtype=np.uint64)
+        for d in range(v.shape[0]):
+            vt = np.ascontiguousarray(v[d][:, :lp])
+            vr = [vt]
+            for g in range(1, G):
+                ge = self.galois_element(tok[g - 1])
+                vr.append(self.rotate(vt, keys[ge], ge))
+            o = self.rescale(self.mul_relin_sum(P, np.stack(vr), rlk))
+            out[d] = self._block_ladder(desc, o, keys)
+        return out
+
+    def attention(self, desc: AttnDesc, q, k, v, scale: float, v_scale: float, shift: float, rounds: int, exp_coeffs, rsqrt_coeffs,
+                  rlk, keys: dict):
+        """Scores, Softmax over the score rows, output channels: attention_scores, softmax_rows, attention_values in a row,
+        with the scales a sequence of doubles: scores scale^2 / q_{l-1}, the Softmax's own, then times v_scale / q_{lp-1}.
+        Returns ([dim_v][2][lp-1][N], scale)."""
+        level = _u64(q).shape[2]
+        S = self.attention_scores(desc, q, k, rlk, keys)
+        ss = scale * scale / float(self.q[level - 1])
+        P, sp = self.softmax_rows(desc, S, ss, shift, rounds, exp_coeffs, rsqrt_coeffs, rlk, keys)
+        lp = P.shape[2]
+        return self.attention_values(desc, P, v, rlk, keys), sp * v_scale / float(self.q[lp - 1])
 
     def automorphism_coeff(self, a, g: int, t: int):
         a = _u64(a); out = np.empty_like(a)

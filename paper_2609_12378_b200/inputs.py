@@ -134,3 +134,26 @@ def pack_feature_major(x: np.ndarray, tokens_per_shard: int, slots: int) -> np.n
         blk = x[c * T:(c + 1) * T, :].T.reshape(-1)          # [f][t] flattened
         out[c] = np.tile(blk, slots // (feats * T))
     return out
+
+
+def attention_slot_index(tokens: int, heads: int, diag_block: int, slots: int):
+    """Index arrays (e, i, h) of every slot of the attention operand layout: slot = ((e * tokens + i) * heads + h) * R + r
+    with R = slots / (diag_block * tokens * heads) trailing copies.  Pure index arithmetic."""
+    E, Tk, H = diag_block, tokens, heads
+    assert slots % (E * Tk * H) == 0 and Tk % E == 0
+    R = slots // (E * Tk * H)
+    s = np.arange(slots) // R
+    return s // (Tk * H), (s // H) % Tk, s % H
+
+
+def pack_attention_operands(Q: np.ndarray, K: np.ndarray, V: np.ndarray, diag_block: int, slots: int):
+    """Lay Q, K [tokens][heads][dim] and V [tokens][heads][dim_v] out as one slot vector per channel in the attention
+    operand layout (slot index as in attention_slot_index): the query operand repeats Q[i, h, d] in every block e, the
+    key and value operands hold token (i + e) mod tokens in block e, so that block e of a product lines query i up with
+    key i + e.  Returns (Qs [dim][slots], Ks [dim][slots], Vs [dim_v][slots]).  Pure data movement."""
+    tokens, heads, _ = Q.shape
+    e, i, h = attention_slot_index(tokens, heads, diag_block, slots)
+    Qs = np.ascontiguousarray(Q[i, h, :].T)
+    Ks = np.ascontiguousarray(K[(i + e) % tokens, h, :].T)
+    Vs = np.ascontiguousarray(V[(i + e) % tokens, h, :].T)
+    return Qs, Ks, Vs

@@ -137,3 +137,39 @@ def softmax_case(P: Params, seed: int, row_len: int = 16, rounds: int = 2, degre
     for i in range(row_len):
         truth[i * stride:(i + 1) * stride] = true[:, i]
     return x, shift, exp_in_z, np.stack(rs), clear, truth
+
+
+# ------------------------------------------------------------ attention in the diagonal-block layout, synthetic case
+
+def attention_case(seed: int, tokens: int, heads: int, dim: int, dim_v: int, rounds: int = 1, degree: int = 4, spread: float = 4.0):
+    """Seeded Q, K [tokens][heads][dim] and V [tokens][heads][dim_v] whose scores Q K^T fall in [shift - spread, shift],
+    polynomial fits as in softmax_case, the pipeline of Algorithm 1 evaluated in the clear on the full score matrix
+    (out_clear [tokens][heads][dim_v]) and plain Softmax attention (out_true).  Returns a dict."""
+    g = inputs.rng(seed, 11)
+    Q = g.uniform(-1.0, 1.0, (tokens, heads, dim))
+    K = g.uniform(-1.0, 1.0, (tokens, heads, dim))
+    V = g.uniform(-1.0, 1.0, (tokens, heads, dim_v))
+    S = np.einsum("ihd,jhd->hij", Q, K)                       # [heads][query][key]
+    Q = Q * (0.5 * spread / np.abs(S).max())                  # scores within +- spread / 2
+    S = np.einsum("ihd,jhd->hij", Q, K)
+    shift = 0.5 * spread
+
+    def fit(f, lo, hi, deg):
+        t = np.cos(np.pi * (np.arange(64) + 0.5) / 64) * (hi - lo) / 2 + (hi + lo) / 2
+        return np.polynomial.polynomial.polyfit(t, f(t), deg)
+
+    ce = fit(np.exp, -spread / 2 ** rounds, 0.0, degree)
+    exp_in_z = ce / (2.0 ** rounds) ** np.arange(degree + 1)
+    pv = np.polynomial.polynomial.polyval
+    u = pv(S - shift, exp_in_z)
+    rs = []
+    for _ in range(rounds):
+        s = (u * u).sum(2)
+        c = fit(lambda t: 1.0 / np.sqrt(t), s.min() / 1.3, s.max() * 1.3, degree)
+        rs.append(c)
+        u = (pv(s, c)[:, :, None] * u) ** 2
+    out_clear = np.einsum("hij,jhd->ihd", u, V)
+    e = np.exp(S - S.max(2, keepdims=True))
+    out_true = np.einsum("hij,jhd->ihd", e / e.sum(2, keepdims=True), V)
+    return dict(Q=Q, K=K, V=V, S=S, shift=shift, exp_coeffs=exp_in_z, rsqrt_coeffs=np.stack(rs), probs_clear=u, out_clear=out_clear,
+                out_true=out_true)

@@ -1,0 +1,96 @@
+"""Pins for the checker's attention in the diagonal-block layout: the layout's index structure in the clear (every
+query meets every key exactly once; rotations as array rolls), the score ciphertexts against Q K^T, and the whole block
+(scores, Softmax by doubling over rows spread across ciphertexts, probability x value) against the same pipeline in the
+clear (tight) and against plain Softmax attention (as good as the synthetic polynomials)."""
+import numpy as np
+import pytest
+
+from oracle.ckks_oracle import AttnDesc
+from paper_2609_12378_b200 import inputs
+from tests.harness import Client, attention_case, params
+
+
+def _key_of(desc, n, g):
+    """Key token met by slot (e, i) of score group g, from the layout's definition: the key operand holds token i + e in
+    block e and is rotated left by g * diag_block token positions of the flattened (e, i) index."""
+    E, Tk = desc.diag_block, desc.tokens
+    e, i, h = inputs.attention_slot_index(Tk, desc.heads, E, n)
+    u = (e * Tk + i + g * E) % (E * Tk)
+    return (u % Tk + u // Tk) % Tk, i, h
+
+
+@pytest.mark.parametrize("tokens,heads,E,n", [(8, 1, 4, 512), (16, 2, 4, 512), (8, 1, 8, 512), (128, 32, 8, 32768), (16, 4, 1, 64)])
+def test_layout_meets_every_key_once_and_rolls_agree(tokens, heads, E, n):
+    desc = AttnDesc(tokens, heads, E)
+    g0 = inputs.rng(5, tokens)
+    Q = g0.integers(1, 50, (tokens, heads, 2)).astype(np.float64)
+    K = g0.integers(1, 50, (tokens, heads, 2)).astype(np.float64)
+    Qs, Ks, _ = inputs.pack_attention_operands(Q, K, K, E, n)
+    R = n // (E * tokens * heads)
+    seen = np.zeros((tokens, heads, tokens), dtype=np.int64)
+    for g in range(desc.groups()):
+        key, i, h = _key_of(desc, n, g)
+        # the rotation as an array roll: left by g * E tokens = g * E * heads * R slots
+        prod = (Qs * np.roll(Ks, -g * E * heads * R, axis=1)).sum(0)
+        want = (Q[i, h, :] * K[key, h, :]).sum(1)
+        assert np.array_equal(prod, want)
+        np.add.at(seen, (i[::R], h[::R], key[::R]), 1)
+    assert (seen == 1).all()          # the score row of (query i, head h) holds every key exactly once
+
+
+def _keys(cl, o, desc):
+    tok, lad = o.attention_rotations(desc)
+    return {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in tok + lad}
+
+
+def _unpack_rows(desc, n, vals_by_group):
+    """[groups][n] slot values -> [tokens][heads][tokens (key)] using the layout's definition."""
+    out = np.full((desc.tokens, desc.heads, desc.tokens), np.nan)
+    for g, vals in enumerate(vals_by_group):
+        key, i, h = _key_of(desc, n, g)
+        out[i, h, key] = vals
+    return out
+
+
+@pytest.mark.parametrize("tokens,heads,E,dim,seed", [(8, 1, 4, 8, 81), (16, 2, 4, 4, 82)])
+def test_attention_against_clear_pipeline_and_softmax_attention(tokens, heads, E, dim, seed):
+    P = params(10, 13, 4, 4)
+    o = P.oracle
+    cl = Client(P, seed)
+    desc = AttnDesc(tokens, heads, E)
+    level, scale, rounds = 13, 2.0 ** 50, 1
+    c = attention_case(seed, tokens, heads, dim, dim, rounds)
+    Qs, Ks, Vs = inputs.pack_attention_operands(c["Q"], c["K"], c["V"], E, P.n)
+    q = np.stack([cl.encrypt_slots(z, scale, level) for z in Qs])
+    k = np.stack([cl.encrypt_slots(z, scale, level) for z in Ks])
+    v = np.stack([cl.encrypt_slots(z, scale, level) for z in Vs])
+    rlk, keys = cl.relin_key(), _keys(cl, o, desc)
+    # scores: slot (e, i, h) of group g is Q[i, h] . K[key, h]
+    S = o.attention_scores(desc, q, k, rlk, keys)
+    ss = scale * scale / float(P.q[level - 1])
+    rows = _unpack_rows(desc, P.n, [cl.decrypt_slots(S[g], ss).real for g in range(desc.groups())])
+    assert np.abs(rows - c["S"].transpose(1, 0, 2)).max() < 2.0 ** -20
+    # Softmax over rows spread across the groups
+    Pr, sp = o.softmax_rows(desc, S, ss, c["shift"], rounds, c["exp_coeffs"], c["rsqrt_coeffs"], rlk, keys)
+    assert Pr.shape[2] == level - 1 - 3 - rounds * 6
+    probs = _unpack_rows(desc, P.n, [cl.decrypt_slots(Pr[g], sp).real for g in range(desc.groups())])
+    assert np.abs(probs - c["probs_clear"].transpose(1, 0, 2)).max() < 2.0 ** -20
+    assert np.abs(probs.sum(2) - 1.0).max() < 0.1
+    # probability x value, and the three steps in one call give the same integers
+    out = o.attention_values(desc, Pr, v, rlk, keys)
+    whole, so = o.attention(desc, q, k, v, scale, scale, c["shift"], rounds, c["exp_coeffs"], c["rsqrt_coeffs"], rlk, keys)
+    assert np.array_equal(out, whole) and out.shape[2] == Pr.shape[2] - 1
+    e, i, h = inputs.attention_slot_index(tokens, heads, E, P.n)
+    for d in range(dim):
+        got = cl.decrypt_slots(out[d], so).real
+        assert np.abs(got - c["out_clear"][i, h, d]).max() < 2.0 ** -19       # every block e holds the output (query layout)
+        assert np.abs(got - c["out_true"][i, h, d]).max() < 0.05
+
+
+def test_single_group_needs_no_token_rotation_and_one_block_no_ladder():
+    P = params(10, 4, 2, 2)
+    o = P.oracle
+    assert o.attention_rotations(AttnDesc(8, 1, 8)) == ([], [8 * 1 * 8 * k for k in (1, 2, 4)])
+    assert o.attention_rotations(AttnDesc(16, 4, 1)) == ([g * 4 * 8 for g in range(1, 16)], [])
+    with pytest.raises(ValueError):
+        o.attention_rotations(AttnDesc(8, 1, 3))
