@@ -532,10 +532,11 @@ def run_cuda(args):
 
     layer = None
     if not args.no_extras and not args.no_layer:
-        del ws, h_cts, h_W, h_outs
+        # the layer's down projection needs most of the device: keep only the rotation keys (reused) and the context
+        del ws, h_cts, h_W, h_outs, hoist_out, polys, probe_scratch, outs, cts, W, rot_out, mul_out, rot_keys, proj_keys
         ctx._ws = None
         torch.cuda.empty_cache()
-        layer = layer_submetrics(ctx, residues, allp, gen, dev, args.layer_reps)
+        layer = layer_submetrics(ctx, residues, allp, gen, dev, args.layer_reps, keys)
 
     pk, pk_kind = peaks()
     limb_ntts = NTT_BATCH * L
@@ -638,7 +639,7 @@ def run_cuda(args):
 
 
 # ----------------------------------------------------------------- one decoder layer's linear work and products
-def layer_submetrics(ctx, residues, allp, gen, dev, reps):
+def layer_submetrics(ctx, residues, allp, gen, dev, reps, have_keys):
     """CUDA-event means of one Llama-3-8B decoder layer's homomorphic linear work at 128 tokens (16 shards of 8, B = 64,
     giant steps summed before one ModDown): query/key/value as one call sharing their baby steps, output, gate and up as
     one call, down; and the attention products as ciphertext x ciphertext multiplies at level 24: 2048 + 2048 products,
@@ -654,8 +655,12 @@ def layer_submetrics(ctx, residues, allp, gen, dev, reps):
         return (torch.randn((d_in, d_out), generator=gen, device=dev, dtype=torch.float64) * 0.02).contiguous()
 
     def keys_for(shapes):
+        """Rotation keys of the shapes: the ones the caller already holds (rotation in slots -> key), new ones otherwise."""
         rots = sorted(set(r for d_in, d_out in shapes for r in ctx.linear_proj_rotations(d_in, d_out, T_SHARD, SHARDS, BABY)))
-        return [binding.SwitchKey(residues(allp, DNUM, 2), ctx.galois_element(r)) for r in rots]
+        for r in rots:
+            if r not in have_keys:
+                have_keys[r] = binding.SwitchKey(residues(allp, DNUM, 2), ctx.galois_element(r))
+        return [have_keys[r] for r in rots]
 
     def timed(f):
         f()

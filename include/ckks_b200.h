@@ -294,6 +294,50 @@ int32_t ckks_softmax(ckks_ctx *ctx, const ckks_softmax_desc *desc, const ckks_ct
                      uint32_t nkeys, ckks_ct *out, void *ws, size_t ws_bytes, void *stream);
 size_t ckks_softmax_workspace_bytes(const ckks_ctx *ctx, const ckks_softmax_desc *desc, uint32_t level);
 
+/* ---- Attention in a diagonal-block layout (Section 2.2: QK^T and PV multiply two encrypted operands; Section 4 names a
+ * layout in which QK^T yields score diagonals that Softmax and PV consume without repacking, and does not define it) ----
+ * The layout built here.  Every operand and score ciphertext uses the slot index
+ *     slot = ((e * tokens + i) * heads + h) * R + r,     R = n / (diag_block * tokens * heads),
+ * i a token position, h a head, e < diag_block, r trailing copies (tokens and diag_block powers of two, diag_block
+ * dividing tokens, diag_block * tokens * heads dividing n).  Operands are one ciphertext per channel d:
+ *     q[d]: Q[i, h, d] in every block e;      k[d], v[d]: token (i + e) mod tokens in block e.
+ * (The 1/sqrt(dim) factor and, for grouped-query attention, the repetition of key/value heads are the caller's: they
+ * are part of the projections that produce the operands.  No causal mask is applied.)
+ *   ckks_attention_scores: S_g = rescale(sum_d q[d] * rot_g(k[d])) for g < groups = tokens / diag_block, rot_g the left
+ *     rotation by g * diag_block * heads * R slots (cyclic over the flattened (e, i) index), the sum over d relinearised
+ *     once (ckks_mul_relin_sum).  Slot (e, i, h) of S_g is the score of query i, head h against one key token; over all
+ *     g and e every key token occurs exactly once, so the score row of (i, h) is the set of slots (e, i, h) of the S_g.
+ *     scores: host array of `groups` descriptors with buffers for level - 1 limbs.  Every rotated operand is bit-identical
+ *     to ckks_rotate's.  Workspace: ckks_attention_scores_workspace_bytes holds all rotated operands at once
+ *     ((groups - 1) * dim ciphertexts); any workspace that holds one group's is accepted and the groups are then taken in passes.
+ *   ckks_softmax_rows: Algorithm 1 on rows spread that way.  Per group u_g = p_exp(S_g - shift); per round
+ *     t = rescale(sum_g u_g^2) (one relinearisation), t += rot(t, tokens * heads * R * 2^k) for k < log2 diag_block (cyclic
+ *     over e: the row sum in every slot of the row), lambda = p_rsqrt_j(t) once for all groups, u_g = rescale(rescale(lambda
+ *     u_g)^2).  desc->row_len, exp_m and rsqrt_m are ignored (both polynomials as ckks_poly_eval_tree).  in, out: host
+ *     arrays of `groups` descriptors; out buffers sized for the input level.
+ *   ckks_attention_values: out[d] = ladder(rescale(sum_g P_g * rot_g(v[d] truncated to P's level))), the same ladder
+ *     over e: slot (e, i, h) of out[d] holds sum over all key tokens of probability x value, in every block e (the query
+ *     operand's layout).  out: dim_v descriptors with buffers for P's level - 1.
+ *   ckks_attention: the three in a row (scores at level - 1, then the Softmax's levels, then one more).
+ * keys must hold the rotations ckks_attention_rotations lists (token rotations first, then the ladder).
+ * Errors: ARG, LEVEL, SCALE, NO_KEY, WORKSPACE, UNSUPPORTED (shape rules above), RANGE (a polynomial constant). */
+typedef struct { uint32_t tokens, heads, diag_block; } ckks_attn_desc;
+int32_t ckks_attention_rotations(const ckks_ctx *ctx, const ckks_attn_desc *desc, int64_t *rots, uint32_t cap);
+int32_t ckks_attention_scores(ckks_ctx *ctx, const ckks_attn_desc *desc, const ckks_ct *q, const ckks_ct *k, uint32_t dim,
+                              const ckks_evk *rlk, const ckks_evk *keys, uint32_t nkeys, ckks_ct *scores, void *ws, size_t ws_bytes, void *stream);
+size_t ckks_attention_scores_workspace_bytes(const ckks_ctx *ctx, const ckks_attn_desc *desc, uint32_t level, uint32_t dim);
+int32_t ckks_attention_values(ckks_ctx *ctx, const ckks_attn_desc *desc, const ckks_ct *probs, const ckks_ct *v, uint32_t dim_v,
+                              const ckks_evk *rlk, const ckks_evk *keys, uint32_t nkeys, ckks_ct *out, void *ws, size_t ws_bytes, void *stream);
+size_t ckks_attention_values_workspace_bytes(const ckks_ctx *ctx, const ckks_attn_desc *desc, uint32_t level);
+
+int32_t ckks_softmax_rows(ckks_ctx *ctx, const ckks_attn_desc *desc, const ckks_softmax_desc *sm, const ckks_ct *in, const ckks_evk *rlk,
+                          const ckks_evk *keys, uint32_t nkeys, ckks_ct *out, void *ws, size_t ws_bytes, void *stream);
+size_t ckks_softmax_rows_workspace_bytes(const ckks_ctx *ctx, const ckks_attn_desc *desc, const ckks_softmax_desc *sm, uint32_t level);
+int32_t ckks_attention(ckks_ctx *ctx, const ckks_attn_desc *desc, const ckks_softmax_desc *sm, const ckks_ct *q, const ckks_ct *k, uint32_t dim,
+                       const ckks_ct *v, uint32_t dim_v, const ckks_evk *rlk, const ckks_evk *keys, uint32_t nkeys, ckks_ct *out,
+                       void *ws, size_t ws_bytes, void *stream);
+size_t ckks_attention_workspace_bytes(const ckks_ctx *ctx, const ckks_attn_desc *desc, const ckks_softmax_desc *sm, uint32_t level, uint32_t dim);
+
 /* ---- Rot_k (Section 2.1, Rot + KeySwitch) ----------------------------------
  * Plain: apply sigma_g (g = key->galois) to both components, key-switch the
  * permuted c1: out = (sigma c0 + k0, k1).  Key switch = iNTT, centred ModUp

@@ -27,6 +27,9 @@ EXPORTS = [
     "ckks_encode_range_flag", "ckks_mul_plain_acc", "ckks_add", "ckks_mul_relin", "ckks_rotate",
     "ckks_rotate_hoisted", "ckks_rescale", "ckks_linear_proj", "ckks_linear_proj_workspace_bytes",
     "ckks_linear_proj_rotations", "ckks_kernel_launches", "ckks_device_status", "ckks_rescale_static",
+    "ckks_attention_rotations", "ckks_attention_scores", "ckks_attention_scores_workspace_bytes", "ckks_attention_values",
+    "ckks_attention_values_workspace_bytes", "ckks_softmax_rows", "ckks_softmax_rows_workspace_bytes", "ckks_attention",
+    "ckks_attention_workspace_bytes",
     "ckks_ntt_butterfly_probe", "ckks_mul_relin_sum", "ckks_mul_relin_batch", "ckks_rotate_batch", "ckks_rotate_sum", "ckks_softmax", "ckks_softmax_workspace_bytes", "ckks_poly_eval_bsgs", "ckks_poly_eval_bsgs_workspace_bytes", "ckks_mul_const", "ckks_add_const", "ckks_poly_eval", "ckks_poly_eval_tree", "ckks_linear_proj_multi", "ckks_linear_proj_multi_workspace_bytes",
 ]
 
@@ -52,6 +55,10 @@ class CSoftmaxDesc(C.Structure):
     _fields_ = [("shift", C.c_double), ("rounds", C.c_uint32), ("row_len", C.c_uint32), ("exp_degree", C.c_uint32),
                 ("rsqrt_degree", C.c_uint32), ("exp_coeffs", C.POINTER(C.c_double)), ("rsqrt_coeffs", C.POINTER(C.c_double)),
                 ("exp_m", C.c_uint32), ("rsqrt_m", C.c_uint32)]
+
+
+class CAttnDesc(C.Structure):
+    _fields_ = [("tokens", C.c_uint32), ("heads", C.c_uint32), ("diag_block", C.c_uint32)]
 
 
 class CProjDesc(C.Structure):
@@ -93,6 +100,19 @@ def load():
         "ckks_poly_eval_bsgs_workspace_bytes": (sz, [vp, u32, u32, u32]),
         "ckks_softmax": (i32, [vp, C.POINTER(CSoftmaxDesc), C.POINTER(CCt), C.POINTER(CEvk), C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
         "ckks_softmax_workspace_bytes": (sz, [vp, C.POINTER(CSoftmaxDesc), u32]),
+        "ckks_attention_rotations": (i32, [vp, C.POINTER(CAttnDesc), C.POINTER(i64), u32]),
+        "ckks_attention_scores": (i32, [vp, C.POINTER(CAttnDesc), C.POINTER(CCt), C.POINTER(CCt), u32, C.POINTER(CEvk), C.POINTER(CEvk), u32,
+                                        C.POINTER(CCt), vp, sz, vp]),
+        "ckks_attention_scores_workspace_bytes": (sz, [vp, C.POINTER(CAttnDesc), u32, u32]),
+        "ckks_attention_values": (i32, [vp, C.POINTER(CAttnDesc), C.POINTER(CCt), C.POINTER(CCt), u32, C.POINTER(CEvk), C.POINTER(CEvk), u32,
+                                        C.POINTER(CCt), vp, sz, vp]),
+        "ckks_attention_values_workspace_bytes": (sz, [vp, C.POINTER(CAttnDesc), u32]),
+        "ckks_softmax_rows": (i32, [vp, C.POINTER(CAttnDesc), C.POINTER(CSoftmaxDesc), C.POINTER(CCt), C.POINTER(CEvk), C.POINTER(CEvk), u32,
+                                    C.POINTER(CCt), vp, sz, vp]),
+        "ckks_softmax_rows_workspace_bytes": (sz, [vp, C.POINTER(CAttnDesc), C.POINTER(CSoftmaxDesc), u32]),
+        "ckks_attention": (i32, [vp, C.POINTER(CAttnDesc), C.POINTER(CSoftmaxDesc), C.POINTER(CCt), C.POINTER(CCt), u32, C.POINTER(CCt), u32,
+                                 C.POINTER(CEvk), C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
+        "ckks_attention_workspace_bytes": (sz, [vp, C.POINTER(CAttnDesc), C.POINTER(CSoftmaxDesc), u32, u32]),
         "ckks_rotate_sum": (i32, [vp, C.POINTER(CCt), C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
         "ckks_rotate_batch": (i32, [vp, C.POINTER(CCt), u32, C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
         "ckks_mul_relin_batch": (i32, [vp, C.POINTER(CCt), C.POINTER(CCt), u32, C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
@@ -389,6 +409,106 @@ class Context:
                                         _stream_ptr(stream)))
         res = Ciphertext(out.data.view(-1)[: 2 * co.level * self.N].view(2, co.level, self.N), co.scale)
         return res
+
+    # ------------------------------------------------------------ attention in the diagonal-block layout
+    @staticmethod
+    def _softmax_desc(shift, rounds, exp_coeffs, rsqrt_coeffs, row_len=0):
+        ec = (C.c_double * len(exp_coeffs))(*[float(v) for v in exp_coeffs])
+        flat = [float(v) for row in rsqrt_coeffs for v in row] if rounds else []
+        rc = (C.c_double * max(1, len(flat)))(*flat)
+        rdeg = (len(rsqrt_coeffs[0]) - 1) if rounds else 0
+        d = CSoftmaxDesc(float(shift), rounds, row_len, len(exp_coeffs) - 1, rdeg, C.cast(ec, C.POINTER(C.c_double)),
+                         C.cast(rc, C.POINTER(C.c_double)), 0, 0)
+        d._keep = (ec, rc)          # the arrays must outlive the descriptor
+        return d
+
+    def _cut(self, out: Ciphertext, c: CCt) -> Ciphertext:
+        """The first c.level limbs per component of a buffer written densely as [2][c.level][N]."""
+        return Ciphertext(out.data.view(-1)[: 2 * c.level * self.N].view(2, c.level, self.N), c.scale)
+
+    def attention_rotations(self, tokens: int, heads: int, diag_block: int):
+        d = CAttnDesc(tokens, heads, diag_block)
+        n = load().ckks_attention_rotations(self._h, C.byref(d), None, 0)
+        if n < 0:
+            raise CkksError(n)
+        buf = (C.c_int64 * max(n, 1))()
+        load().ckks_attention_rotations(self._h, C.byref(d), buf, n)
+        return list(buf)[:n]
+
+    def attention_scores(self, q, k, rlk: SwitchKey, keys, tokens, heads, diag_block, ws: torch.Tensor = None, stream=None):
+        """Score ciphertexts S_g (one per group of diag_block diagonals) from the channel operands q[d], k[d]."""
+        d = CAttnDesc(tokens, heads, diag_block)
+        level, G = q[0].level, tokens // diag_block
+        outs = [self.empty_ct(level - 1) for _ in range(G)]
+        if ws is None:
+            ws = self.workspace(int(load().ckks_attention_scores_workspace_bytes(self._h, C.byref(d), level, len(q))))
+        qa = (CCt * len(q))(*[_cct(x) for x in q])
+        ka = (CCt * len(k))(*[_cct(x) for x in k])
+        oa = (CCt * G)(*[_cct(x) for x in outs])
+        ck = CEvk(_dev_u64(rlk.data).data_ptr(), 0)
+        ra = (CEvk * max(1, len(keys)))(*[CEvk(_dev_u64(x.data).data_ptr(), x.galois) for x in keys])
+        self._check(load().ckks_attention_scores(self._h, C.byref(d), qa, ka, len(q), C.byref(ck), ra, len(keys), oa, ws.data_ptr(), ws.numel(),
+                                                 _stream_ptr(stream)))
+        for o, c in zip(outs, oa):
+            o.scale = c.scale
+        return outs
+
+    def softmax_rows(self, cts, shift, rounds, exp_coeffs, rsqrt_coeffs, rlk: SwitchKey, keys, tokens, heads, diag_block, stream=None):
+        """Softmax by doubling on score rows spread over the groups' ciphertexts (slots (e, i, h) of every group)."""
+        d = CAttnDesc(tokens, heads, diag_block)
+        sd = self._softmax_desc(shift, rounds, exp_coeffs, rsqrt_coeffs)
+        level = cts[0].level
+        need = int(load().ckks_softmax_rows_workspace_bytes(self._h, C.byref(d), C.byref(sd), level))
+        if need == 0:
+            raise CkksError(ERR_ARG)
+        ws = self.workspace(need)
+        outs = [self.empty_ct(level) for _ in cts]
+        ia = (CCt * len(cts))(*[_cct(x) for x in cts])
+        oa = (CCt * len(outs))(*[_cct(x) for x in outs])
+        ck = CEvk(_dev_u64(rlk.data).data_ptr(), 0)
+        ra = (CEvk * max(1, len(keys)))(*[CEvk(_dev_u64(x.data).data_ptr(), x.galois) for x in keys])
+        self._check(load().ckks_softmax_rows(self._h, C.byref(d), C.byref(sd), ia, C.byref(ck), ra, len(keys), oa, ws.data_ptr(), ws.numel(),
+                                             _stream_ptr(stream)))
+        return [self._cut(o, c) for o, c in zip(outs, oa)]
+
+    def attention_values(self, probs, v, rlk: SwitchKey, keys, tokens, heads, diag_block, stream=None):
+        """Output channels sum over key tokens of probability x value, in the query operand's layout."""
+        d = CAttnDesc(tokens, heads, diag_block)
+        lp = probs[0].level
+        ws = self.workspace(int(load().ckks_attention_values_workspace_bytes(self._h, C.byref(d), lp)))
+        outs = [self.empty_ct(lp - 1) for _ in v]
+        pa = (CCt * len(probs))(*[_cct(x) for x in probs])
+        va = (CCt * len(v))(*[_cct(x) for x in v])
+        oa = (CCt * len(outs))(*[_cct(x) for x in outs])
+        ck = CEvk(_dev_u64(rlk.data).data_ptr(), 0)
+        ra = (CEvk * max(1, len(keys)))(*[CEvk(_dev_u64(x.data).data_ptr(), x.galois) for x in keys])
+        self._check(load().ckks_attention_values(self._h, C.byref(d), pa, va, len(v), C.byref(ck), ra, len(keys), oa, ws.data_ptr(), ws.numel(),
+                                                 _stream_ptr(stream)))
+        for o, c in zip(outs, oa):
+            o.scale = c.scale
+        return outs
+
+    def attention(self, q, k, v, shift, rounds, exp_coeffs, rsqrt_coeffs, rlk: SwitchKey, keys, tokens, heads, diag_block,
+                  ws: torch.Tensor = None, stream=None):
+        """Scores, Softmax over the score rows and probability x value in one call; returns the output channels."""
+        d = CAttnDesc(tokens, heads, diag_block)
+        sd = self._softmax_desc(shift, rounds, exp_coeffs, rsqrt_coeffs)
+        level = q[0].level
+        need = int(load().ckks_attention_workspace_bytes(self._h, C.byref(d), C.byref(sd), level, len(q)))
+        if need == 0:
+            raise CkksError(ERR_ARG)
+        if ws is None:
+            ws = self.workspace(need)
+        outs = [self.empty_ct(level - 1) for _ in v]
+        qa = (CCt * len(q))(*[_cct(x) for x in q])
+        ka = (CCt * len(k))(*[_cct(x) for x in k])
+        va = (CCt * len(v))(*[_cct(x) for x in v])
+        oa = (CCt * len(outs))(*[_cct(x) for x in outs])
+        ck = CEvk(_dev_u64(rlk.data).data_ptr(), 0)
+        ra = (CEvk * max(1, len(keys)))(*[CEvk(_dev_u64(x.data).data_ptr(), x.galois) for x in keys])
+        self._check(load().ckks_attention(self._h, C.byref(d), C.byref(sd), qa, ka, len(q), va, len(v), C.byref(ck), ra, len(keys), oa,
+                                          ws.data_ptr(), ws.numel(), _stream_ptr(stream)))
+        return [self._cut(o, c) for o, c in zip(outs, oa)]
 
     def rotate_sum(self, cts, keys, out: Ciphertext = None, ws: torch.Tensor = None, stream=None):
         """sum_i rotate(cts[i], keys[i]) formed in the key-switching basis and divided by P once."""

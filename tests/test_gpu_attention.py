@@ -1,0 +1,131 @@
+"""GPU parity: attention in the diagonal-block layout (scores, Softmax over rows spread across ciphertexts, probability x
+value), every output limb bit-exact against the CPU checker's compositions, stage by stage and in one call."""
+import numpy as np
+import pytest
+
+from oracle.ckks_oracle import AttnDesc
+from paper_2609_12378_b200 import binding, inputs
+from tests.harness import Client, attention_case, params
+
+pytestmark = pytest.mark.gpu
+
+
+def _setup(log_n, L, K, dnum, level, tokens, heads, E, dim, dim_v, seed, rounds=1):
+    from tests.gpu_util import context, ct_dev, key_dev
+    P, ctx = params(log_n, L, K, dnum), context(log_n, L, K, dnum)
+    o = P.oracle
+    cl = Client(P, seed)
+    desc = AttnDesc(tokens, heads, E)
+    scale = 2.0 ** 50
+    c = attention_case(seed, tokens, heads, dim, dim_v, rounds)
+    Qs, Ks, Vs = inputs.pack_attention_operands(c["Q"], c["K"], c["V"], E, P.n)
+    q = np.stack([cl.encrypt_slots(z, scale, level) for z in Qs])
+    k = np.stack([cl.encrypt_slots(z, scale, level) for z in Ks])
+    v = np.stack([cl.encrypt_slots(z, scale, level) for z in Vs])
+    tok, lad = o.attention_rotations(desc)
+    assert ctx.attention_rotations(tokens, heads, E) == tok + lad
+    keys = {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in tok + lad}
+    rlk = cl.relin_key()
+    dev = dict(q=[ct_dev(x, scale) for x in q], k=[ct_dev(x, scale) for x in k], v=[ct_dev(x, scale) for x in v],
+               rlk=key_dev(rlk, 0), keys=[key_dev(kk, ge) for ge, kk in keys.items()])
+    return P, ctx, o, cl, desc, c, scale, q, k, v, rlk, keys, dev
+
+
+@pytest.mark.parametrize("log_n,L,K,dnum,level,tokens,heads,E,dim,dim_v", [
+    (10, 13, 4, 4, 13, 8, 1, 4, 8, 8),        # one head, two groups of four diagonals
+    (10, 13, 4, 4, 13, 16, 2, 4, 4, 3),       # two heads, four groups
+    (10, 13, 4, 4, 12, 8, 2, 8, 2, 2),        # a single group: no token rotation, ladder of three; level below L
+    (10, 13, 4, 4, 13, 16, 4, 1, 2, 1),       # one diagonal per ciphertext: sixteen groups, no ladder
+])
+def test_attention_stages_bit_exact(log_n, L, K, dnum, level, tokens, heads, E, dim, dim_v):
+    from tests.gpu_util import host
+    P, ctx, o, cl, desc, c, scale, q, k, v, rlk, keys, dev = _setup(log_n, L, K, dnum, level, tokens, heads, E, dim, dim_v, 600 + tokens + heads + E)
+    a = (tokens, heads, E)
+    ss = scale * scale / float(P.q[level - 1])
+    S = o.attention_scores(desc, q, k, rlk, keys)
+    dS = ctx.attention_scores(dev["q"], dev["k"], dev["rlk"], dev["keys"], *a)
+    assert len(dS) == desc.groups()
+    for g in range(desc.groups()):
+        assert dS[g].scale == ss and dS[g].level == level - 1
+        assert np.array_equal(host(dS[g].data), S[g]), g
+    Pr, sp = o.softmax_rows(desc, S, ss, c["shift"], 1, c["exp_coeffs"], c["rsqrt_coeffs"], rlk, keys)
+    dP = ctx.softmax_rows(dS, c["shift"], 1, c["exp_coeffs"], c["rsqrt_coeffs"], dev["rlk"], dev["keys"], *a)
+    for g in range(desc.groups()):
+        assert dP[g].scale == sp and dP[g].level == Pr.shape[2]
+        assert np.array_equal(host(dP[g].data), Pr[g]), g
+    out = o.attention_values(desc, Pr, v, rlk, keys)
+    dO = ctx.attention_values(dP, dev["v"], dev["rlk"], dev["keys"], *a)
+    for d in range(dim_v):
+        assert np.array_equal(host(dO[d].data), out[d]), d
+    # the three steps in one call: the same integers, and the decrypted outputs are Softmax attention
+    whole = ctx.attention(dev["q"], dev["k"], dev["v"], c["shift"], 1, c["exp_coeffs"], c["rsqrt_coeffs"], dev["rlk"], dev["keys"], *a)
+    assert ctx.device_status() == binding.OK
+    e, i, h = inputs.attention_slot_index(tokens, heads, E, P.n)
+    for d in range(dim_v):
+        assert whole[d].scale == dO[d].scale
+        arr = host(whole[d].data)
+        assert np.array_equal(arr, out[d]), d
+        got = cl.decrypt_slots(arr, whole[d].scale).real
+        assert np.abs(got - c["out_clear"][i, h, d]).max() < 2.0 ** -19
+        assert np.abs(got - c["out_true"][i, h, d]).max() < 0.05
+
+
+def test_attention_scores_in_passes_and_errors():
+    """A workspace that holds one group's rotated operands at a time gives the same scores; missing keys, short
+    workspaces, shapes that do not tile the slots and operands at different levels are refused before any launch."""
+    import torch
+
+    from tests.gpu_util import host
+    P, ctx, o, cl, desc, c, scale, q, k, v, rlk, keys, dev = _setup(10, 13, 4, 4, 5, 16, 2, 4, 3, 1, 640)
+    a = (16, 2, 4)
+    full = ctx.attention_scores(dev["q"], dev["k"], dev["rlk"], dev["keys"], *a)
+    lib = binding.load()
+    import ctypes as C
+    d = binding.CAttnDesc(*a)
+    need = lib.ckks_attention_scores_workspace_bytes(ctx._h, C.byref(d), 5, 3)
+    ct = 2 * 5 * P.N * 8
+    small = torch.empty(need - 2 * 3 * ct, dtype=torch.uint8, device="cuda")          # room for one group's operands only
+    again = ctx.attention_scores(dev["q"], dev["k"], dev["rlk"], dev["keys"], *a, ws=small)
+    for x, y in zip(full, again):
+        assert np.array_equal(host(x.data), host(y.data))
+    launches = binding.kernel_launches()
+    with pytest.raises(binding.CkksError) as e:
+        ctx.attention_scores(dev["q"], dev["k"], dev["rlk"], dev["keys"][1:], *a)
+    assert e.value.code == binding.ERR_NO_KEY
+    with pytest.raises(binding.CkksError) as e:
+        ctx.attention_scores(dev["q"], dev["k"], dev["rlk"], dev["keys"], *a, ws=torch.empty(1024, dtype=torch.uint8, device="cuda"))
+    assert e.value.code == binding.ERR_WORKSPACE
+    with pytest.raises(binding.CkksError) as e:
+        ctx.attention_scores(dev["q"], dev["k"], dev["rlk"], dev["keys"], 16, 3, 4)        # 4 * 16 * 3 does not divide the slots
+    assert e.value.code == binding.ERR_UNSUPPORTED
+    with pytest.raises(binding.CkksError) as e:
+        ctx.attention_rotations(16, 2, 3)
+    assert e.value.code == binding.ERR_UNSUPPORTED
+    low = binding.Ciphertext(dev["k"][0].data[:, :4].contiguous(), scale)
+    with pytest.raises(binding.CkksError) as e:
+        ctx.attention_scores(dev["q"], [low] + dev["k"][1:], dev["rlk"], dev["keys"], *a)
+    assert e.value.code == binding.ERR_LEVEL
+    with pytest.raises(binding.CkksError) as e:
+        ctx.softmax_rows(full, c["shift"], 1, c["exp_coeffs"], c["rsqrt_coeffs"], dev["rlk"], dev["keys"], *a)   # 4 limbs are too few
+    assert e.value.code == binding.ERR_LEVEL
+    assert binding.kernel_launches() == launches
+
+
+@pytest.mark.slow
+def test_attention_full_ring():
+    """N = 2^16 with the decoder layer's attention shape in the slots (128 tokens, 32 heads, 8 diagonals per ciphertext:
+    16 groups, every slot used) and a few channels: bit-exact in one call, and Softmax attention after decryption."""
+    from tests.gpu_util import host
+    tokens, heads, E, dim, dim_v, level = 128, 32, 8, 2, 1, 13
+    P, ctx, o, cl, desc, c, scale, q, k, v, rlk, keys, dev = _setup(16, 24, 8, 3, level, tokens, heads, E, dim, dim_v, 660)
+    want, so = o.attention(desc, q, k, v, scale, scale, c["shift"], 1, c["exp_coeffs"], c["rsqrt_coeffs"], rlk, keys)
+    got = ctx.attention(dev["q"], dev["k"], dev["v"], c["shift"], 1, c["exp_coeffs"], c["rsqrt_coeffs"], dev["rlk"], dev["keys"], tokens, heads, E)
+    assert ctx.device_status() == binding.OK
+    e, i, h = inputs.attention_slot_index(tokens, heads, E, P.n)
+    for d in range(dim_v):
+        assert got[d].scale == so
+        arr = host(got[d].data)
+        assert np.array_equal(arr, want[d]), d
+        sl = cl.decrypt_slots(arr, so).real
+        assert np.abs(sl - c["out_clear"][i, h, d]).max() < 2.0 ** -14
+        assert np.abs(sl - c["out_true"][i, h, d]).max() < 0.05

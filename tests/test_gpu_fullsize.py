@@ -173,12 +173,12 @@ def test_attention_product_batch_full_size():
     g = inputs.rng(1005, 9)
     rlk = cl.relin_key()
     drlk = key_dev(rlk, 0)
-    # 16 distinct ciphertexts; product i pairs a[i % 16] with b[(5 i + 3) % 16], so all 64 pairs differ
+    # 16 distinct ciphertexts on either side; product i pairs a[i % 16] with b[(5 i + 3 + i / 16) % 16], so all 64 pairs differ
     za, zb = g.uniform(-1, 1, (16, P.n)), g.uniform(-1, 1, (16, P.n))
     a = [cl.encrypt_slots(z, scale, level) for z in za]
     b = [cl.encrypt_slots(z, scale, level) for z in zb]
     da, db = [ct_dev(x, scale) for x in a], [ct_dev(x, scale) for x in b]
-    ia, ib = [i % 16 for i in range(64)], [(5 * i + 3) % 16 for i in range(64)]
+    ia, ib = [i % 16 for i in range(64)], [(5 * i + 3 + i // 16) % 16 for i in range(64)]
     assert len(set(zip(ia, ib))) == 64
     outs = ctx.mul_relin_batch([da[i] for i in ia], [db[j] for j in ib], drlk)
     assert ctx.device_status() == binding.OK
