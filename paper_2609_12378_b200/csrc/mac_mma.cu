@@ -295,10 +295,12 @@ __device__ __forceinline__ void mbar_arrive_cp_async(uint32_t bar) {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long limit) {
     const long long t0 = clock64();
     uint32_t ok = 0;
-    for (;;) {
+    // a non-blocking test first (try_wait may itself sleep for a while, which would make a limit of zero meaningless)
+    asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    while (!ok && clock64() - t0 < limit) {
         asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
                      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-        if (ok || clock64() - t0 > limit) break;
     }
     return __all_sync(0xffffffffu, ok != 0);
 }
