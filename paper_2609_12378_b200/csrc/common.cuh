@@ -26,10 +26,10 @@ struct DevTables {
     const ulonglong2 *tw_fwd;  // [T][N] {psi^bitrev(i), Shoup companion}, index m+i
     const ulonglong2 *tw_inv;  // [T][N] inverses of the same
     const ulonglong2 *n_inv;   // [T] {N^-1, Shoup}
-    // fp64 copies for the double-precision NTT path (N = 2^16 only): w as a double, same indexing (w/q is formed
-    // in the kernel as w * (1/q): half the table bytes for one extra multiply per twiddle)
+    // fp64 copies for the double-precision NTT path (N = 2^16 only): the centred representative of w as a double, same
+    // indexing (w/q is formed in the kernel as w * (1/q): half the table bytes for one extra multiply per twiddle)
     const double *twd_fwd, *twd_inv;    // [T][N]
-    const double2 *n_inv_d;             // [T] {N^-1, N^-1/q}
+    const double2 *n_inv_d;             // [T][2] {N^-1, N^-1/q}, {w N^-1, that/q} for the inverse's last twiddle w, all centred
     // ModUp, per level l (1..L), digit j, source a < alpha:
     const ulonglong2 *up_hat_inv;  // [(L+1)][dnum][alpha]        {qhat^-1 mod q_src, Shoup}
     const u64 *up_hat_mod;         // [(L+1)][dnum][alpha][T]     qhat mod target

@@ -196,14 +196,18 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
     std::vector<ulonglong2> ninv(T), twf((size_t)T * N), twi((size_t)T * N);
     const bool fp = prm->log_n == 16;
     std::vector<double> twdf(fp ? (size_t)T * N : 0), twdi(fp ? (size_t)T * N : 0);
-    std::vector<double2> ninvd(T);
+    std::vector<double2> ninvd((size_t)2 * T);
     for (uint32_t t = 0; t < T; t++) {
         u64 m = mod[t];
         mu[t] = (u64)((((u128)1) << 112) / m);
         mu64[t] = (u64)((((u128)1) << 64) / m);
         modd[t] = make_double2((double)m, 1.0 / (double)m);
         ninv[t] = h_pair(h_inv(N % m, m), m);
-        ninvd[t] = make_double2((double)ninv[t].x, (double)ninv[t].x / (double)m);
+        auto centred_pair = [&](u64 v) {
+            const double d = v > m / 2 ? -(double)(m - v) : (double)v;
+            return make_double2(d, d * (1.0 / (double)m));
+        };
+        ninvd[2 * t] = centred_pair(ninv[t].x);
         u64 psi = h_min_root(m, N), psi_inv = h_inv(psi, m);
         std::vector<u64> pw(N), pwi(N);
         pw[0] = pwi[0] = 1;
@@ -213,8 +217,10 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
             twf[(size_t)t * N + i] = h_pair(pw[r], m);
             twi[(size_t)t * N + i] = h_pair(pwi[r], m);
             if (fp) {
-                twdf[(size_t)t * N + i] = (double)pw[r];
-                twdi[(size_t)t * N + i] = (double)pwi[r];
+                // centred representatives: |w| <= q/2 halves the quotient estimate's error and doubles the input range
+                twdf[(size_t)t * N + i] = pw[r] > m / 2 ? -(double)(m - pw[r]) : (double)pw[r];
+                twdi[(size_t)t * N + i] = pwi[r] > m / 2 ? -(double)(m - pwi[r]) : (double)pwi[r];
+                if (i == 1) ninvd[2 * t + 1] = centred_pair(h_mul(pwi[r], ninv[t].x, m));     // the inverse's last twiddle times N^-1
             }
         }
     }

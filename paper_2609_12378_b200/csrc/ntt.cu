@@ -212,8 +212,19 @@ __device__ __forceinline__ void ldg_4(const u64 *p, u64 &a, u64 &b, u64 &c, u64 
     asm volatile("ld.global.v4.b64 {%0,%1,%2,%3}, [%4];" : "=l"(a), "=l"(b), "=l"(c), "=l"(d) : "l"(p) : "memory");
 }
 
-// 4 Cooley-Tukey stages; inputs of any magnitude below 2^53 (reduced first), outputs below 4.6 q.
-template <uint32_t ML>
+// Range bookkeeping of the double-precision path (B = bound in units of q).  The twiddle tables hold centred
+// representatives, |w| <= q/2, and w/q is known to 2^-52 relative, so for |y| <= B q the product y w - k q comes out below
+//   T(B) = (1/2 + B/8) q   when k is rounded to the nearest integer (needs B <= 4:  |y w/q| < 2^51), and below
+//   Tc(B) = (1 + B/8) q    when k is rounded to the nearest even integer (needs |y w/q| < 2^52, sums below 2^53 ~ 8 q).
+// A Cooley-Tukey stage takes B to B + T(B): from a canonical input (B = 1) four stages reach 1.63, 2.33, 3.12, 4.01;
+// from a reduced one (B = 1/2) 1.06, 1.70, 2.41, 3.21.  The sixteen stages of a transform therefore need the
+// three-instruction reduction only twice on the way (after stage 6 and before stage 13) and once at the end:
+//   column pass  canonical 1 | 1.63 2.33 3.12 4.01 | exchange | 5.51c 7.20c | reduce | 1.06 1.70 | stored as doubles
+//   row pass     1.70 | 2.41 3.21 4.11 5.63c | exchange | reduce | 1.06 1.70 2.41 3.21 | exact reduction, canonical word
+// (c = even rounding).  A Gentleman-Sande stage doubles the bound (x1 = u + v) and multiplies u - v, |u - v| <= 2 B:
+// from a reduced input four stages reach 1, 2, 4, 8 (the last product with even rounding, 8 q < 2^53), so the inverse
+// reduces once per group of four stages.
+template <uint32_t ML, int COARSE>
 __device__ __forceinline__ void fwd_stage_d(double (&x)[16], const double *__restrict__ tw, uint32_t base, double q, double qinv) {
     constexpr uint32_t tl = 8 / ML;
     double2 w[ML];
@@ -223,23 +234,42 @@ __device__ __forceinline__ void fwd_stage_d(double (&x)[16], const double *__res
 #pragma unroll
         for (uint32_t j = 0; j < tl; j++) {
             const uint32_t k1 = 2 * i * tl + j, k2 = k1 + tl;
-            // bounds entering the stages: 0.5, 1.13, 1.9, 2.9 (times q): only the last needs the coarse rounding
-            const double t = ML == 8 ? mulmod_d<1>(x[k2], w[i], q) : mulmod_d<0>(x[k2], w[i], q);
+            const double t = mulmod_d<COARSE>(x[k2], w[i], q);
             x[k2] = __dsub_rn(x[k1], t);
             x[k1] = __dadd_rn(x[k1], t);
         }
 }
-__device__ __forceinline__ void fwd16_d(double (&x)[16], const double *__restrict__ tw, uint32_t base, double q, double qinv) {
+__device__ __forceinline__ void reduce16(double (&x)[16], double q, double qinv) {
 #pragma unroll
     for (uint32_t k = 0; k < 16; k++) x[k] = reduce_d(x[k], q, qinv);
-    fwd_stage_d<1>(x, tw, base, q, qinv);
-    fwd_stage_d<2>(x, tw, base, q, qinv);
-    fwd_stage_d<4>(x, tw, base, q, qinv);
-    fwd_stage_d<8>(x, tw, base, q, qinv);
+}
+// stages 1-4 (canonical or reduced input, bound 4.01 q out) and 9-12 (1.70 q in, 5.63 q out): no reduction
+template <int LAST_COARSE>
+__device__ __forceinline__ void fwd16_open(double (&x)[16], const double *__restrict__ tw, uint32_t base, double q, double qinv) {
+    fwd_stage_d<1, 0>(x, tw, base, q, qinv);
+    fwd_stage_d<2, 0>(x, tw, base, q, qinv);
+    fwd_stage_d<4, 0>(x, tw, base, q, qinv);
+    fwd_stage_d<8, LAST_COARSE>(x, tw, base, q, qinv);
+}
+// stages 5-8: two stages with even rounding (4.01 q in, 7.20 q), the reduction, two more (1.70 q out)
+__device__ __forceinline__ void fwd16_mid(double (&x)[16], const double *__restrict__ tw, uint32_t base, double q, double qinv) {
+    fwd_stage_d<1, 1>(x, tw, base, q, qinv);
+    fwd_stage_d<2, 1>(x, tw, base, q, qinv);
+    reduce16(x, q, qinv);
+    fwd_stage_d<4, 0>(x, tw, base, q, qinv);
+    fwd_stage_d<8, 0>(x, tw, base, q, qinv);
+}
+// stages 13-16, and the groups of the register-resident probe: reduction first, outputs below 3.21 q
+__device__ __forceinline__ void fwd16_d(double (&x)[16], const double *__restrict__ tw, uint32_t base, double q, double qinv) {
+    reduce16(x, q, qinv);
+    fwd_stage_d<1, 0>(x, tw, base, q, qinv);
+    fwd_stage_d<2, 0>(x, tw, base, q, qinv);
+    fwd_stage_d<4, 0>(x, tw, base, q, qinv);
+    fwd_stage_d<8, 0>(x, tw, base, q, qinv);
 }
 
-// 4 Gentleman-Sande stages; reduced at the start and after two stages; outputs below 2 q.
-template <uint32_t ML>
+// 4 Gentleman-Sande stages after one reduction; outputs below 8 q (the last stage's products with even rounding).
+template <uint32_t ML, int COARSE>
 __device__ __forceinline__ void inv_stage_d(double (&x)[16], const double *__restrict__ tw, uint32_t base, double q, double qinv) {
     constexpr uint32_t tl = 8 / ML;
     double2 w[ML];
@@ -251,18 +281,32 @@ __device__ __forceinline__ void inv_stage_d(double (&x)[16], const double *__res
             const uint32_t k1 = 2 * i * tl + j, k2 = k1 + tl;
             const double u = x[k1], v = x[k2];
             x[k1] = __dadd_rn(u, v);
-            x[k2] = mulmod_d<0>(__dsub_rn(u, v), w[i], q);     // |u - v| <= 2q < 2^51
+            x[k2] = mulmod_d<COARSE>(__dsub_rn(u, v), w[i], q);
         }
 }
 __device__ __forceinline__ void inv16_d(double (&x)[16], const double *__restrict__ tw, uint32_t base, double q, double qinv) {
+    reduce16(x, q, qinv);
+    inv_stage_d<8, 0>(x, tw, base, q, qinv);     // |u - v| <= 1 q
+    inv_stage_d<4, 0>(x, tw, base, q, qinv);     // 2 q
+    inv_stage_d<2, 0>(x, tw, base, q, qinv);     // 4 q
+    inv_stage_d<1, 1>(x, tw, base, q, qinv);     // 8 q: even rounding; sums reach 8 q < 2^53
+}
+// The last group of the inverse transform (stages m = 8, 4, 2, 1 of the column pass, twiddle base 1): three stages, a
+// second reduction, and the last stage with N^-1 folded in: x1 = (u + v) N^-1, x2 = (u - v) (w N^-1), both products of
+// values below 1 q, so the results are within 0.63 q and one conditional addition makes them canonical.
+// nw = {N^-1, N^-1/q}, wn = {w_1 N^-1, that / q}, centred.
+__device__ __forceinline__ void inv16_last(double (&x)[16], const double *__restrict__ tw, double q, double qinv, double2 nw, double2 wn) {
+    reduce16(x, q, qinv);
+    inv_stage_d<8, 0>(x, tw, 1, q, qinv);
+    inv_stage_d<4, 0>(x, tw, 1, q, qinv);
+    inv_stage_d<2, 0>(x, tw, 1, q, qinv);
+    reduce16(x, q, qinv);
 #pragma unroll
-    for (uint32_t k = 0; k < 16; k++) x[k] = reduce_d(x[k], q, qinv);
-    inv_stage_d<8>(x, tw, base, q, qinv);
-    inv_stage_d<4>(x, tw, base, q, qinv);
-#pragma unroll
-    for (uint32_t k = 0; k < 16; k++) x[k] = reduce_d(x[k], q, qinv);
-    inv_stage_d<2>(x, tw, base, q, qinv);
-    inv_stage_d<1>(x, tw, base, q, qinv);
+    for (uint32_t j = 0; j < 8; j++) {
+        const double u = x[j], v = x[j + 8];
+        x[j] = mulmod_d<0>(__dadd_rn(u, v), nw, q);
+        x[j + 8] = mulmod_d<0>(__dsub_rn(u, v), wn, q);
+    }
 }
 
 // ---- measurement aid: the forward butterflies of the N = 2^16 kernels on registers only ------------------
@@ -311,13 +355,13 @@ __global__ void __launch_bounds__(F_THREADS, 3) ntt16_fwd_cols(DevTables c, u64 
 #pragma unroll
             for (uint32_t k = 0; k < 16; k++) x[k] = u64_to_d(g[(size_t)(r + 16 * k) * 256]);
         }
-        fwd16_d(x, tw, 1, q, qinv);
+        fwd16_open<0>(x, tw, 1, q, qinv);                 // canonical input: no reduction before stage 1
 #pragma unroll
         for (uint32_t k = 0; k < 16; k++) smd[(r + 16 * k) * 16 + cc] = x[k];
         __syncthreads();
 #pragma unroll
         for (uint32_t k = 0; k < 16; k++) x[k] = smd[(16 * r + k) * 16 + cc];
-        fwd16_d(x, tw, 16 + r, q, qinv);
+        fwd16_mid(x, tw, 16 + r, q, qinv);
 #pragma unroll
         for (uint32_t k = 0; k < 16; k++) reinterpret_cast<double *>(g)[(size_t)(16 * r + k) * 256] = x[k];
         return;
@@ -361,7 +405,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) ntt16_fwd_rows(DevTables c, u64 
         double x[16];
 #pragma unroll
         for (uint32_t k = 0; k < 16; k++) x[k] = reinterpret_cast<const double *>(g)[t + 16 * k];
-        fwd16_d(x, tw, 256 + row, q, qinv);
+        fwd16_open<1>(x, tw, 256 + row, q, qinv);     // 1.70 q in, 5.63 q out
 #pragma unroll
         for (uint32_t k = 0; k < 16; k++) s[padded(t + 16 * k)] = x[k];
         __syncwarp();
@@ -519,10 +563,9 @@ __global__ void __launch_bounds__(F_THREADS, 3) ntt16_inv_cols(DevTables c, u64 
         __syncthreads();
 #pragma unroll
         for (uint32_t k = 0; k < 16; k++) x[k] = smd[(r + 16 * k) * 16 + cc];
-        inv16_d(x, tw, 1, q, qinv);
-        const double2 ni = c.n_inv_d[prime];
+        inv16_last(x, tw, q, qinv, c.n_inv_d[2 * prime], c.n_inv_d[2 * prime + 1]);
 #pragma unroll
-        for (uint32_t k = 0; k < 16; k++) g[(size_t)(r + 16 * k) * 256] = canonical_d(mulmod_d<0>(x[k], ni, q), q);   // |x| <= 2q < 2^51
+        for (uint32_t k = 0; k < 16; k++) g[(size_t)(r + 16 * k) * 256] = canonical_d(x[k], q);
         return;
     }
     if (ALLFP) return;
