@@ -67,6 +67,7 @@ struct ckks_ctx {
     std::string cuda_error;
     // options (ckks_context_set_option); host-side state read when a call is made
     uint32_t ntt_fp_share = 8;               // of every 8 limbs, how many take the double-precision NTT path
+    int ntt_bulk_store = 1;                  // forward row pass (N = 2^16): results leave as 128-byte bulk copies from shared memory
     int conv_kernel = 0;                     // basis conversions: 0 = FP64 pipe, 1 = tensor cores (conv_mma.cu)
     int mac_kernel = 82;                     // projection multiply-accumulate kernel (see launch_mac_mma)
     long long wait_cycles = 2000000000ll;    // clock bound of every device-side wait (about a second)

@@ -131,6 +131,10 @@ extern "C" int32_t ckks_context_set_option(ckks_ctx *ctx, int32_t option, int64_
                 return CKKS_ERR_ARG;
             ctx->mac_kernel = (int)value;
             return CKKS_OK;
+        case CKKS_OPT_NTT_BULK_STORE:
+            if (value != 0 && value != 1) return CKKS_ERR_ARG;
+            ctx->ntt_bulk_store = (int)value;
+            return CKKS_OK;
         case CKKS_OPT_WAIT_CYCLES:
             if (value < 0) return CKKS_ERR_ARG;
             ctx->wait_cycles = (long long)value;
@@ -146,6 +150,7 @@ extern "C" int64_t ckks_context_get_option(const ckks_ctx *ctx, int32_t option) 
         case CKKS_OPT_CONV_KERNEL: return ctx->conv_kernel;
         case CKKS_OPT_MAC_KERNEL: return ctx->mac_kernel;
         case CKKS_OPT_WAIT_CYCLES: return ctx->wait_cycles;
+        case CKKS_OPT_NTT_BULK_STORE: return ctx->ntt_bulk_store;
         case CKKS_OPT_STATIC_SCRATCH_BYTES: return (int64_t)CKKS_STATIC_SCRATCH_BYTES;
         default: return -1;
     }

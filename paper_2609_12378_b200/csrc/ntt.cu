@@ -385,15 +385,27 @@ __global__ void __launch_bounds__(F_THREADS, 3) ntt16_fwd_cols(DevTables c, u64 
     for (uint32_t k = 0; k < 16; k++) g[(size_t)(16 * r + k) * 256] = x[k];
 }
 
-// padded index inside a 256-coefficient row: one spare word per 16 so that both access patterns are conflict free
-__device__ __forceinline__ uint32_t padded(uint32_t i) { return i + (i >> 4); }
-constexpr uint32_t ROW_PAD = 256 + 16;
+// padded index inside a 256-coefficient row: two spare words per 16, so that a thread's 16 consecutive coefficients
+// form a 16-byte aligned block of 128 bytes at a pitch of 144 (strided 8-byte accesses by consecutive lanes and
+// 16-byte accesses to the own block are both conflict free, and the block can be the source of a bulk copy)
+__device__ __forceinline__ uint32_t padded(uint32_t i) { return i + 2 * (i >> 4); }
+constexpr uint32_t ROW_PAD = 256 + 32;
+// Results leave the row pass as one 128-byte bulk copy per thread (shared -> global, no multicast, this GPU's memory):
+// a thread writes its 16 canonical words into its own block of the exchange row with 16-byte stores and hands the
+// block to the copy engine, which takes the stores off the load/store pipe (four 32-byte global stores per thread cost
+// it one pass per lane and sector: the row pass's busiest unit).
+__device__ __forceinline__ void bulk_store_128(u64 *gdst, const void *ssrc) {
+    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], 128;\n" ::"l"(gdst), "r"((uint32_t)__cvta_generic_to_shared(ssrc)) : "memory");
+    asm volatile("cp.async.bulk.commit_group;\n" ::: "memory");
+}
+__device__ __forceinline__ void bulk_store_wait() { asm volatile("cp.async.bulk.wait_group.read 0;\n" ::: "memory"); }
 
 // ---- forward, row pass (stages m = 256..32768): CTA = 16 rows, 16 threads per row ---------
-template <bool ALLFP, int EP>
+template <bool ALLFP, int EP, bool BULK = false>
 __global__ void __launch_bounds__(F_THREADS, 3) ntt16_fwd_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, NttEpilogue ep) {
     constexpr int has_ep = EP;
-    __shared__ u64 sm[16 * ROW_PAD];
+    __shared__ __align__(16) u64 sm[16 * ROW_PAD];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
     if (ALLFP || (blockIdx.y & 7) < fp_share) {
@@ -409,16 +421,36 @@ __global__ void __launch_bounds__(F_THREADS, 3) ntt16_fwd_rows(DevTables c, u64 
 #pragma unroll
         for (uint32_t k = 0; k < 16; k++) s[padded(t + 16 * k)] = x[k];
         __syncwarp();
+        double *blk = s + 18 * t;                 // this thread's 16 consecutive coefficients: 16-byte aligned, 144-byte pitch
 #pragma unroll
-        for (uint32_t k = 0; k < 16; k++) x[k] = s[padded(16 * t + k)];
+        for (uint32_t k = 0; k < 16; k += 2) {
+            const double2 v = *reinterpret_cast<const double2 *>(blk + k);
+            x[k] = v.x; x[k + 1] = v.y;
+        }
         fwd16_d(x, tw, 16 * (256 + row) + t, q, qinv);
+        // four finished words: to the own block (BULK) or straight to global memory
+        auto put4 = [&](u64 *dst, uint32_t k, u64 a, u64 b, u64 cc, u64 d) {
+            if (BULK) {
+                *reinterpret_cast<ulonglong2 *>(blk + k) = make_ulonglong2(a, b);
+                *reinterpret_cast<ulonglong2 *>(blk + k + 2) = make_ulonglong2(cc, d);
+            } else {
+                stg_4(dst + k, a, b, cc, d);
+            }
+        };
+        auto finish = [&](u64 *dst) {
+            if (BULK) {
+                bulk_store_128(dst, blk);
+                bulk_store_wait();
+            }
+        };
         if (has_ep == 2) {     // the result itself, but into a tiled buffer
             const uint32_t y = blockIdx.y, i = y % ep.level, b = y / ep.level;
             u64 *dst = ep.out + tiled_index(ep.tl.R, 65536, ep.tl.row0 + b * ep.tl.row_stride, i, row * 256 + 16 * t);
 #pragma unroll
             for (uint32_t k = 0; k < 16; k += 4)
-                stg_4(dst + k, canonical_d(reduce_d(x[k], q, qinv), q), canonical_d(reduce_d(x[k + 1], q, qinv), q),
-                      canonical_d(reduce_d(x[k + 2], q, qinv), q), canonical_d(reduce_d(x[k + 3], q, qinv), q));
+                put4(dst, k, canonical_d(reduce_d(x[k], q, qinv), q), canonical_d(reduce_d(x[k + 1], q, qinv), q),
+                     canonical_d(reduce_d(x[k + 2], q, qinv), q), canonical_d(reduce_d(x[k + 3], q, qinv), q));
+            finish(dst);
             return;
         }
         if (has_ep) {      // ModDown tail: (u - NTT(conv)) P^-1 + sigma_g(add), written to its final place
@@ -447,15 +479,17 @@ __global__ void __launch_bounds__(F_THREADS, 3) ntt16_fwd_rows(DevTables c, u64 
                     if (ep.accumulate) v = __dadd_rn(v, u64_to_d(old[e]));
                     r[e] = canonical_d(reduce_d(v, q, qinv), q);
                 }
-                stg_4(dst + k, r[0], r[1], r[2], r[3]);
+                put4(dst, k, r[0], r[1], r[2], r[3]);
             }
+            finish(dst);
             return;
         }
-        // a thread ends up with 16 consecutive coefficients: four 32-byte stores, each a full sector
+        // a thread ends up with 16 consecutive coefficients
 #pragma unroll
         for (uint32_t k = 0; k < 16; k += 4)
-            stg_4(g + 16 * t + k, canonical_d(reduce_d(x[k], q, qinv), q), canonical_d(reduce_d(x[k + 1], q, qinv), q),
-                  canonical_d(reduce_d(x[k + 2], q, qinv), q), canonical_d(reduce_d(x[k + 3], q, qinv), q));
+            put4(g + 16 * t, k, canonical_d(reduce_d(x[k], q, qinv), q), canonical_d(reduce_d(x[k + 1], q, qinv), q),
+                 canonical_d(reduce_d(x[k + 2], q, qinv), q), canonical_d(reduce_d(x[k + 3], q, qinv), q));
+        finish(g + 16 * t);
         return;
     }
     if (ALLFP) return;
@@ -487,7 +521,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) ntt16_fwd_rows(DevTables c, u64 
 template <bool ALLFP>
 __global__ void __launch_bounds__(F_THREADS, 3) ntt16_inv_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, const u64 *src,
                                                                 uint32_t src_pitch) {
-    __shared__ u64 sm[16 * ROW_PAD];
+    __shared__ __align__(16) u64 sm[16 * ROW_PAD];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
     if (ALLFP || (blockIdx.y & 7) < fp_share) {
@@ -507,7 +541,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) ntt16_inv_rows(DevTables c, u64 
         }
         inv16_d(x, tw, 16 * (256 + row) + t, q, qinv);
 #pragma unroll
-        for (uint32_t k = 0; k < 16; k++) s[padded(16 * t + k)] = x[k];
+        for (uint32_t k = 0; k < 16; k += 2) *reinterpret_cast<double2 *>(s + 18 * t + k) = make_double2(x[k], x[k + 1]);     // own block, 16-byte stores
         __syncwarp();
 #pragma unroll
         for (uint32_t k = 0; k < 16; k++) x[k] = s[padded(t + 16 * k)];
@@ -605,9 +639,16 @@ void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbM
                 if (share >= 8) ntt16_fwd_cols<true><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, coef_src);
                 else ntt16_fwd_cols<false><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, coef_src);
                 count_launches();
+                // bulk-copy stores need 16-byte aligned destinations (every block is then 128-byte aligned relative to them)
+                bool bulk = c->ntt_bulk_store && ((uintptr_t)(ep ? (const void *)ep->out : (const void *)b) & 15) == 0;
+                if (ep && ep->multi)
+                    for (uint32_t k = 0; k < KS_MULTI; k++) bulk = bulk && ((uintptr_t)ep->mout[k] & 15) == 0;
                 if (share < 8) ntt16_fwd_rows<false, 0><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, NttEpilogue{});
+                else if (!ep && bulk) ntt16_fwd_rows<true, 0, true><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, NttEpilogue{});
                 else if (!ep) ntt16_fwd_rows<true, 0><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, NttEpilogue{});
+                else if (ep->mode == 1 && bulk) ntt16_fwd_rows<true, 1, true><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, *ep);
                 else if (ep->mode == 1) ntt16_fwd_rows<true, 1><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, *ep);
+                else if (bulk) ntt16_fwd_rows<true, 2, true><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, *ep);
                 else ntt16_fwd_rows<true, 2><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, share, *ep);
                 count_launches();
             } else {
