@@ -30,6 +30,10 @@ struct DevTables {
     // indexing (w/q is formed in the kernel as w * (1/q): half the table bytes for one extra multiply per twiddle)
     const double *twd_fwd, *twd_inv;    // [T][N]
     const double2 *n_inv_d;             // [T][2] {N^-1, N^-1/q}, {w N^-1, that/q} for the inverse's last twiddle w, all centred
+    // inverse-transform scalings that deliver the basis conversions' first factor y = [d qhat^-1] (N = 2^16 only), pairs
+    // {N^-1 qhat^-1, last inverse twiddle times that}, each {v, v / prime} centred
+    const double2 *inv_scale_up;   // [(L+1)][L][2]   ModUp: level, limb
+    const double2 *inv_scale_dn;   // [K][2]          ModDown: special limb
     // ModUp, per level l (1..L), digit j, source a < alpha:
     const ulonglong2 *up_hat_inv;  // [(L+1)][dnum][alpha]        {qhat^-1 mod q_src, Shoup}
     const u64 *up_hat_mod;         // [(L+1)][dnum][alpha][T]     qhat mod target
@@ -241,9 +245,11 @@ struct NttEpilogue {
 // index / map.period) and reduces them modulo the limb's prime on the fly instead of reading `base`.
 // inv_src (inverse, N = 2^16 path only): the first pass reads its limbs from another buffer whose periods start
 // inv_src_pitch limbs apart, so the transform runs out of place and the input stays intact.
+// inv_scale (inverse, N = 2^16 path only): pairs [map.period][2] that replace {N^-1, last twiddle N^-1} for limb x of every
+// period (device pointer), so that the output is scaled by a per-limb constant.
 void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbMap &map, bool inverse, cudaStream_t s,
                 const NttEpilogue *ep = nullptr, const long long *coef_src = nullptr, const u64 *inv_src = nullptr,
-                uint32_t inv_src_pitch = 0);
+                uint32_t inv_src_pitch = 0, const double2 *inv_scale = nullptr);
 
 void launch_mul_plain_acc(const ckks_ctx *c, const u64 *const *cts, u64 *const *accs, uint32_t ncts, const u64 *pt,
                           uint32_t level, bool init, cudaStream_t s);

@@ -281,6 +281,33 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
         dn_pmod_d[i] = (double)Pm;
     }
 
+    // ---- The inverse transform can deliver the conversions' first factor directly: its last stage multiplies by
+    // N^-1 anyway, so with N^-1 qhat^-1 (and the last twiddle times that) in its place the coefficient-domain output is
+    // y = [d qhat^-1] instead of d.  Pairs {constant, constant / prime}, centred; index [level][limb][2] and [k][2].
+    std::vector<double2> isc_up(fp ? (size_t)(L + 1) * L * 2 : 0), isc_dn(fp ? (size_t)K * 2 : 0);
+    if (fp) {
+        auto centred_pair_mod = [&](u64 v, u64 m) {
+            const double dd = v > m / 2 ? -(double)(m - v) : (double)v;
+            return make_double2(dd, dd * (1.0 / (double)m));
+        };
+        auto last_tw = [&](uint32_t t) {     // the inverse transform's last twiddle (index 1 of the inverse table)
+            return twi[(size_t)t * N + 1].x;
+        };
+        for (uint32_t l = 1; l <= L; l++)
+            for (uint32_t x = 0; x < l; x++) {
+                const uint32_t j = x / alpha, a = x % alpha;
+                const u64 m = mod[x], h = up_inv[((size_t)l * dn + j) * alpha + a].x;
+                const u64 nh = h_mul(ninv[x].x, h, m);
+                isc_up[((size_t)l * L + x) * 2] = centred_pair_mod(nh, m);
+                isc_up[((size_t)l * L + x) * 2 + 1] = centred_pair_mod(h_mul(last_tw(x), nh, m), m);
+            }
+        for (uint32_t a = 0; a < K; a++) {
+            const u64 m = mod[L + a], nh = h_mul(ninv[L + a].x, dn_inv[a].x, m);
+            isc_dn[(size_t)a * 2] = centred_pair_mod(nh, m);
+            isc_dn[(size_t)a * 2 + 1] = centred_pair_mod(h_mul(last_tw(L + a), nh, m), m);
+        }
+    }
+
     // ---- Byte matrices for the tensor-core basis conversion.  Row k = 8 a + b of the k-dimension is byte b of source
     // a's centred-lift word (b = 7: the "negative" flag); column (x, d) collects the byte products of weight 2^(8 d):
     // byte d - b of the constant C[a][x] for b < 7, and byte d of (-q_a C[a][x]) mod t for the flag, so that the
@@ -357,7 +384,7 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
     std::vector<int> flag(2, 0);
     const int *flag_dev = nullptr;
     if ((rc = upload(c, mod, &d.mod)) || (rc = upload(c, mu, &d.mu)) || (rc = upload(c, mu64, &d.mu64)) || (rc = upload(c, modd, &d.modd)) || (rc = upload(c, twf, &d.tw_fwd)) ||
-        (rc = upload(c, twi, &d.tw_inv)) || (rc = upload(c, twdf, &d.twd_fwd)) || (rc = upload(c, twdi, &d.twd_inv)) || (rc = upload(c, ninvd, &d.n_inv_d)) || (rc = upload(c, ninv, &d.n_inv)) || (rc = upload(c, up_inv, &d.up_hat_inv)) ||
+        (rc = upload(c, twi, &d.tw_inv)) || (rc = upload(c, twdf, &d.twd_fwd)) || (rc = upload(c, twdi, &d.twd_inv)) || (rc = upload(c, ninvd, &d.n_inv_d)) || (rc = upload(c, isc_up, &d.inv_scale_up)) || (rc = upload(c, isc_dn, &d.inv_scale_dn)) || (rc = upload(c, ninv, &d.n_inv)) || (rc = upload(c, up_inv, &d.up_hat_inv)) ||
         (rc = upload(c, up_mod, &d.up_hat_mod)) || (rc = upload(c, up_mod_d, &d.up_hat_mod_d)) || (rc = upload(c, dn_mod_d, &d.dn_hat_mod_d)) || (rc = upload(c, dn_inv, &d.dn_hat_inv)) ||
         (rc = upload(c, dn_mod, &d.dn_hat_mod)) || (rc = upload(c, dn_pinv, &d.dn_p_inv)) || (rc = upload(c, dn_pinv_d, &d.dn_p_inv_d)) || (rc = upload(c, dn_pmod_d, &d.dn_p_mod_d)) || (rc = upload(c, up_bmat, &d.up_bmat)) || (rc = upload(c, dn_bmat, &d.dn_bmat)) || (rc = upload(c, two52, &d.two52_d)) || (rc = upload(c, rs, &d.rs_inv)) ||
         (rc = upload(c, enc_src, &d.enc_src)) || (rc = upload(c, om, &d.enc_omega)) || (rc = upload(c, ze, &d.enc_zeta)) ||

@@ -33,7 +33,8 @@ inline uint32_t conv_chunk(uint32_t nb) { return nb >= 4 ? 32 : 8; }
 // walks a chunk of CHUNK target limbs (blockIdx.y), so the source limbs are read once per chunk.
 constexpr uint32_t CONV_CHUNK_MAX = 32;
 
-template <uint32_t ALPHA>
+// PRE: dcoef already holds [d_a qhat_a^-1] (the inverse transform multiplied it in), so only the centring is left.
+template <uint32_t ALPHA, bool PRE>
 __global__ void __launch_bounds__(THREADS) modup_kernel(DevTables c, const u64 *dcoef, const u64 *deval, size_t deval_stride, u64 g,
                                                         u64 *ext, uint32_t level, uint32_t CHUNK) {
     // the CTA's conversion constants (qhat_a mod t and its quotient by t; t and 1/t), fetched once: as global loads
@@ -60,8 +61,11 @@ __global__ void __launch_bounds__(THREADS) modup_kernel(DevTables c, const u64 *
         y[a] = 0.0;
         if (a < nd) {
             const u64 qa = c.mod[lo + a];
-            const ulonglong2 hinv = c.up_hat_inv[cb + a];
-            const u64 v = mul_shoup(dcoef[(size_t)(lo + a) * c.N + k], hinv.x, hinv.y, qa);
+            u64 v = dcoef[(size_t)(lo + a) * c.N + k];
+            if (!PRE) {
+                const ulonglong2 hinv = c.up_hat_inv[cb + a];
+                v = mul_shoup(v, hinv.x, hinv.y, qa);
+            }
             y[a] = v > (qa >> 1) ? __dsub_rn(u64_to_d(v), (double)qa) : u64_to_d(v);
         }
     }
@@ -88,10 +92,12 @@ __global__ void __launch_bounds__(THREADS) modup_kernel(DevTables c, const u64 *
 
 template <uint32_t ALPHA>
 void launch_modup(const ckks_ctx *c, const u64 *dcoef, const u64 *deval, size_t deval_stride, u64 g, u64 *ext, uint32_t level,
-                  uint32_t nb, cudaStream_t s) {
+                  uint32_t nb, cudaStream_t s, bool pre) {
     const uint32_t nt = level + c->K, beta = (level + c->alpha - 1) / c->alpha;
     const uint32_t CHUNK = conv_chunk(nb);
-    modup_kernel<ALPHA><<<dim3(c->N / THREADS, (nt + CHUNK - 1) / CHUNK, beta * nb), THREADS, 0, s>>>(c->dev, dcoef, deval, deval_stride, g, ext, level, CHUNK);
+    const dim3 grid(c->N / THREADS, (nt + CHUNK - 1) / CHUNK, beta * nb);
+    if (pre) modup_kernel<ALPHA, true><<<grid, THREADS, 0, s>>>(c->dev, dcoef, deval, deval_stride, g, ext, level, CHUNK);
+    else modup_kernel<ALPHA, false><<<grid, THREADS, 0, s>>>(c->dev, dcoef, deval, deval_stride, g, ext, level, CHUNK);
     count_launches();
 }
 
@@ -273,7 +279,7 @@ __global__ void __launch_bounds__(THREADS, 3) inner_product_terms_kernel(DevTabl
 
 // conv[comp][i][k] = sum_a centre([u_{p_a} Phat_a^-1]) (Phat_a mod q_i)  mod q_i   (coefficient domain)
 // Same shape as ModUp: the K centred special residues are formed once per thread, then a chunk of targets is walked.
-template <uint32_t KK>
+template <uint32_t KK, bool PRE>
 __global__ void __launch_bounds__(THREADS, 6) moddown_conv_kernel(DevTables c, const u64 *u, u64 *conv, uint32_t level, uint32_t CHUNK) {
     __shared__ double2 s_w[CONV_CHUNK_MAX][KK];     // Phat_a mod q_i and its quotient by q_i
     __shared__ double2 s_m[CONV_CHUNK_MAX];         // q_i, 1 / q_i
@@ -294,8 +300,11 @@ __global__ void __launch_bounds__(THREADS, 6) moddown_conv_kernel(DevTables c, c
         y[a] = 0.0;
         if (a < c.K) {
             const u64 pa = c.mod[c.L + a];
-            const ulonglong2 hinv = c.dn_hat_inv[a];
-            const u64 v = mul_shoup(u[((size_t)comp * nt + level + a) * c.N + k], hinv.x, hinv.y, pa);
+            u64 v = u[((size_t)comp * nt + level + a) * c.N + k];
+            if (!PRE) {
+                const ulonglong2 hinv = c.dn_hat_inv[a];
+                v = mul_shoup(v, hinv.x, hinv.y, pa);
+            }
             y[a] = v > (pa >> 1) ? __dsub_rn(u64_to_d(v), (double)pa) : u64_to_d(v);
         }
     }
@@ -315,9 +324,11 @@ __global__ void __launch_bounds__(THREADS, 6) moddown_conv_kernel(DevTables c, c
 }
 
 template <uint32_t KK>
-void launch_moddown_conv(const ckks_ctx *c, const u64 *u, u64 *conv, uint32_t level, uint32_t nb, cudaStream_t s) {
+void launch_moddown_conv(const ckks_ctx *c, const u64 *u, u64 *conv, uint32_t level, uint32_t nb, cudaStream_t s, bool pre) {
     const uint32_t CHUNK = conv_chunk(nb);
-    moddown_conv_kernel<KK><<<dim3(c->N / THREADS, (level + CHUNK - 1) / CHUNK, 2 * nb), THREADS, 0, s>>>(c->dev, u, conv, level, CHUNK);
+    const dim3 grid(c->N / THREADS, (level + CHUNK - 1) / CHUNK, 2 * nb);
+    if (pre) moddown_conv_kernel<KK, true><<<grid, THREADS, 0, s>>>(c->dev, u, conv, level, CHUNK);
+    else moddown_conv_kernel<KK, false><<<grid, THREADS, 0, s>>>(c->dev, u, conv, level, CHUNK);
     count_launches();
 }
 
@@ -407,15 +418,18 @@ KsWorkspace ks_carve(const ckks_ctx *c, uint32_t level, void *ws, uint32_t nb) {
 
 void ks_modup(const ckks_ctx *c, const u64 *d, uint32_t level, const KsWorkspace &w, cudaStream_t s, uint32_t nb, size_t d_stride) {
     const uint32_t N = c->N, beta = (level + c->alpha - 1) / c->alpha, nt = level + c->K;
+    // N = 2^16 with the FP64 transform and conversion: the inverse transform's last stage multiplies qhat^-1 in
+    const bool pre = c->log_n == 16 && c->ntt_fp_share >= 8 && c->conv_kernel != CKKS_CONV_TENSOR;
     if (c->log_n == 16) {      // the inverse transform reads d and writes the coefficient copy
-        launch_ntt(c, w.dcoef, nb * level, plain_map(0, level), true, s, nullptr, nullptr, d, (uint32_t)(d_stride / N));
+        launch_ntt(c, w.dcoef, nb * level, plain_map(0, level), true, s, nullptr, nullptr, d, (uint32_t)(d_stride / N),
+                   pre ? c->dev.inv_scale_up + (size_t)level * c->L * 2 : nullptr);
     } else {
         permute_kernel<<<dim3(N / THREADS, level, nb), THREADS, 0, s>>>(c->dev, d, d_stride, w.dcoef, (size_t)level * N, 1); count_launches();
         launch_ntt(c, w.dcoef, nb * level, plain_map(0, level), true, s);
     }
     // the context option CKKS_CONV_TENSOR takes the tensor-core conversion of conv_mma.cu: bit-identical, 2 % slower on B200
     if (c->conv_kernel != CKKS_CONV_TENSOR || !launch_modup_mma(c, w.dcoef, d, d_stride, w.ext, level, nb, s)) {
-#define CALL_UP(A) launch_modup<A>(c, w.dcoef, d, d_stride, 1, w.ext, level, nb, s)
+#define CALL_UP(A) launch_modup<A>(c, w.dcoef, d, d_stride, 1, w.ext, level, nb, s, pre)
         DISPATCH_POW2(c->alpha, CALL_UP);
 #undef CALL_UP
     }
@@ -461,10 +475,13 @@ void ks_inner(const ckks_ctx *c, const u64 *evk, uint32_t level, u64 ext_galois,
 void ks_moddown(const ckks_ctx *c, uint32_t level, const KsWorkspace &w, const u64 *add0, const u64 *add1, u64 add_galois, u64 *out,
                 cudaStream_t s, uint32_t nb, size_t add_stride, size_t out_stride, bool accumulate, TiledOut tiled, const KsMulti *multi) {
     const uint32_t N = c->N, nt = level + c->K, K = c->K;
-    // the K special limbs of every (batch, component): groups of K limbs, nt limbs apart
-    launch_ntt(c, w.u + (size_t)level * N, nb * 2 * K, pitched_map(c->L, K, nt), true, s);
+    // the K special limbs of every (batch, component): groups of K limbs, nt limbs apart; at N = 2^16 the inverse
+    // transform's last stage multiplies Phat^-1 in
+    const bool pre = c->log_n == 16 && c->ntt_fp_share >= 8 && c->conv_kernel != CKKS_CONV_TENSOR;
+    launch_ntt(c, w.u + (size_t)level * N, nb * 2 * K, pitched_map(c->L, K, nt), true, s, nullptr, nullptr, nullptr, 0,
+               pre ? c->dev.inv_scale_dn : nullptr);
     if (c->conv_kernel != CKKS_CONV_TENSOR || !launch_moddown_conv_mma(c, w.u, w.conv, level, nb, s)) {
-#define CALL_DN(A) launch_moddown_conv<A>(c, w.u, w.conv, level, nb, s)
+#define CALL_DN(A) launch_moddown_conv<A>(c, w.u, w.conv, level, nb, s, pre)
         DISPATCH_POW2(K, CALL_DN);
 #undef CALL_DN
     }

@@ -578,7 +578,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) ntt16_inv_rows(DevTables c, u64 
 
 // ---- inverse, column pass (stages m = 128..1), then N^-1 and the exact reduction -----------
 template <bool ALLFP>
-__global__ void __launch_bounds__(F_THREADS, 3) ntt16_inv_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share) {
+__global__ void __launch_bounds__(F_THREADS, 3) ntt16_inv_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, const double2 *scale) {
     __shared__ u64 sm[256 * 16];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
@@ -597,7 +597,8 @@ __global__ void __launch_bounds__(F_THREADS, 3) ntt16_inv_cols(DevTables c, u64 
         __syncthreads();
 #pragma unroll
         for (uint32_t k = 0; k < 16; k++) x[k] = smd[(r + 16 * k) * 16 + cc];
-        inv16_last(x, tw, q, qinv, c.n_inv_d[2 * prime], c.n_inv_d[2 * prime + 1]);
+        const double2 *sc = scale ? scale + 2 * (blockIdx.y % map.period) : c.n_inv_d + 2 * prime;
+        inv16_last(x, tw, q, qinv, sc[0], sc[1]);
 #pragma unroll
         for (uint32_t k = 0; k < 16; k++) g[(size_t)(r + 16 * k) * 256] = canonical_d(x[k], q);
         return;
@@ -625,7 +626,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) ntt16_inv_cols(DevTables c, u64 
 }  // namespace
 
 void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbMap &map, bool inverse, cudaStream_t s,
-                const NttEpilogue *ep, const long long *coef_src, const u64 *inv_src, uint32_t inv_src_pitch) {
+                const NttEpilogue *ep, const long long *coef_src, const u64 *inv_src, uint32_t inv_src_pitch, const double2 *inv_scale) {
     if (nlimbs_total == 0) return;
     if (c->log_n == 16) {
         for (uint32_t y0 = 0; y0 < nlimbs_total;) {
@@ -656,8 +657,8 @@ void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbM
                 if (c->ntt_fp_share >= 8) ntt16_inv_rows<true><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, 8, sb, inv_src_pitch);
                 else ntt16_inv_rows<false><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share, sb, inv_src_pitch);
                 count_launches();
-                if (c->ntt_fp_share >= 8) ntt16_inv_cols<true><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, 8);
-                else ntt16_inv_cols<false><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share);
+                if (c->ntt_fp_share >= 8) ntt16_inv_cols<true><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, 8, inv_scale);
+                else ntt16_inv_cols<false><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share, nullptr);
                 count_launches();
             }
             y0 += ny;
