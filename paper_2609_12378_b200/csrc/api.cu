@@ -79,12 +79,12 @@ int make_plan(const ckks_ctx *c, const ckks_proj_desc *d, ProjPlan &p) {
     return CKKS_OK;
 }
 
-struct ProjWs { size_t baby, xin, pts, ptt, slots, enc, acc, total, tmp, ks, ksx, rs, bytes; uint32_t gg; bool per_block; };
+struct ProjWs { size_t baby, xin, pts, ptt, slots, enc, acc, total, tmp, ks, ksx, rs, bytes; uint32_t gg, gacc; bool per_block, ib_outer; };
 
 constexpr uint32_t BABY_ROTS = 4;            // baby-step rotations per key-switch pass (N = 2^16)
 constexpr uint32_t MAC_GT = 4;               // giants per register tile of the fallback multiply-accumulate kernel
 
-ProjWs proj_layout(const ckks_ctx *c, const ProjPlan &p, uint32_t level, bool lazy) {
+ProjWs proj_layout(const ckks_ctx *c, const ProjPlan &p, uint32_t level, bool lazy, uint32_t nmat = 1) {
     const size_t ct = (size_t)2 * level * c->N * sizeof(u64), pt = (size_t)level * c->N * sizeof(u64);
     const size_t nib = p.ins.size();
     ProjWs w;
@@ -96,21 +96,27 @@ ProjWs proj_layout(const ckks_ctx *c, const ProjPlan &p, uint32_t level, bool la
     if (w.per_block) w.gg = std::max<uint32_t>(1, std::min<uint32_t>(p.gmax, 16));
     else w.gg = std::max<uint32_t>(1, std::min<uint32_t>(p.gmax, 16 / (uint32_t)nib ? 16 / (uint32_t)nib : 1));
     w.gg = (w.gg + MAC_GT - 1) / MAC_GT * MAC_GT;
+    // Several input blocks and one output block (a down-shaped projection): the input blocks are taken in the outer
+    // loop, so that only one block's baby ciphertexts are resident (B per shard instead of nib * B) and the key-switch
+    // buffers serve one block's batch; the accumulators of all giant steps then stay live across the blocks.
+    w.ib_outer = w.per_block && nib > 1 && p.outs.size() == 1 && nmat == 1;
+    w.gacc = w.ib_outer ? (p.gmax + w.gg - 1) / w.gg * w.gg : w.gg;
+    const size_t nbb = w.ib_outer ? 1 : nib;                // input blocks whose baby ciphertexts are resident together
     const size_t npt = (size_t)w.gg * (w.per_block ? 1 : nib) * p.B;
     size_t off = 0;
-    w.baby = off;  off += align256(ct * p.S * nib * p.B);   // tiled: rows (shard * J + j) * 2 + component
+    w.baby = off;  off += align256(ct * p.S * nbb * p.B);   // tiled: rows (shard * J + j) * 2 + component
     w.xin = off;   off += align256(ct * p.S * nib);         // the inputs side by side, plain layout
     w.pts = off;   off += align256(pt * npt);               // encoded plaintexts of a group, plain layout
     w.ptt = off;   off += align256(pt * npt);               // the same, tiled: rows g * J + j
     w.slots = off; off += align256(npt * c->n * sizeof(double));
     w.enc = off;   off += align256(encode_workspace_bytes(c, (uint32_t)npt));
-    w.acc = off;   off += align256(ct * p.S * w.gg);
+    w.acc = off;   off += align256(ct * p.S * w.gacc);
     w.total = off; off += align256(ct * p.S);
     w.tmp = off;   off += align256(ct);
     // all shards' key switches run side by side; the baby steps take BABY_ROTS rotations per pass, which needs that
     // many inner-product and conversion buffers per input ciphertext
     const size_t knt = level + c->K;
-    w.ks = off;    off += align256(ks_bytes(c, level) * p.S * nib + (size_t)(BABY_ROTS - 1) * p.S * nib * (2 * knt + 2 * level) * c->N * sizeof(u64));
+    w.ks = off;    off += align256(ks_bytes(c, level) * p.S * nbb + (size_t)(BABY_ROTS - 1) * p.S * nbb * (2 * knt + 2 * level) * c->N * sizeof(u64));
     // lazy giant steps: coefficient copies and extended digits of IP_TERMS giant steps of every shard
     const size_t kbeta = (level + c->alpha - 1) / c->alpha;
     w.ksx = off;   off += lazy ? align256((size_t)IP_TERMS * p.S * (level + kbeta * (level + c->K)) * c->N * sizeof(u64)) : 0;
@@ -913,7 +919,7 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
     }
     bool any_lazy = false;
     for (uint32_t m = 0; m < nmat; m++) any_lazy = any_lazy || (descs[m].flags & CKKS_PROJ_LAZY_MODDOWN) != 0;
-    const ProjWs L = proj_layout(c, merged, level, any_lazy);
+    const ProjWs L = proj_layout(c, merged, level, any_lazy, nmat);
     if (!ws || ws_bytes < L.bytes) return CKKS_ERR_WORKSPACE;
 
     DeviceGuard g(c->device);
@@ -925,48 +931,54 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
     u64 *total = (u64 *)(base + L.total), *rsw = (u64 *)(base + L.rs);
     double *slots = (double *)(base + L.slots);
     void *encw = base + L.enc;
-    KsWorkspace kw = ks_carve(c, level, base + L.ks, S * nib);
+    // baby row ((sh*nbb + ib)*B + b)*2 + comp = component comp of rho^(b T)(x_{sh,ib}), tiled layout: one ModUp for all
+    // input ciphertexts of the block set at once, then every baby rotation is applied to all of them in one batch (the
+    // key is read once per rotation, not once per shard) and written straight into the tiled buffer.  The block set is
+    // all input blocks, or one block at a time (L.ib_outer): its inputs are then the ciphertexts ib, ib + nib, ..
+    const uint32_t nbb = L.ib_outer ? 1 : nib;
+    const uint32_t Jall = nbb * B, Rx = 2 * S * Jall;
+    for (uint32_t x = 0; x < S * nib; x++)
+        cudaMemcpyAsync(xin + (size_t)x * ctl, in[x].data, ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+    KsWorkspace kw = ks_carve(c, level, base + L.ks, S * nbb);
     // lazy giant steps: digits of IP_TERMS x S accumulators side by side; the running sum and the ModDown use kw's buffers
     const uint32_t kbeta = (level + c->alpha - 1) / c->alpha, knt = level + c->K;
     KsWorkspace kx = kw;
     kx.dcoef = (u64 *)(base + L.ksx);
     kx.ext = kx.dcoef + (size_t)IP_TERMS * S * level * N;
-
-    // baby row ((sh*nib + ib)*B + b)*2 + comp = component comp of rho^(b T)(x_{sh,ib}), tiled layout: one ModUp for all
-    // input ciphertexts at once, then every baby rotation is applied to all of them in one batch (the key is read
-    // once per rotation, not once per shard) and written straight into the tiled buffer
-    const uint32_t Jall = nib * B, Rx = 2 * S * Jall;
-    for (uint32_t x = 0; x < S * nib; x++)
-        cudaMemcpyAsync(xin + (size_t)x * ctl, in[x].data, ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
-    for (uint32_t comp = 0; comp < 2; comp++)
-        launch_to_tiled(c, xin + comp * ptl, ctl, S * nib, baby, Rx, comp, 2 * B, level, s);
-    if (B > 1) {
-        ks_modup(c, xin + ptl, level, kw, s, S * nib, ctl);
+    auto baby_steps = [&](uint32_t ib0) {
+        const u64 *xb = xin + (size_t)ib0 * ctl;                       // first ciphertext of the set
+        const size_t xs = (size_t)(L.ib_outer ? nib : 1) * ctl;       // from one ciphertext of the set to the next
+        const uint32_t nx = S * nbb;
+        for (uint32_t comp = 0; comp < 2; comp++)
+            launch_to_tiled(c, xb + comp * ptl, xs, nx, baby, Rx, comp, 2 * B, level, s);
+        if (B <= 1) return;
+        ks_modup(c, xb + ptl, level, kw, s, nx, xs);
         // N = 2^16: BABY_ROTS rotations of all inputs per pass (the digits of a limb are fetched once for all of them and
         // the launches are four times larger); the inner-product and conversion buffers follow the digits
         const uint32_t rots = c->log_n == 16 ? BABY_ROTS : 1;       // the grouped ModDown tail exists for N = 2^16 only
         KsWorkspace kb = kw;
-        kb.u = kw.ext + (size_t)S * nib * kbeta * knt * N;
-        kb.conv = kb.u + (size_t)rots * S * nib * 2 * knt * N;
+        kb.u = kw.ext + (size_t)nx * kbeta * knt * N;
+        kb.conv = kb.u + (size_t)rots * nx * 2 * knt * N;
         for (uint32_t b = 1; b < B; b += rots) {
             const uint32_t nr = std::min(rots, B - b);
             TiledOut to;
             to.R = Rx; to.row0 = 2 * b; to.row_stride = 2 * B;
             if (rots == 1) {
                 const u64 ge = ckks_galois_element(c, (int64_t)b * T);
-                ks_inner_moddown(c, (const u64 *)find_key(keys, nkeys, ge)->data, level, ge, kw, xin, nullptr, ge, baby, s, S * nib, ctl, 0,
+                ks_inner_moddown(c, (const u64 *)find_key(keys, nkeys, ge)->data, level, ge, kw, xb, nullptr, ge, baby, s, nx, xs, 0,
                                  false, to);
                 continue;
             }
             KsMulti m{};
-            m.group = S * nib; m.rot_rows = 2;
+            m.group = nx; m.rot_rows = 2;
             for (uint32_t r = 0; r < nr; r++) {
                 m.galois[r] = ckks_galois_element(c, (int64_t)(b + r) * T);
                 m.evk[r] = (const u64 *)find_key(keys, nkeys, m.galois[r])->data;
             }
-            ks_inner_moddown(c, nullptr, level, 1, kb, xin, nullptr, 1, baby, s, nr * S * nib, ctl, 0, false, to, &m);
+            ks_inner_moddown(c, nullptr, level, 1, kb, xb, nullptr, 1, baby, s, nr * nx, xs, 0, false, to, &m);
         }
-    }
+    };
+    if (!L.ib_outer) baby_steps(0);
 
     ckks_ct *out_m = out;
     for (uint32_t m = 0; m < nmat; m++) {
@@ -984,6 +996,67 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
                 gcount = std::max(gcount, std::min(i.size, o.size) / B);
                 if (i.size > o.size) fold = i.size / o.size;
             }
+            // the giant steps of a group of accumulators accg (giants g0 .. g0 + ng - 1, all shards)
+            auto giant_steps = [&](u64 *acc, uint32_t g0, uint32_t ng) {
+                for (uint32_t gl = 0; gl < ng && !lazy; gl++) {
+                    const uint32_t gi = g0 + gl;
+                    u64 *ag = acc + (size_t)gl * S * ctl;
+                    if (gi == 0) {
+                        cudaMemcpyAsync(total, ag, (size_t)S * ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+                        continue;
+                    }
+                    const u64 ge = ckks_galois_element(c, (int64_t)gi * B * T);
+                    const u64 *key = (const u64 *)find_key(keys, nkeys, ge)->data;
+                    // total[sh] += rotate(acc_g[sh]) for all shards in one batch
+                    ks_modup(c, ag + ptl, level, kw, s, S, ctl);
+                    ks_inner_moddown(c, key, level, ge, kw, ag, nullptr, ge, total, s, S, ctl, ctl, true);
+                }
+                // lazy: the key-switched parts of up to IP_TERMS giant steps (all shards) are extended in one batch and
+                // added to the running sum in the key-switching basis in one pass, their first components with them
+                for (uint32_t gl = 0; gl < ng && lazy;) {
+                    if (g0 + gl == 0) {
+                        cudaMemcpyAsync(total, acc, (size_t)S * ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+                        gl++;
+                        continue;
+                    }
+                    const uint32_t nterm = std::min(IP_TERMS, ng - gl);
+                    u64 *ag = acc + (size_t)gl * S * ctl;
+                    ks_modup(c, ag + ptl, level, kx, s, nterm * S, ctl);
+                    IpTerms tm{};
+                    for (uint32_t t = 0; t < nterm; t++) {
+                        const u64 ge = ckks_galois_element(c, (int64_t)(g0 + gl + t) * B * T);
+                        tm.evk[t] = (const u64 *)find_key(keys, nkeys, ge)->data;
+                        tm.galois[t] = ge;
+                        tm.c0[t] = ag + (size_t)t * S * ctl;
+                    }
+                    ks_inner_terms(c, level, kx, (size_t)S * kbeta * knt * N, tm, nterm, ctl, s, S, u_live);
+                    u_live = true;
+                    gl += nterm;
+                }
+            };
+            if (L.ib_outer) {
+                // one input block at a time: its baby steps, then its share of every giant step's accumulator (block 0 is a
+                // full block, so its launch initialises every accumulator it reaches); the giant steps follow at the end
+                for (uint32_t ib = 0; ib < nib; ib++) {
+                    const Block &i = p.ins[ib];
+                    const uint32_t cnt = std::min(i.size, o.size) / B;
+                    baby_steps(ib);
+                    for (uint32_t g0 = 0; g0 < cnt; g0 += L.gg) {
+                        const uint32_t ngi = std::min(L.gg, cnt - g0);
+                        u64 *accg = acc + (size_t)g0 * S * ctl;
+                        const bool covered = ib > 0 || ngi == std::min(L.gg, gcount - g0);
+                        if (ib == 0 && !covered) cudaMemsetAsync(accg, 0, (size_t)std::min(L.gg, gcount - g0) * S * ctl * sizeof(u64), s);
+                        for (uint32_t gl = 0; gl < ngi; gl++)
+                            launch_extract_diagonals(c, W, d->d_out, i.start, i.size, o.start, o.size, p.F, T, (g0 + gl) * B, B, (g0 + gl) * B,
+                                                     slots + (size_t)gl * B * c->n, s);
+                        TiledOut to;
+                        to.R = ngi * B; to.row0 = 0; to.row_stride = 1;
+                        launch_encode(c, slots, nullptr, ngi * B, pt_scale, level, pts, encw, s, to, ptt);
+                        launch_mac_mma(c, baby, ptt, accg, B, S, ngi, level, s, B, 0, ib > 0 || !covered);
+                    }
+                }
+                for (uint32_t g0 = 0; g0 < gcount; g0 += L.gg) giant_steps(acc + (size_t)g0 * S * ctl, g0, std::min(L.gg, gcount - g0));
+            } else
             for (uint32_t g0 = 0; g0 < gcount; g0 += L.gg) {
                 const uint32_t ng = std::min(L.gg, gcount - g0);
                 const uint32_t J = nib * B;
@@ -1035,41 +1108,7 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
                 }
                 if (!launch_mac_mma(c, baby, ptt, acc, J, S, ng, level, s)) launch_mac_tile(c, baby, ptt, acc, J, S, ng, level, s);
                 }
-                for (uint32_t gl = 0; gl < ng && !lazy; gl++) {
-                    const uint32_t gi = g0 + gl;
-                    u64 *ag = acc + (size_t)gl * S * ctl;
-                    if (gi == 0) {
-                        cudaMemcpyAsync(total, ag, (size_t)S * ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
-                        continue;
-                    }
-                    const u64 ge = ckks_galois_element(c, (int64_t)gi * B * T);
-                    const u64 *key = (const u64 *)find_key(keys, nkeys, ge)->data;
-                    // total[sh] += rotate(acc_g[sh]) for all shards in one batch
-                    ks_modup(c, ag + ptl, level, kw, s, S, ctl);
-                    ks_inner_moddown(c, key, level, ge, kw, ag, nullptr, ge, total, s, S, ctl, ctl, true);
-                }
-                // lazy: the key-switched parts of up to IP_TERMS giant steps (all shards) are extended in one batch and
-                // added to the running sum in the key-switching basis in one pass, their first components with them
-                for (uint32_t gl = 0; gl < ng && lazy;) {
-                    if (g0 + gl == 0) {
-                        cudaMemcpyAsync(total, acc, (size_t)S * ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
-                        gl++;
-                        continue;
-                    }
-                    const uint32_t nterm = std::min(IP_TERMS, ng - gl);
-                    u64 *ag = acc + (size_t)gl * S * ctl;
-                    ks_modup(c, ag + ptl, level, kx, s, nterm * S, ctl);
-                    IpTerms tm{};
-                    for (uint32_t t = 0; t < nterm; t++) {
-                        const u64 ge = ckks_galois_element(c, (int64_t)(g0 + gl + t) * B * T);
-                        tm.evk[t] = (const u64 *)find_key(keys, nkeys, ge)->data;
-                        tm.galois[t] = ge;
-                        tm.c0[t] = ag + (size_t)t * S * ctl;
-                    }
-                    ks_inner_terms(c, level, kx, (size_t)S * kbeta * knt * N, tm, nterm, ctl, s, S, u_live);
-                    u_live = true;
-                    gl += nterm;
-                }
+                giant_steps(acc, g0, ng);
             }
             if (u_live) ks_moddown(c, level, kw, total, total + ptl, 1, total, s, S, ctl, ctl, false);
             for (uint32_t f = o.size; fold > 1; f *= 2, fold /= 2) {
@@ -1124,5 +1163,5 @@ extern "C" size_t ckks_linear_proj_multi_workspace_bytes(const ckks_ctx *c, cons
         merged.gmax = std::max(merged.gmax, p.gmax);
         lazy = lazy || (descs[m].flags & CKKS_PROJ_LAZY_MODDOWN) != 0;
     }
-    return proj_layout(c, merged, level, lazy).bytes;
+    return proj_layout(c, merged, level, lazy, nmat).bytes;
 }

@@ -25,7 +25,7 @@ __global__ void __launch_bounds__(THREADS) permute_kernel(DevTables c, const u64
 
 // targets per CTA row in the basis-conversion kernels: the source limbs are re-read once per chunk, so large batches
 // take all targets in one chunk and single ciphertexts split them for parallelism
-inline uint32_t conv_chunk(uint32_t nb) { return nb >= 4 ? 32 : 8; }
+inline uint32_t conv_chunk(uint32_t nb) { return nb >= 4 ? 32 : 16; }
 
 // ext[j][x][k] for x over q_0..q_{level-1}, p_0..p_{K-1}.  dcoef: sigma_g(d) in the coefficient domain;
 // deval: d in the evaluation domain, read through sigma_g for the digit's own limbs.
