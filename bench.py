@@ -704,6 +704,28 @@ def layer_submetrics(ctx, residues, allp, gen, dev, reps, have_keys):
     bws = ctx.workspace(ctx.workspace_bytes(binding.OP_MUL_RELIN_BATCH, LEVEL, 128))
     out["ms"]["products_2x2048_each_relinearised"] = timed(lambda: [ctx.mul_relin_batch(pa, pb, rlk, outs=bouts, ws=bws) for _ in range(32)])
     out["layer_linear_and_products_s"] = out["projections_s"] + out["ms"]["products_2x2048_summed_128_per_output"] * 1e-3
+    del bouts, bws, a, b, acc
+    ctx._ws = None
+    torch.cuda.empty_cache()
+    # the same products inside the attention entry points (diagonal-block layout: 128 tokens, 32 heads, 8 diagonals per
+    # ciphertext, 128 channels): scores with the key operands' hoisted rotations, Softmax by doubling over rows spread
+    # across 16 ciphertexts (two rounds, degree-4 polynomials), probability x value with the value operands' rotations
+    tokens, heads, E, dim = 128, 32, 8, 128
+    rots = ctx.attention_rotations(tokens, heads, E)
+    akeys = [binding.SwitchKey(residues(allp, DNUM, 2), ctx.galois_element(r)) for r in rots]
+    q = [binding.Ciphertext(residues(allp[:L], 2), 2.0 ** 50) for _ in range(dim)]
+    k = [binding.Ciphertext(residues(allp[:L], 2), 2.0 ** 50) for _ in range(dim)]
+    v = q                                   # same shape and level; the values' content does not matter to the kernels
+    poly = [1.0, 0.25, 0.03, 0.002, 0.0001]
+    att = {}
+    S = ctx.attention_scores(q, k, rlk, akeys, tokens, heads, E)
+    att["scores"] = timed(lambda: ctx.attention_scores(q, k, rlk, akeys, tokens, heads, E))
+    P = ctx.softmax_rows(S, 3.0, 2, poly, [poly, poly], rlk, akeys, tokens, heads, E)
+    att["softmax_rows"] = timed(lambda: ctx.softmax_rows(S, 3.0, 2, poly, [poly, poly], rlk, akeys, tokens, heads, E))
+    att["values"] = timed(lambda: ctx.attention_values(P, v, rlk, akeys, tokens, heads, E))
+    att["levels"] = {"operands": LEVEL, "scores": S[0].level, "probabilities": P[0].level, "outputs": P[0].level - 1}
+    att["total_s"] = (att["scores"] + att["softmax_rows"] + att["values"]) * 1e-3
+    out["attention_32_heads_128_tokens_dim_128_ms"] = att
     return out
 
 
