@@ -77,11 +77,15 @@ def test_rotate_and_hoisted_bit_exact(log_n, L, K, dnum, levels):
         for k, dk, g in zip(keys, dkeys, gals):
             out = ctx.rotate(dct, dk)
             assert np.array_equal(host(out.data), o.rotate(ct, k, g)), (level, g)
+        plain = []
+        for k, dk, g in zip(keys, dkeys, gals):
+            plain.append(host(ctx.rotate(dct, dk).data))
         outs = ctx.rotate_hoisted(dct, dkeys)
         want = o.rotate_hoisted(ct, keys, gals)
         for i, out in enumerate(outs):
             got = host(out.data)
             assert np.array_equal(got, want[i]), (level, i)
+            assert np.array_equal(got, plain[i]), (level, i)      # the contract: hoisted and plain rotation give the same integers
             if level >= 2:
                 assert np.abs(cl.decrypt_slots(got, 2.0 ** 40).real - np.roll(z, -rots[i])).max() < truth_tol(log_n)
     # error paths: even Galois element, aliasing, short workspace
