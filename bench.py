@@ -730,6 +730,7 @@ def layer_submetrics(ctx, residues, allp, gen, dev, reps, have_keys):
 
 
 def main():
+    global LAZY, NTT_BATCH
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=3)
@@ -737,6 +738,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--parts", default="abc", help="with --profile: which parts of the step to run (a: NTT, b: key switching, c: projection)")
     ap.add_argument("--shards", type=int, default=SHARDS, help="with --profile: token shards in the projection (default 16)")
+    ap.add_argument("--ntt-batch", type=int, default=NTT_BATCH, help="with --profile: polynomials in the NTT part (default 32)")
     ap.add_argument("--eager-moddown", action="store_true",
                     help="one ModDown per giant-step rotation instead of one per output ciphertext")
     ap.add_argument("--no-extras", action="store_true", help="skip the untimed one-off measurements of the composite calls")
@@ -747,8 +749,9 @@ def main():
     ap.add_argument("--profile", action="store_true",
                     help="for profiler captures: honour --warmup below 3 and skip the e2e and CPU legs (prints no bench line)")
     args = ap.parse_args()
-    global LAZY
     LAZY = not args.eager_moddown
+    if args.profile:
+        NTT_BATCH = args.ntt_batch
     if args.impl == "reference":
         run_reference(args)
     else:
