@@ -563,7 +563,7 @@ def run_cuda(args):
     roofline.update({
         "kernel": "ntt16_fwd_cols + ntt16_fwd_rows (forward NTT of 768 limbs, one launch each)",
         # ncu, dram read + write bytes of the two launches; None when no capture of the current kernels is recorded
-        "traffic": profile_figure("ntt16_768limbs.md", "dram_bytes_per_launch_pair"),
+        "traffic": profile_figure("ntt16_384limbs.md", "dram_bytes_per_launch_pair"),
         "ms_per_launch_pair": ntt_fwd_ms,
         "vs_register_resident_butterflies": {
             "achieved_gbfly_s": limb_ntts * BFLY / (ntt_fwd_ms * 1e-3) / 1e9, "peak_gbfly_s": probe_rate / 1e9,
@@ -626,12 +626,12 @@ def run_cuda(args):
                          # recorded with its command: x 16 shards = what the extrapolation should land near
                          "one_shard_anchor_s": profile_figure("oracle_one_shard.md", "one_shard_seconds")},
         # figures copied from ncu captures (profiles/), with the kernels they were taken on: not measured in this run
-        "static_notes": {"source": "profiles/bench_step_launch_list.md, profiles/ntt16_768limbs.md",
+        "static_notes": {"source": "profiles/bench_step_launch_list.md, profiles/ntt16_384limbs.md",
                          "ntt16_family_share_of_step": profile_figure("bench_step_launch_list.md", "ntt16_family_share"),
                          "mac_share_of_step": profile_figure("bench_step_launch_list.md", "mac_share"),
                          "keyswitch_kernels_share_of_step": profile_figure("bench_step_launch_list.md", "keyswitch_kernels_share"),
-                         "fp64_pipe_active_fwd_cols": profile_figure("ntt16_768limbs.md", "fp64_pipe_active_fwd_cols"),
-                         "fp64_pipe_active_fwd_rows": profile_figure("ntt16_768limbs.md", "fp64_pipe_active_fwd_rows")},
+                         "fp64_pipe_active_fwd_cols": profile_figure("ntt16_384limbs.md", "fp64_pipe_active_fwd_cols"),
+                         "fp64_pipe_active_fwd_rows": profile_figure("ntt16_384limbs.md", "fp64_pipe_active_fwd_rows")},
     }
     print(json.dumps(line))
     if world > 1:
