@@ -79,10 +79,11 @@ int make_plan(const ckks_ctx *c, const ckks_proj_desc *d, ProjPlan &p) {
     return CKKS_OK;
 }
 
-struct ProjWs { size_t baby, xin, pts, ptt, slots, enc, acc, total, tmp, ks, ksx, rs, bytes; uint32_t gg, gacc; bool per_block, ib_outer; };
+struct ProjWs { size_t baby, xin, pts, ptt, slots, enc, acc, total, tmp, ks, ksx, rs, bytes; uint32_t gg, gacc, eg; bool per_block, ib_outer; };
 
 constexpr uint32_t BABY_ROTS = 4;            // baby-step rotations per key-switch pass (N = 2^16)
 constexpr uint32_t MAC_GT = 4;               // giants per register tile of the fallback multiply-accumulate kernel
+constexpr uint32_t ENC_PTS = 128;            // plaintexts per encode call of the tensor-core path (its scratch is 13.25 MiB each)
 
 ProjWs proj_layout(const ckks_ctx *c, const ProjPlan &p, uint32_t level, bool lazy, uint32_t nmat = 1) {
     const size_t ct = (size_t)2 * level * c->N * sizeof(u64), pt = (size_t)level * c->N * sizeof(u64);
@@ -103,24 +104,39 @@ ProjWs proj_layout(const ckks_ctx *c, const ProjPlan &p, uint32_t level, bool la
     w.gacc = w.ib_outer ? (p.gmax + w.gg - 1) / w.gg * w.gg : w.gg;
     const size_t nbb = w.ib_outer ? 1 : nib;                // input blocks whose baby ciphertexts are resident together
     const size_t npt = (size_t)w.gg * (w.per_block ? 1 : nib) * p.B;
+    // the tensor-core path encodes a group's plaintexts a few giants at a time straight into the tiled buffer, so the
+    // encoder's scratch (slot values, FFT buffer, coefficients, the words between the two NTT passes) serves ENC_PTS plaintexts
+    w.eg = w.per_block ? std::max<uint32_t>(1, std::min<uint32_t>(w.gg, ENC_PTS / p.B)) : w.gg;
+    const size_t nenc = w.per_block ? (size_t)w.eg * p.B : npt;
+    const size_t knt = level + c->K, kbeta = (level + c->alpha - 1) / c->alpha;
+    // all shards' key switches run side by side; the baby steps take BABY_ROTS rotations per pass, which needs that
+    // many inner-product and conversion buffers per input ciphertext
+    const size_t ks_sz = align256(ks_bytes(c, level) * p.S * nbb + (size_t)(BABY_ROTS - 1) * p.S * nbb * (2 * knt + 2 * level) * c->N * sizeof(u64));
+    // lazy giant steps: coefficient copies and extended digits of IP_TERMS giant steps of every shard
+    const size_t ksx_sz = lazy ? align256((size_t)IP_TERMS * p.S * (level + kbeta * (level + c->K)) * c->N * sizeof(u64)) : 0;
     size_t off = 0;
     w.baby = off;  off += align256(ct * p.S * nbb * p.B);   // tiled: rows (shard * J + j) * 2 + component
-    w.xin = off;   off += align256(ct * p.S * nib);         // the inputs side by side, plain layout
-    w.pts = off;   off += align256(pt * npt);               // encoded plaintexts of a group, plain layout
-    w.ptt = off;   off += align256(pt * npt);               // the same, tiled: rows g * J + j
-    w.slots = off; off += align256(npt * c->n * sizeof(double));
-    w.enc = off;   off += align256(encode_workspace_bytes(c, (uint32_t)npt));
+    w.xin = off;   off += align256(ct * p.S * nbb);         // the inputs of the resident blocks side by side, plain layout
     w.acc = off;   off += align256(ct * p.S * w.gacc);
     w.total = off; off += align256(ct * p.S);
     w.tmp = off;   off += align256(ct);
-    // all shards' key switches run side by side; the baby steps take BABY_ROTS rotations per pass, which needs that
-    // many inner-product and conversion buffers per input ciphertext
-    const size_t knt = level + c->K;
-    w.ks = off;    off += align256(ks_bytes(c, level) * p.S * nbb + (size_t)(BABY_ROTS - 1) * p.S * nbb * (2 * knt + 2 * level) * c->N * sizeof(u64));
-    // lazy giant steps: coefficient copies and extended digits of IP_TERMS giant steps of every shard
-    const size_t kbeta = (level + c->alpha - 1) / c->alpha;
-    w.ksx = off;   off += lazy ? align256((size_t)IP_TERMS * p.S * (level + kbeta * (level + c->K)) * c->N * sizeof(u64)) : 0;
     w.rs = off;    off += align256(rescale_bytes(c, level, 2));
+    const size_t shared = off;
+    w.ptt = off;   off += align256(pt * npt);               // encoded plaintexts of a group, tiled: rows g * J + j
+    w.pts = off;   off += align256(pt * nenc);              // plain layout: the encoder's words between its two NTT passes
+    w.slots = off; off += align256(nenc * c->n * sizeof(double));
+    w.enc = off;   off += align256(encode_workspace_bytes(c, (uint32_t)nenc));
+    // With the input blocks in the outer loop no key switch runs between a block's first encode and its last
+    // multiply-accumulate and nothing of a key switch outlives its phase (the baby steps of a block; the giant steps at
+    // the end), so the key-switch buffers share their bytes with the plaintext buffers.  In the other order the running
+    // sum of the lazy giant steps lives in a key-switch buffer across the groups, so they stay apart.
+    if (w.ib_outer) {
+        w.ks = shared; w.ksx = shared + ks_sz;
+        off = std::max(off, shared + ks_sz + ksx_sz);
+    } else {
+        w.ks = off;    off += ks_sz;
+        w.ksx = off;   off += ksx_sz;
+    }
     w.bytes = off;
     return w;
 }
@@ -937,8 +953,9 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
     // all input blocks, or one block at a time (L.ib_outer): its inputs are then the ciphertexts ib, ib + nib, ..
     const uint32_t nbb = L.ib_outer ? 1 : nib;
     const uint32_t Jall = nbb * B, Rx = 2 * S * Jall;
-    for (uint32_t x = 0; x < S * nib; x++)
-        cudaMemcpyAsync(xin + (size_t)x * ctl, in[x].data, ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
+    if (!L.ib_outer)
+        for (uint32_t x = 0; x < S * nib; x++)
+            cudaMemcpyAsync(xin + (size_t)x * ctl, in[x].data, ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
     KsWorkspace kw = ks_carve(c, level, base + L.ks, S * nbb);
     // lazy giant steps: digits of IP_TERMS x S accumulators side by side; the running sum and the ModDown use kw's buffers
     const uint32_t kbeta = (level + c->alpha - 1) / c->alpha, knt = level + c->K;
@@ -946,9 +963,12 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
     kx.dcoef = (u64 *)(base + L.ksx);
     kx.ext = kx.dcoef + (size_t)IP_TERMS * S * level * N;
     auto baby_steps = [&](uint32_t ib0) {
-        const u64 *xb = xin + (size_t)ib0 * ctl;                       // first ciphertext of the set
-        const size_t xs = (size_t)(L.ib_outer ? nib : 1) * ctl;       // from one ciphertext of the set to the next
+        const u64 *xb = xin;                                           // first ciphertext of the set
+        const size_t xs = ctl;                                         // from one ciphertext of the set to the next
         const uint32_t nx = S * nbb;
+        if (L.ib_outer)
+            for (uint32_t sh = 0; sh < S; sh++)
+                cudaMemcpyAsync(xin + (size_t)sh * ctl, in[sh * nib + ib0].data, ctl * sizeof(u64), cudaMemcpyDeviceToDevice, s);
         for (uint32_t comp = 0; comp < 2; comp++)
             launch_to_tiled(c, xb + comp * ptl, xs, nx, baby, Rx, comp, 2 * B, level, s);
         if (B <= 1) return;
@@ -1034,6 +1054,18 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
                     gl += nterm;
                 }
             };
+            // the diagonals of giants g0 .. g0 + ngi - 1 of a block pair, encoded into rows 0 .. ngi B - 1 of the tiled buffer
+            auto encode_group = [&](const Block &i, uint32_t g0, uint32_t ngi) {
+                for (uint32_t e0 = 0; e0 < ngi; e0 += L.eg) {
+                    const uint32_t ne = std::min(L.eg, ngi - e0);
+                    for (uint32_t gl = 0; gl < ne; gl++)
+                        launch_extract_diagonals(c, W, d->d_out, i.start, i.size, o.start, o.size, p.F, T, (g0 + e0 + gl) * B, B,
+                                                 (g0 + e0 + gl) * B, slots + (size_t)gl * B * c->n, s);
+                    TiledOut to;
+                    to.R = ngi * B; to.row0 = e0 * B; to.row_stride = 1;
+                    launch_encode(c, slots, nullptr, ne * B, pt_scale, level, pts, encw, s, to, ptt);
+                }
+            };
             if (L.ib_outer) {
                 // one input block at a time: its baby steps, then its share of every giant step's accumulator (block 0 is a
                 // full block, so its launch initialises every accumulator it reaches); the giant steps follow at the end
@@ -1046,12 +1078,7 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
                         u64 *accg = acc + (size_t)g0 * S * ctl;
                         const bool covered = ib > 0 || ngi == std::min(L.gg, gcount - g0);
                         if (ib == 0 && !covered) cudaMemsetAsync(accg, 0, (size_t)std::min(L.gg, gcount - g0) * S * ctl * sizeof(u64), s);
-                        for (uint32_t gl = 0; gl < ngi; gl++)
-                            launch_extract_diagonals(c, W, d->d_out, i.start, i.size, o.start, o.size, p.F, T, (g0 + gl) * B, B, (g0 + gl) * B,
-                                                     slots + (size_t)gl * B * c->n, s);
-                        TiledOut to;
-                        to.R = ngi * B; to.row0 = 0; to.row_stride = 1;
-                        launch_encode(c, slots, nullptr, ngi * B, pt_scale, level, pts, encw, s, to, ptt);
+                        encode_group(i, g0, ngi);
                         launch_mac_mma(c, baby, ptt, accg, B, S, ngi, level, s, B, 0, ib > 0 || !covered);
                     }
                 }
@@ -1071,12 +1098,7 @@ static int32_t run_projections(ckks_ctx *c, const ckks_proj_desc *descs, uint32_
                         const uint32_t cnt = std::min(i.size, o.size) / B;
                         if (g0 >= cnt) continue;
                         const uint32_t ngi = std::min(ng, cnt - g0);
-                        for (uint32_t gl = 0; gl < ngi; gl++)
-                            launch_extract_diagonals(c, W, d->d_out, i.start, i.size, o.start, o.size, p.F, T, (g0 + gl) * B, B, (g0 + gl) * B,
-                                                     slots + (size_t)gl * B * c->n, s);
-                        TiledOut to;
-                        to.R = ngi * B; to.row0 = 0; to.row_stride = 1;
-                        launch_encode(c, slots, nullptr, ngi * B, pt_scale, level, pts, encw, s, to, ptt);
+                        encode_group(i, g0, ngi);
                         launch_mac_mma(c, baby, ptt, acc, B, S, ngi, level, s, J, ib * B, !full0 || ib > 0);
                     }
                 } else {
