@@ -27,7 +27,7 @@ struct DevTables {
     const ulonglong2 *tw_inv;  // [T][N] inverses of the same
     const ulonglong2 *n_inv;   // [T] {N^-1, Shoup}
     // fp64 copies for the double-precision NTT path (N = 2^16 only): the centred representative of w as a double, same
-    // indexing (w/q is formed in the kernel as w * (1/q): half the table bytes for one extra multiply per twiddle)
+    // indexing (the transform estimates a product's quotient from the rounded product and 1/q, so the table holds w alone)
     const double *twd_fwd, *twd_inv;    // [T][N]
     const double2 *n_inv_d;             // [T][2] {N^-1, N^-1/q}, {w N^-1, that/q} for the inverse's last twiddle w, all centred
     // inverse-transform scalings that deliver the basis conversions' first factor y = [d qhat^-1] (N = 2^16 only), pairs
@@ -177,6 +177,16 @@ __device__ __forceinline__ double mulmod_d(double y, double2 w, double q) {
     const double e = __fma_rn(y, w.x, -p);
     const double M = COARSE ? MAGIC1 : MAGIC0;
     const double k = __dsub_rn(__fma_rn(y, w.y, M), M);
+    return __dadd_rn(__fma_rn(-k, q, p), e);
+}
+// The same with the quotient estimated from the rounded product, k = round(p * (1/q)): p and 1/q are each within 2^-53
+// relative, so the estimate is as close as with a precomputed w * (1/q), and no per-twiddle multiply is needed.
+template <int COARSE>
+__device__ __forceinline__ double mulmod_pq(double y, double w, double q, double qinv) {
+    const double p = __dmul_rn(y, w);
+    const double e = __fma_rn(y, w, -p);
+    const double M = COARSE ? MAGIC1 : MAGIC0;
+    const double k = __dsub_rn(__fma_rn(p, qinv, M), M);
     return __dadd_rn(__fma_rn(-k, q, p), e);
 }
 // x * y - k q for two variable residues 0 <= x, y < q (as doubles): exact, |result| <= 0.75 q

@@ -119,6 +119,11 @@ __global__ void __launch_bounds__(THREADS) ntt_rows(DevTables c, u64 *base, Limb
 // ===========================================================================
 
 constexpr uint32_t F_THREADS = 256;
+// CTAs per SM the compiler is asked to fit.  The forward kernels take their quotients from the rounded products (no
+// {w, w/q} pairs in registers) and run four CTAs of 64 registers per SM: 0.422 us per limb against 0.440 with pairs at three
+// CTAs.  The row pass with the ModDown tail would spill at 64 registers and the inverse kernels lose at four CTAs
+// (0.447 against 0.440 us per limb), so those stay at three.
+constexpr uint32_t FWD_CTAS = 4, INV_CTAS = 3;
 
 __device__ __forceinline__ u64 mulhi_under(u64 x, u64 a) {
     const uint32_t x0 = (uint32_t)x, x1 = (uint32_t)(x >> 32), a0 = (uint32_t)a, a1 = (uint32_t)(a >> 32);
@@ -181,7 +186,7 @@ __device__ __forceinline__ u64 reduce_exact(u64 x, u64 q, u64 qinv64) {
 // 53-bit operands in one instruction where the integer pipe needs several
 // 32x32 products, so for 50-bit primes a twiddle product is cheaper there:
 //   p = y w (rounded), e = fma(y, w, -p) (exact low part),
-//   k = round(y * (w/q))  by adding and subtracting 1.5 * 2^52 (or 1.5 * 2^53),
+//   k = round(p * (1/q))  by adding and subtracting 1.5 * 2^52 (or 1.5 * 2^53),
 //   r = fma(-k, q, p) + e  =  y w - k q   exactly, |r| <= (1/2 + eps) q  (or (1 + eps) q).
 // Values are signed integers held in doubles; everything is exact while they stay
 // below 2^53 in magnitude, so each group of four stages starts by reducing its 16
@@ -190,11 +195,11 @@ __device__ __forceinline__ u64 reduce_exact(u64 x, u64 q, u64 qinv64) {
 // intermediate written between the passes is a lazy word in one case and a double
 // in the other); the result is the same canonical residue either way.
 // ---------------------------------------------------------------------------
-// ML consecutive twiddles w (ML = 1, 2, 4, 8; the index is a multiple of ML) with the widest loads that fit, each
-// completed to {w, w * (1/q)}.  w * fl(1/q) is within 2^-52 relative of w/q, which the stage bounds allow for.
+// ML consecutive twiddles w (ML = 1, 2, 4, 8; the index is a multiple of ML) with the widest loads that fit.  The quotient
+// of a twiddle product is estimated from the rounded product and fl(1/q) (mulmod_pq): within 2^-52 relative of y w / q,
+// which the stage bounds allow for, and one multiply per twiddle and half the twiddle registers less than with {w, w/q}.
 template <uint32_t ML>
-__device__ __forceinline__ void load_tw(const double *p, double qinv, double2 (&w)[ML]) {
-    double v[ML];
+__device__ __forceinline__ void load_tw(const double *p, double (&v)[ML]) {
     if (ML == 1) v[0] = __ldg(p);
     if (ML == 2) asm volatile("ld.global.nc.v2.f64 {%0,%1}, [%2];" : "=d"(v[0]), "=d"(v[1]) : "l"(p));
     if (ML >= 4) {
@@ -202,8 +207,6 @@ __device__ __forceinline__ void load_tw(const double *p, double qinv, double2 (&
         for (uint32_t i = 0; i < ML; i += 4)
             asm volatile("ld.global.nc.v4.f64 {%0,%1,%2,%3}, [%4];" : "=d"(v[i]), "=d"(v[(i + 1) % ML]), "=d"(v[(i + 2) % ML]), "=d"(v[(i + 3) % ML]) : "l"(p + i));
     }
-#pragma unroll
-    for (uint32_t i = 0; i < ML; i++) w[i] = make_double2(v[i], __dmul_rn(v[i], qinv));
 }
 __device__ __forceinline__ void stg_4(u64 *p, u64 a, u64 b, u64 c, u64 d) {
     asm volatile("st.global.v4.b64 [%0], {%1,%2,%3,%4};" ::"l"(p), "l"(a), "l"(b), "l"(c), "l"(d) : "memory");
@@ -213,7 +216,7 @@ __device__ __forceinline__ void ldg_4(const u64 *p, u64 &a, u64 &b, u64 &c, u64 
 }
 
 // Range bookkeeping of the double-precision path (B = bound in units of q).  The twiddle tables hold centred
-// representatives, |w| <= q/2, and w/q is known to 2^-52 relative, so for |y| <= B q the product y w - k q comes out below
+// representatives, |w| <= q/2, and the quotient estimate is within 2^-52 relative, so for |y| <= B q the product y w - k q comes out below
 //   T(B) = (1/2 + B/8) q   when k is rounded to the nearest integer (needs B <= 4:  |y w/q| < 2^51), and below
 //   Tc(B) = (1 + B/8) q    when k is rounded to the nearest even integer (needs |y w/q| < 2^52, sums below 2^53 ~ 8 q).
 // A Cooley-Tukey stage takes B to B + T(B): from a canonical input (B = 1) four stages reach 1.63, 2.33, 3.12, 4.01;
@@ -227,14 +230,14 @@ __device__ __forceinline__ void ldg_4(const u64 *p, u64 &a, u64 &b, u64 &c, u64 
 template <uint32_t ML, int COARSE>
 __device__ __forceinline__ void fwd_stage_d(double (&x)[16], const double *__restrict__ tw, uint32_t base, double q, double qinv) {
     constexpr uint32_t tl = 8 / ML;
-    double2 w[ML];
-    load_tw<ML>(tw + ML * base, qinv, w);
+    double w[ML];
+    load_tw<ML>(tw + ML * base, w);
 #pragma unroll
     for (uint32_t i = 0; i < ML; i++)
 #pragma unroll
         for (uint32_t j = 0; j < tl; j++) {
             const uint32_t k1 = 2 * i * tl + j, k2 = k1 + tl;
-            const double t = mulmod_d<COARSE>(x[k2], w[i], q);
+                        const double t = mulmod_pq<COARSE>(x[k2], w[i], q, qinv);
             x[k2] = __dsub_rn(x[k1], t);
             x[k1] = __dadd_rn(x[k1], t);
         }
@@ -272,8 +275,8 @@ __device__ __forceinline__ void fwd16_d(double (&x)[16], const double *__restric
 template <uint32_t ML, int COARSE>
 __device__ __forceinline__ void inv_stage_d(double (&x)[16], const double *__restrict__ tw, uint32_t base, double q, double qinv) {
     constexpr uint32_t tl = 8 / ML;
-    double2 w[ML];
-    load_tw<ML>(tw + ML * base, qinv, w);
+    double w[ML];
+    load_tw<ML>(tw + ML * base, w);
 #pragma unroll
     for (uint32_t i = 0; i < ML; i++)
 #pragma unroll
@@ -281,7 +284,7 @@ __device__ __forceinline__ void inv_stage_d(double (&x)[16], const double *__res
             const uint32_t k1 = 2 * i * tl + j, k2 = k1 + tl;
             const double u = x[k1], v = x[k2];
             x[k1] = __dadd_rn(u, v);
-            x[k2] = mulmod_d<COARSE>(__dsub_rn(u, v), w[i], q);
+            x[k2] = mulmod_pq<COARSE>(__dsub_rn(u, v), w[i], q, qinv);
         }
 }
 __device__ __forceinline__ void inv16_d(double (&x)[16], const double *__restrict__ tw, uint32_t base, double q, double qinv) {
@@ -331,7 +334,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) butterfly_probe_kernel(DevTables
 
 // ---- forward, column pass (stages m = 1..128): CTA = strip of 16 columns -----------------
 template <bool ALLFP>
-__global__ void __launch_bounds__(F_THREADS, 3) ntt16_fwd_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, const long long *coef_src) {
+__global__ void __launch_bounds__(F_THREADS, FWD_CTAS) ntt16_fwd_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, const long long *coef_src) {
     __shared__ u64 sm[256 * 16];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
@@ -403,7 +406,7 @@ __device__ __forceinline__ void bulk_store_wait() { asm volatile("cp.async.bulk.
 
 // ---- forward, row pass (stages m = 256..32768): CTA = 16 rows, 16 threads per row ---------
 template <bool ALLFP, int EP, bool BULK = false>
-__global__ void __launch_bounds__(F_THREADS, 3) ntt16_fwd_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, NttEpilogue ep) {
+__global__ void __launch_bounds__(F_THREADS, EP == 1 ? 3 : FWD_CTAS) ntt16_fwd_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, NttEpilogue ep) {
     constexpr int has_ep = EP;
     __shared__ __align__(16) u64 sm[16 * ROW_PAD];
     const int prime = limb_prime(map, blockIdx.y);
@@ -519,7 +522,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) ntt16_fwd_rows(DevTables c, u64 
 
 // ---- inverse, row pass (stages m = 32768..256) ---------------------------------------------
 template <bool ALLFP>
-__global__ void __launch_bounds__(F_THREADS, 3) ntt16_inv_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, const u64 *src,
+__global__ void __launch_bounds__(F_THREADS, INV_CTAS) ntt16_inv_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, const u64 *src,
                                                                 uint32_t src_pitch) {
     __shared__ __align__(16) u64 sm[16 * ROW_PAD];
     const int prime = limb_prime(map, blockIdx.y);
@@ -578,7 +581,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) ntt16_inv_rows(DevTables c, u64 
 
 // ---- inverse, column pass (stages m = 128..1), then N^-1 and the exact reduction -----------
 template <bool ALLFP>
-__global__ void __launch_bounds__(F_THREADS, 3) ntt16_inv_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, const double2 *scale) {
+__global__ void __launch_bounds__(F_THREADS, INV_CTAS) ntt16_inv_cols(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, const double2 *scale) {
     __shared__ u64 sm[256 * 16];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
