@@ -70,6 +70,7 @@ class AttnDesc:
     tokens: int
     heads: int
     diag_block: int
+    group_baby: int = 1      # attention_scores: baby-step count of the split of the score groups (1 = every group by itself)
 
     def groups(self) -> int:
         return self.tokens // self.diag_block
@@ -407,16 +408,52 @@ class Oracle:
             lad.append(Tk * H * R * k); k *= 2
         return tok, lad
 
+    def attention_query_rotations(self, desc: AttnDesc):
+        """Rotations (in slots, negative: to the right) of the query operands when the score groups are split into
+        group_baby baby steps and groups / group_baby giant steps: -g1 * group_baby * diag_block tokens, g1 >= 1."""
+        tok, _ = self.attention_rotations(desc)
+        Gb, G = desc.group_baby, desc.groups()
+        if Gb < 1 or G % Gb:
+            raise ValueError("group_baby must divide the number of score groups")
+        return [-tok[g1 * Gb - 1] for g1 in range(1, G // Gb)] if Gb > 1 else []
+
     def attention_scores(self, desc: AttnDesc, q, k, rlk, keys: dict):
         """Score ciphertexts S_g, g < groups = tokens / diag_block, from the channel operands q[d], k[d] (d < dim,
         [dim][2][level][N], layout of AttnDesc with the query repeated in every block e and the key operand holding token
         i + e in block e):  S_g = rescale(mul_relin_sum_d(q[d], rotate(k[d], g * diag_block tokens))).
         Slot (e, i, h) of S_g is the score of query i and head h against one key token; over all g and e every key token
         occurs exactly once, so the score row of (i, h) is spread over the groups x diag_block slots (e, i, h) of the S_g.
-        One relinearisation per S_g; the products of a group are summed before it.  Returns [groups][2][level-1][N]."""
+        One relinearisation per S_g; the products of a group are summed before it.  With desc.group_baby = Gb > 1 the
+        groups are split g = g1 Gb + g0:  S_g = rotate(rescale(mul_relin_sum_d(rotate(q[d], -g1 Gb diag_block tokens),
+        rotate(k[d], g0 diag_block tokens))), g1 Gb diag_block tokens), the same slot values from other integers (the last
+        rotation is left out for g1 = 0).  Returns [groups][2][level-1][N]."""
         q = _u64(q); k = _u64(k); level = q.shape[2]
         tok, _ = self.attention_rotations(desc)
         out = np.empty((desc.groups(), 2, level - 1, self.N), dtype=np.uint64)
+        if desc.group_baby > 1:
+            # Baby-step / giant-step split of the groups, g = g1 * Gb + g0: a rotation is a ring automorphism, so
+            #   q[d] * rot_g(k[d]) = rot_{g1 Gb}( rot_{-g1 Gb}(q[d]) * rot_{g0}(k[d]) )
+            # and the query operand is the same in every block, so its right rotation is again a query operand (of the
+            # tokens shifted cyclically).  Per channel Gb - 1 key and G / Gb - 1 query rotations instead of G - 1 key
+            # rotations; every group with g1 > 0 is rotated back once, after its rescale.
+            Gb, G = desc.group_baby, desc.groups()
+            neg = self.attention_query_rotations(desc)
+            dim = q.shape[0]
+            kr, qr = [k], [q]
+            for g0 in range(1, Gb):
+                ge = self.galois_element(tok[g0 - 1])
+                kr.append(np.stack([self.rotate(k[d], keys[ge], ge) for d in range(dim)]))
+            for r in neg:
+                ge = self.galois_element(r)
+                qr.append(np.stack([self.rotate(q[d], keys[ge], ge) for d in range(dim)]))
+            for g in range(G):
+                g1, g0 = divmod(g, Gb)
+                t = self.rescale(self.mul_relin_sum(qr[g1], kr[g0], rlk))
+                if g1:
+                    ge = self.galois_element(tok[g1 * Gb - 1])
+                    t = self.rotate(t, keys[ge], ge)
+                out[g] = t
+            return out
         for g in range(desc.groups()):
             if g == 0:
                 kr = k

@@ -94,3 +94,46 @@ def test_single_group_needs_no_token_rotation_and_one_block_no_ladder():
     assert o.attention_rotations(AttnDesc(16, 4, 1)) == ([g * 4 * 8 for g in range(1, 16)], [])
     with pytest.raises(ValueError):
         o.attention_rotations(AttnDesc(8, 1, 3))
+
+
+@pytest.mark.parametrize("tokens,heads,E,dim,Gb,seed", [(16, 2, 4, 4, 2, 83), (16, 1, 2, 4, 4, 84), (16, 2, 4, 4, 4, 85)])
+def test_scores_with_split_groups_hold_the_same_slots(tokens, heads, E, dim, Gb, seed):
+    """The baby-step / giant-step split of the score groups: the same slot values as Q K^T and as the unsplit schedule
+    (other integers), the rotation set it asks for, and the query operand's right rotation being a query operand again."""
+    P = params(10, 6, 2, 3)
+    o = P.oracle
+    cl = Client(P, seed)
+    plain, split = AttnDesc(tokens, heads, E), AttnDesc(tokens, heads, E, Gb)
+    tok, lad = o.attention_rotations(split)
+    assert (tok, lad) == o.attention_rotations(plain)
+    G, R = split.groups(), P.n // (E * tokens * heads)
+    neg = o.attention_query_rotations(split)
+    assert neg == [-g1 * Gb * E * heads * R for g1 in range(1, G // Gb)] and o.attention_query_rotations(plain) == []
+    level, scale = 6, 2.0 ** 50
+    c = attention_case(seed, tokens, heads, dim, dim, 1)
+    Qs, Ks, _ = inputs.pack_attention_operands(c["Q"], c["K"], c["V"], E, P.n)
+    # in the clear: rolling a query operand to the right by s group steps gives the query operand of the tokens shifted by s E
+    for g1 in range(1, G // Gb):
+        Qshift = np.roll(c["Q"], g1 * Gb * E, axis=0)
+        Qs2, _, _ = inputs.pack_attention_operands(Qshift, c["K"], c["V"], E, P.n)
+        assert np.array_equal(np.roll(Qs, -neg[g1 - 1], axis=1), Qs2)
+    q = np.stack([cl.encrypt_slots(z, scale, level) for z in Qs])
+    k = np.stack([cl.encrypt_slots(z, scale, level) for z in Ks])
+    rlk = cl.relin_key()
+    keys = {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in tok + neg}
+    S = o.attention_scores(split, q, k, rlk, keys)
+    S0 = o.attention_scores(plain, q, k, rlk, keys)
+    assert S.shape == S0.shape
+    for g in range(Gb):
+        assert np.array_equal(S[g], S0[g])                 # groups without a giant step are the unsplit schedule's
+    if G > Gb:
+        assert not np.array_equal(S[Gb], S0[Gb])
+    else:
+        assert np.array_equal(S, S0)                      # a single giant step: nothing is rotated back
+    ss = scale * scale / float(P.q[level - 1])
+    rows = _unpack_rows(split, P.n, [cl.decrypt_slots(S[g], ss).real for g in range(G)])
+    assert np.abs(rows - c["S"].transpose(1, 0, 2)).max() < 2.0 ** -20
+    rows0 = _unpack_rows(plain, P.n, [cl.decrypt_slots(S0[g], ss).real for g in range(G)])
+    assert np.abs(rows - rows0).max() < 2.0 ** -22
+    with pytest.raises(ValueError):
+        o.attention_query_rotations(AttnDesc(tokens, heads, E, 3))
