@@ -708,18 +708,22 @@ def layer_submetrics(ctx, residues, allp, gen, dev, reps, have_keys):
     ctx._ws = None
     torch.cuda.empty_cache()
     # the same products inside the attention entry points (diagonal-block layout: 128 tokens, 32 heads, 8 diagonals per
-    # ciphertext, 128 channels): scores with the key operands' hoisted rotations, Softmax by doubling over rows spread
+    # ciphertext, 128 channels): scores with hoisted rotations of the key and query operands (groups split 4 x 4), Softmax by doubling over rows spread
     # across 16 ciphertexts (two rounds, degree-4 polynomials), probability x value with the value operands' rotations
     tokens, heads, E, dim = 128, 32, 8, 128
-    rots = ctx.attention_rotations(tokens, heads, E)
+    GB = 4                                  # score groups split into 4 baby x 4 giant steps
+    rots = ctx.attention_rotations(tokens, heads, E, GB)
     akeys = [binding.SwitchKey(residues(allp, DNUM, 2), ctx.galois_element(r)) for r in rots]
     q = [binding.Ciphertext(residues(allp[:L], 2), 2.0 ** 50) for _ in range(dim)]
     k = [binding.Ciphertext(residues(allp[:L], 2), 2.0 ** 50) for _ in range(dim)]
     v = q                                   # same shape and level; the values' content does not matter to the kernels
     poly = [1.0, 0.25, 0.03, 0.002, 0.0001]
     att = {}
-    S = ctx.attention_scores(q, k, rlk, akeys, tokens, heads, E)
-    att["scores"] = timed(lambda: ctx.attention_scores(q, k, rlk, akeys, tokens, heads, E))
+    att["scores_every_group_by_itself"] = timed(lambda: ctx.attention_scores(q, k, rlk, akeys, tokens, heads, E))
+    ctx._ws = None
+    torch.cuda.empty_cache()
+    S = ctx.attention_scores(q, k, rlk, akeys, tokens, heads, E, group_baby=GB)
+    att["scores"] = timed(lambda: ctx.attention_scores(q, k, rlk, akeys, tokens, heads, E, group_baby=GB))
     P = ctx.softmax_rows(S, 3.0, 2, poly, [poly, poly], rlk, akeys, tokens, heads, E)
     att["softmax_rows"] = timed(lambda: ctx.softmax_rows(S, 3.0, 2, poly, [poly, poly], rlk, akeys, tokens, heads, E))
     att["values"] = timed(lambda: ctx.attention_values(P, v, rlk, akeys, tokens, heads, E))

@@ -312,6 +312,12 @@ size_t ckks_softmax_workspace_bytes(const ckks_ctx *ctx, const ckks_softmax_desc
  *     scores: host array of `groups` descriptors with buffers for level - 1 limbs.  Every rotated operand is bit-identical
  *     to ckks_rotate's.  Workspace: ckks_attention_scores_workspace_bytes holds all rotated operands at once
  *     ((groups - 1) * dim ciphertexts); any workspace that holds one group's is accepted and the groups are then taken in passes.
+ *     desc->group_baby = Gb > 1 (a power of two dividing groups) splits the groups g = g1 Gb + g0 into baby and giant steps:
+ *     S_g = rot_{g1 Gb}( rescale( sum_d rot_{-g1 Gb}(q[d]) * rot_{g0}(k[d]) ) ), the same slot values (a rotation is a ring
+ *     automorphism and a query operand rotated to the right is the query operand of cyclically shifted tokens) from other
+ *     integers: per channel Gb - 1 key and groups / Gb - 1 query rotations instead of groups - 1 key rotations, and one
+ *     rotation per group with g1 > 0 after its rescale.  The workspace then holds all rotated operands
+ *     ((Gb + groups / Gb - 2) * dim ciphertexts) and is needed in full.  group_baby 0 or 1: no split.
  *   ckks_softmax_rows: Algorithm 1 on rows spread that way.  Per group u_g = p_exp(S_g - shift); per round
  *     t = rescale(sum_g u_g^2) (one relinearisation), t += rot(t, tokens * heads * R * 2^k) for k < log2 diag_block (cyclic
  *     over e: the row sum in every slot of the row), lambda = p_rsqrt_j(t) once for all groups, u_g = rescale(rescale(lambda
@@ -321,9 +327,10 @@ size_t ckks_softmax_workspace_bytes(const ckks_ctx *ctx, const ckks_softmax_desc
  *     over e: slot (e, i, h) of out[d] holds sum over all key tokens of probability x value, in every block e (the query
  *     operand's layout).  out: dim_v descriptors with buffers for P's level - 1.
  *   ckks_attention: the three in a row (scores at level - 1, then the Softmax's levels, then one more).
- * keys must hold the rotations ckks_attention_rotations lists (token rotations first, then the ladder).
+ * keys must hold the rotations ckks_attention_rotations lists (token rotations first, then the ladder, then, with
+ * group_baby > 1, the query operands' right rotations as negative numbers).
  * Errors: ARG, LEVEL, SCALE, NO_KEY, WORKSPACE, UNSUPPORTED (shape rules above), RANGE (a polynomial constant). */
-typedef struct { uint32_t tokens, heads, diag_block; } ckks_attn_desc;
+typedef struct { uint32_t tokens, heads, diag_block, group_baby; } ckks_attn_desc;
 int32_t ckks_attention_rotations(const ckks_ctx *ctx, const ckks_attn_desc *desc, int64_t *rots, uint32_t cap);
 int32_t ckks_attention_scores(ckks_ctx *ctx, const ckks_attn_desc *desc, const ckks_ct *q, const ckks_ct *k, uint32_t dim,
                               const ckks_evk *rlk, const ckks_evk *keys, uint32_t nkeys, ckks_ct *scores, void *ws, size_t ws_bytes, void *stream);

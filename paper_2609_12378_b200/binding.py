@@ -58,7 +58,7 @@ class CSoftmaxDesc(C.Structure):
 
 
 class CAttnDesc(C.Structure):
-    _fields_ = [("tokens", C.c_uint32), ("heads", C.c_uint32), ("diag_block", C.c_uint32)]
+    _fields_ = [("tokens", C.c_uint32), ("heads", C.c_uint32), ("diag_block", C.c_uint32), ("group_baby", C.c_uint32)]
 
 
 class CProjDesc(C.Structure):
@@ -426,8 +426,8 @@ class Context:
         """The first c.level limbs per component of a buffer written densely as [2][c.level][N]."""
         return Ciphertext(out.data.view(-1)[: 2 * c.level * self.N].view(2, c.level, self.N), c.scale)
 
-    def attention_rotations(self, tokens: int, heads: int, diag_block: int):
-        d = CAttnDesc(tokens, heads, diag_block)
+    def attention_rotations(self, tokens: int, heads: int, diag_block: int, group_baby: int = 1):
+        d = CAttnDesc(tokens, heads, diag_block, group_baby)
         n = load().ckks_attention_rotations(self._h, C.byref(d), None, 0)
         if n < 0:
             raise CkksError(n)
@@ -435,9 +435,11 @@ class Context:
         load().ckks_attention_rotations(self._h, C.byref(d), buf, n)
         return list(buf)[:n]
 
-    def attention_scores(self, q, k, rlk: SwitchKey, keys, tokens, heads, diag_block, ws: torch.Tensor = None, stream=None):
-        """Score ciphertexts S_g (one per group of diag_block diagonals) from the channel operands q[d], k[d]."""
-        d = CAttnDesc(tokens, heads, diag_block)
+    def attention_scores(self, q, k, rlk: SwitchKey, keys, tokens, heads, diag_block, ws: torch.Tensor = None, stream=None,
+                         group_baby: int = 1):
+        """Score ciphertexts S_g (one per group of diag_block diagonals) from the channel operands q[d], k[d]; group_baby > 1
+        splits the groups into baby and giant steps."""
+        d = CAttnDesc(tokens, heads, diag_block, group_baby)
         level, G = q[0].level, tokens // diag_block
         outs = [self.empty_ct(level - 1) for _ in range(G)]
         if ws is None:
@@ -455,7 +457,7 @@ class Context:
 
     def softmax_rows(self, cts, shift, rounds, exp_coeffs, rsqrt_coeffs, rlk: SwitchKey, keys, tokens, heads, diag_block, stream=None):
         """Softmax by doubling on score rows spread over the groups' ciphertexts (slots (e, i, h) of every group)."""
-        d = CAttnDesc(tokens, heads, diag_block)
+        d = CAttnDesc(tokens, heads, diag_block, 1)
         sd = self._softmax_desc(shift, rounds, exp_coeffs, rsqrt_coeffs)
         level = cts[0].level
         need = int(load().ckks_softmax_rows_workspace_bytes(self._h, C.byref(d), C.byref(sd), level))
@@ -473,7 +475,7 @@ class Context:
 
     def attention_values(self, probs, v, rlk: SwitchKey, keys, tokens, heads, diag_block, stream=None):
         """Output channels sum over key tokens of probability x value, in the query operand's layout."""
-        d = CAttnDesc(tokens, heads, diag_block)
+        d = CAttnDesc(tokens, heads, diag_block, 1)
         lp = probs[0].level
         ws = self.workspace(int(load().ckks_attention_values_workspace_bytes(self._h, C.byref(d), lp)))
         outs = [self.empty_ct(lp - 1) for _ in v]
@@ -489,9 +491,9 @@ class Context:
         return outs
 
     def attention(self, q, k, v, shift, rounds, exp_coeffs, rsqrt_coeffs, rlk: SwitchKey, keys, tokens, heads, diag_block,
-                  ws: torch.Tensor = None, stream=None):
+                  ws: torch.Tensor = None, stream=None, group_baby: int = 1):
         """Scores, Softmax over the score rows and probability x value in one call; returns the output channels."""
-        d = CAttnDesc(tokens, heads, diag_block)
+        d = CAttnDesc(tokens, heads, diag_block, group_baby)
         sd = self._softmax_desc(shift, rounds, exp_coeffs, rsqrt_coeffs)
         level = q[0].level
         need = int(load().ckks_attention_workspace_bytes(self._h, C.byref(d), C.byref(sd), level, len(q)))

@@ -20,8 +20,8 @@
 namespace {
 
 struct AttnPlan {
-    uint32_t E, Tk, H, R, G;
-    std::vector<int64_t> tok, lad;      // rotations in slots
+    uint32_t E, Tk, H, R, G, Gb;
+    std::vector<int64_t> tok, lad, neg;      // rotations in slots (neg: the query operands' right rotations of the split)
 };
 
 bool pow2(uint32_t x) { return x && !(x & (x - 1)); }
@@ -34,6 +34,10 @@ int make_attn_plan(const ckks_ctx *c, const ckks_attn_desc *d, AttnPlan &p) {
     p.E = d->diag_block; p.Tk = d->tokens; p.H = d->heads; p.R = (uint32_t)(c->n / block); p.G = p.Tk / p.E;
     for (uint32_t g = 1; g < p.G; g++) p.tok.push_back((int64_t)g * p.E * p.H * p.R);
     for (uint32_t k = 1; k < p.E; k *= 2) p.lad.push_back((int64_t)p.Tk * p.H * p.R * k);
+    p.Gb = d->group_baby ? d->group_baby : 1;
+    if (!pow2(p.Gb) || p.G % p.Gb) return CKKS_ERR_UNSUPPORTED;
+    if (p.Gb > 1)
+        for (uint32_t g1 = 1; g1 < p.G / p.Gb; g1++) p.neg.push_back(-p.tok[g1 * p.Gb - 1]);
     return CKKS_OK;
 }
 
@@ -90,6 +94,7 @@ extern "C" int32_t ckks_attention_rotations(const ckks_ctx *c, const ckks_attn_d
     uint32_t k = 0;
     for (int64_t r : p.tok) { if (rots && k < cap) rots[k] = r; k++; }
     for (int64_t r : p.lad) { if (rots && k < cap) rots[k] = r; k++; }
+    for (int64_t r : p.neg) { if (rots && k < cap) rots[k] = r; k++; }
     return (int32_t)k;
 }
 
@@ -98,7 +103,49 @@ extern "C" int32_t ckks_attention_rotations(const ckks_ctx *c, const ckks_attn_d
 extern "C" size_t ckks_attention_scores_workspace_bytes(const ckks_ctx *c, const ckks_attn_desc *d, uint32_t level, uint32_t dim) {
     AttnPlan p;
     if (!c || !dim || level < 2 || level > c->L || make_attn_plan(c, d, p)) return 0;
+    // the split holds Gb - 1 rotated key sets, G / Gb - 1 rotated query sets, a product and a rescaled product
+    if (p.Gb > 1) return (size_t)(p.Gb + p.G / p.Gb - 2) * dim * ct_bytes(c, level) + 2 * ct_bytes(c, level) + scratch_bytes(c, level, p.G - 1);
     return (size_t)(p.G - 1) * dim * ct_bytes(c, level) + ct_bytes(c, level) + scratch_bytes(c, level, p.G - 1);
+}
+
+// scores with the groups split into Gb baby and G / Gb giant steps
+static int scores_split(ckks_ctx *c, const AttnPlan &p, const ckks_ct *q, const ckks_ct *k, uint32_t dim, uint32_t level, const ckks_evk *rlk,
+                        const ckks_evk *keys, uint32_t nkeys, ckks_ct *scores, void *ws, size_t ws_bytes, void *stream) {
+    const uint32_t Gb = p.Gb, Gg = p.G / p.Gb;
+    const size_t ctb = ct_bytes(c, level);
+    char *base = (char *)ws;
+    char *kr = base, *qr = base + (size_t)(Gb - 1) * dim * ctb;         // [Gb - 1][dim], [Gg - 1][dim] ciphertexts
+    char *rest = qr + (size_t)(Gg - 1) * dim * ctb;
+    ckks_ct prod{(uint64_t *)rest, level, 2, 0.0}, resc{(uint64_t *)(rest + ctb), level - 1, 2, 0.0};
+    void *sw = rest + 2 * ctb;
+    const size_t sw_bytes = ws_bytes - (size_t)((char *)sw - base);
+    int rc;
+    std::vector<ckks_evk> bk, gk;
+    for (uint32_t g0 = 1; g0 < Gb; g0++) bk.push_back(*find_key(c, keys, nkeys, p.tok[g0 - 1]));
+    for (int64_t r : p.neg) gk.push_back(*find_key(c, keys, nkeys, r));
+    std::vector<ckks_ct> outs(std::max(Gb, Gg));
+    for (uint32_t dd = 0; dd < dim; dd++) {
+        for (uint32_t x = 0; x + 1 < Gb; x++) outs[x] = ckks_ct{(uint64_t *)(kr + ((size_t)x * dim + dd) * ctb), level, 2, 0.0};
+        if (Gb > 1 && (rc = ckks_rotate_hoisted(c, &k[dd], bk.data(), Gb - 1, outs.data(), sw, sw_bytes, stream))) return rc;
+        for (uint32_t y = 0; y + 1 < Gg; y++) outs[y] = ckks_ct{(uint64_t *)(qr + ((size_t)y * dim + dd) * ctb), level, 2, 0.0};
+        if (Gg > 1 && (rc = ckks_rotate_hoisted(c, &q[dd], gk.data(), Gg - 1, outs.data(), sw, sw_bytes, stream))) return rc;
+    }
+    std::vector<ckks_ct> a(dim), b(dim);
+    for (uint32_t g = 0; g < p.G; g++) {
+        const uint32_t g1 = g / Gb, g0 = g % Gb;
+        for (uint32_t dd = 0; dd < dim; dd++) {
+            a[dd] = g1 ? ckks_ct{(uint64_t *)(qr + ((size_t)(g1 - 1) * dim + dd) * ctb), level, 2, q[dd].scale} : q[dd];
+            b[dd] = g0 ? ckks_ct{(uint64_t *)(kr + ((size_t)(g0 - 1) * dim + dd) * ctb), level, 2, k[dd].scale} : k[dd];
+        }
+        if ((rc = ckks_mul_relin_sum(c, a.data(), b.data(), dim, rlk, &prod, sw, sw_bytes, stream))) return rc;
+        if (!g1) {
+            if ((rc = ckks_rescale(c, &prod, &scores[g], sw, sw_bytes, stream))) return rc;
+            continue;
+        }
+        if ((rc = ckks_rescale(c, &prod, &resc, sw, sw_bytes, stream))) return rc;
+        if ((rc = ckks_rotate(c, &resc, find_key(c, keys, nkeys, p.tok[g1 * Gb - 1]), &scores[g], sw, sw_bytes, stream))) return rc;
+    }
+    return CKKS_OK;
 }
 
 extern "C" int32_t ckks_attention_scores(ckks_ctx *c, const ckks_attn_desc *d, const ckks_ct *q, const ckks_ct *k, uint32_t dim,
@@ -114,8 +161,14 @@ extern "C" int32_t ckks_attention_scores(ckks_ctx *c, const ckks_attn_desc *d, c
     if (!rlk_ok(rlk)) return CKKS_ERR_NO_KEY;
     for (int64_t r : p.tok)
         if (!keys || !find_key(c, keys, nkeys, r)) return CKKS_ERR_NO_KEY;
+    for (int64_t r : p.neg)
+        if (!find_key(c, keys, nkeys, r)) return CKKS_ERR_NO_KEY;
     for (uint32_t g = 0; g < p.G; g++)
         if (!scores[g].data) return CKKS_ERR_ARG;
+    if (p.Gb > 1) {
+        if (!ws || ws_bytes < ckks_attention_scores_workspace_bytes(c, d, level, dim)) return CKKS_ERR_WORKSPACE;
+        return scores_split(c, p, q, k, dim, level, rlk, keys, nkeys, scores, ws, ws_bytes, stream);
+    }
     // as many groups per pass as the workspace holds (one at least)
     const size_t ctb = ct_bytes(c, level), fixed = ctb + scratch_bytes(c, level, p.G - 1);
     uint32_t per_pass = p.G > 1 ? (uint32_t)std::min<size_t>(p.G - 1, ws_bytes > fixed ? (ws_bytes - fixed) / ((size_t)dim * ctb) : 0) : 0;

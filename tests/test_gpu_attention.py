@@ -10,12 +10,12 @@ from tests.harness import Client, attention_case, params
 pytestmark = pytest.mark.gpu
 
 
-def _setup(log_n, L, K, dnum, level, tokens, heads, E, dim, dim_v, seed, rounds=1):
+def _setup(log_n, L, K, dnum, level, tokens, heads, E, dim, dim_v, seed, rounds=1, Gb=1):
     from tests.gpu_util import context, ct_dev, key_dev
     P, ctx = params(log_n, L, K, dnum), context(log_n, L, K, dnum)
     o = P.oracle
     cl = Client(P, seed)
-    desc = AttnDesc(tokens, heads, E)
+    desc = AttnDesc(tokens, heads, E, Gb)
     scale = 2.0 ** 50
     c = attention_case(seed, tokens, heads, dim, dim_v, rounds)
     Qs, Ks, Vs = inputs.pack_attention_operands(c["Q"], c["K"], c["V"], E, P.n)
@@ -23,8 +23,9 @@ def _setup(log_n, L, K, dnum, level, tokens, heads, E, dim, dim_v, seed, rounds=
     k = np.stack([cl.encrypt_slots(z, scale, level) for z in Ks])
     v = np.stack([cl.encrypt_slots(z, scale, level) for z in Vs])
     tok, lad = o.attention_rotations(desc)
-    assert ctx.attention_rotations(tokens, heads, E) == tok + lad
-    keys = {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in tok + lad}
+    neg = o.attention_query_rotations(desc)
+    assert ctx.attention_rotations(tokens, heads, E, Gb) == tok + lad + neg
+    keys = {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in tok + lad + neg}
     rlk = cl.relin_key()
     dev = dict(q=[ct_dev(x, scale) for x in q], k=[ct_dev(x, scale) for x in k], v=[ct_dev(x, scale) for x in v],
                rlk=key_dev(rlk, 0), keys=[key_dev(kk, ge) for ge, kk in keys.items()])
@@ -68,6 +69,44 @@ def test_attention_stages_bit_exact(log_n, L, K, dnum, level, tokens, heads, E, 
         got = cl.decrypt_slots(arr, whole[d].scale).real
         assert np.abs(got - c["out_clear"][i, h, d]).max() < 2.0 ** -19
         assert np.abs(got - c["out_true"][i, h, d]).max() < 0.05
+
+
+@pytest.mark.parametrize("tokens,heads,E,dim,Gb", [(16, 2, 4, 3, 2), (16, 4, 1, 2, 4), (16, 1, 2, 2, 8), (8, 2, 4, 2, 2)])
+def test_attention_scores_with_split_groups_bit_exact(tokens, heads, E, dim, Gb):
+    """The score groups split into baby and giant steps (rotated queries, one rotation back per group): every limb equals
+    the checker's, the whole block in one call too, and a workspace short of the full size is refused."""
+    import ctypes as C
+
+    import torch
+
+    from tests.gpu_util import host
+    level = 13
+    P, ctx, o, cl, desc, c, scale, q, k, v, rlk, keys, dev = _setup(10, 13, 4, 4, level, tokens, heads, E, dim, 1, 700 + tokens + E + Gb, Gb=Gb)
+    a = (tokens, heads, E)
+    S = o.attention_scores(desc, q, k, rlk, keys)
+    dS = ctx.attention_scores(dev["q"], dev["k"], dev["rlk"], dev["keys"], *a, group_baby=Gb)
+    ss = scale * scale / float(P.q[level - 1])
+    for g in range(desc.groups()):
+        assert dS[g].scale == ss and dS[g].level == level - 1
+        assert np.array_equal(host(dS[g].data), S[g]), g
+    want, so = o.attention(desc, q, k, v, scale, scale, c["shift"], 1, c["exp_coeffs"], c["rsqrt_coeffs"], rlk, keys)
+    got = ctx.attention(dev["q"], dev["k"], dev["v"], c["shift"], 1, c["exp_coeffs"], c["rsqrt_coeffs"], dev["rlk"], dev["keys"], *a, group_baby=Gb)
+    assert ctx.device_status() == binding.OK
+    e, i, h = inputs.attention_slot_index(tokens, heads, E, P.n)
+    assert got[0].scale == so and np.array_equal(host(got[0].data), want[0])
+    assert np.abs(cl.decrypt_slots(host(got[0].data), so).real - c["out_clear"][i, h, 0]).max() < 2.0 ** -19
+    d = binding.CAttnDesc(*a, Gb)
+    need = binding.load().ckks_attention_scores_workspace_bytes(ctx._h, C.byref(d), level, dim)
+    with pytest.raises(binding.CkksError) as err:
+        ctx.attention_scores(dev["q"], dev["k"], dev["rlk"], dev["keys"], *a, ws=torch.empty(need - 256, dtype=torch.uint8, device="cuda"), group_baby=Gb)
+    assert err.value.code == binding.ERR_WORKSPACE
+    if desc.groups() > Gb:
+        with pytest.raises(binding.CkksError) as err:
+            ctx.attention_scores(dev["q"], dev["k"], dev["rlk"], dev["keys"][:-1], *a, group_baby=Gb)   # a query rotation's key is missing
+        assert err.value.code == binding.ERR_NO_KEY
+    with pytest.raises(binding.CkksError) as err:
+        ctx.attention_rotations(tokens, heads, E, 3)
+    assert err.value.code == binding.ERR_UNSUPPORTED
 
 
 def test_attention_scores_in_passes_and_errors():
@@ -114,12 +153,13 @@ def test_attention_scores_in_passes_and_errors():
 @pytest.mark.slow
 def test_attention_full_ring():
     """N = 2^16 with the decoder layer's attention shape in the slots (128 tokens, 32 heads, 8 diagonals per ciphertext:
-    16 groups, every slot used) and a few channels: bit-exact in one call, and Softmax attention after decryption."""
+    16 groups split into 4 baby and 4 giant steps, every slot used) and a few channels: bit-exact in one call, and Softmax attention after decryption."""
     from tests.gpu_util import host
-    tokens, heads, E, dim, dim_v, level = 128, 32, 8, 2, 1, 13
-    P, ctx, o, cl, desc, c, scale, q, k, v, rlk, keys, dev = _setup(16, 24, 8, 3, level, tokens, heads, E, dim, dim_v, 660)
+    tokens, heads, E, dim, dim_v, level, Gb = 128, 32, 8, 2, 1, 13, 4
+    P, ctx, o, cl, desc, c, scale, q, k, v, rlk, keys, dev = _setup(16, 24, 8, 3, level, tokens, heads, E, dim, dim_v, 660, Gb=Gb)
     want, so = o.attention(desc, q, k, v, scale, scale, c["shift"], 1, c["exp_coeffs"], c["rsqrt_coeffs"], rlk, keys)
-    got = ctx.attention(dev["q"], dev["k"], dev["v"], c["shift"], 1, c["exp_coeffs"], c["rsqrt_coeffs"], dev["rlk"], dev["keys"], tokens, heads, E)
+    got = ctx.attention(dev["q"], dev["k"], dev["v"], c["shift"], 1, c["exp_coeffs"], c["rsqrt_coeffs"], dev["rlk"], dev["keys"], tokens, heads, E,
+                        group_baby=Gb)
     assert ctx.device_status() == binding.OK
     e, i, h = inputs.attention_slot_index(tokens, heads, E, P.n)
     for d in range(dim_v):
