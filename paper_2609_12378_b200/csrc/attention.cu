@@ -283,11 +283,16 @@ extern "C" int32_t ckks_softmax_rows(ckks_ctx *c, const ckks_attn_desc *d, const
 }
 
 // ---- probability x value ------------------------------------------------------------------------------------------
-// workspace: the truncated value operand and its rotated copies, a product, a sum, the scratch of the calls
+// The ladder over the blocks runs for VAL_CHUNK output channels at a time (ckks_rotate_batch: their key switches side by side).
+constexpr uint32_t VAL_CHUNK = 16;
+static size_t values_scratch(const ckks_ctx *c, uint32_t level, uint32_t nrot) {
+    return std::max(scratch_bytes(c, level, nrot), align256(ckks_workspace_bytes(c, CKKS_OP_ROTATE_BATCH, level - 1, VAL_CHUNK)));
+}
+// workspace: the truncated value operand and its rotated copies, a product, the rotated outputs of a chunk, the scratch of the calls
 extern "C" size_t ckks_attention_values_workspace_bytes(const ckks_ctx *c, const ckks_attn_desc *d, uint32_t level) {
     AttnPlan p;
     if (!c || level < 2 || level > c->L || make_attn_plan(c, d, p)) return 0;
-    return (size_t)(p.G + 2) * ct_bytes(c, level) + scratch_bytes(c, level, p.G - 1);
+    return (size_t)(p.G + 1) * ct_bytes(c, level) + (size_t)VAL_CHUNK * ct_bytes(c, level - 1) + values_scratch(c, level, p.G - 1);
 }
 
 extern "C" int32_t ckks_attention_values(ckks_ctx *c, const ckks_attn_desc *d, const ckks_ct *probs, const ckks_ct *v, uint32_t dim_v,
@@ -312,28 +317,37 @@ extern "C" int32_t ckks_attention_values(ckks_ctx *c, const ckks_attn_desc *d, c
     char *base = (char *)ws;
     std::vector<ckks_ct> vr(p.G);
     for (uint32_t g = 0; g < p.G; g++) vr[g] = ckks_ct{(uint64_t *)(base + (size_t)g * ctb), lp, 2, v[0].scale};
-    ckks_ct prod{(uint64_t *)(base + (size_t)p.G * ctb), lp, 2, 0.0}, tmp{(uint64_t *)(base + (size_t)(p.G + 1) * ctb), lp, 2, 0.0};
-    void *sw = base + (size_t)(p.G + 2) * ctb;
-    const size_t sw_bytes = scratch_bytes(c, lp, p.G - 1);
+    ckks_ct prod{(uint64_t *)(base + (size_t)p.G * ctb), lp, 2, 0.0};
+    const size_t ctb1 = ct_bytes(c, lp - 1);
+    char *rot = base + (size_t)(p.G + 1) * ctb;                          // [VAL_CHUNK] rotated outputs of the ladder
+    void *sw = rot + (size_t)VAL_CHUNK * ctb1;
+    const size_t sw_bytes = values_scratch(c, lp, p.G - 1);
     std::vector<ckks_evk> pk;
     for (int64_t r : p.tok) pk.push_back(*find_key(c, keys, nkeys, r));
     cudaStream_t st = (cudaStream_t)stream;
-    for (uint32_t dd = 0; dd < dim_v; dd++) {
-        int prev = 0;
-        cudaGetDevice(&prev);
-        cudaSetDevice(c->device);
-        for (uint32_t comp = 0; comp < 2; comp++)
-            cudaMemcpyAsync(vr[0].data + (size_t)comp * lp * N, v[dd].data + (size_t)comp * lv * N, (size_t)lp * N * sizeof(uint64_t),
-                            cudaMemcpyDeviceToDevice, st);
-        cudaSetDevice(prev);
-        if (p.G > 1 && (rc = ckks_rotate_hoisted(c, &vr[0], pk.data(), p.G - 1, vr.data() + 1, sw, sw_bytes, stream))) return rc;
-        for (uint32_t g = 0; g < p.G; g++) vr[g].scale = v[dd].scale;
-        if ((rc = ckks_mul_relin_sum(c, probs, vr.data(), p.G, rlk, &prod, sw, sw_bytes, stream))) return rc;
-        ckks_ct o = out[dd];
-        if ((rc = ckks_rescale(c, &prod, &o, sw, sw_bytes, stream))) return rc;
-        tmp.level = o.level;
-        if ((rc = block_ladder(c, p, keys, nkeys, &o, &tmp, sw, sw_bytes, stream))) return rc;
-        out[dd] = o;
+    std::vector<ckks_ct> tmp(VAL_CHUNK);
+    for (uint32_t d0 = 0; d0 < dim_v; d0 += VAL_CHUNK) {
+        const uint32_t nd = std::min(VAL_CHUNK, dim_v - d0);
+        for (uint32_t dd = d0; dd < d0 + nd; dd++) {
+            int prev = 0;
+            cudaGetDevice(&prev);
+            cudaSetDevice(c->device);
+            for (uint32_t comp = 0; comp < 2; comp++)
+                cudaMemcpyAsync(vr[0].data + (size_t)comp * lp * N, v[dd].data + (size_t)comp * lv * N, (size_t)lp * N * sizeof(uint64_t),
+                                cudaMemcpyDeviceToDevice, st);
+            cudaSetDevice(prev);
+            if (p.G > 1 && (rc = ckks_rotate_hoisted(c, &vr[0], pk.data(), p.G - 1, vr.data() + 1, sw, sw_bytes, stream))) return rc;
+            for (uint32_t g = 0; g < p.G; g++) vr[g].scale = v[dd].scale;
+            if ((rc = ckks_mul_relin_sum(c, probs, vr.data(), p.G, rlk, &prod, sw, sw_bytes, stream))) return rc;
+            if ((rc = ckks_rescale(c, &prod, &out[dd], sw, sw_bytes, stream))) return rc;
+        }
+        // the ladder over the blocks, a rotation of the whole chunk at a time: out += rotate(out, r), r ascending
+        for (int64_t r : p.lad) {
+            for (uint32_t x = 0; x < nd; x++) tmp[x] = ckks_ct{(uint64_t *)(rot + (size_t)x * ctb1), lp - 1, 2, 0.0};
+            if ((rc = ckks_rotate_batch(c, &out[d0], nd, find_key(c, keys, nkeys, r), tmp.data(), sw, sw_bytes, stream))) return rc;
+            for (uint32_t x = 0; x < nd; x++)
+                if ((rc = ckks_add(c, &out[d0 + x], &tmp[x], &out[d0 + x], stream))) return rc;
+        }
     }
     return CKKS_OK;
 }
