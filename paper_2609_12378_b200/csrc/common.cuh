@@ -57,6 +57,8 @@ struct DevTables {
     // Encode:
     const uint32_t *enc_src;       // [n] slot index feeding FFT input position pos (bit-reversed e_j)
     const double2 *enc_omega;      // [n] exp(2 pi i t / n)
+    const double2 *enc_omega_st;   // [min(n, 1024)] the same values stage by stage: entry half + j = omega^(j n / (2 half)), half = 1, 2, .. (entry 0 unused)
+    const double2 *enc_omega_st2;  // [n] second-pass twiddles by stage and row: entry (hr + jr) * ch + col = omega^((jr ch + col) n / (2 hr ch)), ch = min(n, 1024)
     const double2 *enc_zeta;       // [n] exp(2 pi i k / 2N)
     int *range_flag;               // [0] sticky encode overflow flag, [1] sticky device-side wait timeout flag
 };

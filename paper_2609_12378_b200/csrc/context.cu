@@ -378,6 +378,21 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
         ze[t] = make_double2(cos(2.0 * M_PI * (double)t / (double)(2.0 * N)), sin(2.0 * M_PI * (double)t / (double)(2.0 * N)));
     }
 
+    // the twiddles of the encoder's first pass (stages m = 2 .. min(n, 1024)) laid out stage by stage, so that a CTA
+    // fetches them once into shared memory with contiguous loads
+    const uint32_t enc_ch = std::min<uint32_t>(n, 1024);
+    std::vector<double2> om_st(enc_ch, make_double2(0.0, 0.0));
+    for (uint32_t half = 1; half < enc_ch; half <<= 1)
+        for (uint32_t j = 0; j < half; j++) om_st[half + j] = om[(size_t)j * (n / (2 * half))];
+
+    // the second pass's twiddles (stages m = 2 ch .. n on strips of columns) by stage and row, so that a strip's 16
+    // columns of a row are 16 consecutive entries
+    std::vector<double2> om_st2(n, make_double2(0.0, 0.0));
+    for (uint32_t hr = 1; hr < n / enc_ch; hr <<= 1)
+        for (uint32_t jr = 0; jr < hr; jr++)
+            for (uint32_t col = 0; col < enc_ch; col++)
+                om_st2[(size_t)(hr + jr) * enc_ch + col] = om[((size_t)jr * enc_ch + col) * (n / (2 * hr * enc_ch))];
+
     DevTables &d = c->dev;
     d.conv_groups = conv_groups; d.log_n = prm->log_n; d.N = N; d.L = L; d.K = K; d.alpha = alpha; d.T = T; d.dnum = prm->dnum;
     int rc = CKKS_OK;
@@ -387,7 +402,7 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
         (rc = upload(c, twi, &d.tw_inv)) || (rc = upload(c, twdf, &d.twd_fwd)) || (rc = upload(c, twdi, &d.twd_inv)) || (rc = upload(c, ninvd, &d.n_inv_d)) || (rc = upload(c, isc_up, &d.inv_scale_up)) || (rc = upload(c, isc_dn, &d.inv_scale_dn)) || (rc = upload(c, ninv, &d.n_inv)) || (rc = upload(c, up_inv, &d.up_hat_inv)) ||
         (rc = upload(c, up_mod, &d.up_hat_mod)) || (rc = upload(c, up_mod_d, &d.up_hat_mod_d)) || (rc = upload(c, dn_mod_d, &d.dn_hat_mod_d)) || (rc = upload(c, dn_inv, &d.dn_hat_inv)) ||
         (rc = upload(c, dn_mod, &d.dn_hat_mod)) || (rc = upload(c, dn_pinv, &d.dn_p_inv)) || (rc = upload(c, dn_pinv_d, &d.dn_p_inv_d)) || (rc = upload(c, dn_pmod_d, &d.dn_p_mod_d)) || (rc = upload(c, up_bmat, &d.up_bmat)) || (rc = upload(c, dn_bmat, &d.dn_bmat)) || (rc = upload(c, two52, &d.two52_d)) || (rc = upload(c, rs, &d.rs_inv)) ||
-        (rc = upload(c, enc_src, &d.enc_src)) || (rc = upload(c, om, &d.enc_omega)) || (rc = upload(c, ze, &d.enc_zeta)) ||
+        (rc = upload(c, enc_src, &d.enc_src)) || (rc = upload(c, om, &d.enc_omega)) || (rc = upload(c, om_st, &d.enc_omega_st)) || (rc = upload(c, om_st2, &d.enc_omega_st2)) || (rc = upload(c, ze, &d.enc_zeta)) ||
         (rc = upload(c, flag, &flag_dev))) {
         cudaSetDevice(prev);
         ckks_context_destroy(c);

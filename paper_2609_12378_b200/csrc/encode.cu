@@ -26,20 +26,24 @@ __device__ __forceinline__ double2 cmul_conj_w(double2 w, double2 v) {   // conj
     return make_double2(__dsub_rn(p0, p1), __dadd_rn(p2, p3));
 }
 
-// Pass 1: gather (E1 + bit reversal), stages m = 2 .. min(n, CH) on chunks of CH points.
+// Pass 1: gather (E1 + bit reversal), stages m = 2 .. min(n, CH) on chunks of CH points.  The stages' twiddles come from
+// a copy in shared memory (stage by stage, so that a warp reads consecutive entries): fetched from the full table they
+// were 5120 scattered 16-byte loads per CTA and the kernel was bound by the traffic between L2 and L1.
 __global__ void __launch_bounds__(THREADS) fft_chunks(DevTables c, const double *re, const double *im, double2 *buf, uint32_t n, uint32_t ch) {
     __shared__ double2 sm[CH];
+    __shared__ double2 tw[CH];
     const uint32_t b = blockIdx.y, base = blockIdx.x * ch;
     for (uint32_t x = threadIdx.x; x < ch; x += THREADS) {
         const uint32_t j = c.enc_src[base + x];
         sm[x] = make_double2(re[(size_t)b * n + j], im ? im[(size_t)b * n + j] : 0.0);
+        tw[x] = c.enc_omega_st[x];
     }
     __syncthreads();
     for (uint32_t m = 2; m <= ch; m <<= 1) {
-        const uint32_t half = m >> 1, stride = n / m;
+        const uint32_t half = m >> 1;
         for (uint32_t x = threadIdx.x; x < ch / 2; x += THREADS) {
             const uint32_t j = x & (half - 1), i1 = ((x - j) << 1) + j;
-            const double2 t = cmul_conj_w(c.enc_omega[j * stride], sm[i1 + half]);
+            const double2 t = cmul_conj_w(tw[half + j], sm[i1 + half]);
             const double2 u = sm[i1];
             sm[i1] = make_double2(__dadd_rn(u.x, t.x), __dadd_rn(u.y, t.y));
             sm[i1 + half] = make_double2(__dsub_rn(u.x, t.x), __dsub_rn(u.y, t.y));
@@ -53,15 +57,18 @@ __global__ void __launch_bounds__(THREADS) fft_chunks(DevTables c, const double 
 __global__ void __launch_bounds__(THREADS) fft_strips_round(DevTables c, const double2 *buf, long long *coef, uint32_t n, uint32_t ch, double s) {
     extern __shared__ double2 sm2[];
     const uint32_t b = blockIdx.y, rows = n / ch, col0 = blockIdx.x * COLS;
-    for (uint32_t x = threadIdx.x; x < rows * COLS; x += THREADS)
+    double2 *tw = sm2 + rows * COLS;          // the strip's twiddles, entry (hr + jr) * COLS + column (row 0 unused)
+    for (uint32_t x = threadIdx.x; x < rows * COLS; x += THREADS) {
         sm2[x] = buf[(size_t)b * n + (size_t)(x / COLS) * ch + col0 + x % COLS];
+        tw[x] = c.enc_omega_st2[(size_t)(x / COLS) * ch + col0 + x % COLS];
+    }
     __syncthreads();
     for (uint32_t m = 2 * ch; m <= n; m <<= 1) {
-        const uint32_t half = m >> 1, hr = half / ch, stride = n / m;      // hr = distance in rows
+        const uint32_t half = m >> 1, hr = half / ch;      // hr = distance in rows
         for (uint32_t x = threadIdx.x; x < (rows / 2) * COLS; x += THREADS) {
             const uint32_t cc = x % COLS, y = x / COLS, jr = y & (hr - 1), r1 = ((y - jr) << 1) + jr;
-            const uint32_t j = jr * ch + col0 + cc;                            // position inside the half block
-            const double2 t = cmul_conj_w(c.enc_omega[j * stride], sm2[(r1 + hr) * COLS + cc]);
+            // twiddle omega^(j n / m) of position j = jr ch + col0 + cc inside the half block
+            const double2 t = cmul_conj_w(tw[(hr + jr) * COLS + cc], sm2[(r1 + hr) * COLS + cc]);
             const double2 u = sm2[r1 * COLS + cc];
             sm2[r1 * COLS + cc] = make_double2(__dadd_rn(u.x, t.x), __dadd_rn(u.y, t.y));
             sm2[(r1 + hr) * COLS + cc] = make_double2(__dsub_rn(u.x, t.x), __dsub_rn(u.y, t.y));
@@ -118,7 +125,7 @@ void launch_encode(const ckks_ctx *c, const double *re, const double *im, uint32
         const uint32_t nb = batch - b0 < 32768 ? batch - b0 : 32768;
         fft_chunks<<<dim3(n / ch, nb), THREADS, 0, s>>>(c->dev, re + (size_t)b0 * n, im ? im + (size_t)b0 * n : nullptr,
                                                          buf + (size_t)b0 * n, n, ch); count_launches();
-        fft_strips_round<<<dim3(ch / COLS, nb), THREADS, (size_t)(n / ch) * COLS * sizeof(double2), s>>>(
+        fft_strips_round<<<dim3(ch / COLS, nb), THREADS, (size_t)2 * (n / ch) * COLS * sizeof(double2), s>>>(
             c->dev, buf + (size_t)b0 * n, coef + (size_t)b0 * N, n, ch, sc); count_launches();
     }
     if (c->log_n == 16 && (uint64_t)batch * level <= 32768) {
