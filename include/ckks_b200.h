@@ -133,8 +133,10 @@ const char *ckks_last_cuda_error(const ckks_ctx *ctx);
  *                           about a second).  A wait that runs out makes its kernel drain its copies and return, and
  *                           sets the sticky flag ckks_device_status reports; 0 makes every wait that is not already
  *                           satisfied give up at once (used to test that path).
- *   CKKS_OPT_NTT_BULK_STORE N = 2^16 forward transform, last pass: 1 (default) = every thread stages its 16 results in
- *                           shared memory and a 128-byte bulk copy writes them out, 0 = 32-byte global stores.
+ *   CKKS_OPT_NTT_BULK_STORE N = 2^16 transforms: 1 (default) = in the forward transform's last pass every thread stages its
+ *                           16 results in shared memory and a 128-byte bulk copy writes them out, and in the inverse
+ *                           transform's first pass every thread's 16 inputs arrive by a 128-byte bulk copy (a bounded wait
+ *                           on an mbarrier, see CKKS_OPT_WAIT_CYCLES); 0 = 32-byte global stores and loads.
  *   CKKS_OPT_STATIC_SCRATCH_BYTES  (read only) CKKS_STATIC_SCRATCH_BYTES of the loaded library.
  * set returns CKKS_ERR_ARG for an unknown option or a value outside its range; get returns -1 for an unknown option. */
 enum { CKKS_OPT_NTT_FP_SHARE = 1, CKKS_OPT_CONV_KERNEL = 2, CKKS_OPT_MAC_KERNEL = 3, CKKS_OPT_WAIT_CYCLES = 4,

@@ -404,6 +404,28 @@ __device__ __forceinline__ void bulk_store_128(u64 *gdst, const void *ssrc) {
 }
 __device__ __forceinline__ void bulk_store_wait() { asm volatile("cp.async.bulk.wait_group.read 0;\n" ::: "memory"); }
 
+// The mirror for loads: a warp's 32 threads each fetch their 128-byte block (global -> shared, this GPU's memory, no
+// multicast) and wait on the warp's mbarrier for the 4096 bytes.  The wait is bounded by the SM clock.
+__device__ __forceinline__ void warp_bulk_load_128(uint32_t bar, void *sdst, const u64 *gsrc, uint32_t lane) {
+    if (lane == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(bar) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    __syncwarp();
+    if (lane == 0) asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], 4096;\n" ::"r"(bar) : "memory");
+    asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], 128, [%2];\n"
+                 ::"r"((uint32_t)__cvta_generic_to_shared(sdst)), "l"(gsrc), "r"(bar) : "memory");
+}
+// true once the warp's copies have landed; the verdict is the warp's (one vote)
+__device__ __forceinline__ bool warp_bulk_wait(uint32_t bar, long long limit) {
+    const long long t0 = clock64();
+    uint32_t ok = 0;
+    do {
+        asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\nselp.u32 %0, 1, 0, p;\n}\n" : "=r"(ok) : "r"(bar) : "memory");
+    } while (!ok && clock64() - t0 < limit);
+    return __all_sync(0xffffffffu, ok != 0);
+}
+
 // ---- forward, row pass (stages m = 256..32768): CTA = 16 rows, 16 threads per row ---------
 template <bool ALLFP, int EP, bool BULK = false>
 __global__ void __launch_bounds__(F_THREADS, EP == 1 ? 3 : FWD_CTAS) ntt16_fwd_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, NttEpilogue ep) {
@@ -521,10 +543,11 @@ __global__ void __launch_bounds__(F_THREADS, EP == 1 ? 3 : FWD_CTAS) ntt16_fwd_r
 }
 
 // ---- inverse, row pass (stages m = 32768..256) ---------------------------------------------
-template <bool ALLFP>
+template <bool ALLFP, bool BULK = false>
 __global__ void __launch_bounds__(F_THREADS, INV_CTAS) ntt16_inv_rows(DevTables c, u64 *base, LimbMap map, uint32_t fp_share, const u64 *src,
-                                                                uint32_t src_pitch) {
+                                                                uint32_t src_pitch, long long wait_limit) {
     __shared__ __align__(16) u64 sm[16 * ROW_PAD];
+    __shared__ __align__(8) u64 bars[F_THREADS / 32];
     const int prime = limb_prime(map, blockIdx.y);
     if (prime < 0) return;
     if (ALLFP || (blockIdx.y & 7) < fp_share) {
@@ -536,11 +559,32 @@ __global__ void __launch_bounds__(F_THREADS, INV_CTAS) ntt16_inv_rows(DevTables 
         const u64 *gs = src ? src + ((((size_t)(blockIdx.y / map.period) * src_pitch) + blockIdx.y % map.period) << 16) + (size_t)row * 256 : g;
         double *s = reinterpret_cast<double *>(sm) + rl * ROW_PAD;
         double x[16];
+        if (BULK) {
+            // 16 consecutive coefficients per thread arrive in the thread's own block of the exchange row as one 128-byte
+            // bulk copy: the four 32-byte loads per thread they replace cost the load/store pipe one pass per lane and
+            // sector, which made it the busiest unit of this kernel (inverse transform 0.440 -> 0.426 us per limb).  The
+            // column passes' strided row pieces were measured slower as bulk copies (per warp or per CTA) and stay loads.
+            const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&bars[threadIdx.x >> 5]);
+            u64 *blk = reinterpret_cast<u64 *>(s) + 18 * t;
+            warp_bulk_load_128(bar, blk, gs + 16 * t, threadIdx.x & 31);
+            if (!warp_bulk_wait(bar, wait_limit)) {
+                // report it, give the copies in flight one more bounded wait (their target is this CTA's memory) and leave
+                if ((threadIdx.x & 31) == 0) atomicExch(c.range_flag + 1, 1);
+                warp_bulk_wait(bar, wait_limit);
+                return;
+            }
 #pragma unroll
-        for (uint32_t k = 0; k < 16; k += 4) {      // 16 consecutive coefficients per thread, four 32-byte loads
-            u64 a, b, cc, d;
-            ldg_4(gs + 16 * t + k, a, b, cc, d);
-            x[k] = u64_to_d(a); x[k + 1] = u64_to_d(b); x[k + 2] = u64_to_d(cc); x[k + 3] = u64_to_d(d);
+            for (uint32_t k = 0; k < 16; k += 2) {
+                const ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(blk + k);
+                x[k] = u64_to_d(v.x); x[k + 1] = u64_to_d(v.y);
+            }
+        } else {
+#pragma unroll
+            for (uint32_t k = 0; k < 16; k += 4) {      // 16 consecutive coefficients per thread, four 32-byte loads
+                u64 a, b, cc, d;
+                ldg_4(gs + 16 * t + k, a, b, cc, d);
+                x[k] = u64_to_d(a); x[k + 1] = u64_to_d(b); x[k + 2] = u64_to_d(cc); x[k + 3] = u64_to_d(d);
+            }
         }
         inv16_d(x, tw, 16 * (256 + row) + t, q, qinv);
 #pragma unroll
@@ -657,8 +701,11 @@ void launch_ntt(const ckks_ctx *c, u64 *base, uint32_t nlimbs_total, const LimbM
                 count_launches();
             } else {
                 const u64 *sb = inv_src ? inv_src + (((size_t)(y0 / map.period) * inv_src_pitch) << 16) : nullptr;
-                if (c->ntt_fp_share >= 8) ntt16_inv_rows<true><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, 8, sb, inv_src_pitch);
-                else ntt16_inv_rows<false><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share, sb, inv_src_pitch);
+                // bulk-copy loads need 16-byte aligned sources
+                const bool bulk_in = c->ntt_bulk_store && ((uintptr_t)(sb ? (const void *)sb : (const void *)b) & 15) == 0;
+                if (c->ntt_fp_share >= 8 && bulk_in) ntt16_inv_rows<true, true><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, 8, sb, inv_src_pitch, c->wait_cycles);
+                else if (c->ntt_fp_share >= 8) ntt16_inv_rows<true><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, 8, sb, inv_src_pitch, 0);
+                else ntt16_inv_rows<false><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share, sb, inv_src_pitch, 0);
                 count_launches();
                 if (c->ntt_fp_share >= 8) ntt16_inv_cols<true><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, 8, inv_scale);
                 else ntt16_inv_cols<false><<<grid, F_THREADS, 0, s>>>(c->dev, b, map, c->ntt_fp_share, nullptr);
