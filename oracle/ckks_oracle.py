@@ -71,6 +71,8 @@ class AttnDesc:
     heads: int
     diag_block: int
     group_baby: int = 1      # attention_scores: baby-step count of the split of the score groups (1 = every group by itself)
+    token_inner: int = 1     # tokens kept innermost in the slot index (divides diag_block): slot =
+                             # (((e P + pos) heads + h) token_inner + t) R + r, token = pos token_inner + t, P = tokens / token_inner
 
     def groups(self) -> int:
         return self.tokens // self.diag_block
@@ -401,6 +403,8 @@ class Oracle:
         E, Tk, H = desc.diag_block, desc.tokens, desc.heads
         if Tk % E or self.n % (E * Tk * H) or E & (E - 1) or Tk & (Tk - 1):
             raise ValueError("diag_block must divide tokens, and diag_block * tokens * heads the slot count (powers of two)")
+        if desc.token_inner < 1 or E % desc.token_inner:
+            raise ValueError("token_inner must divide diag_block")
         R = self.n // (E * Tk * H)
         tok = [g * E * H * R for g in range(1, desc.groups())]
         lad, k = [], 1
@@ -531,6 +535,120 @@ class Oracle:
         P, sp = self.softmax_rows(desc, S, ss, shift, rounds, exp_coeffs, rsqrt_coeffs, rlk, keys)
         lp = P.shape[2]
         return self.attention_values(desc, P, v, rlk, keys), sp * v_scale / float(self.q[lp - 1])
+
+    # ---- conversion between the projections' token-shard layout and the attention operands ------------------------
+    def _pack_shape(self, desc: AttnDesc):
+        E, Tk, H, Ti = desc.diag_block, desc.tokens, desc.heads, desc.token_inner
+        self.attention_rotations(desc)
+        if E * Tk * H != self.n:
+            raise ValueError("the conversions need diag_block * tokens * heads = slot count (no trailing copies)")
+        return E, Tk // Ti, H * Ti, Ti                 # blocks, positions per block, slots per position, tokens per position
+
+    def _slot_mask(self, B: int, lo: int, hi: int, Ti: int, t0: int, t1: int):
+        """1.0 on the slots x with lo <= x // B < hi and t0 <= x % Ti < t1, else 0.0."""
+        x = np.arange(self.n)
+        return (((x // B >= lo) & (x // B < hi) & (x % Ti >= t0) & (x % Ti < t1))).astype(np.float64)
+
+    def attention_pack_rotations(self, desc: AttnDesc, kind: int, dim: int):
+        """Rotations (in slots) attention_pack uses.  Block moves (d - c) B for channel d < dim and shard c < P (B = heads *
+        token_inner slots per position); kind 0 (query): the ladder over the blocks; kind 1 (key / value): -P B (a second
+        copy of block 0) and, per block e with e = a token_inner + b, the token shifts a B + b - e P B (slots with
+        t < token_inner - b) and (a + 1) B + b - token_inner - e P B (the others, which take their token from the next
+        position)."""
+        E, P, B, Ti = self._pack_shape(desc)
+        move = sorted({(d - c) * B for d in range(dim) for c in range(P)} - {0})
+        if kind == 0:
+            return move, self.attention_rotations(desc)[1]
+        shift = []
+        for e in range(E):
+            a, b = divmod(e, Ti)
+            shift.append((a * B + b - e * P * B, (a + 1) * B + b - Ti - e * P * B if b else None))
+        return move, ([-P * B] if E > 1 else []), shift
+
+    def _gather_channels(self, desc: AttnDesc, X, dim: int, keys: dict):
+        """Step shared by both kinds: acc[d] = sum_c rotate(X[c], (d - c) B) * mask(position c of block 0), rescaled: block 0
+        of output d holds channel d of every shard at the shard's position.  X: [P][2][level][N] with slot
+        (d heads + h) token_inner + t = value of token c token_inner + t, head h, channel d.  Returns [dim][2][level-1][N]."""
+        E, P, B, Ti = self._pack_shape(desc)
+        X = _u64(X); level = X.shape[2]
+        pt_scale = float(self.q[level - 1])
+        acc = [None] * dim
+        for c in range(P):
+            mask = self.encode(self._slot_mask(B, c, c + 1, Ti, 0, Ti), pt_scale, level)
+            for d in range(dim):
+                r = (d - c) * B
+                if r:
+                    ge = self.galois_element(r)
+                    xr = self.rotate(X[c], keys[ge], ge)
+                else:
+                    xr = X[c]
+                acc[d] = self.mul_plain_acc(xr, mask, acc[d])
+        return np.stack([self.rescale(a) for a in acc])
+
+    def attention_pack(self, desc: AttnDesc, kind: int, X, dim: int, keys: dict):
+        """Attention operands from token-shard ciphertexts in channel-major feature order (the projections' layout with
+        token_inner tokens per shard): X [P][2][level][N], slot (d heads + h) token_inner + t.
+          kind 0 (query):  q[d] = ladder(gathered[d]): channel d of every token in every block e.  Level - 1.
+          kind 1 (key, value): k0 = gathered[d]; k0 = k0 + rotate(k0, -P B) (blocks 0 and 1 hold the tokens); then
+            k[d] = rescale( sum_e [ rotate(k0, sA_e) * mask(block e, t < token_inner - b) + rotate(k0, sB_e) * mask(block e,
+            t >= token_inner - b) ] ) with the shifts of attention_pack_rotations: block e holds token i + e.  Level - 2
+            (level - 1 if diag_block = 1: nothing to shift).
+        Masks are encoded at the scale of the last prime of their level, so that every rescale returns the input's scale.
+        Returns [dim][2][l'][N]."""
+        E, P, B, Ti = self._pack_shape(desc)
+        g = self._gather_channels(desc, X, dim, keys)
+        if kind == 0:
+            return np.stack([self._block_ladder(desc, g[d], keys) for d in range(dim)])
+        if E == 1:
+            return g
+        _, dbl, shift = self.attention_pack_rotations(desc, 1, dim)
+        level = g.shape[2]
+        pt_scale = float(self.q[level - 1])
+        out = []
+        for d in range(dim):
+            ge = self.galois_element(dbl[0])
+            k0 = self.add(g[d], self.rotate(g[d], keys[ge], ge))
+            acc = None
+            for e in range(E):
+                b = e % Ti
+                for part, r in enumerate(shift[e]):
+                    if r is None:
+                        continue
+                    mask = self._slot_mask(B, e * P, (e + 1) * P, Ti, 0, Ti - b) if part == 0 else self._slot_mask(B, e * P, (e + 1) * P, Ti, Ti - b, Ti)
+                    if r % self.n:
+                        ge = self.galois_element(r)
+                        kr = self.rotate(k0, keys[ge], ge)
+                    else:
+                        kr = k0
+                    acc = self.mul_plain_acc(kr, self.encode(mask, pt_scale, level), acc)
+            out.append(self.rescale(acc))
+        return np.stack(out)
+
+    def attention_unpack_rotations(self, desc: AttnDesc, dim: int):
+        """Block moves (c - d) B of attention_unpack, c < P shards, d < dim channels."""
+        E, P, B, Ti = self._pack_shape(desc)
+        return sorted({(c - d) * B for d in range(dim) for c in range(P)} - {0})
+
+    def attention_unpack(self, desc: AttnDesc, O, keys: dict):
+        """Token-shard ciphertexts in channel-major feature order from attention outputs in the query operand's layout
+        (O [dim][2][level][N], every block e alike):  X[c] = rescale( sum_d rotate(O[d], (c - d) B) * mask(slots d B .. d B + B - 1) ):
+        slot (d heads + h) token_inner + t of X[c] holds channel d of token c token_inner + t, head h.  Returns
+        [P][2][level-1][N]."""
+        E, P, B, Ti = self._pack_shape(desc)
+        O = _u64(O); dim, level = O.shape[0], O.shape[2]
+        pt_scale = float(self.q[level - 1])
+        acc = [None] * P
+        for d in range(dim):
+            mask = self.encode(self._slot_mask(B, d, d + 1, Ti, 0, Ti), pt_scale, level)
+            for c in range(P):
+                r = (c - d) * B
+                if r:
+                    ge = self.galois_element(r)
+                    orr = self.rotate(O[d], keys[ge], ge)
+                else:
+                    orr = O[d]
+                acc[c] = self.mul_plain_acc(orr, mask, acc[c])
+        return np.stack([self.rescale(a) for a in acc])
 
     def automorphism_coeff(self, a, g: int, t: int):
         a = _u64(a); out = np.empty_like(a)

@@ -136,24 +136,39 @@ def pack_feature_major(x: np.ndarray, tokens_per_shard: int, slots: int) -> np.n
     return out
 
 
-def attention_slot_index(tokens: int, heads: int, diag_block: int, slots: int):
-    """Index arrays (e, i, h) of every slot of the attention operand layout: slot = ((e * tokens + i) * heads + h) * R + r
-    with R = slots / (diag_block * tokens * heads) trailing copies.  Pure index arithmetic."""
-    E, Tk, H = diag_block, tokens, heads
-    assert slots % (E * Tk * H) == 0 and Tk % E == 0
+def attention_slot_index(tokens: int, heads: int, diag_block: int, slots: int, token_inner: int = 1):
+    """Index arrays (e, i, h) of every slot of the attention operand layout:
+        slot = ((((e * P + pos) * heads + h) * token_inner + t) * R + r,   token i = pos * token_inner + t,
+    P = tokens / token_inner positions per block, R = slots / (diag_block * tokens * heads) trailing copies.  token_inner = 1
+    puts a token's heads side by side; token_inner = T keeps T consecutive tokens innermost, as the projections' token-shard
+    layout does.  Pure index arithmetic."""
+    E, Tk, H, Ti = diag_block, tokens, heads, token_inner
+    assert slots % (E * Tk * H) == 0 and Tk % E == 0 and E % Ti == 0 and Tk % Ti == 0
     R = slots // (E * Tk * H)
     s = np.arange(slots) // R
-    return s // (Tk * H), (s // H) % Tk, s % H
+    t = s % Ti; s = s // Ti
+    h = s % H; s = s // H
+    P = Tk // Ti
+    return s // P, (s % P) * Ti + t, h
 
 
-def pack_attention_operands(Q: np.ndarray, K: np.ndarray, V: np.ndarray, diag_block: int, slots: int):
+def pack_attention_operands(Q: np.ndarray, K: np.ndarray, V: np.ndarray, diag_block: int, slots: int, token_inner: int = 1):
     """Lay Q, K [tokens][heads][dim] and V [tokens][heads][dim_v] out as one slot vector per channel in the attention
     operand layout (slot index as in attention_slot_index): the query operand repeats Q[i, h, d] in every block e, the
     key and value operands hold token (i + e) mod tokens in block e, so that block e of a product lines query i up with
     key i + e.  Returns (Qs [dim][slots], Ks [dim][slots], Vs [dim_v][slots]).  Pure data movement."""
     tokens, heads, _ = Q.shape
-    e, i, h = attention_slot_index(tokens, heads, diag_block, slots)
+    e, i, h = attention_slot_index(tokens, heads, diag_block, slots, token_inner)
     Qs = np.ascontiguousarray(Q[i, h, :].T)
     Ks = np.ascontiguousarray(K[(i + e) % tokens, h, :].T)
     Vs = np.ascontiguousarray(V[(i + e) % tokens, h, :].T)
     return Qs, Ks, Vs
+
+
+def pack_channel_major_shards(X: np.ndarray, tokens_per_shard: int, slots: int) -> np.ndarray:
+    """Lay X [tokens][heads][dim] out as token-shard slot vectors with the features in channel-major order:
+    shard c holds tokens c*T .. c*T+T-1, slot = (d * heads + h) * T + t, which must fill the slots exactly.
+    Returns [tokens / T][slots].  Pure data movement (pack_feature_major with feature index d * heads + h)."""
+    tokens, heads, dim = X.shape
+    assert dim * heads * tokens_per_shard == slots
+    return pack_feature_major(np.ascontiguousarray(X.transpose(0, 2, 1)).reshape(tokens, dim * heads), tokens_per_shard, slots)

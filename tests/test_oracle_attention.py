@@ -13,19 +13,21 @@ from tests.harness import Client, attention_case, params
 def _key_of(desc, n, g):
     """Key token met by slot (e, i) of score group g, from the layout's definition: the key operand holds token i + e in
     block e and is rotated left by g * diag_block token positions of the flattened (e, i) index."""
-    E, Tk = desc.diag_block, desc.tokens
-    e, i, h = inputs.attention_slot_index(Tk, desc.heads, E, n)
-    u = (e * Tk + i + g * E) % (E * Tk)
-    return (u % Tk + u // Tk) % Tk, i, h
+    E, Tk, Ti = desc.diag_block, desc.tokens, desc.token_inner
+    e, i, h = inputs.attention_slot_index(Tk, desc.heads, E, n, Ti)
+    P = Tk // Ti                                       # positions per block, token_inner tokens each
+    u = (e * P + i // Ti + g * (E // Ti)) % (E * P)    # the rotation moves whole positions
+    return ((u % P) * Ti + i % Ti + u // P) % Tk, i, h
 
 
-@pytest.mark.parametrize("tokens,heads,E,n", [(8, 1, 4, 512), (16, 2, 4, 512), (8, 1, 8, 512), (128, 32, 8, 32768), (16, 4, 1, 64)])
-def test_layout_meets_every_key_once_and_rolls_agree(tokens, heads, E, n):
-    desc = AttnDesc(tokens, heads, E)
+@pytest.mark.parametrize("tokens,heads,E,n,Ti", [(8, 1, 4, 512, 1), (16, 2, 4, 512, 1), (8, 1, 8, 512, 1), (128, 32, 8, 32768, 1), (16, 4, 1, 64, 1),
+                                                 (16, 8, 4, 512, 4), (16, 8, 4, 512, 2), (128, 32, 8, 32768, 8)])
+def test_layout_meets_every_key_once_and_rolls_agree(tokens, heads, E, n, Ti):
+    desc = AttnDesc(tokens, heads, E, 1, Ti)
     g0 = inputs.rng(5, tokens)
     Q = g0.integers(1, 50, (tokens, heads, 2)).astype(np.float64)
     K = g0.integers(1, 50, (tokens, heads, 2)).astype(np.float64)
-    Qs, Ks, _ = inputs.pack_attention_operands(Q, K, K, E, n)
+    Qs, Ks, _ = inputs.pack_attention_operands(Q, K, K, E, n, Ti)
     R = n // (E * tokens * heads)
     seen = np.zeros((tokens, heads, tokens), dtype=np.int64)
     for g in range(desc.groups()):
@@ -137,3 +139,79 @@ def test_scores_with_split_groups_hold_the_same_slots(tokens, heads, E, dim, Gb,
     assert np.abs(rows - rows0).max() < 2.0 ** -22
     with pytest.raises(ValueError):
         o.attention_query_rotations(AttnDesc(tokens, heads, E, 3))
+
+
+@pytest.mark.parametrize("tokens,heads,E,Ti,dim,seed", [(16, 8, 4, 4, 3, 91), (16, 8, 4, 2, 2, 92), (16, 8, 4, 1, 2, 93), (32, 16, 1, 1, 2, 94)])
+def test_pack_and_unpack_against_the_clear_layouts(tokens, heads, E, Ti, dim, seed):
+    """Token-shard ciphertexts in channel-major feature order -> attention operands -> back: every operand decrypts to the
+    clear packing of the same tokens (query: every block alike; key: token i + e in block e), the way back to the shards'
+    slots, and the rotation sets are the block moves and token shifts the layout's index arithmetic gives."""
+    P = params(10, 6, 2, 3)
+    o = P.oracle
+    cl = Client(P, seed)
+    desc = AttnDesc(tokens, heads, E, 1, Ti)
+    D = P.n // (heads * Ti)                                  # channels a shard ciphertext holds
+    g0 = inputs.rng(seed, 3)
+    X = g0.uniform(-1.0, 1.0, (tokens, heads, D))
+    shards = inputs.pack_channel_major_shards(X, Ti, P.n)
+    level, scale = 6, 2.0 ** 40
+    cts = np.stack([cl.encrypt_slots(z, scale, level) for z in shards])
+    Qs, Ks, _ = inputs.pack_attention_operands(X[:, :, :dim], X[:, :, :dim], X[:, :, :dim], E, P.n, Ti)
+    B, Pp = heads * Ti, tokens // Ti
+    move, lad = o.attention_pack_rotations(desc, 0, dim)
+    assert move == sorted({(d - c) * B for d in range(dim) for c in range(Pp)} - {0}) and lad == o.attention_rotations(desc)[1]
+    keys = {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in move + lad}
+    q = o.attention_pack(desc, 0, cts, dim, keys)
+    assert q.shape == (dim, 2, level - 1, P.N)
+    for d in range(dim):
+        assert np.abs(cl.decrypt_slots(q[d], scale).real - Qs[d]).max() < 2.0 ** -20
+    move1, dbl, shift = o.attention_pack_rotations(desc, 1, dim)
+    assert move1 == move and dbl == ([-Pp * B] if E > 1 else []) and len(shift) == E and shift[0] == (0, None)
+    more = [r for pair in shift for r in pair if r] + dbl
+    keys.update({o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in more})
+    k = o.attention_pack(desc, 1, cts, dim, keys)
+    assert k.shape == (dim, 2, level - (2 if E > 1 else 1), P.N)
+    for d in range(dim):
+        assert np.abs(cl.decrypt_slots(k[d], scale).real - Ks[d]).max() < 2.0 ** -20
+    # back: the query layout is the attention output's
+    back = o.attention_unpack_rotations(desc, dim)
+    assert back == sorted({(c - d) * B for d in range(dim) for c in range(Pp)} - {0})
+    keys.update({o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in back})
+    Y = o.attention_unpack(desc, q, keys)
+    assert Y.shape == (Pp, 2, level - 2, P.N)
+    keep = np.arange(P.n) < dim * B                           # the channels that were carried along
+    for c in range(Pp):
+        got = cl.decrypt_slots(Y[c], scale).real
+        assert np.abs(got - shards[c] * keep).max() < 2.0 ** -20
+    with pytest.raises(ValueError):
+        o.attention_pack_rotations(AttnDesc(tokens, heads // 2, E, 1, Ti), 0, dim)     # trailing copies: not supported
+
+
+def test_attention_from_packed_shards_is_softmax_attention():
+    """Projection-layout shards of Q, K, V -> operands -> scores, Softmax over the rows, values -> shards again: the decrypted
+    result is the clear pipeline's attention output in the shards' slots."""
+    tokens, heads, E, Ti, dim, seed = 16, 8, 4, 4, 2, 95
+    P = params(10, 16, 4, 4)
+    o = P.oracle
+    cl = Client(P, seed)
+    desc = AttnDesc(tokens, heads, E, 1, Ti)
+    D = P.n // (heads * Ti)
+    c = attention_case(seed, tokens, heads, dim, dim, 1)
+    level, scale = 16, 2.0 ** 50
+    def shards_of(A):
+        full = np.zeros((tokens, heads, D)); full[:, :, :dim] = A
+        return np.stack([cl.encrypt_slots(z, scale, level) for z in inputs.pack_channel_major_shards(full, Ti, P.n)])
+    rots = set(o.attention_rotations(desc)[0] + o.attention_rotations(desc)[1] + o.attention_pack_rotations(desc, 0, dim)[0] + o.attention_unpack_rotations(desc, dim))
+    _, dbl, shift = o.attention_pack_rotations(desc, 1, dim)
+    rots |= set(dbl) | {r for pair in shift for r in pair if r}
+    keys = {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in rots}
+    rlk = cl.relin_key()
+    q = o.attention_pack(desc, 0, shards_of(c["Q"]), dim, keys)[:, :, :level - 2]         # down to the key operands' level
+    k = o.attention_pack(desc, 1, shards_of(c["K"]), dim, keys)
+    v = o.attention_pack(desc, 1, shards_of(c["V"]), dim, keys)
+    out, so = o.attention(desc, np.ascontiguousarray(q), k, v, scale, scale, c["shift"], 1, c["exp_coeffs"], c["rsqrt_coeffs"], rlk, keys)
+    Y = o.attention_unpack(desc, out, keys)
+    want = np.zeros((tokens, heads, D)); want[:, :, :dim] = c["out_clear"]
+    want = inputs.pack_channel_major_shards(want, Ti, P.n)
+    for cc in range(tokens // Ti):
+        assert np.abs(cl.decrypt_slots(Y[cc], so).real - want[cc]).max() < 2.0 ** -18
