@@ -329,10 +329,15 @@ size_t ckks_softmax_workspace_bytes(const ckks_ctx *ctx, const ckks_softmax_desc
  *     over e: slot (e, i, h) of out[d] holds sum over all key tokens of probability x value, in every block e (the query
  *     operand's layout).  out: dim_v descriptors with buffers for P's level - 1.
  *   ckks_attention: the three in a row (scores at level - 1, then the Softmax's levels, then one more).
+ * desc->token_inner = T' > 1 (dividing diag_block) keeps T' consecutive tokens innermost in the slot index,
+ *     slot = ((((e * P + pos) * heads + h) * T' + t) * R + r,   token i = pos * T' + t,   P = tokens / T',
+ * which is the order the projections' token-shard layout has (T' tokens per shard).  Operands are defined as above in terms
+ * of (e, i, h); the four calls are the same for every T' (a group step is diag_block tokens = diag_block * heads * R slots
+ * either way, the ladder steps tokens * heads * R * 2^k).  token_inner 0 or 1: a token's heads side by side.
  * keys must hold the rotations ckks_attention_rotations lists (token rotations first, then the ladder, then, with
  * group_baby > 1, the query operands' right rotations as negative numbers).
  * Errors: ARG, LEVEL, SCALE, NO_KEY, WORKSPACE, UNSUPPORTED (shape rules above), RANGE (a polynomial constant). */
-typedef struct { uint32_t tokens, heads, diag_block, group_baby; } ckks_attn_desc;
+typedef struct { uint32_t tokens, heads, diag_block, group_baby, token_inner; } ckks_attn_desc;
 int32_t ckks_attention_rotations(const ckks_ctx *ctx, const ckks_attn_desc *desc, int64_t *rots, uint32_t cap);
 int32_t ckks_attention_scores(ckks_ctx *ctx, const ckks_attn_desc *desc, const ckks_ct *q, const ckks_ct *k, uint32_t dim,
                               const ckks_evk *rlk, const ckks_evk *keys, uint32_t nkeys, ckks_ct *scores, void *ws, size_t ws_bytes, void *stream);
@@ -348,6 +353,28 @@ int32_t ckks_attention(ckks_ctx *ctx, const ckks_attn_desc *desc, const ckks_sof
                        const ckks_ct *v, uint32_t dim_v, const ckks_evk *rlk, const ckks_evk *keys, uint32_t nkeys, ckks_ct *out,
                        void *ws, size_t ws_bytes, void *stream);
 size_t ckks_attention_workspace_bytes(const ckks_ctx *ctx, const ckks_attn_desc *desc, const ckks_softmax_desc *sm, uint32_t level, uint32_t dim);
+
+/* Conversion between the projections' token-shard layout and the attention operands (Section 6.2 names an adaptation of
+ * the Q/K/V inputs before the attention products and a conversion after them; neither is defined in the text).  Needs
+ * diag_block * tokens * heads = n and token_inner = the shards' tokens per ciphertext.  A shard ciphertext c < P holds, in
+ * slot (d * heads + h) * T' + t, channel d of token c T' + t and head h (the feature-major layout with the features in
+ * channel-major order, which is the caller's choice of the projection's output columns); B = heads * T' slots.
+ *   kind CKKS_ATTN_QUERY:     in: P shards -> out[d], d < dim, at level - 1:
+ *       ladder( rescale( sum_c rot(in[c], (d - c) B) * mask(position c of block 0) ) ): every block e alike.
+ *   kind CKKS_ATTN_KEY_VALUE: in: P shards -> out[d] at level - 2 (level - 1 if diag_block = 1): with k0 the same sum and its
+ *       copy in block 1, rescale( sum_e [ rot(k0, sA_e) * mask(block e, t < T' - b) + rot(k0, sB_e) * mask(block e, t >= T' - b) ] ),
+ *       e = a T' + b, sA_e = a B + b - e P B, sB_e = (a + 1) B + b - T' - e P B: block e holds token i + e.
+ *   kind CKKS_ATTN_TO_SHARDS: in: dim outputs in the query operand's layout -> out[c], c < P, at level - 1:
+ *       rescale( sum_d rot(in[d], (c - d) B) * mask(slots d B .. d B + B - 1) ).
+ * Masks are 0/1 plaintexts encoded at the scale of their level's last prime, so every rescale returns the input's scale;
+ * every rotated ciphertext is bit-identical to ckks_rotate's (all rotations of a ciphertext share one ModUp).  out: host
+ * array of descriptors with buffers for level - 1 limbs.  ckks_attention_pack_rotations lists the rotations a kind needs
+ * (negative = to the right); returns their number.  Errors: ARG, LEVEL (level < 3), SCALE, NO_KEY, WORKSPACE, UNSUPPORTED. */
+enum { CKKS_ATTN_QUERY = 0, CKKS_ATTN_KEY_VALUE = 1, CKKS_ATTN_TO_SHARDS = 2 };
+int32_t ckks_attention_pack_rotations(const ckks_ctx *ctx, const ckks_attn_desc *desc, int32_t kind, uint32_t dim, int64_t *rots, uint32_t cap);
+int32_t ckks_attention_pack(ckks_ctx *ctx, const ckks_attn_desc *desc, int32_t kind, const ckks_ct *in, uint32_t dim, const ckks_evk *keys,
+                            uint32_t nkeys, ckks_ct *out, void *ws, size_t ws_bytes, void *stream);
+size_t ckks_attention_pack_workspace_bytes(const ckks_ctx *ctx, const ckks_attn_desc *desc, int32_t kind, uint32_t level, uint32_t dim);
 
 /* ---- Rot_k (Section 2.1, Rot + KeySwitch) ----------------------------------
  * Plain: apply sigma_g (g = key->galois) to both components, key-switch the

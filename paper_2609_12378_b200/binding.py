@@ -19,6 +19,7 @@ PROJ_LAZY_MODDOWN = 1
 OPT_NTT_FP_SHARE, OPT_CONV_KERNEL, OPT_MAC_KERNEL, OPT_WAIT_CYCLES, OPT_STATIC_SCRATCH_BYTES, OPT_NTT_BULK_STORE = 1, 2, 3, 4, 5, 6
 CONV_FP64, CONV_TENSOR = 0, 1
 MAC_MMA, MAC_MMA_ASYNC, MAC_MMA_SPLIT, MAC_MMA_HALF, MAC_TCGEN05 = 82, 83, 81, 42, 100
+ATTN_QUERY, ATTN_KEY_VALUE, ATTN_TO_SHARDS = 0, 1, 2
 
 EXPORTS = [
     "ckks_context_create", "ckks_context_destroy", "ckks_context_set_option", "ckks_context_get_option", "ckks_status_string",
@@ -27,7 +28,7 @@ EXPORTS = [
     "ckks_encode_range_flag", "ckks_mul_plain_acc", "ckks_add", "ckks_mul_relin", "ckks_rotate",
     "ckks_rotate_hoisted", "ckks_rescale", "ckks_linear_proj", "ckks_linear_proj_workspace_bytes",
     "ckks_linear_proj_rotations", "ckks_kernel_launches", "ckks_device_status", "ckks_rescale_static",
-    "ckks_attention_rotations", "ckks_attention_scores", "ckks_attention_scores_workspace_bytes", "ckks_attention_values",
+    "ckks_attention_pack_rotations", "ckks_attention_pack", "ckks_attention_pack_workspace_bytes", "ckks_attention_rotations", "ckks_attention_scores", "ckks_attention_scores_workspace_bytes", "ckks_attention_values",
     "ckks_attention_values_workspace_bytes", "ckks_softmax_rows", "ckks_softmax_rows_workspace_bytes", "ckks_attention",
     "ckks_attention_workspace_bytes",
     "ckks_ntt_butterfly_probe", "ckks_mul_relin_sum", "ckks_mul_relin_batch", "ckks_rotate_batch", "ckks_rotate_sum", "ckks_softmax", "ckks_softmax_workspace_bytes", "ckks_poly_eval_bsgs", "ckks_poly_eval_bsgs_workspace_bytes", "ckks_mul_const", "ckks_add_const", "ckks_poly_eval", "ckks_poly_eval_tree", "ckks_linear_proj_multi", "ckks_linear_proj_multi_workspace_bytes",
@@ -58,7 +59,7 @@ class CSoftmaxDesc(C.Structure):
 
 
 class CAttnDesc(C.Structure):
-    _fields_ = [("tokens", C.c_uint32), ("heads", C.c_uint32), ("diag_block", C.c_uint32), ("group_baby", C.c_uint32)]
+    _fields_ = [("tokens", C.c_uint32), ("heads", C.c_uint32), ("diag_block", C.c_uint32), ("group_baby", C.c_uint32), ("token_inner", C.c_uint32)]
 
 
 class CProjDesc(C.Structure):
@@ -101,6 +102,9 @@ def load():
         "ckks_softmax": (i32, [vp, C.POINTER(CSoftmaxDesc), C.POINTER(CCt), C.POINTER(CEvk), C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
         "ckks_softmax_workspace_bytes": (sz, [vp, C.POINTER(CSoftmaxDesc), u32]),
         "ckks_attention_rotations": (i32, [vp, C.POINTER(CAttnDesc), C.POINTER(i64), u32]),
+        "ckks_attention_pack_rotations": (i32, [vp, C.POINTER(CAttnDesc), i32, u32, C.POINTER(i64), u32]),
+        "ckks_attention_pack": (i32, [vp, C.POINTER(CAttnDesc), i32, C.POINTER(CCt), u32, C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
+        "ckks_attention_pack_workspace_bytes": (sz, [vp, C.POINTER(CAttnDesc), i32, u32, u32]),
         "ckks_attention_scores": (i32, [vp, C.POINTER(CAttnDesc), C.POINTER(CCt), C.POINTER(CCt), u32, C.POINTER(CEvk), C.POINTER(CEvk), u32,
                                         C.POINTER(CCt), vp, sz, vp]),
         "ckks_attention_scores_workspace_bytes": (sz, [vp, C.POINTER(CAttnDesc), u32, u32]),
@@ -434,6 +438,32 @@ class Context:
         buf = (C.c_int64 * max(n, 1))()
         load().ckks_attention_rotations(self._h, C.byref(d), buf, n)
         return list(buf)[:n]
+
+    def attention_pack_rotations(self, kind: int, dim: int, tokens: int, heads: int, diag_block: int, token_inner: int):
+        d = CAttnDesc(tokens, heads, diag_block, 1, token_inner)
+        n = load().ckks_attention_pack_rotations(self._h, C.byref(d), kind, dim, None, 0)
+        if n < 0:
+            raise CkksError(n)
+        buf = (C.c_int64 * max(n, 1))()
+        load().ckks_attention_pack_rotations(self._h, C.byref(d), kind, dim, buf, n)
+        return list(buf)[:n]
+
+    def attention_pack(self, kind: int, cts, dim: int, keys, tokens: int, heads: int, diag_block: int, token_inner: int, stream=None):
+        """Conversion between token-shard ciphertexts in channel-major feature order and the attention operands: kind
+        ATTN_QUERY / ATTN_KEY_VALUE take the shards to dim operands, ATTN_TO_SHARDS takes dim outputs back to the shards."""
+        d = CAttnDesc(tokens, heads, diag_block, 1, token_inner)
+        level = cts[0].level
+        need = int(load().ckks_attention_pack_workspace_bytes(self._h, C.byref(d), kind, level, dim))
+        if need == 0:
+            raise CkksError(ERR_UNSUPPORTED)
+        ws = self.workspace(need)
+        nout = tokens // max(1, token_inner) if kind == ATTN_TO_SHARDS else dim
+        outs = [self.empty_ct(level - 1) for _ in range(nout)]
+        ia = (CCt * len(cts))(*[_cct(x) for x in cts])
+        oa = (CCt * nout)(*[_cct(x) for x in outs])
+        ra = (CEvk * max(1, len(keys)))(*[CEvk(_dev_u64(x.data).data_ptr(), x.galois) for x in keys])
+        self._check(load().ckks_attention_pack(self._h, C.byref(d), kind, ia, dim, ra, len(keys), oa, ws.data_ptr(), ws.numel(), _stream_ptr(stream)))
+        return [self._cut(o, c) for o, c in zip(outs, oa)]
 
     def attention_scores(self, q, k, rlk: SwitchKey, keys, tokens, heads, diag_block, ws: torch.Tensor = None, stream=None,
                          group_baby: int = 1):

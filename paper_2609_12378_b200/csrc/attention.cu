@@ -20,7 +20,7 @@
 namespace {
 
 struct AttnPlan {
-    uint32_t E, Tk, H, R, G, Gb;
+    uint32_t E, Tk, H, R, G, Gb, Ti;
     std::vector<int64_t> tok, lad, neg;      // rotations in slots (neg: the query operands' right rotations of the split)
 };
 
@@ -38,6 +38,10 @@ int make_attn_plan(const ckks_ctx *c, const ckks_attn_desc *d, AttnPlan &p) {
     if (!pow2(p.Gb) || p.G % p.Gb) return CKKS_ERR_UNSUPPORTED;
     if (p.Gb > 1)
         for (uint32_t g1 = 1; g1 < p.G / p.Gb; g1++) p.neg.push_back(-p.tok[g1 * p.Gb - 1]);
+    // tokens kept innermost in the slot index: the products, rotations and ladders above are the same for every value (a
+    // group step is diag_block tokens = diag_block * heads * R slots either way); only the conversions below use it
+    p.Ti = d->token_inner ? d->token_inner : 1;
+    if (p.E % p.Ti) return CKKS_ERR_UNSUPPORTED;
     return CKKS_OK;
 }
 
@@ -386,4 +390,227 @@ extern "C" int32_t ckks_attention(ckks_ctx *c, const ckks_attn_desc *d, const ck
     if ((rc = ckks_attention_scores(c, d, q, k, dim, rlk, keys, nkeys, S.data(), sw, sw_bytes, stream))) return rc;
     if ((rc = ckks_softmax_rows(c, d, s, S.data(), rlk, keys, nkeys, P.data(), sw, sw_bytes, stream))) return rc;
     return ckks_attention_values(c, d, P.data(), v, dim_v, rlk, keys, nkeys, out, sw, sw_bytes, stream);
+}
+
+// ---- conversion between the projections' token-shard layout and the attention operands ---------------------------------
+// Shard ciphertext c (c < P = tokens / token_inner) holds, in slot (d * heads + h) * token_inner + t, channel d of token
+// c * token_inner + t and head h (the feature-major layout with the features in channel-major order).  The operands keep
+// token_inner tokens innermost:  slot = ((e * P + pos) * heads + h) * token_inner + t,  so that a channel's share of a
+// shard (B = heads * token_inner slots) moves as one block:
+//   gathered[d] = rescale( sum_c rotate(in[c], (d - c) B) * mask(position c of block 0) )
+//   query:      q[d] = ladder(gathered[d])                               (every block alike)
+//   key, value: k0 = gathered[d] + rotate(gathered[d], -P B);  k[d] = rescale( sum_e [ rotate(k0, sA_e) * mask(block e,
+//               t < token_inner - b) + rotate(k0, sB_e) * mask(block e, t >= token_inner - b) ] ),  e = a token_inner + b,
+//               sA_e = a B + b - e P B,  sB_e = (a + 1) B + b - token_inner - e P B  (the token of the next position)
+//   back:       out[c] = rescale( sum_d rotate(o[d], (c - d) B) * mask(slots d B .. d B + B - 1) )
+// Masks are encoded at the scale of their level's last prime, so every rescale returns the input's scale.  All rotations
+// of a ciphertext run off one ModUp (ckks_rotate_hoisted).  Needs diag_block * tokens * heads = n (no trailing copies).
+namespace {
+
+struct PackPlan {
+    uint32_t E, P, B, Ti;
+    std::vector<int64_t> move, dbl, shA, shB;       // shB[e] = 0 where block e needs no second part (sA of block 0 is 0 too)
+};
+
+int make_pack_plan(const ckks_ctx *c, const ckks_attn_desc *d, uint32_t dim, bool back, AttnPlan &ap, PackPlan &p) {
+    int rc = make_attn_plan(c, d, ap);
+    if (rc) return rc;
+    if (ap.R != 1 || !dim) return CKKS_ERR_UNSUPPORTED;
+    p.E = ap.E; p.Ti = ap.Ti; p.P = ap.Tk / ap.Ti; p.B = ap.H * ap.Ti;
+    if ((uint64_t)dim * p.B > c->n) return CKKS_ERR_UNSUPPORTED;
+    std::vector<int64_t> mv;
+    for (uint32_t dd = 0; dd < dim; dd++)
+        for (uint32_t cc = 0; cc < p.P; cc++)
+            if (dd != cc) mv.push_back(((int64_t)dd - (int64_t)cc) * p.B * (back ? -1 : 1));
+    std::sort(mv.begin(), mv.end());
+    mv.erase(std::unique(mv.begin(), mv.end()), mv.end());
+    p.move = mv;
+    if (p.E > 1) p.dbl.push_back(-(int64_t)p.P * p.B);
+    for (uint32_t e = 0; e < p.E; e++) {
+        const int64_t a = e / p.Ti, b = e % p.Ti, back_e = (int64_t)e * p.P * p.B;
+        p.shA.push_back(a * p.B + b - back_e);
+        p.shB.push_back(b ? (a + 1) * p.B + b - p.Ti - back_e : 0);
+    }
+    return CKKS_OK;
+}
+
+int list_rots(const std::vector<int64_t> &v, int64_t *rots, uint32_t cap, uint32_t &k) {
+    for (int64_t r : v) { if (r) { if (rots && k < cap) rots[k] = r; k++; } }
+    return 0;
+}
+
+size_t pt_bytes(const ckks_ctx *c, uint32_t level) { return align256((size_t)level * c->N * sizeof(uint64_t)); }
+size_t mask_scratch(const ckks_ctx *c, uint32_t level) {
+    return align256((size_t)c->n * sizeof(double)) + align256(ckks_workspace_bytes(c, CKKS_OP_ENCODE, level, 1));
+}
+
+// pt = encode(mask) at `level` with the scale of that level's last prime; scratch: mask_scratch bytes
+int encode_mask(ckks_ctx *c, uint32_t level, uint32_t B, uint32_t lo, uint32_t hi, uint32_t Ti, uint32_t t0, uint32_t t1, ckks_pt *pt, void *scratch,
+                void *stream) {
+    double *slots = (double *)scratch;
+    void *ew = (char *)scratch + align256((size_t)c->n * sizeof(double));
+    {
+        int prev = 0;
+        cudaGetDevice(&prev);
+        cudaSetDevice(c->device);
+        launch_slot_mask(c, slots, B, lo, hi, Ti, t0, t1, (cudaStream_t)stream);
+        cudaSetDevice(prev);
+    }
+    pt->level = level;
+    pt->scale = (double)c->mod[level - 1];
+    return ckks_encode(c, slots, nullptr, 1, pt->scale, level, pt->data, ew, ckks_workspace_bytes(c, CKKS_OP_ENCODE, level, 1), stream);
+}
+
+// outs[x] = rotate(in, rots[x]) for the non-zero rotations, in chunks of 16 off one ModUp each; outs[x] = in's descriptor for a zero rotation
+int rotate_many(ckks_ctx *c, const ckks_ct *in, const std::vector<int64_t> &rots, const ckks_evk *keys, uint32_t nkeys, ckks_ct *outs, void *sw,
+                size_t sw_bytes, void *stream) {
+    std::vector<ckks_evk> ks;
+    std::vector<ckks_ct> os;
+    for (size_t x = 0; x < rots.size(); x++) {
+        if (rots[x] % (int64_t)c->n == 0) { outs[x] = *in; continue; }
+        ks.push_back(*find_key(c, keys, nkeys, rots[x]));
+        os.push_back(outs[x]);
+    }
+    if (ks.empty()) return CKKS_OK;
+    int rc = ckks_rotate_hoisted(c, in, ks.data(), (uint32_t)ks.size(), os.data(), sw, sw_bytes, stream);
+    if (rc) return rc;
+    size_t y = 0;
+    for (size_t x = 0; x < rots.size(); x++)
+        if (rots[x] % (int64_t)c->n != 0) outs[x] = os[y++];
+    return CKKS_OK;
+}
+
+bool have_keys(const ckks_ctx *c, const std::vector<int64_t> &v, const ckks_evk *keys, uint32_t nkeys) {
+    for (int64_t r : v)
+        if (r % (int64_t)c->n != 0 && (!keys || !find_key(c, keys, nkeys, r))) return false;
+    return true;
+}
+
+struct PackWs { size_t rot, acc, gat, pts, mask, sw, sw_bytes, bytes; uint32_t nrot; };
+
+// kind 0 / 1: pack; kind 2: back
+PackWs pack_layout(const ckks_ctx *c, const PackPlan &p, int kind, uint32_t level, uint32_t dim) {
+    PackWs w;
+    const uint32_t fan = kind == 2 ? p.P : dim;                 // rotated copies and accumulators of the first step
+    w.nrot = std::max<uint32_t>(fan, 2 * p.E);
+    size_t off = 0;
+    w.rot = off;  off += (size_t)w.nrot * ct_bytes(c, level);
+    w.acc = off;  off += (size_t)fan * ct_bytes(c, level);
+    w.gat = off;  off += kind == 1 ? (size_t)dim * ct_bytes(c, level - 1) + 2 * ct_bytes(c, level - 1) : 0;     // gathered[d], k0, a sum
+    w.pts = off;  off += (size_t)(kind == 1 ? 2 * p.E : 1) * pt_bytes(c, level);
+    w.mask = off; off += mask_scratch(c, level);
+    w.sw = off;
+    w.sw_bytes = align256(std::max({ckks_workspace_bytes(c, CKKS_OP_ROTATE_HOISTED, level, 16), ckks_workspace_bytes(c, CKKS_OP_RESCALE, level, 0),
+                                    ckks_workspace_bytes(c, CKKS_OP_ROTATE, level, 0), ckks_workspace_bytes(c, CKKS_OP_ROTATE_BATCH, level, 16)}));
+    w.bytes = off + w.sw_bytes;
+    return w;
+}
+
+}  // namespace
+
+extern "C" int32_t ckks_attention_pack_rotations(const ckks_ctx *c, const ckks_attn_desc *d, int32_t kind, uint32_t dim, int64_t *rots, uint32_t cap) {
+    if (!c || kind < 0 || kind > 2) return CKKS_ERR_ARG;
+    AttnPlan ap;
+    PackPlan p;
+    int rc = make_pack_plan(c, d, dim, kind == 2, ap, p);
+    if (rc) return rc;
+    uint32_t k = 0;
+    list_rots(p.move, rots, cap, k);
+    if (kind == 0) list_rots(ap.lad, rots, cap, k);
+    if (kind == 1) { list_rots(p.dbl, rots, cap, k); list_rots(p.shA, rots, cap, k); list_rots(p.shB, rots, cap, k); }
+    return (int32_t)k;
+}
+
+extern "C" size_t ckks_attention_pack_workspace_bytes(const ckks_ctx *c, const ckks_attn_desc *d, int32_t kind, uint32_t level, uint32_t dim) {
+    AttnPlan ap;
+    PackPlan p;
+    if (!c || kind < 0 || kind > 2 || level < 3 || level > c->L || make_pack_plan(c, d, dim, kind == 2, ap, p)) return 0;
+    return pack_layout(c, p, kind, level, dim).bytes;
+}
+
+extern "C" int32_t ckks_attention_pack(ckks_ctx *c, const ckks_attn_desc *d, int32_t kind, const ckks_ct *in, uint32_t dim, const ckks_evk *keys,
+                                       uint32_t nkeys, ckks_ct *out, void *ws, size_t ws_bytes, void *stream) {
+    if (!c || !out || kind < 0 || kind > 2) return CKKS_ERR_ARG;
+    AttnPlan ap;
+    PackPlan p;
+    int rc = make_pack_plan(c, d, dim, kind == 2, ap, p);
+    if (rc) return rc;
+    const uint32_t nin = kind == 2 ? dim : p.P, nout = kind == 2 ? p.P : dim;
+    uint32_t level;
+    if ((rc = check_cts(c, in, nin, &level, true))) return rc;
+    if (level < 3) return CKKS_ERR_LEVEL;
+    for (uint32_t x = 0; x < nout; x++)
+        if (!out[x].data) return CKKS_ERR_ARG;
+    if (!have_keys(c, p.move, keys, nkeys)) return CKKS_ERR_NO_KEY;
+    if (kind == 0 && !have_keys(c, ap.lad, keys, nkeys)) return CKKS_ERR_NO_KEY;
+    if (kind == 1 && (!have_keys(c, p.dbl, keys, nkeys) || !have_keys(c, p.shA, keys, nkeys) || !have_keys(c, p.shB, keys, nkeys))) return CKKS_ERR_NO_KEY;
+    const PackWs L = pack_layout(c, p, kind, level, dim);
+    if (!ws || ws_bytes < L.bytes) return CKKS_ERR_WORKSPACE;
+    char *base = (char *)ws;
+    const size_t ctb = ct_bytes(c, level), ctb1 = ct_bytes(c, level - 1);
+    void *sw = base + L.sw;
+    const uint32_t fan = nout;
+    std::vector<ckks_ct> rot(L.nrot), acc(fan);
+    for (uint32_t x = 0; x < L.nrot; x++) rot[x] = ckks_ct{(uint64_t *)(base + L.rot + (size_t)x * ctb), level, 2, 0.0};
+    for (uint32_t x = 0; x < fan; x++) acc[x] = ckks_ct{(uint64_t *)(base + L.acc + (size_t)x * ctb), level, 2, 0.0};
+    ckks_pt pt{(uint64_t *)(base + L.pts), level, 0.0};
+    // first step, the same in both directions: every input is rotated to its `fan` targets and added in under the mask of
+    // its own place (pack: position c of block 0; back: the channel's slots)
+    std::vector<int64_t> rr(fan);
+    std::vector<ckks_ct> ro(fan);
+    for (uint32_t x = 0; x < nin; x++) {
+        for (uint32_t y = 0; y < fan; y++) {
+            rr[y] = kind == 2 ? ((int64_t)y - (int64_t)x) * p.B : ((int64_t)y - (int64_t)x) * p.B;      // target y, source x
+            ro[y] = rot[y];
+        }
+        if ((rc = rotate_many(c, &in[x], rr, keys, nkeys, ro.data(), sw, L.sw_bytes, stream))) return rc;
+        if ((rc = encode_mask(c, level, p.B, x, x + 1, p.Ti, 0, p.Ti, &pt, base + L.mask, stream))) return rc;
+        if ((rc = ckks_mul_plain_acc(c, ro.data(), fan, &pt, acc.data(), x == 0, stream))) return rc;
+    }
+    if (kind != 1 || p.E == 1) {
+        for (uint32_t y = 0; y < fan; y++)
+            if ((rc = ckks_rescale(c, &acc[y], &out[y], sw, L.sw_bytes, stream))) return rc;
+        if (kind != 0) return CKKS_OK;
+        // query: the ladder over the blocks, 16 channels at a time
+        std::vector<ckks_ct> tmp(16);
+        for (uint32_t d0 = 0; d0 < dim; d0 += 16) {
+            const uint32_t nd = std::min<uint32_t>(16, dim - d0);
+            for (int64_t r : ap.lad) {
+                for (uint32_t x = 0; x < nd; x++) tmp[x] = ckks_ct{(uint64_t *)(base + L.rot + (size_t)x * ctb), level - 1, 2, 0.0};
+                if ((rc = ckks_rotate_batch(c, &out[d0], nd, find_key(c, keys, nkeys, r), tmp.data(), sw, L.sw_bytes, stream))) return rc;
+                for (uint32_t x = 0; x < nd; x++)
+                    if ((rc = ckks_add(c, &out[d0 + x], &tmp[x], &out[d0 + x], stream))) return rc;
+            }
+        }
+        return CKKS_OK;
+    }
+    // key, value: the token shifts, one level down
+    const uint32_t l1 = level - 1;
+    std::vector<ckks_pt> mA(p.E), mB(p.E);
+    for (uint32_t e = 0; e < p.E; e++) {
+        const uint32_t b = e % p.Ti;
+        mA[e] = ckks_pt{(uint64_t *)(base + L.pts + (size_t)(2 * e) * pt_bytes(c, level)), l1, 0.0};
+        mB[e] = ckks_pt{(uint64_t *)(base + L.pts + (size_t)(2 * e + 1) * pt_bytes(c, level)), l1, 0.0};
+        if ((rc = encode_mask(c, l1, p.B, e * p.P, (e + 1) * p.P, p.Ti, 0, p.Ti - b, &mA[e], base + L.mask, stream))) return rc;
+        if (b && (rc = encode_mask(c, l1, p.B, e * p.P, (e + 1) * p.P, p.Ti, p.Ti - b, p.Ti, &mB[e], base + L.mask, stream))) return rc;
+    }
+    ckks_ct k0{(uint64_t *)(base + L.gat + (size_t)dim * ctb1), l1, 2, 0.0}, sum{(uint64_t *)(base + L.gat + (size_t)(dim + 1) * ctb1), l1, 2, 0.0};
+    std::vector<int64_t> sr;
+    for (uint32_t e = 0; e < p.E; e++) { sr.push_back(p.shA[e]); if (e % p.Ti) sr.push_back(p.shB[e]); }
+    std::vector<ckks_ct> so(sr.size());
+    for (uint32_t dd = 0; dd < dim; dd++) {
+        ckks_ct g{(uint64_t *)(base + L.gat + (size_t)dd * ctb1), l1, 2, 0.0};
+        if ((rc = ckks_rescale(c, &acc[dd], &g, sw, L.sw_bytes, stream))) return rc;
+        if ((rc = ckks_rotate(c, &g, find_key(c, keys, nkeys, p.dbl[0]), &k0, sw, L.sw_bytes, stream))) return rc;
+        if ((rc = ckks_add(c, &g, &k0, &k0, stream))) return rc;
+        for (size_t x = 0; x < sr.size(); x++) so[x] = ckks_ct{(uint64_t *)(base + L.rot + x * ctb), l1, 2, 0.0};
+        if ((rc = rotate_many(c, &k0, sr, keys, nkeys, so.data(), sw, L.sw_bytes, stream))) return rc;
+        size_t x = 0;
+        for (uint32_t e = 0; e < p.E; e++) {
+            if ((rc = ckks_mul_plain_acc(c, &so[x++], 1, &mA[e], &sum, e == 0, stream))) return rc;
+            if (e % p.Ti && (rc = ckks_mul_plain_acc(c, &so[x++], 1, &mB[e], &sum, 0, stream))) return rc;
+        }
+        if ((rc = ckks_rescale(c, &sum, &out[dd], sw, L.sw_bytes, stream))) return rc;
+    }
+    return CKKS_OK;
 }

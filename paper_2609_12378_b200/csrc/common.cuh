@@ -268,6 +268,8 @@ void launch_mul_plain_acc(const ckks_ctx *c, const u64 *const *cts, u64 *const *
 void launch_add(const ckks_ctx *c, const u64 *a, const u64 *b, u64 *out, uint32_t ncomp, uint32_t level, cudaStream_t s);
 void launch_automorphism(const ckks_ctx *c, const u64 *in, u64 *out, uint32_t nlimbs, u64 galois, cudaStream_t s);
 void launch_tensor(const ckks_ctx *c, const u64 *a, const u64 *b, u64 *e01, u64 *e2, uint32_t level, cudaStream_t s);
+// slot values 1.0 on the slots x with lo <= x / B < hi and t0 <= x % Ti < t1, else 0.0 (n doubles on the device)
+void launch_slot_mask(const ckks_ctx *c, double *out, uint32_t B, uint32_t lo, uint32_t hi, uint32_t Ti, uint32_t t0, uint32_t t1, cudaStream_t s);
 // out = in * v or in + v (component 0 only) for the constant polynomial v
 void launch_const(const ckks_ctx *c, const u64 *in, long long v, bool mul, u64 *out, uint32_t ncomp, uint32_t level, cudaStream_t s);
 // e01, e2 = sum_i tensor(a_i, b_i) (host arrays of n device pointers, [2][level][N] each)

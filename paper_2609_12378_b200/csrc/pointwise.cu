@@ -119,6 +119,20 @@ __global__ void __launch_bounds__(THREADS) tensor_sum_kernel(DevTables c, Tensor
 
 }  // namespace
 
+// out[x] = 1.0 where lo <= x / B < hi and t0 <= x % Ti < t1, else 0.0 (slot masks of the attention layout's conversions)
+__global__ void __launch_bounds__(THREADS) slot_mask_kernel(double *out, uint32_t n, uint32_t B, uint32_t lo, uint32_t hi, uint32_t Ti, uint32_t t0,
+                                                            uint32_t t1) {
+    const uint32_t x = blockIdx.x * THREADS + threadIdx.x;
+    if (x >= n) return;
+    const uint32_t blk = x / B, t = x % Ti;
+    out[x] = (blk >= lo && blk < hi && t >= t0 && t < t1) ? 1.0 : 0.0;
+}
+
+void launch_slot_mask(const ckks_ctx *c, double *out, uint32_t B, uint32_t lo, uint32_t hi, uint32_t Ti, uint32_t t0, uint32_t t1, cudaStream_t s) {
+    slot_mask_kernel<<<(c->n + THREADS - 1) / THREADS, THREADS, 0, s>>>(out, c->n, B, lo, hi, Ti, t0, t1);
+    count_launches();
+}
+
 void launch_const(const ckks_ctx *c, const u64 *in, long long v, bool mul, u64 *out, uint32_t ncomp, uint32_t level, cudaStream_t s) {
     dim3 grid((c->N / 2 + THREADS - 1) / THREADS, ncomp * level);
     if (mul) const_kernel<true><<<grid, THREADS, 0, s>>>(c->dev, in, v, out, level);

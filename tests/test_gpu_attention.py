@@ -169,3 +169,57 @@ def test_attention_full_ring():
         sl = cl.decrypt_slots(arr, so).real
         assert np.abs(sl - c["out_clear"][i, h, d]).max() < 2.0 ** -14
         assert np.abs(sl - c["out_true"][i, h, d]).max() < 0.05
+
+
+@pytest.mark.parametrize("tokens,heads,E,Ti,dim", [(16, 8, 4, 4, 3), (16, 8, 4, 2, 2), (16, 8, 4, 1, 2), (32, 16, 1, 1, 2)])
+def test_pack_and_unpack_bit_exact(tokens, heads, E, Ti, dim):
+    """Token-shard ciphertexts in channel-major feature order -> query and key operands -> shards again: every limb equals the
+    checker's composition, the rotation lists agree, and the operands decrypt to the clear packings."""
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    P, ctx = params(10, 6, 2, 3), context(10, 6, 2, 3)
+    o = P.oracle
+    cl = Client(P, 800 + tokens + E + Ti)
+    desc = AttnDesc(tokens, heads, E, 1, Ti)
+    D = P.n // (heads * Ti)
+    X = inputs.rng(800 + Ti, 3).uniform(-1.0, 1.0, (tokens, heads, D))
+    shards = inputs.pack_channel_major_shards(X, Ti, P.n)
+    level, scale = 6, 2.0 ** 40
+    cts = np.stack([cl.encrypt_slots(z, scale, level) for z in shards])
+    a = (tokens, heads, E, Ti)
+    move, lad = o.attention_pack_rotations(desc, 0, dim)
+    _, dbl, shift = o.attention_pack_rotations(desc, 1, dim)
+    back = o.attention_unpack_rotations(desc, dim)
+    shifts = [r for pair in shift for r in pair if r]
+    assert set(ctx.attention_pack_rotations(binding.ATTN_QUERY, dim, *a)) == set(move + lad)
+    assert set(ctx.attention_pack_rotations(binding.ATTN_KEY_VALUE, dim, *a)) == set(move + dbl + shifts)
+    assert set(ctx.attention_pack_rotations(binding.ATTN_TO_SHARDS, dim, *a)) == set(back)
+    keys = {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in set(move + lad + dbl + shifts + back)}
+    dkeys = [key_dev(kk, ge) for ge, kk in keys.items()]
+    dcts = [ct_dev(x, scale) for x in cts]
+    Qs, Ks, _ = inputs.pack_attention_operands(X[:, :, :dim], X[:, :, :dim], X[:, :, :dim], E, P.n, Ti)
+    q = o.attention_pack(desc, 0, cts, dim, keys)
+    dq = ctx.attention_pack(binding.ATTN_QUERY, dcts, dim, dkeys, *a)
+    k = o.attention_pack(desc, 1, cts, dim, keys)
+    dk = ctx.attention_pack(binding.ATTN_KEY_VALUE, dcts, dim, dkeys, *a)
+    for d in range(dim):
+        assert dq[d].level == level - 1 and abs(dq[d].scale / scale - 1.0) < 1e-12
+        assert np.array_equal(host(dq[d].data), q[d]), d
+        assert dk[d].level == k.shape[2] and np.array_equal(host(dk[d].data), k[d]), d
+        assert np.abs(cl.decrypt_slots(host(dk[d].data), scale).real - Ks[d]).max() < 2.0 ** -20
+    Y = o.attention_unpack(desc, q, keys)
+    dY = ctx.attention_pack(binding.ATTN_TO_SHARDS, dq, dim, dkeys, *a)
+    assert len(dY) == tokens // Ti
+    for c in range(tokens // Ti):
+        assert np.array_equal(host(dY[c].data), Y[c]), c
+    assert ctx.device_status() == binding.OK
+    launches = binding.kernel_launches()
+    with pytest.raises(binding.CkksError) as err:
+        ctx.attention_pack(binding.ATTN_KEY_VALUE, dcts, dim, dkeys[:1], *a)
+    assert err.value.code == binding.ERR_NO_KEY
+    with pytest.raises(binding.CkksError) as err:
+        ctx.attention_pack(binding.ATTN_QUERY, dcts, dim, dkeys, tokens, heads // 2, E, Ti)        # trailing copies
+    assert err.value.code == binding.ERR_UNSUPPORTED
+    with pytest.raises(binding.CkksError) as err:
+        ctx.attention_pack_rotations(binding.ATTN_QUERY, dim, tokens, heads, E, 3)
+    assert err.value.code == binding.ERR_UNSUPPORTED
+    assert binding.kernel_launches() == launches
