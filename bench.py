@@ -729,6 +729,33 @@ def layer_submetrics(ctx, residues, allp, gen, dev, reps, have_keys):
     att["values"] = timed(lambda: ctx.attention_values(P, v, rlk, akeys, tokens, heads, E))
     att["levels"] = {"operands": LEVEL, "scores": S[0].level, "probabilities": P[0].level, "outputs": P[0].level - 1}
     att["total_s"] = (att["scores"] + att["softmax_rows"] + att["values"]) * 1e-3
+    # the conversions around it: 16 token-shard ciphertexts (8 tokens each, channel-major features) -> 128 query operands,
+    # 128 key (or value) operands, and 128 outputs at the values' level back to 16 shards; timed once each (one call is
+    # 2048 hoisted rotations), with their own rotation keys
+    del S, akeys, k
+    ctx._ws = None
+    torch.cuda.empty_cache()
+    TI = 8
+    shape = (tokens, heads, E, TI)
+    conv = {}
+    for name, kind, level in (("query_operands", binding.ATTN_QUERY, LEVEL), ("key_or_value_operands", binding.ATTN_KEY_VALUE, LEVEL),
+                              ("outputs_to_shards", binding.ATTN_TO_SHARDS, P[0].level - 1)):
+        rots = ctx.attention_pack_rotations(kind, dim, *shape)
+        ckeys = [binding.SwitchKey(residues(allp, DNUM, 2), ctx.galois_element(r)) for r in rots]
+        nin = dim if kind == binding.ATTN_TO_SHARDS else tokens // TI
+        src = [binding.Ciphertext(q[x % dim].data[:, :level].contiguous(), 2.0 ** 40) for x in range(nin)]
+        ctx.attention_pack(kind, src, dim, ckeys, *shape)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); ctx.attention_pack(kind, src, dim, ckeys, *shape); b.record()
+        torch.cuda.synchronize()
+        conv[name] = a.elapsed_time(b)
+        conv[name + "_rotation_keys"] = len(rots)
+        del ckeys, src
+        ctx._ws = None
+        torch.cuda.empty_cache()
+    conv["q_k_v_and_back_s"] = (conv["query_operands"] + 2 * conv["key_or_value_operands"] + conv["outputs_to_shards"]) * 1e-3
+    att["layout_conversions_ms"] = conv
     out["attention_32_heads_128_tokens_dim_128_ms"] = att
     return out
 

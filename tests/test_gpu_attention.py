@@ -223,3 +223,37 @@ def test_pack_and_unpack_bit_exact(tokens, heads, E, Ti, dim):
         ctx.attention_pack_rotations(binding.ATTN_QUERY, dim, tokens, heads, E, 3)
     assert err.value.code == binding.ERR_UNSUPPORTED
     assert binding.kernel_launches() == launches
+
+
+@pytest.mark.slow
+def test_pack_full_ring():
+    """N = 2^16 with the decoder layer's shape (128 tokens in 16 shards of 8, 32 heads, 8 diagonals per ciphertext) and two
+    channels: key operands from the shards bit-exact (block moves, the copy of block 0, fifteen token shifts), and back."""
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    tokens, heads, E, Ti, dim, level = 128, 32, 8, 8, 2, 6
+    P, ctx = params(16, 24, 8, 3), context(16, 24, 8, 3)
+    o = P.oracle
+    cl = Client(P, 880)
+    desc = AttnDesc(tokens, heads, E, 1, Ti)
+    D = P.n // (heads * Ti)
+    X = inputs.rng(881, 3).uniform(-1.0, 1.0, (tokens, heads, D))
+    shards = inputs.pack_channel_major_shards(X, Ti, P.n)
+    scale = 2.0 ** 40
+    cts = np.stack([cl.encrypt_slots(z, scale, level) for z in shards])
+    a = (tokens, heads, E, Ti)
+    rots = set(ctx.attention_pack_rotations(binding.ATTN_KEY_VALUE, dim, *a)) | set(ctx.attention_pack_rotations(binding.ATTN_TO_SHARDS, dim, *a))
+    keys = {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in rots}
+    dkeys = [key_dev(kk, ge) for ge, kk in keys.items()]
+    dcts = [ct_dev(x, scale) for x in cts]
+    k = o.attention_pack(desc, 1, cts, dim, keys)
+    dk = ctx.attention_pack(binding.ATTN_KEY_VALUE, dcts, dim, dkeys, *a)
+    _, Ks, _ = inputs.pack_attention_operands(X[:, :, :dim], X[:, :, :dim], X[:, :, :dim], E, P.n, Ti)
+    for d in range(dim):
+        arr = host(dk[d].data)
+        assert dk[d].level == level - 2 and np.array_equal(arr, k[d]), d
+        assert np.abs(cl.decrypt_slots(arr, scale).real - Ks[d]).max() < 2.0 ** -14
+    Y = o.attention_unpack(desc, k, keys)               # any ciphertexts in the operands' slots serve as input of the way back
+    dY = ctx.attention_pack(binding.ATTN_TO_SHARDS, dk, dim, dkeys, *a)
+    for c in (0, 7, 15):
+        assert np.array_equal(host(dY[c].data), Y[c]), c
+    assert ctx.device_status() == binding.OK
