@@ -550,13 +550,13 @@ class Oracle:
         return (((x // B >= lo) & (x // B < hi) & (x % Ti >= t0) & (x % Ti < t1))).astype(np.float64)
 
     def attention_pack_rotations(self, desc: AttnDesc, kind: int, dim: int):
-        """Rotations (in slots) attention_pack uses.  Block moves (d - c) B for channel d < dim and shard c < P (B = heads *
-        token_inner slots per position); kind 0 (query): the ladder over the blocks; kind 1 (key / value): -P B (a second
+        """Rotations (in slots) attention_pack uses.  Block moves: -c B for shard c < P and d B for channel d < dim (B = heads
+        * token_inner slots per position); kind 0 (query): the ladder over the blocks; kind 1 (key / value): -P B (a second
         copy of block 0) and, per block e with e = a token_inner + b, the token shifts a B + b - e P B (slots with
         t < token_inner - b) and (a + 1) B + b - token_inner - e P B (the others, which take their token from the next
         position)."""
         E, P, B, Ti = self._pack_shape(desc)
-        move = sorted({(d - c) * B for d in range(dim) for c in range(P)} - {0})
+        move = [-c * B for c in range(1, P)] + [d * B for d in range(1, dim)]
         if kind == 0:
             return move, self.attention_rotations(desc)[1]
         shift = []
@@ -565,29 +565,52 @@ class Oracle:
             shift.append((a * B + b - e * P * B, (a + 1) * B + b - Ti - e * P * B if b else None))
         return move, ([-P * B] if E > 1 else []), shift
 
-    def _gather_channels(self, desc: AttnDesc, X, dim: int, keys: dict):
-        """Step shared by both kinds: acc[d] = sum_c rotate(X[c], (d - c) B) * mask(position c of block 0), rescaled: block 0
-        of output d holds channel d of every shard at the shard's position.  X: [P][2][level][N] with slot
-        (d heads + h) token_inner + t = value of token c token_inner + t, head h, channel d.  Returns [dim][2][level-1][N]."""
+    def _move_blocks(self, desc: AttnDesc, X, nout: int, keys: dict):
+        """out[y] = rotate( rescale( sum_x rotate(X[x], -x B) * mask(block x + y) ), y B ),  y < nout: block y of input x ends up
+        as block x of output y (a transpose between the ciphertext index and the block index).  Every input and every
+        output is rotated once; the sums in between are plaintext multiplications by 0/1 masks (encoded at the scale of the
+        level's last prime) and additions.  Blocks are counted cyclically over the n / B blocks of a ciphertext."""
         E, P, B, Ti = self._pack_shape(desc)
-        X = _u64(X); level = X.shape[2]
+        X = _u64(X); nin, level = X.shape[0], X.shape[2]
         pt_scale = float(self.q[level - 1])
-        acc = [None] * dim
-        for c in range(P):
-            mask = self.encode(self._slot_mask(B, c, c + 1, Ti, 0, Ti), pt_scale, level)
-            for d in range(dim):
-                r = (d - c) * B
-                if r:
-                    ge = self.galois_element(r)
-                    xr = self.rotate(X[c], keys[ge], ge)
-                else:
-                    xr = X[c]
-                acc[d] = self.mul_plain_acc(xr, mask, acc[d])
-        return np.stack([self.rescale(a) for a in acc])
+        nblk = self.n // B
+        Xp = []
+        for x in range(nin):
+            if x:
+                ge = self.galois_element(-x * B)
+                Xp.append(self.rotate(X[x], keys[ge], ge))
+            else:
+                Xp.append(X[0])
+        acc = [None] * nout
+        for j in range(min(nin + nout - 1, nblk)):
+            mask = None
+            for x in range(nin):
+                for y in range(nout):
+                    if (x + y) % nblk != j:
+                        continue
+                    if mask is None:
+                        mask = self.encode(self._slot_mask(B, j, j + 1, Ti, 0, Ti), pt_scale, level)
+                    acc[y] = self.mul_plain_acc(Xp[x], mask, acc[y])
+        out = []
+        for y in range(nout):
+            w = self.rescale(acc[y])
+            if y:
+                ge = self.galois_element(y * B)
+                w = self.rotate(w, keys[ge], ge)
+            out.append(w)
+        return np.stack(out)
+
+    def _gather_channels(self, desc: AttnDesc, X, dim: int, keys: dict):
+        """gathered[d], d < dim: block 0 holds channel d of every shard at the shard's position (position c = shard c).
+        X: [P][2][level][N] with slot (d heads + h) token_inner + t = value of token c token_inner + t, head h, channel d.
+        Returns [dim][2][level-1][N]."""
+        return self._move_blocks(desc, X, dim, keys)
 
     def attention_pack(self, desc: AttnDesc, kind: int, X, dim: int, keys: dict):
         """Attention operands from token-shard ciphertexts in channel-major feature order (the projections' layout with
         token_inner tokens per shard): X [P][2][level][N], slot (d heads + h) token_inner + t.
+        gathered[d] = rotate( rescale( sum_c rotate(X[c], -c B) * mask(block c + d) ), d B ) (_move_blocks): position c of block
+        0 holds channel d of shard c.
           kind 0 (query):  q[d] = ladder(gathered[d]): channel d of every token in every block e.  Level - 1.
           kind 1 (key, value): k0 = gathered[d]; k0 = k0 + rotate(k0, -P B) (blocks 0 and 1 hold the tokens); then
             k[d] = rescale( sum_e [ rotate(k0, sA_e) * mask(block e, t < token_inner - b) + rotate(k0, sB_e) * mask(block e,
@@ -625,30 +648,17 @@ class Oracle:
         return np.stack(out)
 
     def attention_unpack_rotations(self, desc: AttnDesc, dim: int):
-        """Block moves (c - d) B of attention_unpack, c < P shards, d < dim channels."""
+        """Block moves of attention_unpack: -d B for channel d < dim, c B for shard c < P."""
         E, P, B, Ti = self._pack_shape(desc)
-        return sorted({(c - d) * B for d in range(dim) for c in range(P)} - {0})
+        return [-d * B for d in range(1, dim)] + [c * B for c in range(1, P)]
 
     def attention_unpack(self, desc: AttnDesc, O, keys: dict):
         """Token-shard ciphertexts in channel-major feature order from attention outputs in the query operand's layout
-        (O [dim][2][level][N], every block e alike):  X[c] = rescale( sum_d rotate(O[d], (c - d) B) * mask(slots d B .. d B + B - 1) ):
-        slot (d heads + h) token_inner + t of X[c] holds channel d of token c token_inner + t, head h.  Returns
-        [P][2][level-1][N]."""
+        (O [dim][2][level][N], every block e alike): the same transpose between ciphertext index and block index the other
+        way, X[c] = rotate( rescale( sum_d rotate(O[d], -d B) * mask(block c + d) ), c B ): slot (d heads + h) token_inner + t
+        of X[c] holds channel d of token c token_inner + t, head h.  Returns [P][2][level-1][N]."""
         E, P, B, Ti = self._pack_shape(desc)
-        O = _u64(O); dim, level = O.shape[0], O.shape[2]
-        pt_scale = float(self.q[level - 1])
-        acc = [None] * P
-        for d in range(dim):
-            mask = self.encode(self._slot_mask(B, d, d + 1, Ti, 0, Ti), pt_scale, level)
-            for c in range(P):
-                r = (c - d) * B
-                if r:
-                    ge = self.galois_element(r)
-                    orr = self.rotate(O[d], keys[ge], ge)
-                else:
-                    orr = O[d]
-                acc[c] = self.mul_plain_acc(orr, mask, acc[c])
-        return np.stack([self.rescale(a) for a in acc])
+        return self._move_blocks(desc, O, P, keys)
 
     def automorphism_coeff(self, a, g: int, t: int):
         a = _u64(a); out = np.empty_like(a)
