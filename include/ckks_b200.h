@@ -359,15 +359,16 @@ size_t ckks_attention_workspace_bytes(const ckks_ctx *ctx, const ckks_attn_desc 
  * diag_block * tokens * heads = n and token_inner = the shards' tokens per ciphertext.  A shard ciphertext c < P holds, in
  * slot (d * heads + h) * T' + t, channel d of token c T' + t and head h (the feature-major layout with the features in
  * channel-major order, which is the caller's choice of the projection's output columns); B = heads * T' slots.
- *   kind CKKS_ATTN_QUERY:     in: P shards -> out[d], d < dim, at level - 1:
- *       ladder( rescale( sum_c rot(in[c], (d - c) B) * mask(position c of block 0) ) ): every block e alike.
- *   kind CKKS_ATTN_KEY_VALUE: in: P shards -> out[d] at level - 2 (level - 1 if diag_block = 1): with k0 the same sum and its
+ *   Both directions start with a transpose between the ciphertext index and the block index:
+ *       moved[y] = rot( rescale( sum_x rot(in[x], -x B) * mask(block x + y) ), y B ),
+ *   one rotation per input and per output ciphertext, blocks counted cyclically over the n / B blocks.
+ *   kind CKKS_ATTN_QUERY:     in: P shards -> out[d], d < dim, at level - 1: ladder(moved[d]): every block e alike.
+ *   kind CKKS_ATTN_KEY_VALUE: in: P shards -> out[d] at level - 2 (level - 1 if diag_block = 1): with k0 = moved[d] and its
  *       copy in block 1, rescale( sum_e [ rot(k0, sA_e) * mask(block e, t < T' - b) + rot(k0, sB_e) * mask(block e, t >= T' - b) ] ),
  *       e = a T' + b, sA_e = a B + b - e P B, sB_e = (a + 1) B + b - T' - e P B: block e holds token i + e.
- *   kind CKKS_ATTN_TO_SHARDS: in: dim outputs in the query operand's layout -> out[c], c < P, at level - 1:
- *       rescale( sum_d rot(in[d], (c - d) B) * mask(slots d B .. d B + B - 1) ).
+ *   kind CKKS_ATTN_TO_SHARDS: in: dim outputs in the query operand's layout -> out[c] = moved[c], c < P, at level - 1.
  * Masks are 0/1 plaintexts encoded at the scale of their level's last prime, so every rescale returns the input's scale;
- * every rotated ciphertext is bit-identical to ckks_rotate's (all rotations of a ciphertext share one ModUp).  out: host
+ * every rotated ciphertext is bit-identical to ckks_rotate's (the token shifts of an operand share one ModUp).  out: host
  * array of descriptors with buffers for level - 1 limbs.  ckks_attention_pack_rotations lists the rotations a kind needs
  * (negative = to the right); returns their number.  Errors: ARG, LEVEL (level < 3), SCALE, NO_KEY, WORKSPACE, UNSUPPORTED. */
 enum { CKKS_ATTN_QUERY = 0, CKKS_ATTN_KEY_VALUE = 1, CKKS_ATTN_TO_SHARDS = 2 };

@@ -397,13 +397,13 @@ extern "C" int32_t ckks_attention(ckks_ctx *c, const ckks_attn_desc *d, const ck
 // c * token_inner + t and head h (the feature-major layout with the features in channel-major order).  The operands keep
 // token_inner tokens innermost:  slot = ((e * P + pos) * heads + h) * token_inner + t,  so that a channel's share of a
 // shard (B = heads * token_inner slots) moves as one block:
-//   gathered[d] = rescale( sum_c rotate(in[c], (d - c) B) * mask(position c of block 0) )
+//   gathered[d] = rotate( rescale( sum_c rotate(in[c], -c B) * mask(block c + d) ), d B )     (one rotation per input and output)
 //   query:      q[d] = ladder(gathered[d])                               (every block alike)
 //   key, value: k0 = gathered[d] + rotate(gathered[d], -P B);  k[d] = rescale( sum_e [ rotate(k0, sA_e) * mask(block e,
 //               t < token_inner - b) + rotate(k0, sB_e) * mask(block e, t >= token_inner - b) ] ),  e = a token_inner + b,
 //               sA_e = a B + b - e P B,  sB_e = (a + 1) B + b - token_inner - e P B  (the token of the next position)
-//   back:       out[c] = rescale( sum_d rotate(o[d], (c - d) B) * mask(slots d B .. d B + B - 1) )
-// Masks are encoded at the scale of their level's last prime, so every rescale returns the input's scale.  All rotations
+//   back:       out[c] = rotate( rescale( sum_d rotate(o[d], -d B) * mask(block c + d) ), c B )
+// Masks are encoded at the scale of their level's last prime, so every rescale returns the input's scale.  The token shifts
 // of a ciphertext run off one ModUp (ckks_rotate_hoisted).  Needs diag_block * tokens * heads = n (no trailing copies).
 namespace {
 
@@ -418,13 +418,10 @@ int make_pack_plan(const ckks_ctx *c, const ckks_attn_desc *d, uint32_t dim, boo
     if (ap.R != 1 || !dim) return CKKS_ERR_UNSUPPORTED;
     p.E = ap.E; p.Ti = ap.Ti; p.P = ap.Tk / ap.Ti; p.B = ap.H * ap.Ti;
     if ((uint64_t)dim * p.B > c->n) return CKKS_ERR_UNSUPPORTED;
-    std::vector<int64_t> mv;
-    for (uint32_t dd = 0; dd < dim; dd++)
-        for (uint32_t cc = 0; cc < p.P; cc++)
-            if (dd != cc) mv.push_back(((int64_t)dd - (int64_t)cc) * p.B * (back ? -1 : 1));
-    std::sort(mv.begin(), mv.end());
-    mv.erase(std::unique(mv.begin(), mv.end()), mv.end());
-    p.move = mv;
+    // block moves: every input x is rotated by -x B, every output y by y B (pack: inputs = shards, outputs = channels)
+    const uint32_t nin = back ? dim : p.P, nout = back ? p.P : dim;
+    for (uint32_t x = 1; x < nin; x++) p.move.push_back(-(int64_t)x * p.B);
+    for (uint32_t y = 1; y < nout; y++) p.move.push_back((int64_t)y * p.B);
     if (p.E > 1) p.dbl.push_back(-(int64_t)p.P * p.B);
     for (uint32_t e = 0; e < p.E; e++) {
         const int64_t a = e / p.Ti, b = e % p.Ti, back_e = (int64_t)e * p.P * p.B;
@@ -486,16 +483,17 @@ bool have_keys(const ckks_ctx *c, const std::vector<int64_t> &v, const ckks_evk 
     return true;
 }
 
-struct PackWs { size_t rot, acc, gat, pts, mask, sw, sw_bytes, bytes; uint32_t nrot; };
+struct PackWs { size_t rot, acc, tmp, gat, pts, mask, sw, sw_bytes, bytes; uint32_t nrot; };
 
 // kind 0 / 1: pack; kind 2: back
 PackWs pack_layout(const ckks_ctx *c, const PackPlan &p, int kind, uint32_t level, uint32_t dim) {
     PackWs w;
-    const uint32_t fan = kind == 2 ? p.P : dim;                 // rotated copies and accumulators of the first step
-    w.nrot = std::max<uint32_t>(fan, 2 * p.E);
+    const uint32_t nin = kind == 2 ? dim : p.P, nout = kind == 2 ? p.P : dim;
+    w.nrot = std::max<uint32_t>({nin, 2 * p.E, 16});            // rotated inputs; later the token shifts or a ladder's chunk
     size_t off = 0;
     w.rot = off;  off += (size_t)w.nrot * ct_bytes(c, level);
-    w.acc = off;  off += (size_t)fan * ct_bytes(c, level);
+    w.acc = off;  off += (size_t)nout * ct_bytes(c, level);
+    w.tmp = off;  off += ct_bytes(c, level);
     w.gat = off;  off += kind == 1 ? (size_t)dim * ct_bytes(c, level - 1) + 2 * ct_bytes(c, level - 1) : 0;     // gathered[d], k0, a sum
     w.pts = off;  off += (size_t)(kind == 1 ? 2 * p.E : 1) * pt_bytes(c, level);
     w.mask = off; off += mask_scratch(c, level);
@@ -549,27 +547,49 @@ extern "C" int32_t ckks_attention_pack(ckks_ctx *c, const ckks_attn_desc *d, int
     char *base = (char *)ws;
     const size_t ctb = ct_bytes(c, level), ctb1 = ct_bytes(c, level - 1);
     void *sw = base + L.sw;
-    const uint32_t fan = nout;
-    std::vector<ckks_ct> rot(L.nrot), acc(fan);
-    for (uint32_t x = 0; x < L.nrot; x++) rot[x] = ckks_ct{(uint64_t *)(base + L.rot + (size_t)x * ctb), level, 2, 0.0};
-    for (uint32_t x = 0; x < fan; x++) acc[x] = ckks_ct{(uint64_t *)(base + L.acc + (size_t)x * ctb), level, 2, 0.0};
+    // First step, the same in both directions: a transpose between the ciphertext index and the block index.  Input x is
+    // rotated by -x B (its block y then sits at block x + y), output y collects block x + y of every rotated input under a
+    // 0/1 mask, is rescaled and rotated by y B, so that input x's share lands in block x.  Blocks count cyclically.
+    const uint32_t nblk = c->n / p.B;
+    std::vector<ckks_ct> xp(nin), acc(nout);
+    xp[0] = in[0];
+    for (uint32_t x = 1; x < nin; x++) {
+        xp[x] = ckks_ct{(uint64_t *)(base + L.rot + (size_t)x * ctb), level, 2, 0.0};
+        if ((rc = ckks_rotate(c, &in[x], find_key(c, keys, nkeys, -(int64_t)x * p.B), &xp[x], sw, L.sw_bytes, stream))) return rc;
+    }
     ckks_pt pt{(uint64_t *)(base + L.pts), level, 0.0};
-    // first step, the same in both directions: every input is rotated to its `fan` targets and added in under the mask of
-    // its own place (pack: position c of block 0; back: the channel's slots)
-    std::vector<int64_t> rr(fan);
-    std::vector<ckks_ct> ro(fan);
-    for (uint32_t x = 0; x < nin; x++) {
-        for (uint32_t y = 0; y < fan; y++) {
-            rr[y] = kind == 2 ? ((int64_t)y - (int64_t)x) * p.B : ((int64_t)y - (int64_t)x) * p.B;      // target y, source x
-            ro[y] = rot[y];
+    {
+        int prev = 0;
+        cudaGetDevice(&prev);
+        cudaSetDevice(c->device);
+        cudaMemsetAsync(base + L.acc, 0, (size_t)nout * ctb, (cudaStream_t)stream);
+        cudaSetDevice(prev);
+    }
+    for (uint32_t y = 0; y < nout; y++) acc[y] = ckks_ct{(uint64_t *)(base + L.acc + (size_t)y * ctb), level, 2, in[0].scale * (double)c->mod[level - 1]};
+    std::vector<ckks_ct> mc, ma;
+    for (uint32_t j = 0; j < std::min(nin + nout - 1, nblk); j++) {
+        mc.clear(); ma.clear();
+        for (uint32_t x = 0; x < nin; x++)
+            for (uint32_t y = 0; y < nout; y++)
+                if ((x + y) % nblk == j) { mc.push_back(xp[x]); ma.push_back(acc[y]); }
+        if (mc.empty()) continue;
+        if ((rc = encode_mask(c, level, p.B, j, j + 1, p.Ti, 0, p.Ti, &pt, base + L.mask, stream))) return rc;
+        if ((rc = ckks_mul_plain_acc(c, mc.data(), (uint32_t)mc.size(), &pt, ma.data(), 0, stream))) return rc;
+    }
+    // rescaled and rotated into place: straight to the outputs, or (key, value) to the buffer the token shifts read
+    ckks_ct tmp{(uint64_t *)(base + L.tmp), level - 1, 2, 0.0};
+    std::vector<ckks_ct> moved(nout);
+    for (uint32_t y = 0; y < nout; y++) {
+        moved[y] = (kind == 1 && p.E > 1) ? ckks_ct{(uint64_t *)(base + L.gat + (size_t)y * ctb1), level - 1, 2, 0.0} : out[y];
+        if (y == 0) {
+            if ((rc = ckks_rescale(c, &acc[0], &moved[0], sw, L.sw_bytes, stream))) return rc;
+            continue;
         }
-        if ((rc = rotate_many(c, &in[x], rr, keys, nkeys, ro.data(), sw, L.sw_bytes, stream))) return rc;
-        if ((rc = encode_mask(c, level, p.B, x, x + 1, p.Ti, 0, p.Ti, &pt, base + L.mask, stream))) return rc;
-        if ((rc = ckks_mul_plain_acc(c, ro.data(), fan, &pt, acc.data(), x == 0, stream))) return rc;
+        if ((rc = ckks_rescale(c, &acc[y], &tmp, sw, L.sw_bytes, stream))) return rc;
+        if ((rc = ckks_rotate(c, &tmp, find_key(c, keys, nkeys, (int64_t)y * p.B), &moved[y], sw, L.sw_bytes, stream))) return rc;
     }
     if (kind != 1 || p.E == 1) {
-        for (uint32_t y = 0; y < fan; y++)
-            if ((rc = ckks_rescale(c, &acc[y], &out[y], sw, L.sw_bytes, stream))) return rc;
+        for (uint32_t y = 0; y < nout; y++) out[y] = moved[y];
         if (kind != 0) return CKKS_OK;
         // query: the ladder over the blocks, 16 channels at a time
         std::vector<ckks_ct> tmp(16);
@@ -599,8 +619,7 @@ extern "C" int32_t ckks_attention_pack(ckks_ctx *c, const ckks_attn_desc *d, int
     for (uint32_t e = 0; e < p.E; e++) { sr.push_back(p.shA[e]); if (e % p.Ti) sr.push_back(p.shB[e]); }
     std::vector<ckks_ct> so(sr.size());
     for (uint32_t dd = 0; dd < dim; dd++) {
-        ckks_ct g{(uint64_t *)(base + L.gat + (size_t)dd * ctb1), l1, 2, 0.0};
-        if ((rc = ckks_rescale(c, &acc[dd], &g, sw, L.sw_bytes, stream))) return rc;
+        ckks_ct g = moved[dd];
         if ((rc = ckks_rotate(c, &g, find_key(c, keys, nkeys, p.dbl[0]), &k0, sw, L.sw_bytes, stream))) return rc;
         if ((rc = ckks_add(c, &g, &k0, &k0, stream))) return rc;
         for (size_t x = 0; x < sr.size(); x++) so[x] = ckks_ct{(uint64_t *)(base + L.rot + x * ctb), l1, 2, 0.0};
