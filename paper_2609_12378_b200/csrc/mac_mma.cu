@@ -290,7 +290,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_cp_async(uint32_t bar) {
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(bar) : "memory");
 }
-// Bounded wait, called by all 32 lanes of a warp together; the verdict is the warp's (every lane gets the same answer, so
+// Bounded wait, called by all 32 lanes of a warp together; the answer is the warp's (every lane gets the same one, so
 // a timeout never splits a warp in front of a warp-wide instruction).  limit: SM clock cycles.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long limit) {
     const long long t0 = clock64();

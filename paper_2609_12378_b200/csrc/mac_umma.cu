@@ -72,7 +72,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) { asm volatile("mbarri
 __device__ __forceinline__ void mbar_arrive_cp_async(uint32_t bar) {
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(bar) : "memory");
 }
-// Bounded wait (limit in SM clock cycles).  WARP = true: all 32 lanes call it together and get the warp's common verdict,
+// Bounded wait (limit in SM clock cycles).  WARP = true: all 32 lanes call it together and get the warp's common answer,
 // so a timeout never splits a warp in front of a warp-wide instruction; WARP = false: a single thread waits (the MMA issuer).
 template <bool WARP>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long limit) {

@@ -416,7 +416,7 @@ __device__ __forceinline__ void warp_bulk_load_128(uint32_t bar, void *sdst, con
     asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], 128, [%2];\n"
                  ::"r"((uint32_t)__cvta_generic_to_shared(sdst)), "l"(gsrc), "r"(bar) : "memory");
 }
-// true once the warp's copies have landed; the verdict is the warp's (one vote)
+// true once the warp's copies have landed; the answer is the warp's (one vote)
 __device__ __forceinline__ bool warp_bulk_wait(uint32_t bar, long long limit) {
     const long long t0 = clock64();
     uint32_t ok = 0;
