@@ -151,7 +151,13 @@ def attention_case(seed: int, tokens: int, heads: int, dim: int, dim_v: int, rou
     V = g.uniform(-1.0, 1.0, (tokens, heads, dim_v))
     S = np.einsum("ihd,jhd->hij", Q, K)                       # [heads][query][key]
     Q = Q * (0.5 * spread / np.abs(S).max())                  # scores within +- spread / 2
+    return attention_case_from(Q, K, V, rounds, degree, spread)
+
+
+def attention_case_from(Q, K, V, rounds: int = 1, degree: int = 4, spread: float = 4.0):
+    """The same dict for given Q, K [tokens][heads][dim], V [tokens][heads][dim_v] whose scores lie within +- spread / 2."""
     S = np.einsum("ihd,jhd->hij", Q, K)
+    assert np.abs(S).max() <= 0.5 * spread * (1 + 1e-9)
     shift = 0.5 * spread
 
     def fit(f, lo, hi, deg):

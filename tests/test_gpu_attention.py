@@ -257,3 +257,68 @@ def test_pack_full_ring():
     for c in (0, 7, 15):
         assert np.array_equal(host(dY[c].data), Y[c]), c
     assert ctx.device_status() == binding.OK
+
+
+def test_attention_block_from_projections_to_projection_bit_exact():
+    """The attention block of a decoder layer through the C ABI on a small ring: query/key/value projections in one call
+    (channel-major output columns), operands, scores - Softmax - values, back to shards, output projection.  Every stage's
+    limbs equal the checker's, and the decrypted result is the clear pipeline's attention(X W_q, X W_k, X W_v) W_o."""
+    import torch
+
+    from oracle.ckks_oracle import ProjDesc
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    from tests.test_oracle_attention import layer_attention_case
+    tokens, heads, E, T, seed = 16, 8, 4, 4, 96
+    P, ctx = params(10, 18, 6, 3), context(10, 18, 6, 3)
+    o = P.oracle
+    cl = Client(P, seed)
+    desc = AttnDesc(tokens, heads, E, 1, T)
+    D = P.n // (heads * T)
+    hidden, C_ = heads * D, tokens // T
+    X, W, c, Z = layer_attention_case(seed, tokens, heads, T, P.n)
+    level, scale = 18, 2.0 ** 50
+    pd = ProjDesc(hidden, hidden, T, C_, 8)
+    a = (tokens, heads, E, T)
+    rots = set(ctx.linear_proj_rotations(hidden, hidden, T, C_, 8)) | set(ctx.attention_rotations(tokens, heads, E))
+    for kind in (binding.ATTN_QUERY, binding.ATTN_KEY_VALUE, binding.ATTN_TO_SHARDS):
+        rots |= set(ctx.attention_pack_rotations(kind, D, *a))
+    keys = {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in rots}
+    dkeys = [key_dev(kk, ge) for ge, kk in keys.items()]
+    rlk = cl.relin_key()
+    drlk = key_dev(rlk, 0)
+    x = np.stack([cl.encrypt_slots(z, scale, level) for z in inputs.pack_feature_major(X, T, P.n)])
+    dx = [ct_dev(z, scale) for z in x]
+    dW = {k: torch.tensor(W[k], dtype=torch.float64, device="cuda").contiguous() for k in "qkvo"}
+    # projections
+    dproj = ctx.linear_proj_multi(dx, [dW["q"], dW["k"], dW["v"]], dkeys, hidden, [hidden] * 3, T, C_, 8)
+    proj = {k: o.linear_proj(pd, x, W[k], keys, scale)[0] for k in "qkv"}
+    for i, k in enumerate("qkv"):
+        for cc in range(C_):
+            assert np.array_equal(host(dproj[i][cc].data), proj[k][cc]), (k, cc)
+    # operands
+    q = o.attention_pack(desc, 0, proj["q"], D, keys)
+    kk = o.attention_pack(desc, 1, proj["k"], D, keys)
+    v = o.attention_pack(desc, 1, proj["v"], D, keys)
+    dq = ctx.attention_pack(binding.ATTN_QUERY, dproj[0], D, dkeys, *a)
+    dk = ctx.attention_pack(binding.ATTN_KEY_VALUE, dproj[1], D, dkeys, *a)
+    dv = ctx.attention_pack(binding.ATTN_KEY_VALUE, dproj[2], D, dkeys, *a)
+    for d in range(D):
+        assert np.array_equal(host(dq[d].data), q[d]) and np.array_equal(host(dk[d].data), kk[d]) and np.array_equal(host(dv[d].data), v[d]), d
+    lk = dk[0].level
+    dq = [binding.Ciphertext(z.data[:, :lk].contiguous(), z.scale) for z in dq]          # down to the key operands' level
+    # attention
+    out, so = o.attention(desc, np.ascontiguousarray(q[:, :, :lk]), kk, v, scale, scale, c["shift"], 1, c["exp_coeffs"], c["rsqrt_coeffs"], rlk, keys)
+    dout = ctx.attention(dq, dk, dv, c["shift"], 1, c["exp_coeffs"], c["rsqrt_coeffs"], drlk, dkeys, tokens, heads, E)
+    for d in range(D):
+        assert np.array_equal(host(dout[d].data), out[d]), d
+    # back to shards, output projection
+    Y = o.attention_unpack(desc, out, keys)
+    dY = ctx.attention_pack(binding.ATTN_TO_SHARDS, dout, D, dkeys, *a)
+    z, sz = o.linear_proj(pd, Y, W["o"], keys, so)
+    dz = ctx.linear_proj(dY, dW["o"], dkeys, hidden, hidden, T, C_, 8)
+    assert ctx.device_status() == binding.OK
+    want = inputs.pack_feature_major(Z, T, P.n)
+    for cc in range(C_):
+        arr = host(dz[cc].data)
+        assert np.array_equal(host(dY[cc].data), Y[cc]) and np.array_equal(arr, z[cc]), cc
+        assert np.abs(cl.decrypt_slots(arr, dz[cc].scale).real - want[cc]).max() < 2.0 ** -14

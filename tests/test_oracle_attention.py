@@ -7,7 +7,7 @@ import pytest
 
 from oracle.ckks_oracle import AttnDesc
 from paper_2609_12378_b200 import inputs
-from tests.harness import Client, attention_case, params
+from tests.harness import Client, attention_case, attention_case_from, params
 
 
 def _key_of(desc, n, g):
@@ -215,3 +215,55 @@ def test_attention_from_packed_shards_is_softmax_attention():
     want = inputs.pack_channel_major_shards(want, Ti, P.n)
     for cc in range(tokens // Ti):
         assert np.abs(cl.decrypt_slots(Y[cc], so).real - want[cc]).max() < 2.0 ** -18
+
+
+def layer_attention_case(seed: int, tokens: int, heads: int, T: int, n: int):
+    """Synthetic attention block of a decoder layer in the projections' layout: X [tokens][hidden], W_q, W_k, W_v with their
+    output columns in channel-major order d * heads + h, W_o with its input rows in that order; the clear pipeline's
+    result Z = attention(X W_q, X W_k, X W_v) W_o with the Softmax by doubling of attention_case_from."""
+    D = n // (heads * T)
+    hidden = heads * D
+    g = inputs.rng(seed, 13)
+    X = g.uniform(-1.0, 1.0, (tokens, hidden))
+    W = {k: g.normal(0.0, 1.0 / np.sqrt(hidden), (hidden, hidden)) for k in "qkvo"}
+    split = lambda A: A.reshape(tokens, D, heads).transpose(0, 2, 1)          # [tokens][d * heads + h] -> [tokens][heads][D]
+    S = np.einsum("ihd,jhd->hij", split(X @ W["q"]), split(X @ W["k"]))
+    W["q"] = W["q"] * (1.9 / np.abs(S).max())                                 # scores within +- 2 (the 1/sqrt(dim) of the model)
+    c = attention_case_from(split(X @ W["q"]), split(X @ W["k"]), split(X @ W["v"]), 1)
+    Yf = c["out_clear"].transpose(0, 2, 1).reshape(tokens, hidden)
+    return X, W, c, Yf @ W["o"]
+
+
+def test_attention_block_from_projections_to_projection():
+    """X -> Q, K, V projections (channel-major output columns) -> operands -> scores, Softmax, values -> shards -> output
+    projection, everything in the checker: the decrypted shards hold the clear pipeline's Z = attention(X W_q, X W_k, X W_v) W_o."""
+    from oracle.ckks_oracle import ProjDesc
+    tokens, heads, E, T, seed = 16, 8, 4, 4, 96
+    P = params(10, 18, 6, 3)
+    o = P.oracle
+    cl = Client(P, seed)
+    desc = AttnDesc(tokens, heads, E, 1, T)
+    D = P.n // (heads * T)
+    hidden, C_ = heads * D, tokens // T
+    X, W, c, Z = layer_attention_case(seed, tokens, heads, T, P.n)
+    level, scale = 18, 2.0 ** 50
+    pd = ProjDesc(hidden, hidden, T, C_, 8)
+    rots = set(o.proj_rotations(pd)) | set(sum(o.attention_rotations(desc), [])) | set(o.attention_pack_rotations(desc, 0, D)[0]) | set(o.attention_unpack_rotations(desc, D))
+    _, dbl, shift = o.attention_pack_rotations(desc, 1, D)
+    rots |= set(dbl) | {r for pair in shift for r in pair if r}
+    keys = {o.galois_element(r): cl.rotation_key(o.galois_element(r)) for r in rots}
+    rlk = cl.relin_key()
+    x = np.stack([cl.encrypt_slots(z, scale, level) for z in inputs.pack_feature_major(X, T, P.n)])
+    proj = {k: o.linear_proj(pd, x, W[k], keys, scale) for k in "qkv"}
+    for k in "qkv":
+        assert proj[k][1] == scale
+    q = np.ascontiguousarray(o.attention_pack(desc, 0, proj["q"][0], D, keys)[:, :, :level - 3])
+    kk = o.attention_pack(desc, 1, proj["k"][0], D, keys)
+    v = o.attention_pack(desc, 1, proj["v"][0], D, keys)
+    out, so = o.attention(desc, q, kk, v, scale, scale, c["shift"], 1, c["exp_coeffs"], c["rsqrt_coeffs"], rlk, keys)
+    Y = o.attention_unpack(desc, out, keys)
+    z, sz = o.linear_proj(pd, Y, W["o"], keys, so)
+    assert z.shape[2] == level - 16
+    want = inputs.pack_feature_major(Z, T, P.n)
+    for cc in range(C_):
+        assert np.abs(cl.decrypt_slots(z[cc], sz).real - want[cc]).max() < 2.0 ** -14
