@@ -704,7 +704,15 @@ def layer_submetrics(ctx, residues, allp, gen, dev, reps, have_keys):
     bws = ctx.workspace(ctx.workspace_bytes(binding.OP_MUL_RELIN_BATCH, LEVEL, 128))
     out["ms"]["products_2x2048_each_relinearised"] = timed(lambda: [ctx.mul_relin_batch(pa, pb, rlk, outs=bouts, ws=bws) for _ in range(32)])
     out["layer_linear_and_products_s"] = out["projections_s"] + out["ms"]["products_2x2048_summed_128_per_output"] * 1e-3
-    del bouts, bws, a, b, acc
+    # the element-wise product of the gate and up branches (SiLU's polynomial not included): 4 blocks x 16 shards of
+    # ciphertext pairs at the projections' output level, relinearised in batches of 16
+    g1 = [binding.Ciphertext(a[i % 16].data[:, :LEVEL - 1].contiguous(), 2.0 ** 40) for i in range(16)]
+    g2 = [binding.Ciphertext(b[i % 16].data[:, :LEVEL - 1].contiguous(), 2.0 ** 40) for i in range(16)]
+    ga, gb = [g1[i % 16] for i in range(nib * SHARDS)], [g2[(5 * i + 1) % 16] for i in range(nib * SHARDS)]
+    gouts = [ctx.empty_ct(LEVEL - 1) for _ in range(16)] * (nib * SHARDS // 16)
+    gws = ctx.workspace(ctx.workspace_bytes(binding.OP_MUL_RELIN_BATCH, LEVEL - 1, nib * SHARDS))
+    out["ms"]["gate_times_up_64_products"] = timed(lambda: ctx.mul_relin_batch(ga, gb, rlk, outs=gouts, ws=gws))
+    del bouts, bws, a, b, acc, g1, g2, ga, gb, gouts, gws
     ctx._ws = None
     torch.cuda.empty_cache()
     # the same products inside the attention entry points (diagonal-block layout: 128 tokens, 32 heads, 8 diagonals per
