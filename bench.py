@@ -712,6 +712,12 @@ def layer_submetrics(ctx, residues, allp, gen, dev, reps, have_keys):
     gouts = [ctx.empty_ct(LEVEL - 1) for _ in range(16)] * (nib * SHARDS // 16)
     gws = ctx.workspace(ctx.workspace_bytes(binding.OP_MUL_RELIN_BATCH, LEVEL - 1, nib * SHARDS))
     out["ms"]["gate_times_up_64_products"] = timed(lambda: ctx.mul_relin_batch(ga, gb, rlk, outs=gouts, ws=gws))
+    # a degree-63 polynomial (the size the paper's Table 7 gives SiLU) of one gate ciphertext by baby and giant steps of 8,
+    # synthetic coefficients; a layer evaluates it on all 64 gate ciphertexts
+    pc = [0.5 ** (k // 4) / (1 + k) for k in range(64)]
+    xg = binding.Ciphertext(g1[0].data, 2.0 ** 50)
+    out["ms"]["polynomial_degree_63_one_ciphertext"] = timed(lambda: ctx.poly_eval_bsgs(xg, pc, 8, rlk))
+    del xg
     del bouts, bws, a, b, acc, g1, g2, ga, gb, gouts, gws
     ctx._ws = None
     torch.cuda.empty_cache()
