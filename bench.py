@@ -452,6 +452,24 @@ def run_cuda(args):
         extras["rotate_64_calls_ms"] = once(lambda: [ctx.rotate(x_, rot_keys[0], out=rot_out) for x_ in rin])
         extras["rotate_batch_64_ms"] = once(lambda: ctx.rotate_batch(rin, rot_keys[0], outs=routs, ws=rws))
         del routs, rws
+        # the same 64 independent rotations issued on four streams, a context (tables and scratch) per stream: kernels of
+        # single-ciphertext calls fill the GPU for at most one wave, so independent calls overlap
+        sctx = [ctx] + [binding.Context(LOG_N, q, p, DNUM, device=local) for _ in range(3)]
+        sts = [torch.cuda.Stream() for _ in range(4)]
+        souts = [ctx.empty_ct(LEVEL) for _ in range(4)]
+
+        def on_streams():
+            cur = torch.cuda.current_stream()
+            for s_ in sts:
+                s_.wait_stream(cur)
+            for i_, x_ in enumerate(rin):
+                with torch.cuda.stream(sts[i_ % 4]):
+                    sctx[i_ % 4].rotate(x_, rot_keys[0], out=souts[i_ % 4], stream=sts[i_ % 4])
+            for s_ in sts:
+                cur.wait_stream(s_)
+
+        extras["rotate_64_calls_on_4_streams_ms"] = once(on_streams)
+        del sctx, sts, souts
         # a degree-63 polynomial (the paper's SiLU degree per layer) by the power tree and by baby steps / giant steps
         c63 = [1.0 / (1 + k) for k in range(64)]
         extras["poly_degree63_tree_ms"] = once(lambda: ctx.poly_eval_tree(binding.Ciphertext(cta.data, 2.0 ** 50), c63, rlk))
