@@ -137,10 +137,15 @@ const char *ckks_last_cuda_error(const ckks_ctx *ctx);
  *                           16 results in shared memory and a 128-byte bulk copy writes them out, and in the inverse
  *                           transform's first pass every thread's 16 inputs arrive by a 128-byte bulk copy (a bounded wait
  *                           on an mbarrier, see CKKS_OPT_WAIT_CYCLES); 0 = 32-byte global stores and loads.
+ *   CKKS_OPT_LANES          1..4 (default 4): streams over which the attention entry points spread their independent
+ *                           single-ciphertext chains (per channel, per score group).  Lane 0 is the caller's stream, the
+ *                           others belong to the context; they are forked from and joined to the caller's stream by events
+ *                           inside the call, so the call still behaves as work on the caller's stream.  The workspace sizes
+ *                           of those calls depend on it: set it before asking for them.  Results do not depend on it.
  *   CKKS_OPT_STATIC_SCRATCH_BYTES  (read only) CKKS_STATIC_SCRATCH_BYTES of the loaded library.
  * set returns CKKS_ERR_ARG for an unknown option or a value outside its range; get returns -1 for an unknown option. */
 enum { CKKS_OPT_NTT_FP_SHARE = 1, CKKS_OPT_CONV_KERNEL = 2, CKKS_OPT_MAC_KERNEL = 3, CKKS_OPT_WAIT_CYCLES = 4,
-       CKKS_OPT_STATIC_SCRATCH_BYTES = 5, CKKS_OPT_NTT_BULK_STORE = 6 };
+       CKKS_OPT_STATIC_SCRATCH_BYTES = 5, CKKS_OPT_NTT_BULK_STORE = 6, CKKS_OPT_LANES = 7 };
 enum { CKKS_CONV_FP64 = 0, CKKS_CONV_TENSOR = 1 };
 enum { CKKS_MAC_MMA = 82, CKKS_MAC_MMA_ASYNC = 83, CKKS_MAC_MMA_SPLIT = 81, CKKS_MAC_MMA_HALF = 42, CKKS_MAC_TCGEN05 = 100 };
 int32_t ckks_context_set_option(ckks_ctx *ctx, int32_t option, int64_t value);

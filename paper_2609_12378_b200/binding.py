@@ -16,7 +16,7 @@ OK, ERR_ARG, ERR_LEVEL, ERR_SCALE, ERR_NO_KEY, ERR_WORKSPACE, ERR_RANGE, ERR_UNS
     0, -1, -2, -3, -4, -5, -6, -7, -8, -9)
 OP_ENCODE, OP_MUL_RELIN, OP_ROTATE, OP_ROTATE_HOISTED, OP_RESCALE, OP_LINEAR_PROJ, OP_POLY_EVAL, OP_POLY_EVAL_TREE, OP_MUL_RELIN_BATCH, OP_ROTATE_BATCH, OP_ROTATE_SUM = 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11
 PROJ_LAZY_MODDOWN = 1
-OPT_NTT_FP_SHARE, OPT_CONV_KERNEL, OPT_MAC_KERNEL, OPT_WAIT_CYCLES, OPT_STATIC_SCRATCH_BYTES, OPT_NTT_BULK_STORE = 1, 2, 3, 4, 5, 6
+OPT_NTT_FP_SHARE, OPT_CONV_KERNEL, OPT_MAC_KERNEL, OPT_WAIT_CYCLES, OPT_STATIC_SCRATCH_BYTES, OPT_NTT_BULK_STORE, OPT_LANES = 1, 2, 3, 4, 5, 6, 7
 CONV_FP64, CONV_TENSOR = 0, 1
 MAC_MMA, MAC_MMA_ASYNC, MAC_MMA_SPLIT, MAC_MMA_HALF, MAC_TCGEN05 = 82, 83, 81, 42, 100
 ATTN_QUERY, ATTN_KEY_VALUE, ATTN_TO_SHARDS = 0, 1, 2

@@ -86,6 +86,37 @@ int check_cts(const ckks_ctx *c, const ckks_ct *cts, uint32_t n, uint32_t *level
 
 bool rlk_ok(const ckks_evk *rlk) { return rlk && rlk->data && rlk->galois == 0; }
 
+// The context's streams as lanes for independent chains: lane 0 is the caller's stream.  fork() makes the other lanes wait
+// for what the caller's stream has been given so far, join() makes the caller's stream wait for all of them.
+struct Lanes {
+    ckks_ctx *c;
+    cudaStream_t caller;
+    uint32_t n;
+    Lanes(ckks_ctx *ctx, void *stream) : c(ctx), caller((cudaStream_t)stream), n((uint32_t)std::max(1, std::min(ctx->lanes, 4))) {}
+    void *at(uint32_t i) const { return i % n == 0 ? (void *)caller : (void *)c->lane_stream[i % n - 1]; }
+    void fork() const {
+        if (n == 1) return;
+        int prev = 0;
+        cudaGetDevice(&prev);
+        cudaSetDevice(c->device);
+        cudaEventRecord(c->lane_event[0], caller);
+        for (uint32_t i = 1; i < n; i++) cudaStreamWaitEvent(c->lane_stream[i - 1], c->lane_event[0], 0);
+        cudaSetDevice(prev);
+    }
+    void join() const {
+        if (n == 1) return;
+        int prev = 0;
+        cudaGetDevice(&prev);
+        cudaSetDevice(c->device);
+        for (uint32_t i = 1; i < n; i++) {
+            cudaEventRecord(c->lane_event[i], c->lane_stream[i - 1]);
+            cudaStreamWaitEvent(caller, c->lane_event[i], 0);
+        }
+        cudaSetDevice(prev);
+    }
+};
+uint32_t lane_count(const ckks_ctx *c) { return (uint32_t)std::max(1, std::min(c->lanes, 4)); }
+
 uint32_t log2_ceil(uint32_t x) { uint32_t d = 0; while ((1u << d) < x) d++; return d; }
 
 }  // namespace
@@ -108,7 +139,8 @@ extern "C" size_t ckks_attention_scores_workspace_bytes(const ckks_ctx *c, const
     AttnPlan p;
     if (!c || !dim || level < 2 || level > c->L || make_attn_plan(c, d, p)) return 0;
     // the split holds Gb - 1 rotated key sets, G / Gb - 1 rotated query sets, a product and a rescaled product
-    if (p.Gb > 1) return (size_t)(p.Gb + p.G / p.Gb - 2) * dim * ct_bytes(c, level) + 2 * ct_bytes(c, level) + scratch_bytes(c, level, p.G - 1);
+    if (p.Gb > 1)
+        return (size_t)(p.Gb + p.G / p.Gb - 2) * dim * ct_bytes(c, level) + 2 * ct_bytes(c, level) + lane_count(c) * scratch_bytes(c, level, p.G - 1);
     return (size_t)(p.G - 1) * dim * ct_bytes(c, level) + ct_bytes(c, level) + scratch_bytes(c, level, p.G - 1);
 }
 
@@ -122,18 +154,24 @@ static int scores_split(ckks_ctx *c, const AttnPlan &p, const ckks_ct *q, const 
     char *rest = qr + (size_t)(Gg - 1) * dim * ctb;
     ckks_ct prod{(uint64_t *)rest, level, 2, 0.0}, resc{(uint64_t *)(rest + ctb), level - 1, 2, 0.0};
     void *sw = rest + 2 * ctb;
-    const size_t sw_bytes = ws_bytes - (size_t)((char *)sw - base);
-    int rc;
+    const size_t sw_bytes = scratch_bytes(c, level, p.G - 1);
+    int rc = CKKS_OK;
     std::vector<ckks_evk> bk, gk;
     for (uint32_t g0 = 1; g0 < Gb; g0++) bk.push_back(*find_key(c, keys, nkeys, p.tok[g0 - 1]));
     for (int64_t r : p.neg) gk.push_back(*find_key(c, keys, nkeys, r));
     std::vector<ckks_ct> outs(std::max(Gb, Gg));
-    for (uint32_t dd = 0; dd < dim; dd++) {
+    // the channels' rotations are independent: spread over the lanes, each with its own scratch
+    const Lanes lanes(c, stream);
+    lanes.fork();
+    for (uint32_t dd = 0; dd < dim && !rc; dd++) {
+        void *lw = (char *)sw + (dd % lanes.n) * sw_bytes, *ls = lanes.at(dd);
         for (uint32_t x = 0; x + 1 < Gb; x++) outs[x] = ckks_ct{(uint64_t *)(kr + ((size_t)x * dim + dd) * ctb), level, 2, 0.0};
-        if (Gb > 1 && (rc = ckks_rotate_hoisted(c, &k[dd], bk.data(), Gb - 1, outs.data(), sw, sw_bytes, stream))) return rc;
+        if (Gb > 1) rc = ckks_rotate_hoisted(c, &k[dd], bk.data(), Gb - 1, outs.data(), lw, sw_bytes, ls);
         for (uint32_t y = 0; y + 1 < Gg; y++) outs[y] = ckks_ct{(uint64_t *)(qr + ((size_t)y * dim + dd) * ctb), level, 2, 0.0};
-        if (Gg > 1 && (rc = ckks_rotate_hoisted(c, &q[dd], gk.data(), Gg - 1, outs.data(), sw, sw_bytes, stream))) return rc;
+        if (!rc && Gg > 1) rc = ckks_rotate_hoisted(c, &q[dd], gk.data(), Gg - 1, outs.data(), lw, sw_bytes, ls);
     }
+    lanes.join();
+    if (rc) return rc;
     std::vector<ckks_ct> a(dim), b(dim);
     for (uint32_t g = 0; g < p.G; g++) {
         const uint32_t g1 = g / Gb, g0 = g % Gb;
@@ -218,7 +256,8 @@ static size_t rows_scratch(const ckks_ctx *c, const ckks_softmax_desc *s, uint32
 extern "C" size_t ckks_softmax_rows_workspace_bytes(const ckks_ctx *c, const ckks_attn_desc *d, const ckks_softmax_desc *s, uint32_t level) {
     AttnPlan p;
     if (!c || level < 1 || level > c->L || !rows_desc_ok(s) || make_attn_plan(c, d, p)) return 0;
-    return (size_t)(p.G + 4) * ct_bytes(c, level) + rows_scratch(c, s, level);
+    // the groups' running ciphertexts u_g, the row sums and lambda, then per lane two temporaries and the scratch of the calls
+    return (size_t)(p.G + 2) * ct_bytes(c, level) + lane_count(c) * (2 * ct_bytes(c, level) + rows_scratch(c, s, level));
 }
 
 extern "C" int32_t ckks_softmax_rows(ckks_ctx *c, const ckks_attn_desc *d, const ckks_softmax_desc *s, const ckks_ct *in, const ckks_evk *rlk,
@@ -241,16 +280,28 @@ extern "C" int32_t ckks_softmax_rows(ckks_ctx *c, const ckks_attn_desc *d, const
     char *base = (char *)ws;
     std::vector<ckks_ct> u(p.G);
     for (uint32_t g = 0; g < p.G; g++) u[g] = ckks_ct{(uint64_t *)(base + (size_t)g * ctb), level, 2, 0.0};
-    ckks_ct A{(uint64_t *)(base + (size_t)p.G * ctb), level, 2, 0.0}, B{(uint64_t *)(base + (size_t)(p.G + 1) * ctb), level, 2, 0.0},
-        T{(uint64_t *)(base + (size_t)(p.G + 2) * ctb), level, 2, 0.0}, X{(uint64_t *)(base + (size_t)(p.G + 3) * ctb), level, 2, 0.0};
-    void *sw = base + (size_t)(p.G + 4) * ctb;
-    const size_t sw_bytes = rows_scratch(c, s, level);
+    ckks_ct B{(uint64_t *)(base + (size_t)p.G * ctb), level, 2, 0.0}, T{(uint64_t *)(base + (size_t)(p.G + 1) * ctb), level, 2, 0.0};
+    const Lanes lanes(c, stream);
+    const size_t sw_bytes = rows_scratch(c, s, level), lane_bytes = 2 * ctb + sw_bytes;
+    char *lane0 = base + (size_t)(p.G + 2) * ctb;
+    // lane l: temporaries A and X, then the scratch
+    auto lane_A = [&](uint32_t l) { return ckks_ct{(uint64_t *)(lane0 + l * lane_bytes), level, 2, 0.0}; };
+    auto lane_X = [&](uint32_t l) { return ckks_ct{(uint64_t *)(lane0 + l * lane_bytes + ctb), level, 2, 0.0}; };
+    auto lane_sw = [&](uint32_t l) { return (void *)(lane0 + l * lane_bytes + 2 * ctb); };
     cudaStream_t st = (cudaStream_t)stream;
-    for (uint32_t g = 0; g < p.G; g++) {
-        if ((rc = ckks_add_const(c, &in[g], -s->shift, &A, stream))) return rc;
-        if ((rc = ckks_poly_eval_tree(c, &A, s->exp_coeffs, s->exp_degree, rlk, &u[g], sw, sw_bytes, stream))) return rc;
+    // the groups' exponentials are independent: spread over the lanes
+    lanes.fork();
+    for (uint32_t g = 0; g < p.G && !rc; g++) {
+        const uint32_t l = g % lanes.n;
+        ckks_ct A = lane_A(l);
+        if ((rc = ckks_add_const(c, &in[g], -s->shift, &A, lanes.at(g)))) break;
+        rc = ckks_poly_eval_tree(c, &A, s->exp_coeffs, s->exp_degree, rlk, &u[g], lane_sw(l), sw_bytes, lanes.at(g));
     }
+    lanes.join();
+    if (rc) return rc;
     for (uint32_t j = 0; j < s->rounds; j++) {
+        ckks_ct A = lane_A(0);
+        void *sw = lane_sw(0);
         // t = row sums of u^2: one relinearisation for the sum over the groups, then the ladder over the blocks
         if ((rc = ckks_mul_relin_sum(c, u.data(), u.data(), p.G, rlk, &A, sw, sw_bytes, stream))) return rc;
         if ((rc = ckks_rescale(c, &A, &T, sw, sw_bytes, stream))) return rc;
@@ -258,21 +309,28 @@ extern "C" int32_t ckks_softmax_rows(ckks_ctx *c, const ckks_attn_desc *d, const
         // lambda = p_rsqrt_j(t), once for all groups
         if ((rc = ckks_poly_eval_tree(c, &T, s->rsqrt_coeffs + (size_t)j * (s->rsqrt_degree + 1), s->rsqrt_degree, rlk, &B, sw, sw_bytes, stream)))
             return rc;
-        for (uint32_t g = 0; g < p.G; g++) {
+        // u_g = rescale(rescale(lambda u_g)^2): independent over the groups
+        lanes.fork();
+        for (uint32_t g = 0; g < p.G && !rc; g++) {
+            const uint32_t l = g % lanes.n;
+            ckks_ct Al = lane_A(l), X = lane_X(l);
+            void *ls = lanes.at(g), *lw = lane_sw(l);
             // u_g truncated to lambda's level
             int prev = 0;
             cudaGetDevice(&prev);
             cudaSetDevice(c->device);
             for (uint32_t comp = 0; comp < 2; comp++)
                 cudaMemcpyAsync(X.data + (size_t)comp * B.level * N, u[g].data + (size_t)comp * u[g].level * N, (size_t)B.level * N * sizeof(uint64_t),
-                                cudaMemcpyDeviceToDevice, st);
+                                cudaMemcpyDeviceToDevice, (cudaStream_t)ls);
             cudaSetDevice(prev);
             X.level = B.level; X.ncomp = 2; X.scale = u[g].scale;
-            if ((rc = ckks_mul_relin(c, &B, &X, rlk, &A, sw, sw_bytes, stream))) return rc;
-            if ((rc = ckks_rescale(c, &A, &X, sw, sw_bytes, stream))) return rc;
-            if ((rc = ckks_mul_relin(c, &X, &X, rlk, &A, sw, sw_bytes, stream))) return rc;
-            if ((rc = ckks_rescale(c, &A, &u[g], sw, sw_bytes, stream))) return rc;
+            if ((rc = ckks_mul_relin(c, &B, &X, rlk, &Al, lw, sw_bytes, ls))) break;
+            if ((rc = ckks_rescale(c, &Al, &X, lw, sw_bytes, ls))) break;
+            if ((rc = ckks_mul_relin(c, &X, &X, rlk, &Al, lw, sw_bytes, ls))) break;
+            rc = ckks_rescale(c, &Al, &u[g], lw, sw_bytes, ls);
         }
+        lanes.join();
+        if (rc) return rc;
     }
     int prev = 0;
     cudaGetDevice(&prev);
@@ -296,7 +354,8 @@ static size_t values_scratch(const ckks_ctx *c, uint32_t level, uint32_t nrot) {
 extern "C" size_t ckks_attention_values_workspace_bytes(const ckks_ctx *c, const ckks_attn_desc *d, uint32_t level) {
     AttnPlan p;
     if (!c || level < 2 || level > c->L || make_attn_plan(c, d, p)) return 0;
-    return (size_t)(p.G + 1) * ct_bytes(c, level) + (size_t)VAL_CHUNK * ct_bytes(c, level - 1) + values_scratch(c, level, p.G - 1);
+    // per lane: the truncated value operand with its rotated copies, a product, the scratch of the calls; then a ladder chunk
+    return lane_count(c) * ((size_t)(p.G + 1) * ct_bytes(c, level) + values_scratch(c, level, p.G - 1)) + (size_t)VAL_CHUNK * ct_bytes(c, level - 1);
 }
 
 extern "C" int32_t ckks_attention_values(ckks_ctx *c, const ckks_attn_desc *d, const ckks_ct *probs, const ckks_ct *v, uint32_t dim_v,
@@ -317,38 +376,44 @@ extern "C" int32_t ckks_attention_values(ckks_ctx *c, const ckks_attn_desc *d, c
     for (uint32_t dd = 0; dd < dim_v; dd++)
         if (!out[dd].data) return CKKS_ERR_ARG;
     if (!ws || ws_bytes < ckks_attention_values_workspace_bytes(c, d, lp)) return CKKS_ERR_WORKSPACE;
-    const size_t ctb = ct_bytes(c, lp), N = c->N;
+    const size_t ctb = ct_bytes(c, lp), ctb1 = ct_bytes(c, lp - 1), N = c->N;
     char *base = (char *)ws;
-    std::vector<ckks_ct> vr(p.G);
-    for (uint32_t g = 0; g < p.G; g++) vr[g] = ckks_ct{(uint64_t *)(base + (size_t)g * ctb), lp, 2, v[0].scale};
-    ckks_ct prod{(uint64_t *)(base + (size_t)p.G * ctb), lp, 2, 0.0};
-    const size_t ctb1 = ct_bytes(c, lp - 1);
-    char *rot = base + (size_t)(p.G + 1) * ctb;                          // [VAL_CHUNK] rotated outputs of the ladder
-    void *sw = rot + (size_t)VAL_CHUNK * ctb1;
-    const size_t sw_bytes = values_scratch(c, lp, p.G - 1);
+    const Lanes lanes(c, stream);
+    const size_t sw_bytes = values_scratch(c, lp, p.G - 1), lane_bytes = (size_t)(p.G + 1) * ctb + sw_bytes;
+    char *rot = base + lanes.n * lane_bytes;                           // [VAL_CHUNK] rotated outputs of the ladder
     std::vector<ckks_evk> pk;
     for (int64_t r : p.tok) pk.push_back(*find_key(c, keys, nkeys, r));
-    cudaStream_t st = (cudaStream_t)stream;
+    // the channels are independent up to the ladder: spread over the lanes, each with its own buffers
+    lanes.fork();
+    std::vector<ckks_ct> vr(p.G);
+    for (uint32_t dd = 0; dd < dim_v; dd++) {
+        char *lb = base + (dd % lanes.n) * lane_bytes;
+        void *ls = lanes.at(dd);
+        for (uint32_t g = 0; g < p.G; g++) vr[g] = ckks_ct{(uint64_t *)(lb + (size_t)g * ctb), lp, 2, v[dd].scale};
+        ckks_ct prod{(uint64_t *)(lb + (size_t)p.G * ctb), lp, 2, 0.0};
+        void *sw = lb + (size_t)(p.G + 1) * ctb;
+        int prev = 0;
+        cudaGetDevice(&prev);
+        cudaSetDevice(c->device);
+        for (uint32_t comp = 0; comp < 2; comp++)
+            cudaMemcpyAsync(vr[0].data + (size_t)comp * lp * N, v[dd].data + (size_t)comp * lv * N, (size_t)lp * N * sizeof(uint64_t),
+                            cudaMemcpyDeviceToDevice, (cudaStream_t)ls);
+        cudaSetDevice(prev);
+        if (p.G > 1 && (rc = ckks_rotate_hoisted(c, &vr[0], pk.data(), p.G - 1, vr.data() + 1, sw, sw_bytes, ls))) break;
+        for (uint32_t g = 0; g < p.G; g++) vr[g].scale = v[dd].scale;
+        if ((rc = ckks_mul_relin_sum(c, probs, vr.data(), p.G, rlk, &prod, sw, sw_bytes, ls))) break;
+        if ((rc = ckks_rescale(c, &prod, &out[dd], sw, sw_bytes, ls))) break;
+    }
+    lanes.join();
+    if (rc) return rc;
+    // the ladder over the blocks, a rotation of a whole chunk of channels at a time: out += rotate(out, r), r ascending
+    void *sw = base;                                                   // lane 0's buffers are free again
     std::vector<ckks_ct> tmp(VAL_CHUNK);
     for (uint32_t d0 = 0; d0 < dim_v; d0 += VAL_CHUNK) {
         const uint32_t nd = std::min(VAL_CHUNK, dim_v - d0);
-        for (uint32_t dd = d0; dd < d0 + nd; dd++) {
-            int prev = 0;
-            cudaGetDevice(&prev);
-            cudaSetDevice(c->device);
-            for (uint32_t comp = 0; comp < 2; comp++)
-                cudaMemcpyAsync(vr[0].data + (size_t)comp * lp * N, v[dd].data + (size_t)comp * lv * N, (size_t)lp * N * sizeof(uint64_t),
-                                cudaMemcpyDeviceToDevice, st);
-            cudaSetDevice(prev);
-            if (p.G > 1 && (rc = ckks_rotate_hoisted(c, &vr[0], pk.data(), p.G - 1, vr.data() + 1, sw, sw_bytes, stream))) return rc;
-            for (uint32_t g = 0; g < p.G; g++) vr[g].scale = v[dd].scale;
-            if ((rc = ckks_mul_relin_sum(c, probs, vr.data(), p.G, rlk, &prod, sw, sw_bytes, stream))) return rc;
-            if ((rc = ckks_rescale(c, &prod, &out[dd], sw, sw_bytes, stream))) return rc;
-        }
-        // the ladder over the blocks, a rotation of the whole chunk at a time: out += rotate(out, r), r ascending
         for (int64_t r : p.lad) {
             for (uint32_t x = 0; x < nd; x++) tmp[x] = ckks_ct{(uint64_t *)(rot + (size_t)x * ctb1), lp - 1, 2, 0.0};
-            if ((rc = ckks_rotate_batch(c, &out[d0], nd, find_key(c, keys, nkeys, r), tmp.data(), sw, sw_bytes, stream))) return rc;
+            if ((rc = ckks_rotate_batch(c, &out[d0], nd, find_key(c, keys, nkeys, r), tmp.data(), sw, lane_bytes, stream))) return rc;
             for (uint32_t x = 0; x < nd; x++)
                 if ((rc = ckks_add(c, &out[d0 + x], &tmp[x], &out[d0 + x], stream))) return rc;
         }
@@ -483,7 +548,7 @@ bool have_keys(const ckks_ctx *c, const std::vector<int64_t> &v, const ckks_evk 
     return true;
 }
 
-struct PackWs { size_t rot, acc, tmp, gat, pts, mask, sw, sw_bytes, bytes; uint32_t nrot; };
+struct PackWs { size_t rot, acc, tmp, gat, pts, mask, sw, sw_bytes, lane, lane_bytes, bytes; uint32_t nrot; };
 
 // kind 0 / 1: pack; kind 2: back
 PackWs pack_layout(const ckks_ctx *c, const PackPlan &p, int kind, uint32_t level, uint32_t dim) {
@@ -494,13 +559,18 @@ PackWs pack_layout(const ckks_ctx *c, const PackPlan &p, int kind, uint32_t leve
     w.rot = off;  off += (size_t)w.nrot * ct_bytes(c, level);
     w.acc = off;  off += (size_t)nout * ct_bytes(c, level);
     w.tmp = off;  off += ct_bytes(c, level);
-    w.gat = off;  off += kind == 1 ? (size_t)dim * ct_bytes(c, level - 1) + 2 * ct_bytes(c, level - 1) : 0;     // gathered[d], k0, a sum
+    w.gat = off;  off += kind == 1 ? (size_t)dim * ct_bytes(c, level - 1) : 0;                                  // gathered[d]
     w.pts = off;  off += (size_t)(kind == 1 ? 2 * p.E : 1) * pt_bytes(c, level);
     w.mask = off; off += mask_scratch(c, level);
     w.sw = off;
     w.sw_bytes = align256(std::max({ckks_workspace_bytes(c, CKKS_OP_ROTATE_HOISTED, level, 16), ckks_workspace_bytes(c, CKKS_OP_RESCALE, level, 0),
                                     ckks_workspace_bytes(c, CKKS_OP_ROTATE, level, 0), ckks_workspace_bytes(c, CKKS_OP_ROTATE_BATCH, level, 16)}));
-    w.bytes = off + w.sw_bytes;
+    off += w.sw_bytes;
+    // key, value: per lane the rotated copies of the token shifts, k0, a sum and the scratch of the calls
+    w.lane = off;
+    w.lane_bytes = (size_t)2 * p.E * ct_bytes(c, level - 1) + 2 * ct_bytes(c, level - 1) + w.sw_bytes;
+    if (kind == 1) off += lane_count(c) * w.lane_bytes;
+    w.bytes = off;
     return w;
 }
 
@@ -614,22 +684,28 @@ extern "C" int32_t ckks_attention_pack(ckks_ctx *c, const ckks_attn_desc *d, int
         if ((rc = encode_mask(c, l1, p.B, e * p.P, (e + 1) * p.P, p.Ti, 0, p.Ti - b, &mA[e], base + L.mask, stream))) return rc;
         if (b && (rc = encode_mask(c, l1, p.B, e * p.P, (e + 1) * p.P, p.Ti, p.Ti - b, p.Ti, &mB[e], base + L.mask, stream))) return rc;
     }
-    ckks_ct k0{(uint64_t *)(base + L.gat + (size_t)dim * ctb1), l1, 2, 0.0}, sum{(uint64_t *)(base + L.gat + (size_t)(dim + 1) * ctb1), l1, 2, 0.0};
     std::vector<int64_t> sr;
     for (uint32_t e = 0; e < p.E; e++) { sr.push_back(p.shA[e]); if (e % p.Ti) sr.push_back(p.shB[e]); }
     std::vector<ckks_ct> so(sr.size());
-    for (uint32_t dd = 0; dd < dim; dd++) {
+    // the channels are independent: spread over the lanes, each with its own buffers
+    const Lanes lanes(c, stream);
+    lanes.fork();
+    for (uint32_t dd = 0; dd < dim && !rc; dd++) {
+        char *lb = base + L.lane + (dd % lanes.n) * L.lane_bytes;
+        void *ls = lanes.at(dd), *lw = lb + (size_t)(2 * p.E + 2) * ctb1;
+        ckks_ct k0{(uint64_t *)(lb + (size_t)(2 * p.E) * ctb1), l1, 2, 0.0}, sum{(uint64_t *)(lb + (size_t)(2 * p.E + 1) * ctb1), l1, 2, 0.0};
         ckks_ct g = moved[dd];
-        if ((rc = ckks_rotate(c, &g, find_key(c, keys, nkeys, p.dbl[0]), &k0, sw, L.sw_bytes, stream))) return rc;
-        if ((rc = ckks_add(c, &g, &k0, &k0, stream))) return rc;
-        for (size_t x = 0; x < sr.size(); x++) so[x] = ckks_ct{(uint64_t *)(base + L.rot + x * ctb), l1, 2, 0.0};
-        if ((rc = rotate_many(c, &k0, sr, keys, nkeys, so.data(), sw, L.sw_bytes, stream))) return rc;
+        if ((rc = ckks_rotate(c, &g, find_key(c, keys, nkeys, p.dbl[0]), &k0, lw, L.sw_bytes, ls))) break;
+        if ((rc = ckks_add(c, &g, &k0, &k0, ls))) break;
+        for (size_t x = 0; x < sr.size(); x++) so[x] = ckks_ct{(uint64_t *)(lb + x * ctb1), l1, 2, 0.0};
+        if ((rc = rotate_many(c, &k0, sr, keys, nkeys, so.data(), lw, L.sw_bytes, ls))) break;
         size_t x = 0;
-        for (uint32_t e = 0; e < p.E; e++) {
-            if ((rc = ckks_mul_plain_acc(c, &so[x++], 1, &mA[e], &sum, e == 0, stream))) return rc;
-            if (e % p.Ti && (rc = ckks_mul_plain_acc(c, &so[x++], 1, &mB[e], &sum, 0, stream))) return rc;
+        for (uint32_t e = 0; e < p.E && !rc; e++) {
+            rc = ckks_mul_plain_acc(c, &so[x++], 1, &mA[e], &sum, e == 0, ls);
+            if (!rc && e % p.Ti) rc = ckks_mul_plain_acc(c, &so[x++], 1, &mB[e], &sum, 0, ls);
         }
-        if ((rc = ckks_rescale(c, &sum, &out[dd], sw, L.sw_bytes, stream))) return rc;
+        if (!rc) rc = ckks_rescale(c, &sum, &out[dd], lw, L.sw_bytes, ls);
     }
-    return CKKS_OK;
+    lanes.join();
+    return rc;
 }

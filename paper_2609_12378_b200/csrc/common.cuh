@@ -77,6 +77,12 @@ struct ckks_ctx {
     int conv_kernel = 0;                     // basis conversions: 0 = FP64 pipe, 1 = tensor cores (conv_mma.cu)
     int mac_kernel = 82;                     // projection multiply-accumulate kernel (see launch_mac_mma)
     long long wait_cycles = 2000000000ll;    // clock bound of every device-side wait (about a second)
+    // Streams of the context.  Composite calls whose work is many independent single-ciphertext chains (the attention
+    // entry points) spread those chains over `lanes` streams, lane 0 being the caller's: a single ciphertext's kernels fill
+    // the GPU for at most one wave, so independent chains overlap.  Forked from and joined to the caller's stream by events.
+    int lanes = 4;
+    cudaStream_t lane_stream[3] = {nullptr, nullptr, nullptr};
+    cudaEvent_t lane_event[4] = {nullptr, nullptr, nullptr, nullptr};
 };
 
 // ---------------------------------------------------------------------------

@@ -110,6 +110,10 @@ extern "C" void ckks_context_destroy(ckks_ctx *ctx) {
     cudaGetDevice(&prev);
     cudaSetDevice(ctx->device);
     for (void *p : ctx->allocs) cudaFree(p);
+    for (cudaStream_t s : ctx->lane_stream)
+        if (s) cudaStreamDestroy(s);
+    for (cudaEvent_t e : ctx->lane_event)
+        if (e) cudaEventDestroy(e);
     cudaSetDevice(prev);
     delete ctx;
 }
@@ -139,6 +143,10 @@ extern "C" int32_t ckks_context_set_option(ckks_ctx *ctx, int32_t option, int64_
             if (value < 0) return CKKS_ERR_ARG;
             ctx->wait_cycles = (long long)value;
             return CKKS_OK;
+        case CKKS_OPT_LANES:
+            if (value < 1 || value > 4) return CKKS_ERR_ARG;
+            ctx->lanes = (int)value;
+            return CKKS_OK;
         default: return CKKS_ERR_ARG;
     }
 }
@@ -151,6 +159,7 @@ extern "C" int64_t ckks_context_get_option(const ckks_ctx *ctx, int32_t option) 
         case CKKS_OPT_MAC_KERNEL: return ctx->mac_kernel;
         case CKKS_OPT_WAIT_CYCLES: return ctx->wait_cycles;
         case CKKS_OPT_NTT_BULK_STORE: return ctx->ntt_bulk_store;
+        case CKKS_OPT_LANES: return ctx->lanes;
         case CKKS_OPT_STATIC_SCRATCH_BYTES: return (int64_t)CKKS_STATIC_SCRATCH_BYTES;
         default: return -1;
     }
@@ -409,6 +418,14 @@ extern "C" int32_t ckks_context_create(const ckks_params *prm, ckks_ctx **out) {
         return rc;
     }
     d.range_flag = const_cast<int *>(flag_dev);
+    bool lanes_ok = true;
+    for (cudaStream_t &ls : c->lane_stream) lanes_ok = lanes_ok && cudaStreamCreateWithFlags(&ls, cudaStreamNonBlocking) == cudaSuccess;
+    for (cudaEvent_t &le : c->lane_event) lanes_ok = lanes_ok && cudaEventCreateWithFlags(&le, cudaEventDisableTiming) == cudaSuccess;
+    if (!lanes_ok) {
+        cudaSetDevice(prev);
+        ckks_context_destroy(c);
+        return CKKS_ERR_CUDA;
+    }
     cudaSetDevice(prev);
     *out = c;
     return CKKS_OK;

@@ -322,3 +322,27 @@ def test_attention_block_from_projections_to_projection_bit_exact():
         arr = host(dz[cc].data)
         assert np.array_equal(host(dY[cc].data), Y[cc]) and np.array_equal(arr, z[cc]), cc
         assert np.abs(cl.decrypt_slots(arr, dz[cc].scale).real - want[cc]).max() < 2.0 ** -14
+
+
+def test_lanes_do_not_change_results():
+    """The attention entry points spread independent chains over the context's streams (option CKKS_OPT_LANES); one lane
+    (the caller's stream only) and four give the same limbs, on the caller's stream in both cases."""
+    from tests.gpu_util import host
+    P, ctx, o, cl, desc, c, scale, q, k, v, rlk, keys, dev = _setup(10, 13, 4, 4, 13, 16, 2, 4, 4, 3, 641)
+    a = (16, 2, 4)
+    assert ctx.get_option(binding.OPT_LANES) == 4
+    res = {}
+    try:
+        for lanes in (1, 4, 2):
+            ctx.set_option(binding.OPT_LANES, lanes)
+            out = ctx.attention(dev["q"], dev["k"], dev["v"], c["shift"], 1, c["exp_coeffs"], c["rsqrt_coeffs"], dev["rlk"], dev["keys"], *a)
+            res[lanes] = [host(x.data) for x in out]
+    finally:
+        ctx.set_option(binding.OPT_LANES, 4)
+    want, _ = o.attention(desc, q, k, v, scale, scale, c["shift"], 1, c["exp_coeffs"], c["rsqrt_coeffs"], rlk, keys)
+    for lanes in (1, 2, 4):
+        for d in range(3):
+            assert np.array_equal(res[lanes][d], want[d]), (lanes, d)
+    with pytest.raises(binding.CkksError):
+        ctx.set_option(binding.OPT_LANES, 5)
+    assert ctx.device_status() == binding.OK
