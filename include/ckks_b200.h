@@ -142,6 +142,8 @@ const char *ckks_last_cuda_error(const ckks_ctx *ctx);
  *                           others belong to the context; they are forked from and joined to the caller's stream by events
  *                           inside the call, so the call still behaves as work on the caller's stream.  The workspace sizes
  *                           of those calls depend on it: set it before asking for them.  Results do not depend on it.
+ *                           The lanes' streams and events belong to the context: two host threads must not run attention
+ *                           entry points on the same context at the same time (use a context per thread).
  *   CKKS_OPT_STATIC_SCRATCH_BYTES  (read only) CKKS_STATIC_SCRATCH_BYTES of the loaded library.
  * set returns CKKS_ERR_ARG for an unknown option or a value outside its range; get returns -1 for an unknown option. */
 enum { CKKS_OPT_NTT_FP_SHARE = 1, CKKS_OPT_CONV_KERNEL = 2, CKKS_OPT_MAC_KERNEL = 3, CKKS_OPT_WAIT_CYCLES = 4,
