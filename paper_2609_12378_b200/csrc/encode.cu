@@ -39,7 +39,33 @@ __global__ void __launch_bounds__(THREADS) fft_chunks(DevTables c, const double 
         tw[x] = c.enc_omega_st[x];
     }
     __syncthreads();
-    for (uint32_t m = 2; m <= ch; m <<= 1) {
+    // two stages per pass over shared memory: a thread takes the four points j, j + h, j + 2h, j + 3h of a block of 4h and does
+    // the two butterflies of span h and the two of span 2h on registers (the same butterflies with the same operands as one
+    // stage at a time; the kernel is bound by shared-memory traffic, which this halves)
+    uint32_t m = 2;
+    for (; 2 * m <= ch; m <<= 2) {
+        const uint32_t h = m >> 1;
+        for (uint32_t x = threadIdx.x; x < ch / 4; x += THREADS) {
+            const uint32_t j = x & (h - 1), i0 = ((x - j) << 2) + j;
+            double2 a0 = sm[i0], a1 = sm[i0 + h], a2 = sm[i0 + 2 * h], a3 = sm[i0 + 3 * h];
+            const double2 w1 = tw[h + j];
+            double2 t = cmul_conj_w(w1, a1);
+            a1 = make_double2(__dsub_rn(a0.x, t.x), __dsub_rn(a0.y, t.y));
+            a0 = make_double2(__dadd_rn(a0.x, t.x), __dadd_rn(a0.y, t.y));
+            t = cmul_conj_w(w1, a3);
+            a3 = make_double2(__dsub_rn(a2.x, t.x), __dsub_rn(a2.y, t.y));
+            a2 = make_double2(__dadd_rn(a2.x, t.x), __dadd_rn(a2.y, t.y));
+            t = cmul_conj_w(tw[2 * h + j], a2);
+            a2 = make_double2(__dsub_rn(a0.x, t.x), __dsub_rn(a0.y, t.y));
+            a0 = make_double2(__dadd_rn(a0.x, t.x), __dadd_rn(a0.y, t.y));
+            t = cmul_conj_w(tw[2 * h + j + h], a3);
+            a3 = make_double2(__dsub_rn(a1.x, t.x), __dsub_rn(a1.y, t.y));
+            a1 = make_double2(__dadd_rn(a1.x, t.x), __dadd_rn(a1.y, t.y));
+            sm[i0] = a0; sm[i0 + h] = a1; sm[i0 + 2 * h] = a2; sm[i0 + 3 * h] = a3;
+        }
+        __syncthreads();
+    }
+    for (; m <= ch; m <<= 1) {             // a last single stage when the number of stages is odd
         const uint32_t half = m >> 1;
         for (uint32_t x = threadIdx.x; x < ch / 2; x += THREADS) {
             const uint32_t j = x & (half - 1), i1 = ((x - j) << 1) + j;
