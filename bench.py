@@ -289,6 +289,10 @@ def run_cuda(args):
     q, p = inputs.prime_chain(LOG_N, L, K)
     allp = [int(x) for x in q] + [int(x) for x in p]
     ctx = binding.Context(LOG_N, q, p, DNUM, device=local)
+    if args.profile and args.mac_kernel:
+        ctx.set_option(binding.OPT_MAC_KERNEL, args.mac_kernel)
+    if args.profile and args.conv_kernel >= 0:
+        ctx.set_option(binding.OPT_CONV_KERNEL, args.conv_kernel)
     gen = torch.Generator(device=dev)
     gen.manual_seed(1004 + rank)
 
@@ -802,6 +806,8 @@ def main():
     ap.add_argument("--parts", default="abc", help="with --profile: which parts of the step to run (a: NTT, b: key switching, c: projection)")
     ap.add_argument("--shards", type=int, default=SHARDS, help="with --profile: token shards in the projection (default 16)")
     ap.add_argument("--ntt-batch", type=int, default=NTT_BATCH, help="with --profile: polynomials in the NTT part (default 32)")
+    ap.add_argument("--mac-kernel", type=int, default=0, help="with --profile: CKKS_OPT_MAC_KERNEL value (82, 83, 81, 42, 100); 0 = the default")
+    ap.add_argument("--conv-kernel", type=int, default=-1, help="with --profile: CKKS_OPT_CONV_KERNEL value (0 = FP64, 1 = tensor cores)")
     ap.add_argument("--eager-moddown", action="store_true",
                     help="one ModDown per giant-step rotation instead of one per output ciphertext")
     ap.add_argument("--no-extras", action="store_true", help="skip the untimed one-off measurements of the composite calls")
