@@ -739,7 +739,9 @@ def layer_submetrics(ctx, residues, allp, gen, dev, reps, have_keys):
     pc = [0.5 ** (k // 4) / (1 + k) for k in range(64)]
     xg = binding.Ciphertext(g1[0].data, 2.0 ** 50)
     out["ms"]["polynomial_degree_63_one_ciphertext"] = timed(lambda: ctx.poly_eval_bsgs(xg, pc, 8, rlk))
-    del xg
+    xs = [binding.Ciphertext(g1[i % 16].data, 2.0 ** 50) for i in range(nib * SHARDS)]
+    out["ms"]["polynomial_degree_63_of_64_ciphertexts"] = timed(lambda: ctx.poly_eval_bsgs_batch(xs, pc, 8, rlk))
+    del xg, xs
     del bouts, bws, a, b, acc, g1, g2, ga, gb, gouts, gws
     ctx._ws = None
     torch.cuda.empty_cache()

@@ -281,6 +281,12 @@ int32_t ckks_poly_eval_tree(ckks_ctx *ctx, const ckks_ct *x, const double *coeff
 int32_t ckks_poly_eval_bsgs(ckks_ctx *ctx, const ckks_ct *x, const double *coeffs, uint32_t degree, uint32_t m, const ckks_evk *rlk,
                             ckks_ct *out, void *ws, size_t ws_bytes, void *stream);
 size_t ckks_poly_eval_bsgs_workspace_bytes(const ckks_ctx *ctx, uint32_t level, uint32_t degree, uint32_t m);
+/* The same polynomial of n ciphertexts at one level (an activation function over a layer's ciphertexts): every out[i] is
+ * bit-identical to ckks_poly_eval_bsgs(x[i]); the n independent chains are spread over the context's lanes
+ * (CKKS_OPT_LANES), each with a workspace of its own.  Errors as ckks_poly_eval_bsgs. */
+int32_t ckks_poly_eval_bsgs_batch(ckks_ctx *ctx, const ckks_ct *x, uint32_t n, const double *coeffs, uint32_t degree, uint32_t m,
+                                  const ckks_evk *rlk, ckks_ct *out, void *ws, size_t ws_bytes, void *stream);
+size_t ckks_poly_eval_bsgs_batch_workspace_bytes(const ckks_ctx *ctx, uint32_t level, uint32_t degree, uint32_t m, uint32_t n);
 
 /* ---- Softmax by doubling with a public shift (Algorithm 1) --------------------
  * One ciphertext of score rows: row r holds its row_len scores (a power of two dividing n) in slots

@@ -28,7 +28,7 @@ EXPORTS = [
     "ckks_encode_range_flag", "ckks_mul_plain_acc", "ckks_add", "ckks_mul_relin", "ckks_rotate",
     "ckks_rotate_hoisted", "ckks_rescale", "ckks_linear_proj", "ckks_linear_proj_workspace_bytes",
     "ckks_linear_proj_rotations", "ckks_kernel_launches", "ckks_device_status", "ckks_rescale_static",
-    "ckks_attention_pack_rotations", "ckks_attention_pack", "ckks_attention_pack_workspace_bytes", "ckks_attention_rotations", "ckks_attention_scores", "ckks_attention_scores_workspace_bytes", "ckks_attention_values",
+    "ckks_poly_eval_bsgs_batch", "ckks_poly_eval_bsgs_batch_workspace_bytes", "ckks_attention_pack_rotations", "ckks_attention_pack", "ckks_attention_pack_workspace_bytes", "ckks_attention_rotations", "ckks_attention_scores", "ckks_attention_scores_workspace_bytes", "ckks_attention_values",
     "ckks_attention_values_workspace_bytes", "ckks_softmax_rows", "ckks_softmax_rows_workspace_bytes", "ckks_attention",
     "ckks_attention_workspace_bytes",
     "ckks_ntt_butterfly_probe", "ckks_mul_relin_sum", "ckks_mul_relin_batch", "ckks_rotate_batch", "ckks_rotate_sum", "ckks_softmax", "ckks_softmax_workspace_bytes", "ckks_poly_eval_bsgs", "ckks_poly_eval_bsgs_workspace_bytes", "ckks_mul_const", "ckks_add_const", "ckks_poly_eval", "ckks_poly_eval_tree", "ckks_linear_proj_multi", "ckks_linear_proj_multi_workspace_bytes",
@@ -102,6 +102,8 @@ def load():
         "ckks_softmax": (i32, [vp, C.POINTER(CSoftmaxDesc), C.POINTER(CCt), C.POINTER(CEvk), C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
         "ckks_softmax_workspace_bytes": (sz, [vp, C.POINTER(CSoftmaxDesc), u32]),
         "ckks_attention_rotations": (i32, [vp, C.POINTER(CAttnDesc), C.POINTER(i64), u32]),
+        "ckks_poly_eval_bsgs_batch": (i32, [vp, C.POINTER(CCt), u32, C.POINTER(C.c_double), u32, u32, C.POINTER(CEvk), C.POINTER(CCt), vp, sz, vp]),
+        "ckks_poly_eval_bsgs_batch_workspace_bytes": (sz, [vp, u32, u32, u32, u32]),
         "ckks_attention_pack_rotations": (i32, [vp, C.POINTER(CAttnDesc), i32, u32, C.POINTER(i64), u32]),
         "ckks_attention_pack": (i32, [vp, C.POINTER(CAttnDesc), i32, C.POINTER(CCt), u32, C.POINTER(CEvk), u32, C.POINTER(CCt), vp, sz, vp]),
         "ckks_attention_pack_workspace_bytes": (sz, [vp, C.POINTER(CAttnDesc), i32, u32, u32]),
@@ -389,6 +391,21 @@ class Context:
         self._check(load().ckks_poly_eval_bsgs(self._h, C.byref(_cct(x)), ca, d, m, C.byref(ck), C.byref(co), ws.data_ptr(), ws.numel(),
                                                _stream_ptr(stream)))
         return Ciphertext(out.data.view(-1)[: 2 * co.level * self.N].view(2, co.level, self.N), co.scale)
+
+    def poly_eval_bsgs_batch(self, xs, coeffs, m: int, rlk: SwitchKey, stream=None):
+        """[poly_eval_bsgs(x, coeffs, m) for x in xs], the independent evaluations spread over the context's lanes."""
+        d, n, level = len(coeffs) - 1, len(xs), xs[0].level
+        need = int(load().ckks_poly_eval_bsgs_batch_workspace_bytes(self._h, level, d, m, n))
+        if need == 0:
+            raise CkksError(ERR_ARG)
+        ws = self.workspace(need)
+        outs = [self.empty_ct(level) for _ in xs]
+        ca = (C.c_double * (d + 1))(*[float(v) for v in coeffs])
+        xa = (CCt * n)(*[_cct(x) for x in xs])
+        oa = (CCt * n)(*[_cct(o) for o in outs])
+        ck = CEvk(_dev_u64(rlk.data).data_ptr(), rlk.galois)
+        self._check(load().ckks_poly_eval_bsgs_batch(self._h, xa, n, ca, d, m, C.byref(ck), oa, ws.data_ptr(), ws.numel(), _stream_ptr(stream)))
+        return [self._cut(o, c) for o, c in zip(outs, oa)]
 
     def softmax(self, ct: Ciphertext, shift: float, rounds: int, row_len: int, exp_coeffs, rsqrt_coeffs, rlk: SwitchKey, keys,
                 ws: torch.Tensor = None, stream=None, exp_m: int = 0, rsqrt_m: int = 0):

@@ -677,6 +677,30 @@ static bool softmax_desc_ok(const ckks_ctx *c, const ckks_softmax_desc *d) {
            (!d->rsqrt_m || !d->rounds || bsgs_shape_ok(d->rsqrt_degree, d->rsqrt_m));
 }
 
+// The same polynomial of n ciphertexts: independent chains, spread over the context's lanes with a workspace each.
+extern "C" size_t ckks_poly_eval_bsgs_batch_workspace_bytes(const ckks_ctx *c, uint32_t level, uint32_t degree, uint32_t m, uint32_t n) {
+    const size_t one = ckks_poly_eval_bsgs_workspace_bytes(c, level, degree, m);
+    return one ? align256(one) * std::min<uint32_t>(std::max<uint32_t>(n, 1), lane_count(c)) : 0;
+}
+
+extern "C" int32_t ckks_poly_eval_bsgs_batch(ckks_ctx *c, const ckks_ct *x, uint32_t n, const double *coeffs, uint32_t degree, uint32_t m,
+                                             const ckks_evk *rlk, ckks_ct *out, void *ws, size_t ws_bytes, void *stream) {
+    if (!c || !x || !out || !n) return CKKS_ERR_ARG;
+    for (uint32_t i = 0; i < n; i++)
+        if (!ct_ok(&x[i]) || !ct_ok(&out[i]) || x[i].level != x[0].level) return x && ct_ok(&x[i]) && ct_ok(&out[i]) ? CKKS_ERR_LEVEL : CKKS_ERR_ARG;
+    const size_t one = align256(ckks_poly_eval_bsgs_workspace_bytes(c, x[0].level, degree, m));
+    if (!one) return CKKS_ERR_ARG;
+    const Lanes lanes(c, stream);
+    const uint32_t nl = std::min<uint32_t>(n, lanes.n);
+    if (!ws || ws_bytes < one * nl) return CKKS_ERR_WORKSPACE;
+    int rc = CKKS_OK;
+    lanes.fork();
+    for (uint32_t i = 0; i < n && !rc; i++)
+        rc = ckks_poly_eval_bsgs(c, &x[i], coeffs, degree, m, rlk, &out[i], (char *)ws + (size_t)(i % nl) * one, one, lanes.at(i % nl));
+    lanes.join();
+    return rc;
+}
+
 extern "C" size_t ckks_softmax_workspace_bytes(const ckks_ctx *c, const ckks_softmax_desc *d, uint32_t level) {
     if (!c || !softmax_desc_ok(c, d) || !level_ok(c, level)) return 0;
     return 4 * align256((size_t)2 * level * c->N * sizeof(u64)) + softmax_scratch_bytes(c, d, level);

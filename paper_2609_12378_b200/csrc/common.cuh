@@ -1,6 +1,7 @@
 // Shared declarations of the ckks_b200 library: context, device tables,
 // modular arithmetic for 50-bit primes, kernel launch entry points.
 #pragma once
+#include <algorithm>
 
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -84,6 +85,37 @@ struct ckks_ctx {
     cudaStream_t lane_stream[3] = {nullptr, nullptr, nullptr};
     cudaEvent_t lane_event[4] = {nullptr, nullptr, nullptr, nullptr};
 };
+
+// The context's streams as lanes for independent chains: lane 0 is the caller's stream.  fork() makes the other lanes wait
+// for what the caller's stream has been given so far, join() makes the caller's stream wait for all of them.
+struct Lanes {
+    ckks_ctx *c;
+    cudaStream_t caller;
+    uint32_t n;
+    Lanes(ckks_ctx *ctx, void *stream) : c(ctx), caller((cudaStream_t)stream), n((uint32_t)std::max(1, std::min(ctx->lanes, 4))) {}
+    void *at(uint32_t i) const { return i % n == 0 ? (void *)caller : (void *)c->lane_stream[i % n - 1]; }
+    void fork() const {
+        if (n == 1) return;
+        int prev = 0;
+        cudaGetDevice(&prev);
+        cudaSetDevice(c->device);
+        cudaEventRecord(c->lane_event[0], caller);
+        for (uint32_t i = 1; i < n; i++) cudaStreamWaitEvent(c->lane_stream[i - 1], c->lane_event[0], 0);
+        cudaSetDevice(prev);
+    }
+    void join() const {
+        if (n == 1) return;
+        int prev = 0;
+        cudaGetDevice(&prev);
+        cudaSetDevice(c->device);
+        for (uint32_t i = 1; i < n; i++) {
+            cudaEventRecord(c->lane_event[i], c->lane_stream[i - 1]);
+            cudaStreamWaitEvent(caller, c->lane_event[i], 0);
+        }
+        cudaSetDevice(prev);
+    }
+};
+inline uint32_t lane_count(const ckks_ctx *c) { return (uint32_t)std::max(1, std::min(c->lanes, 4)); }
 
 // ---------------------------------------------------------------------------
 // "Tiled" operand layout of the projection's multiply-accumulate.  R rows (one row = one plaintext, or one

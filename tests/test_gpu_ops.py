@@ -335,6 +335,35 @@ def test_poly_eval_bsgs_bit_exact(log_n, d, m):
         assert e.value.code == binding.ERR_LEVEL
 
 
+def test_poly_eval_bsgs_batch_bit_exact():
+    """The same polynomial of several ciphertexts, spread over the context's lanes: every output equals the checker's
+    evaluation of its own input (seven ciphertexts on four lanes, then on one)."""
+    from tests.gpu_util import context, ct_dev, host, key_dev
+    cfg = (11, 9, 3, 3)
+    P, ctx = params(*cfg), context(*cfg)
+    o = P.oracle
+    cl = Client(P, 83)
+    g = inputs.rng(83, 2)
+    level, scale, d, m = 9, 2.0 ** 50, 15, 4
+    coeffs = g.uniform(-1, 1, d + 1) / (1 + np.arange(d + 1))
+    rlk = cl.relin_key()
+    cts = [cl.encrypt_slots(g.uniform(-1, 1, P.n), scale, level) for _ in range(7)]
+    want = [o.poly_eval_bsgs(c, scale, coeffs, rlk, m) for c in cts]
+    dev = [ct_dev(c, scale) for c in cts]
+    try:
+        for lanes in (4, 1):
+            ctx.set_option(binding.OPT_LANES, lanes)
+            got = ctx.poly_eval_bsgs_batch(dev, coeffs, m, key_dev(rlk, 0))
+            for x, (w, so) in zip(got, want):
+                assert x.level == w.shape[1] and x.scale == so and np.array_equal(host(x.data), w)
+    finally:
+        ctx.set_option(binding.OPT_LANES, 4)
+    assert ctx.device_status() == binding.OK
+    with pytest.raises(binding.CkksError) as e:
+        ctx.poly_eval_bsgs_batch(dev, coeffs, 3, key_dev(rlk, 0))
+    assert e.value.code == binding.ERR_ARG
+
+
 def test_softmax_by_doubling_bit_exact():
     """Algorithm 1 with synthetic polynomials on 32 rows of 16 scores (two rounds, degree 4): the composite entry point
     returns the checker's integers, which decrypt to the same pipeline in the clear and to the Softmax of every row."""
