@@ -2,7 +2,7 @@
 dnum 3, 16 token shards of 8, B = 64) through the public binding: query/key/value as one call sharing their baby
 steps, output, gate/up as one call, down.  Synthetic inputs (uniform residues for ciphertexts and keys, normal weights):
 the kernels do the same work on them as on real ones.  Needs one B200-class GPU (the down projection's workspace is
-about 150 GiB with B = 64; pass --down-baby 32 for 90 GiB).
+62.5 GiB with B = 64, next to 11.8 GiB of rotation keys).
 
     python -m paper_2609_12378_b200.examples.llama_layer_projections [--eager] [--down-baby 32]
 """
