@@ -657,16 +657,25 @@ extern "C" int32_t ckks_attention_pack(ckks_ctx *c, const ckks_attn_desc *d, int
     std::vector<int64_t> sr;
     for (uint32_t e = 0; e < p.E; e++) { sr.push_back(p.shA[e]); if (e % p.Ti) sr.push_back(p.shB[e]); }
     std::vector<ckks_ct> so(sr.size());
+    // the copy of block 0 in block 1, k0 = moved + rotate(moved, -P B), in place and 16 channels at a time (one key)
+    {
+        std::vector<ckks_ct> tmp16(16);
+        for (uint32_t d0 = 0; d0 < dim; d0 += 16) {
+            const uint32_t nd = std::min<uint32_t>(16, dim - d0);
+            for (uint32_t x = 0; x < nd; x++) tmp16[x] = ckks_ct{(uint64_t *)(base + L.rot + (size_t)x * ctb), l1, 2, 0.0};
+            if ((rc = ckks_rotate_batch(c, &moved[d0], nd, find_key(c, keys, nkeys, p.dbl[0]), tmp16.data(), sw, L.sw_bytes, stream))) return rc;
+            for (uint32_t x = 0; x < nd; x++)
+                if ((rc = ckks_add(c, &moved[d0 + x], &tmp16[x], &moved[d0 + x], stream))) return rc;
+        }
+    }
     // the channels are independent: spread over the lanes, each with its own buffers
     const Lanes lanes(c, stream);
     lanes.fork();
     for (uint32_t dd = 0; dd < dim && !rc; dd++) {
         char *lb = base + L.lane + (dd % lanes.n) * L.lane_bytes;
         void *ls = lanes.at(dd), *lw = lb + (size_t)(2 * p.E + 2) * ctb1;
-        ckks_ct k0{(uint64_t *)(lb + (size_t)(2 * p.E) * ctb1), l1, 2, 0.0}, sum{(uint64_t *)(lb + (size_t)(2 * p.E + 1) * ctb1), l1, 2, 0.0};
-        ckks_ct g = moved[dd];
-        if ((rc = ckks_rotate(c, &g, find_key(c, keys, nkeys, p.dbl[0]), &k0, lw, L.sw_bytes, ls))) break;
-        if ((rc = ckks_add(c, &g, &k0, &k0, ls))) break;
+        ckks_ct sum{(uint64_t *)(lb + (size_t)(2 * p.E + 1) * ctb1), l1, 2, 0.0};
+        ckks_ct k0 = moved[dd];
         for (size_t x = 0; x < sr.size(); x++) so[x] = ckks_ct{(uint64_t *)(lb + x * ctb1), l1, 2, 0.0};
         if ((rc = rotate_many(c, &k0, sr, keys, nkeys, so.data(), lw, L.sw_bytes, ls))) break;
         size_t x = 0;
